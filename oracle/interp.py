@@ -1,0 +1,260 @@
+"""Reference interpreter for operator graphs (TEST INFRASTRUCTURE, not product).
+
+This is the oracle the CUDA path is checked against.  It executes the
+ORIGINAL graph -- unrewritten, unfused -- one operator at a time in
+topological order, every intermediate fully materialised as its own fp64
+array.  Operator fusion and index rewriting are exact transformations of that
+function (paper Section 1: fusion removes materialisation of intermediates;
+Section 4.2: rewriting keeps the mathematical function), so the plain
+definition of each operator, composed, is what a fused block must reproduce.
+
+It shares no code with the CUDA library and imports nothing from it; only
+tests, the smoke check and the CPU-baseline leg of the benchmark may call it.
+
+Operator semantics follow the ONNX vocabulary the paper classifies in Table 2
+(Section 3.1).  Operators the paper uses in Table 4 (Recip, Square, Abs,
+BitShift, ReduceSum, ReduceProd, Exp) are included so that both sides of each
+rewrite identity can be evaluated.
+
+Pinned by tests/test_oracle_*.py against closed forms, invariants and
+brute-force index loops; whole-workload outputs have no printed values in the
+paper ("parity unpinned" beyond the per-operator pins and composition).
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+_erf = np.vectorize(math.erf, otypes=[np.float64])
+
+
+def _axis(a, rank):
+    return a + rank if a < 0 else a
+
+
+# ---- One-to-One operators (Table 2, first row) ---------------------------
+
+def op_add(a, b): return a + b            # multidirectional broadcasting (Table 2: elementwise w/ broadcast)
+def op_sub(a, b): return a - b
+def op_mul(a, b): return a * b
+def op_div(a, b): return a / b
+def op_mulc(a, c): return a * float(c)
+def op_addc(a, c): return a + float(c)
+def op_sigmoid(a): return 1.0 / (1.0 + np.exp(-a))
+def op_tanh(a): return np.tanh(a)
+def op_erf(a): return _erf(a)
+def op_exp(a): return np.exp(a)
+def op_log(a): return np.log(a)
+def op_sqrt(a): return np.sqrt(a)
+def op_abs(a): return np.abs(a)
+def op_neg(a): return -a
+def op_recip(a): return 1.0 / a
+def op_square(a): return a * a
+def op_relu(a): return np.maximum(a, 0.0)
+def op_clip(a, lo, hi): return np.minimum(np.maximum(a, float(lo)), float(hi))
+def op_pow(a, p): return np.power(a, float(p))
+
+
+def op_bitshift(a, bits, direction="left"):
+    """Element-wise shift of integer-valued entries (Table 4, Commutative rows)."""
+    ai = np.rint(a).astype(np.int64)
+    r = ai << int(bits) if direction == "left" else ai >> int(bits)
+    return r.astype(np.float64)
+
+
+def op_gelu(a, approx="erf"):
+    if approx == "erf":
+        return 0.5 * a * (1.0 + _erf(a / math.sqrt(2.0)))
+    k = math.sqrt(2.0 / math.pi)
+    return 0.5 * a * (1.0 + np.tanh(k * (a + 0.044715 * a * a * a)))
+
+
+def op_scaleshift(x, scale, shift, axis=-1):
+    """Inference-time BatchNormalization folded to y = x*scale[c] + shift[c] (Table 2: One-to-One)."""
+    ax = _axis(axis, x.ndim)
+    shp = [1] * x.ndim
+    shp[ax] = x.shape[ax]
+    return x * scale.reshape(shp) + shift.reshape(shp)
+
+
+# ---- Reorganize / Shuffle (Table 2; definitions in Section 3.1) -----------
+
+def op_transpose(x, perm):
+    """out[i_0..i_{n-1}] = in[j] with j[perm[k]] = i_k  (Shuffle: permutation of the index tuple)."""
+    return np.ascontiguousarray(np.transpose(x, tuple(perm)))
+
+
+def op_reshape(x, shape):
+    """Same row-major element order under new dimensions (Reorganize)."""
+    return np.ascontiguousarray(x).reshape(tuple(int(s) for s in shape)).copy()
+
+
+def op_flatten(x, axis=1):
+    ax = _axis(axis, x.ndim)
+    lead = int(np.prod(x.shape[:ax])) if ax > 0 else 1
+    return op_reshape(x, (lead, -1))
+
+
+def op_squeeze(x, axes):
+    axes = sorted(_axis(a, x.ndim) for a in axes)
+    shp = [s for i, s in enumerate(x.shape) if i not in axes]
+    return op_reshape(x, shp)
+
+
+def op_unsqueeze(x, axes):
+    rank = x.ndim + len(axes)
+    axes = sorted(_axis(a, rank) for a in axes)
+    shp = list(x.shape)
+    for a in axes:
+        shp.insert(a, 1)
+    return op_reshape(x, shp)
+
+
+def op_split(x, axis, sizes):
+    ax = _axis(axis, x.ndim)
+    outs, start = [], 0
+    for s in sizes:
+        idx = [slice(None)] * x.ndim
+        idx[ax] = slice(start, start + int(s))
+        outs.append(np.ascontiguousarray(x[tuple(idx)]))
+        start += int(s)
+    assert start == x.shape[ax]
+    return outs
+
+
+def op_concat(xs, axis):
+    return np.concatenate(xs, axis=_axis(axis, xs[0].ndim))
+
+
+def op_slice(x, axis, start, end):
+    ax = _axis(axis, x.ndim)
+    idx = [slice(None)] * x.ndim
+    idx[ax] = slice(int(start), int(end))
+    return np.ascontiguousarray(x[tuple(idx)])
+
+
+# ---- One-to-Many -----------------------------------------------------------
+
+def op_expand(x, shape):
+    return np.ascontiguousarray(np.broadcast_to(x, tuple(int(s) for s in shape)))
+
+
+def op_gather(x, indices, axis=0):
+    return np.take(x, np.rint(indices).astype(np.int64), axis=_axis(axis, x.ndim))
+
+
+# ---- Many-to-Many (Table 2) ------------------------------------------------
+
+def op_matmul(a, b):
+    """C[..., i, j] = sum_k A[..., i, k] * B[..., k, j], leading dims broadcast."""
+    return np.matmul(a, b)
+
+
+def op_conv1x1(x, w):
+    """NHWC pointwise convolution: y[n,h,w,o] = sum_c x[n,h,w,c] * W[c,o]."""
+    return np.einsum("nhwc,co->nhwo", x, w)
+
+
+def op_dwconv3x3(x, k):
+    """NHWC depthwise 3x3, stride 1, zero padding 1:
+    y[n,h,w,c] = sum_{dh,dw in -1..1} x[n,h+dh,w+dw,c] * K[dh+1,dw+1,c]."""
+    n, h, w, c = x.shape
+    xp = np.zeros((n, h + 2, w + 2, c), dtype=np.float64)
+    xp[:, 1:h + 1, 1:w + 1, :] = x
+    y = np.zeros_like(x, dtype=np.float64)
+    for dh in range(3):
+        for dw in range(3):
+            y += xp[:, dh:dh + h, dw:dw + w, :] * k[dh, dw, :]
+    return y
+
+
+def op_softmax(x, axis=-1):
+    ax = _axis(axis, x.ndim)
+    m = np.max(x, axis=ax, keepdims=True)
+    e = np.exp(x - m)
+    return e / np.sum(e, axis=ax, keepdims=True)
+
+
+def op_layernorm(x, gamma, beta, axis=-1, eps=1e-5):
+    """Biased variance, eps inside the square root, over the last axis."""
+    ax = _axis(axis, x.ndim)
+    assert ax == x.ndim - 1
+    mu = np.mean(x, axis=ax, keepdims=True)
+    xc = x - mu
+    var = np.mean(xc * xc, axis=ax, keepdims=True)
+    return xc / np.sqrt(var + float(eps)) * gamma + beta
+
+
+def _reduce(fn, x, axis, keepdims):
+    return fn(x, axis=_axis(axis, x.ndim), keepdims=bool(keepdims))
+
+
+def op_reducesum(x, axis=-1, keepdims=1): return _reduce(np.sum, x, axis, keepdims)
+def op_reducemean(x, axis=-1, keepdims=1): return _reduce(np.mean, x, axis, keepdims)
+def op_reduceprod(x, axis=-1, keepdims=1): return _reduce(np.prod, x, axis, keepdims)
+def op_reducemax(x, axis=-1, keepdims=1): return _reduce(np.max, x, axis, keepdims)
+
+
+# ---- dispatcher -------------------------------------------------------------
+
+def _apply(op, ins, at):
+    g = at.get
+    if op == "Add": return [op_add(*ins)]
+    if op == "Sub": return [op_sub(*ins)]
+    if op == "Mul": return [op_mul(*ins)]
+    if op == "Div": return [op_div(*ins)]
+    if op == "MulC": return [op_mulc(ins[0], at["c"])]
+    if op == "AddC": return [op_addc(ins[0], at["c"])]
+    if op == "Sigmoid": return [op_sigmoid(ins[0])]
+    if op == "Tanh": return [op_tanh(ins[0])]
+    if op == "Erf": return [op_erf(ins[0])]
+    if op == "Exp": return [op_exp(ins[0])]
+    if op == "Log": return [op_log(ins[0])]
+    if op == "Sqrt": return [op_sqrt(ins[0])]
+    if op == "Abs": return [op_abs(ins[0])]
+    if op == "Neg": return [op_neg(ins[0])]
+    if op == "Recip": return [op_recip(ins[0])]
+    if op == "Square": return [op_square(ins[0])]
+    if op == "Relu": return [op_relu(ins[0])]
+    if op == "Clip": return [op_clip(ins[0], at["lo"], at["hi"])]
+    if op == "Pow": return [op_pow(ins[0], at["p"])]
+    if op == "BitShift": return [op_bitshift(ins[0], at["bits"], g("direction", "left"))]
+    if op == "Gelu": return [op_gelu(ins[0], g("approx", "erf"))]
+    if op == "ScaleShift": return [op_scaleshift(ins[0], ins[1], ins[2], g("axis", -1))]
+    if op == "Transpose": return [op_transpose(ins[0], at["perm"])]
+    if op == "Reshape": return [op_reshape(ins[0], at["shape"])]
+    if op == "Flatten": return [op_flatten(ins[0], g("axis", 1))]
+    if op == "Squeeze": return [op_squeeze(ins[0], at["axes"])]
+    if op == "Unsqueeze": return [op_unsqueeze(ins[0], at["axes"])]
+    if op == "Split": return op_split(ins[0], at["axis"], at["sizes"])
+    if op == "Concat": return [op_concat(ins, at["axis"])]
+    if op == "Slice": return [op_slice(ins[0], at["axis"], at["start"], at["end"])]
+    if op == "Expand": return [op_expand(ins[0], at["shape"])]
+    if op == "Gather": return [op_gather(ins[0], ins[1], g("axis", 0))]
+    if op == "MatMul": return [op_matmul(ins[0], ins[1])]
+    if op == "Conv1x1": return [op_conv1x1(ins[0], ins[1])]
+    if op == "DwConv3x3": return [op_dwconv3x3(ins[0], ins[1])]
+    if op == "Softmax": return [op_softmax(ins[0], g("axis", -1))]
+    if op == "LayerNorm": return [op_layernorm(ins[0], ins[1], ins[2], g("axis", -1), g("eps", 1e-5))]
+    if op == "ReduceSum": return [op_reducesum(ins[0], g("axis", -1), g("keepdims", 1))]
+    if op == "ReduceMean": return [op_reducemean(ins[0], g("axis", -1), g("keepdims", 1))]
+    if op == "ReduceProd": return [op_reduceprod(ins[0], g("axis", -1), g("keepdims", 1))]
+    if op == "ReduceMax": return [op_reducemax(ins[0], g("axis", -1), g("keepdims", 1))]
+    raise KeyError(f"oracle: unknown operator {op}")
+
+
+def run_graph(graph, inputs, keep_all=False):
+    """Evaluate `graph` (an object with .ops, .outputs; each op has .op, .inputs,
+    .outputs, .attrs) on `inputs` (name -> array).  Returns name -> fp64 array
+    for the marked outputs (or every tensor when keep_all)."""
+    env = {k: np.asarray(v, dtype=np.float64) for k, v in inputs.items()}
+    for o in graph.ops:
+        ins = [env[n] for n in o.inputs]
+        outs = _apply(o.op, ins, o.attrs)
+        assert len(outs) == len(o.outputs), (o.op, len(outs), len(o.outputs))
+        for n, v in zip(o.outputs, outs):
+            env[n] = np.asarray(v, dtype=np.float64)
+    if keep_all:
+        return env
+    return {n: env[n] for n in graph.outputs}
