@@ -1,0 +1,252 @@
+/*
+ * dnnf.h -- C ABI of the fused operator-block executor.
+ *
+ * The library takes a computational graph (operators with type and parameters,
+ * tensors, data-flow; paper Section 4.1), annotates every operator with its
+ * mapping type (Section 3.1, Table 2) to form the Extended Computational Graph,
+ * optionally rewrites it with mathematical-property rules (Section 4.2,
+ * Table 4), groups operators into fusion blocks (Section 4.3, Listing 1,
+ * Table 3) and runs every block as ONE CUDA kernel that keeps the block's
+ * intermediates in registers / shared memory / tensor memory (Section 4.4).
+ *
+ * Conventions
+ *  - Every function returns a dnnf_status_t; DNNF_OK is 0.  No exception crosses
+ *    this boundary; a failed call leaves the graph usable and stores a message
+ *    retrievable with dnnf_last_error().
+ *  - Pointers named host_* are host memory; pointers named dev_* are device
+ *    memory owned by the caller.  The library never allocates device memory and
+ *    never synchronises inside dnnf_run().
+ *  - Tensors are dense, row-major (last dimension contiguous).
+ *  - Call order: create -> add_tensor/add_op/mark_output -> [rewrite] -> plan ->
+ *    bind/bind_workspace -> run.  add_* after plan returns DNNF_ERR_STATE.
+ *  - A handle is not thread-safe; distinct handles are independent.
+ *  - There is no CPU fallback: a block with no kernel family makes dnnf_plan()
+ *    fail with DNNF_ERR_UNSUPPORTED_OP.
+ */
+#ifndef DNNF_H_
+#define DNNF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define DNNF_API __attribute__((visibility("default")))
+#else
+#define DNNF_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dnnf_graph dnnf_graph;   /* opaque; freed by dnnf_graph_destroy */
+
+typedef enum {
+  DNNF_OK = 0,
+  DNNF_ERR_INVALID_ARG = 1,
+  DNNF_ERR_SHAPE = 2,
+  DNNF_ERR_UNSUPPORTED_OP = 3,
+  DNNF_ERR_STATE = 4,
+  DNNF_ERR_UNBOUND = 5,
+  DNNF_ERR_WORKSPACE = 6,
+  DNNF_ERR_CUDA = 7,
+  DNNF_ERR_TIMEOUT = 8
+} dnnf_status_t;
+
+typedef enum { DNNF_F32 = 0, DNNF_BF16 = 1 } dnnf_dtype_t;
+typedef enum { DNNF_INPUT = 0, DNNF_WEIGHT = 1 } dnnf_tensor_kind_t;
+
+/* The five mapping types of Section 3.1, in the paper's order of increasing
+ * complexity (used to type an operator with mixed input/output pairs). */
+typedef enum {
+  DNNF_ONE_TO_ONE = 0, DNNF_REORGANIZE = 1, DNNF_SHUFFLE = 2,
+  DNNF_ONE_TO_MANY = 3, DNNF_MANY_TO_MANY = 4
+} dnnf_mapping_t;
+
+/* Table 3 cell colours. */
+typedef enum { DNNF_FUSE_THROUGH = 0 /*green*/, DNNF_FUSE_DEPEND = 1 /*yellow*/, DNNF_FUSE_BREAK = 2 /*red*/ } dnnf_fuse_t;
+
+/* Operator vocabulary (ONNX names as classified in Table 2, plus the
+ * element-wise operators Table 4 uses). */
+typedef enum {
+  DNNF_OP_ADD = 1, DNNF_OP_SUB, DNNF_OP_MUL, DNNF_OP_DIV,
+  DNNF_OP_MULC, DNNF_OP_ADDC,                       /* scalar attribute C */
+  DNNF_OP_SIGMOID, DNNF_OP_TANH, DNNF_OP_ERF, DNNF_OP_EXP, DNNF_OP_LOG, DNNF_OP_SQRT,
+  DNNF_OP_ABS, DNNF_OP_NEG, DNNF_OP_RECIP, DNNF_OP_SQUARE, DNNF_OP_RELU,
+  DNNF_OP_CLIP,                                     /* attributes LO, HI */
+  DNNF_OP_POW,                                      /* attribute P */
+  DNNF_OP_GELU,                                     /* attribute APPROX: 0 erf, 1 tanh */
+  DNNF_OP_SCALESHIFT,                               /* (x, scale[c], shift[c]); attribute AXIS */
+  DNNF_OP_TRANSPOSE,                                /* attribute PERM */
+  DNNF_OP_RESHAPE,                                  /* attribute SHAPE (one -1 allowed) */
+  DNNF_OP_FLATTEN, DNNF_OP_SQUEEZE, DNNF_OP_UNSQUEEZE, /* attribute AXIS / AXES */
+  DNNF_OP_SPLIT,                                    /* attributes AXIS, SIZES; several outputs */
+  DNNF_OP_SLICE,                                    /* attributes AXIS, START, END */
+  DNNF_OP_MATMUL,
+  DNNF_OP_CONV1X1,                                  /* NHWC x [Cin,Cout] */
+  DNNF_OP_DWCONV3X3,                                /* NHWC x [3,3,C], stride 1, zero pad 1 */
+  DNNF_OP_SOFTMAX,                                  /* attribute AXIS (last axis only) */
+  DNNF_OP_LAYERNORM,                                /* (x, gamma, beta); attributes AXIS, EPS */
+  DNNF_OP_REDUCESUM, DNNF_OP_REDUCEMEAN, DNNF_OP_REDUCEMAX, DNNF_OP_REDUCEPROD, /* AXIS (last), KEEPDIMS */
+  DNNF_OP_EXPAND,                                   /* attribute SHAPE */
+  DNNF_OP_BITSHIFT,                                 /* attribute BITS; planning/rewriting only */
+  DNNF_OP__COUNT
+} dnnf_op_t;
+
+typedef enum {
+  DNNF_ATTR_C = 1, DNNF_ATTR_LO, DNNF_ATTR_HI, DNNF_ATTR_P, DNNF_ATTR_EPS,   /* use f */
+  DNNF_ATTR_APPROX, DNNF_ATTR_AXIS, DNNF_ATTR_KEEPDIMS, DNNF_ATTR_START, DNNF_ATTR_END, DNNF_ATTR_BITS, /* use i[0] */
+  DNNF_ATTR_PERM, DNNF_ATTR_SHAPE, DNNF_ATTR_SIZES, DNNF_ATTR_AXES            /* use i[0..n) */
+} dnnf_attr_key_t;
+
+typedef struct {
+  int32_t key;      /* dnnf_attr_key_t */
+  int32_t n;        /* number of valid entries in i[] */
+  int64_t i[8];
+  double  f;
+} dnnf_attr;
+
+/* dnnf_rewrite flags */
+#define DNNF_REWRITE_DEFAULT        0u
+#define DNNF_REWRITE_NONE           1u   /* leave the graph as given */
+#define DNNF_REWRITE_CANON_MACRO    2u   /* also fold the 9-operator LayerNorm expansion into one LayerNorm
+                                            operator (an extension beyond the paper's printed rules) */
+/* dnnf_plan flags */
+#define DNNF_PLAN_FUSED             0u
+#define DNNF_PLAN_UNFUSED           1u   /* one block per operator: the no-fusion baseline of Section 5 ("OurB") */
+#define DNNF_PLAN_STRICT_TABLE3     2u   /* type a broadcast operand's consumer One-to-Many on every edge */
+#define DNNF_PLAN_ALLOW_PROLOGUE    4u   /* planning only: let One-to-One predecessors fuse in front of a
+                                            GEMM/conv anchor (Listing 1 literal); such plans cannot be run */
+
+typedef struct {
+  int32_t ops_before, ops_after;
+  int64_t flops_before, flops_after;       /* Table 4's #FLOPS model */
+  int32_t rules_applied;
+  int32_t applied_by_rule[16];             /* index: see dnnf_rule_name() */
+  int32_t folded_constants;
+} dnnf_rewrite_stats;
+
+typedef struct {
+  int32_t n_ops;               /* original operators (a Split counts once) */
+  int32_t n_blocks;            /* fusion blocks */
+  int32_t n_kernels;           /* blocks that launch a kernel (an isolated Reshape launches none) */
+  double  fusion_rate;         /* n_ops / n_blocks (Section 5.2) */
+  int64_t irs_bytes_unfused;   /* bytes of all operator outputs that are not graph outputs */
+  int64_t irs_bytes_fused;     /* bytes of intermediates still materialised between blocks */
+  int64_t workspace_bytes;
+  int32_t n_yellow_decisions;  /* Table 3 yellow cells resolved by the cost model */
+  int32_t n_yellow_fused;
+} dnnf_plan_stats;
+
+typedef enum {
+  DNNF_FAMILY_ALIAS = 0,       /* pure Reorganize: zero-copy */
+  DNNF_FAMILY_ELEMENTWISE = 1, /* One-to-One / broadcast chain, contiguous */
+  DNNF_FAMILY_TRANSPOSE = 2,   /* chain with a Shuffle staged through shared memory */
+  DNNF_FAMILY_ROW = 3,         /* chain around a last-axis reduction (Softmax, LayerNorm, Reduce*) */
+  DNNF_FAMILY_GEMM = 4,        /* tensor-core GEMM anchor with an epilogue chain */
+  DNNF_FAMILY_CONV1X1 = 5,     /* fp32 pointwise convolution with an epilogue chain */
+  DNNF_FAMILY_DWCONV = 6       /* fp32 depthwise 3x3 with an epilogue chain */
+} dnnf_family_t;
+
+typedef struct {
+  int32_t family;              /* dnnf_family_t */
+  int32_t mapping;             /* dnnf_mapping_t of the fused block */
+  int32_t n_ops;
+  int32_t op_kinds[48];        /* dnnf_op_t of the first 48 operators */
+  int32_t n_inputs, n_outputs;
+  int64_t bytes_in, bytes_out; /* algorithmic HBM bytes: each external input/output once */
+  int64_t flops;               /* 2*M*N*K for contraction anchors, else 0 */
+  int32_t n_microops;
+  int32_t grid, threads;
+  int32_t variant;             /* kernel specialisation chosen (family-specific) */
+} dnnf_block_desc;
+
+/* ---- graph construction (Section 4.1: the computational graph handed over by a
+ *      host framework) ------------------------------------------------------- */
+
+/* Creates an empty graph.  *out is owned by the library until dnnf_graph_destroy. */
+DNNF_API int dnnf_graph_create(dnnf_graph** out);
+DNNF_API int dnnf_graph_destroy(dnnf_graph* g);
+
+/* Declares an external tensor (model input or weight).  host_dims has `rank`
+ * entries (rank <= 6).  Returns its id in *tensor_id. */
+DNNF_API int dnnf_add_tensor(dnnf_graph* g, const char* name, int dtype, int rank,
+                    const int64_t* host_dims, int kind, int* tensor_id);
+
+/* Appends an operator.  host_in_ids are ids returned earlier; outputs are created
+ * by shape inference and their ids written to host_out_ids (capacity max_out),
+ * their count to *n_out.  The operator is tagged with its mapping type
+ * (Table 2; an operator with mixed input/output pairs takes the most complex
+ * one, Section 3.1).  Output dtype is the dtype of input 0. */
+DNNF_API int dnnf_add_op(dnnf_graph* g, int op_kind, int n_in, const int* host_in_ids,
+                const dnnf_attr* host_attrs, int n_attrs,
+                int max_out, int* host_out_ids, int* n_out);
+
+/* Marks a tensor as a result the caller wants (never removable, Section 3.2
+ * "IR_removable"). */
+DNNF_API int dnnf_mark_output(dnnf_graph* g, int tensor_id);
+
+/* Tensor introspection: rank and dims (capacity 6), dtype. */
+DNNF_API int dnnf_tensor_info(const dnnf_graph* g, int tensor_id, int* dtype, int* rank, int64_t* host_dims);
+/* Mapping type the ECG holds for operator `op_index` (insertion order). */
+DNNF_API int dnnf_op_mapping(const dnnf_graph* g, int op_index, int* mapping);
+
+/* ---- Table 3 ------------------------------------------------------------------ */
+
+/* Mapping-type analysis of fusing `first` then `second` (both dnnf_mapping_t):
+ * writes the fused block's mapping type and the cell colour. */
+DNNF_API int dnnf_mapping_check(int first, int second, int* fused_mapping, int* colour);
+
+/* ---- Section 4.2: mathematical-property graph rewriting ------------------------ */
+
+/* Partitions the graph at operators with no associative/commutative/distributive
+ * property, matches the printed rules of Table 4 inside each partition, applies
+ * the match with the largest #FLOPS reduction and repeats to a fixed point.
+ * stats may be NULL. */
+DNNF_API int dnnf_rewrite(dnnf_graph* g, uint32_t flags, dnnf_rewrite_stats* host_stats);
+DNNF_API const char* dnnf_rule_name(int rule_index);
+
+/* ---- Section 4.3: fusion-plan generation ---------------------------------------- */
+
+/* Listing 1: seed = One-to-One operator with the smallest intermediate result;
+ * grow along successors, then predecessors, consulting Table 3 (green: fuse,
+ * red: stop, yellow: cost model) and a constraint check; repeat over seeds.
+ * Then lowers every block to one kernel launch (data-flow-tree traversal of
+ * Section 4.4).  stats may be NULL. */
+DNNF_API int dnnf_plan(dnnf_graph* g, uint32_t flags, dnnf_plan_stats* host_stats);
+DNNF_API int dnnf_block_count(const dnnf_graph* g, int* n_blocks);
+DNNF_API int dnnf_block_info(const dnnf_graph* g, int block, dnnf_block_desc* host_out);
+/* Block index that holds operator `op_index` (insertion order), after dnnf_plan. */
+DNNF_API int dnnf_op_block(const dnnf_graph* g, int op_index, int* block);
+/* Number of operators currently alive (after rewriting) and their kinds. */
+DNNF_API int dnnf_op_count(const dnnf_graph* g, int* n_ops);
+DNNF_API int dnnf_op_kind(const dnnf_graph* g, int op_index, int* kind, int* alive);
+
+/* ---- binding and execution (Section 4.4: one generated kernel per block) -------- */
+
+/* Bytes of caller-provided device workspace the plan needs for intermediates
+ * that stay materialised between blocks plus a small status area. */
+DNNF_API int dnnf_workspace_size(const dnnf_graph* g, size_t* bytes);
+/* dev_ptr: device memory of the tensor's full size, 16-byte aligned, caller-owned. */
+DNNF_API int dnnf_bind(dnnf_graph* g, int tensor_id, void* dev_ptr);
+/* dev_ptr: device memory, 256-byte aligned, at least dnnf_workspace_size bytes. */
+DNNF_API int dnnf_bind_workspace(dnnf_graph* g, void* dev_ptr, size_t bytes);
+/* Launches every block's kernel in topological order on `cuda_stream`
+ * (a cudaStream_t; NULL = default stream).  Asynchronous. */
+DNNF_API int dnnf_run(dnnf_graph* g, void* cuda_stream);
+/* Launches only block `block` (for per-block timing). */
+DNNF_API int dnnf_run_block(dnnf_graph* g, int block, void* cuda_stream);
+/* After the caller synchronised the stream: device-side status word
+ * (0 = ok, DNNF_ERR_TIMEOUT if a bounded wait inside a kernel ran out) and the
+ * block that reported it. */
+DNNF_API int dnnf_status(dnnf_graph* g, int* device_status, int* block);
+/* Number of kernels one dnnf_run launches. */
+DNNF_API int dnnf_launch_count(const dnnf_graph* g, int* n);
+
+DNNF_API const char* dnnf_last_error(const dnnf_graph* g);
+DNNF_API const char* dnnf_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DNNF_H_ */

@@ -1,0 +1,299 @@
+// C ABI: argument checking, state machine, error messages.  No exception leaves
+// this file.
+#include <cstring>
+#include <exception>
+
+#include "ir.h"
+
+using namespace dnnf;
+
+namespace dnnf {
+int run_blocks(Graph& g, int only_block, void* stream);
+int read_status(Graph& g, int* status, int* block);
+}
+
+#define DNNF_TRY try {
+#define DNNF_CATCH(gptr)                                                              \
+  } catch (const std::exception& e) { if (gptr) (gptr)->g.err = e.what(); return DNNF_ERR_INVALID_ARG; } \
+    catch (...) { if (gptr) (gptr)->g.err = "unknown exception"; return DNNF_ERR_INVALID_ARG; }
+
+static int fail(dnnf_graph* g, int code, const char* msg) { if (g) g->g.err = msg; return code; }
+
+extern "C" {
+
+const char* dnnf_version(void) { return "dnnf-b200 0.1"; }
+
+int dnnf_graph_create(dnnf_graph** out) {
+  if (!out) return DNNF_ERR_INVALID_ARG;
+  DNNF_TRY
+  *out = new dnnf_graph();
+  return DNNF_OK;
+  DNNF_CATCH((dnnf_graph*)nullptr)
+}
+
+int dnnf_graph_destroy(dnnf_graph* g) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  delete g;
+  return DNNF_OK;
+}
+
+const char* dnnf_last_error(const dnnf_graph* g) { return g ? g->g.err.c_str() : "null graph"; }
+
+int dnnf_add_tensor(dnnf_graph* g, const char* name, int dtype, int rank, const int64_t* dims, int kind, int* tensor_id) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  DNNF_TRY
+  if (g->g.planned || !g->g.blocks.empty()) return fail(g, DNNF_ERR_STATE, "graph is already planned");
+  if (!dims || !tensor_id || rank < 0 || rank > kMaxDims) return fail(g, DNNF_ERR_INVALID_ARG, "bad rank or null pointer");
+  if (dtype != DNNF_F32 && dtype != DNNF_BF16) return fail(g, DNNF_ERR_INVALID_ARG, "unknown dtype");
+  std::vector<int64_t> d(dims, dims + rank);
+  for (auto v : d) if (v <= 0) return fail(g, DNNF_ERR_SHAPE, "dimensions must be positive");
+  int id = g->g.add_tensor(name ? name : "", dtype, d);
+  g->g.tensors[id].external = true;
+  g->g.tensors[id].weight = (kind == DNNF_WEIGHT);
+  *tensor_id = id;
+  return DNNF_OK;
+  DNNF_CATCH(g)
+}
+
+static int parse_attrs(const dnnf_attr* a, int n, Attrs& at, std::string& err) {
+  for (int i = 0; i < n; ++i) {
+    const dnnf_attr& x = a[i];
+    if (x.n < 0 || x.n > 8) { err = "attribute length"; return DNNF_ERR_INVALID_ARG; }
+    std::vector<int64_t> v(x.i, x.i + x.n);
+    switch (x.key) {
+      case DNNF_ATTR_C: at.c = x.f; break;
+      case DNNF_ATTR_LO: at.lo = x.f; break;
+      case DNNF_ATTR_HI: at.hi = x.f; break;
+      case DNNF_ATTR_P: at.p = x.f; break;
+      case DNNF_ATTR_EPS: at.eps = x.f; break;
+      case DNNF_ATTR_APPROX: at.approx = x.i[0]; break;
+      case DNNF_ATTR_AXIS: at.axis = x.i[0]; break;
+      case DNNF_ATTR_KEEPDIMS: at.keepdims = x.i[0]; break;
+      case DNNF_ATTR_START: at.start = x.i[0]; break;
+      case DNNF_ATTR_END: at.end = x.i[0]; break;
+      case DNNF_ATTR_BITS: at.bits = x.i[0]; break;
+      case DNNF_ATTR_PERM: at.perm = v; break;
+      case DNNF_ATTR_SHAPE: at.shape = v; break;
+      case DNNF_ATTR_SIZES: at.sizes = v; break;
+      case DNNF_ATTR_AXES: at.axes = v; break;
+      default: err = "unknown attribute key"; return DNNF_ERR_INVALID_ARG;
+    }
+  }
+  return DNNF_OK;
+}
+
+int dnnf_add_op(dnnf_graph* g, int op_kind, int n_in, const int* in_ids, const dnnf_attr* attrs, int n_attrs,
+                int max_out, int* out_ids, int* n_out) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  DNNF_TRY
+  Graph& G = g->g;
+  if (G.planned || !G.blocks.empty()) return fail(g, DNNF_ERR_STATE, "graph is already planned");
+  if (op_kind <= 0 || op_kind >= DNNF_OP__COUNT) return fail(g, DNNF_ERR_UNSUPPORTED_OP, "unknown operator kind");
+  if (n_in <= 0 || n_in > 4 || !in_ids || !out_ids || !n_out || (n_attrs > 0 && !attrs)) return fail(g, DNNF_ERR_INVALID_ARG, "bad argument");
+  for (int i = 0; i < n_in; ++i) if (in_ids[i] < 0 || in_ids[i] >= (int)G.tensors.size()) return fail(g, DNNF_ERR_INVALID_ARG, "input id out of range");
+  Attrs at;
+  std::string err;
+  int rc = parse_attrs(attrs, n_attrs, at, err);
+  if (rc) { G.err = err; return rc; }
+  size_t n_tensors_before = G.tensors.size(), n_ops_before = G.ops.size();
+  auto rollback = [&]() { G.tensors.resize(n_tensors_before); G.ops.resize(n_ops_before); };
+  int source = G.n_source_ops;
+  std::vector<int> outs;
+  if (op_kind == DNNF_OP_SPLIT) {
+    // A Split is n Slices of one tensor (Table 2 lists both as One-to-One); the ECG holds the Slices.
+    const Tensor& X = G.tensors[in_ids[0]];
+    int rank = (int)X.dims.size();
+    int64_t ax = at.axis < 0 ? at.axis + rank : at.axis;
+    if (ax < 0 || ax >= rank || at.sizes.empty()) return fail(g, DNNF_ERR_SHAPE, "Split: axis or sizes");
+    int64_t tot = 0;
+    for (auto s : at.sizes) tot += s;
+    if (tot != X.dims[ax]) return fail(g, DNNF_ERR_SHAPE, "Split: sizes do not sum to the axis length");
+    int64_t start = 0;
+    for (auto s : at.sizes) {
+      Op o; o.id = (int)G.ops.size(); o.kind = DNNF_OP_SLICE; o.source_id = source; o.in = {in_ids[0]};
+      o.at.axis = ax; o.at.start = start; o.at.end = start + s;
+      rc = infer_shapes(G, o, err);
+      if (rc) { rollback(); G.err = err; return rc; }
+      outs.push_back(o.out[0]);
+      G.ops.push_back(o);
+      start += s;
+    }
+  } else {
+    Op o; o.id = (int)G.ops.size(); o.kind = op_kind; o.source_id = source; o.in.assign(in_ids, in_ids + n_in); o.at = at;
+    rc = infer_shapes(G, o, err);
+    if (rc) { rollback(); G.err = err; return rc; }
+    outs = o.out;
+    G.ops.push_back(o);
+  }
+  if ((int)outs.size() > max_out) { rollback(); return fail(g, DNNF_ERR_INVALID_ARG, "out_ids capacity too small"); }
+  for (size_t i = n_ops_before; i < G.ops.size(); ++i) { G.ops[i].mapping = node_mapping(G, G.ops[i]); G.ops[i].props = math_props(G.ops[i].kind); }
+  for (size_t i = 0; i < outs.size(); ++i) out_ids[i] = outs[i];
+  *n_out = (int)outs.size();
+  G.n_source_ops++;
+  return DNNF_OK;
+  DNNF_CATCH(g)
+}
+
+int dnnf_mark_output(dnnf_graph* g, int t) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  if (g->g.planned || !g->g.blocks.empty()) return fail(g, DNNF_ERR_STATE, "graph is already planned");
+  if (t < 0 || t >= (int)g->g.tensors.size()) return fail(g, DNNF_ERR_INVALID_ARG, "tensor id out of range");
+  if (g->g.tensors[t].external) return fail(g, DNNF_ERR_INVALID_ARG, "an external tensor cannot be an output");
+  g->g.tensors[t].is_output = true;
+  return DNNF_OK;
+}
+
+int dnnf_tensor_info(const dnnf_graph* g, int t, int* dtype, int* rank, int64_t* dims) {
+  if (!g || t < 0 || t >= (int)g->g.tensors.size()) return DNNF_ERR_INVALID_ARG;
+  const Tensor& T = g->g.tensors[t];
+  if (dtype) *dtype = T.dtype;
+  if (rank) *rank = (int)T.dims.size();
+  if (dims) for (size_t i = 0; i < T.dims.size(); ++i) dims[i] = T.dims[i];
+  return DNNF_OK;
+}
+
+int dnnf_op_mapping(const dnnf_graph* g, int op, int* mapping) {
+  if (!g || !mapping || op < 0 || op >= (int)g->g.ops.size()) return DNNF_ERR_INVALID_ARG;
+  *mapping = node_mapping(g->g, g->g.ops[op]);
+  return DNNF_OK;
+}
+
+int dnnf_mapping_check(int first, int second, int* fused, int* colour) {
+  if (first < 0 || first > 4 || second < 0 || second > 4 || !fused || !colour) return DNNF_ERR_INVALID_ARG;
+  table3(first, second, fused, colour);
+  return DNNF_OK;
+}
+
+int dnnf_rewrite(dnnf_graph* g, uint32_t flags, dnnf_rewrite_stats* st) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  DNNF_TRY
+  if (g->g.planned || !g->g.blocks.empty()) return fail(g, DNNF_ERR_STATE, "rewrite must come before plan");
+  return rewrite_graph(g->g, flags, st);
+  DNNF_CATCH(g)
+}
+
+int dnnf_plan(dnnf_graph* g, uint32_t flags, dnnf_plan_stats* st) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  DNNF_TRY
+  if (g->g.ops.empty()) return fail(g, DNNF_ERR_STATE, "empty graph");
+  bool any_out = false;
+  for (auto& t : g->g.tensors) any_out |= t.is_output;
+  if (!any_out) return fail(g, DNNF_ERR_STATE, "no output marked");
+  int rc = plan_graph(g->g, flags);
+  if (rc == DNNF_OK && st) *st = g->g.pstats;
+  return rc;
+  DNNF_CATCH(g)
+}
+
+int dnnf_block_count(const dnnf_graph* g, int* n) {
+  if (!g || !n) return DNNF_ERR_INVALID_ARG;
+  *n = (int)g->g.blocks.size();
+  return DNNF_OK;
+}
+
+int dnnf_block_info(const dnnf_graph* g, int bi, dnnf_block_desc* out) {
+  if (!g || !out || bi < 0 || bi >= (int)g->g.blocks.size()) return DNNF_ERR_INVALID_ARG;
+  const Graph& G = g->g;
+  const Block& b = G.blocks[bi];
+  std::memset(out, 0, sizeof *out);
+  out->family = b.launch.family;
+  out->mapping = b.mapping;
+  out->n_ops = (int)b.ops.size();
+  for (size_t i = 0; i < b.ops.size() && i < 48; ++i) out->op_kinds[i] = G.ops[b.ops[i]].kind;
+  out->n_inputs = (int)b.inputs.size();
+  out->n_outputs = (int)b.outputs.size();
+  for (int t : b.inputs) out->bytes_in += G.tensors[t].bytes();
+  for (int t : b.outputs) out->bytes_out += G.tensors[t].bytes();
+  out->flops = b.launch.flops;
+  out->n_microops = b.launch.family == DNNF_FAMILY_ROW ? b.launch.row.prog.n : b.launch.ew.prog.n;
+  out->grid = b.launch.grid;
+  out->threads = b.launch.threads;
+  out->variant = b.launch.variant;
+  return DNNF_OK;
+}
+
+int dnnf_op_block(const dnnf_graph* g, int op, int* block) {
+  if (!g || !block || op < 0 || op >= (int)g->g.ops.size()) return DNNF_ERR_INVALID_ARG;
+  *block = g->g.ops[op].block;
+  return DNNF_OK;
+}
+
+int dnnf_op_count(const dnnf_graph* g, int* n) {
+  if (!g || !n) return DNNF_ERR_INVALID_ARG;
+  *n = (int)g->g.ops.size();
+  return DNNF_OK;
+}
+
+int dnnf_op_kind(const dnnf_graph* g, int op, int* kind, int* alive) {
+  if (!g || op < 0 || op >= (int)g->g.ops.size()) return DNNF_ERR_INVALID_ARG;
+  if (kind) *kind = g->g.ops[op].kind;
+  if (alive) *alive = g->g.ops[op].alive ? 1 : 0;
+  return DNNF_OK;
+}
+
+int dnnf_workspace_size(const dnnf_graph* g, size_t* bytes) {
+  if (!g || !bytes) return DNNF_ERR_INVALID_ARG;
+  if (!g->g.planned) return DNNF_ERR_STATE;
+  *bytes = g->g.ws_bytes;
+  return DNNF_OK;
+}
+
+int dnnf_bind(dnnf_graph* g, int t, void* dev_ptr) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  Graph& G = g->g;
+  if (t < 0 || t >= (int)G.tensors.size()) return fail(g, DNNF_ERR_INVALID_ARG, "tensor id out of range");
+  if (!dev_ptr || ((uintptr_t)dev_ptr & 15)) return fail(g, DNNF_ERR_INVALID_ARG, "device pointer must be non-null and 16-byte aligned");
+  if (!G.tensors[t].external && !G.tensors[t].is_output) return fail(g, DNNF_ERR_INVALID_ARG, "only external tensors and marked outputs can be bound");
+  G.tensors[t].bound = dev_ptr;
+  return DNNF_OK;
+}
+
+int dnnf_bind_workspace(dnnf_graph* g, void* dev_ptr, size_t bytes) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  Graph& G = g->g;
+  if (!G.planned) return fail(g, DNNF_ERR_STATE, "plan first");
+  if (!dev_ptr || ((uintptr_t)dev_ptr & 255)) return fail(g, DNNF_ERR_INVALID_ARG, "workspace must be non-null and 256-byte aligned");
+  if (bytes < G.ws_bytes) return fail(g, DNNF_ERR_WORKSPACE, "workspace too small");
+  G.ws_ptr = dev_ptr; G.ws_bound_bytes = bytes;
+  return DNNF_OK;
+}
+
+int dnnf_run(dnnf_graph* g, void* stream) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  DNNF_TRY
+  return run_blocks(g->g, -1, stream);
+  DNNF_CATCH(g)
+}
+
+int dnnf_run_block(dnnf_graph* g, int block, void* stream) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  DNNF_TRY
+  if (block < 0 || block >= (int)g->g.blocks.size()) return fail(g, DNNF_ERR_INVALID_ARG, "block index out of range");
+  return run_blocks(g->g, block, stream);
+  DNNF_CATCH(g)
+}
+
+int dnnf_status(dnnf_graph* g, int* status, int* block) {
+  if (!g || !status) return DNNF_ERR_INVALID_ARG;
+  DNNF_TRY
+  return read_status(g->g, status, block);
+  DNNF_CATCH(g)
+}
+
+int dnnf_launch_count(const dnnf_graph* g, int* n) {
+  if (!g || !n) return DNNF_ERR_INVALID_ARG;
+  if (!g->g.planned) return DNNF_ERR_STATE;
+  *n = g->g.pstats.n_kernels;
+  return DNNF_OK;
+}
+
+const char* dnnf_rule_name(int i) {
+  static const char* names[] = {"assoc:recip-recip-mul", "assoc:sqrt-sqrt", "assoc:abs-abs", "assoc:reducesum-square",
+                                "dist:common-factor", "dist:a-plus-a-mul-b", "dist:square-minus-product",
+                                "comm:swap-operands", "comm:reducesum-bitshift", "comm:reduceprod-exp",
+                                "strength:pow-to-square-sqrt", "fold:constant", "canon:layernorm"};
+  if (i < 0 || i >= (int)(sizeof names / sizeof names[0])) return "";
+  return names[i];
+}
+
+}  // extern "C"

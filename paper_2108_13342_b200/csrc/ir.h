@@ -1,0 +1,130 @@
+// Extended Computational Graph (Section 3.2): operators, tensors, data-flow, plus
+// mapping type per operator, IR_removable per tensor and mathematical-property
+// flags; fusion blocks and their lowered launches.
+#pragma once
+#include <cstdint>
+#include <map>
+#include <string>
+#include <vector>
+
+#include "../../include/dnnf.h"
+#include "microop.h"
+
+namespace dnnf {
+
+struct Attrs {
+  double c = 0, lo = 0, hi = 0, p = 0, eps = 1e-5;
+  int64_t approx = 0, axis = -1, keepdims = 1, start = 0, end = 0, bits = 0;
+  std::vector<int64_t> perm, shape, sizes, axes;
+};
+
+struct Tensor {
+  int id = -1;
+  std::string name;
+  int dtype = DNNF_F32;
+  std::vector<int64_t> dims;
+  bool external = false;       // declared by dnnf_add_tensor
+  bool weight = false;
+  bool is_output = false;      // marked by the caller
+  int producer = -1;           // op id, -1 for externals
+  std::vector<int> consumers;  // op ids (alive ops only; rebuilt by Graph::relink)
+  bool removable = false;      // IR_removable: all consumers sit in the producer's block
+  int64_t ws_offset = -1;      // workspace offset (bytes) when materialised between blocks
+  int alias_of = -1;           // zero-copy Reorganize result: shares storage with this tensor
+  void* bound = nullptr;       // caller-bound device pointer (externals and outputs)
+  int64_t numel() const { int64_t n = 1; for (auto d : dims) n *= d; return n; }
+  int64_t bytes() const { return numel() * (dtype == DNNF_BF16 ? 2 : 4); }
+};
+
+enum MathProp : uint32_t { P_ASSOC = 1, P_COMM = 2, P_DIST = 4 };
+
+struct Op {
+  int id = -1;
+  int kind = 0;
+  int source_id = -1;          // original operator this came from (a Split expands to Slices)
+  std::vector<int> in, out;
+  Attrs at;
+  int mapping = DNNF_ONE_TO_ONE;
+  uint32_t props = 0;
+  bool alive = true;
+  int block = -1;
+};
+
+// A lowered block = one kernel launch (or none for a zero-copy alias).
+struct ArgRef { int tensor; };   // which tensor supplies TensorArg.ptr at bind time
+
+struct GemmLaunch;   // defined in gemm_host.h
+struct ConvLaunch;
+
+struct Launch {
+  int family = DNNF_FAMILY_ALIAS;
+  int variant = 0;
+  int grid = 0, threads = 0;
+  size_t smem = 0;
+  EwParams ew{};
+  RowParams row{};
+  std::vector<int> in_tensors, out_tensors;     // parallel to params.in[] / out[]
+  std::vector<uint8_t> blob;                    // family-specific parameter block (GEMM / conv)
+  int64_t flops = 0;
+};
+
+struct Block {
+  std::vector<int> ops;        // op ids, topological
+  int mapping = DNNF_ONE_TO_ONE;
+  std::vector<int> inputs, outputs;   // external tensor ids of the block
+  Launch launch;
+  bool lowered = false;
+};
+
+struct Graph {
+  std::vector<Tensor> tensors;
+  std::vector<Op> ops;
+  std::vector<Block> blocks;
+  std::vector<int> run_order;            // block indices in execution order
+  int n_source_ops = 0;
+  bool planned = false;
+  uint32_t plan_flags = 0;
+  size_t ws_bytes = 0;
+  void* ws_ptr = nullptr;
+  size_t ws_bound_bytes = 0;
+  dnnf_plan_stats pstats{};
+  std::string err;
+
+  int add_tensor(const std::string& name, int dtype, const std::vector<int64_t>& dims);
+  void relink();                          // rebuild producer/consumer lists over alive ops
+  std::vector<int> topo_order() const;    // alive ops in topological order
+};
+
+// ---- mapping types (ir.cpp) ----
+int node_mapping(const Graph& g, const Op& op);                 // Table 2 + most-complex-pair rule
+int edge_mapping(const Graph& g, const Op& op, int in_slot);    // mapping of one (input, output) pair
+uint32_t math_props(int kind);
+void table3(int first, int second, int* fused, int* colour);
+bool is_index_only(int kind);       // Reorganize / Shuffle / Slice: no arithmetic
+bool is_elementwise(int kind);
+bool is_row_anchor(int kind);
+bool is_contraction(int kind);
+const char* op_name(int kind);
+int infer_shapes(Graph& g, Op& op, std::string& err);           // creates output tensors
+
+// ---- rewrite.cpp ----
+int rewrite_graph(Graph& g, uint32_t flags, dnnf_rewrite_stats* st);
+int64_t graph_flops(const Graph& g);
+
+// ---- plan.cpp ----
+int plan_graph(Graph& g, uint32_t flags);
+
+// ---- lower.cpp ----
+// Lowers `ops` (a candidate block) into a launch.  Returns DNNF_OK or an error;
+// `why` explains a refusal (used as the constraint check of Listing 1, Step 2.2).
+int lower_block(const Graph& g, const std::vector<int>& ops, uint32_t flags, Block& out, std::string& why);
+double block_cost_us(const Graph& g, const Block& b);
+
+// ---- launch (kernels_*.cu) ----
+int launch_block(Graph& g, Block& b, void* stream, std::string& err);
+
+}  // namespace dnnf
+
+struct dnnf_graph {
+  dnnf::Graph g;
+};

@@ -1,0 +1,352 @@
+// Fusion-plan generation (Section 4.3, Listing 1) and plan finalisation.
+#include <algorithm>
+#include <cstring>
+#include <functional>
+#include <set>
+
+#include "ir.h"
+
+namespace dnnf {
+
+namespace {
+
+struct Bits {
+  std::vector<uint64_t> w;
+  explicit Bits(int n = 0) : w((n + 63) / 64, 0) {}
+  void set(int i) { w[i >> 6] |= 1ull << (i & 63); }
+  bool get(int i) const { return (w[i >> 6] >> (i & 63)) & 1; }
+  void or_with(const Bits& o) { for (size_t i = 0; i < w.size(); ++i) w[i] |= o.w[i]; }
+};
+
+struct Planner {
+  Graph& g;
+  uint32_t flags;
+  std::vector<int> order;            // topological
+  std::vector<int> pos;              // op id -> topological position
+  std::vector<Bits> anc, desc;       // strict ancestors / descendants per op
+  std::vector<int> block_of;         // op id -> block index or -1
+  std::vector<std::vector<int>> blocks;
+  std::vector<int> btype;
+  int yellow = 0, yellow_fused = 0;
+
+  Planner(Graph& gg, uint32_t f) : g(gg), flags(f) {}
+
+  std::vector<int> successors(int o) const {
+    std::vector<int> s;
+    for (int t : g.ops[o].out) for (int c : g.tensors[t].consumers) if (std::find(s.begin(), s.end(), c) == s.end()) s.push_back(c);
+    std::sort(s.begin(), s.end(), [&](int a, int b) { return pos[a] < pos[b]; });
+    return s;
+  }
+  std::vector<int> predecessors(int o) const {
+    std::vector<int> s;
+    for (int t : g.ops[o].in) { int p = g.tensors[t].producer; if (p >= 0 && g.ops[p].alive && std::find(s.begin(), s.end(), p) == s.end()) s.push_back(p); }
+    std::sort(s.begin(), s.end(), [&](int a, int b) { return pos[a] < pos[b]; });
+    return s;
+  }
+
+  void reachability() {
+    int n = (int)g.ops.size();
+    anc.assign(n, Bits(n)); desc.assign(n, Bits(n));
+    for (int o : order) for (int p : predecessors(o)) { anc[o].or_with(anc[p]); anc[o].set(p); }
+    for (auto it = order.rbegin(); it != order.rend(); ++it) for (int s : successors(*it)) { desc[*it].or_with(desc[s]); desc[*it].set(s); }
+  }
+
+  // A block must stay convex: no path between two members may leave the block,
+  // otherwise the fused kernel would have to run both before and after an
+  // outside operator.  (The paper does not spell this legality rule out.)
+  bool convex(const std::vector<int>& members) const {
+    int n = (int)g.ops.size();
+    Bits in(n), a(n), d(n);
+    for (int m : members) { in.set(m); a.or_with(anc[m]); d.or_with(desc[m]); }
+    for (size_t i = 0; i < a.w.size(); ++i) if (a.w[i] & d.w[i] & ~in.w[i]) return false;
+    return true;
+  }
+
+  // Mapping type of `op` as met along the edge from `from` (Section 3.1 defines
+  // types per input/output pair).  With STRICT_TABLE3 the node type is used.
+  int type_along(int op, int from_tensor) const {
+    const Op& o = g.ops[op];
+    if (flags & DNNF_PLAN_STRICT_TABLE3) return o.mapping;
+    int best = -1;
+    for (size_t s = 0; s < o.in.size(); ++s) if (o.in[s] == from_tensor) { int m = edge_mapping(g, o, (int)s); if (best < 0 || m < best) best = m; }
+    return best < 0 ? o.mapping : best;
+  }
+  // Type of a predecessor as seen from its output: the simplest pair it offers.
+  int type_as_pred(int op) const {
+    const Op& o = g.ops[op];
+    if (flags & DNNF_PLAN_STRICT_TABLE3) return o.mapping;
+    int best = o.mapping;
+    for (size_t s = 0; s < o.in.size(); ++s) best = std::min(best, edge_mapping(g, o, (int)s));
+    return best;
+  }
+  bool seed_eligible(int op) const {
+    const Op& o = g.ops[op];
+    if (o.mapping == DNNF_ONE_TO_ONE) return true;
+    if (flags & DNNF_PLAN_STRICT_TABLE3) return false;
+    return is_elementwise(o.kind) && type_as_pred(op) == DNNF_ONE_TO_ONE;
+  }
+  int64_t irs_size(int op) const { int64_t b = 0; for (int t : g.ops[op].out) b += g.tensors[t].bytes(); return b; }
+
+  bool lowers(const std::vector<int>& members, Block* out = nullptr) {
+    Block tmp; std::string why;
+    Block& b = out ? *out : tmp;
+    return lower_block(g, members, flags, b, why) == DNNF_OK;
+  }
+
+  // Step 2.2: the constraint check.  The paper's "empirically determined
+  // threshold" (register pressure etc.) becomes: the merged block must lower
+  // to one kernel within the register / argument / program-length budgets.
+  bool check_constraint(const std::vector<int>& merged) {
+    if (!convex(merged)) return false;
+    int anchors = 0;
+    for (int m : merged) if (g.ops[m].mapping == DNNF_MANY_TO_MANY) anchors++;
+    if (anchors > 1) return false;
+    if (flags & DNNF_PLAN_ALLOW_PROLOGUE) return true;
+    return lowers(merged);
+  }
+
+  // Step 2.3 for yellow cells.  The paper looks the combination up in a
+  // profiling database; this build uses an analytic stand-in: HBM bytes over
+  // bandwidth plus a launch cost per kernel.
+  bool profitable(const std::vector<int>& cur, int cand, const std::vector<int>& merged) {
+    yellow++;
+    if (flags & DNNF_PLAN_ALLOW_PROLOGUE) { yellow_fused++; return true; }
+    Block a, b, m;
+    if (!lowers(merged, &m)) return false;
+    if (!lowers(cur, &a) || !lowers({cand}, &b)) { yellow_fused++; return true; }
+    bool ok = block_cost_us(g, m) <= block_cost_us(g, a) + block_cost_us(g, b);
+    if (ok) yellow_fused++;
+    return ok;
+  }
+
+  bool try_add(int bi, int cand, int first_type, int second_type, bool cand_is_second) {
+    int fused, colour;
+    table3(first_type, second_type, &fused, &colour);
+    if (colour == DNNF_FUSE_BREAK) return false;
+    std::vector<int> merged = blocks[bi];
+    merged.push_back(cand);
+    if (!check_constraint(merged)) return false;
+    if (colour == DNNF_FUSE_DEPEND && !profitable(blocks[bi], cand, merged)) return false;
+    (void)cand_is_second;
+    blocks[bi] = merged;
+    block_of[cand] = bi;
+    btype[bi] = fused;
+    return true;
+  }
+
+  void fuse_successor(int op, int succ, int bi) {
+    if (block_of[succ] >= 0) return;
+    int via = -1;
+    for (int t : g.ops[op].out) if (std::find(g.ops[succ].in.begin(), g.ops[succ].in.end(), t) != g.ops[succ].in.end()) via = t;
+    if (!try_add(bi, succ, btype[bi], type_along(succ, via), true)) return;
+    for (int s : successors(succ)) fuse_successor(succ, s, bi);     // Step 2.4
+  }
+  void fuse_predecessor(int op, int pred, int bi) {
+    (void)op;
+    if (block_of[pred] >= 0) return;
+    if (!try_add(bi, pred, type_as_pred(pred), btype[bi], false)) return;
+    for (int p : predecessors(pred)) fuse_predecessor(pred, p, bi);
+  }
+
+  void run_listing1() {
+    for (;;) {
+      // Step 1: One-to-One operator with the smallest intermediate result; ties in graph order.
+      int seed = -1;
+      for (int o : order) {
+        if (block_of[o] >= 0 || !seed_eligible(o)) continue;
+        if (seed < 0 || irs_size(o) < irs_size(seed)) seed = o;
+      }
+      if (seed < 0) break;
+      int bi = (int)blocks.size();
+      blocks.push_back({seed});
+      btype.push_back(flags & DNNF_PLAN_STRICT_TABLE3 ? g.ops[seed].mapping : DNNF_ONE_TO_ONE);
+      block_of[seed] = bi;
+      for (int s : successors(seed)) fuse_successor(seed, s, bi);       // Step 2
+      for (int p : predecessors(seed)) fuse_predecessor(seed, p, bi);   // Step 3
+    }
+    for (int o : order) if (block_of[o] < 0) { block_of[o] = (int)blocks.size(); blocks.push_back({o}); btype.push_back(g.ops[o].mapping); }
+  }
+
+  // Intra-block optimisation of Section 4.4.2: a Reorganize/Shuffle operator with a
+  // single consumer is replaced by changed indexing.  Operators of these types are
+  // never seeds, so ones no seed reached are folded here into the block of their
+  // producer (as store indexing) or else of their consumer (as load indexing).
+  void absorb_index_ops() {
+    bool changed = true;
+    while (changed) {
+      changed = false;
+      for (int o : order) {
+        int bi = block_of[o];
+        if (blocks[bi].size() != 1 || !is_index_only(g.ops[o].kind)) continue;
+        std::vector<int> targets;
+        for (int p : predecessors(o)) targets.push_back(block_of[p]);
+        auto succ = successors(o);
+        if (succ.size() == 1) targets.push_back(block_of[succ[0]]);
+        for (int tb : targets) {
+          if (tb == bi) continue;
+          std::vector<int> merged = blocks[tb];
+          merged.push_back(o);
+          if (!convex(merged)) continue;
+          Block m, a, b;
+          if (!lowers(merged, &m)) continue;
+          if (lowers(blocks[tb], &a) && lowers({o}, &b) && block_cost_us(g, m) > block_cost_us(g, a) + block_cost_us(g, b)) continue;
+          blocks[tb] = merged; blocks[bi].clear(); block_of[o] = tb;
+          changed = true;
+          break;
+        }
+      }
+    }
+  }
+};
+
+}  // namespace
+
+// Analytic block cost: algorithmic bytes over HBM bandwidth (element-wise gathers
+// pay a sector per element), contraction flops over tensor/FMA peak, one launch.
+double block_cost_us(const Graph& g, const Block& b) {
+  const Launch& L = b.launch;
+  if (L.family == DNNF_FAMILY_ALIAS) return 0.0;
+  double bytes = 0;
+  auto add = [&](int tensor, int mode) {
+    const Tensor& T = g.tensors[tensor];
+    double e = (double)T.bytes();
+    if (mode == 2) e = (double)T.numel() * 32.0;
+    bytes += e;
+  };
+  if (L.family == DNNF_FAMILY_ELEMENTWISE || L.family == DNNF_FAMILY_TRANSPOSE) {
+    for (int i = 0; i < L.ew.n_in; ++i) add(L.in_tensors[i], L.ew.in[i].mode);
+    for (int i = 0; i < L.ew.n_out; ++i) add(L.out_tensors[i], L.ew.out[i].mode);
+  } else {
+    for (int t : b.inputs) add(t, 0);
+    for (int t : b.outputs) add(t, 0);
+  }
+  double t_mem = bytes / 6.5e6;                       // us at 6.5 TB/s
+  double t_cmp = (double)L.flops / 1.4e9;             // us at 1.4 PFLOP/s
+  return std::max(t_mem, t_cmp) + 2.0;
+}
+
+int plan_graph(Graph& g, uint32_t flags) {
+  g.relink();
+  g.blocks.clear(); g.run_order.clear();
+  g.planned = false;
+  for (auto& o : g.ops) { o.block = -1; if (o.alive) o.mapping = node_mapping(g, o); }
+  for (auto& t : g.tensors) { t.ws_offset = -1; t.alias_of = -1; t.removable = false; }
+
+  Planner P(g, flags);
+  P.order = g.topo_order();
+  P.pos.assign(g.ops.size(), -1);
+  for (size_t i = 0; i < P.order.size(); ++i) P.pos[P.order[i]] = (int)i;
+  P.block_of.assign(g.ops.size(), -1);
+  P.reachability();
+  if (flags & DNNF_PLAN_UNFUSED) {
+    for (int o : P.order) { P.block_of[o] = (int)P.blocks.size(); P.blocks.push_back({o}); P.btype.push_back(g.ops[o].mapping); }
+  } else {
+    P.run_listing1();
+    if (!(flags & DNNF_PLAN_ALLOW_PROLOGUE)) P.absorb_index_ops();
+  }
+
+  // Materialise blocks in an order that respects dependencies (first member's position
+  // is not enough after predecessor fusion: sort blocks topologically).
+  std::vector<std::vector<int>> live;
+  for (auto& b : P.blocks) if (!b.empty()) live.push_back(b);
+  int nb = (int)live.size();
+  std::vector<int> bo(g.ops.size(), -1);
+  for (int i = 0; i < nb; ++i) for (int o : live[i]) bo[o] = i;
+  std::vector<std::set<int>> deps(nb);
+  for (int i = 0; i < nb; ++i)
+    for (int o : live[i]) for (int t : g.ops[o].in) { int p = g.tensors[t].producer; if (p >= 0 && g.ops[p].alive && bo[p] != i) deps[i].insert(bo[p]); }
+  std::vector<int> first_pos(nb, 1 << 30);
+  for (int i = 0; i < nb; ++i) for (int o : live[i]) first_pos[i] = std::min(first_pos[i], P.pos[o]);
+  std::vector<int> done(nb, 0), border;
+  for (int round = 0; round < nb; ++round) {
+    int pick = -1;
+    for (int i = 0; i < nb; ++i) {
+      if (done[i]) continue;
+      bool ready = true;
+      for (int d : deps[i]) if (!done[d]) ready = false;
+      if (ready && (pick < 0 || first_pos[i] < first_pos[pick])) pick = i;
+    }
+    if (pick < 0) { g.err = "internal: cyclic block dependencies"; return DNNF_ERR_STATE; }
+    done[pick] = 1; border.push_back(pick);
+  }
+
+  bool runnable = true;
+  for (int bi : border) {
+    Block b; std::string why;
+    int rc = lower_block(g, live[bi], flags, b, why);
+    if (rc != DNNF_OK) {
+      if (flags & DNNF_PLAN_ALLOW_PROLOGUE) { b.ops = live[bi]; b.lowered = false; runnable = false; }
+      else {
+        g.err = "cannot lower block starting at " + std::string(op_name(g.ops[live[bi][0]].kind)) + ": " + why;
+        return DNNF_ERR_UNSUPPORTED_OP;
+      }
+    }
+    b.mapping = P.btype[P.block_of[live[bi][0]]];
+    int idx = (int)g.blocks.size();
+    for (int o : b.ops) g.ops[o].block = idx;
+    g.blocks.push_back(std::move(b));
+    g.run_order.push_back(idx);
+  }
+
+  // IR_removable (Section 3.2): an intermediate disappears iff every consumer sits in
+  // its producer's block.  What remains is materialised in the workspace.
+  int64_t irs_unfused = 0, irs_fused = 0;
+  for (auto& t : g.tensors) {
+    if (t.external || t.producer < 0 || !g.ops[t.producer].alive) continue;
+    bool outside = false;
+    for (int c : t.consumers) if (g.ops[c].block != g.ops[t.producer].block) outside = true;
+    t.removable = !outside && !t.is_output;
+    if (!t.is_output) { irs_unfused += t.bytes(); if (!t.removable) irs_fused += t.bytes(); }
+  }
+  // zero-copy aliases
+  for (auto& b : g.blocks) if (b.lowered && b.launch.family == DNNF_FAMILY_ALIAS) {
+    g.tensors[b.launch.out_tensors[0]].alias_of = b.launch.in_tensors[0];
+    irs_fused -= g.tensors[b.launch.out_tensors[0]].bytes();
+  }
+  // Workspace: first-fit over live ranges in block order.
+  struct Range { int64_t off, size; int last_use; };
+  std::vector<Range> active;
+  int64_t ws = 256;                       // status words live in the first 256 bytes
+  auto root = [&](int t) { while (g.tensors[t].alias_of >= 0) t = g.tensors[t].alias_of; return t; };
+  std::vector<int> last_use(g.tensors.size(), -1);
+  for (size_t bi = 0; bi < g.blocks.size(); ++bi) for (int t : g.blocks[bi].inputs) last_use[root(t)] = (int)bi;
+  for (size_t bi = 0; bi < g.blocks.size(); ++bi) {
+    Block& b = g.blocks[bi];
+    if (!b.lowered || b.launch.family == DNNF_FAMILY_ALIAS) continue;
+    for (int t : b.outputs) {
+      Tensor& T = g.tensors[t];
+      if (T.is_output) continue;          // bound by the caller
+      int64_t size = (T.bytes() + 255) / 256 * 256;
+      // free ranges whose last use is before this block
+      std::vector<Range> keep;
+      for (auto& r : active) if (r.last_use >= (int)bi) keep.push_back(r);
+      active.swap(keep);
+      std::sort(active.begin(), active.end(), [](const Range& a, const Range& c) { return a.off < c.off; });
+      int64_t off = 256;
+      for (auto& r : active) { if (off + size <= r.off) break; off = std::max(off, r.off + r.size); }
+      active.push_back({off, size, std::max(last_use[t], (int)bi)});
+      T.ws_offset = off;
+      ws = std::max(ws, off + size);
+    }
+  }
+  g.ws_bytes = (size_t)ws;
+  g.plan_flags = flags;
+  g.planned = runnable;
+
+  dnnf_plan_stats& s = g.pstats;
+  std::memset(&s, 0, sizeof s);
+  std::set<int> src;
+  for (auto& o : g.ops) if (o.alive) src.insert(o.source_id);
+  s.n_ops = (int)src.size();
+  s.n_blocks = (int)g.blocks.size();
+  for (auto& b : g.blocks) if (!b.lowered || b.launch.family != DNNF_FAMILY_ALIAS) s.n_kernels++;
+  s.fusion_rate = s.n_blocks ? (double)s.n_ops / s.n_blocks : 0.0;
+  s.irs_bytes_unfused = irs_unfused;
+  s.irs_bytes_fused = irs_fused;
+  s.workspace_bytes = ws;
+  s.n_yellow_decisions = P.yellow;
+  s.n_yellow_fused = P.yellow_fused;
+  return DNNF_OK;
+}
+
+}  // namespace dnnf
