@@ -1,0 +1,291 @@
+#!/usr/bin/env python
+"""Benchmark of the fused-block executor on one B200 ("Measurement").
+
+Default arm: `python bench.py --gpus N --steps K --warmup W` prints ONE JSON line.
+A step is one pass of the hot path -- dnnf_run of the fused scale+mask+softmax
+block and of the fused add+LayerNorm+GELU block (fp32, the attention-score /
+norm configuration) -- over a batch of R independent instances that live in
+distinct buffers larger than L2.  `value` is algorithmic GB/s over the whole
+step, inputs already in HBM; `e2e` is the same through host buffers.
+
+`--impl reference` times the CPU oracle on the same workload (bounded sample).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "fused-block GB/s (algorithmic bytes / time) on the attention-score and norm blocks; % of HBM peak in roofline"
+UNIT = "GB/s"
+R_INSTANCES = 24
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"], "bf16_tflops_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    def __init__(self, index=0):
+        self.samples = []
+        self.reasons = set()
+        self.stop = threading.Event()
+        self.index = index
+        self.th = None
+
+    def _run(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        while not self.stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-i", str(self.index)],
+                                     capture_output=True, text=True, timeout=5).stdout.strip().split(",")
+                self.samples.append((float(out[0]), float(out[1])))
+                for n, v in zip(names, out[2:]):
+                    if v.strip().lower().startswith("active"):
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            self.stop.wait(0.1)
+
+    def __enter__(self):
+        self.th = threading.Thread(target=self._run, daemon=True)
+        self.th.start()
+        return self
+
+    def __exit__(self, *a):
+        self.stop.set()
+        self.th.join(timeout=6)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": sorted(self.reasons)}
+        sm = sorted(s[0] for s in self.samples)
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(s[1] for s in self.samples), "reasons": sorted(self.reasons),
+                "samples": len(sm)}
+
+
+def block_bytes(sess):
+    tot = 0
+    for b in range(sess.g.block_count()):
+        d = sess.g.block_info(b)
+        tot += d.bytes_in + d.bytes_out
+    return tot
+
+
+# --------------------------------------------------------------------------------------
+def run_reference(args):
+    """CPU oracle arm: the unfused fp64 interpreter on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import interp as O
+    from paper_2108_13342_b200 import workloads as W
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = 1
+    wa, wb = W.masked_softmax(), W.add_layernorm_gelu()
+    bytes_step = 12648448 + 9443328
+    for _ in range(max(1, min(args.warmup, 1))):
+        O.run_graph(wa.graph, wa.inputs); O.run_graph(wb.graph, wb.inputs)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        O.run_graph(wa.graph, wa.inputs); O.run_graph(wb.graph, wb.inputs)
+    dt = (time.perf_counter() - t0) / args.steps
+    val = bytes_step / dt / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "configs[1]: scale+mask+softmax [8,12,128,128] + add+LayerNorm+GELU [1024,768]; "
+                                   "one instance per step (bounded sample of the 24-instance GPU step)"},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": "1 of 24 instances per step, numpy fp64 unfused interpreter"},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="dnnf")
+    ap.add_argument("--no-detail", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2108_13342_b200 import binding as B
+    from paper_2108_13342_b200 import workloads as W
+    from paper_2108_13342_b200.runtime import Session
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    pk = peaks()
+    steps, warm = args.steps, max(args.warmup, 3)
+
+    # ---- the step: R instances of each block, distinct buffers (footprint > L2) ------------------
+    wa, wb = W.masked_softmax(seed=W.BASE_SEED + 100 * rank), W.add_layernorm_gelu(seed=W.BASE_SEED + 100 * rank)
+    A = [Session(wa, rewrite_flags=B.REWRITE_NONE, device=dev) for _ in range(R_INSTANCES)]
+    Bn = [Session(wb, rewrite_flags=B.REWRITE_NONE, device=dev) for _ in range(R_INSTANCES)]
+    bytes_a, bytes_b = block_bytes(A[0]), block_bytes(Bn[0])
+    bytes_step = R_INSTANCES * (bytes_a + bytes_b)
+    stream = torch.cuda.current_stream(dev)
+    sptr = stream.cuda_stream
+
+    def part_a():
+        for s in A:
+            s.g.run(sptr)
+
+    def part_b():
+        for s in Bn:
+            s.g.run(sptr)
+
+    for _ in range(warm):
+        part_a(); part_b()
+    torch.cuda.synchronize(dev)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize(dev)
+    with ClockSampler(local) as clk:
+        for i in range(steps):
+            ev[i][0].record(stream); part_a(); ev[i][1].record(stream); part_b(); ev[i][2].record(stream)
+        torch.cuda.synchronize(dev)
+        t_total = ev[0][0].elapsed_time(ev[-1][2])                      # ms, whole timed region
+        # keep the GPU busy a little longer so the sampler sees clocks under load
+        t_end = time.time() + 1.0
+        while time.time() < t_end:
+            part_a(); part_b()
+        torch.cuda.synchronize(dev)
+    if world > 1:
+        dist.barrier()
+    t_a = sum(e[0].elapsed_time(e[1]) for e in ev) / steps             # ms per step in part a
+    t_b = sum(e[1].elapsed_time(e[2]) for e in ev) / steps
+    ms_step = t_total / steps
+    if world > 1:
+        t = torch.tensor([ms_step], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t.item())
+    value = world * bytes_step / (ms_step * 1e-3) / 1e9
+
+    # ---- roofline of the dominant kernel (the softmax row kernel) ---------------------------------
+    dur_a = t_a * 1e-3 / R_INSTANCES
+    ach = bytes_a / dur_a / 1e9
+    roof = {"bound": "hbm", "kernel": "row_kernel<4,1,1> (scale+mask+softmax)", "achieved": ach, "peak": pk["hbm_gbs"],
+            "unit": "GB/s", "frac": ach / pk["hbm_gbs"], "peak_source": pk["source"], "traffic": None,
+            "bytes_per_launch": bytes_a, "us_per_launch": dur_a * 1e6,
+            "second_kernel": {"kernel": "row_kernel<4,6,1> (add+LayerNorm+GELU)", "bytes_per_launch": bytes_b,
+                              "us_per_launch": t_b * 1e3 / R_INSTANCES, "achieved": bytes_b / (t_b * 1e-3 / R_INSTANCES) / 1e9,
+                              "frac": bytes_b / (t_b * 1e-3 / R_INSTANCES) / 1e9 / pk["hbm_gbs"]}}
+    tp = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tp):
+        with open(tp) as f:
+            roof["traffic"] = json.load(f).get("masked_softmax_bytes_per_launch")
+
+    # ---- end to end: host buffers in, host result out, through the same C-ABI calls -----------------
+    hin_a = [torch.from_numpy(wa.inputs["S"]).pin_memory() for _ in range(2)]
+    hin_b = [(torch.from_numpy(wb.inputs["H"]).pin_memory(), torch.from_numpy(wb.inputs["R"]).pin_memory()) for _ in range(2)]
+    hout_a = torch.empty_like(hin_a[0]).pin_memory()
+    hout_b = torch.empty_like(hin_b[0][0]).pin_memory()
+    h2d = R_INSTANCES * (hin_a[0].numel() + 2 * hin_b[0][0].numel()) * 4
+    d2h = R_INSTANCES * (hout_a.numel() + hout_b.numel()) * 4
+
+    def e2e_step():
+        for i, s in enumerate(A):
+            s.buffers["S"].copy_(hin_a[i & 1], non_blocking=True)
+            s.g.run(sptr)
+            hout_a.copy_(s.buffers["P"], non_blocking=True)
+        for i, s in enumerate(Bn):
+            s.buffers["H"].copy_(hin_b[i & 1][0], non_blocking=True)
+            s.buffers["R"].copy_(hin_b[i & 1][1], non_blocking=True)
+            s.g.run(sptr)
+            hout_b.copy_(s.buffers["Y"], non_blocking=True)
+
+    e2e_steps = max(3, min(steps, 10))
+    for _ in range(2):
+        e2e_step()
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e = {"value": world * bytes_step / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": f"configs[1]: fused scale+mask+softmax [8,12,128,128] and fused add+LayerNorm+GELU "
+                                   f"[1024,768], fp32; {R_INSTANCES} independent instances of each per step",
+                       "l2": f"inputs larger than L2: {bytes_step / 1e6:.0f} MB of distinct buffers per step",
+                       "bytes_per_step": bytes_step, "launches_per_step": 2 * R_INSTANCES},
+            "clocks": clk.summary(), "e2e": e2e, "gpu_launches": steps * 2 * R_INSTANCES, "roofline": roof}
+
+    if rank == 0 and not args.no_cpu:
+        line["cpu_baseline"] = cpu_baseline(wa, wb, bytes_a + bytes_b)
+    if rank == 0 and not args.no_detail:
+        from paper_2108_13342_b200 import report
+        line["detail"] = report.per_config(dev, pk)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(wa, wb, bytes_instance):
+    from oracle import interp as O
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = 1
+    O.run_graph(wa.graph, wa.inputs); O.run_graph(wb.graph, wb.inputs)
+    n, t0 = 0, time.perf_counter()
+    while time.perf_counter() - t0 < 10.0 or n < 2:
+        O.run_graph(wa.graph, wa.inputs); O.run_graph(wb.graph, wb.inputs)
+        n += 1
+    dt = (time.perf_counter() - t0) / n
+    return {"value": bytes_instance / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n} passes over 1 of the {R_INSTANCES} instances (about {dt * n:.0f} s of CPU work)",
+            "ms_per_instance": dt * 1e3}
+
+
+if __name__ == "__main__":
+    main()

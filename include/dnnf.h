@@ -216,6 +216,10 @@ DNNF_API const char* dnnf_rule_name(int rule_index);
 DNNF_API int dnnf_plan(dnnf_graph* g, uint32_t flags, dnnf_plan_stats* host_stats);
 DNNF_API int dnnf_block_count(const dnnf_graph* g, int* n_blocks);
 DNNF_API int dnnf_block_info(const dnnf_graph* g, int block, dnnf_block_desc* host_out);
+/* Writes the block's micro-op program as text ("MOV in0; ADD in1; MUL c0=0.5; ...")
+ * into host_buf (capacity bytes, NUL-terminated, truncated if needed): the linearised
+ * data-flow tree of Section 4.4, every value computed once. */
+DNNF_API int dnnf_block_program(const dnnf_graph* g, int block, char* host_buf, size_t capacity);
 /* Block index that holds operator `op_index` (insertion order), after dnnf_plan. */
 DNNF_API int dnnf_op_block(const dnnf_graph* g, int op_index, int* block);
 /* Number of operators currently alive (after rewriting) and their kinds. */

@@ -67,7 +67,7 @@ class BlockDesc(C.Structure):
 
 EXPORTS = ["dnnf_graph_create", "dnnf_graph_destroy", "dnnf_add_tensor", "dnnf_add_op", "dnnf_mark_output",
            "dnnf_tensor_info", "dnnf_op_mapping", "dnnf_mapping_check", "dnnf_rewrite", "dnnf_rule_name", "dnnf_plan",
-           "dnnf_block_count", "dnnf_block_info", "dnnf_op_block", "dnnf_op_count", "dnnf_op_kind",
+           "dnnf_block_count", "dnnf_block_info", "dnnf_block_program", "dnnf_op_block", "dnnf_op_count", "dnnf_op_kind",
            "dnnf_workspace_size", "dnnf_bind", "dnnf_bind_workspace", "dnnf_run", "dnnf_run_block", "dnnf_status",
            "dnnf_launch_count", "dnnf_last_error", "dnnf_version"]
 
@@ -95,6 +95,7 @@ def _load():
     lib.dnnf_plan.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(PlanStats)]
     lib.dnnf_block_count.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
     lib.dnnf_block_info.argtypes = [C.c_void_p, C.c_int, C.POINTER(BlockDesc)]
+    lib.dnnf_block_program.argtypes = [C.c_void_p, C.c_int, C.c_char_p, C.c_size_t]
     lib.dnnf_op_block.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int)]
     lib.dnnf_op_count.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
     lib.dnnf_op_kind.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
@@ -204,6 +205,11 @@ class Graph:
         d = BlockDesc()
         self._check(lib.dnnf_block_info(self.h, b, C.byref(d)))
         return d
+
+    def block_program(self, b):
+        buf = C.create_string_buffer(4096)
+        self._check(lib.dnnf_block_program(self.h, b, buf, 4096))
+        return buf.value.decode()
 
     def op_block(self, op_index):
         b = C.c_int()

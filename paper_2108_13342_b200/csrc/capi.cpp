@@ -1,5 +1,6 @@
 // C ABI: argument checking, state machine, error messages.  No exception leaves
 // this file.
+#include <cstdio>
 #include <cstring>
 #include <exception>
 
@@ -205,10 +206,35 @@ int dnnf_block_info(const dnnf_graph* g, int bi, dnnf_block_desc* out) {
   for (int t : b.inputs) out->bytes_in += G.tensors[t].bytes();
   for (int t : b.outputs) out->bytes_out += G.tensors[t].bytes();
   out->flops = b.launch.flops;
-  out->n_microops = b.launch.family == DNNF_FAMILY_ROW ? b.launch.row.prog.n : b.launch.ew.prog.n;
+  { const Program* pr = program_of(b.launch); out->n_microops = pr ? pr->n : 0; }
   out->grid = b.launch.grid;
   out->threads = b.launch.threads;
   out->variant = b.launch.variant;
+  return DNNF_OK;
+}
+
+int dnnf_block_program(const dnnf_graph* g, int bi, char* buf, size_t cap) {
+  if (!g || !buf || cap == 0 || bi < 0 || bi >= (int)g->g.blocks.size()) return DNNF_ERR_INVALID_ARG;
+  static const char* on[] = {"END", "MOV", "SAVE", "STORE", "ADD", "SUB", "RSUB", "MUL", "DIV", "RDIV", "MAX", "MIN", "NEG", "ABS",
+    "RECIP", "SQUARE", "SQRT", "EXP", "LOG", "TANH", "ERF", "SIGMOID", "RELU", "GELU_ERF", "GELU_TANH", "CLIP", "POW",
+    "ROWSUM", "ROWMEAN", "ROWMAX", "ROWPROD"};
+  const Block& b = g->g.blocks[bi];
+  const Program* pr = program_of(b.launch);
+  std::string s;
+  if (pr) for (int i = 0; i < pr->n; ++i) {
+    const MicroOp& m = pr->ops[i];
+    if (i) s += "; ";
+    s += on[m.op < M__COUNT ? m.op : 0];
+    char t[48] = "";
+    if (m.op == M_SAVE) snprintf(t, sizeof t, " t%d", m.idx);
+    else if (m.op == M_STORE) snprintf(t, sizeof t, " out%d", m.idx);
+    else if (m.src == S_IN) snprintf(t, sizeof t, " in%d", m.idx);
+    else if (m.src == S_TMP) snprintf(t, sizeof t, " t%d", m.idx);
+    else if (m.src == S_CONST) snprintf(t, sizeof t, " c%d=%g", m.idx, pr->consts[m.idx]);
+    else if (m.src == S_ANCHOR) snprintf(t, sizeof t, " anchor");
+    s += t;
+  }
+  snprintf(buf, cap, "%s", s.c_str());
   return DNNF_OK;
 }
 

@@ -10,13 +10,9 @@
 #include <math_constants.h>
 
 #include "microop.h"
+#include "static_programs.h"
 
 namespace dnnf {
-
-struct FastDiv {
-  uint32_t m, s, d;
-  __device__ __forceinline__ uint32_t div(uint32_t n) const { return d == 1 ? n : (__umulhi(n, m) >> s); }
-};
 
 __device__ __forceinline__ float op_sigmoid(float x) { return __fdividef(1.0f, 1.0f + __expf(-x)); }
 __device__ __forceinline__ float op_gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
@@ -134,72 +130,75 @@ __device__ __forceinline__ void apply_op(int op, float (&acc)[VV], const float (
 //   void anchor(float (&dst)[VV]);               contraction result (S_ANCHOR)
 //   void store(int out_idx, const float (&v)[VV]);
 //   void row_reduce(int op, float (&acc)[VV]);   M_ROW* (row kernels only)
-template <int VV, int NT, class IO>
-__device__ __forceinline__ void run_program(const Program& prog, IO& io) {
-  // Saved values sit in separately named arrays selected by a switch, so that they
-  // stay in registers (an array indexed by the slot number would go to local memory).
-  float acc[VV], t0[VV], t1[VV], t2[VV], t3[VV];
+//
+// Saved values sit in separately named arrays selected by a switch, so that they stay
+// in registers (an array indexed by the slot number would go to local memory).
+template <int VV>
+struct ChainState {
+  float acc[VV], t0[VV], t1[VV];
+};
+
+template <int VV, class IO>
+__device__ __forceinline__ void exec_one(const MicroOp m, ChainState<VV>& st, IO& io, const Program& prog) {
+  if (m.op == M_SAVE) {
+    if (m.idx == 0) {
 #pragma unroll
-  for (int v = 0; v < VV; ++v) { acc[v] = 0.0f; t0[v] = 0.0f; t1[v] = 0.0f; t2[v] = 0.0f; t3[v] = 0.0f; }
-  const int n = prog.n;
-#pragma unroll 1
-  for (int pc = 0; pc < n; ++pc) {
-    const MicroOp m = prog.ops[pc];
-    if (m.op == M_SAVE) {
-      switch (m.idx) {
-        case 0:
-#pragma unroll
-          for (int v = 0; v < VV; ++v) t0[v] = acc[v];
-          break;
-        case 1:
-          if (NT > 1) {
-#pragma unroll
-            for (int v = 0; v < VV; ++v) t1[v] = acc[v];
-          }
-          break;
-        case 2:
-          if (NT > 2) {
-#pragma unroll
-            for (int v = 0; v < VV; ++v) t2[v] = acc[v];
-          }
-          break;
-        default:
-          if (NT > 3) {
-#pragma unroll
-            for (int v = 0; v < VV; ++v) t3[v] = acc[v];
-          }
-          break;
-      }
-      continue;
-    }
-    if (m.op == M_STORE) { io.store(m.idx, acc); continue; }
-    if (m.op >= M_ROWSUM) { io.row_reduce(m.op, acc); continue; }
-    float c0 = 0.0f, c1 = 0.0f;
-    if (m.src == S_IN) {
-      float src[VV];
-      io.load(m.idx, src);
-      apply_op<VV>(m.op, acc, src, c0, c1);
-    } else if (m.src == S_TMP) {
-      switch (m.idx) {
-        case 0: apply_op<VV>(m.op, acc, t0, c0, c1); break;
-        case 1: if (NT > 1) apply_op<VV>(m.op, acc, t1, c0, c1); break;
-        case 2: if (NT > 2) apply_op<VV>(m.op, acc, t2, c0, c1); break;
-        default: if (NT > 3) apply_op<VV>(m.op, acc, t3, c0, c1); break;
-      }
-    } else if (m.src == S_ANCHOR) {
-      float src[VV];
-      io.anchor(src);
-      apply_op<VV>(m.op, acc, src, c0, c1);
+      for (int v = 0; v < VV; ++v) st.t0[v] = st.acc[v];
     } else {
-      float src[VV];
-      if (m.src == S_CONST) {
-        c0 = prog.consts[m.idx];
-        c1 = prog.consts[m.idx + 1 < kMaxConst ? m.idx + 1 : m.idx];
-      }
 #pragma unroll
-      for (int v = 0; v < VV; ++v) src[v] = c0;
-      apply_op<VV>(m.op, acc, src, c0, c1);
+      for (int v = 0; v < VV; ++v) st.t1[v] = st.acc[v];
     }
+    return;
+  }
+  if (m.op == M_STORE) { io.store(m.idx, st.acc); return; }
+  if (m.op >= M_ROWSUM) { io.row_reduce(m.op, st.acc); return; }
+  float c0 = 0.0f, c1 = 0.0f;
+  if (m.src == S_IN) {
+    float src[VV];
+    io.load(m.idx, src);
+    apply_op<VV>(m.op, st.acc, src, c0, c1);
+  } else if (m.src == S_TMP) {
+    if (m.idx == 0) apply_op<VV>(m.op, st.acc, st.t0, c0, c1);
+    else apply_op<VV>(m.op, st.acc, st.t1, c0, c1);
+  } else if (m.src == S_ANCHOR) {
+    float src[VV];
+    io.anchor(src);
+    apply_op<VV>(m.op, st.acc, src, c0, c1);
+  } else {
+    float src[VV];
+    if (m.src == S_CONST) {
+      c0 = prog.consts[m.idx];
+      c1 = prog.consts[m.idx + 1 < kMaxConst ? m.idx + 1 : m.idx];
+    }
+#pragma unroll
+    for (int v = 0; v < VV; ++v) src[v] = c0;
+    apply_op<VV>(m.op, st.acc, src, c0, c1);
+  }
+}
+
+template <class SP, int I, int VV, class IO>
+__device__ __forceinline__ void static_step(ChainState<VV>& st, IO& io, const Program& prog) {
+  constexpr MicroOp m = SP::op(I);
+  exec_one<VV>(m, st, io, prog);
+}
+template <class SP, int VV, class IO, int... I>
+__device__ __forceinline__ void run_static(ChainState<VV>& st, IO& io, const Program& prog, std::integer_sequence<int, I...>) {
+  (static_step<SP, I, VV>(st, io, prog), ...);
+}
+
+// SP = DynProg: interpret prog at run time.  Otherwise SP is a compile-time table with
+// the same opcodes as prog (the host checked), and the whole chain is straight-line code.
+template <int VV, class SP, class IO>
+__device__ __forceinline__ void run_program(const Program& prog, IO& io) {
+  ChainState<VV> st;
+#pragma unroll
+  for (int v = 0; v < VV; ++v) { st.acc[v] = 0.0f; st.t0[v] = 0.0f; st.t1[v] = 0.0f; }
+  if constexpr (SP::n == 0) {
+    const int n = prog.n;
+#pragma unroll 1
+    for (int pc = 0; pc < n; ++pc) exec_one<VV>(prog.ops[pc], st, io, prog);
+  } else {
+    run_static<SP, VV>(st, io, prog, std::make_integer_sequence<int, SP::n>{});
   }
 }
 

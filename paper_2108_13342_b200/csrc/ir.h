@@ -59,6 +59,7 @@ struct ConvLaunch;
 struct Launch {
   int family = DNNF_FAMILY_ALIAS;
   int variant = 0;
+  int static_id = 0;          // compile-time program table the block runs on (0: interpreted)
   int grid = 0, threads = 0;
   size_t smem = 0;
   EwParams ew{};
@@ -119,6 +120,8 @@ int plan_graph(Graph& g, uint32_t flags);
 // `why` explains a refusal (used as the constraint check of Listing 1, Step 2.2).
 int lower_block(const Graph& g, const std::vector<int>& ops, uint32_t flags, Block& out, std::string& why);
 double block_cost_us(const Graph& g, const Block& b);
+
+const Program* program_of(const Launch& L);     // the block's micro-op program, wherever the family keeps it
 
 // ---- launch (kernels_*.cu) ----
 int launch_block(Graph& g, Block& b, void* stream, std::string& err);

@@ -224,7 +224,8 @@ static bool derive_once(LowerCtx& cx, int ref, const std::set<int>& stop_ops) {
     int t = q.front(); q.pop_front();
     const Tensor& T = g.tensors[t];
     int p = T.producer;
-    if (p >= 0 && cx.in_block.count(p) && !stop_ops.count(p)) {
+    const bool p_is_reduce = p >= 0 && g.ops[p].kind >= DNNF_OP_REDUCESUM && g.ops[p].kind <= DNNF_OP_REDUCEPROD;
+    if (p >= 0 && cx.in_block.count(p) && !stop_ops.count(p) && !p_is_reduce) {   // a reduction's input is the reference
       std::vector<View> vin;
       if (!backward_views(cx, g.ops[p], cx.views[t], vin)) return false;
       for (size_t s = 0; s < vin.size(); ++s) {
@@ -279,7 +280,7 @@ struct Emitter {
   int max_tmp;
   std::map<Val, int> uses;          // remaining arithmetic uses
   std::map<Val, int> tmp_of;        // value -> tmp slot
-  bool tmp_busy[kMaxTmp] = {false, false, false, false};
+  bool tmp_busy[kMaxTmp] = {false, false};
   Val acc{-1, -1};
   bool acc_valid = false;
   std::map<int, Val> root_of;       // in-block tensor -> value
@@ -527,7 +528,7 @@ bool emit_program(LowerCtx& cx, int anchor_out, int max_tmp) {
         E.load_acc(v[0]); E.protect_operand_in_acc(v[0], 1);
         int t = E.alloc_tmp(); if (E.fail) break;
         E.push(M_SAVE, S_TMP, (uint8_t)t); E.push(M_ROWMAX); E.push(M_RSUB, S_TMP, (uint8_t)t); E.push(M_EXP);
-        E.push(M_SAVE, S_TMP, (uint8_t)t); E.push(M_ROWSUM); E.push(M_RDIV, S_TMP, (uint8_t)t);
+        E.push(M_SAVE, S_TMP, (uint8_t)t); E.push(M_ROWSUM); E.push(M_RECIP); E.push(M_MUL, S_TMP, (uint8_t)t);
         E.tmp_busy[t] = false;
         E.consume(v[0]);
         break;
@@ -538,7 +539,7 @@ bool emit_program(LowerCtx& cx, int anchor_out, int max_tmp) {
         // two-pass statistics on the register-resident row: mean, then mean of squared deviations
         E.push(M_SAVE, S_TMP, (uint8_t)t); E.push(M_ROWMEAN); E.push(M_RSUB, S_TMP, (uint8_t)t);
         E.push(M_SAVE, S_TMP, (uint8_t)t); E.push(M_SQUARE); E.push(M_ROWMEAN);
-        E.push(M_ADD, S_CONST, (uint8_t)E.cst((float)op.at.eps)); E.push(M_SQRT); E.push(M_RDIV, S_TMP, (uint8_t)t);
+        E.push(M_ADD, S_CONST, (uint8_t)E.cst((float)op.at.eps)); E.push(M_SQRT); E.push(M_RECIP); E.push(M_MUL, S_TMP, (uint8_t)t);
         E.tmp_busy[t] = false;
         uint8_t s, i;
         if (!E.src_of(v[1], s, i)) break; E.push(M_MUL, s, i);
@@ -748,6 +749,12 @@ static int lower_elementwise_or_row(const Graph& g, const std::vector<int>& ops,
   finalize_ew(L_);
   out.lowered = true;
   return DNNF_OK;
+}
+
+const Program* program_of(const Launch& L) {
+  if (L.family == DNNF_FAMILY_ALIAS) return nullptr;
+  if (L.family == DNNF_FAMILY_ROW) return &L.row.prog;
+  return &L.ew.prog;     // contraction families keep their epilogue program here too
 }
 
 int lower_block(const Graph& g, const std::vector<int>& ops_in, uint32_t flags, Block& out, std::string& why) {

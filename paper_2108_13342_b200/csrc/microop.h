@@ -18,7 +18,7 @@ constexpr int kMaxIn = 8;        // external inputs of a block
 constexpr int kMaxOut = 4;       // external outputs of a block
 constexpr int kMaxOps = 40;      // micro-ops per program
 constexpr int kMaxConst = 12;
-constexpr int kMaxTmp = 4;
+constexpr int kMaxTmp = 2;      // saved values live in registers: two per element
 
 enum MOp : uint8_t {
   M_END = 0,

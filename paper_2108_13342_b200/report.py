@@ -1,0 +1,107 @@
+"""Per-configuration measurements printed beside the headline benchmark number:
+each fused block's time, GB/s (or TFLOP/s) and roofline fraction; the same graph
+unfused, one kernel per operator; plain launches and CUDA-graph replay."""
+from __future__ import annotations
+
+import numpy as np
+
+from . import binding as B
+from . import workloads as W
+from .runtime import Session
+
+L2_BYTES = 126 * 1024 * 1024
+
+
+def _time_region(torch, dev, fn, iters):
+    st = torch.cuda.current_stream(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    e0.record(st)
+    for _ in range(iters):
+        fn()
+    e1.record(st)
+    torch.cuda.synchronize(dev)
+    return e0.elapsed_time(e1) * 1e3 / iters          # us per call
+
+
+def _graph_of(torch, dev, fn):
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream(dev)
+    s.wait_stream(torch.cuda.current_stream(dev))
+    with torch.cuda.stream(s):
+        fn_s = lambda: fn(s.cuda_stream)
+        fn_s()                                         # warm-up on the side stream
+        torch.cuda.synchronize(dev)
+        with torch.cuda.graph(g, stream=s):
+            fn_s()
+    torch.cuda.current_stream(dev).wait_stream(s)
+    return g
+
+
+def measure_workload(torch, dev, wl, pk, flags, copies, iters=20, rewrite=B.REWRITE_NONE):
+    """`copies` sessions with distinct buffers, run round-robin so that every launch
+    sees cold data when copies * footprint exceeds L2."""
+    sess = [Session(wl, plan_flags=flags, rewrite_flags=rewrite, device=dev) for _ in range(copies)]
+    s0 = sess[0]
+    nb = s0.g.block_count()
+    blocks = s0.g.blocks()
+
+    def all_plain():
+        sp = torch.cuda.current_stream(dev).cuda_stream
+        for s in sess:
+            s.g.run(sp)
+
+    def all_on(sp):
+        for s in sess:
+            s.g.run(sp)
+
+    for _ in range(3):
+        all_plain()
+    t_plain = _time_region(torch, dev, all_plain, iters) / copies
+    cg = _graph_of(torch, dev, all_on)
+    t_graph = _time_region(torch, dev, cg.replay, iters) / copies
+    per_block = []
+    if nb <= 16:
+        for b in range(nb):
+            if blocks[b]["family"] == "alias":
+                continue
+
+            def one(sp, b=b):
+                for s in sess:
+                    s.g.run_block(b, sp)
+
+            cgb = _graph_of(torch, dev, one)
+            cgb.replay()
+            t = _time_region(torch, dev, cgb.replay, iters) / copies
+            by, fl = blocks[b]["bytes"], blocks[b]["flops"]
+            roof_us = max(by / (pk["hbm_gbs"] * 1e3), fl / (pk["bf16_tflops"] * 1e6))
+            per_block.append({"ops": "+".join(blocks[b]["ops"][:8]), "family": blocks[b]["family"], "us": round(t, 3),
+                              "bytes": by, "GBps": round(by / t / 1e3, 1), "flops": fl,
+                              "TFLOPs": round(fl / t / 1e6, 1) if fl else 0, "roofline_us": round(roof_us, 3),
+                              "frac_of_roofline": round(roof_us / t, 3)})
+    return {"kernels": s0.plan_stats.n_kernels, "ops": s0.plan_stats.n_ops, "fusion_rate": round(s0.plan_stats.fusion_rate, 2),
+            "us_plain_launches": round(t_plain, 3), "us_cuda_graph": round(t_graph, 3), "copies": copies,
+            "irs_bytes": int(s0.plan_stats.irs_bytes_fused), "blocks": per_block}
+
+
+def per_config(dev, pk):
+    import torch
+    out = {}
+    cases = [
+        ("cfg1 swish+transpose [1,64,56,56]", W.swish_transpose(), 96),
+        ("cfg1 batch-512 variant", W.swish_transpose(n=512), 1),
+        ("cfg2a scale+mask+softmax [8,12,128,128]", W.masked_softmax(), 24),
+        ("cfg2a batch-512 variant", W.masked_softmax(batch=512), 1),
+        ("cfg2b add+LayerNorm+GELU [1024,768]", W.add_layernorm_gelu(), 24),
+        ("cfg2b 131072-row variant", W.add_layernorm_gelu(rows=131072), 1),
+    ]
+    for name, wl, copies in cases:
+        try:
+            fused = measure_workload(torch, dev, wl, pk, B.PLAN_FUSED, copies)
+            unfused = measure_workload(torch, dev, wl, pk, B.PLAN_UNFUSED, copies)
+            out[name] = {"fused": fused, "unfused": unfused,
+                         "speedup_fused_vs_unfused_graph": round(unfused["us_cuda_graph"] / fused["us_cuda_graph"], 2)}
+        except Exception as e:      # report, never hide
+            out[name] = {"error": repr(e)}
+        torch.cuda.empty_cache()
+    return out

@@ -151,7 +151,7 @@ def test_long_chain_with_shared_subexpressions_and_two_outputs():
     o = g.add("Add", [t3, t5], out="Out")
     g.mark_output(o); g.mark_output(t1)
     s = check(W.Workload(g, ins), RTOL_F32, expect_blocks=1)
-    assert s.g.blocks()[0]["n_microops"] <= 10
+    assert s.g.blocks()[0]["n_microops"] <= 11      # 5 arithmetic ops, 2 stores, 2 saves, 2 moves
 
 
 def test_chain_of_24_ops():
