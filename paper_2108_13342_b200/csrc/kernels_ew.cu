@@ -14,21 +14,20 @@ __device__ __forceinline__ uint32_t fdiv(const IterSpace& it, int d, uint32_t n)
 // Contiguous chain.  Each thread owns U vectors of V elements, U*256*V elements
 // per CTA, consecutive lanes on consecutive vectors.
 // ---------------------------------------------------------------------------
-template <int V, int U>
+template <int V, int U, bool F32>
 struct EwIO {
   const EwParams& p;
   uint32_t coord[U][kMaxDims];
   bool valid[U];
-  __device__ __forceinline__ int64_t offset(const TensorArg& a, int u) const {
-    int64_t off = a.base;
+  __device__ __forceinline__ uint32_t offset(const TensorArg& a, int u) const {
+    uint32_t off = (uint32_t)a.base;
 #pragma unroll
-    for (int d = 0; d < kMaxDims; ++d)
-      if (d < p.it.ndim) off += (int64_t)coord[u][d] * a.stride[d];
+    for (int d = 0; d < kMaxDims; ++d) off += coord[u][d] * (uint32_t)a.stride[d];   // unused dims: coord 0
     return off;
   }
   __device__ __forceinline__ void load(int idx, float (&dst)[V * U]) const {
     const TensorArg& a = p.in[idx];
-    const int64_t si = a.stride[0];
+    const int si = a.stride[0];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       if (!valid[u]) {
@@ -36,16 +35,16 @@ struct EwIO {
         for (int v = 0; v < V; ++v) dst[u * V + v] = 0.0f;
         continue;
       }
-      int64_t off = offset(a, u);
+      uint32_t off = offset(a, u);
       if (V == 4 && si == 1 && a.mode == 0) {
-        load_vec4(a, off, &dst[u * V]);
+        load_vec4<F32>(a, off, &dst[u * V]);
       } else if (si == 0) {
-        float x = load_scalar(a, off);
+        float x = load_scalar<F32>(a, off);
 #pragma unroll
         for (int v = 0; v < V; ++v) dst[u * V + v] = x;
       } else {
 #pragma unroll
-        for (int v = 0; v < V; ++v) dst[u * V + v] = load_scalar(a, off + v * si);
+        for (int v = 0; v < V; ++v) dst[u * V + v] = load_scalar<F32>(a, off + v * si);
       }
     }
   }
@@ -55,16 +54,16 @@ struct EwIO {
   }
   __device__ __forceinline__ void store(int idx, const float (&val)[V * U]) const {
     const TensorArg& a = p.out[idx];
-    const int64_t si = a.stride[0];
+    const int si = a.stride[0];
     const bool exact = p.prog.flags & kProgPureMove;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       if (!valid[u]) continue;
-      int64_t off = offset(a, u);
-      if (V == 4 && si == 1 && a.mode == 0) store_vec4(a, off, &val[u * V], exact);
+      uint32_t off = offset(a, u);
+      if (V == 4 && si == 1 && a.mode == 0) store_vec4<F32>(a, off, &val[u * V], exact);
       else {
 #pragma unroll
-        for (int v = 0; v < V; ++v) store_scalar(a, off + v * si, val[u * V + v], exact);
+        for (int v = 0; v < V; ++v) store_scalar<F32>(a, off + v * si, val[u * V + v], exact);
       }
     }
   }
@@ -73,9 +72,9 @@ struct EwIO {
 
 // NOTE: on the device the iteration dims are stored INNERMOST FIRST (dim 0 is the
 // contiguous one), so that every index below is a compile-time constant.
-template <int V, int U, class SP>
+template <int V, int U, class SP, bool F32>
 __global__ void __launch_bounds__(256) ew_kernel(const __grid_constant__ EwParams p) {
-  EwIO<V, U> io{p};
+  EwIO<V, U, F32> io{p};
   const uint32_t nvec = (uint32_t)(p.total / V);
 #pragma unroll
   for (int u = 0; u < U; ++u) {
@@ -110,25 +109,23 @@ __global__ void __launch_bounds__(256) ew_kernel(const __grid_constant__ EwParam
 // ---------------------------------------------------------------------------
 constexpr int TT = 64, TI = 64, TPITCH = TI + 1;
 
-template <int V, int K>      // K vectors per thread
+template <int V, int K, bool F32>      // K vectors per thread
 struct TrIO {
   const EwParams& p;
   const float* smem;       // [n_staged][TT][TPITCH]
-  int64_t outer_dummy;
   uint32_t outer[kMaxDims];
   uint32_t t0, i0;         // tile origin
   uint32_t tt[K], ti;      // this thread's elements within the tile
   bool valid[K];
-  __device__ __forceinline__ int64_t offset(const TensorArg& a, int k) const {
-    int64_t off = a.base + (int64_t)(t0 + tt[k]) * a.stride[1] + (int64_t)(i0 + ti) * a.stride[0];
+  __device__ __forceinline__ uint32_t offset(const TensorArg& a, int k) const {
+    uint32_t off = (uint32_t)a.base + (t0 + tt[k]) * (uint32_t)a.stride[1] + (i0 + ti) * (uint32_t)a.stride[0];
 #pragma unroll
-    for (int d = 2; d < kMaxDims; ++d)
-      if (d < p.it.ndim) off += (int64_t)outer[d] * a.stride[d];
+    for (int d = 2; d < kMaxDims; ++d) off += outer[d] * (uint32_t)a.stride[d];
     return off;
   }
   __device__ __forceinline__ void load(int idx, float (&dst)[V * K]) const {
     const TensorArg& a = p.in[idx];
-    const int64_t si = a.stride[0];
+    const int si = a.stride[0];
 #pragma unroll
     for (int k = 0; k < K; ++k) {
       if (!valid[k]) {
@@ -142,15 +139,15 @@ struct TrIO {
         for (int v = 0; v < V; ++v) dst[k * V + v] = s[v];
         continue;
       }
-      int64_t off = offset(a, k);
-      if (V == 4 && si == 1 && a.mode == 0) load_vec4(a, off, &dst[k * V]);
+      uint32_t off = offset(a, k);
+      if (V == 4 && si == 1 && a.mode == 0) load_vec4<F32>(a, off, &dst[k * V]);
       else if (si == 0) {
-        float x = load_scalar(a, off);
+        float x = load_scalar<F32>(a, off);
 #pragma unroll
         for (int v = 0; v < V; ++v) dst[k * V + v] = x;
       } else {
 #pragma unroll
-        for (int v = 0; v < V; ++v) dst[k * V + v] = load_scalar(a, off + v * si);
+        for (int v = 0; v < V; ++v) dst[k * V + v] = load_scalar<F32>(a, off + v * si);
       }
     }
   }
@@ -160,27 +157,27 @@ struct TrIO {
   }
   __device__ __forceinline__ void store(int idx, const float (&val)[V * K]) const {
     const TensorArg& a = p.out[idx];
-    const int64_t si = a.stride[0];
+    const int si = a.stride[0];
     const bool exact = p.prog.flags & kProgPureMove;
 #pragma unroll
     for (int k = 0; k < K; ++k) {
       if (!valid[k]) continue;
-      int64_t off = offset(a, k);
-      if (V == 4 && si == 1 && a.mode == 0) store_vec4(a, off, &val[k * V], exact);
+      uint32_t off = offset(a, k);
+      if (V == 4 && si == 1 && a.mode == 0) store_vec4<F32>(a, off, &val[k * V], exact);
       else {
 #pragma unroll
-        for (int v = 0; v < V; ++v) store_scalar(a, off + v * si, val[k * V + v], exact);
+        for (int v = 0; v < V; ++v) store_scalar<F32>(a, off + v * si, val[k * V + v], exact);
       }
     }
   }
   __device__ __forceinline__ void row_reduce(int, float (&)[V * K]) const {}
 };
 
-template <int V, class SP>
+template <int V, class SP, bool F32>
 __global__ void __launch_bounds__(256) tr_kernel(const __grid_constant__ EwParams p) {
   extern __shared__ float smem[];
   constexpr int K = 4;
-  TrIO<V, K> io{p, smem};
+  TrIO<V, K, F32> io{p, smem};
   uint32_t b = blockIdx.x;
   uint32_t tile_i = b % (uint32_t)p.tiles_i; b /= (uint32_t)p.tiles_i;
   uint32_t tile_t = b % (uint32_t)p.tiles_t; b /= (uint32_t)p.tiles_t;
@@ -201,10 +198,9 @@ __global__ void __launch_bounds__(256) tr_kernel(const __grid_constant__ EwParam
     const TensorArg& a = p.in[k];
     if (!(a.mode & 1)) continue;
     float* s = smem + ((a.mode >> 1) & 1) * TT * TPITCH;
-    int64_t base = a.base + (int64_t)io.t0 * a.stride[1] + (int64_t)io.i0 * a.stride[0];
+    uint32_t base = (uint32_t)a.base + io.t0 * (uint32_t)a.stride[1] + io.i0 * (uint32_t)a.stride[0];
 #pragma unroll
-    for (int d = 2; d < kMaxDims; ++d)
-      if (d < p.it.ndim) base += (int64_t)io.outer[d] * a.stride[d];
+    for (int d = 2; d < kMaxDims; ++d) base += io.outer[d] * (uint32_t)a.stride[d];
     const bool full = io.t0 + TT <= ext_t && io.i0 + TI <= ext_i;
     if (V == 4 && a.mode >= 5 && full) {          // 128-bit loads along t (host verified alignment)
 #pragma unroll
@@ -212,7 +208,7 @@ __global__ void __launch_bounds__(256) tr_kernel(const __grid_constant__ EwParam
         int idx = threadIdx.x + 256 * r;
         int t4 = (idx % (TT / 4)) * 4, ti = idx / (TT / 4);
         float x[4];
-        load_vec4(a, base + t4 + (int64_t)ti * a.stride[0], x);
+        load_vec4<F32>(a, base + t4 + ti * (uint32_t)a.stride[0], x);
 #pragma unroll
         for (int j = 0; j < 4; ++j) s[(t4 + j) * TPITCH + ti] = x[j];
       }
@@ -224,7 +220,7 @@ __global__ void __launch_bounds__(256) tr_kernel(const __grid_constant__ EwParam
         for (int h = 0; h < TT / 32; ++h) {
           int tt = lane + 32 * h;
           float x = 0.0f;
-          if (iok && io.t0 + tt < ext_t) x = load_scalar(a, base + (int64_t)tt * a.stride[1] + (int64_t)ti * a.stride[0]);
+          if (iok && io.t0 + tt < ext_t) x = load_scalar<F32>(a, base + tt * (uint32_t)a.stride[1] + ti * (uint32_t)a.stride[0]);
           s[tt * TPITCH + ti] = x;
         }
       }
@@ -255,22 +251,34 @@ __global__ void __launch_bounds__(256) tr_kernel(const __grid_constant__ EwParam
 }
 
 // ---------------------------------------------------------------------------
+template <bool F32>
 struct EwLauncher {
   const Launch& L; cudaStream_t st;
   template <class SP> void run() {
-    if (L.family == DNNF_FAMILY_ELEMENTWISE) ew_kernel<4, 2, SP><<<L.grid, 256, 0, st>>>(L.ew);
-    else tr_kernel<4, SP><<<L.grid, 256, L.smem, st>>>(L.ew);
+    if (L.family == DNNF_FAMILY_ELEMENTWISE) ew_kernel<4, 2, SP, F32><<<L.grid, 256, 0, st>>>(L.ew);
+    else tr_kernel<4, SP, F32><<<L.grid, 256, L.smem, st>>>(L.ew);
   }
 };
 
+static bool all_f32(const EwParams& p) {
+  for (int i = 0; i < p.n_in; ++i) if (p.in[i].dtype != 0) return false;
+  for (int i = 0; i < p.n_out; ++i) if (p.out[i].dtype != 0) return false;
+  return true;
+}
+
 int launch_ew(const Launch& L, cudaStream_t st) {
   const EwParams& p = L.ew;
-  EwLauncher F{L, st};
   if (p.vec == 4) {
-    if (!(L.static_id > 0 && StaticSet<EwStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
+    if (all_f32(p)) {
+      EwLauncher<true> F{L, st};
+      if (!(L.static_id > 0 && StaticSet<EwStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
+    } else {
+      EwLauncher<false> F{L, st};
+      if (!(L.static_id > 0 && StaticSet<EwStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
+    }
   } else {
-    if (L.family == DNNF_FAMILY_ELEMENTWISE) ew_kernel<1, 4, DynProg><<<L.grid, 256, 0, st>>>(p);
-    else tr_kernel<1, DynProg><<<L.grid, 256, L.smem, st>>>(p);
+    if (L.family == DNNF_FAMILY_ELEMENTWISE) ew_kernel<1, 4, DynProg, false><<<L.grid, 256, 0, st>>>(p);
+    else tr_kernel<1, DynProg, false><<<L.grid, 256, L.smem, st>>>(p);
   }
   return cudaGetLastError() == cudaSuccess ? 0 : 1;
 }

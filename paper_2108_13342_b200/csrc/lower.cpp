@@ -601,8 +601,9 @@ void collapse(Packed& p) {
 
 bool fill_arg(TensorArg& a, const Graph& g, const ExtArg& e, const std::vector<int64_t>& coef) {
   a.ptr = nullptr;
-  a.base = e.view.c0;
-  for (int d = 0; d < kMaxDims; ++d) a.stride[d] = d < (int)coef.size() ? coef[d] : 0;
+  if (g.tensors[e.tensor].numel() >= (1ll << 31)) return false;
+  a.base = (int32_t)e.view.c0;
+  for (int d = 0; d < kMaxDims; ++d) a.stride[d] = d < (int)coef.size() ? (int32_t)coef[d] : 0;
   a.dtype = g.tensors[e.tensor].dtype;
   a.mode = 0;
   return true;
@@ -681,8 +682,10 @@ static int lower_elementwise_or_row(const Graph& g, const std::vector<int>& ops,
     rp.it.ndim = nd;
     for (int d = 0; d < nd; ++d) rp.it.extent[d] = (uint32_t)p.ext[d];
     rp.n_in = n_in; rp.n_out = n_out;
-    for (int i = 0; i < n_in; ++i) fill_arg(rp.in[i], g, cx.ins[i], p.coefs[i]);
-    for (int i = 0; i < n_out; ++i) fill_arg(rp.out[i], g, cx.outs[i], p.coefs[n_in + i]);
+    bool fits = true;
+    for (int i = 0; i < n_in; ++i) fits &= fill_arg(rp.in[i], g, cx.ins[i], p.coefs[i]);
+    for (int i = 0; i < n_out; ++i) fits &= fill_arg(rp.out[i], g, cx.outs[i], p.coefs[n_in + i]);
+    if (!fits) { why = "tensor with 2^31 or more elements"; return DNNF_ERR_UNSUPPORTED_OP; }
     rp.prog = cx.prog;
     rp.L = (int)L; rp.rows = total / L;
     int inner = nd - 1;
@@ -707,8 +710,10 @@ static int lower_elementwise_or_row(const Graph& g, const std::vector<int>& ops,
   ep.it.ndim = nd;
   for (int d = 0; d < nd; ++d) ep.it.extent[d] = (uint32_t)p.ext[d];
   ep.n_in = n_in; ep.n_out = n_out;
-  for (int i = 0; i < n_in; ++i) fill_arg(ep.in[i], g, cx.ins[i], p.coefs[i]);
-  for (int i = 0; i < n_out; ++i) fill_arg(ep.out[i], g, cx.outs[i], p.coefs[n_in + i]);
+  bool fits = true;
+  for (int i = 0; i < n_in; ++i) fits &= fill_arg(ep.in[i], g, cx.ins[i], p.coefs[i]);
+  for (int i = 0; i < n_out; ++i) fits &= fill_arg(ep.out[i], g, cx.outs[i], p.coefs[n_in + i]);
+  if (!fits) { why = "tensor with 2^31 or more elements"; return DNNF_ERR_UNSUPPORTED_OP; }
   ep.prog = cx.prog;
   ep.total = total;
   int inner = nd - 1;

@@ -50,10 +50,12 @@ constexpr int kProgPureMove = 1;
 
 // One external tensor as seen from the block's iteration space: element offset
 //   off = base + sum_d idx[d] * stride[d]
+// (element counts below 2^31 per tensor are checked at lowering time, so 32-bit
+// offsets are enough on the device.)
 struct TensorArg {
   void* ptr;
-  int64_t base;
-  int64_t stride[kMaxDims];
+  int32_t base;
+  int32_t stride[kMaxDims];
   int32_t dtype;       // 0 f32, 1 bf16
   int32_t mode;        // 0 direct; 2 element-wise gather; 1 / 3 staged through shared-memory slot 0 / 1
 };
