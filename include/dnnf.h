@@ -240,6 +240,28 @@ DNNF_API int dnnf_bind_workspace(dnnf_graph* g, void* dev_ptr, size_t bytes);
 DNNF_API int dnnf_run(dnnf_graph* g, void* cuda_stream);
 /* Launches only block `block` (for per-block timing). */
 DNNF_API int dnnf_run_block(dnnf_graph* g, int block, void* cuda_stream);
+/* No counterpart in the paper: a convenience for callers that cannot allocate.
+ * Same as dnnf_run(), but the intermediates that stay materialised between blocks
+ * live in a fixed array inside the library instead of a caller-provided workspace,
+ * so nothing has to be allocated or bound (a workspace bound earlier is ignored for
+ * this call and left bound).  Meant for code running where cudaMalloc is off limits:
+ * inside a memory pool's out-of-memory handler, in a plugin whose host forbids
+ * allocation after initialisation, or between the capture-begin and capture-end of
+ * somebody else's stream.
+ *  - The array is DNNF_STATIC_WS_BYTES long and is reserved on every GPU that loads
+ *    the library, until the process exits.  A plan that needs more returns
+ *    DNNF_ERR_WORKSPACE and launches nothing.
+ *  - The first call on each device looks the array's address up (with that device
+ *    current); make that first call outside any stream capture.
+ *  - All graphs and all calls share the one array.  It keeps whatever the previous call
+ *    left; the status words at its start are cleared on `cuda_stream` before the
+ *    kernels run.  Two calls whose kernels can overlap on the GPU (different streams,
+ *    no ordering between them) race on it.
+ *  - Inputs and outputs are still the caller's bound tensors.  The call allocates
+ *    nothing on host-visible CUDA paths: no cudaMalloc, cudaFree or library routine
+ *    that allocates. */
+#define DNNF_STATIC_WS_BYTES (32u << 20)
+DNNF_API int dnnf_run_static_ws(dnnf_graph* g, void* cuda_stream);
 /* After the caller synchronised the stream: device-side status word
  * (0 = ok, DNNF_ERR_TIMEOUT if a bounded wait inside a kernel ran out) and the
  * block that reported it. */

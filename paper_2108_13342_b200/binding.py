@@ -40,6 +40,7 @@ _FLOAT_ATTRS = {"c", "lo", "hi", "p", "eps"}
 
 REWRITE_DEFAULT, REWRITE_NONE, REWRITE_CANON_MACRO = 0, 1, 2
 PLAN_FUSED, PLAN_UNFUSED, PLAN_STRICT_TABLE3, PLAN_ALLOW_PROLOGUE = 0, 1, 2, 4
+STATIC_WS_BYTES = 32 << 20
 
 
 class Attr(C.Structure):
@@ -68,7 +69,7 @@ class BlockDesc(C.Structure):
 EXPORTS = ["dnnf_graph_create", "dnnf_graph_destroy", "dnnf_add_tensor", "dnnf_add_op", "dnnf_mark_output",
            "dnnf_tensor_info", "dnnf_op_mapping", "dnnf_mapping_check", "dnnf_rewrite", "dnnf_rule_name", "dnnf_plan",
            "dnnf_block_count", "dnnf_block_info", "dnnf_block_program", "dnnf_op_block", "dnnf_op_count", "dnnf_op_kind",
-           "dnnf_workspace_size", "dnnf_bind", "dnnf_bind_workspace", "dnnf_run", "dnnf_run_block", "dnnf_status",
+           "dnnf_workspace_size", "dnnf_bind", "dnnf_bind_workspace", "dnnf_run", "dnnf_run_static_ws", "dnnf_run_block", "dnnf_status",
            "dnnf_launch_count", "dnnf_last_error", "dnnf_version"]
 
 
@@ -103,6 +104,7 @@ def _load():
     lib.dnnf_bind.argtypes = [C.c_void_p, C.c_int, C.c_void_p]
     lib.dnnf_bind_workspace.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
     lib.dnnf_run.argtypes = [C.c_void_p, C.c_void_p]
+    lib.dnnf_run_static_ws.argtypes = [C.c_void_p, C.c_void_p]
     lib.dnnf_run_block.argtypes = [C.c_void_p, C.c_int, C.c_void_p]
     lib.dnnf_status.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     lib.dnnf_launch_count.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
@@ -239,6 +241,10 @@ class Graph:
 
     def run(self, stream=0):
         self._check(lib.dnnf_run(self.h, C.c_void_p(stream)))
+
+    def run_static_ws(self, stream=0):
+        """dnnf_run with the between-block intermediates in the library's built-in array (no workspace needed)."""
+        self._check(lib.dnnf_run_static_ws(self.h, C.c_void_p(stream)))
 
     def run_block(self, b, stream=0):
         self._check(lib.dnnf_run_block(self.h, b, C.c_void_p(stream)))
