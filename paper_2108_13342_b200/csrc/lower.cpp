@@ -197,8 +197,19 @@ static int forward_view_i(LowerCtx& cx, const Op& op, int slot, const View& vi, 
   if (k == DNNF_OP_SOFTMAX) { vo = vi; return 1; }
   if (k == DNNF_OP_LAYERNORM || k == DNNF_OP_SCALESHIFT) { if (slot != 0) return 0; vo = vi; return 1; }
   if (is_elementwise(k)) {
-    if (in.dims != out.dims) return 0;
-    vo = vi; return 1;
+    if (in.dims == out.dims) { vo = vi; return 1; }
+    // Coming from a broadcast operand (e.g. a per-row statistic): the result covers the whole
+    // iteration space.  Accept the identity map if walking it back reproduces this operand's view.
+    int64_t tot = 1, no = 1;
+    for (auto e : cx.ext) tot *= e;
+    for (auto e : out.dims) no *= e;
+    if (tot != no) return 0;
+    View cand; cand.coef = contiguous_strides(cx.ext);
+    std::vector<View> vin;
+    SplitRequest keep = cx.split;
+    if (!backward_views(cx, op, cand, vin)) { if (cx.split.dim >= 0) return -1; cx.split = keep; cx.why.clear(); return 0; }
+    if (!(vin[slot] == vi)) return 0;
+    vo = cand; return 1;
   }
   cx.why = std::string("no index map through ") + op_name(k);
   return -1;

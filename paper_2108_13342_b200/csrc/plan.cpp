@@ -1,9 +1,12 @@
 // Fusion-plan generation (Section 4.3, Listing 1) and plan finalisation.
 #include <algorithm>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <functional>
 #include <set>
 
+#include "gemm_params.h"
 #include "ir.h"
 
 namespace dnnf {
@@ -28,6 +31,7 @@ struct Planner {
   std::vector<std::vector<int>> blocks;
   std::vector<int> btype;
   int yellow = 0, yellow_fused = 0;
+  bool debug = getenv("DNNF_DEBUG_PLAN") != nullptr;
 
   Planner(Graph& gg, uint32_t f) : g(gg), flags(f) {}
 
@@ -90,7 +94,13 @@ struct Planner {
   bool lowers(const std::vector<int>& members, Block* out = nullptr) {
     Block tmp; std::string why;
     Block& b = out ? *out : tmp;
-    return lower_block(g, members, flags, b, why) == DNNF_OK;
+    bool ok = lower_block(g, members, flags, b, why) == DNNF_OK;
+    if (!ok && debug) {
+      fprintf(stderr, "[dnnf plan] cannot lower {");
+      for (int m : members) fprintf(stderr, " %s#%d", op_name(g.ops[m].kind), m);
+      fprintf(stderr, " }: %s\n", why.c_str());
+    }
+    return ok;
   }
 
   // Step 2.2: the constraint check.  The paper's "empirically determined
@@ -197,6 +207,74 @@ struct Planner {
       }
     }
   }
+
+  double cost_of(const std::vector<int>& members) {
+    if (members.empty()) return 0.0;
+    Block b;
+    if (!lowers(members, &b)) return 1e30;
+    return block_cost_us(g, b);
+  }
+
+  // Second half of the same intra-block optimisation: an index-only operator at the END of
+  // a block whose result is read only by one other block moves into that block, where it
+  // becomes the consumer's load indexing (for a GEMM: the operand's strides).
+  void migrate_index_tails() {
+    bool changed = true;
+    int guard = 0;
+    while (changed && guard++ < 10000) {
+      changed = false;
+      for (auto it = order.rbegin(); it != order.rend() && !changed; ++it) {
+        int o = *it;
+        if (!is_index_only(g.ops[o].kind)) continue;
+        int x = block_of[o];
+        int y = -1; bool ok = true;
+        for (int t : g.ops[o].out) {
+          if (g.tensors[t].is_output) ok = false;
+          for (int c : g.tensors[t].consumers) { if (block_of[c] == x) ok = false; else if (y < 0) y = block_of[c]; else if (y != block_of[c]) ok = false; }
+        }
+        if (!ok || y < 0) continue;
+        std::vector<int> xs, ys = blocks[y];
+        for (int m : blocks[x]) if (m != o) xs.push_back(m);
+        ys.push_back(o);
+        if (!convex(ys) || (!xs.empty() && !convex(xs))) continue;
+        double before = cost_of(blocks[x]) + cost_of(blocks[y]);
+        double after = cost_of(xs) + cost_of(ys);
+        if (after >= 1e30 || after > before) continue;
+        blocks[x] = xs; blocks[y] = ys; block_of[o] = y;
+        changed = true;
+      }
+    }
+  }
+
+  // Listing 1 applied once more with whole blocks as the operators: a producer block and a
+  // consumer block merge when Table 3 allows the pair of block types, the union stays convex,
+  // passes the constraint check and is not slower by the cost model.
+  void merge_blocks() {
+    bool changed = true;
+    int guard = 0;
+    while (changed && guard++ < 10000) {
+      changed = false;
+      for (int o : order) {
+        int x = block_of[o];
+        for (int s : successors(o)) {
+          int y = block_of[s];
+          if (y == x) continue;
+          int fused, colour;
+          table3(btype[x], btype[y], &fused, &colour);
+          if (colour == DNNF_FUSE_BREAK) continue;
+          std::vector<int> merged = blocks[x];
+          merged.insert(merged.end(), blocks[y].begin(), blocks[y].end());
+          if (!check_constraint(merged)) continue;
+          if (cost_of(merged) > cost_of(blocks[x]) + cost_of(blocks[y])) continue;
+          for (int m : blocks[y]) block_of[m] = x;
+          blocks[x] = merged; blocks[y].clear(); btype[x] = fused;
+          changed = true;
+          break;
+        }
+        if (changed) break;
+      }
+    }
+  }
 };
 
 }  // namespace
@@ -216,6 +294,14 @@ double block_cost_us(const Graph& g, const Block& b) {
   if (L.family == DNNF_FAMILY_ELEMENTWISE || L.family == DNNF_FAMILY_TRANSPOSE) {
     for (int i = 0; i < L.ew.n_in; ++i) add(L.in_tensors[i], L.ew.in[i].mode);
     for (int i = 0; i < L.ew.n_out; ++i) add(L.out_tensors[i], L.ew.out[i].mode);
+  } else if (L.family == DNNF_FAMILY_GEMM || L.family == DNNF_FAMILY_CONV1X1) {
+    // operands: what the contraction reads (a strided view may cover part of a larger tensor)
+    const GemmParams& gp = *reinterpret_cast<const GemmParams*>(L.blob.data());
+    double nb = (double)gp.batch_ext[0] * gp.batch_ext[1];
+    bytes += nb * gp.M * gp.K * (gp.A.dtype ? 2 : 4) * ((gp.A.batch_stride[0] || gp.A.batch_stride[1] || nb == 1) ? 1.0 : 1.0 / nb);
+    bytes += nb * gp.K * gp.N * (gp.B.dtype ? 2 : 4) * ((gp.B.batch_stride[0] || gp.B.batch_stride[1] || nb == 1) ? 1.0 : 1.0 / nb);
+    for (size_t i = 2; i < L.in_tensors.size(); ++i) add(L.in_tensors[i], 0);
+    for (int t : L.out_tensors) add(t, 0);
   } else {
     for (int t : b.inputs) add(t, 0);
     for (int t : b.outputs) add(t, 0);
@@ -242,7 +328,7 @@ int plan_graph(Graph& g, uint32_t flags) {
     for (int o : P.order) { P.block_of[o] = (int)P.blocks.size(); P.blocks.push_back({o}); P.btype.push_back(g.ops[o].mapping); }
   } else {
     P.run_listing1();
-    if (!(flags & DNNF_PLAN_ALLOW_PROLOGUE)) P.absorb_index_ops();
+    if (!(flags & DNNF_PLAN_ALLOW_PROLOGUE)) { P.absorb_index_ops(); P.migrate_index_tails(); P.merge_blocks(); }
   }
 
   // Materialise blocks in an order that respects dependencies (first member's position

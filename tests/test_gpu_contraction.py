@@ -1,0 +1,99 @@
+"""Parity of contraction-anchored blocks (GEMM / pointwise convolution with fused
+epilogues, strided operands, permuted stores) with the oracle."""
+import numpy as np
+import pytest
+
+from paper_2108_13342_b200 import binding as B
+from paper_2108_13342_b200 import workloads as W
+from util import RTOL_BF16, RTOL_F32, check, close, graph, rnd, run_both
+
+pytestmark = pytest.mark.gpu
+FUSED, UNFUSED = B.PLAN_FUSED, B.PLAN_UNFUSED
+
+
+def _bf(x):
+    return W.round_to_bf16(x)
+
+
+@pytest.mark.parametrize("mnk", [(128, 128, 64), (256, 256, 256), (1, 17, 8), (129, 257, 72), (17, 129, 264), (300, 40, 1024),
+                                 (512, 768, 768)])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_plain_matmul(mnk, dtype):
+    m, n, k = mnk
+    a, b = rnd((m, k), 1, -1, 1), rnd((k, n), 2, -1, 1)
+    if dtype == "bf16":
+        a, b = _bf(a), _bf(b)
+    g = graph()
+    g.ext("A", (m, k), dtype); g.ext("B", (k, n), dtype)
+    g.mark_output(g.add("MatMul", ["A", "B"], out="C"))
+    check(W.Workload(g, {"A": a, "B": b}), RTOL_BF16 if dtype == "bf16" else 1e-4)
+
+
+@pytest.mark.parametrize("cfg", [(256, 64, 128), (129, 72, 136), (512, 768, 3072)])
+@pytest.mark.parametrize("flags", [FUSED, UNFUSED])
+def test_ffn_block(cfg, flags):
+    m, hidden, ffn = cfg
+    s = check(W.ffn_block(m, hidden, ffn), RTOL_BF16, flags, expect_blocks=2 if flags == FUSED else 6)
+    if flags == FUSED:
+        assert [b["family"] for b in s.g.blocks()] == ["gemm", "gemm"]
+
+
+def test_batched_matmul_with_transposed_and_strided_operands():
+    # scores = (Q K^T) * scale + mask with Q, K sliced out of one [B,S,3*H*D] tensor -- all index
+    # operators fold into operand strides; P V is stored straight into [B,S,H*D]
+    bsz, s, h, d = 2, 32, 3, 16
+    qkv = _bf(rnd((bsz, s, 3 * h * d), 5, -1, 1))
+    g = graph()
+    g.ext("QKV", qkv.shape, "bf16"); g.ext("mask", (s, s), "f32")
+    q, k, v = g.add("Split", ["QKV"], n_out=3, axis=-1, sizes=(h * d,) * 3)
+    hs = []
+    for t in (q, k, v):
+        t = g.add("Reshape", [t], shape=(bsz, s, h, d))
+        hs.append(g.add("Transpose", [t], perm=(0, 2, 1, 3)))
+    q, k, v = hs
+    kt = g.add("Transpose", [k], perm=(0, 1, 3, 2))
+    sc = g.add("MatMul", [q, kt])
+    sc = g.add("MulC", [sc], c=0.25)
+    sc = g.add("Add", [sc, "mask"])
+    p = g.add("Softmax", [sc], axis=-1)
+    a = g.add("MatMul", [p, v])
+    a = g.add("Transpose", [a], perm=(0, 2, 1, 3))
+    a = g.add("Reshape", [a], shape=(bsz, s, h * d), out="O")
+    g.mark_output(a)
+    wl = W.Workload(g, {"QKV": qkv, "mask": W.causal_mask(s)})
+    sess = check(wl, RTOL_BF16, FUSED, expect_blocks=3)
+    assert [b["family"] for b in sess.g.blocks()] == ["gemm", "row", "gemm"]
+    check(wl, RTOL_BF16, UNFUSED)
+
+
+def test_matmul_broadcast_weight_over_batch_and_f32_epilogue_operands():
+    x = _bf(rnd((3, 40, 64), 7, -1, 1)); w = _bf(rnd((64, 48), 8, -0.2, 0.2))
+    g = graph()
+    g.ext("X", x.shape, "bf16"); g.ext("Wt", w.shape, "bf16", kind="weight"); g.ext("b", (48,), "f32"); g.ext("R", (3, 40, 48), "bf16")
+    t = g.add("MatMul", ["X", "Wt"])
+    t = g.add("Add", [t, "b"])
+    t = g.add("Relu", [t])
+    g.mark_output(g.add("Add", [t, "R"], out="Y"))
+    check(W.Workload(g, {"X": x, "Wt": w, "b": rnd((48,), 9), "R": _bf(rnd((3, 40, 48), 10))}), RTOL_BF16, FUSED, expect_blocks=1)
+
+
+@pytest.mark.parametrize("cfg", [(1, 5, 6, 24, 144), (2, 7, 3, 144, 24), (1, 4, 4, 3, 5)])
+def test_conv1x1_with_epilogue(cfg):
+    n, h, w, ci, co = cfg
+    g = graph()
+    g.ext("X", (n, h, w, ci)); g.ext("Wc", (ci, co)); g.ext("s", (co,)); g.ext("t", (co,))
+    e = g.add("Conv1x1", ["X", "Wc"])
+    e = g.add("ScaleShift", [e, "s", "t"], axis=-1)
+    g.mark_output(g.add("Clip", [e], lo=0.0, hi=6.0, out="Y"))
+    ins = {"X": rnd((n, h, w, ci), 11, 0, 1), "Wc": rnd((ci, co), 12, -0.5, 0.5), "s": rnd((co,), 13, 0.5, 1.5), "t": rnd((co,), 14, -0.5, 0.5)}
+    check(W.Workload(g, ins), RTOL_F32, FUSED, expect_blocks=1)
+
+
+@pytest.mark.parametrize("flags,rewrite", [(FUSED, B.REWRITE_NONE), (UNFUSED, B.REWRITE_NONE), (FUSED, B.REWRITE_CANON_MACRO)])
+def test_encoder_small(flags, rewrite):
+    wl = W.encoder(layers=2, batch=2, seq=32, hidden=64, heads=4, ffn=128)
+    s, got, ref = run_both(wl, flags, rewrite)
+    (name,) = wl.graph.outputs
+    close(got[name], ref[name], RTOL_BF16)
+    if flags == FUSED:
+        assert s.plan_stats.n_kernels <= 2 * 11
