@@ -34,7 +34,20 @@ __device__ __forceinline__ float op_gelu_tanh(float x) {
   return x * op_sigmoid(2.0f * u);
 }
 
-template <int VV>
+// tanh.approx: 2^-11 relative error -- for epilogues whose result is rounded to bf16 anyway
+__device__ __forceinline__ float fast_tanh(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float op_gelu_tanh_fast(float x) {
+  float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
+  float h = 0.5f * x;
+  return fmaf(h, fast_tanh(u), h);
+}
+
+// kFast: the caller rounds results to bf16 (2e-2 budget), so MUFU-approximate forms are used.
+template <int VV, bool kFast = false>
 __device__ __forceinline__ void apply_op(int op, float (&acc)[VV], const float (&src)[VV], float c0, float c1) {
   switch (op) {
     case M_MOV:
@@ -123,7 +136,7 @@ __device__ __forceinline__ void apply_op(int op, float (&acc)[VV], const float (
       break;
     case M_GELU_TANH:
 #pragma unroll
-      for (int v = 0; v < VV; ++v) acc[v] = op_gelu_tanh(acc[v]);
+      for (int v = 0; v < VV; ++v) acc[v] = kFast ? op_gelu_tanh_fast(acc[v]) : op_gelu_tanh(acc[v]);
       break;
     case M_CLIP:
 #pragma unroll
@@ -150,7 +163,7 @@ struct ChainState {
   float acc[VV], t0[VV], t1[VV];
 };
 
-template <int VV, class IO>
+template <int VV, bool kFast, class IO>
 __device__ __forceinline__ void exec_one(const MicroOp m, ChainState<VV>& st, IO& io, const Program& prog) {
   if (m.op == M_SAVE) {
     if (m.idx == 0) {
@@ -168,14 +181,14 @@ __device__ __forceinline__ void exec_one(const MicroOp m, ChainState<VV>& st, IO
   if (m.src == S_IN) {
     float src[VV];
     io.load(m.idx, src);
-    apply_op<VV>(m.op, st.acc, src, c0, c1);
+    apply_op<VV, kFast>(m.op, st.acc, src, c0, c1);
   } else if (m.src == S_TMP) {
-    if (m.idx == 0) apply_op<VV>(m.op, st.acc, st.t0, c0, c1);
-    else apply_op<VV>(m.op, st.acc, st.t1, c0, c1);
+    if (m.idx == 0) apply_op<VV, kFast>(m.op, st.acc, st.t0, c0, c1);
+    else apply_op<VV, kFast>(m.op, st.acc, st.t1, c0, c1);
   } else if (m.src == S_ANCHOR) {
     float src[VV];
     io.anchor(src);
-    apply_op<VV>(m.op, st.acc, src, c0, c1);
+    apply_op<VV, kFast>(m.op, st.acc, src, c0, c1);
   } else {
     float src[VV];
     if (m.src == S_CONST) {
@@ -184,23 +197,23 @@ __device__ __forceinline__ void exec_one(const MicroOp m, ChainState<VV>& st, IO
     }
 #pragma unroll
     for (int v = 0; v < VV; ++v) src[v] = c0;
-    apply_op<VV>(m.op, st.acc, src, c0, c1);
+    apply_op<VV, kFast>(m.op, st.acc, src, c0, c1);
   }
 }
 
-template <class SP, int I, int VV, class IO>
+template <class SP, int I, int VV, bool kFast, class IO>
 __device__ __forceinline__ void static_step(ChainState<VV>& st, IO& io, const Program& prog) {
   constexpr MicroOp m = SP::op(I);
-  exec_one<VV>(m, st, io, prog);
+  exec_one<VV, kFast>(m, st, io, prog);
 }
-template <class SP, int VV, class IO, int... I>
+template <class SP, int VV, bool kFast, class IO, int... I>
 __device__ __forceinline__ void run_static(ChainState<VV>& st, IO& io, const Program& prog, std::integer_sequence<int, I...>) {
-  (static_step<SP, I, VV>(st, io, prog), ...);
+  (static_step<SP, I, VV, kFast>(st, io, prog), ...);
 }
 
 // SP = DynProg: interpret prog at run time.  Otherwise SP is a compile-time table with
 // the same opcodes as prog (the host checked), and the whole chain is straight-line code.
-template <int VV, class SP, class IO>
+template <int VV, class SP, bool kFast = false, class IO>
 __device__ __forceinline__ void run_program(const Program& prog, IO& io) {
   ChainState<VV> st;
 #pragma unroll
@@ -208,9 +221,9 @@ __device__ __forceinline__ void run_program(const Program& prog, IO& io) {
   if constexpr (SP::n == 0) {
     const int n = prog.n;
 #pragma unroll 1
-    for (int pc = 0; pc < n; ++pc) exec_one<VV>(prog.ops[pc], st, io, prog);
+    for (int pc = 0; pc < n; ++pc) exec_one<VV, kFast>(prog.ops[pc], st, io, prog);
   } else {
-    run_static<SP, VV>(st, io, prog, std::make_integer_sequence<int, SP::n>{});
+    run_static<SP, VV, kFast>(st, io, prog, std::make_integer_sequence<int, SP::n>{});
   }
 }
 

@@ -1,10 +1,499 @@
-// Tensor-core GEMM path (tcgen05 + TMA + TMEM).  Placeholder until the kernel lands:
-// nothing is eligible, so every contraction takes the CUDA-core kernel.
+// Tensor-core GEMM-anchored blocks for sm_100a: TMA -> 128B-swizzled shared memory ->
+// tcgen05.mma (bf16 x bf16 -> fp32 in tensor memory) -> tcgen05.ld epilogue that runs
+// the block's micro-op program (bias, GELU, residual, scale, mask ...) on the
+// accumulator and stores through the block's output index map.
+//
+// One persistent CTA per SM, 320 threads, warp-specialised:
+//   warp 0      TMA producer (one elected lane)
+//   warp 1      TMEM allocation, then MMA issue (one elected lane)
+//   warps 2..9  epilogue; warp w reads TMEM lanes 32*(w%4) .. 32*(w%4)+31, warps 2..5 the first
+//               half of the tile's columns, warps 6..9 the second half
+// A BK=64 shared-memory ring feeds the MMA; two accumulator stages in TMEM let the
+// epilogue of tile i overlap the main loop of tile i+1.  Every wait is bounded: when a
+// bound runs out the CTA records DNNF_ERR_TIMEOUT in the status words, stops issuing
+// work, releases tensor memory and returns.
+//
+// No TMA multicast and no clusters are used anywhere in this file.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <mutex>
+
+#include "chain.cuh"
 #include "gemm_params.h"
 #include "ir.h"
+
 namespace dnnf {
-bool tc_gemm_eligible(const GemmParams&) { return false; }
-bool tc_gemm_prepare(Launch&, std::string&) { return true; }
-int tc_gemm_launch(const Launch&, cudaStream_t) { return 1; }
-void tc_gemm_plan(Launch&) {}
+
+constexpr int TC_BM = 128, TC_BK = 64, TC_EPI_WARPS = 8, TC_THREADS = 64 + 32 * TC_EPI_WARPS;
+constexpr uint32_t kSpinLimit = 1u << 27;
+constexpr int kSmemMax = 227 * 1024;                       // dynamic shared memory per CTA
+constexpr int kStageWords = 32 * 33;                       // per epilogue warp: 32 rows x (32 + 1 pad) words
+constexpr int kSmemFixed = 1024 + 256 + TC_EPI_WARPS * kStageWords * 4;   // alignment slack, barriers, staging
+constexpr int kSmemBudget = kSmemMax - kSmemFixed;         // left for the operand ring
+
+// ---- PTX wrappers -------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the bound ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 1023u) == 1023u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* tm, uint64_t* bar, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+               ::"r"(smem_u32(dst)), "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+               ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+                 "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+               : "r"(taddr));
+}
+__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+                 "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]),
+                 "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]),
+                 "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+               : "r"(taddr));
+}
+__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (sm_100 format: version 1, 128-byte swizzle).
+//  K-major tile  [rows][64 bf16]: rows 128 B apart, 8-row groups 1024 B apart (SBO); LBO unused.
+//  MN-major tile [64 k][64 n] blocks: k rows 128 B apart, 8-row groups 1024 B apart (SBO),
+//                next 64-wide n block `lbo_bytes` further (LBO).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= 1ull << 46;          // descriptor version
+  d |= 2ull << 61;          // SWIZZLE_128B
+  return d;
+}
+
+// ---- epilogue IO ------------------------------------------------------------------------------
+// After the transpose through shared memory a lane owns, for each of 8 row groups i, four
+// consecutive columns of row (lane/8 + 4i) of the warp's 32 x 32 chunk: value index i*4 + v.
+// Neighbouring lanes sit on neighbouring columns, so epilogue loads and stores are coalesced
+// and all of a chunk's loads are in flight together.
+struct TcEpiIO {
+  static constexpr int VV = 32;
+  const GemmParams& p;
+  float accv[32];                                 // the 32 accumulator values of this lane (by value: stays in registers)
+  uint32_t row_in[kMaxIn], row_out[kMaxOut];      // offsets of the row this lane owns in TMEM layout (lane = row)
+  int m_first;                                    // global row of the warp's first row
+  uint32_t n0;                                    // first column of the chunk
+  int lane;
+  __device__ __forceinline__ uint32_t n_offset(const TensorArg& a, uint32_t n) const {
+    if (p.n_nd == 1) return n * (uint32_t)a.stride[0];
+    uint32_t off = 0, lin = n;
+#pragma unroll
+    for (int d = 0; d < 3; ++d) {
+      if (d < p.n_nd) {
+        uint32_t e = p.it.extent[d];
+        uint32_t q = (d == p.n_nd - 1) ? 0u : (__umulhi(lin, p.it.div_m[d]) >> p.it.div_s[d]);
+        if (d != p.n_nd - 1 && e == 1) q = lin;
+        off += (lin - q * e) * (uint32_t)a.stride[d];
+        lin = q;
+      }
+    }
+    return off;
+  }
+  __device__ __forceinline__ void load(int idx, float (&dst)[VV]) const {
+    const TensorArg& a = p.in[idx];
+    const uint32_t nn = n0 + (uint32_t)(lane & 7) * 4;
+    const uint32_t mine = row_in[idx];
+    const bool vec = p.vec_ok && (int)nn + 4 <= p.N;
+    const uint32_t noff = vec ? n_offset(a, nn) : 0u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int r = (lane >> 3) + 4 * i;
+      const uint32_t ro = __shfl_sync(0xffffffffu, mine, r);
+      float* d = &dst[i * 4];
+      if (m_first + r >= p.M || (int)nn >= p.N) { d[0] = d[1] = d[2] = d[3] = 0.0f; continue; }
+      if (vec) {
+        if (a.stride[0] == 0) { float x = load_scalar<false>(a, ro + noff); d[0] = d[1] = d[2] = d[3] = x; }
+        else load_vec4<false>(a, ro + noff, d);
+      } else {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) d[v] = ((int)nn + v < p.N) ? load_scalar<false>(a, ro + n_offset(a, nn + v)) : 0.0f;
+      }
+    }
+  }
+  __device__ __forceinline__ void anchor(float (&dst)[VV]) const {
+#pragma unroll
+    for (int v = 0; v < VV; ++v) dst[v] = accv[v];
+  }
+  __device__ __forceinline__ void store(int idx, const float (&val)[VV]) const {
+    const TensorArg& a = p.out[idx];
+    const uint32_t nn = n0 + (uint32_t)(lane & 7) * 4;
+    const uint32_t mine = row_out[idx];
+    const bool vec = p.vec_ok && (int)nn + 4 <= p.N;
+    const uint32_t noff = vec ? n_offset(a, nn) : 0u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int r = (lane >> 3) + 4 * i;
+      const uint32_t ro = __shfl_sync(0xffffffffu, mine, r);
+      if (m_first + r >= p.M || (int)nn >= p.N) continue;
+      if (vec) store_vec4<false>(a, ro + noff, &val[i * 4], false);
+      else {
+#pragma unroll
+        for (int v = 0; v < 4; ++v)
+          if ((int)nn + v < p.N) store_scalar<false>(a, ro + n_offset(a, nn + v), val[i * 4 + v], false);
+      }
+    }
+  }
+  __device__ __forceinline__ void row_reduce(int, float (&)[VV]) const {}
+};
+
+__device__ __forceinline__ uint32_t tc_digits(const GemmParams& p, const TensorArg& a, int first, int count, uint32_t lin) {
+  uint32_t off = 0;
+  for (int d = first; d < first + count; ++d) {
+    uint32_t e = p.it.extent[d];
+    uint32_t q = (d == first + count - 1) ? 0u : lin / e;
+    off += (lin - q * e) * (uint32_t)a.stride[d];
+    lin = q;
+  }
+  return off;
+}
+
+// ---- the kernel ---------------------------------------------------------------------------------
+template <class SP>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ GemmTcParams q, const __grid_constant__ CUtensorMap tmA,
+               const __grid_constant__ CUtensorMap tmB, int stages) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  // carve: [stages][A tile 16 KB][B tile BN*128 B], then barriers
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int BN = q.bn;
+  const uint32_t a_bytes = TC_BM * TC_BK * 2, b_bytes = (uint32_t)BN * TC_BK * 2, stage_bytes = a_bytes + b_bytes;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
+  uint64_t* empty_bar = full_bar + stages;
+  uint64_t* tfull_bar = empty_bar + stages;      // [2]
+  uint64_t* tempty_bar = tfull_bar + 2;          // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  uint32_t* stage_area = tmem_slot + 8;          // TC_EPI_WARPS x kStageWords
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&tfull_bar[s], 1); mbar_init(&tempty_bar[s], TC_EPI_WARPS); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int tiles_mn = p.tiles_m * p.tiles_n;
+  const int total_tiles = q.persistent_tiles;
+  const int k_tiles = q.k_tiles;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---------------- TMA producer ----------------
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int batch = tile / tiles_mn, r = tile - batch * tiles_mn;
+        const int tm = r / p.tiles_n, tn = r - tm * p.tiles_n;
+        const int b0 = batch % p.batch_ext[0], b1 = batch / p.batch_ext[0];
+        // a batch dim an operand is broadcast over has stride 0 and extent 1 in its tensor map
+        const int ab0 = p.A.batch_stride[0] ? b0 : 0, ab1 = p.A.batch_stride[1] ? b1 : 0;
+        const int bb0 = p.B.batch_stride[0] ? b0 : 0, bb1 = p.B.batch_stride[1] ? b1 : 0;
+        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+          const int s = it % stages;
+          const uint32_t ph = (it / stages) & 1;
+          if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_flag)) { ok = false; break; }
+          uint8_t* sa = smem + (size_t)s * stage_bytes;
+          uint8_t* sb = sa + a_bytes;
+          mbar_expect_tx(&full_bar[s], stage_bytes);
+          tma_load_4d(sa, &tmA, &full_bar[s], kt * TC_BK, tm * TC_BM, ab0, ab1);
+          if (q.b_kmajor) {
+            tma_load_4d(sb, &tmB, &full_bar[s], kt * TC_BK, tn * BN, bb0, bb1);
+          } else {
+            for (int j = 0; j < BN / 64; ++j)
+              tma_load_4d(sb + j * (64 * TC_BK * 2), &tmB, &full_bar[s], tn * BN + j * 64, kt * TC_BK, bb0, bb1);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---------------- MMA issuer ----------------
+      // instruction descriptor: D fp32, A/B bf16, A K-major, B per operand, N, M=128
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((q.b_kmajor ? 0u : 1u) << 16) | ((uint32_t)(BN >> 3) << 17) |
+                             ((uint32_t)(TC_BM >> 4) << 24);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+        const int acc = tcount & 1;
+        const uint32_t aph = (tcount >> 1) & 1;
+        if (!mbar_wait(&tempty_bar[acc], aph ^ 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+          const int s = it % stages;
+          const uint32_t ph = (it / stages) & 1;
+          if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+          const uint32_t sb = sa + a_bytes;
+#pragma unroll
+          for (int kk = 0; kk < TC_BK / 16; ++kk) {
+            const uint64_t da = make_desc(sa + kk * 32, 16, 1024);
+            const uint64_t db = q.b_kmajor ? make_desc(sb + kk * 32, 16, 1024) : make_desc(sb + kk * 2048, 64 * TC_BK * 2, 1024);
+            tc_mma_bf16(d_tmem, da, db, idesc, (kt | kk) ? 1u : 0u);
+          }
+          tc_commit(&empty_bar[s]);          // frees the smem stage once these MMAs have read it
+        }
+        if (ok) tc_commit(&tfull_bar[acc]);  // accumulator complete
+      }
+    }
+  } else {
+    // ---------------- epilogue warps ----------------
+    const int sub = warp & 3;                 // TMEM sub-partition this warp may read
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      const int batch = tile / tiles_mn, r = tile - batch * tiles_mn;
+      const int tm = r / p.tiles_n, tn = r - tm * p.tiles_n;
+      const int acc = tcount & 1;
+      const uint32_t aph = (tcount >> 1) & 1;
+      if (!mbar_wait(&tfull_bar[acc], aph, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      TcEpiIO io{p};
+      uint32_t* stage = stage_area + (warp - 2) * kStageWords;
+      io.lane = lane;
+      io.m_first = tm * TC_BM + sub * 32;
+      const int m = io.m_first + lane;
+      const uint32_t mm = m < p.M ? (uint32_t)m : 0u;
+      // (fully unrolled with constant indices so that the offset tables stay in registers)
+#pragma unroll
+      for (int k = 0; k < kMaxIn; ++k) {
+        io.row_in[k] = 0;
+        if (k < p.n_in)
+          io.row_in[k] = (uint32_t)p.in[k].base + tc_digits(p, p.in[k], p.n_nd, p.m_nd, mm) + tc_digits(p, p.in[k], p.n_nd + p.m_nd, p.b_nd, (uint32_t)batch);
+      }
+#pragma unroll
+      for (int k = 0; k < kMaxOut; ++k) {
+        io.row_out[k] = 0;
+        if (k < p.n_out)
+          io.row_out[k] = (uint32_t)p.out[k].base + tc_digits(p, p.out[k], p.n_nd, p.m_nd, mm) + tc_digits(p, p.out[k], p.n_nd + p.m_nd, p.b_nd, (uint32_t)batch);
+      }
+      const int half = (warp - 2) >> 2;        // which half of the tile's columns
+      const int c_begin = half * (BN / 2), c_end = c_begin + BN / 2;
+      const uint32_t t_row = tmem_base + ((uint32_t)(sub * 32) << 16) + (uint32_t)(acc * BN);
+      for (int c = c_begin; c < c_end; c += 32) {
+        const int n0 = tn * BN + c;
+        if (n0 >= p.N) break;                  // uniform across the warp
+        uint32_t raw[32];
+        tc_ld32_issue(t_row + c, raw);
+        tc_ld_wait();
+        // transpose: lane = row  ->  lane = (row group, 4-column piece)
+#pragma unroll
+        for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = raw[j];
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) io.accv[i * 4 + e] = __uint_as_float(stage[((lane >> 3) + 4 * i) * 33 + (lane & 7) * 4 + e]);
+        __syncwarp();
+        io.n0 = (uint32_t)n0;
+        run_program<32, SP, true>(p.prog, io);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+    }
+  }
+
+  // ---------------- teardown ----------------
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0 && p.status) { atomicExch(&p.status[0], DNNF_ERR_TIMEOUT); atomicExch(&p.status[1], p.block_index); }
+    // give copies that are still in flight time to land before shared memory is released
+    if (threadIdx.x == 0) { long long t0 = clock64(); while (clock64() - t0 < 2000000) {} }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// ---- static epilogue programs -----------------------------------------------------------------------
+#define MO(o, s, i) MicroOp{o, s, i, 0}
+DNNF_SP_BEGIN(EP_Store, 2) MO(M_MOV, S_ANCHOR, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(EP_Bias, 3) MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(EP_BiasGeluTanh, 4) MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_GELU_TANH, S_NONE, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(EP_BiasResidual, 4) MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(EP_ScaleMask, 4) MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_CONST, 0), MO(M_ADD, S_IN, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(EP_BiasGeluPrimitives, 9)
+  MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_SAVE, S_TMP, 0), MO(M_MUL, S_CONST, 0), MO(M_ERF, S_NONE, 0), MO(M_ADD, S_CONST, 1),
+  MO(M_MUL, S_TMP, 0), MO(M_MUL, S_CONST, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+#undef MO
+using EpiStatic = TypeList<EP_Store, EP_Bias, EP_BiasGeluTanh, EP_BiasResidual, EP_ScaleMask, EP_BiasGeluPrimitives>;
+
+// ---- host side --------------------------------------------------------------------------------------
+static GemmParams& gp_of(Launch& L) { return *reinterpret_cast<GemmParams*>(L.blob.data()); }
+static const GemmParams& gp_of(const Launch& L) { return *reinterpret_cast<const GemmParams*>(L.blob.data()); }
+static GemmTcParams& tc_of(Launch& L) { return *reinterpret_cast<GemmTcParams*>(L.blob.data() + sizeof(GemmParams)); }
+static const GemmTcParams& tc_of(const Launch& L) { return *reinterpret_cast<const GemmTcParams*>(L.blob.data() + sizeof(GemmParams)); }
+
+bool tc_gemm_eligible(const GemmParams& gp) {
+  if (gp.A.dtype != DNNF_BF16 || gp.B.dtype != DNNF_BF16) return false;
+  auto ok8 = [](int64_t v) { return v % 8 == 0; };
+  // A: K-major only
+  if (gp.A.stride_col != 1 || !ok8(gp.A.stride_row) || !ok8(gp.A.base) || !ok8(gp.A.batch_stride[0]) || !ok8(gp.A.batch_stride[1])) return false;
+  bool b_k = gp.B.stride_row == 1, b_n = gp.B.stride_col == 1;
+  if (gp.K == 1 && b_n) b_k = false;
+  if (!b_k && !b_n) return false;
+  int64_t other = b_n ? gp.B.stride_row : gp.B.stride_col;
+  if (!ok8(other) || !ok8(gp.B.base) || !ok8(gp.B.batch_stride[0]) || !ok8(gp.B.batch_stride[1])) return false;
+  if (gp.A.stride_row <= 0 || other <= 0) return false;
+  if (gp.K % 8 || (b_n && gp.N % 8)) return false;       // tensor-map extents in 16-byte units
+  return true;
+}
+
+void tc_gemm_plan(Launch& L) {
+  GemmParams& gp = gp_of(L);
+  GemmTcParams& tc = tc_of(L);
+  tc.a_kmajor = 1;
+  tc.b_kmajor = (gp.B.stride_col != 1) ? 1 : 0;
+  tc.k_tiles = (gp.K + TC_BK - 1) / TC_BK;
+  int nb = gp.batch_ext[0] * gp.batch_ext[1];
+  int tiles_m = (gp.M + TC_BM - 1) / TC_BM;
+  // N tile: the candidate with the best SM utilisation over whole waves; larger tiles win ties
+  int best_bn = 64; double best = -1;
+  for (int bn : {256, 192, 128, 64}) {
+    if (bn > 64 && bn / 2 >= gp.N) continue;
+    int tiles = tiles_m * ((gp.N + bn - 1) / bn) * nb;
+    int waves = (tiles + 147) / 148;
+    double useful = (double)gp.N / (((gp.N + bn - 1) / bn) * bn);
+    double eff = (double)tiles / (waves * 148.0) * useful * (bn >= 128 ? 1.0 : 0.9);
+    if (eff > best + 1e-9) { best = eff; best_bn = bn; }
+  }
+  tc.bn = best_bn;
+  gp.tiles_m = tiles_m;
+  gp.tiles_n = (gp.N + tc.bn - 1) / tc.bn;
+  tc.persistent_tiles = gp.tiles_m * gp.tiles_n * nb;
+  L.grid = std::min(tc.persistent_tiles, 148);
+  L.threads = TC_THREADS;
+  int stage_bytes = TC_BM * TC_BK * 2 + tc.bn * TC_BK * 2;
+  int stages = std::min(8, kSmemBudget / stage_bytes);
+  L.smem = (size_t)stages * stage_bytes + kSmemFixed;
+  L.variant = 1;
+  L.static_id = StaticSet<EpiStatic>::find(gp.prog);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess && qr == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// dims innermost first: {inner, outer, b0, b1}
+static bool encode(CUtensorMap* tm, void* base, int64_t ext_inner, int64_t ext_outer, int64_t stride_outer, const int32_t* bext,
+                   const int64_t* bstride, int box_inner, int box_outer, std::string& err) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) { err = "cuTensorMapEncodeTiled is not available"; return false; }
+  cuuint64_t dims[4] = {(cuuint64_t)ext_inner, (cuuint64_t)ext_outer, (cuuint64_t)bext[0], (cuuint64_t)bext[1]};
+  // a broadcast (stride 0) batch dim is addressed with coordinate 0 only; give it extent 1 and any legal stride
+  cuuint64_t s1 = (cuuint64_t)stride_outer * 2;
+  cuuint64_t s2 = bstride[0] ? (cuuint64_t)bstride[0] * 2 : s1 * ext_outer;
+  cuuint64_t s3 = bstride[1] ? (cuuint64_t)bstride[1] * 2 : s2 * bext[0];
+  if (!bstride[0]) dims[2] = 1;
+  if (!bstride[1]) dims[3] = 1;
+  cuuint64_t strides[3] = {s1, s2, s3};
+  cuuint32_t box[4] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult rc = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (rc != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)rc); return false; }
+  return true;
+}
+
+bool tc_gemm_prepare(Launch& L, std::string& err) {
+  GemmParams& gp = gp_of(L);
+  GemmTcParams& tc = tc_of(L);
+  uint16_t* a = reinterpret_cast<uint16_t*>(gp.A.ptr) + gp.A.base;
+  uint16_t* b = reinterpret_cast<uint16_t*>(gp.B.ptr) + gp.B.base;
+  if (((uintptr_t)a & 15) || ((uintptr_t)b & 15)) { err = "GEMM operand is not 16-byte aligned"; return false; }
+  if (!encode(&tc.tmA, a, gp.K, gp.M, gp.A.stride_row, gp.batch_ext, gp.A.batch_stride, TC_BK, TC_BM, err)) return false;
+  if (tc.b_kmajor) {
+    if (!encode(&tc.tmB, b, gp.K, gp.N, gp.B.stride_col, gp.batch_ext, gp.B.batch_stride, TC_BK, tc.bn, err)) return false;
+  } else {
+    if (!encode(&tc.tmB, b, gp.N, gp.K, gp.B.stride_row, gp.batch_ext, gp.B.batch_stride, 64, TC_BK, err)) return false;
+  }
+  return true;
+}
+
+struct TcLauncher {
+  const Launch& L; cudaStream_t st; int stages;
+  template <class SP> void run() {
+    static bool attr_set = false;     // per instantiation
+    if (!attr_set) { cudaFuncSetAttribute(gemm_tc_kernel<SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax); attr_set = true; }
+    gemm_tc_kernel<SP><<<L.grid, TC_THREADS, L.smem, st>>>(gp_of(L), tc_of(L), tc_of(L).tmA, tc_of(L).tmB, stages);
+  }
+};
+
+int tc_gemm_launch(const Launch& L, cudaStream_t st) {
+  const GemmTcParams& tc = tc_of(L);
+  int stage_bytes = TC_BM * TC_BK * 2 + tc.bn * TC_BK * 2;
+  int stages = (int)((L.smem - kSmemFixed) / stage_bytes);
+  TcLauncher F{L, st, stages};
+  if (!(L.static_id > 0 && StaticSet<EpiStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
+  return cudaGetLastError() == cudaSuccess ? 0 : 1;
+}
+
+}  // namespace dnnf

@@ -84,7 +84,7 @@ def measure_workload(torch, dev, wl, pk, flags, copies, iters=20, rewrite=B.REWR
             "irs_bytes": int(s0.plan_stats.irs_bytes_fused), "blocks": per_block}
 
 
-def per_config(dev, pk):
+def per_config(dev, pk, only=None):
     import torch
     out = {}
     cases = [
@@ -94,8 +94,11 @@ def per_config(dev, pk):
         ("cfg2a batch-512 variant", W.masked_softmax(batch=512), 1),
         ("cfg2b add+LayerNorm+GELU [1024,768]", W.add_layernorm_gelu(), 24),
         ("cfg2b 131072-row variant", W.add_layernorm_gelu(rows=131072), 1),
+        ("cfg3 GEMM+bias+GELU ; GEMM+bias+residual bf16 [4096,768,3072]", W.ffn_block(), 8),
     ]
     for name, wl, copies in cases:
+        if only and only not in name:
+            continue
         try:
             fused = measure_workload(torch, dev, wl, pk, B.PLAN_FUSED, copies)
             unfused = measure_workload(torch, dev, wl, pk, B.PLAN_UNFUSED, copies)

@@ -36,6 +36,7 @@ def test_ffn_block(cfg, flags):
     s = check(W.ffn_block(m, hidden, ffn), RTOL_BF16, flags, expect_blocks=2 if flags == FUSED else 6)
     if flags == FUSED:
         assert [b["family"] for b in s.g.blocks()] == ["gemm", "gemm"]
+        assert all(b["variant"] == 1 for b in s.g.blocks()), "expected the tensor-core kernel"
 
 
 def test_batched_matmul_with_transposed_and_strided_operands():
