@@ -22,6 +22,12 @@ bool tc_gemm_eligible(const GemmParams& gp);
 bool tc_gemm_prepare(Launch& L, std::string& err);                  // encode tensor maps after pointers are known
 int tc_gemm_launch(const Launch& L, cudaStream_t st);
 void tc_gemm_plan(Launch& L);                                        // choose tiles / grid
+bool conv1x1_direct_eligible(const GemmParams& gp);
+void conv1x1_direct_plan(Launch& L);
+int conv1x1_direct_launch(const Launch& L, cudaStream_t st);
+int lower_dwconv(const Graph& g, const std::vector<int>& ops, int anchor, Block& out, std::string& why);
+int dwconv_launch(const Launch& L, cudaStream_t st);
+void dwconv_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
 
 static GemmParams& gp_of(Launch& L) { return *reinterpret_cast<GemmParams*>(L.blob.data()); }
 static const GemmParams& gp_of(const Launch& L) { return *reinterpret_cast<const GemmParams*>(L.blob.data()); }
@@ -217,7 +223,7 @@ bool pack_operand(const Graph& g, const std::vector<int64_t>& orig_dims, const s
 int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flags, int anchor, Block& out, std::string& why) {
   (void)flags;
   const Op& A = g.ops[anchor];
-  if (A.kind == DNNF_OP_DWCONV3X3) { why = "depthwise convolution kernels not built"; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (A.kind == DNNF_OP_DWCONV3X3) return lower_dwconv(g, ops, anchor, out, why);
   std::set<int> in_block(ops.begin(), ops.end());
   const Tensor& C = g.tensors[A.out[0]];
   const Tensor& TA = g.tensors[A.in[0]];
@@ -405,6 +411,8 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
   if (tc_gemm_eligible(gp)) {
     L.variant = 1;
     tc_gemm_plan(L);
+  } else if (A.kind == DNNF_OP_CONV1X1 && conv1x1_direct_eligible(gp)) {
+    conv1x1_direct_plan(L);
   } else {
     L.variant = 0;
     gp.tiles_m = (gp.M + FB_T - 1) / FB_T; gp.tiles_n = (gp.N + FB_T - 1) / FB_T;
@@ -415,6 +423,7 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
 }
 
 void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op, std::string& err) {
+  if (L.family == DNNF_FAMILY_DWCONV) { dwconv_patch(L, ip, op); return; }
   GemmParams& gp = gp_of(L);
   bool changed = gp.A.ptr != ip[0] || gp.B.ptr != ip[1];
   gp.A.ptr = ip[0]; gp.B.ptr = ip[1];
@@ -424,6 +433,8 @@ void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vecto
 }
 
 int launch_contraction(const Launch& L, void* status_words, int block_index, cudaStream_t st, std::string& err) {
+  if (L.family == DNNF_FAMILY_DWCONV) { int rc = dwconv_launch(L, st); if (rc) err = "depthwise convolution launch failed"; return rc; }
+  if (L.variant == 2) { int rc = conv1x1_direct_launch(L, st); if (rc) err = "pointwise convolution launch failed"; return rc; }
   GemmParams gp = gp_of(L);
   gp.status = reinterpret_cast<int32_t*>(status_words);
   gp.block_index = block_index;

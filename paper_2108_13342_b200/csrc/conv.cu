@@ -1,0 +1,339 @@
+// fp32 NHWC convolution anchors on CUDA cores, each with the block's epilogue program:
+//  * pointwise (1x1) convolution, pixel-stationary: a lane keeps one pixel's partial sums
+//    for a slice of the output channels in registers, the [Cin x Cout] weights sit in
+//    shared memory and are read as broadcast 128-bit words;
+//  * depthwise 3x3, stride 1, zero padding 1: a thread owns one (image, column, 4-channel
+//    group) and walks down the rows with a rolling 3x3 window, so every input value is
+//    loaded three times from L1/L2 instead of nine.
+// Both are bound by HBM traffic at the shapes of a MobileNet block (K = 24 / 144).
+#include <cuda_runtime.h>
+
+#include <algorithm>
+
+#include "chain.cuh"
+#include "gemm_params.h"
+#include "lower.h"
+
+namespace dnnf {
+
+// ---------------------------------------------------------------------------
+// Pointwise convolution: [P x K] * [K x N], fp32, rows contiguous.
+// LPP lanes share a pixel; lane q of them owns float4 columns f = j*LPP + q, j < NPT.
+// ---------------------------------------------------------------------------
+template <int NPT, int LPP>
+struct PwIO {
+  static constexpr int VV = 4 * NPT;
+  const GemmParams& p;
+  float accv[VV];
+  uint32_t pix;            // pixel index (row of the [P x N] result)
+  int q;                   // lane's slot among the LPP lanes of the pixel
+  bool ok;
+  __device__ __forceinline__ uint32_t off(const TensorArg& a, int j) const {
+    return (uint32_t)a.base + pix * (uint32_t)a.stride[1] + (uint32_t)(4 * (j * LPP + q)) * (uint32_t)a.stride[0];
+  }
+  __device__ __forceinline__ void load(int idx, float (&dst)[VV]) const {
+    const TensorArg& a = p.in[idx];
+#pragma unroll
+    for (int j = 0; j < NPT; ++j) {
+      float* d = &dst[4 * j];
+      if (!ok) { d[0] = d[1] = d[2] = d[3] = 0.0f; continue; }
+      if (a.stride[0] == 0) { float x = load_scalar<true>(a, off(a, j)); d[0] = d[1] = d[2] = d[3] = x; }
+      else load_vec4<true>(a, off(a, j), d);
+    }
+  }
+  __device__ __forceinline__ void anchor(float (&dst)[VV]) const {
+#pragma unroll
+    for (int v = 0; v < VV; ++v) dst[v] = accv[v];
+  }
+  __device__ __forceinline__ void store(int idx, const float (&val)[VV]) const {
+    if (!ok) return;
+    const TensorArg& a = p.out[idx];
+#pragma unroll
+    for (int j = 0; j < NPT; ++j) store_vec4<true>(a, off(a, j), &val[4 * j], false);
+  }
+  __device__ __forceinline__ void row_reduce(int, float (&)[VV]) const {}
+};
+
+template <int NPT, int LPP, class SP>
+__global__ void __launch_bounds__(256) conv1x1_kernel(const __grid_constant__ GemmParams p) {
+  extern __shared__ float wsm[];                 // [K][N]
+  const int K = p.K, N = p.N;
+  const float* W = reinterpret_cast<const float*>(p.B.ptr) + p.B.base;
+  for (int i = threadIdx.x * 4; i < K * N; i += 256 * 4)
+    *reinterpret_cast<float4*>(&wsm[i]) = __ldg(reinterpret_cast<const float4*>(W + i));
+  __syncthreads();
+  const float* X = reinterpret_cast<const float*>(p.A.ptr) + p.A.base;
+  constexpr int PPW = 32 / LPP;                  // pixels per warp
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int warps_total = gridDim.x * 8;
+  PwIO<NPT, LPP> io{p};
+  io.q = lane % LPP;
+  for (int64_t base = (int64_t)(blockIdx.x * 8 + warp) * PPW; base < p.M; base += (int64_t)warps_total * PPW) {
+    const int64_t pix = base + lane / LPP;
+    io.ok = pix < p.M;
+    io.pix = (uint32_t)(io.ok ? pix : 0);
+    const float* xr = X + (int64_t)io.pix * p.A.stride_row;
+#pragma unroll
+    for (int v = 0; v < 4 * NPT; ++v) io.accv[v] = 0.0f;
+    for (int k0 = 0; k0 < K; k0 += 8) {
+      float x[8];
+      {
+        float4 a = __ldg(reinterpret_cast<const float4*>(xr + k0));
+        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+        if (k0 + 4 < K) { float4 b = __ldg(reinterpret_cast<const float4*>(xr + k0 + 4)); x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w; }
+        else { x[4] = x[5] = x[6] = x[7] = 0.0f; }
+      }
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        if (k0 + kk < K) {
+          const float* wr = wsm + (k0 + kk) * N + 4 * io.q;
+#pragma unroll
+          for (int j = 0; j < NPT; ++j) {
+            float4 w = *reinterpret_cast<const float4*>(wr + 4 * j * LPP);
+            io.accv[4 * j + 0] = fmaf(x[kk], w.x, io.accv[4 * j + 0]);
+            io.accv[4 * j + 1] = fmaf(x[kk], w.y, io.accv[4 * j + 1]);
+            io.accv[4 * j + 2] = fmaf(x[kk], w.z, io.accv[4 * j + 2]);
+            io.accv[4 * j + 3] = fmaf(x[kk], w.w, io.accv[4 * j + 3]);
+          }
+        }
+      }
+    }
+    run_program<4 * NPT, SP>(p.prog, io);
+  }
+}
+
+#define MO(o, s, i) MicroOp{o, s, i, 0}
+DNNF_SP_BEGIN(CP_ScaleShiftClip, 5)
+  MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_CLIP, S_CONST, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(CP_ScaleShiftResidual, 5)
+  MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_ADD, S_IN, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(CP_Store, 2) MO(M_MOV, S_ANCHOR, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+#undef MO
+using ConvStatic = TypeList<CP_ScaleShiftClip, CP_ScaleShiftResidual, CP_Store>;
+
+static const GemmParams& gp_of(const Launch& L) { return *reinterpret_cast<const GemmParams*>(L.blob.data()); }
+
+// (NPT, LPP) pairs that are instantiated; the host picks one with NPT*LPP == N/4
+static bool pw_shape(int n4, int& npt, int& lpp) {
+  static const int table[][2] = {{9, 4}, {3, 2}, {6, 4}, {4, 4}, {8, 4}, {2, 4}, {1, 4}, {5, 4}, {1, 2}, {1, 1}, {3, 1}};
+  for (auto& t : table) if (t[0] * t[1] == n4) { npt = t[0]; lpp = t[1]; return true; }
+  return false;
+}
+
+bool conv1x1_direct_eligible(const GemmParams& gp) {
+  if (gp.A.dtype != 0 || gp.B.dtype != 0) return false;
+  if (gp.batch_ext[0] * gp.batch_ext[1] != 1) return false;
+  if (gp.A.stride_col != 1 || gp.A.stride_row % 4 || gp.A.base % 4) return false;
+  if (gp.B.stride_col != 1 || gp.B.stride_row != gp.N || gp.B.base % 4) return false;
+  if (gp.N % 4 || gp.K % 4 || (int64_t)gp.K * gp.N * 4 > 96 * 1024) return false;
+  if (gp.n_nd != 1 || gp.m_nd != 1 || gp.b_nd != 1 || !gp.vec_ok) return false;
+  for (int i = 0; i < gp.n_in; ++i) if (gp.in[i].dtype != 0) return false;
+  for (int i = 0; i < gp.n_out; ++i) if (gp.out[i].dtype != 0) return false;
+  int a, b;
+  return pw_shape(gp.N / 4, a, b);
+}
+
+void conv1x1_direct_plan(Launch& L) {
+  GemmParams& gp = *reinterpret_cast<GemmParams*>(L.blob.data());
+  L.variant = 2;
+  L.threads = 256;
+  L.smem = (size_t)gp.K * gp.N * 4;
+  int npt, lpp;
+  pw_shape(gp.N / 4, npt, lpp);
+  int64_t warps = (gp.M + (32 / lpp) - 1) / (32 / lpp);
+  int64_t ctas = (warps + 7) / 8;
+  L.grid = (int)std::min<int64_t>(ctas, 148 * 4);
+  L.static_id = StaticSet<ConvStatic>::find(gp.prog);
+}
+
+template <int NPT, int LPP>
+struct PwLauncher {
+  const Launch& L; cudaStream_t st;
+  template <class SP> void run() {
+    static bool attr = false;
+    if (!attr) { cudaFuncSetAttribute(conv1x1_kernel<NPT, LPP, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); attr = true; }
+    conv1x1_kernel<NPT, LPP, SP><<<L.grid, 256, L.smem, st>>>(gp_of(L));
+  }
+};
+template <int NPT, int LPP, bool kStatic>
+static void pw_launch(const Launch& L, cudaStream_t st) {
+  PwLauncher<NPT, LPP> F{L, st};
+  if (kStatic && L.static_id > 0 && StaticSet<ConvStatic>::dispatch(L.static_id, F)) return;
+  F.template run<DynProg>();
+}
+
+int conv1x1_direct_launch(const Launch& L, cudaStream_t st) {
+  const GemmParams& gp = gp_of(L);
+  int npt = 0, lpp = 0;
+  pw_shape(gp.N / 4, npt, lpp);
+  switch (npt * 10 + lpp) {
+    case 94: pw_launch<9, 4, true>(L, st); break;
+    case 32: pw_launch<3, 2, true>(L, st); break;
+    case 64: pw_launch<6, 4, false>(L, st); break;
+    case 44: pw_launch<4, 4, false>(L, st); break;
+    case 84: pw_launch<8, 4, false>(L, st); break;
+    case 24: pw_launch<2, 4, false>(L, st); break;
+    case 14: pw_launch<1, 4, false>(L, st); break;
+    case 54: pw_launch<5, 4, false>(L, st); break;
+    case 12: pw_launch<1, 2, false>(L, st); break;
+    case 11: pw_launch<1, 1, false>(L, st); break;
+    case 31: pw_launch<3, 1, false>(L, st); break;
+    default: return 2;
+  }
+  return cudaGetLastError() == cudaSuccess ? 0 : 1;
+}
+
+// ---------------------------------------------------------------------------
+// Depthwise 3x3
+// ---------------------------------------------------------------------------
+struct DwParams {
+  int32_t N, H, W, C;
+  const float* x;
+  const float* k;          // [3][3][C]
+  int32_t n_in, n_out;
+  TensorArg in[kMaxIn];    // strides over (c, w, h, n), innermost first
+  TensorArg out[kMaxOut];
+  Program prog;
+};
+
+struct DwIO {
+  const DwParams& p;
+  float accv[4];
+  uint32_t n, h, w, c;
+  __device__ __forceinline__ uint32_t off(const TensorArg& a) const {
+    return (uint32_t)a.base + c * (uint32_t)a.stride[0] + w * (uint32_t)a.stride[1] + h * (uint32_t)a.stride[2] + n * (uint32_t)a.stride[3];
+  }
+  __device__ __forceinline__ void load(int idx, float (&dst)[4]) const {
+    const TensorArg& a = p.in[idx];
+    if (a.stride[0] == 0) { float x = load_scalar<true>(a, off(a)); dst[0] = dst[1] = dst[2] = dst[3] = x; }
+    else load_vec4<true>(a, off(a), dst);
+  }
+  __device__ __forceinline__ void anchor(float (&dst)[4]) const {
+#pragma unroll
+    for (int v = 0; v < 4; ++v) dst[v] = accv[v];
+  }
+  __device__ __forceinline__ void store(int idx, const float (&val)[4]) const { store_vec4<true>(p.out[idx], off(p.out[idx]), val, false); }
+  __device__ __forceinline__ void row_reduce(int, float (&)[4]) const {}
+};
+
+__device__ __forceinline__ float4 ld4_or_zero(const float* p, bool ok) {
+  return ok ? __ldg(reinterpret_cast<const float4*>(p)) : make_float4(0.f, 0.f, 0.f, 0.f);
+}
+__device__ __forceinline__ void fma4(float (&acc)[4], const float4& x, const float4& k) {
+  acc[0] = fmaf(x.x, k.x, acc[0]); acc[1] = fmaf(x.y, k.y, acc[1]); acc[2] = fmaf(x.z, k.z, acc[2]); acc[3] = fmaf(x.w, k.w, acc[3]);
+}
+
+// HS rows per thread: the grid covers (n, h-strip, w, c4)
+template <class SP>
+__global__ void __launch_bounds__(256) dwconv_kernel(const __grid_constant__ DwParams p, int HS) {
+  const int C4 = p.C / 4;
+  const int strips = (p.H + HS - 1) / HS;
+  int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  const int64_t total = (int64_t)p.N * strips * p.W * C4;
+  if (t >= total) return;
+  const int c4 = (int)(t % C4); t /= C4;
+  const int w = (int)(t % p.W); t /= p.W;
+  const int s = (int)(t % strips); const int n = (int)(t / strips);
+  const int h0 = s * HS, h1 = min(p.H, h0 + HS);
+  float4 kw[9];
+#pragma unroll
+  for (int i = 0; i < 9; ++i) kw[i] = __ldg(reinterpret_cast<const float4*>(p.k + i * p.C + c4 * 4));
+  const float* xb = p.x + ((int64_t)n * p.H * p.W) * p.C + c4 * 4;
+  const bool wl = w > 0, wr = w + 1 < p.W;
+  auto row = [&](int h, float4 (&r)[3]) {
+    const bool ok = h >= 0 && h < p.H;
+    const float* q = xb + ((int64_t)h * p.W + w) * p.C;
+    r[0] = ld4_or_zero(q - p.C, ok && wl); r[1] = ld4_or_zero(q, ok); r[2] = ld4_or_zero(q + p.C, ok && wr);
+  };
+  float4 r0[3], r1[3], r2[3];
+  row(h0 - 1, r0); row(h0, r1);
+  DwIO io{p};
+  io.n = n; io.w = w; io.c = c4 * 4;
+  for (int h = h0; h < h1; ++h) {
+    row(h + 1, r2);
+    io.accv[0] = io.accv[1] = io.accv[2] = io.accv[3] = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 3; ++j) { fma4(io.accv, r0[j], kw[j]); fma4(io.accv, r1[j], kw[3 + j]); fma4(io.accv, r2[j], kw[6 + j]); }
+    io.h = h;
+    run_program<4, SP>(p.prog, io);
+#pragma unroll
+    for (int j = 0; j < 3; ++j) { r0[j] = r1[j]; r1[j] = r2[j]; }
+  }
+}
+
+static const DwParams& dw_of(const Launch& L) { return *reinterpret_cast<const DwParams*>(L.blob.data()); }
+
+struct DwLauncher {
+  const Launch& L; cudaStream_t st; int hs;
+  template <class SP> void run() { dwconv_kernel<SP><<<L.grid, 256, 0, st>>>(dw_of(L), hs); }
+};
+
+int dwconv_launch(const Launch& L, cudaStream_t st) {
+  DwLauncher F{L, st, L.variant};
+  if (!(L.static_id > 0 && StaticSet<ConvStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
+  return cudaGetLastError() == cudaSuccess ? 0 : 1;
+}
+
+void dwconv_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op) {
+  DwParams& dp = *reinterpret_cast<DwParams*>(L.blob.data());
+  dp.x = reinterpret_cast<const float*>(ip[0]);
+  dp.k = reinterpret_cast<const float*>(ip[1]);
+  for (int i = 0; i < dp.n_in; ++i) dp.in[i].ptr = ip[2 + i];
+  for (int i = 0; i < dp.n_out; ++i) dp.out[i].ptr = op[i];
+}
+
+int lower_dwconv(const Graph& g, const std::vector<int>& ops, int anchor, Block& out, std::string& why) {
+  const Op& A = g.ops[anchor];
+  const Tensor& X = g.tensors[A.in[0]];
+  const Tensor& Kt = g.tensors[A.in[1]];
+  const Tensor& Y = g.tensors[A.out[0]];
+  std::set<int> in_block(ops.begin(), ops.end());
+  if (X.dtype != DNNF_F32 || Kt.dtype != DNNF_F32) { why = "depthwise convolution is fp32 only"; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (X.dims[3] % 4) { why = "depthwise convolution needs a channel count that is a multiple of 4"; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (in_block.count(X.producer) || in_block.count(Kt.producer)) { why = "operators in front of a convolution anchor (no prologue fusion)"; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (X.numel() >= (1ll << 31)) { why = "tensor too large"; return DNNF_ERR_UNSUPPORTED_OP; }
+  LowerCtx cx(g);
+  cx.ops = ops; cx.in_block = in_block;
+  cx.ext = Y.dims;
+  if (!derive_views(cx, A.out[0], {anchor})) { why = cx.why; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (cx.ext != Y.dims) { why = "epilogue reshapes a depthwise convolution's result"; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (!emit_program(cx, A.out[0], 2)) { why = cx.why; return DNNF_ERR_UNSUPPORTED_OP; }
+  Launch& L = out.launch;
+  L = Launch{};
+  L.blob.assign(sizeof(DwParams), 0);
+  DwParams& dp = *reinterpret_cast<DwParams*>(L.blob.data());
+  dp.N = (int)Y.dims[0]; dp.H = (int)Y.dims[1]; dp.W = (int)Y.dims[2]; dp.C = (int)Y.dims[3];
+  dp.n_in = (int)cx.ins.size(); dp.n_out = (int)cx.outs.size();
+  auto fill = [&](TensorArg& a, const ExtArg& e, bool is_out) {
+    a.ptr = nullptr; a.base = (int32_t)e.view.c0; a.dtype = g.tensors[e.tensor].dtype; a.mode = 0;
+    for (int d = 0; d < kMaxDims; ++d) a.stride[d] = d < 4 ? (int32_t)e.view.coef[3 - d] : 0;
+    if (a.dtype != DNNF_F32) return false;
+    if (a.stride[0] == 1) { if (a.base % 4) return false; for (int d = 1; d < 4; ++d) if (a.stride[d] % 4) return false; }
+    else if (!(a.stride[0] == 0 && !is_out)) return false;
+    return true;
+  };
+  for (size_t i = 0; i < cx.ins.size(); ++i) if (!fill(dp.in[i], cx.ins[i], false)) { why = "depthwise epilogue operand is not fp32 / channel-contiguous"; return DNNF_ERR_UNSUPPORTED_OP; }
+  for (size_t i = 0; i < cx.outs.size(); ++i) if (!fill(dp.out[i], cx.outs[i], true)) { why = "depthwise epilogue output is not fp32 / channel-contiguous"; return DNNF_ERR_UNSUPPORTED_OP; }
+  dp.prog = cx.prog;
+  L.ew.prog = cx.prog;
+  L.in_tensors = {A.in[0], A.in[1]};
+  out.inputs = {A.in[0], A.in[1]};
+  out.outputs.clear();
+  for (auto& a : cx.ins) { L.in_tensors.push_back(a.tensor); if (std::find(out.inputs.begin(), out.inputs.end(), a.tensor) == out.inputs.end()) out.inputs.push_back(a.tensor); }
+  for (auto& a : cx.outs) { L.out_tensors.push_back(a.tensor); out.outputs.push_back(a.tensor); }
+  L.family = DNNF_FAMILY_DWCONV;
+  // rows per thread: enough threads to fill the machine, long enough strips to reuse the window
+  int hs = dp.H;
+  int64_t threads_full = (int64_t)dp.N * dp.W * (dp.C / 4);
+  while (hs > 7 && threads_full * ((dp.H + hs - 1) / hs) < 148 * 2048 * 2) hs = (hs + 1) / 2;
+  L.variant = hs;
+  int64_t total = threads_full * ((dp.H + hs - 1) / hs);
+  L.grid = (int)((total + 255) / 256);
+  L.threads = 256;
+  L.flops = 2ll * 9 * Y.numel();
+  L.static_id = StaticSet<ConvStatic>::find(dp.prog);
+  out.lowered = true;
+  return DNNF_OK;
+}
+
+}  // namespace dnnf

@@ -95,6 +95,7 @@ def per_config(dev, pk, only=None):
         ("cfg2b add+LayerNorm+GELU [1024,768]", W.add_layernorm_gelu(), 24),
         ("cfg2b 131072-row variant", W.add_layernorm_gelu(rows=131072), 1),
         ("cfg3 GEMM+bias+GELU ; GEMM+bias+residual bf16 [4096,768,3072]", W.ffn_block(), 8),
+        ("cfg4 MBConv fp32 NHWC [32,56,56,24->144->24]", W.mbconv_block(), 2),
     ]
     for name, wl, copies in cases:
         if only and only not in name:

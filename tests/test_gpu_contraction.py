@@ -90,6 +90,28 @@ def test_conv1x1_with_epilogue(cfg):
     check(W.Workload(g, ins), RTOL_F32, FUSED, expect_blocks=1)
 
 
+@pytest.mark.parametrize("cfg", [(1, 5, 6, 8), (2, 7, 9, 144), (1, 1, 1, 4), (1, 3, 1, 12), (2, 30, 17, 24)])
+def test_dwconv3x3_with_epilogue(cfg):
+    n, h, w, c = cfg
+    g = graph()
+    g.ext("X", (n, h, w, c)); g.ext("Kd", (3, 3, c)); g.ext("s", (c,)); g.ext("t", (c,))
+    e = g.add("DwConv3x3", ["X", "Kd"])
+    e = g.add("ScaleShift", [e, "s", "t"], axis=-1)
+    g.mark_output(g.add("Clip", [e], lo=0.0, hi=6.0, out="Y"))
+    ins = {"X": rnd((n, h, w, c), 21, 0, 1), "Kd": rnd((3, 3, c), 22, -0.5, 0.5), "s": rnd((c,), 23, 0.5, 1.5), "t": rnd((c,), 24, -0.5, 0.5)}
+    check(W.Workload(g, ins), RTOL_F32, FUSED, expect_blocks=1)
+    check(W.Workload(g, ins), RTOL_F32, UNFUSED, expect_blocks=3)
+
+
+@pytest.mark.parametrize("cfg", [(2, 14, 14, 24, 144), (32, 56, 56, 24, 144), (1, 3, 5, 8, 16)])
+@pytest.mark.parametrize("flags", [FUSED, UNFUSED])
+def test_mbconv_block(cfg, flags):
+    n, h, w, cin, cexp = cfg
+    s = check(W.mbconv_block(n, h, w, cin, cexp), RTOL_F32, flags, expect_blocks=3 if flags == FUSED else 9)
+    if flags == FUSED:
+        assert [b["family"] for b in s.g.blocks()] == ["conv1x1", "dwconv", "conv1x1"]
+
+
 @pytest.mark.parametrize("flags,rewrite", [(FUSED, B.REWRITE_NONE), (UNFUSED, B.REWRITE_NONE), (FUSED, B.REWRITE_CANON_MACRO)])
 def test_encoder_small(flags, rewrite):
     wl = W.encoder(layers=2, batch=2, seq=32, hidden=64, heads=4, ffn=128)

@@ -1,0 +1,330 @@
+"""Host-side logic through the C ABI (no GPU needed): exported symbols, mapping types
+(Table 2), the Table 3 reconstruction, graph rewriting (Table 4 with its #FLOPS counts),
+fusion-plan generation (Listing 1 and the worked examples in the text), IR_removable,
+the data-flow-tree linearisation, and the error / state behaviour of the boundary."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2108_13342_b200 import binding as B
+from paper_2108_13342_b200 import workloads as W
+from paper_2108_13342_b200.runtime import build_graph
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+OO, RE, SH, OM, MM = B.ONE_TO_ONE, B.REORGANIZE, B.SHUFFLE, B.ONE_TO_MANY, B.MANY_TO_MANY
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "dnnf.h")).read()
+    declared = set(re.findall(r"DNNF_API\s+[\w\s\*]+?\b(dnnf_\w+)\s*\(", hdr))
+    assert len(declared) >= 25
+    lib = ctypes.CDLL(B.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert declared == set(B.EXPORTS), declared ^ set(B.EXPORTS)
+
+
+# ---- Table 2 and the most-complex-pair rule ------------------------------------------------
+
+def _one_op_graph(op, in_shapes, **attrs):
+    g = B.Graph()
+    ids = [g.add_tensor(f"i{k}", B.F32, s) for k, s in enumerate(in_shapes)]
+    g.add_op(op, ids, **attrs)
+    return g
+
+
+@pytest.mark.parametrize("op,shapes,attrs,expect", [
+    ("Add", [(4, 8), (4, 8)], {}, OO), ("Relu", [(4, 8)], {}, OO), ("Clip", [(4, 8)], {"lo": 0, "hi": 6}, OO),
+    ("Erf", [(4, 8)], {}, OO), ("Exp", [(4, 8)], {}, OO), ("Sigmoid", [(4, 8)], {}, OO), ("Sqrt", [(4, 8)], {}, OO),
+    ("Tanh", [(4, 8)], {}, OO), ("Recip", [(4, 8)], {}, OO), ("Slice", [(4, 8)], {"axis": 1, "start": 0, "end": 4}, OO),
+    ("ScaleShift", [(2, 4, 4, 8), (8,), (8,)], {"axis": -1}, OO),
+    ("Add", [(4, 8), (8,)], {}, OM), ("Mul", [(4, 8), (4, 1)], {}, OM), ("Expand", [(1, 8)], {"shape": (4, 8)}, OM),
+    ("MatMul", [(4, 8), (8, 16)], {}, MM), ("Conv1x1", [(1, 4, 4, 8), (8, 16)], {}, MM), ("Softmax", [(4, 8)], {"axis": -1}, MM),
+    ("ReduceSum", [(4, 8)], {"axis": -1}, MM), ("ReduceMean", [(4, 8)], {"axis": -1}, MM), ("ReduceProd", [(4, 8)], {"axis": -1}, MM),
+    ("LayerNorm", [(4, 8), (8,), (8,)], {"axis": -1}, MM), ("DwConv3x3", [(1, 4, 4, 8), (3, 3, 8)], {}, MM),
+    ("Reshape", [(4, 8)], {"shape": (8, 4)}, RE), ("Flatten", [(2, 4, 8)], {"axis": 1}, RE), ("Squeeze", [(4, 1, 8)], {"axes": (1,)}, RE),
+    ("Unsqueeze", [(4, 8)], {"axes": (0,)}, RE), ("Transpose", [(4, 8)], {"perm": (1, 0)}, SH)])
+def test_operator_mapping_types(op, shapes, attrs, expect):
+    assert _one_op_graph(op, shapes, **attrs).op_mapping(0) == expect
+
+
+# ---- Table 3 ------------------------------------------------------------------------------------
+
+def test_table3_has_23_fusable_cells_and_the_two_named_red_ones():
+    cells = {(a, b): B.mapping_check(a, b) for a in range(5) for b in range(5)}
+    red = [k for k, v in cells.items() if v[1] == B.RED]
+    assert sorted(red) == [(OM, MM), (MM, MM)]          # Expand->Conv and Conv->Conv
+    assert sum(1 for v in cells.values() if v[1] != B.RED) == 23     # one code-generation rule each
+    for t in range(5):                                  # One-to-One takes the partner's type, green, either order
+        assert cells[(OO, t)] == (t, B.GREEN) and cells[(t, OO)] == (t, B.GREEN)
+    for rs in (RE, SH):                                 # Reorganize/Shuffle with One-to-Many / Many-to-Many: profile
+        for strong in (OM, MM):
+            assert cells[(rs, strong)] == (strong, B.YELLOW) and cells[(strong, rs)] == (strong, B.YELLOW)
+    assert cells[(MM, OM)][1] == B.YELLOW               # Conv -> Expand / Resize
+    assert cells[(RE, SH)][1] == B.GREEN and cells[(SH, SH)] == (SH, B.GREEN)
+
+
+# ---- Table 4 -----------------------------------------------------------------------------------
+
+M_, N_ = 6, 10
+MN = M_ * N_
+
+
+def _g(names=("A", "B", "C")):
+    g = W.GraphDesc()
+    for n in names:
+        g.ext(n, (M_, N_))
+    return g
+
+
+def _rewrite(desc, flags=B.REWRITE_DEFAULT):
+    g, ids = build_graph(desc)
+    st = g.rewrite(flags)
+    kinds = sorted(B.OP_NAMES[k] for k, alive in (g.op_kind(i) for i in range(g.op_count())) if alive)
+    return g, st, kinds
+
+
+def test_rewrite_associative_rows():
+    g = _g(("A", "B"))
+    g.mark_output(g.add("Mul", [g.add("Recip", ["A"]), g.add("Recip", [g.add("Mul", ["A", "B"])])]))
+    _, st, kinds = _rewrite(g)
+    assert (st.flops_before, st.flops_after) == (4 * MN, 4 * MN) and kinds == ["Mul", "Recip", "Recip", "Square"]
+
+    g = _g()
+    g.mark_output(g.add("Mul", [g.add("Mul", ["A", g.add("Sqrt", ["B"])]), g.add("Mul", [g.add("Sqrt", ["B"]), "C"])]))
+    _, st, kinds = _rewrite(g)
+    assert (st.flops_before, st.flops_after) == (5 * MN, 2 * MN) and kinds == ["Mul", "Mul"]
+
+    g = _g()
+    g.mark_output(g.add("Mul", [g.add("Mul", [g.add("Abs", ["A"]), "B"]), g.add("Abs", ["C"])]))
+    _, st, kinds = _rewrite(g)
+    assert (st.flops_before, st.flops_after) == (4 * MN, 3 * MN) and kinds == ["Abs", "Mul", "Mul"]
+
+    g = _g()
+    r1 = g.add("ReduceSum", ["B"], axis=-1, keepdims=1); r2 = g.add("ReduceSum", ["B"], axis=-1, keepdims=1)
+    g.mark_output(g.add("Mul", [g.add("Mul", ["A", r1]), g.add("Mul", [r2, "C"])]))
+    _, st, kinds = _rewrite(g)
+    assert (st.flops_before, st.flops_after) == (5 * MN, 3 * MN + M_) and kinds == ["Mul", "Mul", "ReduceSum", "Square"]
+
+
+def test_rewrite_distributive_rows():
+    g = _g()
+    g.mark_output(g.add("Add", [g.add("Mul", ["A", "C"]), g.add("Mul", ["B", "C"])]))
+    _, st, kinds = _rewrite(g)
+    assert (st.flops_before, st.flops_after) == (3 * MN, 2 * MN) and kinds == ["Add", "Mul"]
+
+    g = _g(("A", "B"))
+    g.mark_output(g.add("Add", ["A", g.add("Mul", ["A", "B"])]))
+    _, st, kinds = _rewrite(g)
+    assert (st.flops_before, st.flops_after) == (2 * MN, 2 * MN) and kinds == ["AddC", "Mul"]
+
+    g = _g()
+    s1 = g.add("Add", ["A", "B"]); s2 = g.add("Add", ["A", "B"])
+    g.mark_output(g.add("Sub", [g.add("Square", [s1]), g.add("Mul", [s2, "C"])]))
+    _, st, kinds = _rewrite(g)
+    assert (st.flops_before, st.flops_after) == (5 * MN, 3 * MN) and kinds == ["Add", "Mul", "Sub"]
+
+
+def test_rewrite_commutative_rows():
+    g = _g(("A",))
+    g.mark_output(g.add("ReduceSum", [g.add("BitShift", ["A"], bits=3)], axis=-1, keepdims=1))
+    gg, st, kinds = _rewrite(g)
+    assert (st.flops_before, st.flops_after) == (2 * MN, MN + M_) and kinds == ["BitShift", "ReduceSum"]
+    order = [B.OP_NAMES[gg.op_kind(i)[0]] for i in range(gg.op_count()) if gg.op_kind(i)[1]]
+    assert order == ["ReduceSum", "BitShift"]
+
+    g = _g(("A",))
+    g.mark_output(g.add("ReduceProd", [g.add("Exp", ["A"])], axis=-1, keepdims=1))
+    _, st, kinds = _rewrite(g)
+    assert (st.flops_before, st.flops_after) == (2 * MN, MN + M_) and kinds == ["Exp", "ReduceSum"]
+
+
+def test_rewrite_is_greedy_largest_gain_first_and_reaches_a_fixed_point():
+    # two independent sites: the sqrt pair saves 3mn, the common factor 1mn; both must be gone at the end
+    g = _g(("A", "B", "C", "D"))
+    p = g.add("Mul", [g.add("Mul", ["A", g.add("Sqrt", ["B"])]), g.add("Mul", [g.add("Sqrt", ["B"]), "C"])])
+    q = g.add("Add", [g.add("Mul", ["A", "D"]), g.add("Mul", ["C", "D"])])
+    g.mark_output(g.add("Sub", [p, q]))
+    gg, st, kinds = _rewrite(g)
+    assert st.flops_before == 9 * MN and st.flops_after == 5 * MN and st.rules_applied >= 2
+    st2 = gg.rewrite(B.REWRITE_DEFAULT)
+    assert st2.rules_applied == 0 and st2.flops_after == 5 * MN
+    _, st3, _ = _rewrite(g, B.REWRITE_NONE)
+    assert st3.flops_after == 9 * MN and st3.rules_applied == 0
+
+
+def test_canonicalise_layernorm_flag():
+    wl = W.encoder(layers=1, batch=2, seq=8, hidden=16, heads=2, ffn=32)
+    g, st, kinds = _rewrite(wl.graph, B.REWRITE_CANON_MACRO)
+    assert kinds.count("LayerNorm") == 2 and "ReduceMean" not in kinds and st.ops_after == st.ops_before - 16
+    g2, st2, kinds2 = _rewrite(wl.graph)
+    assert "LayerNorm" not in kinds2 and kinds2.count("Square") == 2 and "Pow" not in kinds2     # Pow(x,2) -> Square only
+
+
+# ---- Listing 1 -----------------------------------------------------------------------------------
+
+def _block_sets(g):
+    return [tuple(b["ops"]) for b in g.blocks()]
+
+
+def test_plan_example_of_section_4_3():
+    # GEMM -> Add -> Conv -> Relu -> Mul -> Sub with equal result sizes: Add is the first seed, the successor pass
+    # gives {Add, Conv, Relu, Mul, Sub} (Many-to-Many), and the predecessor GEMM is refused (Many-to-Many with
+    # Many-to-Many is red).  Add sits in FRONT of Conv, so the plan is made with the literal Listing 1 (planning only).
+    g = W.GraphDesc()
+    g.ext("X", (1, 4, 4, 8)); g.ext("Wg", (8, 8)); g.ext("b", (1, 4, 4, 8)); g.ext("Wc", (8, 8)); g.ext("s", (1, 4, 4, 8)); g.ext("t", (1, 4, 4, 8))
+    y = g.add("MatMul", ["X", "Wg"])
+    y = g.add("Add", [y, "b"]); y = g.add("Conv1x1", [y, "Wc"]); y = g.add("Relu", [y]); y = g.add("Mul", [y, "s"])
+    g.mark_output(g.add("Sub", [y, "t"]))
+    gg, _ = build_graph(g)
+    st = gg.plan(B.PLAN_ALLOW_PROLOGUE)
+    assert st.n_blocks == 2
+    assert sorted(_block_sets(gg), key=len) == [("MatMul",), ("Add", "Conv1x1", "Relu", "Mul", "Sub")]
+    assert [b["mapping"] for b in gg.blocks() if len(b["ops"]) == 5] == ["Many-to-Many"]
+    with pytest.raises(B.DnnfError) as e:          # such a plan is not executable here
+        gg.workspace_size()
+    assert e.value.code == B.ERR_STATE
+    # the executable profile keeps One-to-One operators out of the front of a contraction anchor
+    gg, _ = build_graph(g)
+    gg.plan(B.PLAN_FUSED)
+    assert sorted(_block_sets(gg)) == [("Conv1x1", "Relu", "Mul", "Sub"), ("MatMul", "Add")]
+
+
+def test_chains_the_paper_names_fuse_into_one_block():
+    # MatMul + Reshape + Transpose + Add (GPT-2)
+    g = W.GraphDesc()
+    g.ext("X", (16, 32), "bf16"); g.ext("Wt", (32, 64), "bf16"); g.ext("b", (64,))
+    y = g.add("MatMul", ["X", "Wt"]); y = g.add("Add", [y, "b"]); y = g.add("Reshape", [y], shape=(16, 4, 16))
+    g.mark_output(g.add("Transpose", [y], perm=(1, 0, 2)))
+    gg, _ = build_graph(g)
+    assert gg.plan().n_blocks == 1 and gg.blocks()[0]["family"] == "gemm"
+    # Sub + Pow + ReduceMean + Add + Sqrt (TinyBERT)
+    g = W.GraphDesc()
+    g.ext("X", (8, 64)); g.ext("mu", (8, 1))
+    y = g.add("Sub", ["X", "mu"]); y = g.add("Pow", [y], p=2.0); y = g.add("ReduceMean", [y], axis=-1, keepdims=1)
+    y = g.add("AddC", [y], c=1e-5); g.mark_output(g.add("Sqrt", [y]))
+    gg, _ = build_graph(g)
+    assert gg.plan().n_blocks == 1 and gg.blocks()[0]["family"] == "row"
+    # GEMM + Div + Transpose: Transpose and Div fuse first (Shuffle), GEMM stores through the resulting index map
+    g = W.GraphDesc()
+    g.ext("X", (16, 32), "bf16"); g.ext("Wt", (32, 64), "bf16"); g.ext("d", (16, 64))
+    y = g.add("MatMul", ["X", "Wt"]); y = g.add("Div", [y, "d"]); g.mark_output(g.add("Transpose", [y], perm=(1, 0)))
+    gg, _ = build_graph(g)
+    assert gg.plan().n_blocks == 1 and gg.block_program(0) == "MOV anchor; DIV in0; STORE out0"
+
+
+def test_config_plans_and_strict_table3():
+    cases = [(W.swish_transpose(), 1, 1), (W.masked_softmax(), 1, 2), (W.add_layernorm_gelu(), 1, 1),
+             (W.ffn_block(m=256, hidden=64, ffn=128), 2, 2), (W.mbconv_block(n=1, h=8, w=8), 3, 3)]
+    for wl, fused, strict in cases:
+        g, _ = build_graph(wl.graph)
+        assert g.plan(B.PLAN_FUSED).n_kernels == fused, wl.graph.name
+        g, _ = build_graph(wl.graph)
+        assert g.plan(B.PLAN_STRICT_TABLE3).n_kernels == strict, wl.graph.name
+        g, _ = build_graph(wl.graph)
+        st = g.plan(B.PLAN_UNFUSED)
+        assert st.n_kernels == len(wl.graph.ops) and abs(st.fusion_rate - 1.0) < 1e-9
+
+
+def test_encoder_plan_kernel_counts_and_fusion_rate():
+    wl = W.encoder(layers=2, batch=2, seq=16, hidden=32, heads=2, ffn=64)
+    g, _ = build_graph(wl.graph)
+    g.rewrite(B.REWRITE_CANON_MACRO)
+    st = g.plan()
+    assert st.n_kernels == 2 * 9 and st.n_ops == 2 * 32 and st.irs_bytes_fused < st.irs_bytes_unfused / 3
+    g, _ = build_graph(wl.graph)
+    g.rewrite(B.REWRITE_NONE)
+    st = g.plan()
+    assert st.n_kernels == 2 * 11 and abs(st.fusion_rate - 96 / 22) < 1e-9
+    fams = [b["family"] for b in g.blocks()][:11]
+    assert fams == ["gemm", "gemm", "row", "gemm", "gemm", "row", "row", "gemm", "gemm", "row", "row"]
+
+
+def test_ir_removable_a_tensor_with_an_outside_consumer_is_stored():
+    g = W.GraphDesc()
+    g.ext("X", (8, 32)); g.ext("Y", (8, 32)); g.ext("Wm", (32, 16))
+    t = g.add("Add", ["X", "Y"], out="T")
+    g.mark_output(g.add("Relu", [t], out="R"))
+    g.mark_output(g.add("MatMul", [t, "Wm"], out="S"))         # second consumer: a contraction takes no prologue, other block
+    gg, ids = build_graph(g)
+    st = gg.plan()
+    progs = [gg.block_program(b) for b in range(gg.block_count())]
+    assert st.irs_bytes_fused == 8 * 32 * 4 and any(p.count("STORE") == 2 for p in progs)
+
+
+def test_data_flow_tree_shares_common_subtrees():
+    # Out = Recip(A*B*C) + (A*B)*D : A*B feeds both products and is evaluated once (Section 4.4)
+    g = W.GraphDesc()
+    for n in "ABCD":
+        g.ext(n, (8, 16))
+    t1 = g.add("Mul", ["A", "B"]); t3 = g.add("Recip", [g.add("Mul", [t1, "C"])]); t5 = g.add("Mul", [t1, "D"])
+    g.mark_output(g.add("Add", [t3, t5]))
+    gg, _ = build_graph(g)
+    assert gg.plan().n_blocks == 1
+    prog = gg.block_program(0)
+    assert prog.count("MUL") == 3 and prog.count("in0") == 1 and prog.count("in1") == 1 and "SAVE t0" in prog
+    assert gg.blocks()[0]["mapping"] == "One-to-One"
+
+
+# ---- errors and the state machine ------------------------------------------------------------
+
+def test_errors_leave_the_graph_usable():
+    g = B.Graph()
+    a = g.add_tensor("a", B.F32, (4, 8)); b = g.add_tensor("b", B.F32, (5, 8))
+    with pytest.raises(B.DnnfError) as e:
+        g.add_op("Add", [a, b])
+    assert e.value.code == B.ERR_SHAPE
+    with pytest.raises(B.DnnfError) as e:
+        g.add_op("Transpose", [a], perm=(0, 0))
+    assert e.value.code == B.ERR_SHAPE
+    with pytest.raises(B.DnnfError) as e:
+        g.add_op(999, [a])
+    assert e.value.code == B.ERR_UNSUPPORTED_OP
+    with pytest.raises(B.DnnfError) as e:
+        g.add_op("Relu", [77])
+    assert e.value.code == B.ERR_INVALID_ARG
+    with pytest.raises(B.DnnfError) as e:
+        g.plan()
+    assert e.value.code == B.ERR_STATE                      # nothing added yet
+    (y,) = g.add_op("Relu", [a])
+    with pytest.raises(B.DnnfError) as e:
+        g.plan()
+    assert e.value.code == B.ERR_STATE                      # no output marked
+    with pytest.raises(B.DnnfError) as e:
+        g.mark_output(a)
+    assert e.value.code == B.ERR_INVALID_ARG
+    g.mark_output(y)
+    with pytest.raises(B.DnnfError) as e:
+        g.run(0)
+    assert e.value.code == B.ERR_STATE                      # run before plan
+    assert g.plan().n_blocks == 1
+    with pytest.raises(B.DnnfError) as e:
+        g.add_op("Relu", [y])
+    assert e.value.code == B.ERR_STATE                      # graph is frozen after plan
+    with pytest.raises(B.DnnfError) as e:
+        g.rewrite()
+    assert e.value.code == B.ERR_STATE
+    with pytest.raises(B.DnnfError) as e:
+        g.bind(a, 0)
+    assert e.value.code == B.ERR_INVALID_ARG
+    with pytest.raises(B.DnnfError) as e:
+        g.bind(a, 0x1008)                                   # not 16-byte aligned
+    assert e.value.code == B.ERR_INVALID_ARG
+    with pytest.raises(B.DnnfError) as e:
+        g.run(0)
+    assert e.value.code == B.ERR_UNBOUND and "not bound" in str(e.value)
+    with pytest.raises(B.DnnfError) as e:
+        g.bind_workspace(0x1000, 0)
+    assert e.value.code == B.ERR_WORKSPACE
+
+
+def test_unsupported_block_fails_the_plan_instead_of_falling_back():
+    g = W.GraphDesc()
+    g.ext("A", (4, 8))
+    g.mark_output(g.add("BitShift", ["A"], bits=2))
+    gg, _ = build_graph(g)
+    with pytest.raises(B.DnnfError) as e:
+        gg.plan()
+    assert e.value.code == B.ERR_UNSUPPORTED_OP
