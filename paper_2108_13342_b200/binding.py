@@ -131,7 +131,7 @@ class Graph:
         self.names = {}          # tensor name -> id
 
     def __del__(self):
-        if getattr(self, "h", None):
+        if getattr(self, "h", None) and lib is not None:      # `lib` is gone during interpreter shutdown
             lib.dnnf_graph_destroy(self.h)
             self.h = None
 

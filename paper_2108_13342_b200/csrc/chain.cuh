@@ -9,6 +9,7 @@
 #include <cuda_runtime.h>
 #include <math_constants.h>
 
+#include "launch_util.h"
 #include "microop.h"
 #include "static_programs.h"
 
@@ -262,8 +263,14 @@ __device__ __forceinline__ void store_vec4(const TensorArg& a, uint32_t off, con
   if (F32 || a.dtype == 0) {
     *reinterpret_cast<float4*>(reinterpret_cast<float*>(a.ptr) + off) = make_float4(v[0], v[1], v[2], v[3]);
   } else {
-    uint32_t lo = (uint32_t)float_to_bf16_bits(v[0], exact) | ((uint32_t)float_to_bf16_bits(v[1], exact) << 16);
-    uint32_t hi = (uint32_t)float_to_bf16_bits(v[2], exact) | ((uint32_t)float_to_bf16_bits(v[3], exact) << 16);
+    uint32_t lo, hi;
+    if (exact) {
+      lo = (uint32_t)float_to_bf16_bits(v[0], true) | ((uint32_t)float_to_bf16_bits(v[1], true) << 16);
+      hi = (uint32_t)float_to_bf16_bits(v[2], true) | ((uint32_t)float_to_bf16_bits(v[3], true) << 16);
+    } else {                                   // one packed conversion per pair (full-rate pipe)
+      __nv_bfloat162 p0 = __floats2bfloat162_rn(v[0], v[1]), p1 = __floats2bfloat162_rn(v[2], v[3]);
+      lo = *reinterpret_cast<uint32_t*>(&p0); hi = *reinterpret_cast<uint32_t*>(&p1);
+    }
     *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(a.ptr) + off) = make_uint2(lo, hi);
   }
 }

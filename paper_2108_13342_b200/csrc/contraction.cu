@@ -22,6 +22,11 @@ bool tc_gemm_eligible(const GemmParams& gp);
 bool tc_gemm_prepare(Launch& L, std::string& err);                  // encode tensor maps after pointers are known
 int tc_gemm_launch(const Launch& L, cudaStream_t st);
 void tc_gemm_plan(Launch& L);                                        // choose tiles / grid
+size_t tc2_blob_bytes();
+bool tc2_gemm_eligible(const GemmParams& gp);
+void tc2_gemm_plan(Launch& L);
+bool tc2_gemm_prepare(Launch& L, std::string& err);
+int tc2_gemm_launch(const Launch& L, cudaStream_t st);
 bool conv1x1_direct_eligible(const GemmParams& gp);
 void conv1x1_direct_plan(Launch& L);
 int conv1x1_direct_launch(const Launch& L, cudaStream_t st);
@@ -97,6 +102,8 @@ __device__ __forceinline__ uint32_t digits_offset(const GemmParams& p, const Ten
 __global__ void __launch_bounds__(256) gemm_fallback_kernel(const __grid_constant__ GemmParams p) {
   __shared__ float As[FB_K][FB_T + 1];
   __shared__ float Bs[FB_K][FB_T + 1];
+  pdl_launch_dependents();
+  pdl_wait();
   const int tile_n = blockIdx.x % p.tiles_n, tile_m = blockIdx.x / p.tiles_n;
   const int batch = blockIdx.y;
   const int b0 = batch % p.batch_ext[0], b1 = batch / p.batch_ext[0];
@@ -231,7 +238,7 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
 
   Launch& L = out.launch;
   L = Launch{};
-  L.blob.assign(sizeof(GemmParams) + sizeof(GemmTcParams), 0);
+  L.blob.assign(sizeof(GemmParams) + sizeof(GemmTcParams) + tc2_blob_bytes(), 0);
   GemmParams& gp = gp_of(L);
 
   // ---- operands ----------------------------------------------------------------
@@ -389,6 +396,10 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
     for (int d = 0; d < kMaxDims; ++d) a.stride[d] = d < nd ? (int32_t)dims[nd - 1 - d].coef[ai] : 0;
     if (g.tensors[e.tensor].numel() >= (1ll << 31)) return false;
     bool is_out = ai >= cx.ins.size();
+    // mode 1: the operand does not depend on the row or the batch (a bias vector)
+    bool row_invariant = !is_out;
+    for (int d = n_nd; d < nd; ++d) if (a.stride[d] != 0) row_invariant = false;
+    a.mode = row_invariant ? 1 : 0;
     if (a.stride[0] != 1 && !(a.stride[0] == 0 && !is_out)) vec_ok = false;
     if (a.stride[0] == 1) { if (a.base % 8) vec_ok = false; for (int d = 1; d < nd; ++d) if (a.stride[d] % 8) vec_ok = false; }
     return true;
@@ -408,7 +419,9 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
   L.flops = 2ll * gp.M * gp.N * gp.K * nbatch;
   L.family = A.kind == DNNF_OP_CONV1X1 ? DNNF_FAMILY_CONV1X1 : DNNF_FAMILY_GEMM;
 
-  if (tc_gemm_eligible(gp)) {
+  if (tc2_gemm_eligible(gp)) {
+    tc2_gemm_plan(L);
+  } else if (tc_gemm_eligible(gp)) {
     L.variant = 1;
     tc_gemm_plan(L);
   } else if (A.kind == DNNF_OP_CONV1X1 && conv1x1_direct_eligible(gp)) {
@@ -429,7 +442,12 @@ void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vecto
   gp.A.ptr = ip[0]; gp.B.ptr = ip[1];
   for (int i = 0; i < gp.n_in; ++i) gp.in[i].ptr = ip[2 + i];
   for (int i = 0; i < gp.n_out; ++i) gp.out[i].ptr = op[i];
+  if (L.variant == 3) changed = changed || !L.tc_ready || gp.out[0].ptr != L.last_out || (gp.n_in > 0 && gp.in[0].ptr != L.last_in0) || (gp.n_in > 1 && gp.in[1].ptr != L.last_in1);
   if (L.variant == 1 && (changed || !L.tc_ready)) { if (tc_gemm_prepare(L, err)) L.tc_ready = true; }
+  if (L.variant == 3 && changed) {
+    if (tc2_gemm_prepare(L, err)) L.tc_ready = true;
+    L.last_out = gp.out[0].ptr; L.last_in0 = gp.n_in > 0 ? gp.in[0].ptr : nullptr; L.last_in1 = gp.n_in > 1 ? gp.in[1].ptr : nullptr;
+  }
 }
 
 int launch_contraction(const Launch& L, void* status_words, int block_index, cudaStream_t st, std::string& err) {
@@ -438,6 +456,13 @@ int launch_contraction(const Launch& L, void* status_words, int block_index, cud
   GemmParams gp = gp_of(L);
   gp.status = reinterpret_cast<int32_t*>(status_words);
   gp.block_index = block_index;
+  if (L.variant == 3) {
+    Launch& M = const_cast<Launch&>(L);
+    gp_of(M).status = gp.status; gp_of(M).block_index = block_index;
+    int rc = tc2_gemm_launch(L, st);
+    if (rc) err = "tensor-core pair GEMM launch failed";
+    return rc;
+  }
   if (L.variant == 1) {
     Launch& M = const_cast<Launch&>(L);
     gp_of(M).status = gp.status; gp_of(M).block_index = block_index;
@@ -446,7 +471,7 @@ int launch_contraction(const Launch& L, void* status_words, int block_index, cud
     return rc;
   }
   dim3 grid(L.grid, gp.batch_ext[0] * gp.batch_ext[1]);
-  gemm_fallback_kernel<<<grid, 256, 0, st>>>(gp);
+  launch_pdl(gemm_fallback_kernel, grid, 256, 0, st, gp);
   if (cudaGetLastError() != cudaSuccess) { err = "fallback GEMM launch failed"; return 1; }
   return 0;
 }

@@ -57,6 +57,8 @@ struct PwIO {
 template <int NPT, int LPP, class SP>
 __global__ void __launch_bounds__(256) conv1x1_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ float wsm[];                 // [K][N]
+  pdl_launch_dependents();
+  pdl_wait();
   const int K = p.K, N = p.N;
   const float* W = reinterpret_cast<const float*>(p.B.ptr) + p.B.base;
   for (int i = threadIdx.x * 4; i < K * N; i += 256 * 4)
@@ -152,7 +154,7 @@ struct PwLauncher {
   template <class SP> void run() {
     static bool attr = false;
     if (!attr) { cudaFuncSetAttribute(conv1x1_kernel<NPT, LPP, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); attr = true; }
-    conv1x1_kernel<NPT, LPP, SP><<<L.grid, 256, L.smem, st>>>(gp_of(L));
+    launch_pdl(conv1x1_kernel<NPT, LPP, SP>, L.grid, 256, L.smem, st, gp_of(L));
   }
 };
 template <int NPT, int LPP, bool kStatic>
@@ -226,6 +228,8 @@ __device__ __forceinline__ void fma4(float (&acc)[4], const float4& x, const flo
 // HS rows per thread: the grid covers (n, h-strip, w, c4)
 template <class SP>
 __global__ void __launch_bounds__(256) dwconv_kernel(const __grid_constant__ DwParams p, int HS) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int C4 = p.C / 4;
   const int strips = (p.H + HS - 1) / HS;
   int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
@@ -265,7 +269,7 @@ static const DwParams& dw_of(const Launch& L) { return *reinterpret_cast<const D
 
 struct DwLauncher {
   const Launch& L; cudaStream_t st; int hs;
-  template <class SP> void run() { dwconv_kernel<SP><<<L.grid, 256, 0, st>>>(dw_of(L), hs); }
+  template <class SP> void run() { launch_pdl(dwconv_kernel<SP>, L.grid, 256, 0, st, dw_of(L), hs); }
 };
 
 int dwconv_launch(const Launch& L, cudaStream_t st) {

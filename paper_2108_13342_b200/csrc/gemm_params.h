@@ -41,6 +41,7 @@ struct GemmTcParams {
   int32_t k_tiles;
   int32_t bn;                      // N tile
   int32_t persistent_tiles;        // total output tiles
+  int32_t debug;                   // ablation switches (development only)
 };
 
 }  // namespace dnnf

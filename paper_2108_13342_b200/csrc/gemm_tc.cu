@@ -17,6 +17,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cstdlib>
 #include <mutex>
 
 #include "chain.cuh"
@@ -136,6 +137,14 @@ struct TcEpiIO {
     const uint32_t mine = row_in[idx];
     const bool vec = p.vec_ok && (int)nn + 4 <= p.N;
     const uint32_t noff = vec ? n_offset(a, nn) : 0u;
+    if (vec && a.mode == 1) {                   // the same for every row (a bias): load once
+      float x[4];
+      if (a.stride[0] == 0) { x[0] = x[1] = x[2] = x[3] = load_scalar<false>(a, mine + noff); }
+      else load_vec4<false>(a, mine + noff, x);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { dst[i * 4] = x[0]; dst[i * 4 + 1] = x[1]; dst[i * 4 + 2] = x[2]; dst[i * 4 + 3] = x[3]; }
+      return;
+    }
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int r = (lane >> 3) + 4 * i;
@@ -188,6 +197,13 @@ __device__ __forceinline__ uint32_t tc_digits(const GemmParams& p, const TensorA
   return off;
 }
 
+#ifdef DNNF_TRACE
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define TRACE(slot) do { if (blockIdx.x == 0 && p.status) reinterpret_cast<unsigned long long*>(p.status)[4 + (slot)] = gtime(); } while (0)
+#else
+#define TRACE(slot) do {} while (0)
+#endif
+
 // ---- the kernel ---------------------------------------------------------------------------------
 template <class SP>
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -207,6 +223,8 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
   uint32_t* stage_area = tmem_slot + 8;          // TC_EPI_WARPS x kStageWords
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_launch_dependents();
+  if (threadIdx.x == 0) TRACE(0);
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(&tfull_bar[s], 1); mbar_init(&tempty_bar[s], TC_EPI_WARPS); }
@@ -221,6 +239,9 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) TRACE(1);
+  // set-up above overlaps the previous kernel's tail; nothing below may touch global memory earlier
+  pdl_wait();
 
   const int tiles_mn = p.tiles_m * p.tiles_n;
   const int total_tiles = q.persistent_tiles;
@@ -244,6 +265,7 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
           if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + (size_t)s * stage_bytes;
           uint8_t* sb = sa + a_bytes;
+          if (it == 0) TRACE(2);
           mbar_expect_tx(&full_bar[s], stage_bytes);
           tma_load_4d(sa, &tmA, &full_bar[s], kt * TC_BK, tm * TC_BM, ab0, ab1);
           if (q.b_kmajor) {
@@ -273,6 +295,7 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
           const int s = it % stages;
           const uint32_t ph = (it / stages) & 1;
           if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
+          if (it == 0) TRACE(3);
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
           const uint32_t sb = sa + a_bytes;
@@ -285,6 +308,7 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
           tc_commit(&empty_bar[s]);          // frees the smem stage once these MMAs have read it
         }
         if (ok) tc_commit(&tfull_bar[acc]);  // accumulator complete
+        if (tcount == 0) TRACE(4);
       }
     }
   } else {
@@ -298,6 +322,7 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
       const int acc = tcount & 1;
       const uint32_t aph = (tcount >> 1) & 1;
       if (!mbar_wait(&tfull_bar[acc], aph, abort_flag)) { ok = false; break; }
+      if (tcount == 0 && warp == 2 && lane == 0) TRACE(5);
       tc_fence_after();
       TcEpiIO io{p};
       uint32_t* stage = stage_area + (warp - 2) * kStageWords;
@@ -324,10 +349,14 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
       for (int c = c_begin; c < c_end; c += 32) {
         const int n0 = tn * BN + c;
         if (n0 >= p.N) break;                  // uniform across the warp
+        if (q.debug & 4) continue;
         uint32_t raw[32];
+        if (tcount == 0 && warp == 2 && lane == 0 && c == c_begin) TRACE(8);
         tc_ld32_issue(t_row + c, raw);
         tc_ld_wait();
+        if (tcount == 0 && warp == 2 && lane == 0 && c == c_begin) TRACE(9);
         // transpose: lane = row  ->  lane = (row group, 4-column piece)
+        if (!(q.debug & 2)) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = raw[j];
         __syncwarp();
@@ -336,11 +365,15 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
 #pragma unroll
           for (int e = 0; e < 4; ++e) io.accv[i * 4 + e] = __uint_as_float(stage[((lane >> 3) + 4 * i) * 33 + (lane & 7) * 4 + e]);
         __syncwarp();
+        }
+        if (tcount == 0 && warp == 2 && lane == 0 && c == c_begin) TRACE(10);
         io.n0 = (uint32_t)n0;
-        run_program<32, SP, true>(p.prog, io);
+        if (!(q.debug & 1)) run_program<32, SP, true>(p.prog, io);
+        if (tcount == 0 && warp == 2 && lane == 0 && c == c_begin) TRACE(11);
       }
       tc_fence_before();
       __syncwarp();
+      if (tcount == 0 && warp == 2 && lane == 0) TRACE(6);
       if (lane == 0) mbar_arrive(&tempty_bar[acc]);
     }
   }
@@ -349,6 +382,7 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
   __syncwarp();
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) TRACE(7);
   if (*abort_flag) {
     if (threadIdx.x == 0 && p.status) { atomicExch(&p.status[0], DNNF_ERR_TIMEOUT); atomicExch(&p.status[1], p.block_index); }
     // give copies that are still in flight time to land before shared memory is released
@@ -424,6 +458,7 @@ void tc_gemm_plan(Launch& L) {
   L.smem = (size_t)stages * stage_bytes + kSmemFixed;
   L.variant = 1;
   L.static_id = StaticSet<EpiStatic>::find(gp.prog);
+  tc.debug = getenv("DNNF_GEMM_DEBUG") ? atoi(getenv("DNNF_GEMM_DEBUG")) : 0;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -483,7 +518,7 @@ struct TcLauncher {
   template <class SP> void run() {
     static bool attr_set = false;     // per instantiation
     if (!attr_set) { cudaFuncSetAttribute(gemm_tc_kernel<SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax); attr_set = true; }
-    gemm_tc_kernel<SP><<<L.grid, TC_THREADS, L.smem, st>>>(gp_of(L), tc_of(L), tc_of(L).tmA, tc_of(L).tmB, stages);
+    launch_pdl(gemm_tc_kernel<SP>, L.grid, TC_THREADS, L.smem, st, gp_of(L), tc_of(L), tc_of(L).tmA, tc_of(L).tmB, stages);
   }
 };
 

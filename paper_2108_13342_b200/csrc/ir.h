@@ -60,6 +60,7 @@ struct Launch {
   int family = DNNF_FAMILY_ALIAS;
   int variant = 0;
   bool tc_ready = false;      // tensor maps encoded for the currently bound pointers
+  void *last_out = nullptr, *last_in0 = nullptr, *last_in1 = nullptr;
   int static_id = 0;          // compile-time program table the block runs on (0: interpreted)
   int grid = 0, threads = 0;
   size_t smem = 0;

@@ -74,6 +74,7 @@ struct EwIO {
 // contiguous one), so that every index below is a compile-time constant.
 template <int V, int U, class SP, bool F32>
 __global__ void __launch_bounds__(256) ew_kernel(const __grid_constant__ EwParams p) {
+  pdl_launch_dependents();
   EwIO<V, U, F32> io{p};
   const uint32_t nvec = (uint32_t)(p.total / V);
 #pragma unroll
@@ -97,6 +98,7 @@ __global__ void __launch_bounds__(256) ew_kernel(const __grid_constant__ EwParam
       }
     }
   }
+  pdl_wait();
   run_program<V * U, SP>(p.prog, io);
 }
 
@@ -176,6 +178,7 @@ struct TrIO {
 template <int V, class SP, bool F32>
 __global__ void __launch_bounds__(256) tr_kernel(const __grid_constant__ EwParams p) {
   extern __shared__ float smem[];
+  pdl_launch_dependents();
   constexpr int K = 4;
   TrIO<V, K, F32> io{p, smem};
   uint32_t b = blockIdx.x;
@@ -193,6 +196,7 @@ __global__ void __launch_bounds__(256) tr_kernel(const __grid_constant__ EwParam
   io.t0 = tile_t * TT; io.i0 = tile_i * TI;
   const uint32_t ext_t = p.it.extent[1], ext_i = p.it.extent[0];
 
+  pdl_wait();
   // Phase 1: staged inputs, lanes along t (their contiguous dim).
   for (int k = 0; k < p.n_in; ++k) {
     const TensorArg& a = p.in[k];
@@ -255,8 +259,8 @@ template <bool F32>
 struct EwLauncher {
   const Launch& L; cudaStream_t st;
   template <class SP> void run() {
-    if (L.family == DNNF_FAMILY_ELEMENTWISE) ew_kernel<4, 2, SP, F32><<<L.grid, 256, 0, st>>>(L.ew);
-    else tr_kernel<4, SP, F32><<<L.grid, 256, L.smem, st>>>(L.ew);
+    if (L.family == DNNF_FAMILY_ELEMENTWISE) launch_pdl(ew_kernel<4, 2, SP, F32>, L.grid, 256, 0, st, L.ew);
+    else launch_pdl(tr_kernel<4, SP, F32>, L.grid, 256, L.smem, st, L.ew);
   }
 };
 
@@ -277,8 +281,8 @@ int launch_ew(const Launch& L, cudaStream_t st) {
       if (!(L.static_id > 0 && StaticSet<EwStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
     }
   } else {
-    if (L.family == DNNF_FAMILY_ELEMENTWISE) ew_kernel<1, 4, DynProg, false><<<L.grid, 256, 0, st>>>(p);
-    else tr_kernel<1, DynProg, false><<<L.grid, 256, L.smem, st>>>(p);
+    if (L.family == DNNF_FAMILY_ELEMENTWISE) launch_pdl(ew_kernel<1, 4, DynProg, false>, L.grid, 256, 0, st, p);
+    else launch_pdl(tr_kernel<1, DynProg, false>, L.grid, 256, L.smem, st, p);
   }
   return cudaGetLastError() == cudaSuccess ? 0 : 1;
 }

@@ -135,6 +135,7 @@ template <int V, int NV, int WPR, int RPW, class SP, bool F32>
 __global__ void __launch_bounds__(WPR > 1 ? 32 * WPR : 32 * kRowWarpsPerCta)
 row_kernel(const __grid_constant__ RowParams p) {
   __shared__ float xchg[WPR > 1 ? WPR : 1];
+  pdl_launch_dependents();
   RowIO<V, NV, WPR, RPW, F32> io{p};
   io.xchg = xchg;
   uint32_t row0;
@@ -155,6 +156,7 @@ row_kernel(const __grid_constant__ RowParams p) {
       }
     }
   }
+  pdl_wait();
   run_program<V * NV * RPW, SP>(p.prog, io);
 }
 
@@ -162,7 +164,7 @@ template <int V, int NV, int WPR, int RPW, bool F32>
 struct RowLauncher {
   const Launch& L; cudaStream_t st;
   template <class SP> void run() {
-    row_kernel<V, NV, WPR, RPW, SP, F32><<<L.grid, L.threads, 0, st>>>(L.row);
+    launch_pdl(row_kernel<V, NV, WPR, RPW, SP, F32>, L.grid, L.threads, 0, st, L.row);
   }
 };
 

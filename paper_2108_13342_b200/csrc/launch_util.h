@@ -1,0 +1,26 @@
+// Kernel launch with programmatic dependent launch: a block's kernel may start while the
+// previous kernel on the stream is still draining, and blocks at pdl_wait() until that kernel
+// has completed and its writes are visible.  Every kernel of this library calls pdl_wait()
+// before its first global-memory access, so the result equals plain stream order; only the
+// launch latency and the prologue (index set-up, barrier and tensor-memory set-up) overlap
+// the predecessor's tail.  Works in plain streams and under stream capture.
+#pragma once
+#include <cuda_runtime.h>
+
+namespace dnnf {
+
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+}
+
+}  // namespace dnnf

@@ -38,7 +38,7 @@ def _graph_of(torch, dev, fn):
     return g
 
 
-def measure_workload(torch, dev, wl, pk, flags, copies, iters=20, rewrite=B.REWRITE_NONE):
+def measure_workload(torch, dev, wl, pk, flags, copies, iters=20, rewrite=B.REWRITE_NONE, per_block_limit=16):
     """`copies` sessions with distinct buffers, run round-robin so that every launch
     sees cold data when copies * footprint exceeds L2."""
     sess = [Session(wl, plan_flags=flags, rewrite_flags=rewrite, device=dev) for _ in range(copies)]
@@ -61,7 +61,7 @@ def measure_workload(torch, dev, wl, pk, flags, copies, iters=20, rewrite=B.REWR
     cg = _graph_of(torch, dev, all_on)
     t_graph = _time_region(torch, dev, cg.replay, iters) / copies
     per_block = []
-    if nb <= 16:
+    if nb <= per_block_limit:
         for b in range(nb):
             if blocks[b]["family"] == "alias":
                 continue
@@ -108,4 +108,36 @@ def per_config(dev, pk, only=None):
         except Exception as e:      # report, never hide
             out[name] = {"error": repr(e)}
         torch.cuda.empty_cache()
+    return out
+
+
+def encoder_report(dev, pk, layers=12):
+    """Whole-graph workload: the 12-layer encoder as primitive operators, through rewriting,
+    planning and fused execution; compared with one kernel per operator."""
+    import torch
+    wl = W.encoder(layers=layers)
+    out = {}
+    for name, flags, rw in [("fused", B.PLAN_FUSED, B.REWRITE_DEFAULT), ("fused+layernorm-canon", B.PLAN_FUSED, B.REWRITE_CANON_MACRO),
+                            ("unfused", B.PLAN_UNFUSED, B.REWRITE_NONE)]:
+        r = measure_workload(torch, dev, wl, pk, flags, 1, iters=10, rewrite=rw, per_block_limit=0)
+        out[name] = r
+        torch.cuda.empty_cache()
+    # per-block table for one layer of the canonicalised plan
+    s = Session(wl, rewrite_flags=B.REWRITE_CANON_MACRO, device=dev)
+    blocks = s.g.blocks()
+    per = []
+    nb_layer = max(1, s.g.block_count() // layers)
+    for b in range(nb_layer, 2 * nb_layer if layers > 1 else nb_layer):
+        if blocks[b]["family"] == "alias":
+            continue
+        cg = _graph_of(torch, dev, lambda sp, b=b: s.g.run_block(b, sp))
+        cg.replay()
+        t = _time_region(torch, dev, cg.replay, 50)
+        by, fl = blocks[b]["bytes"], blocks[b]["flops"]
+        roof = max(by / (pk["hbm_gbs"] * 1e3), fl / (pk["bf16_tflops"] * 1e6))
+        per.append({"ops": "+".join(blocks[b]["ops"][:10]), "family": blocks[b]["family"], "us_warm_l2": round(t, 3), "bytes": by,
+                    "flops": fl, "roofline_us": round(roof, 3), "frac_of_roofline": round(roof / t, 3)})
+    out["layer_blocks_canon_plan"] = per
+    out["speedup_fused_vs_unfused_graph"] = round(out["unfused"]["us_cuda_graph"] / out["fused+layernorm-canon"]["us_cuda_graph"], 2)
+    out["speedup_fused_vs_unfused_plain"] = round(out["unfused"]["us_plain_launches"] / out["fused+layernorm-canon"]["us_plain_launches"], 2)
     return out
