@@ -27,7 +27,7 @@
 namespace dnnf {
 
 constexpr int TC_BM = 128, TC_BK = 64, TC_EPI_WARPS = 8, TC_THREADS = 64 + 32 * TC_EPI_WARPS;
-constexpr uint32_t kSpinLimit = 1u << 27;
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // 1 s
 constexpr int kSmemMax = 227 * 1024;                       // dynamic shared memory per CTA
 constexpr int kStageWords = 32 * 33;                       // per epilogue warp: 32 rows x (32 + 1 pad) words
 constexpr int kSmemFixed = 1024 + 256 + TC_EPI_WARPS * kStageWords * 4;   // alignment slack, barriers, staging
@@ -52,13 +52,18 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false when the bound ran out or another role already gave up.
+__device__ __forceinline__ unsigned long long wall_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+// Bounded wait: gives up after kWaitLimitNs of wall-clock time (or as soon as another role of the
+// CTA gave up), sets the CTA's abort flag and returns false.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (mbar_try(bar, parity)) return true;
-    if ((it & 1023u) == 1023u && *abort_flag) return false;
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = wall_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i) if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (wall_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
   }
-  *abort_flag = 1;
-  return false;
 }
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* tm, uint64_t* bar, int c0, int c1, int c2, int c3) {
   asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
@@ -137,10 +142,16 @@ struct TcEpiIO {
     const uint32_t mine = row_in[idx];
     const bool vec = p.vec_ok && (int)nn + 4 <= p.N;
     const uint32_t noff = vec ? n_offset(a, nn) : 0u;
-    if (vec && a.mode == 1) {                   // the same for every row (a bias): load once
+    if (a.mode == 1) {                          // the same for every row (a bias): load once.
+      // (a.mode is uniform over the warp: no lane may leave before the shuffles of the general path)
       float x[4];
-      if (a.stride[0] == 0) { x[0] = x[1] = x[2] = x[3] = load_scalar<false>(a, mine + noff); }
-      else load_vec4<false>(a, mine + noff, x);
+      if (vec) {
+        if (a.stride[0] == 0) { x[0] = x[1] = x[2] = x[3] = load_scalar<false>(a, mine + noff); }
+        else load_vec4<false>(a, mine + noff, x);
+      } else {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) x[v] = ((int)nn + v < p.N) ? load_scalar<false>(a, mine + n_offset(a, nn + v)) : 0.0f;
+      }
 #pragma unroll
       for (int i = 0; i < 8; ++i) { dst[i * 4] = x[0]; dst[i * 4 + 1] = x[1]; dst[i * 4 + 2] = x[2]; dst[i * 4 + 3] = x[3]; }
       return;

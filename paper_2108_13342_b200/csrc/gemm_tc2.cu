@@ -31,8 +31,14 @@ namespace dnnf {
 
 namespace tc2 {
 
+#ifdef DNNF_TRACE
+#define T2ACC(slot, v) do { if (blockIdx.x == 0 && p.status) atomicAdd(reinterpret_cast<unsigned long long*>(p.status) + 4 + (slot), (unsigned long long)(v)); } while (0)
+#else
+#define T2ACC(slot, v) do {} while (0)
+#endif
+
 constexpr int BM = 128, BK = 64, EPI_WARPS = 8, THREADS = 64 + 32 * EPI_WARPS;
-constexpr uint32_t kSpin = 1u << 27;
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // 1 s
 constexpr int kSmemMax = 227 * 1024;
 constexpr int kChunkBytes = 32 * 128;                        // 32 rows x 64 bf16
 constexpr int kBiasFloats = 128;                             // per warp, per row-invariant operand
@@ -78,13 +84,18 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
                : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ unsigned long long wall_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+// Bounded wait: gives up after kWaitLimitNs of wall-clock time (or as soon as another role of the
+// CTA gave up), sets the CTA's abort flag and returns false.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kSpin; ++it) {
-    if (mbar_try(bar, parity)) return true;
-    if ((it & 1023u) == 1023u && *abort_flag) return false;
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = wall_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i) if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (wall_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
   }
-  *abort_flag = 1;
-  return false;
 }
 // Operand load of a CTA pair: the bytes land in THIS CTA's shared memory, the completion is
 // counted on the LEADER's barrier (cluster address), so the MMA thread waits on one barrier only.
@@ -226,6 +237,7 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();
+  const long long t_begin = clock64();
 
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int total = q.total_tiles, k_tiles = q.k_tiles, tiles_n = q.tiles_n;
@@ -241,7 +253,7 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
         for (int kt = 0; kt < k_tiles; ++kt, ++it) {
           const int s = it % stages;
           const uint32_t ph = (it / stages) & 1;
-          if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_flag)) { ok = false; break; }
+          { long long t0 = clock64(); if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_flag)) { ok = false; break; } T2ACC(0, clock64() - t0); }
           uint8_t* sa = smem + (size_t)s * stage_bytes;
           uint8_t* sb = sa + a_bytes;
           const uint32_t lbar = mapa(smem_u32(&full_bar[s]), 0);
@@ -266,13 +278,13 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
         for (int tile = pair; tile < total && ok; tile += n_pairs, ++tcount) {
           const int acc = tcount & 1;
           const uint32_t aph = (tcount >> 1) & 1;
-          if (!mbar_wait(&tempty_bar[acc], aph ^ 1, abort_flag)) { ok = false; break; }
+          { long long t0 = clock64(); if (!mbar_wait(&tempty_bar[acc], aph ^ 1, abort_flag)) { ok = false; break; } T2ACC(1, clock64() - t0); }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
           for (int kt = 0; kt < k_tiles; ++kt, ++it) {
             const int s = it % stages;
             const uint32_t ph = (it / stages) & 1;
-            if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }   // own bytes landed and the peer reported its own
+            { long long t0 = clock64(); if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; } T2ACC(2, clock64() - t0); T2ACC(3, 1); }
             tc_fence_after();
             const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
             const uint32_t sb = sa + a_bytes;
@@ -326,7 +338,7 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
       __syncwarp();
       const int acc = tcount & 1;
       const uint32_t aph = (tcount >> 1) & 1;
-      if (!mbar_wait(&tfull_bar[acc], aph, abort_flag)) { ok = false; break; }
+      { long long t0 = clock64(); if (!mbar_wait(&tfull_bar[acc], aph, abort_flag)) { ok = false; break; } if (warp == 2 && lane == 0) T2ACC(4, clock64() - t0); }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(sub * 32) << 16) + (uint32_t)(acc * BN + half * cols_per_warp);
       for (int c = 0; c < chunks && ok; ++c, ++ccount) {
@@ -373,6 +385,7 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
   __syncwarp();
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) T2ACC(5, clock64() - t_begin);
   cluster_sync();                              // the peer may still be signalling our barriers / reading our shared memory
   if (*abort_flag) {
     if (threadIdx.x == 0 && p.status) { atomicExch(&p.status[0], DNNF_ERR_TIMEOUT); atomicExch(&p.status[1], p.block_index); }

@@ -36,7 +36,35 @@ def test_ffn_block(cfg, flags):
     s = check(W.ffn_block(m, hidden, ffn), RTOL_BF16, flags, expect_blocks=2 if flags == FUSED else 6)
     if flags == FUSED:
         assert [b["family"] for b in s.g.blocks()] == ["gemm", "gemm"]
-        assert all(b["variant"] == 1 for b in s.g.blocks()), "expected the tensor-core kernel"
+        assert all(b["variant"] in (1, 3) for b in s.g.blocks()), "expected a tensor-core kernel"
+
+
+@pytest.mark.parametrize("mnk", [(256, 128, 64), (300, 200, 72), (1000, 328, 264), (257, 136, 8), (512, 2304, 768)])
+@pytest.mark.parametrize("kmajor_b", [False, True])
+@pytest.mark.parametrize("epi", ["none", "bias_gelu", "bias_residual"])
+def test_pair_gemm_shapes_and_epilogues(mnk, kmajor_b, epi):
+    """The CTA-pair kernel (M >= 256, N >= 128): ragged edges in M, N and K, both operand layouts for B."""
+    m, n, k = mnk
+    g = graph()
+    g.ext("A", (m, k), "bf16")
+    ins = {"A": _bf(rnd((m, k), 31, -1, 1))}
+    if kmajor_b:
+        g.ext("Bt", (n, k), "bf16"); ins["Bt"] = _bf(rnd((n, k), 32, -0.1, 0.1))
+        b = g.add("Transpose", ["Bt"], perm=(1, 0))
+    else:
+        g.ext("Bm", (k, n), "bf16"); ins["Bm"] = _bf(rnd((k, n), 32, -0.1, 0.1)); b = "Bm"
+    t = g.add("MatMul", ["A", b])
+    if epi != "none":
+        g.ext("bias", (n,), "f32"); ins["bias"] = rnd((n,), 33, -0.5, 0.5)
+        t = g.add("Add", [t, "bias"])
+    if epi == "bias_gelu":
+        t = g.add("Gelu", [t], approx="tanh")
+    if epi == "bias_residual":
+        g.ext("R", (m, n), "bf16"); ins["R"] = _bf(rnd((m, n), 34, -1, 1))
+        t = g.add("Add", [t, "R"])
+    g.mark_output(t)
+    s = check(W.Workload(g, ins), RTOL_BF16, FUSED, expect_blocks=1)
+    assert s.g.blocks()[0]["variant"] == 3, s.g.blocks()
 
 
 def test_batched_matmul_with_transposed_and_strided_operands():
