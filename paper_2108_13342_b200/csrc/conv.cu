@@ -1,7 +1,7 @@
 // fp32 NHWC convolution anchors on CUDA cores, each with the block's epilogue program:
-//  * pointwise (1x1) convolution, pixel-stationary: a lane keeps one pixel's partial sums
-//    for a slice of the output channels in registers, the [Cin x Cout] weights sit in
-//    shared memory and are read as broadcast 128-bit words;
+//  * pointwise (1x1) convolution as a register-tiled FMA GEMM for tall-skinny shapes: weights
+//    resident in shared memory, pixel tile streamed through shared memory, 8 pixels x TN
+//    channels per thread;
 //  * depthwise 3x3, stride 1, zero padding 1: a thread owns one (image, column, 4-channel
 //    group) and walks down the rows with a rolling 3x3 window, so every input value is
 //    loaded three times from L1/L2 instead of nine.
@@ -18,23 +18,30 @@ namespace dnnf {
 
 // ---------------------------------------------------------------------------
 // Pointwise convolution: [P x K] * [K x N], fp32, rows contiguous.
-// LPP lanes share a pixel; lane q of them owns float4 columns f = j*LPP + q, j < NPT.
+// Register-tiled FMA kernel for tall-skinny problems (K, N small): a CTA owns BM = PG*8
+// pixels and all N channels; the [K x N] weights sit in shared memory for the CTA's
+// lifetime, the pixel tile streams through shared memory 8 input channels at a time
+// (transposed, so a thread reads its 8 pixels as two 128-bit words); a thread accumulates
+// 8 pixels x TN channels.  Thread `chg` owns the float4 channel groups chg + CG*j, so the
+// lanes of a warp write neighbouring 16-byte pieces of a pixel's row.
 // ---------------------------------------------------------------------------
-template <int NPT, int LPP>
+constexpr int PW_TM = 8, PW_KC = 8;
+
+template <int TN>
 struct PwIO {
-  static constexpr int VV = 4 * NPT;
+  static constexpr int VV = TN;
   const GemmParams& p;
-  float accv[VV];
+  float accv[TN];
   uint32_t pix;            // pixel index (row of the [P x N] result)
-  int q;                   // lane's slot among the LPP lanes of the pixel
+  int chg, cg;
   bool ok;
   __device__ __forceinline__ uint32_t off(const TensorArg& a, int j) const {
-    return (uint32_t)a.base + pix * (uint32_t)a.stride[1] + (uint32_t)(4 * (j * LPP + q)) * (uint32_t)a.stride[0];
+    return (uint32_t)a.base + pix * (uint32_t)a.stride[1] + (uint32_t)(4 * (chg + cg * j)) * (uint32_t)a.stride[0];
   }
   __device__ __forceinline__ void load(int idx, float (&dst)[VV]) const {
     const TensorArg& a = p.in[idx];
 #pragma unroll
-    for (int j = 0; j < NPT; ++j) {
+    for (int j = 0; j < TN / 4; ++j) {
       float* d = &dst[4 * j];
       if (!ok) { d[0] = d[1] = d[2] = d[3] = 0.0f; continue; }
       if (a.stride[0] == 0) { float x = load_scalar<true>(a, off(a, j)); d[0] = d[1] = d[2] = d[3] = x; }
@@ -49,58 +56,93 @@ struct PwIO {
     if (!ok) return;
     const TensorArg& a = p.out[idx];
 #pragma unroll
-    for (int j = 0; j < NPT; ++j) store_vec4<true>(a, off(a, j), &val[4 * j], false);
+    for (int j = 0; j < TN / 4; ++j) store_vec4<true>(a, off(a, j), &val[4 * j], false);
   }
   __device__ __forceinline__ void row_reduce(int, float (&)[VV]) const {}
 };
 
-template <int NPT, int LPP, class SP>
-__global__ void __launch_bounds__(256) conv1x1_kernel(const __grid_constant__ GemmParams p) {
-  extern __shared__ float wsm[];                 // [K][N]
+// THREADS = CG * PG; BM = PG * 8 pixels per CTA
+template <int TN, int CG, int PG, class SP>
+__global__ void __launch_bounds__(CG * PG) conv1x1_kernel(const __grid_constant__ GemmParams p) {
+  constexpr int THREADS = CG * PG, BM = PG * PW_TM, APITCH = BM + 16;
+  extern __shared__ float wsm[];                 // [K][N] weights, then [2][KC][APITCH] pixel chunks
   pdl_launch_dependents();
   pdl_wait();
   const int K = p.K, N = p.N;
+  float* as = wsm + K * N;
   const float* W = reinterpret_cast<const float*>(p.B.ptr) + p.B.base;
-  for (int i = threadIdx.x * 4; i < K * N; i += 256 * 4)
+  for (int i = threadIdx.x * 4; i < K * N; i += THREADS * 4)
     *reinterpret_cast<float4*>(&wsm[i]) = __ldg(reinterpret_cast<const float4*>(W + i));
-  __syncthreads();
   const float* X = reinterpret_cast<const float*>(p.A.ptr) + p.A.base;
-  constexpr int PPW = 32 / LPP;                  // pixels per warp
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int warps_total = gridDim.x * 8;
-  PwIO<NPT, LPP> io{p};
-  io.q = lane % LPP;
-  for (int64_t base = (int64_t)(blockIdx.x * 8 + warp) * PPW; base < p.M; base += (int64_t)warps_total * PPW) {
-    const int64_t pix = base + lane / LPP;
-    io.ok = pix < p.M;
-    io.pix = (uint32_t)(io.ok ? pix : 0);
-    const float* xr = X + (int64_t)io.pix * p.A.stride_row;
+  const int chg = threadIdx.x % CG, pxg = threadIdx.x / CG;
+  const int64_t m0 = (int64_t)blockIdx.x * BM;
+  // chunk loader: BM pixels x 8 input channels = 2*BM float4; thread t takes float4 (pixel t/2 + i*THREADS/2, half t%2)
+  constexpr int LD = (2 * BM + THREADS - 1) / THREADS;
+  float4 pre[LD];
+  auto fetch = [&](int k0) {
 #pragma unroll
-    for (int v = 0; v < 4 * NPT; ++v) io.accv[v] = 0.0f;
-    for (int k0 = 0; k0 < K; k0 += 8) {
-      float x[8];
-      {
-        float4 a = __ldg(reinterpret_cast<const float4*>(xr + k0));
-        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
-        if (k0 + 4 < K) { float4 b = __ldg(reinterpret_cast<const float4*>(xr + k0 + 4)); x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w; }
-        else { x[4] = x[5] = x[6] = x[7] = 0.0f; }
-      }
+    for (int i = 0; i < LD; ++i) {
+      int idx = threadIdx.x + i * THREADS;
+      int px = idx >> 1, half = idx & 1;
+      bool ok = idx < 2 * BM && m0 + px < p.M && k0 + half * 4 < K;
+      pre[i] = ok ? __ldg(reinterpret_cast<const float4*>(X + (m0 + px) * p.A.stride_row + k0 + half * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  auto stash = [&](int buf) {
+    float* dst = as + buf * (PW_KC * APITCH);
 #pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-        if (k0 + kk < K) {
-          const float* wr = wsm + (k0 + kk) * N + 4 * io.q;
-#pragma unroll
-          for (int j = 0; j < NPT; ++j) {
-            float4 w = *reinterpret_cast<const float4*>(wr + 4 * j * LPP);
-            io.accv[4 * j + 0] = fmaf(x[kk], w.x, io.accv[4 * j + 0]);
-            io.accv[4 * j + 1] = fmaf(x[kk], w.y, io.accv[4 * j + 1]);
-            io.accv[4 * j + 2] = fmaf(x[kk], w.z, io.accv[4 * j + 2]);
-            io.accv[4 * j + 3] = fmaf(x[kk], w.w, io.accv[4 * j + 3]);
-          }
-        }
+    for (int i = 0; i < LD; ++i) {
+      int idx = threadIdx.x + i * THREADS;
+      if (idx < 2 * BM) {
+        int px = idx >> 1, half = idx & 1;
+        dst[(half * 4 + 0) * APITCH + px] = pre[i].x; dst[(half * 4 + 1) * APITCH + px] = pre[i].y;
+        dst[(half * 4 + 2) * APITCH + px] = pre[i].z; dst[(half * 4 + 3) * APITCH + px] = pre[i].w;
       }
     }
-    run_program<4 * NPT, SP>(p.prog, io);
+  };
+  float acc[PW_TM][TN];
+#pragma unroll
+  for (int i = 0; i < PW_TM; ++i)
+#pragma unroll
+    for (int j = 0; j < TN; ++j) acc[i][j] = 0.0f;
+  fetch(0);
+  stash(0);
+  __syncthreads();
+  const int nchunks = (K + PW_KC - 1) / PW_KC;
+  for (int c = 0; c < nchunks; ++c) {
+    if (c + 1 < nchunks) fetch((c + 1) * PW_KC);          // next chunk's global loads overlap this chunk's FMAs
+    const float* a_s = as + (c & 1) * (PW_KC * APITCH) + pxg * PW_TM;
+#pragma unroll
+    for (int kk = 0; kk < PW_KC; ++kk) {
+      const int k = c * PW_KC + kk;
+      if (k < K) {
+        float4 a0 = *reinterpret_cast<const float4*>(a_s + kk * APITCH), a1 = *reinterpret_cast<const float4*>(a_s + kk * APITCH + 4);
+        const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+        float b[TN];
+#pragma unroll
+        for (int j = 0; j < TN / 4; ++j) {
+          float4 w = *reinterpret_cast<const float4*>(wsm + k * N + 4 * (chg + CG * j));
+          b[4 * j] = w.x; b[4 * j + 1] = w.y; b[4 * j + 2] = w.z; b[4 * j + 3] = w.w;
+        }
+#pragma unroll
+        for (int i = 0; i < PW_TM; ++i)
+#pragma unroll
+          for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+      }
+    }
+    if (c + 1 < nchunks) stash((c + 1) & 1);
+    __syncthreads();
+  }
+  PwIO<TN> io{p};
+  io.chg = chg; io.cg = CG;
+#pragma unroll
+  for (int i = 0; i < PW_TM; ++i) {
+    const int64_t pix = m0 + pxg * PW_TM + i;
+    io.ok = pix < p.M;
+    io.pix = (uint32_t)(io.ok ? pix : 0);
+#pragma unroll
+    for (int j = 0; j < TN; ++j) io.accv[j] = acc[i][j];
+    run_program<TN, SP>(p.prog, io);
   }
 }
 
@@ -115,10 +157,11 @@ using ConvStatic = TypeList<CP_ScaleShiftClip, CP_ScaleShiftResidual, CP_Store>;
 
 static const GemmParams& gp_of(const Launch& L) { return *reinterpret_cast<const GemmParams*>(L.blob.data()); }
 
-// (NPT, LPP) pairs that are instantiated; the host picks one with NPT*LPP == N/4
-static bool pw_shape(int n4, int& npt, int& lpp) {
-  static const int table[][2] = {{9, 4}, {3, 2}, {6, 4}, {4, 4}, {8, 4}, {2, 4}, {1, 4}, {5, 4}, {1, 2}, {1, 1}, {3, 1}};
-  for (auto& t : table) if (t[0] * t[1] == n4) { npt = t[0]; lpp = t[1]; return true; }
+// Instantiated (TN, CG, PG) shapes; the host picks one with TN*CG == N.
+struct PwShape { int tn, cg, pg; };
+static bool pw_shape(int n, PwShape& s) {
+  static const PwShape table[] = {{12, 12, 16}, {4, 6, 32}, {8, 8, 24}, {8, 16, 16}, {4, 4, 32}, {4, 8, 32}, {8, 4, 32}, {4, 2, 64}, {4, 1, 64}, {12, 4, 32}};
+  for (auto& t : table) if (t.tn * t.cg == n) { s = t; return true; }
   return false;
 }
 
@@ -131,55 +174,53 @@ bool conv1x1_direct_eligible(const GemmParams& gp) {
   if (gp.n_nd != 1 || gp.m_nd != 1 || gp.b_nd != 1 || !gp.vec_ok) return false;
   for (int i = 0; i < gp.n_in; ++i) if (gp.in[i].dtype != 0) return false;
   for (int i = 0; i < gp.n_out; ++i) if (gp.out[i].dtype != 0) return false;
-  int a, b;
-  return pw_shape(gp.N / 4, a, b);
+  PwShape s;
+  return pw_shape(gp.N, s);
 }
 
 void conv1x1_direct_plan(Launch& L) {
   GemmParams& gp = *reinterpret_cast<GemmParams*>(L.blob.data());
+  PwShape s;
+  pw_shape(gp.N, s);
   L.variant = 2;
-  L.threads = 256;
-  L.smem = (size_t)gp.K * gp.N * 4;
-  int npt, lpp;
-  pw_shape(gp.N / 4, npt, lpp);
-  int64_t warps = (gp.M + (32 / lpp) - 1) / (32 / lpp);
-  int64_t ctas = (warps + 7) / 8;
-  L.grid = (int)std::min<int64_t>(ctas, 148 * 4);
+  L.threads = s.cg * s.pg;
+  const int bm = s.pg * PW_TM;
+  L.smem = (size_t)gp.K * gp.N * 4 + 2 * PW_KC * (bm + 16) * 4;
+  L.grid = (int)((gp.M + bm - 1) / bm);
   L.static_id = StaticSet<ConvStatic>::find(gp.prog);
 }
 
-template <int NPT, int LPP>
+template <int TN, int CG, int PG>
 struct PwLauncher {
   const Launch& L; cudaStream_t st;
   template <class SP> void run() {
     static bool attr = false;
-    if (!attr) { cudaFuncSetAttribute(conv1x1_kernel<NPT, LPP, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); attr = true; }
-    launch_pdl(conv1x1_kernel<NPT, LPP, SP>, L.grid, 256, L.smem, st, gp_of(L));
+    if (!attr) { cudaFuncSetAttribute(conv1x1_kernel<TN, CG, PG, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024); attr = true; }
+    launch_pdl(conv1x1_kernel<TN, CG, PG, SP>, L.grid, CG * PG, L.smem, st, gp_of(L));
   }
 };
-template <int NPT, int LPP, bool kStatic>
+template <int TN, int CG, int PG, bool kStatic>
 static void pw_launch(const Launch& L, cudaStream_t st) {
-  PwLauncher<NPT, LPP> F{L, st};
+  PwLauncher<TN, CG, PG> F{L, st};
   if (kStatic && L.static_id > 0 && StaticSet<ConvStatic>::dispatch(L.static_id, F)) return;
   F.template run<DynProg>();
 }
 
 int conv1x1_direct_launch(const Launch& L, cudaStream_t st) {
   const GemmParams& gp = gp_of(L);
-  int npt = 0, lpp = 0;
-  pw_shape(gp.N / 4, npt, lpp);
-  switch (npt * 10 + lpp) {
-    case 94: pw_launch<9, 4, true>(L, st); break;
-    case 32: pw_launch<3, 2, true>(L, st); break;
-    case 64: pw_launch<6, 4, false>(L, st); break;
-    case 44: pw_launch<4, 4, false>(L, st); break;
-    case 84: pw_launch<8, 4, false>(L, st); break;
-    case 24: pw_launch<2, 4, false>(L, st); break;
-    case 14: pw_launch<1, 4, false>(L, st); break;
-    case 54: pw_launch<5, 4, false>(L, st); break;
-    case 12: pw_launch<1, 2, false>(L, st); break;
-    case 11: pw_launch<1, 1, false>(L, st); break;
-    case 31: pw_launch<3, 1, false>(L, st); break;
+  PwShape s{0, 0, 0};
+  pw_shape(gp.N, s);
+  switch (s.tn * 10000 + s.cg * 100 + s.pg) {
+    case 121216: pw_launch<12, 12, 16, true>(L, st); break;
+    case 40632: pw_launch<4, 6, 32, true>(L, st); break;
+    case 80824: pw_launch<8, 8, 24, false>(L, st); break;
+    case 81616: pw_launch<8, 16, 16, false>(L, st); break;
+    case 40432: pw_launch<4, 4, 32, false>(L, st); break;
+    case 40832: pw_launch<4, 8, 32, false>(L, st); break;
+    case 80432: pw_launch<8, 4, 32, false>(L, st); break;
+    case 40264: pw_launch<4, 2, 64, false>(L, st); break;
+    case 40164: pw_launch<4, 1, 64, false>(L, st); break;
+    case 120432: pw_launch<12, 4, 32, false>(L, st); break;
     default: return 2;
   }
   return cudaGetLastError() == cudaSuccess ? 0 : 1;
@@ -249,19 +290,19 @@ __global__ void __launch_bounds__(256) dwconv_kernel(const __grid_constant__ DwP
     const float* q = xb + ((int64_t)h * p.W + w) * p.C;
     r[0] = ld4_or_zero(q - p.C, ok && wl); r[1] = ld4_or_zero(q, ok); r[2] = ld4_or_zero(q + p.C, ok && wr);
   };
-  float4 r0[3], r1[3], r2[3];
-  row(h0 - 1, r0); row(h0, r1);
+  float4 r0[3], r1[3], r2[3], r3[3];
+  row(h0 - 1, r0); row(h0, r1); row(h0 + 1, r2);
   DwIO io{p};
   io.n = n; io.w = w; io.c = c4 * 4;
   for (int h = h0; h < h1; ++h) {
-    row(h + 1, r2);
+    row(h + 2, r3);                              // the row needed by the NEXT output: in flight during this one
     io.accv[0] = io.accv[1] = io.accv[2] = io.accv[3] = 0.0f;
 #pragma unroll
     for (int j = 0; j < 3; ++j) { fma4(io.accv, r0[j], kw[j]); fma4(io.accv, r1[j], kw[3 + j]); fma4(io.accv, r2[j], kw[6 + j]); }
     io.h = h;
     run_program<4, SP>(p.prog, io);
 #pragma unroll
-    for (int j = 0; j < 3; ++j) { r0[j] = r1[j]; r1[j] = r2[j]; }
+    for (int j = 0; j < 3; ++j) { r0[j] = r1[j]; r1[j] = r2[j]; r2[j] = r3[j]; }
   }
 }
 
