@@ -317,6 +317,17 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
   }
   gp.batch_ext[0] = bext.size() > 0 ? (int)bext[bext.size() - 1] : 1;
   gp.batch_ext[1] = bext.size() > 1 ? (int)bext[0] : 1;
+  // A weight shared by every batch and an activation whose batches follow each other row after row
+  // is one tall 2-D GEMM: fold the batch dims into M (one wave of large tiles instead of many small ones).
+  bool fold_batch = false;
+  if (A.kind == DNNF_OP_MATMUL && nbatch > 1 && gp.B.batch_stride[0] == 0 && gp.B.batch_stride[1] == 0 &&
+      gp.A.batch_stride[0] == (int64_t)gp.M * gp.A.stride_row &&
+      (bext.size() < 2 || gp.A.batch_stride[1] == gp.batch_ext[0] * gp.A.batch_stride[0]) && (int64_t)gp.M * nbatch < (1ll << 31)) {
+    fold_batch = true;
+    gp.M = (int)(gp.M * nbatch);
+    gp.batch_ext[0] = gp.batch_ext[1] = 1;
+    gp.A.batch_stride[0] = gp.A.batch_stride[1] = 0;
+  }
 
   // ---- epilogue ------------------------------------------------------------------
   LowerCtx cx(g);
@@ -353,7 +364,7 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
       int64_t p = 1;
       int gk;
       if (A.kind == DNNF_OP_CONV1X1) gk = k < 3 ? 1 : 2;
-      else gk = k + 2 < C.dims.size() ? 0 : (k + 2 == C.dims.size() ? 1 : 2);
+      else gk = k + 2 < C.dims.size() ? (fold_batch ? 1 : 0) : (k + 2 == C.dims.size() ? 1 : 2);
       bool first = true;
       while (p < C.dims[k] || (first && d < cx.ext.size() && cx.ext[d] == 1 && C.dims[k] == 1)) {
         if (d >= cx.ext.size()) { why = "internal: refinement mismatch"; return DNNF_ERR_UNSUPPORTED_OP; }
@@ -416,7 +427,7 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
   out.inputs = {srcA, srcB};
   for (auto& a : cx.ins) { L.in_tensors.push_back(a.tensor); if (std::find(out.inputs.begin(), out.inputs.end(), a.tensor) == out.inputs.end()) out.inputs.push_back(a.tensor); }
   for (auto& a : cx.outs) { L.out_tensors.push_back(a.tensor); out.outputs.push_back(a.tensor); }
-  L.flops = 2ll * gp.M * gp.N * gp.K * nbatch;
+  L.flops = 2ll * gp.M * gp.N * gp.K * (fold_batch ? 1 : nbatch);
   L.family = A.kind == DNNF_OP_CONV1X1 ? DNNF_FAMILY_CONV1X1 : DNNF_FAMILY_GEMM;
 
   if (tc2_gemm_eligible(gp)) {

@@ -130,9 +130,10 @@ def encoder_report(dev, pk, layers=12):
     for b in range(nb_layer, 2 * nb_layer if layers > 1 else nb_layer):
         if blocks[b]["family"] == "alias":
             continue
-        cg = _graph_of(torch, dev, lambda sp, b=b: s.g.run_block(b, sp))
+        reps = 20        # several launches per replay: a one-node graph is bound by the replay overhead itself
+        cg = _graph_of(torch, dev, lambda sp, b=b: [s.g.run_block(b, sp) for _ in range(reps)])
         cg.replay()
-        t = _time_region(torch, dev, cg.replay, 50)
+        t = _time_region(torch, dev, cg.replay, 10) / reps
         by, fl = blocks[b]["bytes"], blocks[b]["flops"]
         roof = max(by / (pk["hbm_gbs"] * 1e3), fl / (pk["bf16_tflops"] * 1e6))
         per.append({"ops": "+".join(blocks[b]["ops"][:10]), "family": blocks[b]["family"], "us_warm_l2": round(t, 3), "bytes": by,
