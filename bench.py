@@ -1,5 +1,5 @@
 #!/usr/bin/env python
-"""Benchmark of the fused-block executor on one B200 ("Measurement").
+"""Benchmark of the fused-block executor on one B200.
 
 Default arm: `python bench.py --gpus N --steps K --warmup W` prints ONE JSON line.
 A step is one pass of the hot path -- dnnf_run of the fused scale+mask+softmax
@@ -81,6 +81,27 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def max_over_ranks(value, device=None):
+    """Slowest rank's time (all ranks get it).  Works with any initialised backend (nccl on GPUs, gloo on CPU)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(bytes_per_rank_step, ms_step_max, world):
+    """Whole-job GB/s when every rank processes its own replica of the step (weak scaling, no exchange step)."""
+    return world * bytes_per_rank_step / (ms_step_max * 1e-3) / 1e9
+
+
+def rank_seed(base_seed, rank):
+    """Each replica draws its own inputs."""
+    return base_seed + 100 * rank
+
+
 def block_bytes(sess):
     tot = 0
     for b in range(sess.g.block_count()):
@@ -155,7 +176,7 @@ def main():
     steps, warm = args.steps, max(args.warmup, 3)
 
     # ---- the step: R instances of each block, distinct buffers (footprint > L2) ------------------
-    wa, wb = W.masked_softmax(seed=W.BASE_SEED + 100 * rank), W.add_layernorm_gelu(seed=W.BASE_SEED + 100 * rank)
+    wa, wb = W.masked_softmax(seed=rank_seed(W.BASE_SEED, rank)), W.add_layernorm_gelu(seed=rank_seed(W.BASE_SEED, rank))
     A = [Session(wa, rewrite_flags=B.REWRITE_NONE, device=dev) for _ in range(R_INSTANCES)]
     Bn = [Session(wb, rewrite_flags=B.REWRITE_NONE, device=dev) for _ in range(R_INSTANCES)]
     bytes_a, bytes_b = block_bytes(A[0]), block_bytes(Bn[0])
@@ -212,11 +233,8 @@ def main():
     t_a = sum(e[0].elapsed_time(e[1]) for e in ev) / steps             # ms per step in part a
     t_b = sum(e[1].elapsed_time(e[2]) for e in ev) / steps
     ms_step = t_total / steps
-    if world > 1:
-        t = torch.tensor([ms_step], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step = float(t.item())
-    value = world * bytes_step / (ms_step * 1e-3) / 1e9
+    ms_step = max_over_ranks(ms_step, dev)
+    value = aggregate_throughput(bytes_step, ms_step, world)
 
     # ---- roofline of the dominant kernel (the softmax row kernel) ---------------------------------
     dur_a = t_a * 1e-3 / R_INSTANCES
@@ -264,11 +282,8 @@ def main():
     e1.record(stream)
     torch.cuda.synchronize(dev)
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e = {"value": world * bytes_step / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+    e2e_ms = max_over_ranks(e2e_ms, dev)
+    e2e = {"value": aggregate_throughput(bytes_step, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,

@@ -255,13 +255,21 @@ __global__ void __launch_bounds__(256) tr_kernel(const __grid_constant__ EwParam
 }
 
 // ---------------------------------------------------------------------------
+// Vectors per thread for interpreted programs.
+constexpr int kDynU = 2;     // (4 was measured: occupancy halves and it gets slower)
+
 template <bool F32>
 struct EwLauncher {
   const Launch& L; cudaStream_t st;
   template <class SP> void run() {
-    if (L.family == DNNF_FAMILY_ELEMENTWISE) launch_pdl(ew_kernel<4, 2, SP, F32>, L.grid, 256, 0, st, L.ew);
-    else launch_pdl(tr_kernel<4, SP, F32>, L.grid, 256, L.smem, st, L.ew);
+    if (SP::n == 0) launch_pdl(ew_kernel<4, kDynU, SP, F32>, L.grid, 256, 0, st, L.ew);
+    else launch_pdl(ew_kernel<4, 2, SP, F32>, L.grid, 256, 0, st, L.ew);
   }
+};
+template <bool F32>
+struct TrLauncher {
+  const Launch& L; cudaStream_t st;
+  template <class SP> void run() { launch_pdl(tr_kernel<4, SP, F32>, L.grid, 256, L.smem, st, L.ew); }
 };
 
 static bool all_f32(const EwParams& p) {
@@ -272,7 +280,15 @@ static bool all_f32(const EwParams& p) {
 
 int launch_ew(const Launch& L, cudaStream_t st) {
   const EwParams& p = L.ew;
-  if (p.vec == 4) {
+  if (p.vec == 4 && L.family == DNNF_FAMILY_TRANSPOSE) {
+    if (all_f32(p)) {
+      TrLauncher<true> F{L, st};
+      if (!(L.static_id > 0 && StaticSet<TrStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
+    } else {
+      TrLauncher<false> F{L, st};
+      if (!(L.static_id > 0 && StaticSet<TrStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
+    }
+  } else if (p.vec == 4) {
     if (all_f32(p)) {
       EwLauncher<true> F{L, st};
       if (!(L.static_id > 0 && StaticSet<EwStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
@@ -321,15 +337,16 @@ void finalize_ew(Launch& L) {
     }
     L.smem = (size_t)staged * TT * TPITCH * sizeof(float);
     L.grid = (int)grid; L.threads = 256;
-  } else {
-    int U = p.vec == 4 ? 2 : 4;
+  }
+  L.static_id = p.vec != 4 ? 0 : (L.family == DNNF_FAMILY_TRANSPOSE ? StaticSet<TrStatic>::find(p.prog) : StaticSet<EwStatic>::find(p.prog));
+  if (L.family != DNNF_FAMILY_TRANSPOSE) {
+    int U = p.vec == 4 ? (L.static_id > 0 ? 2 : kDynU) : 4;
     int64_t nvec = p.total / p.vec;
     L.grid = (int)((nvec + 256 * U - 1) / (256 * U));
     L.threads = 256;
     p.inner_vecs = p.it.extent[0] / p.vec;
     fastdiv_for(p.inner_vecs, p.inner_m, p.inner_s);
   }
-  L.static_id = p.vec == 4 ? StaticSet<EwStatic>::find(p.prog) : 0;
   L.variant = p.vec * 100 + L.static_id;
   set_fastdiv(p.it);
 }

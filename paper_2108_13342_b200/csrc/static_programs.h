@@ -46,6 +46,18 @@ DNNF_SP_BEGIN(SP_GeluPrimitives, 8)
   MO(M_MOV, S_IN, 0), MO(M_SAVE, S_TMP, 0), MO(M_MUL, S_CONST, 0), MO(M_ERF, S_NONE, 0), MO(M_ADD, S_CONST, 1),
   MO(M_MUL, S_TMP, 0), MO(M_MUL, S_CONST, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
 
+// single operators (the one-kernel-per-operator baseline must not be handicapped by the interpreter)
+DNNF_SP_BEGIN(SP_ScaleShift, 4) MO(M_MOV, S_IN, 0), MO(M_MUL, S_IN, 1), MO(M_ADD, S_IN, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(SP_Clip, 3) MO(M_MOV, S_IN, 0), MO(M_CLIP, S_CONST, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(SP_AddC, 3) MO(M_MOV, S_IN, 0), MO(M_ADD, S_CONST, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(SP_Erf, 3) MO(M_MOV, S_IN, 0), MO(M_ERF, S_NONE, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(SP_GeluTanh, 3) MO(M_MOV, S_IN, 0), MO(M_GELU_TANH, S_NONE, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(SP_SubIn, 3) MO(M_MOV, S_IN, 0), MO(M_SUB, S_IN, 1), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(SP_DivIn, 3) MO(M_MOV, S_IN, 0), MO(M_DIV, S_IN, 1), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(SP_Square, 3) MO(M_MOV, S_IN, 0), MO(M_SQUARE, S_NONE, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(SP_Sqrt, 3) MO(M_MOV, S_IN, 0), MO(M_SQRT, S_NONE, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(SP_Relu, 3) MO(M_MOV, S_IN, 0), MO(M_RELU, S_NONE, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+
 // ---- row family --------------------------------------------------------------------------
 DNNF_SP_BEGIN(SP_ScaleMaskSoftmax, 12)
   MO(M_MOV, S_IN, 0), MO(M_MUL, S_CONST, 0), MO(M_ADD, S_IN, 1), MO(M_SAVE, S_TMP, 0), MO(M_ROWMAX, S_NONE, 0),
@@ -72,7 +84,9 @@ DNNF_SP_BEGIN(SP_BiasResidualLayerNorm, 16)
 
 template <class... T> struct TypeList {};
 using EwStatic = TypeList<SP_Move, SP_BiasScaleSwish, SP_AddIn, SP_MulIn, SP_MulC, SP_Sigmoid, SP_GeluErf, SP_ScaleShiftClip,
-                          SP_GeluPrimitives>;
+                          SP_GeluPrimitives, SP_ScaleShift, SP_Clip, SP_AddC, SP_Erf, SP_GeluTanh, SP_SubIn, SP_DivIn, SP_Square, SP_Sqrt,
+                          SP_Relu>;
+using TrStatic = TypeList<SP_Move, SP_BiasScaleSwish>;
 using RowStatic = TypeList<SP_ScaleMaskSoftmax, SP_Softmax, SP_AddLayerNormGelu, SP_LayerNorm, SP_BiasResidualLayerNorm>;
 
 template <class SP>
