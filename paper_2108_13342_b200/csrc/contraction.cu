@@ -27,6 +27,11 @@ bool tc2_gemm_eligible(const GemmParams& gp);
 void tc2_gemm_plan(Launch& L);
 bool tc2_gemm_prepare(Launch& L, std::string& err);
 int tc2_gemm_launch(const Launch& L, cudaStream_t st);
+size_t tf32_blob_bytes();
+bool tf32_gemm_eligible(const GemmParams& gp);
+void tf32_gemm_plan(Launch& L);
+bool tf32_gemm_prepare(Launch& L, std::string& err);
+int tf32_gemm_launch(const Launch& L, cudaStream_t st);
 bool conv1x1_direct_eligible(const GemmParams& gp);
 void conv1x1_direct_plan(Launch& L);
 int conv1x1_direct_launch(const Launch& L, cudaStream_t st);
@@ -238,7 +243,7 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
 
   Launch& L = out.launch;
   L = Launch{};
-  L.blob.assign(sizeof(GemmParams) + sizeof(GemmTcParams) + tc2_blob_bytes(), 0);
+  L.blob.assign(sizeof(GemmParams) + sizeof(GemmTcParams) + std::max(tc2_blob_bytes(), tf32_blob_bytes()), 0);
   GemmParams& gp = gp_of(L);
 
   // ---- operands ----------------------------------------------------------------
@@ -419,6 +424,9 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
   for (size_t i = 0; i < cx.outs.size(); ++i) if (!fill(gp.out[i], cx.outs[i], cx.ins.size() + i)) { why = "tensor too large"; return DNNF_ERR_UNSUPPORTED_OP; }
   if (gp.it.extent[0] % 8) vec_ok = false;
   gp.vec_ok = vec_ok;
+  auto is_static = [&](int t) { return g.tensors[t].external && g.tensors[t].producer < 0 && !g.tensors[t].is_output; };
+  gp.static_mask = is_static(srcB) ? 1u : 0u;
+  for (size_t i = 0; i < cx.ins.size(); ++i) if (is_static(cx.ins[i].tensor)) gp.static_mask |= 2u << i;
   gp.prog = cx.prog;
   L.ew.prog = cx.prog;            // introspection (dnnf_block_program)
 
@@ -435,6 +443,8 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
   } else if (tc_gemm_eligible(gp)) {
     L.variant = 1;
     tc_gemm_plan(L);
+  } else if (tf32_gemm_eligible(gp)) {
+    tf32_gemm_plan(L);
   } else if (A.kind == DNNF_OP_CONV1X1 && conv1x1_direct_eligible(gp)) {
     conv1x1_direct_plan(L);
   } else {
@@ -455,6 +465,10 @@ void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vecto
   for (int i = 0; i < gp.n_out; ++i) gp.out[i].ptr = op[i];
   if (L.variant == 3) changed = changed || !L.tc_ready || gp.out[0].ptr != L.last_out || (gp.n_in > 0 && gp.in[0].ptr != L.last_in0) || (gp.n_in > 1 && gp.in[1].ptr != L.last_in1);
   if (L.variant == 1 && (changed || !L.tc_ready)) { if (tc_gemm_prepare(L, err)) L.tc_ready = true; }
+  if (L.variant == 4 && (changed || !L.tc_ready || gp.out[0].ptr != L.last_out)) {
+    if (tf32_gemm_prepare(L, err)) L.tc_ready = true;
+    L.last_out = gp.out[0].ptr;
+  }
   if (L.variant == 3 && changed) {
     if (tc2_gemm_prepare(L, err)) L.tc_ready = true;
     L.last_out = gp.out[0].ptr; L.last_in0 = gp.n_in > 0 ? gp.in[0].ptr : nullptr; L.last_in1 = gp.n_in > 1 ? gp.in[1].ptr : nullptr;
@@ -472,6 +486,13 @@ int launch_contraction(const Launch& L, void* status_words, int block_index, cud
     gp_of(M).status = gp.status; gp_of(M).block_index = block_index;
     int rc = tc2_gemm_launch(L, st);
     if (rc) err = "tensor-core pair GEMM launch failed";
+    return rc;
+  }
+  if (L.variant == 4) {
+    Launch& M = const_cast<Launch&>(L);
+    gp_of(M).status = gp.status; gp_of(M).block_index = block_index;
+    int rc = tf32_gemm_launch(L, st);
+    if (rc) err = "tensor-core fp32 GEMM launch failed";
     return rc;
   }
   if (L.variant == 1) {

@@ -32,6 +32,7 @@ struct GemmParams {
   int32_t tiles_m, tiles_n;
   int32_t* status;         // device status words (bounded-wait failures)
   int32_t block_index;
+  uint32_t static_mask;     // bit 0: B, bit 1+i: epilogue input i is an external input of the graph (never written by a kernel)
 };
 
 // Tensor-core path extras (kept apart so the common block stays small).

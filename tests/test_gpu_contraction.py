@@ -118,6 +118,40 @@ def test_conv1x1_with_epilogue(cfg):
     check(W.Workload(g, ins), RTOL_F32, FUSED, expect_blocks=1)
 
 
+# fp32 blocks on the tensor cores (split-TF32): tall-and-skinny shapes, ragged M, N and K
+@pytest.mark.parametrize("cfg", [(2, 16, 16, 24, 144), (3, 19, 23, 144, 24), (1, 30, 31, 12, 20), (1, 40, 40, 36, 160), (4, 16, 16, 32, 192),
+                                 (1, 33, 33, 100, 8), (2, 24, 24, 96, 48)])
+@pytest.mark.parametrize("epi", ["clip", "residual", "none"])
+def test_conv1x1_tensor_core_fp32(cfg, epi):
+    n, h, w, ci, co = cfg
+    g = graph()
+    g.ext("X", (n, h, w, ci)); g.ext("Wc", (ci, co)); g.ext("s", (co,)); g.ext("t", (co,))
+    ins = {"X": rnd((n, h, w, ci), 11, -1, 1), "Wc": rnd((ci, co), 12, -0.5, 0.5), "s": rnd((co,), 13, 0.5, 1.5), "t": rnd((co,), 14, -0.5, 0.5)}
+    e = g.add("Conv1x1", ["X", "Wc"])
+    if epi == "none":
+        g.mark_output(e)
+    else:
+        e = g.add("ScaleShift", [e, "s", "t"], axis=-1)
+        if epi == "clip":
+            g.mark_output(g.add("Clip", [e], lo=0.0, hi=6.0, out="Y"))
+        else:
+            g.ext("R", (n, h, w, co)); ins["R"] = rnd((n, h, w, co), 15, -1, 1)
+            g.mark_output(g.add("Add", [e, "R"], out="Y"))
+    s = check(W.Workload(g, ins), RTOL_F32, FUSED, expect_blocks=1)
+    assert s.g.blocks()[0]["variant"] == 4, s.g.blocks()
+
+
+def test_matmul_fp32_tall_skinny_uses_tensor_cores():
+    m, k, n = 1000, 52, 72
+    g = graph()
+    g.ext("X", (m, k)); g.ext("Wt", (k, n), kind="weight"); g.ext("b", (n,))
+    t = g.add("MatMul", ["X", "Wt"])
+    t = g.add("Add", [t, "b"])
+    g.mark_output(g.add("Tanh", [t], out="Y"))
+    s = check(W.Workload(g, {"X": rnd((m, k), 3, -1, 1), "Wt": rnd((k, n), 4, -0.3, 0.3), "b": rnd((n,), 5)}), RTOL_F32, FUSED, expect_blocks=1)
+    assert s.g.blocks()[0]["variant"] == 4
+
+
 @pytest.mark.parametrize("cfg", [(1, 5, 6, 8), (2, 7, 9, 144), (1, 1, 1, 4), (1, 3, 1, 12), (2, 30, 17, 24)])
 def test_dwconv3x3_with_epilogue(cfg):
     n, h, w, c = cfg
