@@ -36,7 +36,7 @@ bool conv1x1_direct_eligible(const GemmParams& gp);
 void conv1x1_direct_plan(Launch& L);
 int conv1x1_direct_launch(const Launch& L, cudaStream_t st);
 int lower_dwconv(const Graph& g, const std::vector<int>& ops, int anchor, Block& out, std::string& why);
-int dwconv_launch(const Launch& L, cudaStream_t st);
+int dwconv_launch(const Launch& L, void* status_words, int block_index, cudaStream_t st);
 void dwconv_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
 
 static GemmParams& gp_of(Launch& L) { return *reinterpret_cast<GemmParams*>(L.blob.data()); }
@@ -476,7 +476,7 @@ void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vecto
 }
 
 int launch_contraction(const Launch& L, void* status_words, int block_index, cudaStream_t st, std::string& err) {
-  if (L.family == DNNF_FAMILY_DWCONV) { int rc = dwconv_launch(L, st); if (rc) err = "depthwise convolution launch failed"; return rc; }
+  if (L.family == DNNF_FAMILY_DWCONV) { int rc = dwconv_launch(L, status_words, block_index, st); if (rc) err = "depthwise convolution launch failed"; return rc; }
   if (L.variant == 2) { int rc = conv1x1_direct_launch(L, st); if (rc) err = "pointwise convolution launch failed"; return rc; }
   GemmParams gp = gp_of(L);
   gp.status = reinterpret_cast<int32_t*>(status_words);

@@ -11,6 +11,7 @@
 #include <algorithm>
 
 #include "chain.cuh"
+#include "conv_params.h"
 #include "gemm_params.h"
 #include "lower.h"
 
@@ -146,15 +147,6 @@ __global__ void __launch_bounds__(CG * PG) conv1x1_kernel(const __grid_constant_
   }
 }
 
-#define MO(o, s, i) MicroOp{o, s, i, 0}
-DNNF_SP_BEGIN(CP_ScaleShiftClip, 5)
-  MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_CLIP, S_CONST, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-DNNF_SP_BEGIN(CP_ScaleShiftResidual, 5)
-  MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_ADD, S_IN, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-DNNF_SP_BEGIN(CP_Store, 2) MO(M_MOV, S_ANCHOR, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-#undef MO
-using ConvStatic = TypeList<CP_ScaleShiftClip, CP_ScaleShiftResidual, CP_Store>;
-
 static const GemmParams& gp_of(const Launch& L) { return *reinterpret_cast<const GemmParams*>(L.blob.data()); }
 
 // Instantiated (TN, CG, PG) shapes; the host picks one with TN*CG == N.
@@ -229,36 +221,6 @@ int conv1x1_direct_launch(const Launch& L, cudaStream_t st) {
 // ---------------------------------------------------------------------------
 // Depthwise 3x3
 // ---------------------------------------------------------------------------
-struct DwParams {
-  int32_t N, H, W, C;
-  const float* x;
-  const float* k;          // [3][3][C]
-  int32_t n_in, n_out;
-  TensorArg in[kMaxIn];    // strides over (c, w, h, n), innermost first
-  TensorArg out[kMaxOut];
-  Program prog;
-};
-
-struct DwIO {
-  const DwParams& p;
-  float accv[4];
-  uint32_t n, h, w, c;
-  __device__ __forceinline__ uint32_t off(const TensorArg& a) const {
-    return (uint32_t)a.base + c * (uint32_t)a.stride[0] + w * (uint32_t)a.stride[1] + h * (uint32_t)a.stride[2] + n * (uint32_t)a.stride[3];
-  }
-  __device__ __forceinline__ void load(int idx, float (&dst)[4]) const {
-    const TensorArg& a = p.in[idx];
-    if (a.stride[0] == 0) { float x = load_scalar<true>(a, off(a)); dst[0] = dst[1] = dst[2] = dst[3] = x; }
-    else load_vec4<true>(a, off(a), dst);
-  }
-  __device__ __forceinline__ void anchor(float (&dst)[4]) const {
-#pragma unroll
-    for (int v = 0; v < 4; ++v) dst[v] = accv[v];
-  }
-  __device__ __forceinline__ void store(int idx, const float (&val)[4]) const { store_vec4<true>(p.out[idx], off(p.out[idx]), val, false); }
-  __device__ __forceinline__ void row_reduce(int, float (&)[4]) const {}
-};
-
 __device__ __forceinline__ float4 ld4_or_zero(const float* p, bool ok) {
   return ok ? __ldg(reinterpret_cast<const float4*>(p)) : make_float4(0.f, 0.f, 0.f, 0.f);
 }
@@ -266,12 +228,18 @@ __device__ __forceinline__ void fma4(float (&acc)[4], const float4& x, const flo
   acc[0] = fmaf(x.x, k.x, acc[0]); acc[1] = fmaf(x.y, k.y, acc[1]); acc[2] = fmaf(x.z, k.z, acc[2]); acc[3] = fmaf(x.w, k.w, acc[3]);
 }
 
-// HS rows per thread: the grid covers (n, h-strip, w, c4)
+// HS rows per thread: the grid covers (n, h-strip, w, c4).  The 3x3 weights sit in shared memory
+// (a thread re-reads its nine 128-bit words per output row: conflict-free, neighbouring lanes hold
+// neighbouring channels), which keeps the thread at 64 registers so that four CTAs fit an SM and
+// enough loads are in flight to cover the memory latency.
 template <class SP>
-__global__ void __launch_bounds__(256) dwconv_kernel(const __grid_constant__ DwParams p, int HS) {
+__global__ void __launch_bounds__(256, 4) dwconv_kernel(const __grid_constant__ DwParams p, int HS) {
+  extern __shared__ float4 kws[];                // [9][C/4]
   pdl_launch_dependents();
   pdl_wait();
   const int C4 = p.C / 4;
+  for (int i = threadIdx.x; i < 9 * C4; i += 256) kws[i] = __ldg(reinterpret_cast<const float4*>(p.k) + i);
+  __syncthreads();
   const int strips = (p.H + HS - 1) / HS;
   int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
   const int64_t total = (int64_t)p.N * strips * p.W * C4;
@@ -280,9 +248,7 @@ __global__ void __launch_bounds__(256) dwconv_kernel(const __grid_constant__ DwP
   const int w = (int)(t % p.W); t /= p.W;
   const int s = (int)(t % strips); const int n = (int)(t / strips);
   const int h0 = s * HS, h1 = min(p.H, h0 + HS);
-  float4 kw[9];
-#pragma unroll
-  for (int i = 0; i < 9; ++i) kw[i] = __ldg(reinterpret_cast<const float4*>(p.k + i * p.C + c4 * 4));
+  const float4* kw = kws + c4;
   const float* xb = p.x + ((int64_t)n * p.H * p.W) * p.C + c4 * 4;
   const bool wl = w > 0, wr = w + 1 < p.W;
   auto row = [&](int h, float4 (&r)[3]) {
@@ -298,7 +264,7 @@ __global__ void __launch_bounds__(256) dwconv_kernel(const __grid_constant__ DwP
     row(h + 2, r3);                              // the row needed by the NEXT output: in flight during this one
     io.accv[0] = io.accv[1] = io.accv[2] = io.accv[3] = 0.0f;
 #pragma unroll
-    for (int j = 0; j < 3; ++j) { fma4(io.accv, r0[j], kw[j]); fma4(io.accv, r1[j], kw[3 + j]); fma4(io.accv, r2[j], kw[6 + j]); }
+    for (int j = 0; j < 3; ++j) { fma4(io.accv, r0[j], kw[j * C4]); fma4(io.accv, r1[j], kw[(3 + j) * C4]); fma4(io.accv, r2[j], kw[(6 + j) * C4]); }
     io.h = h;
     run_program<4, SP>(p.prog, io);
 #pragma unroll
@@ -306,14 +272,20 @@ __global__ void __launch_bounds__(256) dwconv_kernel(const __grid_constant__ DwP
   }
 }
 
+size_t dwconv_tma_blob_bytes();
+bool dwconv_tma_plan(Launch& L);
+bool dwconv_tma_prepare(Launch& L, std::string& err);
+int dwconv_tma_launch(const Launch& L, int32_t* status, int block_index, cudaStream_t st);
+
 static const DwParams& dw_of(const Launch& L) { return *reinterpret_cast<const DwParams*>(L.blob.data()); }
 
 struct DwLauncher {
   const Launch& L; cudaStream_t st; int hs;
-  template <class SP> void run() { launch_pdl(dwconv_kernel<SP>, L.grid, 256, 0, st, dw_of(L), hs); }
+  template <class SP> void run() { launch_pdl(dwconv_kernel<SP>, L.grid, 256, (size_t)9 * dw_of(L).C * 4, st, dw_of(L), hs); }
 };
 
-int dwconv_launch(const Launch& L, cudaStream_t st) {
+int dwconv_launch(const Launch& L, void* status_words, int block_index, cudaStream_t st) {
+  if (L.variant < 0) return dwconv_tma_launch(L, reinterpret_cast<int32_t*>(status_words), block_index, st);
   DwLauncher F{L, st, L.variant};
   if (!(L.static_id > 0 && StaticSet<ConvStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
   return cudaGetLastError() == cudaSuccess ? 0 : 1;
@@ -321,6 +293,11 @@ int dwconv_launch(const Launch& L, cudaStream_t st) {
 
 void dwconv_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op) {
   DwParams& dp = *reinterpret_cast<DwParams*>(L.blob.data());
+  if (L.variant < 0 && (dp.x != ip[0] || !L.tc_ready)) {
+    dp.x = reinterpret_cast<const float*>(ip[0]);
+    std::string err;
+    L.tc_ready = dwconv_tma_prepare(L, err);
+  }
   dp.x = reinterpret_cast<const float*>(ip[0]);
   dp.k = reinterpret_cast<const float*>(ip[1]);
   for (int i = 0; i < dp.n_in; ++i) dp.in[i].ptr = ip[2 + i];
@@ -335,6 +312,7 @@ int lower_dwconv(const Graph& g, const std::vector<int>& ops, int anchor, Block&
   std::set<int> in_block(ops.begin(), ops.end());
   if (X.dtype != DNNF_F32 || Kt.dtype != DNNF_F32) { why = "depthwise convolution is fp32 only"; return DNNF_ERR_UNSUPPORTED_OP; }
   if (X.dims[3] % 4) { why = "depthwise convolution needs a channel count that is a multiple of 4"; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (X.dims[3] > 1280) { why = "depthwise convolution: more than 1280 channels"; return DNNF_ERR_UNSUPPORTED_OP; }   // weights in 48 KB of shared memory
   if (in_block.count(X.producer) || in_block.count(Kt.producer)) { why = "operators in front of a convolution anchor (no prologue fusion)"; return DNNF_ERR_UNSUPPORTED_OP; }
   if (X.numel() >= (1ll << 31)) { why = "tensor too large"; return DNNF_ERR_UNSUPPORTED_OP; }
   LowerCtx cx(g);
@@ -345,7 +323,7 @@ int lower_dwconv(const Graph& g, const std::vector<int>& ops, int anchor, Block&
   if (!emit_program(cx, A.out[0], 2)) { why = cx.why; return DNNF_ERR_UNSUPPORTED_OP; }
   Launch& L = out.launch;
   L = Launch{};
-  L.blob.assign(sizeof(DwParams), 0);
+  L.blob.assign(sizeof(DwParams) + dwconv_tma_blob_bytes(), 0);
   DwParams& dp = *reinterpret_cast<DwParams*>(L.blob.data());
   dp.N = (int)Y.dims[0]; dp.H = (int)Y.dims[1]; dp.W = (int)Y.dims[2]; dp.C = (int)Y.dims[3];
   dp.n_in = (int)cx.ins.size(); dp.n_out = (int)cx.outs.size();
@@ -367,10 +345,12 @@ int lower_dwconv(const Graph& g, const std::vector<int>& ops, int anchor, Block&
   for (auto& a : cx.ins) { L.in_tensors.push_back(a.tensor); if (std::find(out.inputs.begin(), out.inputs.end(), a.tensor) == out.inputs.end()) out.inputs.push_back(a.tensor); }
   for (auto& a : cx.outs) { L.out_tensors.push_back(a.tensor); out.outputs.push_back(a.tensor); }
   L.family = DNNF_FAMILY_DWCONV;
+  L.flops = 2ll * 9 * Y.numel();
+  if (dwconv_tma_plan(L)) { out.lowered = true; return DNNF_OK; }
   // rows per thread: enough threads to fill the machine, long enough strips to reuse the window
   int hs = dp.H;
   int64_t threads_full = (int64_t)dp.N * dp.W * (dp.C / 4);
-  while (hs > 7 && threads_full * ((dp.H + hs - 1) / hs) < 148 * 2048 * 2) hs = (hs + 1) / 2;
+  while (hs > 7 && threads_full * ((dp.H + hs - 1) / hs) < 148 * 1024 * 4) hs = (hs + 1) / 2;
   L.variant = hs;
   int64_t total = threads_full * ((dp.H + hs - 1) / hs);
   L.grid = (int)((total + 255) / 256);

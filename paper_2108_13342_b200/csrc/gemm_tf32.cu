@@ -42,6 +42,11 @@ namespace dnnf {
 
 namespace tf32 {
 
+#ifdef DNNF_TRACE_LITE
+#define FACC3(slot, v) do {} while (0)
+#else
+#define FACC3(slot, v) FACC(slot, v)
+#endif
 #ifdef DNNF_TRACE
 #define FACC(slot, v) do { if (blockIdx.x == 0 && p.status) atomicAdd(reinterpret_cast<unsigned long long*>(p.status) + 4 + (slot), (unsigned long long)(v)); } while (0)
 #else
@@ -64,6 +69,7 @@ struct Params {
   int32_t npad;              // N rounded up to 16
   int32_t total_tiles;
   int32_t stages;            // raw row blocks in the shared-memory ring
+  int32_t epi_warps;         // 8 epilogue + 4 converter warps, or 4 + 8 when the tile is one 32-column chunk wide
   int32_t rb;                // rows per raw block: 128, 64 or 32
   int32_t pitch;             // floats per shared-memory row of a raw block (the TMA box width; >= K, zero beyond K)
   int32_t unit_stride;       // bytes between ring stages
@@ -207,13 +213,14 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
   uint32_t* stage_area = reinterpret_cast<uint32_t*>(epi);       // general form: EPI_WARPS x kStageWords
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_epi = q.epi_warps, conv_sets = (EPI_WARPS + CONV_WARPS - n_epi) / 4;   // converter sets take chunks in turn
   const int rb = q.rb, units = BM / rb;                            // a raw block holds rb rows; `units` blocks per tile
   pdl_launch_dependents();
   const long long t_begin = clock64();
   if (threadIdx.x == 0) {
-    for (int s = 0; s < stages; ++s) { mbar_init(&raw_bar[s], 1); mbar_init(&empty_bar[s], (uint32_t)(rb / 32)); }
-    for (int s = 0; s < a_stages; ++s) { mbar_init(&conv_bar[s], CONV_WARPS); mbar_init(&afree_bar[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&tfull_bar[s], 1); mbar_init(&tempty_bar[s], EPI_WARPS); }
+    for (int s = 0; s < stages; ++s) { mbar_init(&raw_bar[s], 1); mbar_init(&empty_bar[s], (uint32_t)(rb / 32 * conv_sets)); }
+    for (int s = 0; s < a_stages; ++s) { mbar_init(&conv_bar[s], 4); mbar_init(&afree_bar[s], 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&tfull_bar[s], 1); mbar_init(&tempty_bar[s], (uint32_t)n_epi); }
     mbar_init(b_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -330,10 +337,11 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
         { long long t0 = clock64(); if (!mbar_wait(&tempty_bar[acc], aph ^ 1, abort_flag)) { ok = false; break; } FACC(2, clock64() - t0); }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * acc_cols);
+        const long long t_tile = clock64();
         for (int kc = 0; kc < k_chunks; ++kc, ++it) {
           const int s = it % a_stages;
           const uint32_t ph = (it / a_stages) & 1;
-          { long long t0 = clock64(); if (!mbar_wait(&conv_bar[s], ph, abort_flag)) { ok = false; break; } FACC(3, clock64() - t0); }
+          { long long t0 = clock64(); if (!mbar_wait(&conv_bar[s], ph, abort_flag)) { ok = false; break; } FACC3(3, clock64() - t0); }
           tc_fence_after();
           const long long t_issue = clock64();
           const int ksteps = min(BK, p.K - kc * BK + 7) >> 3;            // 8 tf32 per MMA
@@ -354,15 +362,18 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
             }
           }
           tc_commit(&afree_bar[s]);          // frees the A stage once these MMAs have read it
-          FACC(4, clock64() - t_issue);
+          FACC3(4, clock64() - t_issue);
         }
+        FACC(10, clock64() - t_tile);
         if (ok) tc_commit(&tfull_bar[acc]);  // accumulator complete
       }
+      FACC(11, clock64() - t_begin);
     }
-  } else if (warp >= 2 && warp < 2 + EPI_WARPS) {
+  } else if (warp >= 2 && warp < 2 + n_epi) {
     // ---------------- epilogue warps ----------------
     const int sub = warp & 3;                 // TMEM sub-partition this warp may read
-    const int cgroup = (warp - 2) >> 2;       // takes every second 32-column chunk
+    const int cgroup = (warp - 2) >> 2;       // with 8 warps: takes every second 32-column chunk
+    const int cstep = 8 * n_epi;              // 64 or 32 columns
     uint32_t tcount = 0, nstore = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
@@ -382,7 +393,7 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
         io.row = io.row_ok ? (uint32_t)m : 0u;
         uint32_t raw[32];
         if (cgroup * 32 < p.N) tc_ld32_issue(t_row + cgroup * 32, raw);
-        for (int c = cgroup * 32; c < p.N; c += 64, ++nstore) {
+        for (int c = cgroup * 32; c < p.N; c += cstep, ++nstore) {
           tc_ld_wait();
 #pragma unroll
           for (int j = 0; j < 32; ++j) io.accv[j] = __uint_as_float(raw[j]);
@@ -392,7 +403,7 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
 #pragma unroll
             for (int j = 0; j < 32; ++j) io.accv[j] += __uint_as_float(raw[j]);
           }
-          if (c + 64 < p.N) tc_ld32_issue(t_row + c + 64, raw);      // the next chunk's accumulators fly in during this chunk's work
+          if (c + cstep < p.N) tc_ld32_issue(t_row + c + cstep, raw);      // the next chunk's accumulators fly in during this chunk's work
           io.c = c;
           io.chunk = epi + ((warp - 2) * 2 + (nstore & 1)) * kChunkBytes;
           // the store issued two chunks ago read this buffer: it must have finished reading
@@ -420,7 +431,7 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
           io.row_out[k] = 0;
           if (k < p.n_out) io.row_out[k] = (uint32_t)p.out[k].base + tc_digits(p, p.out[k], p.n_nd, p.m_nd, mm);
         }
-        for (int c = cgroup * 32; c < p.N; c += 64) {
+        for (int c = cgroup * 32; c < p.N; c += cstep) {
           uint32_t raw[32];
           tc_ld32_issue(t_row + c, raw);
           tc_ld_wait();
@@ -451,9 +462,10 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
     }
     if (kFast && lane == 0) tma_store_wait_all();     // shared memory must outlive the last stores' reads
     (void)nstore;
-  } else if (warp >= 2 + EPI_WARPS) {
+  } else if (warp >= 2 + n_epi) {
     // ---------------- converters ----------------
     const int sub = warp & 3;                                  // TMEM sub-partition this warp may write
+    const int set = (warp - 2 - n_epi) >> 2;                   // this set converts the chunks with ia % conv_sets == set
     const int unit = (sub * 32) / rb;                          // which raw block of the tile holds this warp's rows
     const int row = (sub * 32) % rb + lane;                    // this lane's row inside it
     const int pieces = q.pitch >> 2;                           // 16-byte pieces per shared-memory row
@@ -463,9 +475,13 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
       const uint32_t it = tcount * (uint32_t)units + (uint32_t)unit;
       const int s = it % stages;
       // (votes keep the warp together: the tensor-memory stores below are warp-wide)
-      { long long t0 = clock64(); if (!__all_sync(0xffffffffu, mbar_wait(&raw_bar[s], (it / stages) & 1, abort_flag))) { ok = false; break; } if (warp == 10 && lane == 0) FACC(7, clock64() - t0); }
+      { long long t0 = clock64(); if (!__all_sync(0xffffffffu, mbar_wait(&raw_bar[s], (it / stages) & 1, abort_flag))) { ok = false; break; } if (warp == 13 && lane == 0) FACC(7, clock64() - t0); }
       const float4* src = reinterpret_cast<const float4*>(ring + (size_t)s * q.unit_stride) + row * pieces;
       for (int kc = 0; kc < k_chunks; ++kc, ++ia) {
+        if ((int)(ia % (uint32_t)conv_sets) != set) {
+          if (kc == k_chunks - 1) { __syncwarp(); if (lane == 0) mbar_arrive(&empty_bar[s]); }
+          continue;
+        }
         const long long t_cv = clock64();
         const int as = ia % a_stages;
         uint32_t hi[32], lo[32];
@@ -498,7 +514,7 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&conv_bar[as]);
-        if (warp == 10 && lane == 0) FACC(8, clock64() - t_cv);
+        if (warp == 13 && lane == 0) FACC(8, clock64() - t_cv);
       }
     }
   }
@@ -582,6 +598,7 @@ void tf32_gemm_plan(Launch& L) {
   q.dual = 2 * q.npad <= 256 && !getenv("DNNF_TF32_NO_DUAL");
   q.fast_epi = fast_epilogue(gp, q.slot) && !getenv("DNNF_TF32_GENERAL_EPILOGUE");
   q.b_static = gp.static_mask & 1u;
+  q.epi_warps = (gp.N <= 32 && !getenv("DNNF_TF32_EPI8")) ? 4 : 8;
   q.debug = getenv("DNNF_TF32_DEBUG") ? atoi(getenv("DNNF_TF32_DEBUG")) : 0;
   gp.tiles_m = (gp.M + tf32::BM - 1) / tf32::BM;
   gp.tiles_n = 1;

@@ -165,6 +165,22 @@ def test_dwconv3x3_with_epilogue(cfg):
     check(W.Workload(g, ins), RTOL_F32, UNFUSED, expect_blocks=3)
 
 
+# shapes with enough tiles for the TMA-tiled depthwise kernel: ragged H and W, several channel blocks, several items per thread
+@pytest.mark.parametrize("cfg", [(64, 20, 9, 12), (10, 16, 16, 320), (80, 9, 10, 36), (3, 56, 56, 144), (100, 12, 31, 8)])
+def test_dwconv3x3_tma_tiled(cfg):
+    n, h, w, c = cfg
+    g = graph()
+    g.ext("X", (n, h, w, c)); g.ext("Kd", (3, 3, c)); g.ext("s", (c,)); g.ext("t", (c,)); g.ext("R", (n, h, w, c))
+    e = g.add("DwConv3x3", ["X", "Kd"])
+    e = g.add("ScaleShift", [e, "s", "t"], axis=-1)
+    g.mark_output(g.add("Add", [e, "R"], out="Y"))
+    ins = {"X": rnd((n, h, w, c), 21, -1, 1), "Kd": rnd((3, 3, c), 22, -0.5, 0.5), "s": rnd((c,), 23, 0.5, 1.5), "t": rnd((c,), 24, -0.5, 0.5),
+           "R": rnd((n, h, w, c), 25, -1, 1)}
+    s = check(W.Workload(g, ins), RTOL_F32, FUSED, expect_blocks=1)
+    assert s.g.blocks()[0]["variant"] == -1, s.g.blocks()
+    check(W.Workload(g, ins), RTOL_F32, UNFUSED, expect_blocks=3)
+
+
 @pytest.mark.parametrize("cfg", [(2, 14, 14, 24, 144), (32, 56, 56, 24, 144), (1, 3, 5, 8, 16)])
 @pytest.mark.parametrize("flags", [FUSED, UNFUSED])
 def test_mbconv_block(cfg, flags):
