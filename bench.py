@@ -153,6 +153,8 @@ def main():
     ap.add_argument("--no-detail", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time plain dnnf_run launches instead of a captured CUDA graph")
+    ap.add_argument("--branches", type=int, default=4,
+                    help="parallel branches of the captured graph: the step's instances are independent, so they may overlap on the GPU")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -199,15 +201,24 @@ def main():
     if not args.no_graph:
         # The step is launch-bound (48 kernels of a few microseconds): capture it once, replay it.
         # dnnf_run neither allocates nor synchronises, so it can be captured as is.
+        # The instances of a step share no buffer, so the graph gets `branches` parallel chains: a kernel
+        # of one instance may run beside a kernel of another (each fills about a third of the SMs).
         side = torch.cuda.Stream(dev)
+        nbr = max(1, min(args.branches, R_INSTANCES))
+        lanes = [torch.cuda.Stream(dev) for _ in range(nbr - 1)]
         side.wait_stream(stream)
         graphs = []
         with torch.cuda.stream(side):
             for sess in (A, Bn):
                 cg = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(cg, stream=side):
-                    for x in sess:
-                        x.g.run(side.cuda_stream)
+                    for ln in lanes:
+                        ln.wait_stream(side)                       # fork
+                    for i, x in enumerate(sess):
+                        st = side if i % nbr == 0 else lanes[i % nbr - 1]
+                        x.g.run(st.cuda_stream)
+                    for ln in lanes:
+                        side.wait_stream(ln)                       # join
                 graphs.append(cg)
         stream.wait_stream(side)
         part_a, part_b = graphs[0].replay, graphs[1].replay
@@ -239,10 +250,15 @@ def main():
     # ---- roofline of the dominant kernel (the softmax row kernel) ---------------------------------
     dur_a = t_a * 1e-3 / R_INSTANCES
     ach = bytes_a / dur_a / 1e9
-    roof = {"bound": "hbm", "kernel": "row_kernel<4,1,1,4,SP_ScaleMaskSoftmax,true> (scale+mask+softmax, one launch per instance)", "achieved": ach, "peak": pk["hbm_gbs"],
+    def kernel_name(sess):
+        b = sess.g.blocks()[0]
+        v = b["variant"]                          # row family: V*100000 + NV*1000 + WPR*10 + RPW
+        return "row_kernel<V=%d,NV=%d,WPR=%d,RPW=%d> running %s, one launch per instance" % (
+            v // 100000, v // 1000 % 100, v // 10 % 100, v % 10, "+".join(b["ops"]))
+    roof = {"bound": "hbm", "kernel": kernel_name(A[0]), "achieved": ach, "peak": pk["hbm_gbs"],
             "unit": "GB/s", "frac": ach / pk["hbm_gbs"], "peak_source": pk["source"], "traffic": None,
             "bytes_per_launch": bytes_a, "us_per_launch": dur_a * 1e6,
-            "second_kernel": {"kernel": "row_kernel<4,6,1,1,SP_AddLayerNormGelu,true> (add+LayerNorm+GELU)", "bytes_per_launch": bytes_b,
+            "second_kernel": {"kernel": kernel_name(Bn[0]), "bytes_per_launch": bytes_b,
                               "us_per_launch": t_b * 1e3 / R_INSTANCES, "achieved": bytes_b / (t_b * 1e-3 / R_INSTANCES) / 1e9,
                               "frac": bytes_b / (t_b * 1e-3 / R_INSTANCES) / 1e9 / pk["hbm_gbs"]}}
     tp = os.path.join(ROOT, "profiles", "traffic.json")
@@ -294,7 +310,8 @@ def main():
                        "l2": f"inputs larger than L2: {bytes_step / 1e6:.0f} MB of distinct buffers per step",
                        "bytes_per_step": bytes_step, "launches_per_step": 2 * R_INSTANCES,
                        "launch_mode": "plain stream launches" if args.no_graph else
-                       "CUDA-graph replay of the captured step; kernels use programmatic dependent launch"},
+                       ("CUDA-graph replay of the captured step with %d parallel branches over the step's independent instances; "
+                        "kernels use programmatic dependent launch" % max(1, min(args.branches, R_INSTANCES)))},
             "clocks": clk.summary(), "e2e": e2e, "gpu_launches": steps * 2 * R_INSTANCES, "roofline": roof}
 
     if rank == 0 and not args.no_cpu:
