@@ -39,7 +39,9 @@ bool finalize_row(Launch& L) {
   int nv = 0, wpr = 1, rpw = 1;
   // Enough warps to keep every scheduler busy: with few rows a row is split over several warps
   // (shorter per-thread chains), with many short rows a warp takes several rows (more loads in flight).
-  static const long target = getenv("DNNF_ROW_TARGET_WARPS") ? atol(getenv("DNNF_ROW_TARGET_WARPS")) : 148L * 32;
+  // 4000 (27 warps per SM): measured best when independent blocks overlap on the GPU, 6 % slower than
+  // 148 * 32 for a lone 1024-row launch.
+  static const long target = getenv("DNNF_ROW_TARGET_WARPS") ? atol(getenv("DNNF_ROW_TARGET_WARPS")) : 4000L;
   if (V == 4) {
     const int vectors = (Lr + 3) / 4;
     auto fit = [&](int w) { int need = (vectors + 32 * w - 1) / (32 * w); return need; };   // vectors per lane with w warps per row
