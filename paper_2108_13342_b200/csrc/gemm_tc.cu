@@ -83,7 +83,9 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
   if (warp == 0) {
     if (lane == 0) {
       // ---------------- TMA producer ----------------
-      uint32_t it = 0;
+      // (stage index and phase advance by increments: a division by the run-time stage count costs this
+      // single thread some 200 cycles of dependent instructions per k-tile)
+      int s = 0; uint32_t ph = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const int batch = tile / tiles_mn, r = tile - batch * tiles_mn;
@@ -92,13 +94,10 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
         // a batch dim an operand is broadcast over has stride 0 and extent 1 in its tensor map
         const int ab0 = p.A.batch_stride[0] ? b0 : 0, ab1 = p.A.batch_stride[1] ? b1 : 0;
         const int bb0 = p.B.batch_stride[0] ? b0 : 0, bb1 = p.B.batch_stride[1] ? b1 : 0;
-        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
-          const int s = it % stages;
-          const uint32_t ph = (it / stages) & 1;
+        for (int kt = 0; kt < k_tiles; ++kt) {
           if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + (size_t)s * stage_bytes;
           uint8_t* sb = sa + a_bytes;
-          if (it == 0) TRACE(2);
           mbar_expect_tx(&full_bar[s], stage_bytes);
           tma_load_4d(sa, &tmA, &full_bar[s], kt * TC_BK, tm * TC_BM, ab0, ab1);
           if (q.b_kmajor) {
@@ -107,6 +106,7 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
             for (int j = 0; j < BN / 64; ++j)
               tma_load_4d(sb + j * (64 * TC_BK * 2), &tmB, &full_bar[s], tn * BN + j * 64, kt * TC_BK, bb0, bb1);
           }
+          if (++s == stages) { s = 0; ph ^= 1; }
         }
       }
     }
@@ -116,29 +116,30 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
       // instruction descriptor: D fp32, A/B bf16, A K-major, B per operand, N, M=128
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((q.b_kmajor ? 0u : 1u) << 16) | ((uint32_t)(BN >> 3) << 17) |
                              ((uint32_t)(TC_BM >> 4) << 24);
-      uint32_t it = 0, tcount = 0;
+      uint32_t tcount = 0;
+      int s = 0; uint32_t ph = 0;
       bool ok = true;
+      // descriptors of stage 0; a stage further on adds stage_bytes / 16 to the address field, a k-step 2 (32 bytes)
+      // or, for an MN-major B, 128 (2048 bytes)
+      const uint64_t da0 = make_desc(smem_u32(smem), 16, 1024);
+      const uint64_t db0 = q.b_kmajor ? make_desc(smem_u32(smem) + a_bytes, 16, 1024) : make_desc(smem_u32(smem) + a_bytes, 64 * TC_BK * 2, 1024);
+      const uint64_t dstage = stage_bytes >> 4, dbk = q.b_kmajor ? 2 : 128;
+      uint64_t da_s = da0, db_s = db0;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
         const int acc = tcount & 1;
         const uint32_t aph = (tcount >> 1) & 1;
         if (!mbar_wait(&tempty_bar[acc], aph ^ 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
-          const int s = it % stages;
-          const uint32_t ph = (it / stages) & 1;
+        for (int kt = 0; kt < k_tiles; ++kt) {
           if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
-          if (it == 0) TRACE(3);
           tc_fence_after();
-          const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-          const uint32_t sb = sa + a_bytes;
 #pragma unroll
-          for (int kk = 0; kk < TC_BK / 16; ++kk) {
-            const uint64_t da = make_desc(sa + kk * 32, 16, 1024);
-            const uint64_t db = q.b_kmajor ? make_desc(sb + kk * 32, 16, 1024) : make_desc(sb + kk * 2048, 64 * TC_BK * 2, 1024);
-            tc_mma_bf16(d_tmem, da, db, idesc, (kt | kk) ? 1u : 0u);
-          }
+          for (int kk = 0; kk < TC_BK / 16; ++kk)
+            tc_mma_bf16(d_tmem, da_s + 2 * kk, db_s + dbk * kk, idesc, (kt | kk) ? 1u : 0u);
           tc_commit(&empty_bar[s]);          // frees the smem stage once these MMAs have read it
+          da_s += dstage; db_s += dstage;
+          if (++s == stages) { s = 0; ph ^= 1; da_s = da0; db_s = db0; }
         }
         if (ok) tc_commit(&tfull_bar[acc]);  // accumulator complete
         if (tcount == 0) TRACE(4);

@@ -245,14 +245,14 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
   if (warp == 0) {
     if (lane == 0) {
       // ---------------- TMA producer (both CTAs): own 128 rows of A, own half of B ----------------
-      uint32_t it = 0;
+      // (stage index and phase advance by increments: a division by the run-time stage count costs this
+      // single thread some 200 cycles of dependent instructions per k-tile)
+      int s = 0; uint32_t ph = 0;
       bool ok = true;
       for (int tile = pair; tile < total && ok; tile += n_pairs) {
         const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
         const int m0 = tm * 256 + (int)rank * BM, n0 = tn * BN + (int)rank * HB;
-        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
-          const int s = it % stages;
-          const uint32_t ph = (it / stages) & 1;
+        for (int kt = 0; kt < k_tiles; ++kt) {
           { long long t0 = clock64(); if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_flag)) { ok = false; break; } T2ACC(0, clock64() - t0); }
           uint8_t* sa = smem + (size_t)s * stage_bytes;
           uint8_t* sb = sa + a_bytes;
@@ -264,6 +264,7 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
           } else {
             for (int j = 0; j < HB / 64; ++j) tma_load_2d_pair(sb + j * (64 * BK * 2), &q.tmB, lbar, n0 + j * 64, kt * BK);
           }
+          if (++s == stages) { s = 0; ph ^= 1; }
         }
       }
     }
@@ -273,31 +274,34 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
         // ---------------- MMA issuer (leader CTA only) ----------------
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((q.b_kmajor ? 0u : 1u) << 16) | ((uint32_t)(BN >> 3) << 17) |
                                ((uint32_t)(256 >> 4) << 24);
-        uint32_t it = 0, tcount = 0;
+        uint32_t tcount = 0;
+        int s = 0; uint32_t ph = 0;
         bool ok = true;
+        // descriptors of stage 0; a stage further on adds stage_bytes / 16 to the address field, a k-step 2 (32 bytes)
+        // or, for an MN-major B, 128 (2048 bytes); the barriers' cluster addresses are 8 bytes apart
+        const uint64_t da0 = make_desc(smem_u32(smem), 16, 1024);
+        const uint64_t db0 = q.b_kmajor ? make_desc(smem_u32(smem) + a_bytes, 16, 1024) : make_desc(smem_u32(smem) + a_bytes, 64 * BK * 2, 1024);
+        const uint64_t dstage = stage_bytes >> 4, dbk = q.b_kmajor ? 2 : 128;
+        const uint32_t e0 = mapa(smem_u32(&empty_bar[0]), 0), e1 = mapa(smem_u32(&empty_bar[0]), 1);
+        uint64_t da_s = da0, db_s = db0;
         for (int tile = pair; tile < total && ok; tile += n_pairs, ++tcount) {
           const int acc = tcount & 1;
           const uint32_t aph = (tcount >> 1) & 1;
           { long long t0 = clock64(); if (!mbar_wait(&tempty_bar[acc], aph ^ 1, abort_flag)) { ok = false; break; } T2ACC(1, clock64() - t0); }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-          for (int kt = 0; kt < k_tiles; ++kt, ++it) {
-            const int s = it % stages;
-            const uint32_t ph = (it / stages) & 1;
+          for (int kt = 0; kt < k_tiles; ++kt) {
             { long long t0 = clock64(); if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; } T2ACC(2, clock64() - t0); T2ACC(3, 1); }
             tc_fence_after();
-            const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-            const uint32_t sb = sa + a_bytes;
 #pragma unroll
-            for (int kk = 0; kk < BK / 16; ++kk) {
-              const uint64_t da = make_desc(sa + kk * 32, 16, 1024);
-              const uint64_t db = q.b_kmajor ? make_desc(sb + kk * 32, 16, 1024) : make_desc(sb + kk * 2048, 64 * BK * 2, 1024);
-              tc_mma2(d_tmem, da, db, idesc, (kt | kk) ? 1u : 0u);
-            }
+            for (int kk = 0; kk < BK / 16; ++kk)
+              tc_mma2(d_tmem, da_s + 2 * kk, db_s + dbk * kk, idesc, (kt | kk) ? 1u : 0u);
             // stage free in both CTAs once these MMAs have read it.  (Relaying the peer's signal through a helper
             // warp instead of a second commit was measured: the extra hop starves the peer's producer, 40 % slower.)
-            tc_commit2(mapa(smem_u32(&empty_bar[s]), 0));
-            tc_commit2(mapa(smem_u32(&empty_bar[s]), 1));
+            tc_commit2(e0 + 8u * (uint32_t)s);
+            tc_commit2(e1 + 8u * (uint32_t)s);
+            da_s += dstage; db_s += dstage;
+            if (++s == stages) { s = 0; ph ^= 1; da_s = da0; db_s = db0; }
           }
           if (ok) { tc_commit2(mapa(smem_u32(&tfull_bar[acc]), 0)); tc_commit2(mapa(smem_u32(&tfull_bar[acc]), 1)); }
         }

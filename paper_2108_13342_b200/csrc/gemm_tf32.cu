@@ -239,15 +239,16 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
     // ---------------- TMA producer: starts at once, while the other warps still prepare B ----------------
     if (lane == 0) {
       pdl_wait();
-      uint32_t it = 0;
+      // (ring positions and phases advance by increments everywhere: a division by a run-time stage count
+      // costs a lone thread some 200 cycles of dependent instructions)
+      int s = 0; uint32_t ph = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        for (int u = 0; u < units; ++u, ++it) {
-          const int s = it % stages;
-          const uint32_t ph = (it / stages) & 1;
+        for (int u = 0; u < units; ++u) {
           { long long t0 = clock64(); if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_flag)) { ok = false; break; } FACC(1, clock64() - t0); }
           mbar_expect_tx(&raw_bar[s], (uint32_t)(rb * q.pitch * 4));
           tma_load_2d(ring + (size_t)s * q.unit_stride, &q.tmA, &raw_bar[s], 0, tile * BM + u * rb);
+          if (++s == stages) { s = 0; ph ^= 1; }
         }
       }
     }
@@ -329,8 +330,10 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
       const uint32_t idesc = idesc0 | ((uint32_t)(NP >> 3) << 17), idesc2 = idesc0 | ((uint32_t)(NP >> 2) << 17);
       const uint32_t b_base = smem_u32(smem);
       const bool dual = q.dual != 0;
-      uint32_t it = 0, tcount = 0;
+      uint32_t tcount = 0;
+      int s = 0; uint32_t ph = 0;
       bool ok = true;
+      const uint64_t db0 = make_desc(b_base, 16, 1024);          // B_hi of K atom 0; + atom_bytes / 16 per atom, + lo_off / 16 for B_lo
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
         const int acc = tcount & 1;
         const uint32_t aph = (tcount >> 1) & 1;
@@ -338,30 +341,37 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * acc_cols);
         const long long t_tile = clock64();
-        for (int kc = 0; kc < k_chunks; ++kc, ++it) {
-          const int s = it % a_stages;
-          const uint32_t ph = (it / a_stages) & 1;
+        uint64_t dbh = db0;
+        int k_left = p.K;
+        for (int kc = 0; kc < k_chunks; ++kc, k_left -= BK, dbh += atom_bytes >> 4) {
           { long long t0 = clock64(); if (!mbar_wait(&conv_bar[s], ph, abort_flag)) { ok = false; break; } FACC3(3, clock64() - t0); }
           tc_fence_after();
           const long long t_issue = clock64();
-          const int ksteps = min(BK, p.K - kc * BK + 7) >> 3;            // 8 tf32 per MMA
-          uint32_t a_hi = tmem_base + a_cols0 + (uint32_t)(s * kAStageCols), a_lo = a_hi + BK;
+          const int ksteps = min(BK, k_left + 7) >> 3;                   // 8 tf32 per MMA
+          const uint32_t a_hi = tmem_base + a_cols0 + (uint32_t)(s * kAStageCols), a_lo = a_hi + BK;
           // B descriptors advance by 32 bytes (2 units of 16) per k-step inside the swizzled atom
-          uint64_t dbh = make_desc(b_base + (uint32_t)kc * atom_bytes, 16, 1024), dbl = make_desc(b_base + (uint32_t)kc * atom_bytes + lo_off, 16, 1024);
+          const uint64_t dbl = dbh + (lo_off >> 4);
           if (q.debug & 2) {
           } else if (dual) {
-            for (int kk = 0; kk < ksteps; ++kk, a_hi += 8, a_lo += 8, dbh += 2) {
-              mma_tf32_ts(d_tmem, a_hi, dbh, idesc2, (kc | kk) ? 1u : 0u);   // [A_hi B_hi | A_hi B_lo]
-              mma_tf32_ts(d_tmem, a_lo, dbh, idesc, 1u);                    // + A_lo B_hi on the first range
+#pragma unroll
+            for (int kk = 0; kk < BK / 8; ++kk) {
+              if (kk < ksteps) {
+                mma_tf32_ts(d_tmem, a_hi + 8 * kk, dbh + 2 * kk, idesc2, (kc | kk) ? 1u : 0u);   // [A_hi B_hi | A_hi B_lo]
+                mma_tf32_ts(d_tmem, a_lo + 8 * kk, dbh + 2 * kk, idesc, 1u);                    // + A_lo B_hi on the first range
+              }
             }
           } else {
-            for (int kk = 0; kk < ksteps; ++kk, a_hi += 8, a_lo += 8, dbh += 2, dbl += 2) {
-              mma_tf32_ts(d_tmem, a_lo, dbh, idesc, (kc | kk) ? 1u : 0u);   // small terms first
-              mma_tf32_ts(d_tmem, a_hi, dbl, idesc, 1u);
-              mma_tf32_ts(d_tmem, a_hi, dbh, idesc, 1u);
+#pragma unroll
+            for (int kk = 0; kk < BK / 8; ++kk) {
+              if (kk < ksteps) {
+                mma_tf32_ts(d_tmem, a_lo + 8 * kk, dbh + 2 * kk, idesc, (kc | kk) ? 1u : 0u);   // small terms first
+                mma_tf32_ts(d_tmem, a_hi + 8 * kk, dbl + 2 * kk, idesc, 1u);
+                mma_tf32_ts(d_tmem, a_hi + 8 * kk, dbh + 2 * kk, idesc, 1u);
+              }
             }
           }
           tc_commit(&afree_bar[s]);          // frees the A stage once these MMAs have read it
+          if (++s == a_stages) { s = 0; ph ^= 1; }
           FACC3(4, clock64() - t_issue);
         }
         FACC(10, clock64() - t_tile);
@@ -469,21 +479,23 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
     const int unit = (sub * 32) / rb;                          // which raw block of the tile holds this warp's rows
     const int row = (sub * 32) % rb + lane;                    // this lane's row inside it
     const int pieces = q.pitch >> 2;                           // 16-byte pieces per shared-memory row
-    uint32_t tcount = 0, ia = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-      const uint32_t it = tcount * (uint32_t)units + (uint32_t)unit;
-      const int s = it % stages;
+    // raw-block ring position of this warp's block (advances by `units` per tile) and A-stage ring position
+    int s = unit % stages; uint32_t rph = (uint32_t)(unit / stages) & 1;
+    int as = 0, turn = 0; uint32_t aph = 0;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       // (votes keep the warp together: the tensor-memory stores below are warp-wide)
-      { long long t0 = clock64(); if (!__all_sync(0xffffffffu, mbar_wait(&raw_bar[s], (it / stages) & 1, abort_flag))) { ok = false; break; } if (warp == 13 && lane == 0) FACC(7, clock64() - t0); }
+      { long long t0 = clock64(); if (!__all_sync(0xffffffffu, mbar_wait(&raw_bar[s], rph, abort_flag))) { ok = false; break; } if (warp == 13 && lane == 0) FACC(7, clock64() - t0); }
       const float4* src = reinterpret_cast<const float4*>(ring + (size_t)s * q.unit_stride) + row * pieces;
-      for (int kc = 0; kc < k_chunks; ++kc, ++ia) {
-        if ((int)(ia % (uint32_t)conv_sets) != set) {
+      for (int kc = 0; kc < k_chunks; ++kc) {
+        const bool mine = turn == set;
+        if (++turn == conv_sets) turn = 0;
+        if (!mine) {
           if (kc == k_chunks - 1) { __syncwarp(); if (lane == 0) mbar_arrive(&empty_bar[s]); }
+          if (++as == a_stages) { as = 0; aph ^= 1; }
           continue;
         }
         const long long t_cv = clock64();
-        const int as = ia % a_stages;
         uint32_t hi[32], lo[32];
         if (!(q.debug & 1)) {
 #pragma unroll
@@ -503,7 +515,7 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
           __syncwarp();
           if (lane == 0) mbar_arrive(&empty_bar[s]);
         }
-        if (!__all_sync(0xffffffffu, mbar_wait(&afree_bar[as], ((ia / a_stages) & 1) ^ 1, abort_flag))) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait(&afree_bar[as], aph ^ 1, abort_flag))) { ok = false; break; }
         if (!(q.debug & 1)) {
           tc_fence_after();
           const uint32_t t_a = tmem_base + ((uint32_t)(sub * 32) << 16) + a_cols0 + (uint32_t)(as * kAStageCols);
@@ -515,7 +527,10 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
         __syncwarp();
         if (lane == 0) mbar_arrive(&conv_bar[as]);
         if (warp == 13 && lane == 0) FACC(8, clock64() - t_cv);
+        if (++as == a_stages) { as = 0; aph ^= 1; }
       }
+      s += units;
+      while (s >= stages) { s -= stages; rph ^= 1; }
     }
   }
 

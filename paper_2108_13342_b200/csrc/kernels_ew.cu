@@ -53,6 +53,7 @@ struct EwIO {
     for (int v = 0; v < V * U; ++v) dst[v] = 0.0f;
   }
   __device__ __forceinline__ void store(int idx, const float (&val)[V * U]) const {
+    pdl_launch_dependents();       // loads are done: the next kernel's CTAs may start arriving (first trigger counts)
     const TensorArg& a = p.out[idx];
     const int si = a.stride[0];
     const bool exact = p.prog.flags & kProgPureMove;
@@ -74,7 +75,6 @@ struct EwIO {
 // contiguous one), so that every index below is a compile-time constant.
 template <int V, int U, class SP, bool F32>
 __global__ void __launch_bounds__(256) ew_kernel(const __grid_constant__ EwParams p) {
-  pdl_launch_dependents();
   EwIO<V, U, F32> io{p};
   const uint32_t nvec = (uint32_t)(p.total / V);
 #pragma unroll

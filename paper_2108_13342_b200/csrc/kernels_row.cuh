@@ -83,6 +83,10 @@ struct RowIO {
     }
   }
   __device__ __forceinline__ void row_reduce(int op, float (&acc)[VV]) const {
+    // The row's loads have been issued by now: let the next kernel's CTAs start arriving.  (Triggering at
+    // kernel entry parks them on the SMs for this kernel's whole load latency, where they take the
+    // slots of independent kernels that could run.)  Only the first trigger of a CTA counts.
+    pdl_launch_dependents();
     float red[RPW];
 #pragma unroll
     for (int r = 0; r < RPW; ++r) {
@@ -135,7 +139,6 @@ template <int V, int NV, int WPR, int RPW, class SP, bool F32>
 __global__ void __launch_bounds__(WPR > 1 ? 32 * WPR : 32 * kRowWarpsPerCta)
 row_kernel(const __grid_constant__ RowParams p) {
   __shared__ float xchg[WPR > 1 ? WPR : 1];
-  pdl_launch_dependents();
   RowIO<V, NV, WPR, RPW, F32> io{p};
   io.xchg = xchg;
   uint32_t row0;
