@@ -52,6 +52,7 @@ struct Params {
   int32_t b_kmajor, k_tiles, bn, total_tiles, tiles_n;
   int32_t c_input;           // index of the epilogue input that is a full tile (TMA-loaded), or -1
   int32_t stages;
+  int32_t kpack;             // 64-wide k-tiles per ring stage (1 or 2): one wait, one pair of commits per stage
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -204,8 +205,8 @@ __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Params q) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int BN = q.bn, HB = BN / 2, stages = q.stages;
-  const uint32_t a_bytes = BM * BK * 2, b_bytes = (uint32_t)HB * BK * 2, stage_bytes = a_bytes + b_bytes;
+  const int BN = q.bn, HB = BN / 2, stages = q.stages, kpack = q.kpack;
+  const uint32_t a_bytes = BM * BK * 2, b_bytes = (uint32_t)HB * BK * 2, sub_bytes = a_bytes + b_bytes, stage_bytes = sub_bytes * (uint32_t)kpack;
   uint8_t* epi = smem + (size_t)stages * stage_bytes;                  // 1024-aligned (stage_bytes is a multiple of 1024)
   uint64_t* bars = reinterpret_cast<uint64_t*>(epi + kEpiBytes);
   uint64_t* full_bar = bars;                  // [stages]  used in the leader only: 1 arrival + the bytes of BOTH CTAs
@@ -252,17 +253,21 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
       for (int tile = pair; tile < total && ok; tile += n_pairs) {
         const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
         const int m0 = tm * 256 + (int)rank * BM, n0 = tn * BN + (int)rank * HB;
-        for (int kt = 0; kt < k_tiles; ++kt) {
+        for (int kt = 0; kt < k_tiles; kt += kpack) {
           { long long t0 = clock64(); if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_flag)) { ok = false; break; } T2ACC(0, clock64() - t0); }
-          uint8_t* sa = smem + (size_t)s * stage_bytes;
-          uint8_t* sb = sa + a_bytes;
           const uint32_t lbar = mapa(smem_u32(&full_bar[s]), 0);
           if (leader) mbar_expect_tx(&full_bar[s], 2 * stage_bytes);
-          tma_load_2d_pair(sa, &q.tmA, lbar, kt * BK, m0);
-          if (q.b_kmajor) {
-            tma_load_2d_pair(sb, &q.tmB, lbar, kt * BK, n0);
-          } else {
-            for (int j = 0; j < HB / 64; ++j) tma_load_2d_pair(sb + j * (64 * BK * 2), &q.tmB, lbar, n0 + j * 64, kt * BK);
+          // (a k-tile past K, when k_tiles is odd and kpack is 2, arrives as zeros: its MMAs add nothing)
+          for (int u = 0; u < kpack; ++u) {
+            uint8_t* sa = smem + (size_t)s * stage_bytes + (size_t)u * sub_bytes;
+            uint8_t* sb = sa + a_bytes;
+            const int k0 = (kt + u) * BK;
+            tma_load_2d_pair(sa, &q.tmA, lbar, k0, m0);
+            if (q.b_kmajor) {
+              tma_load_2d_pair(sb, &q.tmB, lbar, k0, n0);
+            } else {
+              for (int j = 0; j < HB / 64; ++j) tma_load_2d_pair(sb + j * (64 * BK * 2), &q.tmB, lbar, n0 + j * 64, k0);
+            }
           }
           if (++s == stages) { s = 0; ph ^= 1; }
         }
@@ -281,7 +286,7 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
         // or, for an MN-major B, 128 (2048 bytes); the barriers' cluster addresses are 8 bytes apart
         const uint64_t da0 = make_desc(smem_u32(smem), 16, 1024);
         const uint64_t db0 = q.b_kmajor ? make_desc(smem_u32(smem) + a_bytes, 16, 1024) : make_desc(smem_u32(smem) + a_bytes, 64 * BK * 2, 1024);
-        const uint64_t dstage = stage_bytes >> 4, dbk = q.b_kmajor ? 2 : 128;
+        const uint64_t dstage = stage_bytes >> 4, dsub = sub_bytes >> 4, dbk = q.b_kmajor ? 2 : 128;
         const uint32_t e0 = mapa(smem_u32(&empty_bar[0]), 0), e1 = mapa(smem_u32(&empty_bar[0]), 1);
         uint64_t da_s = da0, db_s = db0;
         for (int tile = pair; tile < total && ok; tile += n_pairs, ++tcount) {
@@ -290,12 +295,17 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
           { long long t0 = clock64(); if (!mbar_wait(&tempty_bar[acc], aph ^ 1, abort_flag)) { ok = false; break; } T2ACC(1, clock64() - t0); }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-          for (int kt = 0; kt < k_tiles; ++kt) {
+          for (int kt = 0; kt < k_tiles; kt += kpack) {
             { long long t0 = clock64(); if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; } T2ACC(2, clock64() - t0); T2ACC(3, 1); }
             tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < BK / 16; ++kk)
               tc_mma2(d_tmem, da_s + 2 * kk, db_s + dbk * kk, idesc, (kt | kk) ? 1u : 0u);
+            if (kpack == 2) {
+#pragma unroll
+              for (int kk = 0; kk < BK / 16; ++kk)
+                tc_mma2(d_tmem, da_s + dsub + 2 * kk, db_s + dsub + dbk * kk, idesc, 1u);
+            }
             // stage free in both CTAs once these MMAs have read it.  (Relaying the peer's signal through a helper
             // warp instead of a second commit was measured: the extra hop starves the peer's producer, 40 % slower.)
             tc_commit2(e0 + 8u * (uint32_t)s);
@@ -470,7 +480,12 @@ void tc2_gemm_plan(Launch& L) {
   q.tiles_n = (gp.N + q.bn - 1) / q.bn;
   q.total_tiles = tiles_m * q.tiles_n;
   gp.tiles_m = tiles_m; gp.tiles_n = q.tiles_n;
-  const int stage_bytes = tc2::BM * tc2::BK * 2 + (q.bn / 2) * tc2::BK * 2;
+  const int sub_bytes = tc2::BM * tc2::BK * 2 + (q.bn / 2) * tc2::BK * 2;
+  // two k-tiles per stage halve the issuing thread's per-stage cost (wait, fence, two commits); worth it when its
+  // MMAs are short (BN = 128) or the k loop is long, as long as three stages still fit
+  q.kpack = (q.k_tiles >= 4 && tc2::kRingBudget / (2 * sub_bytes) >= 3) ? 2 : 1;
+  if (getenv("DNNF_PAIR_KPACK")) q.kpack = atoi(getenv("DNNF_PAIR_KPACK")) == 2 ? 2 : 1;
+  const int stage_bytes = sub_bytes * q.kpack;
   q.stages = std::min(8, tc2::kRingBudget / stage_bytes);
   q.c_input = -1;
   int vec_slot = 0;
