@@ -401,9 +401,9 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
         const int m = tile * BM + sub * 32 + lane;
         io.row_ok = m < p.M;
         io.row = io.row_ok ? (uint32_t)m : 0u;
-        uint32_t raw[32];
-        if (cgroup * 32 < p.N) tc_ld32_issue(t_row + cgroup * 32, raw);
         for (int c = cgroup * 32; c < p.N; c += cstep, ++nstore) {
+          uint32_t raw[32];
+          tc_ld32_issue(t_row + c, raw);
           tc_ld_wait();
 #pragma unroll
           for (int j = 0; j < 32; ++j) io.accv[j] = __uint_as_float(raw[j]);
@@ -413,7 +413,6 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
 #pragma unroll
             for (int j = 0; j < 32; ++j) io.accv[j] += __uint_as_float(raw[j]);
           }
-          if (c + cstep < p.N) tc_ld32_issue(t_row + c + cstep, raw);      // the next chunk's accumulators fly in during this chunk's work
           io.c = c;
           io.chunk = epi + ((warp - 2) * 2 + (nstore & 1)) * kChunkBytes;
           // the store issued two chunks ago read this buffer: it must have finished reading

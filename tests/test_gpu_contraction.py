@@ -39,7 +39,7 @@ def test_ffn_block(cfg, flags):
         assert all(b["variant"] in (1, 3) for b in s.g.blocks()), "expected a tensor-core kernel"
 
 
-@pytest.mark.parametrize("mnk", [(256, 128, 64), (300, 200, 72), (1000, 328, 264), (257, 136, 8), (512, 2304, 768)])
+@pytest.mark.parametrize("mnk", [(256, 128, 64), (300, 200, 72), (1000, 328, 264), (257, 136, 8), (512, 2304, 768), (512, 128, 448)])
 @pytest.mark.parametrize("kmajor_b", [False, True])
 @pytest.mark.parametrize("epi", ["none", "bias_gelu", "bias_residual"])
 def test_pair_gemm_shapes_and_epilogues(mnk, kmajor_b, epi):
