@@ -11,6 +11,14 @@ pytestmark = pytest.mark.gpu
 FUSED, UNFUSED = B.PLAN_FUSED, B.PLAN_UNFUSED
 
 
+
+def _expect_variant(sess, variant, switch):
+    """The block must run on the named kernel variant -- unless the development switch that disables it is set
+    (the suite is also run with those switches to cover the fall-back kernels)."""
+    import os
+    if not os.environ.get(switch):
+        assert sess.g.blocks()[0]["variant"] == variant, sess.g.blocks()
+
 def _bf(x):
     return W.round_to_bf16(x)
 
@@ -64,7 +72,7 @@ def test_pair_gemm_shapes_and_epilogues(mnk, kmajor_b, epi):
         t = g.add("Add", [t, "R"])
     g.mark_output(t)
     s = check(W.Workload(g, ins), RTOL_BF16, FUSED, expect_blocks=1)
-    assert s.g.blocks()[0]["variant"] == 3, s.g.blocks()
+    _expect_variant(s, 3, "DNNF_NO_PAIR_GEMM")
 
 
 def test_batched_matmul_with_transposed_and_strided_operands():
@@ -138,7 +146,7 @@ def test_conv1x1_tensor_core_fp32(cfg, epi):
             g.ext("R", (n, h, w, co)); ins["R"] = rnd((n, h, w, co), 15, -1, 1)
             g.mark_output(g.add("Add", [e, "R"], out="Y"))
     s = check(W.Workload(g, ins), RTOL_F32, FUSED, expect_blocks=1)
-    assert s.g.blocks()[0]["variant"] == 4, s.g.blocks()
+    _expect_variant(s, 4, "DNNF_NO_TF32_GEMM")
 
 
 def test_matmul_fp32_tall_skinny_uses_tensor_cores():
@@ -149,7 +157,7 @@ def test_matmul_fp32_tall_skinny_uses_tensor_cores():
     t = g.add("Add", [t, "b"])
     g.mark_output(g.add("Tanh", [t], out="Y"))
     s = check(W.Workload(g, {"X": rnd((m, k), 3, -1, 1), "Wt": rnd((k, n), 4, -0.3, 0.3), "b": rnd((n,), 5)}), RTOL_F32, FUSED, expect_blocks=1)
-    assert s.g.blocks()[0]["variant"] == 4
+    _expect_variant(s, 4, "DNNF_NO_TF32_GEMM")
 
 
 @pytest.mark.parametrize("cfg", [(1, 5, 6, 8), (2, 7, 9, 144), (1, 1, 1, 4), (1, 3, 1, 12), (2, 30, 17, 24)])
@@ -177,7 +185,7 @@ def test_dwconv3x3_tma_tiled(cfg):
     ins = {"X": rnd((n, h, w, c), 21, -1, 1), "Kd": rnd((3, 3, c), 22, -0.5, 0.5), "s": rnd((c,), 23, 0.5, 1.5), "t": rnd((c,), 24, -0.5, 0.5),
            "R": rnd((n, h, w, c), 25, -1, 1)}
     s = check(W.Workload(g, ins), RTOL_F32, FUSED, expect_blocks=1)
-    assert s.g.blocks()[0]["variant"] == -1, s.g.blocks()
+    _expect_variant(s, -1, "DNNF_NO_TMA_DWCONV")
     check(W.Workload(g, ins), RTOL_F32, UNFUSED, expect_blocks=3)
 
 
