@@ -233,7 +233,12 @@ DNNF_API int dnnf_op_kind(const dnnf_graph* g, int op_index, int* kind, int* ali
 DNNF_API int dnnf_workspace_size(const dnnf_graph* g, size_t* bytes);
 /* dev_ptr: device memory of the tensor's full size, 16-byte aligned, caller-owned. */
 DNNF_API int dnnf_bind(dnnf_graph* g, int tensor_id, void* dev_ptr);
-/* dev_ptr: device memory, 256-byte aligned, at least dnnf_workspace_size bytes. */
+/* The first *bytes of the workspace (status words, then arrival counters of split-K GEMM blocks;
+ * at least 256) must be zero when a run starts.  A run that returns DNNF_OK leaves them zero; after
+ * a failed run (dnnf_status != DNNF_OK) the caller clears them again. */
+DNNF_API int dnnf_workspace_zero_bytes(const dnnf_graph* g, size_t* bytes);
+/* dev_ptr: device memory, 256-byte aligned, at least dnnf_workspace_size bytes, its first
+ * dnnf_workspace_zero_bytes bytes zero. */
 DNNF_API int dnnf_bind_workspace(dnnf_graph* g, void* dev_ptr, size_t bytes);
 /* Launches every block's kernel in topological order on `cuda_stream`
  * (a cudaStream_t; NULL = default stream).  Asynchronous. */

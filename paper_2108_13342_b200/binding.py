@@ -69,7 +69,7 @@ class BlockDesc(C.Structure):
 EXPORTS = ["dnnf_graph_create", "dnnf_graph_destroy", "dnnf_add_tensor", "dnnf_add_op", "dnnf_mark_output",
            "dnnf_tensor_info", "dnnf_op_mapping", "dnnf_mapping_check", "dnnf_rewrite", "dnnf_rule_name", "dnnf_plan",
            "dnnf_block_count", "dnnf_block_info", "dnnf_block_program", "dnnf_op_block", "dnnf_op_count", "dnnf_op_kind",
-           "dnnf_workspace_size", "dnnf_bind", "dnnf_bind_workspace", "dnnf_run", "dnnf_run_static_ws", "dnnf_run_block", "dnnf_status",
+           "dnnf_workspace_size", "dnnf_workspace_zero_bytes", "dnnf_bind", "dnnf_bind_workspace", "dnnf_run", "dnnf_run_static_ws", "dnnf_run_block", "dnnf_status",
            "dnnf_launch_count", "dnnf_last_error", "dnnf_version"]
 
 
@@ -101,6 +101,7 @@ def _load():
     lib.dnnf_op_count.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
     lib.dnnf_op_kind.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     lib.dnnf_workspace_size.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
+    lib.dnnf_workspace_zero_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
     lib.dnnf_bind.argtypes = [C.c_void_p, C.c_int, C.c_void_p]
     lib.dnnf_bind_workspace.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
     lib.dnnf_run.argtypes = [C.c_void_p, C.c_void_p]
@@ -231,6 +232,11 @@ class Graph:
     def workspace_size(self):
         n = C.c_size_t()
         self._check(lib.dnnf_workspace_size(self.h, C.byref(n)))
+        return n.value
+
+    def workspace_zero_bytes(self):
+        n = C.c_size_t(0)
+        self._check(lib.dnnf_workspace_zero_bytes(self.h, C.byref(n)))
         return n.value
 
     def bind(self, tid, dev_ptr):

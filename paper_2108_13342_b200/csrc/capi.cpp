@@ -274,6 +274,13 @@ int dnnf_bind(dnnf_graph* g, int t, void* dev_ptr) {
   return DNNF_OK;
 }
 
+int dnnf_workspace_zero_bytes(const dnnf_graph* g, size_t* bytes) {
+  if (!g || !bytes) return DNNF_ERR_INVALID_ARG;
+  if (!g->g.planned) return DNNF_ERR_STATE;
+  *bytes = g->g.ws_zero_bytes;
+  return DNNF_OK;
+}
+
 int dnnf_bind_workspace(dnnf_graph* g, void* dev_ptr, size_t bytes) {
   if (!g) return DNNF_ERR_INVALID_ARG;
   Graph& G = g->g;

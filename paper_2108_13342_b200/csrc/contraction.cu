@@ -27,6 +27,7 @@ bool tc2_gemm_eligible(const GemmParams& gp);
 void tc2_gemm_plan(Launch& L);
 bool tc2_gemm_prepare(Launch& L, std::string& err);
 int tc2_gemm_launch(const Launch& L, cudaStream_t st);
+void tc2_set_scratch(Launch& L, void* ws_base);
 size_t tf32_blob_bytes();
 bool tf32_gemm_eligible(const GemmParams& gp);
 void tf32_gemm_plan(Launch& L);
@@ -484,6 +485,7 @@ int launch_contraction(const Launch& L, void* status_words, int block_index, cud
   if (L.variant == 3) {
     Launch& M = const_cast<Launch&>(L);
     gp_of(M).status = gp.status; gp_of(M).block_index = block_index;
+    tc2_set_scratch(M, status_words);
     int rc = tc2_gemm_launch(L, st);
     if (rc) err = "tensor-core pair GEMM launch failed";
     return rc;

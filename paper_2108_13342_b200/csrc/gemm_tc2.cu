@@ -15,6 +15,10 @@
 // Both CTAs' operand loads count their bytes on the leader's barrier (cta_group::2 form of the
 // TMA load, single destination); stage release and accumulator hand-over use single-target
 // tcgen05.commit / mbarrier arrives on cluster shared-memory addresses.
+// Split-K (few output tiles, long K): `ksplit` CTA pairs each accumulate a slice of K for the same tile.  Per
+// 32 x 64 chunk a warp writes its partial accumulators to scratch and bumps the chunk's counter; the warp whose
+// bump is the last adds the other partials to its own (L2 reads), runs the epilogue program and stores.
+// Nobody waits for anybody, and the last warp puts the counter back to zero.
 // Every wait is bounded; on expiry the CTA pair records DNNF_ERR_TIMEOUT, stops and releases
 // tensor memory.
 #include <cuda.h>
@@ -53,6 +57,10 @@ struct Params {
   int32_t c_input;           // index of the epilogue input that is a full tile (TMA-loaded), or -1
   int32_t stages;
   int32_t kpack;             // 64-wide k-tiles per ring stage (1 or 2): one wait, one pair of commits per stage
+  int32_t ksplit;            // CTA pairs that share one output tile, each with kt_per k-tiles of the K range (1: no split)
+  int32_t kt_per;
+  float* scratch;            // split-K partial accumulators: [unit][ksplit][64 cols][32 rows] fp32
+  int32_t* counters;         // split-K arrival counters, one per unit (a warp's 32 x 64 chunk); zero between runs
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -241,7 +249,8 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
   const long long t_begin = clock64();
 
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int total = q.total_tiles, k_tiles = q.k_tiles, tiles_n = q.tiles_n;
+  const int n_tiles = q.total_tiles, k_tiles = q.k_tiles, tiles_n = q.tiles_n;
+  const int total = n_tiles * q.ksplit;        // work items: (tile, K slice); item = slice * n_tiles + tile
 
   if (warp == 0) {
     if (lane == 0) {
@@ -250,10 +259,12 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
       // single thread some 200 cycles of dependent instructions per k-tile)
       int s = 0; uint32_t ph = 0;
       bool ok = true;
-      for (int tile = pair; tile < total && ok; tile += n_pairs) {
+      for (int item = pair; item < total && ok; item += n_pairs) {
+        const int ks = item / n_tiles, tile = item - ks * n_tiles;
         const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
         const int m0 = tm * 256 + (int)rank * BM, n0 = tn * BN + (int)rank * HB;
-        for (int kt = 0; kt < k_tiles; kt += kpack) {
+        const int kt_end = min(k_tiles, (ks + 1) * q.kt_per);
+        for (int kt = ks * q.kt_per; kt < kt_end; kt += kpack) {
           { long long t0 = clock64(); if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_flag)) { ok = false; break; } T2ACC(0, clock64() - t0); }
           const uint32_t lbar = mapa(smem_u32(&full_bar[s]), 0);
           if (leader) mbar_expect_tx(&full_bar[s], 2 * stage_bytes);
@@ -289,18 +300,20 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
         const uint64_t dstage = stage_bytes >> 4, dsub = sub_bytes >> 4, dbk = q.b_kmajor ? 2 : 128;
         const uint32_t e0 = mapa(smem_u32(&empty_bar[0]), 0), e1 = mapa(smem_u32(&empty_bar[0]), 1);
         uint64_t da_s = da0, db_s = db0;
-        for (int tile = pair; tile < total && ok; tile += n_pairs, ++tcount) {
+        for (int item = pair; item < total && ok; item += n_pairs, ++tcount) {
           const int acc = tcount & 1;
           const uint32_t aph = (tcount >> 1) & 1;
           { long long t0 = clock64(); if (!mbar_wait(&tempty_bar[acc], aph ^ 1, abort_flag)) { ok = false; break; } T2ACC(1, clock64() - t0); }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-          for (int kt = 0; kt < k_tiles; kt += kpack) {
+          const int ks = item / n_tiles;
+          const int kt_begin = ks * q.kt_per, kt_end = min(k_tiles, kt_begin + q.kt_per);
+          for (int kt = kt_begin; kt < kt_end; kt += kpack) {
             { long long t0 = clock64(); if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; } T2ACC(2, clock64() - t0); T2ACC(3, 1); }
             tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < BK / 16; ++kk)
-              tc_mma2(d_tmem, da_s + 2 * kk, db_s + dbk * kk, idesc, (kt | kk) ? 1u : 0u);
+              tc_mma2(d_tmem, da_s + 2 * kk, db_s + dbk * kk, idesc, ((kt - kt_begin) | kk) ? 1u : 0u);
             if (kpack == 2) {
 #pragma unroll
               for (int kk = 0; kk < BK / 16; ++kk)
@@ -330,15 +343,18 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
     uint32_t tcount = 0, ccount = 0;                                // tiles and chunks processed by this warp
     bool ok = true;
     // prefetch of the residual chunk `g` (global chunk counter of this warp) into buffer g & 1
-    auto prefetch = [&](int tile, int c, uint32_t g) {
+    auto prefetch = [&](int item, int c, uint32_t g) {
       if (q.c_input < 0 || lane != 0) return;
+      const int tile = item % n_tiles;
       const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
       const int m0 = tm * 256 + (int)rank * BM + sub * 32, n0 = tn * BN + half * cols_per_warp + c * 64;
       mbar_expect_tx(&my_cbar[g & 1], kChunkBytes);
       tma_load_2d(cbuf + (g & 1) * kChunkBytes, &q.tmC, &my_cbar[g & 1], n0, m0);
     };
+    const int S = q.ksplit;
     if (pair < total) prefetch(pair, 0, 0);
-    for (int tile = pair; tile < total && ok; tile += n_pairs, ++tcount) {
+    for (int item = pair; item < total && ok; item += n_pairs, ++tcount) {
+      const int ks = item / n_tiles, tile = item - ks * n_tiles;
       const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
       const int m0 = tm * 256 + (int)rank * BM + sub * 32;
       const int nw0 = tn * BN + half * cols_per_warp;
@@ -363,22 +379,50 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
         // the other buffer is free once the store issued from it two chunks ago has been read out
         if (lane == 0) tma_store_wait_read();
         __syncwarp();
-        {   // prefetch the next residual chunk (possibly of the next tile) into the other buffer
-          int nt = tile, nc = c + 1;
-          if (nc == chunks) { nt = tile + n_pairs; nc = 0; }
+        {   // prefetch the next residual chunk (possibly of the next item) into the other buffer
+          int nt = item, nc = c + 1;
+          if (nc == chunks) { nt = item + n_pairs; nc = 0; }
           if (nt < total) prefetch(nt, nc, ccount + 1);
         }
         if (q.c_input >= 0) { if (!mbar_wait(&my_cbar[buf], (ccount >> 1) & 1, abort_flag)) { ok = false; break; } }
+        // ---- split-K: hand in this slice's partial chunk; only the last slice to arrive carries on ----
+        const float* others = nullptr;
+        if (S > 1) {
+          const uint32_t unit = (((uint32_t)tile * 2u + rank) * EPI_WARPS + (uint32_t)ew) * (uint32_t)chunks + (uint32_t)c;
+          float* mine = q.scratch + ((size_t)unit * S + ks) * 2048;
+#pragma unroll 1
+          for (int h = 0; h < 2; ++h) {
+            uint32_t raw[32];
+            tc_ld32(t_row + c * 64 + h * 32, raw);
+            tc_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mine[(h * 32 + i) * 32 + lane] = __uint_as_float(raw[i]);     // a 128-byte line per instruction
+          }
+          __threadfence();                       // this lane's partials are visible before the counter moves
+          __syncwarp();
+          int old = 0;
+          if (lane == 0) old = atomicAdd(&q.counters[unit], 1);
+          old = __shfl_sync(0xffffffffu, old, 0);
+          if (old != S - 1) continue;            // somebody else finishes this chunk (uniform over the warp)
+          if (lane == 0) q.counters[unit] = 0;   // all S slices have arrived: ready for the next run
+          __threadfence();
+          others = q.scratch + (size_t)unit * S * 2048;
+        }
 #pragma unroll 1
         for (int h = 0; h < 2; ++h) {
-          if (tn * BN + half * cols_per_warp + c * 64 + h * 32 >= p.N && h == 1) {
-            // columns beyond N in the second half: still fill the buffer with zeros (TMA clips them anyway)
-          }
           uint32_t raw[32];
           tc_ld32(t_row + c * 64 + h * 32, raw);
           tc_ld_wait();
 #pragma unroll
           for (int i = 0; i < 32; ++i) io.accv[i] = __uint_as_float(raw[i]);
+          if (others) {
+            for (int s2 = 0; s2 < S; ++s2) {
+              if (s2 == ks) continue;
+              const float* o = others + (size_t)s2 * 2048 + (h * 32) * 32 + lane;
+#pragma unroll
+              for (int i = 0; i < 32; ++i) io.accv[i] += __ldcg(o + i * 32);       // written by another SM: read from L2
+            }
+          }
           io.col_in_chunk = h * 32;
           io.col_in_half = c * 64 + h * 32;
           run_program<32, SP, true>(p.prog, io);
@@ -487,13 +531,34 @@ void tc2_gemm_plan(Launch& L) {
   if (getenv("DNNF_PAIR_KPACK")) q.kpack = atoi(getenv("DNNF_PAIR_KPACK")) == 2 ? 2 : 1;
   const int stage_bytes = sub_bytes * q.kpack;
   q.stages = std::min(8, tc2::kRingBudget / stage_bytes);
+  // split-K when fewer than half of the 74 CTA pairs would have a tile and the k loop is long.  Handing partial
+  // tiles over through L2 costs about 3 us (measured), a k-tile about 0.22 us: it pays from 32 k-tiles up, with
+  // two or three slices (1024 x 768 x 3072: 15.7 -> 13.2 us; 1024 x 768 x 768: 7.2 -> 9.2 us, so not there).
+  q.ksplit = 1; q.kt_per = q.k_tiles;
+  if (q.total_tiles * 2 <= 74 && q.k_tiles >= 32 && !getenv("DNNF_NO_SPLIT_K")) {
+    int want = std::min(3, 74 / q.total_tiles);
+    if (getenv("DNNF_SPLIT_K")) want = std::max(1, std::min(8, atoi(getenv("DNNF_SPLIT_K"))));
+    if (want > 1) {
+      int per = (q.k_tiles + want - 1) / want;
+      per = (per + q.kpack - 1) / q.kpack * q.kpack;
+      q.kt_per = per;
+      q.ksplit = (q.k_tiles + per - 1) / per;
+    }
+  }
+  if (q.ksplit > 1) {
+    const int64_t units = (int64_t)q.total_tiles * 2 * tc2::EPI_WARPS * std::max(1, q.bn / 2 / 64);
+    L.counter_bytes = units * 4;
+    L.scratch_bytes = units * q.ksplit * 2048 * 4;
+  } else {
+    L.counter_bytes = L.scratch_bytes = 0;
+  }
   q.c_input = -1;
   int vec_slot = 0;
   for (int i = 0; i < gp.n_in; ++i) {
     if (gp.in[i].mode == 1) gp.in[i].mode = vec_slot++;      // from here on: slot in the staged-vector area
     else { q.c_input = i; gp.in[i].mode = 0; }
   }
-  L.grid = 2 * std::min(q.total_tiles, 74);
+  L.grid = 2 * std::min(q.total_tiles * q.ksplit, 74);
   L.threads = tc2::THREADS;
   L.smem = (size_t)q.stages * stage_bytes + tc2::kFixed;
   L.variant = 3;
@@ -566,6 +631,13 @@ struct Tc2Launcher {
     rc = cudaLaunchKernelEx(&cfg, tc2::gemm_tc2_kernel<SP>, gp_of(L), t2_of(L));
   }
 };
+
+// split-K scratch and counters live in the bound workspace at the offsets the planner chose
+void tc2_set_scratch(Launch& L, void* ws_base) {
+  tc2::Params& q = t2_of(L);
+  q.scratch = L.scratch_off >= 0 ? reinterpret_cast<float*>(reinterpret_cast<char*>(ws_base) + L.scratch_off) : nullptr;
+  q.counters = L.counter_off >= 0 ? reinterpret_cast<int32_t*>(reinterpret_cast<char*>(ws_base) + L.counter_off) : nullptr;
+}
 
 int tc2_gemm_launch(const Launch& L, cudaStream_t st) {
   Tc2Launcher F{L, st, cudaSuccess};

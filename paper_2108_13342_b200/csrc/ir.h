@@ -69,6 +69,9 @@ struct Launch {
   std::vector<int> in_tensors, out_tensors;     // parallel to params.in[] / out[]
   std::vector<uint8_t> blob;                    // family-specific parameter block (GEMM / conv)
   int64_t flops = 0;
+  // device scratch of the kernel itself, placed in the workspace by the planner: `counter_bytes` sit in the
+  // workspace's zeroed header, `scratch_bytes` behind the tensors
+  int64_t scratch_bytes = 0, counter_bytes = 0, scratch_off = -1, counter_off = -1;
 };
 
 struct Block {
@@ -88,6 +91,7 @@ struct Graph {
   bool planned = false;
   uint32_t plan_flags = 0;
   size_t ws_bytes = 0;
+  size_t ws_zero_bytes = 256;            // leading bytes of the workspace that must be zero when a run starts
   void* ws_ptr = nullptr;
   size_t ws_bound_bytes = 0;
   dnnf_plan_stats pstats{};

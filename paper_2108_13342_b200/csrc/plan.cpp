@@ -392,7 +392,11 @@ int plan_graph(Graph& g, uint32_t flags) {
   // Workspace: first-fit over live ranges in block order.
   struct Range { int64_t off, size; int last_use; };
   std::vector<Range> active;
-  int64_t ws = 256;                       // status words live in the first 256 bytes
+  int64_t ws = 256;                       // status words live in the first 256 bytes,
+  for (auto& b : g.blocks)                // kernels' arrival counters right behind them (the zeroed header)
+    if (b.lowered && b.launch.counter_bytes > 0) { b.launch.counter_off = ws; ws += (b.launch.counter_bytes + 255) / 256 * 256; }
+  const int64_t header = ws;
+  g.ws_zero_bytes = (size_t)header;
   auto root = [&](int t) { while (g.tensors[t].alias_of >= 0) t = g.tensors[t].alias_of; return t; };
   std::vector<int> last_use(g.tensors.size(), -1);
   for (size_t bi = 0; bi < g.blocks.size(); ++bi) for (int t : g.blocks[bi].inputs) last_use[root(t)] = (int)bi;
@@ -408,13 +412,15 @@ int plan_graph(Graph& g, uint32_t flags) {
       for (auto& r : active) if (r.last_use >= (int)bi) keep.push_back(r);
       active.swap(keep);
       std::sort(active.begin(), active.end(), [](const Range& a, const Range& c) { return a.off < c.off; });
-      int64_t off = 256;
+      int64_t off = header;
       for (auto& r : active) { if (off + size <= r.off) break; off = std::max(off, r.off + r.size); }
       active.push_back({off, size, std::max(last_use[t], (int)bi)});
       T.ws_offset = off;
       ws = std::max(ws, off + size);
     }
   }
+  for (auto& b : g.blocks)                // kernels' own scratch (split-K partials) behind the tensors, never shared
+    if (b.lowered && b.launch.scratch_bytes > 0) { b.launch.scratch_off = ws; ws += (b.launch.scratch_bytes + 255) / 256 * 256; }
   g.ws_bytes = (size_t)ws;
   g.plan_flags = flags;
   g.planned = runnable;

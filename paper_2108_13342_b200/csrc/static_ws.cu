@@ -50,8 +50,8 @@ extern "C" DNNF_API int dnnf_run_static_ws(dnnf_graph* g, void* cuda_stream) {
     void* ws = nullptr;
     int rc = static_ws_address(&ws, G.err);
     if (rc != DNNF_OK) return rc;
-    // the status words must start at zero; everything else is written before it is read
-    if (cudaMemsetAsync(ws, 0, 256, (cudaStream_t)cuda_stream) != cudaSuccess) { G.err = "cannot clear the status words"; return DNNF_ERR_CUDA; }
+    // the status words and the kernels' arrival counters must start at zero; everything else is written before it is read
+    if (cudaMemsetAsync(ws, 0, G.ws_zero_bytes, (cudaStream_t)cuda_stream) != cudaSuccess) { G.err = "cannot clear the status words"; return DNNF_ERR_CUDA; }
     void* saved_ptr = G.ws_ptr;
     size_t saved_bytes = G.ws_bound_bytes;
     G.ws_ptr = ws; G.ws_bound_bytes = DNNF_STATIC_WS_BYTES;

@@ -75,6 +75,38 @@ def test_pair_gemm_shapes_and_epilogues(mnk, kmajor_b, epi):
     _expect_variant(s, 3, "DNNF_NO_PAIR_GEMM")
 
 
+@pytest.mark.parametrize("mnk", [(512, 128, 2048), (256, 256, 2304), (1024, 768, 3072), (300, 136, 2120), (512, 384, 2056)])
+@pytest.mark.parametrize("epi", ["none", "bias_gelu", "bias_residual"])
+def test_pair_gemm_split_k(mnk, epi):
+    """Few output tiles and a long K: several CTA pairs share a tile (split-K).  Three runs in a row on the same
+    workspace: the arrival counters must come back to zero by themselves."""
+    import os
+    m, n, k = mnk
+    g = graph()
+    g.ext("A", (m, k), "bf16"); g.ext("Bm", (k, n), "bf16")
+    ins = {"A": _bf(rnd((m, k), 41, -1, 1)), "Bm": _bf(rnd((k, n), 42, -0.1, 0.1))}
+    t = g.add("MatMul", ["A", "Bm"])
+    if epi != "none":
+        g.ext("bias", (n,), "f32"); ins["bias"] = rnd((n,), 43, -0.5, 0.5)
+        t = g.add("Add", [t, "bias"])
+    if epi == "bias_gelu":
+        t = g.add("Gelu", [t], approx="tanh")
+    if epi == "bias_residual":
+        g.ext("R", (m, n), "bf16"); ins["R"] = _bf(rnd((m, n), 44, -1, 1))
+        t = g.add("Add", [t, "R"])
+    g.mark_output(t)
+    wl = W.Workload(g, ins)
+    s, got, ref = run_both(wl, FUSED)
+    (name,) = wl.graph.outputs
+    close(got[name], ref[name], RTOL_BF16)
+    if not (os.environ.get("DNNF_NO_PAIR_GEMM") or os.environ.get("DNNF_NO_SPLIT_K")):
+        assert s.g.blocks()[0]["variant"] == 3 and s.g.workspace_zero_bytes() > 256, (s.g.blocks(), s.g.workspace_zero_bytes())
+    for _ in range(2):
+        s.run()
+        close(s.output(name), ref[name], RTOL_BF16)
+        assert s.g.status()[0] == 0
+
+
 def test_batched_matmul_with_transposed_and_strided_operands():
     # scores = (Q K^T) * scale + mask with Q, K sliced out of one [B,S,3*H*D] tensor -- all index
     # operators fold into operand strides; P V is stored straight into [B,S,H*D]
