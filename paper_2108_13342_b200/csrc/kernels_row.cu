@@ -36,19 +36,21 @@ bool finalize_row(Launch& L) {
   for (int i = 0; i < p.n_in; ++i) rev(p.in[i].stride);
   for (int i = 0; i < p.n_out; ++i) rev(p.out[i].stride);
   const int V = p.vec, Lr = p.L;
+  p.inv_L = 1.0f / (float)p.L;
   int nv = 0, wpr = 1, rpw = 1;
   // Enough warps to keep every scheduler busy: with few rows a row is split over several warps
   // (shorter per-thread chains), with many short rows a warp takes several rows (more loads in flight).
   // 4000 (27 warps per SM): measured best when independent blocks overlap on the GPU, 6 % slower than
   // 148 * 32 for a lone 1024-row launch.
   static const long target = getenv("DNNF_ROW_TARGET_WARPS") ? atol(getenv("DNNF_ROW_TARGET_WARPS")) : 4000L;
+  static const long split_target = getenv("DNNF_ROW_SPLIT_TARGET") ? atol(getenv("DNNF_ROW_SPLIT_TARGET")) : 2000L;   // splitting a row costs a barrier per reduction: only below 2000 rows
   if (V == 4) {
     const int vectors = (Lr + 3) / 4;
     auto fit = [&](int w) { int need = (vectors + 32 * w - 1) / (32 * w); return need; };   // vectors per lane with w warps per row
     int need = fit(1);
     if (need <= 8) {
       wpr = 1;
-      while (wpr < 8 && p.rows * wpr < target && fit(wpr) > 1) wpr *= 2;
+      while (wpr < 8 && p.rows * wpr < split_target && fit(wpr) > 1) wpr *= 2;
       need = fit(wpr);
       if (wpr == 1) { nv = need <= 1 ? 1 : need <= 2 ? 2 : need <= 4 ? 4 : need <= 6 ? 6 : 8; }
       else if (wpr == 2) { nv = need <= 1 ? 1 : need <= 2 ? 2 : need <= 3 ? 3 : 4; }

@@ -23,7 +23,8 @@ struct RowIO {
   uint32_t outer[kMaxDims];        // coordinates of the warp's first row; its other rows follow along dim 1
   bool row_ok[RPW];
   int lane_in_row;                 // 0 .. 32*WPR-1
-  float* xchg;                     // shared memory, WPR floats (WPR > 1)
+  float* xchg;                     // shared memory, 2 x WPR floats (WPR > 1)
+  mutable int xslot = 0;
   __device__ __forceinline__ int col(int j) const { return (j * 32 * WPR + lane_in_row) * V; }
   __device__ __forceinline__ uint32_t row_offset(const TensorArg& a, int r) const {
     uint32_t off = (uint32_t)a.base + (uint32_t)r * (uint32_t)a.stride[1];
@@ -113,20 +114,23 @@ struct RowIO {
       }
     }
     if (WPR > 1) {                                   // RPW == 1 here
-      __syncthreads();                               // previous exchange fully consumed
-      if ((threadIdx.x & 31) == 0) xchg[threadIdx.x >> 5] = red[0];
+      // two exchange areas used in turn: the barrier of this exchange also tells that everybody has
+      // finished reading the one before, so one barrier per reduction is enough
+      float* x = xchg + xslot * WPR;
+      xslot ^= 1;
+      if ((threadIdx.x & 31) == 0) x[threadIdx.x >> 5] = red[0];
       __syncthreads();
-      float t = xchg[0];
+      float t = x[0];
 #pragma unroll
       for (int w = 1; w < WPR; ++w) {
-        float y = xchg[w];
+        float y = x[w];
         if (op == M_ROWMAX) t = fmaxf(t, y); else if (op == M_ROWPROD) t *= y; else t += y;
       }
       red[0] = t;
     }
 #pragma unroll
     for (int r = 0; r < RPW; ++r) {
-      float x = op == M_ROWMEAN ? red[r] / (float)p.L : red[r];
+      float x = op == M_ROWMEAN ? red[r] * p.inv_L : red[r];
 #pragma unroll
       for (int e = 0; e < V * NV; ++e) acc[r * V * NV + e] = x;
     }
@@ -138,7 +142,7 @@ constexpr int kRowWarpsPerCta = 4;
 template <int V, int NV, int WPR, int RPW, class SP, bool F32>
 __global__ void __launch_bounds__(WPR > 1 ? 32 * WPR : 32 * kRowWarpsPerCta)
 row_kernel(const __grid_constant__ RowParams p) {
-  __shared__ float xchg[WPR > 1 ? WPR : 1];
+  __shared__ float xchg[WPR > 1 ? 2 * WPR : 1];
   RowIO<V, NV, WPR, RPW, F32> io{p};
   io.xchg = xchg;
   uint32_t row0;

@@ -110,6 +110,7 @@ struct RowParams {
   int64_t rows;
   int32_t L;
   int32_t vec;          // 4 if L % 4 == 0 and all accesses 16B-aligned, else 1
+  float inv_L;          // 1 / L (row means multiply by it)
 };
 
 }  // namespace dnnf
