@@ -20,6 +20,7 @@
 #include <string>
 
 #include "conv_params.h"
+#include "tma_host.h"
 
 namespace dnnf {
 
@@ -236,35 +237,13 @@ bool dwconv_tma_plan(Launch& L) {
   return true;
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qr;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess && qr == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  });
-  return fn;
-}
-
 bool dwconv_tma_prepare(Launch& L, std::string& err) {
   const DwParams& dp = dw_of(L);
   dwt::Params& q = tq_of(L);
-  if ((uintptr_t)dp.x & 15) { err = "depthwise convolution input is not 16-byte aligned"; return false; }
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) { err = "cuTensorMapEncodeTiled is not available"; return false; }
   cuuint64_t dims[4] = {(cuuint64_t)dp.C, (cuuint64_t)dp.W, (cuuint64_t)dp.H, (cuuint64_t)dp.N};
   cuuint64_t strides[3] = {(cuuint64_t)dp.C * 4, (cuuint64_t)dp.W * dp.C * 4, (cuuint64_t)dp.H * dp.W * dp.C * 4};
   cuuint32_t box[4] = {(cuuint32_t)q.cb, (cuuint32_t)(q.wt + 2), (cuuint32_t)(dwt::HT + 2), 1};
-  cuuint32_t estr[4] = {1, 1, 1, 1};
-  CUresult rc = fn(&q.tmX, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(dp.x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (rc != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)rc); return false; }
+  if (!tma_encode(&q.tmX, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(dp.x), dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE, err)) return false;
   return true;
 }
 

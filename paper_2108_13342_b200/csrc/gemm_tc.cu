@@ -22,6 +22,7 @@
 
 #include "ir.h"
 #include "tc_common.cuh"
+#include "tma_host.h"
 
 namespace dnnf {
 
@@ -295,27 +296,9 @@ void tc_gemm_plan(Launch& L) {
   tc.debug = getenv("DNNF_GEMM_DEBUG") ? atoi(getenv("DNNF_GEMM_DEBUG")) : 0;
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qr;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess && qr == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  });
-  return fn;
-}
-
 // dims innermost first: {inner, outer, b0, b1}
 static bool encode(CUtensorMap* tm, void* base, int64_t ext_inner, int64_t ext_outer, int64_t stride_outer, const int32_t* bext,
                    const int64_t* bstride, int box_inner, int box_outer, std::string& err) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) { err = "cuTensorMapEncodeTiled is not available"; return false; }
   cuuint64_t dims[4] = {(cuuint64_t)ext_inner, (cuuint64_t)ext_outer, (cuuint64_t)bext[0], (cuuint64_t)bext[1]};
   // a broadcast (stride 0) batch dim is addressed with coordinate 0 only; give it extent 1 and any legal stride
   cuuint64_t s1 = (cuuint64_t)stride_outer * 2;
@@ -325,11 +308,7 @@ static bool encode(CUtensorMap* tm, void* base, int64_t ext_inner, int64_t ext_o
   if (!bstride[1]) dims[3] = 1;
   cuuint64_t strides[3] = {s1, s2, s3};
   cuuint32_t box[4] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer, 1, 1};
-  cuuint32_t estr[4] = {1, 1, 1, 1};
-  CUresult rc = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (rc != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)rc); return false; }
-  return true;
+  return tma_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, err);
 }
 
 bool tc_gemm_prepare(Launch& L, std::string& err) {

@@ -30,6 +30,7 @@
 #include "chain.cuh"
 #include "gemm_params.h"
 #include "ir.h"
+#include "tma_host.h"
 
 namespace dnnf {
 
@@ -565,32 +566,12 @@ void tc2_gemm_plan(Launch& L) {
   L.static_id = StaticSet<Epi2Static>::find(gp.prog);
 }
 
-typedef CUresult (*EncodeTiledFn2)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-static EncodeTiledFn2 encode_fn2() {
-  static EncodeTiledFn2 fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qr;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess && qr == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn2>(p);
-  });
-  return fn;
-}
 static bool encode2d(CUtensorMap* tm, void* base, int64_t ext_inner, int64_t ext_outer, int64_t stride_outer_elems, int box_inner, int box_outer,
                      std::string& err) {
-  EncodeTiledFn2 fn = encode_fn2();
-  if (!fn) { err = "cuTensorMapEncodeTiled is not available"; return false; }
   cuuint64_t dims[2] = {(cuuint64_t)ext_inner, (cuuint64_t)ext_outer};
   cuuint64_t strides[1] = {(cuuint64_t)stride_outer_elems * 2};
   cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult rc = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (rc != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)rc); return false; }
-  return true;
+  return tma_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, err);
 }
 
 bool tc2_gemm_prepare(Launch& L, std::string& err) {

@@ -37,6 +37,7 @@
 
 #include "ir.h"
 #include "tc_common.cuh"
+#include "tma_host.h"
 
 namespace dnnf {
 
@@ -635,36 +636,13 @@ void tf32_gemm_plan(Launch& L) {
   L.static_id = StaticSet<tf32::Static>::find(gp.prog);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qr;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess && qr == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  });
-  return fn;
-}
-
 // fp32 [rows x cols] matrix, unit stride along cols, box = box_cols x box_rows
 static bool encode_f32(CUtensorMap* tm, float* base, int64_t cols, int64_t rows, int64_t row_stride, int box_cols, int box_rows,
                        CUtensorMapSwizzle swizzle, std::string& err) {
-  if ((uintptr_t)base & 15) { err = "GEMM operand is not 16-byte aligned"; return false; }
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) { err = "cuTensorMapEncodeTiled is not available"; return false; }
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)row_stride * 4};
   cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult rc = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (rc != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)rc); return false; }
-  return true;
+  return tma_encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, swizzle, err);
 }
 
 bool tf32_gemm_prepare(Launch& L, std::string& err) {
