@@ -11,7 +11,7 @@
 // tile (plus halo) and never through the L1 load path.  Per-channel epilogue operands
 // (scale, shift) are read once per thread, not once per output.
 //
-// No TMA multicast and no clusters are used anywhere in this file.
+// Every TMA load in this file is a plain per-CTA load; no clusters are used.
 #include <cuda.h>
 #include <cuda_runtime.h>
 

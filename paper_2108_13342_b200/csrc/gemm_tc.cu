@@ -13,7 +13,7 @@
 // bound runs out the CTA records DNNF_ERR_TIMEOUT in the status words, stops issuing
 // work, releases tensor memory and returns.
 //
-// No TMA multicast and no clusters are used anywhere in this file.
+// Every TMA load in this file is a plain per-CTA load; no clusters are used.
 #include <cuda.h>
 #include <cuda_runtime.h>
 

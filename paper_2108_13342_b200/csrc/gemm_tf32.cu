@@ -28,7 +28,7 @@
 // Two accumulator stages in TMEM overlap the epilogue of tile i with the main loop of tile i+1.
 // Every wait is bounded: on expiry the CTA records DNNF_ERR_TIMEOUT, stops and frees TMEM.
 //
-// No TMA multicast and no clusters are used anywhere in this file.
+// Every TMA load in this file is a plain per-CTA load; no clusters are used.
 #include <cuda.h>
 #include <cuda_runtime.h>
 

@@ -2,7 +2,7 @@
 // TMA loads and tcgen05, the shared-memory matrix descriptor, and the epilogue IO that maps
 // a warp's 32 x 32 accumulator chunk onto the block's input/output index maps.
 //
-// No TMA multicast and no clusters are used anywhere in this file.
+// Every TMA load in this file is a plain per-CTA load; no clusters are used.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
