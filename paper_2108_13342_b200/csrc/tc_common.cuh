@@ -182,8 +182,9 @@ struct TcEpiIO {
 __device__ __forceinline__ uint32_t tc_digits(const GemmParams& p, const TensorArg& a, int first, int count, uint32_t lin) {
   uint32_t off = 0;
   for (int d = first; d < first + count; ++d) {
-    uint32_t e = p.it.extent[d];
-    uint32_t q = (d == first + count - 1) ? 0u : lin / e;
+    const uint32_t e = p.it.extent[d];
+    // (multiply-shift division: a run-time divide is some 40 dependent instructions)
+    const uint32_t q = (d == first + count - 1) ? 0u : (e == 1 ? lin : (__umulhi(lin, p.it.div_m[d]) >> p.it.div_s[d]));
     off += (lin - q * e) * (uint32_t)a.stride[d];
     lin = q;
   }
