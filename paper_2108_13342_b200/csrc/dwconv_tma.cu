@@ -33,6 +33,7 @@ struct Params {
   CUtensorMap tmX;           // dims (C, W, H, N), box (cb, wt + 2, HT + 2, 1), no swizzle
   int32_t cb, wt;            // channels and columns per tile
   int32_t tiles_c, tiles_w, tiles_h, total_tiles;
+  FastDiv fd_c, fd_w, fd_h, fd_c4; // tile index -> (channel block, column block, row block, image); item -> (column, channel group)
   int32_t invariant[kMaxIn]; // epilogue input i depends on the channel only
 };
 
@@ -118,10 +119,10 @@ __global__ void __launch_bounds__(THREADS, 2) dwconv_tma_kernel(const __grid_con
   pdl_wait();
 
   auto issue = [&](int tile, int buf) {
-    int t = tile;
-    const int tc = t % q.tiles_c; t /= q.tiles_c;
-    const int tw = t % q.tiles_w; t /= q.tiles_w;
-    const int th = t % q.tiles_h; const int n = t / q.tiles_h;
+    uint32_t t = (uint32_t)tile, u;
+    u = fd_div(t, q.fd_c); const int tc = (int)(t - u * q.tiles_c); t = u;
+    u = fd_div(t, q.fd_w); const int tw = (int)(t - u * q.tiles_w); t = u;
+    u = fd_div(t, q.fd_h); const int th = (int)(t - u * q.tiles_h); const int n = (int)u;
     mbar_expect_tx(&full_bar[buf], patch_bytes);
     // the halo may start at -1: rows and columns outside the image arrive as zeros (the convolution's padding)
     tma_load_4d(smem + (size_t)buf * patch_stride, &q.tmX, &full_bar[buf], tc * cb, tw * wt - 1, th * HT - 1, n);
@@ -143,7 +144,7 @@ __global__ void __launch_bounds__(THREADS, 2) dwconv_tma_kernel(const __grid_con
     for (int i = 0; i < 3; ++i)
       if (i < p.n_in && q.invariant[i]) { float v[4]; io.fetch(i, v); io.inv[i] = make_float4(v[0], v[1], v[2], v[3]); }
   };
-  if (hoist && (int)threadIdx.x < items) load_consts(((int)threadIdx.x % c4n) * 4);
+  if (hoist && (int)threadIdx.x < items) load_consts(((int)threadIdx.x - (int)fd_div(threadIdx.x, q.fd_c4) * c4n) * 4);
   uint32_t k = 0;
   for (int tile = blockIdx.x; tile < q.total_tiles; tile += gridDim.x, ++k) {
     const int buf = k & 1;
@@ -153,13 +154,13 @@ __global__ void __launch_bounds__(THREADS, 2) dwconv_tma_kernel(const __grid_con
     if (!mbar_wait(&full_bar[buf], (k >> 1) & 1)) failed = 1;
     __syncthreads();
     if (failed) break;
-    int t = tile;
-    const int tc = t % q.tiles_c; t /= q.tiles_c;
-    const int tw = t % q.tiles_w; t /= q.tiles_w;
-    const int th = t % q.tiles_h; const int n = t / q.tiles_h;
+    uint32_t t = (uint32_t)tile, u;
+    u = fd_div(t, q.fd_c); const int tc = (int)(t - u * q.tiles_c); t = u;
+    u = fd_div(t, q.fd_w); const int tw = (int)(t - u * q.tiles_w); t = u;
+    u = fd_div(t, q.fd_h); const int th = (int)(t - u * q.tiles_h); const int n = (int)u;
     const float4* patch = reinterpret_cast<const float4*>(smem + (size_t)buf * patch_stride);
     for (int item = threadIdx.x; item < items; item += THREADS) {
-      const int c4 = item % c4n, wl = item / c4n;
+      const int wl = (int)fd_div((uint32_t)item, q.fd_c4), c4 = item - wl * c4n;
       const int w = tw * wt + wl, c = tc * cb + c4 * 4;
       if (w >= p.W || c >= p.C) continue;
       if (!hoist) load_consts(c);
@@ -221,6 +222,8 @@ bool dwconv_tma_plan(Launch& L) {
   q.tiles_c = (dp.C + cb - 1) / cb;
   q.tiles_w = (dp.W + wt - 1) / wt;
   q.tiles_h = (dp.H + dwt::HT - 1) / dwt::HT;
+  q.fd_c = make_fastdiv((uint32_t)q.tiles_c); q.fd_w = make_fastdiv((uint32_t)q.tiles_w); q.fd_h = make_fastdiv((uint32_t)q.tiles_h);
+  q.fd_c4 = make_fastdiv((uint32_t)(cb / 4));
   const int64_t total = (int64_t)q.tiles_c * q.tiles_w * q.tiles_h * dp.N;
   if (total >= (1ll << 31) || total < 148) return false;        // too small to fill the machine: the direct kernel is better
   q.total_tiles = (int)total;

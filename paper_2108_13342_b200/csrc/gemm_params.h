@@ -43,6 +43,7 @@ struct GemmTcParams {
   int32_t bn;                      // N tile
   int32_t persistent_tiles;        // total output tiles
   int32_t debug;                   // ablation switches (development only)
+  FastDiv fd_tiles_mn, fd_tiles_n, fd_batch0;   // tile index -> (batch, tile row, tile column), batch -> (b0, b1)
 };
 
 }  // namespace dnnf

@@ -89,9 +89,9 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
       int s = 0; uint32_t ph = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int batch = tile / tiles_mn, r = tile - batch * tiles_mn;
-        const int tm = r / p.tiles_n, tn = r - tm * p.tiles_n;
-        const int b0 = batch % p.batch_ext[0], b1 = batch / p.batch_ext[0];
+        const int batch = (int)fd_div((uint32_t)tile, q.fd_tiles_mn), r = tile - batch * tiles_mn;
+        const int tm = (int)fd_div((uint32_t)r, q.fd_tiles_n), tn = r - tm * p.tiles_n;
+        const int b1 = (int)fd_div((uint32_t)batch, q.fd_batch0), b0 = batch - b1 * p.batch_ext[0];
         // a batch dim an operand is broadcast over has stride 0 and extent 1 in its tensor map
         const int ab0 = p.A.batch_stride[0] ? b0 : 0, ab1 = p.A.batch_stride[1] ? b1 : 0;
         const int bb0 = p.B.batch_stride[0] ? b0 : 0, bb1 = p.B.batch_stride[1] ? b1 : 0;
@@ -152,8 +152,8 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-      const int batch = tile / tiles_mn, r = tile - batch * tiles_mn;
-      const int tm = r / p.tiles_n, tn = r - tm * p.tiles_n;
+      const int batch = (int)fd_div((uint32_t)tile, q.fd_tiles_mn), r = tile - batch * tiles_mn;
+      const int tm = (int)fd_div((uint32_t)r, q.fd_tiles_n), tn = r - tm * p.tiles_n;
       const int acc = tcount & 1;
       const uint32_t aph = (tcount >> 1) & 1;
       if (!mbar_wait(&tfull_bar[acc], aph, abort_flag)) { ok = false; break; }
@@ -286,6 +286,9 @@ void tc_gemm_plan(Launch& L) {
   gp.tiles_m = tiles_m;
   gp.tiles_n = (gp.N + tc.bn - 1) / tc.bn;
   tc.persistent_tiles = gp.tiles_m * gp.tiles_n * nb;
+  tc.fd_tiles_mn = make_fastdiv((uint32_t)(gp.tiles_m * gp.tiles_n));
+  tc.fd_tiles_n = make_fastdiv((uint32_t)gp.tiles_n);
+  tc.fd_batch0 = make_fastdiv((uint32_t)gp.batch_ext[0]);
   L.grid = std::min(tc.persistent_tiles, 148);
   L.threads = TC_THREADS;
   int stage_bytes = TC_BM * TC_BK * 2 + tc.bn * TC_BK * 2;

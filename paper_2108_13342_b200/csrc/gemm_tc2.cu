@@ -60,6 +60,7 @@ struct Params {
   int32_t kpack;             // 64-wide k-tiles per ring stage (1 or 2): one wait, one pair of commits per stage
   int32_t ksplit;            // CTA pairs that share one output tile, each with kt_per k-tiles of the K range (1: no split)
   int32_t kt_per;
+  FastDiv fd_tiles, fd_tiles_n;   // item -> (K slice, tile), tile -> (tile row, tile column)
   float* scratch;            // split-K partial accumulators: [unit][ksplit][64 cols][32 rows] fp32
   int32_t* counters;         // split-K arrival counters, one per unit (a warp's 32 x 64 chunk); zero between runs
 };
@@ -261,8 +262,8 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
       int s = 0; uint32_t ph = 0;
       bool ok = true;
       for (int item = pair; item < total && ok; item += n_pairs) {
-        const int ks = item / n_tiles, tile = item - ks * n_tiles;
-        const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
+        const int ks = (int)fd_div((uint32_t)item, q.fd_tiles), tile = item - ks * n_tiles;
+        const int tm = (int)fd_div((uint32_t)tile, q.fd_tiles_n), tn = tile - tm * tiles_n;
         const int m0 = tm * 256 + (int)rank * BM, n0 = tn * BN + (int)rank * HB;
         const int kt_end = min(k_tiles, (ks + 1) * q.kt_per);
         for (int kt = ks * q.kt_per; kt < kt_end; kt += kpack) {
@@ -307,7 +308,7 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
           { long long t0 = clock64(); if (!mbar_wait(&tempty_bar[acc], aph ^ 1, abort_flag)) { ok = false; break; } T2ACC(1, clock64() - t0); }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-          const int ks = item / n_tiles;
+          const int ks = (int)fd_div((uint32_t)item, q.fd_tiles);
           const int kt_begin = ks * q.kt_per, kt_end = min(k_tiles, kt_begin + q.kt_per);
           for (int kt = kt_begin; kt < kt_end; kt += kpack) {
             { long long t0 = clock64(); if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; } T2ACC(2, clock64() - t0); T2ACC(3, 1); }
@@ -346,8 +347,8 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
     // prefetch of the residual chunk `g` (global chunk counter of this warp) into buffer g & 1
     auto prefetch = [&](int item, int c, uint32_t g) {
       if (q.c_input < 0 || lane != 0) return;
-      const int tile = item % n_tiles;
-      const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
+      const int tile = item - (int)fd_div((uint32_t)item, q.fd_tiles) * n_tiles;
+      const int tm = (int)fd_div((uint32_t)tile, q.fd_tiles_n), tn = tile - tm * tiles_n;
       const int m0 = tm * 256 + (int)rank * BM + sub * 32, n0 = tn * BN + half * cols_per_warp + c * 64;
       mbar_expect_tx(&my_cbar[g & 1], kChunkBytes);
       tma_load_2d(cbuf + (g & 1) * kChunkBytes, &q.tmC, &my_cbar[g & 1], n0, m0);
@@ -355,8 +356,8 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
     const int S = q.ksplit;
     if (pair < total) prefetch(pair, 0, 0);
     for (int item = pair; item < total && ok; item += n_pairs, ++tcount) {
-      const int ks = item / n_tiles, tile = item - ks * n_tiles;
-      const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
+      const int ks = (int)fd_div((uint32_t)item, q.fd_tiles), tile = item - ks * n_tiles;
+      const int tm = (int)fd_div((uint32_t)tile, q.fd_tiles_n), tn = tile - tm * tiles_n;
       const int m0 = tm * 256 + (int)rank * BM + sub * 32;
       const int nw0 = tn * BN + half * cols_per_warp;
       // stage this tile's row-invariant operands (this warp's columns)
@@ -524,6 +525,8 @@ void tc2_gemm_plan(Launch& L) {
   q.bn = best_bn;
   q.tiles_n = (gp.N + q.bn - 1) / q.bn;
   q.total_tiles = tiles_m * q.tiles_n;
+  q.fd_tiles = make_fastdiv((uint32_t)q.total_tiles);
+  q.fd_tiles_n = make_fastdiv((uint32_t)q.tiles_n);
   gp.tiles_m = tiles_m; gp.tiles_n = q.tiles_n;
   const int sub_bytes = tc2::BM * tc2::BK * 2 + (q.bn / 2) * tc2::BK * 2;
   // two k-tiles per stage halve the issuing thread's per-stage cost (wait, fence, two commits); worth it when its

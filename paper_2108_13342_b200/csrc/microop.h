@@ -67,6 +67,23 @@ struct IterSpace {
   uint32_t div_m[kMaxDims], div_s[kMaxDims];   // n / extent[d] == umulhi(n, div_m[d]) >> div_s[d] for n < 2^31
 };
 
+// Division by a run-time constant as multiply-high and shift (valid for n < 2^31): a hardware-less integer
+// divide is some 40 dependent instructions, which a single issuing thread feels on every tile.
+struct FastDiv { uint32_t d, m, s; };
+inline FastDiv make_fastdiv(uint32_t d) {
+  FastDiv f{d, 0, 0};
+  if (d <= 1) return f;
+  uint32_t lg = 0;
+  while ((1ull << lg) < d) ++lg;
+  const uint64_t p = 31 + lg;
+  f.m = (uint32_t)(((1ull << p) + d - 1) / d);
+  f.s = (uint32_t)(p - 32);
+  return f;
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ uint32_t fd_div(uint32_t n, const FastDiv& f) { return f.d <= 1 ? n : (__umulhi(n, f.m) >> f.s); }
+#endif
+
 inline void set_fastdiv(IterSpace& it) {
   for (int d = 0; d < it.ndim; ++d) {
     uint32_t e = it.extent[d];
