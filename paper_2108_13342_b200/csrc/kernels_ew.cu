@@ -182,8 +182,10 @@ __global__ void __launch_bounds__(256) tr_kernel(const __grid_constant__ EwParam
   constexpr int K = 4;
   TrIO<V, K, F32> io{p, smem};
   uint32_t b = blockIdx.x;
-  uint32_t tile_i = b % (uint32_t)p.tiles_i; b /= (uint32_t)p.tiles_i;
-  uint32_t tile_t = b % (uint32_t)p.tiles_t; b /= (uint32_t)p.tiles_t;
+  uint32_t u = fd_div(b, p.fd_tiles_i);
+  const uint32_t tile_i = b - u * (uint32_t)p.tiles_i; b = u;
+  u = fd_div(b, p.fd_tiles_t);
+  const uint32_t tile_t = b - u * (uint32_t)p.tiles_t; b = u;
 #pragma unroll
   for (int d = 2; d < kMaxDims; ++d) {
     io.outer[d] = 0;
@@ -325,6 +327,7 @@ void finalize_ew(Launch& L) {
   if (L.family == DNNF_FAMILY_TRANSPOSE) {
     p.tiles_t = (p.it.extent[1] + TT - 1) / TT;
     p.tiles_i = (p.it.extent[0] + TI - 1) / TI;
+    p.fd_tiles_t = make_fastdiv((uint32_t)p.tiles_t); p.fd_tiles_i = make_fastdiv((uint32_t)p.tiles_i);
     int64_t grid = (int64_t)p.tiles_t * p.tiles_i;
     for (int d = 2; d < nd; ++d) grid *= p.it.extent[d];
     int staged = 0;

@@ -106,6 +106,7 @@ struct EwParams {
   int32_t tdim;         // transpose family: iteration dim along which staged inputs are contiguous
   int64_t total;        // product of extents
   int32_t tiles_t, tiles_i;   // transpose family: tiles along tdim / innermost dim
+  FastDiv fd_tiles_t, fd_tiles_i;
   uint32_t inner_vecs, inner_m, inner_s;   // vectors along the innermost dim and its fast divisor
 };
 
