@@ -79,6 +79,7 @@ struct Params {
   int32_t b_dense;           // B is a dense row-major [K x N] block: fetched with one bulk copy
   int32_t fast_epi;          // the fast epilogue form applies
   int32_t debug;             // ablation switches (development only)
+  FastDiv fd_n, fd_npad, fd_kpad;   // element index of B -> (k, n)
   int32_t b_static;          // B is an external input: it may be read before the previous kernel ends
   int8_t slot[kMaxIn];       // fast form: staged-vector slot of epilogue input i, or -1 for a dense operand
 };
@@ -281,7 +282,7 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
         for (int u = 0; u < 4; ++u) {
           const int i = i0 + u * nthr;
           int k, n;
-          if (n_fast) { k = i / NP; n = i - k * NP; } else { n = i / kpad; k = i - n * kpad; }
+          if (n_fast) { k = (int)fd_div((uint32_t)i, q.fd_npad); n = i - k * NP; } else { n = (int)fd_div((uint32_t)i, q.fd_kpad); k = i - n * kpad; }
           kk[u] = k; nn[u] = n;
           x[u] = (i < total && k < p.K && n < p.N) ? __ldg(W + (int64_t)k * p.B.stride_row + (int64_t)n * p.B.stride_col) : 0.0f;
         }
@@ -315,7 +316,7 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
       if (mbar_wait(b_bar, 0, abort_flag)) {
         const float* raw = reinterpret_cast<const float*>(epi);
         const int total = p.K * p.N;
-        for (int i = tid; i < total; i += nthr) { const int k = i / p.N; put_b(k, i - k * p.N, raw[i]); }
+        for (int i = tid; i < total; i += nthr) { const int k = (int)fd_div((uint32_t)i, q.fd_n); put_b(k, i - k * p.N, raw[i]); }
       }
     }
     fence_async_smem();
@@ -613,6 +614,7 @@ void tf32_gemm_plan(Launch& L) {
   q.dual = 2 * q.npad <= 256 && !getenv("DNNF_TF32_NO_DUAL");
   q.fast_epi = fast_epilogue(gp, q.slot) && !getenv("DNNF_TF32_GENERAL_EPILOGUE");
   q.b_static = gp.static_mask & 1u;
+  q.fd_n = make_fastdiv((uint32_t)gp.N); q.fd_npad = make_fastdiv((uint32_t)q.npad); q.fd_kpad = make_fastdiv((uint32_t)(q.k_chunks * tf32::BK));
   q.epi_warps = (gp.N <= 32 && !getenv("DNNF_TF32_EPI8")) ? 4 : 8;
   q.debug = getenv("DNNF_TF32_DEBUG") ? atoi(getenv("DNNF_TF32_DEBUG")) : 0;
   gp.tiles_m = (gp.M + tf32::BM - 1) / tf32::BM;
