@@ -192,6 +192,21 @@ def test_matmul_fp32_tall_skinny_uses_tensor_cores():
     _expect_variant(s, 4, "DNNF_NO_TF32_GEMM")
 
 
+def test_matmul_fp32_tall_skinny_transposed_weight_and_second_output():
+    """fp32 tensor-core kernel with a K-major weight (strided B: split by the strided loader) and a block with two
+    outputs (general, transposing epilogue)."""
+    m, k, n = 777, 40, 56
+    g = graph()
+    g.ext("X", (m, k)); g.ext("Wt", (n, k), kind="weight"); g.ext("b", (n,))
+    w = g.add("Transpose", ["Wt"], perm=(1, 0))
+    t = g.add("MatMul", ["X", w])
+    t = g.add("Add", [t, "b"], out="Z")
+    g.mark_output(t)
+    g.mark_output(g.add("Relu", [t], out="Y"))
+    s = check(W.Workload(g, {"X": rnd((m, k), 3, -1, 1), "Wt": rnd((n, k), 4, -0.3, 0.3), "b": rnd((n,), 5)}), RTOL_F32, FUSED, expect_blocks=1)
+    _expect_variant(s, 4, "DNNF_NO_TF32_GEMM")
+
+
 @pytest.mark.parametrize("cfg", [(1, 5, 6, 8), (2, 7, 9, 144), (1, 1, 1, 4), (1, 3, 1, 12), (2, 30, 17, 24)])
 def test_dwconv3x3_with_epilogue(cfg):
     n, h, w, c = cfg
