@@ -136,6 +136,8 @@ typedef struct {
   int64_t workspace_bytes;
   int32_t n_yellow_decisions;  /* Table 3 yellow cells resolved by the cost model */
   int32_t n_yellow_fused;
+  int32_t n_profile_hits;      /* candidate-block costs answered by the profiling database */
+  int32_t n_profile_misses;    /* distinct candidate signatures it did not have (analytic cost used) */
 } dnnf_plan_stats;
 
 typedef enum {
@@ -225,6 +227,29 @@ DNNF_API int dnnf_op_block(const dnnf_graph* g, int op_index, int* block);
 /* Number of operators currently alive (after rewriting) and their kinds. */
 DNNF_API int dnnf_op_count(const dnnf_graph* g, int* n_ops);
 DNNF_API int dnnf_op_kind(const dnnf_graph* g, int op_index, int* kind, int* alive);
+
+/* ---- profiling database (Section 4.3: "fusion profitability ... looked up in a profiling database") ----
+ * Process-wide map from a block signature (kernel family | operators | data types | shape) to a measured
+ * latency in microseconds.  dnnf_plan asks it for the cost of every candidate block of a yellow
+ * (profile-dependent) Table 3 decision and of block merging; what it does not find is costed by the
+ * analytic model and remembered in the graph as a miss.  All strings are host pointers, NUL-terminated. */
+DNNF_API int dnnf_profile_db_set(const char* signature, double microseconds);
+DNNF_API int dnnf_profile_db_get(const char* signature, double* microseconds);   /* DNNF_ERR_INVALID_ARG if absent */
+DNNF_API int dnnf_profile_db_size(size_t* n_entries);
+DNNF_API int dnnf_profile_db_clear(void);
+/* Text file, one "signature<TAB>microseconds" line per entry; load adds to / overwrites the current entries. */
+DNNF_API int dnnf_profile_db_save(const char* path);
+DNNF_API int dnnf_profile_db_load(const char* path, int* n_loaded);
+/* Signature of a planned block, and of the i-th miss of the last dnnf_plan (capacity bytes, truncated). */
+DNNF_API int dnnf_block_signature(const dnnf_graph* g, int block, char* host_buf, size_t capacity);
+DNNF_API int dnnf_profile_miss_count(const dnnf_graph* g, int* n);
+DNNF_API int dnnf_profile_miss(const dnnf_graph* g, int index, char* host_buf, size_t capacity);
+/* Runs every missed candidate block of the last dnnf_plan on the device and stores its per-launch time in the
+ * database: `iters` back-to-back launches between two CUDA events on `cuda_stream`, best of three, after two
+ * warm-up launches.  The block's
+ * tensors are placed in `scratch` (device memory, 256-byte aligned, contents irrelevant and overwritten);
+ * candidates that need more than scratch_bytes are skipped.  Synchronises the stream.  n_measured may be NULL. */
+DNNF_API int dnnf_profile_measure(dnnf_graph* g, void* scratch, size_t scratch_bytes, void* cuda_stream, int iters, int* n_measured);
 
 /* ---- binding and execution (Section 4.4: one generated kernel per block) -------- */
 

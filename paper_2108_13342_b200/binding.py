@@ -56,7 +56,8 @@ class RewriteStats(C.Structure):
 class PlanStats(C.Structure):
     _fields_ = [("n_ops", C.c_int32), ("n_blocks", C.c_int32), ("n_kernels", C.c_int32), ("fusion_rate", C.c_double),
                 ("irs_bytes_unfused", C.c_int64), ("irs_bytes_fused", C.c_int64), ("workspace_bytes", C.c_int64),
-                ("n_yellow_decisions", C.c_int32), ("n_yellow_fused", C.c_int32)]
+                ("n_yellow_decisions", C.c_int32), ("n_yellow_fused", C.c_int32),
+                ("n_profile_hits", C.c_int32), ("n_profile_misses", C.c_int32)]
 
 
 class BlockDesc(C.Structure):
@@ -70,7 +71,9 @@ EXPORTS = ["dnnf_graph_create", "dnnf_graph_destroy", "dnnf_add_tensor", "dnnf_a
            "dnnf_tensor_info", "dnnf_op_mapping", "dnnf_mapping_check", "dnnf_rewrite", "dnnf_rule_name", "dnnf_plan",
            "dnnf_block_count", "dnnf_block_info", "dnnf_block_program", "dnnf_op_block", "dnnf_op_count", "dnnf_op_kind",
            "dnnf_workspace_size", "dnnf_workspace_zero_bytes", "dnnf_bind", "dnnf_bind_workspace", "dnnf_run", "dnnf_run_static_ws", "dnnf_run_block", "dnnf_status",
-           "dnnf_launch_count", "dnnf_last_error", "dnnf_version"]
+           "dnnf_launch_count", "dnnf_last_error", "dnnf_version",
+           "dnnf_profile_db_set", "dnnf_profile_db_get", "dnnf_profile_db_size", "dnnf_profile_db_clear", "dnnf_profile_db_save",
+           "dnnf_profile_db_load", "dnnf_block_signature", "dnnf_profile_miss_count", "dnnf_profile_miss", "dnnf_profile_measure"]
 
 
 def _load():
@@ -102,6 +105,15 @@ def _load():
     lib.dnnf_op_kind.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     lib.dnnf_workspace_size.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
     lib.dnnf_workspace_zero_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
+    lib.dnnf_profile_db_set.argtypes = [C.c_char_p, C.c_double]
+    lib.dnnf_profile_db_get.argtypes = [C.c_char_p, C.POINTER(C.c_double)]
+    lib.dnnf_profile_db_size.argtypes = [C.POINTER(C.c_size_t)]
+    lib.dnnf_profile_db_save.argtypes = [C.c_char_p]
+    lib.dnnf_profile_db_load.argtypes = [C.c_char_p, C.POINTER(C.c_int)]
+    lib.dnnf_block_signature.argtypes = [C.c_void_p, C.c_int, C.c_char_p, C.c_size_t]
+    lib.dnnf_profile_miss_count.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
+    lib.dnnf_profile_miss.argtypes = [C.c_void_p, C.c_int, C.c_char_p, C.c_size_t]
+    lib.dnnf_profile_measure.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_int, C.POINTER(C.c_int)]
     lib.dnnf_bind.argtypes = [C.c_void_p, C.c_int, C.c_void_p]
     lib.dnnf_bind_workspace.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
     lib.dnnf_run.argtypes = [C.c_void_p, C.c_void_p]
@@ -239,6 +251,26 @@ class Graph:
         self._check(lib.dnnf_workspace_zero_bytes(self.h, C.byref(n)))
         return n.value
 
+    def block_signature(self, block):
+        buf = C.create_string_buffer(4096)
+        self._check(lib.dnnf_block_signature(self.h, block, buf, 4096))
+        return buf.value.decode()
+
+    def profile_misses(self):
+        n = C.c_int(0)
+        self._check(lib.dnnf_profile_miss_count(self.h, C.byref(n)))
+        out = []
+        for i in range(n.value):
+            buf = C.create_string_buffer(4096)
+            self._check(lib.dnnf_profile_miss(self.h, i, buf, 4096))
+            out.append(buf.value.decode())
+        return out
+
+    def profile_measure(self, scratch_ptr, scratch_bytes, stream=0, iters=20):
+        n = C.c_int(0)
+        self._check(lib.dnnf_profile_measure(self.h, C.c_void_p(scratch_ptr), scratch_bytes, C.c_void_p(stream), iters, C.byref(n)))
+        return n.value
+
     def bind(self, tid, dev_ptr):
         self._check(lib.dnnf_bind(self.h, tid, C.c_void_p(dev_ptr)))
 
@@ -274,3 +306,36 @@ class Graph:
                         "bytes": d.bytes_in + d.bytes_out, "flops": d.flops, "grid": d.grid,
                         "threads": d.threads, "variant": d.variant, "n_microops": d.n_microops})
         return out
+
+
+# ---- profiling database (process-wide) -------------------------------------------------------------
+def profile_db_set(signature, us):
+    if lib.dnnf_profile_db_set(signature.encode(), float(us)) != 0:
+        raise ValueError("bad profiling-database entry")
+
+
+def profile_db_get(signature):
+    v = C.c_double(0)
+    return v.value if lib.dnnf_profile_db_get(signature.encode(), C.byref(v)) == 0 else None
+
+
+def profile_db_size():
+    n = C.c_size_t(0)
+    lib.dnnf_profile_db_size(C.byref(n))
+    return n.value
+
+
+def profile_db_clear():
+    lib.dnnf_profile_db_clear()
+
+
+def profile_db_save(path):
+    if lib.dnnf_profile_db_save(path.encode()) != 0:
+        raise OSError(f"cannot write {path}")
+
+
+def profile_db_load(path):
+    n = C.c_int(0)
+    if lib.dnnf_profile_db_load(path.encode(), C.byref(n)) != 0:
+        raise OSError(f"cannot read {path}")
+    return n.value

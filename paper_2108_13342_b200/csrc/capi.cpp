@@ -1,5 +1,6 @@
 // C ABI: argument checking, state machine, error messages.  No exception leaves
 // this file.
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <exception>
@@ -11,6 +12,7 @@ using namespace dnnf;
 namespace dnnf {
 int run_blocks(Graph& g, int only_block, void* stream);
 int read_status(Graph& g, int* status, int* block);
+int profile_measure(Graph& g, void* scratch, size_t scratch_bytes, void* stream, int iters, int* n_measured);
 }
 
 #define DNNF_TRY try {
@@ -272,6 +274,54 @@ int dnnf_bind(dnnf_graph* g, int t, void* dev_ptr) {
   if (!G.tensors[t].external && !G.tensors[t].is_output) return fail(g, DNNF_ERR_INVALID_ARG, "only external tensors and marked outputs can be bound");
   G.tensors[t].bound = dev_ptr;
   return DNNF_OK;
+}
+
+int dnnf_profile_db_set(const char* signature, double microseconds) {
+  if (!signature || !(microseconds > 0)) return DNNF_ERR_INVALID_ARG;
+  profile_db_set(signature, microseconds);
+  return DNNF_OK;
+}
+int dnnf_profile_db_get(const char* signature, double* microseconds) {
+  if (!signature || !microseconds) return DNNF_ERR_INVALID_ARG;
+  return profile_db_get(signature, microseconds) ? DNNF_OK : DNNF_ERR_INVALID_ARG;
+}
+int dnnf_profile_db_size(size_t* n_entries) {
+  if (!n_entries) return DNNF_ERR_INVALID_ARG;
+  *n_entries = profile_db_size();
+  return DNNF_OK;
+}
+int dnnf_profile_db_clear(void) { profile_db_clear(); return DNNF_OK; }
+int dnnf_profile_db_save(const char* path) { return path ? profile_db_save(path) : DNNF_ERR_INVALID_ARG; }
+int dnnf_profile_db_load(const char* path, int* n_loaded) { return path ? profile_db_load(path, n_loaded) : DNNF_ERR_INVALID_ARG; }
+
+static int copy_out(const std::string& s, char* buf, size_t cap) {
+  if (!buf || cap == 0) return DNNF_ERR_INVALID_ARG;
+  size_t n = std::min(cap - 1, s.size());
+  memcpy(buf, s.data(), n);
+  buf[n] = 0;
+  return DNNF_OK;
+}
+int dnnf_block_signature(const dnnf_graph* g, int block, char* host_buf, size_t capacity) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  const Graph& G = g->g;
+  if (!G.planned && G.blocks.empty()) return DNNF_ERR_STATE;
+  if (block < 0 || block >= (int)G.blocks.size()) return DNNF_ERR_INVALID_ARG;
+  return copy_out(block_signature(G, G.blocks[block]), host_buf, capacity);
+}
+int dnnf_profile_miss_count(const dnnf_graph* g, int* n) {
+  if (!g || !n) return DNNF_ERR_INVALID_ARG;
+  *n = (int)g->g.profile_misses.size();
+  return DNNF_OK;
+}
+int dnnf_profile_miss(const dnnf_graph* g, int index, char* host_buf, size_t capacity) {
+  if (!g || index < 0 || index >= (int)g->g.profile_misses.size()) return DNNF_ERR_INVALID_ARG;
+  return copy_out(g->g.profile_misses[index].signature, host_buf, capacity);
+}
+int dnnf_profile_measure(dnnf_graph* g, void* scratch, size_t scratch_bytes, void* cuda_stream, int iters, int* n_measured) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  DNNF_TRY
+  return profile_measure(g->g, scratch, scratch_bytes, cuda_stream, iters, n_measured);
+  DNNF_CATCH(g)
 }
 
 int dnnf_workspace_zero_bytes(const dnnf_graph* g, size_t* bytes) {

@@ -82,6 +82,9 @@ struct Block {
   bool lowered = false;
 };
 
+// A candidate block whose cost the planner wanted from the profiling database and did not find.
+struct ProfileMiss { std::string signature; std::vector<int> ops; };
+
 struct Graph {
   std::vector<Tensor> tensors;
   std::vector<Op> ops;
@@ -95,6 +98,8 @@ struct Graph {
   void* ws_ptr = nullptr;
   size_t ws_bound_bytes = 0;
   dnnf_plan_stats pstats{};
+  std::vector<ProfileMiss> profile_misses;   // of the last dnnf_plan, one per distinct signature
+  int profile_hits = 0;
   std::string err;
 
   int add_tensor(const std::string& name, int dtype, const std::vector<int64_t>& dims);
@@ -125,6 +130,15 @@ int plan_graph(Graph& g, uint32_t flags);
 // Lowers `ops` (a candidate block) into a launch.  Returns DNNF_OK or an error;
 // `why` explains a refusal (used as the constraint check of Listing 1, Step 2.2).
 int lower_block(const Graph& g, const std::vector<int>& ops, uint32_t flags, Block& out, std::string& why);
+
+// ---- profiling database (profile_db.cpp) ----
+std::string block_signature(const Graph& g, const Block& b);
+bool profile_db_get(const std::string& sig, double* us);
+void profile_db_set(const std::string& sig, double us);
+size_t profile_db_size();
+void profile_db_clear();
+int profile_db_save(const char* path);
+int profile_db_load(const char* path, int* n_loaded);
 double block_cost_us(const Graph& g, const Block& b);
 
 const Program* program_of(const Launch& L);     // the block's micro-op program, wherever the family keeps it

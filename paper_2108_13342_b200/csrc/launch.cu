@@ -2,6 +2,9 @@
 // caller's stream.  Nothing here allocates or synchronises.
 #include <cuda_runtime.h>
 
+#include <algorithm>
+#include <map>
+
 #include "ir.h"
 
 namespace dnnf {
@@ -62,6 +65,80 @@ int run_blocks(Graph& g, int only, void* stream) {
     }
   }
   return DNNF_OK;
+}
+
+// Fills the profiling database: every candidate block the last plan asked about and did not find is lowered
+// again, given device memory from the caller's scratch area, launched and timed with CUDA events.
+int profile_measure(Graph& g, void* scratch, size_t scratch_bytes, void* stream, int iters, int* n_measured) {
+  cudaStream_t st = (cudaStream_t)stream;
+  if (n_measured) *n_measured = 0;
+  if (!scratch || ((uintptr_t)scratch & 255)) { g.err = "scratch must be non-null and 256-byte aligned"; return DNNF_ERR_INVALID_ARG; }
+  if (iters < 1) iters = 1;
+  cudaEvent_t e0, e1;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) { g.err = "cannot create events"; return DNNF_ERR_CUDA; }
+  int rc_all = DNNF_OK, done = 0;
+  for (const ProfileMiss& miss : g.profile_misses) {
+    Block b; std::string why;
+    if (lower_block(g, miss.ops, g.plan_flags, b, why) != DNNF_OK) continue;
+    b.ops = miss.ops;
+    Launch& L = b.launch;
+    if (L.family == DNNF_FAMILY_ALIAS) continue;
+    // arena: status words, arrival counters (both zero), the block's tensors, the kernel's own scratch
+    size_t off = 256;
+    if (L.counter_bytes > 0) { L.counter_off = (int64_t)off; off += (size_t)(L.counter_bytes + 255) / 256 * 256; }
+    const size_t zero_bytes = off;
+    std::map<int, size_t> place;
+    auto put = [&](int t) { if (!place.count(t)) { place[t] = off; off += ((size_t)g.tensors[t].bytes() + 255) / 256 * 256; } };
+    for (int t : L.in_tensors) put(t);
+    for (int t : L.out_tensors) put(t);
+    if (L.scratch_bytes > 0) { L.scratch_off = (int64_t)off; off += (size_t)(L.scratch_bytes + 255) / 256 * 256; }
+    if (off > scratch_bytes) continue;                       // does not fit: stays a miss
+    std::vector<void*> ip, op;
+    for (int t : L.in_tensors) ip.push_back((char*)scratch + place[t]);
+    for (int t : L.out_tensors) op.push_back((char*)scratch + place[t]);
+    if (L.family == DNNF_FAMILY_ROW) {
+      for (size_t i = 0; i < ip.size(); ++i) L.row.in[i].ptr = ip[i];
+      for (size_t i = 0; i < op.size(); ++i) L.row.out[i].ptr = op[i];
+    } else if (L.family == DNNF_FAMILY_ELEMENTWISE || L.family == DNNF_FAMILY_TRANSPOSE) {
+      for (size_t i = 0; i < ip.size(); ++i) L.ew.in[i].ptr = ip[i];
+      for (size_t i = 0; i < op.size(); ++i) L.ew.out[i].ptr = op[i];
+    } else {
+      std::string err;
+      patch_contraction(L, ip, op, err);
+      if (!err.empty()) continue;
+    }
+    if (cudaMemsetAsync(scratch, 0, zero_bytes, st) != cudaSuccess) { rc_all = DNNF_ERR_CUDA; break; }
+    auto launch = [&]() -> int {
+      switch (L.family) {
+        case DNNF_FAMILY_ELEMENTWISE: case DNNF_FAMILY_TRANSPOSE: return launch_ew(L, st);
+        case DNNF_FAMILY_ROW: return launch_row(L, st);
+        default: { std::string err; return launch_contraction(L, scratch, -1, st, err); }
+      }
+    };
+    bool ok = true;
+    for (int i = 0; i < 2 && ok; ++i) ok = launch() == 0;
+    // `iters` launches back to back between two events (what a graph of blocks looks like to the GPU: the next
+    // launch is queued while this one runs), three times; the best per-launch time is kept.
+    std::vector<float> ms;
+    for (int rep = 0; rep < 3 && ok; ++rep) {
+      cudaEventRecord(e0, st);
+      for (int i = 0; i < iters && ok; ++i) ok = launch() == 0;
+      cudaEventRecord(e1, st);
+      if (cudaEventSynchronize(e1) != cudaSuccess) { ok = false; break; }
+      float t = 0.f;
+      cudaEventElapsedTime(&t, e0, e1);
+      ms.push_back(t / (float)iters);
+    }
+    if (!ok || ms.empty()) { cudaGetLastError(); continue; }
+    std::sort(ms.begin(), ms.end());
+    profile_db_set(miss.signature, (double)ms[0] * 1000.0);
+    ++done;
+  }
+  cudaStreamSynchronize(st);
+  cudaEventDestroy(e0); cudaEventDestroy(e1);
+  if (n_measured) *n_measured = done;
+  if (rc_all != DNNF_OK) g.err = "profiling run failed";
+  return rc_all;
 }
 
 int read_status(Graph& g, int* status, int* block) {

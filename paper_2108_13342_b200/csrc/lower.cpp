@@ -483,6 +483,14 @@ bool emit_program(LowerCtx& cx, int anchor_out, int max_tmp) {
       if (!outside) continue;
       auto vit = cx.views.find(t);
       if (vit == cx.views.end()) { cx.why = "output not reachable"; return false; }
+      // A tensor that leaves the block must be written completely: the iteration space has to cover all of it.
+      // (With a Slice further down the block the space is the slice's, and a tensor in front of the Slice that
+      // is also read outside would be written only in part.)
+      {
+        int64_t covered = 1;
+        for (size_t d = 0; d < vit->second.coef.size() && d < cx.ext.size(); ++d) if (vit->second.coef[d] != 0) covered *= cx.ext[d];
+        if (covered != T.numel() || vit->second.c0 != 0) { cx.why = "a tensor that is read outside the block would be written only in part"; return false; }
+      }
       int oi = find_or_add_arg(cx.outs, t, vit->second);
       E.stores[E.root_of[t]].push_back(oi);
     }

@@ -4,7 +4,9 @@
 #include <cstdlib>
 #include <cstring>
 #include <functional>
+#include <map>
 #include <set>
+#include <string>
 
 #include "gemm_params.h"
 #include "ir.h"
@@ -95,12 +97,26 @@ struct Planner {
     Block tmp; std::string why;
     Block& b = out ? *out : tmp;
     bool ok = lower_block(g, members, flags, b, why) == DNNF_OK;
+    if (ok) b.ops = members;
     if (!ok && debug) {
       fprintf(stderr, "[dnnf plan] cannot lower {");
       for (int m : members) fprintf(stderr, " %s#%d", op_name(g.ops[m].kind), m);
       fprintf(stderr, " }: %s\n", why.c_str());
     }
     return ok;
+  }
+
+  // Cost of a lowered candidate block: the profiling database's measured latency when it has the block's
+  // signature (Section 4.3), else the analytic model -- and the miss is remembered so that it can be measured.
+  std::map<std::string, std::vector<int>> misses;
+  int hits = 0;
+  double cost(const Block& b) {
+    if (b.launch.family == DNNF_FAMILY_ALIAS) return 0.0;
+    const std::string sig = block_signature(g, b);
+    double us;
+    if (profile_db_get(sig, &us)) { ++hits; return us; }
+    misses.emplace(sig, b.ops);
+    return block_cost_us(g, b);
   }
 
   // Step 2.2: the constraint check.  The paper's "empirically determined
@@ -124,7 +140,7 @@ struct Planner {
     Block a, b, m;
     if (!lowers(merged, &m)) return false;
     if (!lowers(cur, &a) || !lowers({cand}, &b)) { yellow_fused++; return true; }
-    bool ok = block_cost_us(g, m) <= block_cost_us(g, a) + block_cost_us(g, b);
+    bool ok = cost(m) <= cost(a) + cost(b);
     if (ok) yellow_fused++;
     return ok;
   }
@@ -199,7 +215,7 @@ struct Planner {
           if (!convex(merged)) continue;
           Block m, a, b;
           if (!lowers(merged, &m)) continue;
-          if (lowers(blocks[tb], &a) && lowers({o}, &b) && block_cost_us(g, m) > block_cost_us(g, a) + block_cost_us(g, b)) continue;
+          if (lowers(blocks[tb], &a) && lowers({o}, &b) && cost(m) > cost(a) + cost(b)) continue;
           blocks[tb] = merged; blocks[bi].clear(); block_of[o] = tb;
           changed = true;
           break;
@@ -212,7 +228,7 @@ struct Planner {
     if (members.empty()) return 0.0;
     Block b;
     if (!lowers(members, &b)) return 1e30;
-    return block_cost_us(g, b);
+    return cost(b);
   }
 
   // Second half of the same intra-block optimisation: an index-only operator at the END of
@@ -438,6 +454,11 @@ int plan_graph(Graph& g, uint32_t flags) {
   s.workspace_bytes = ws;
   s.n_yellow_decisions = P.yellow;
   s.n_yellow_fused = P.yellow_fused;
+  s.n_profile_hits = P.hits;
+  s.n_profile_misses = (int32_t)P.misses.size();
+  g.profile_hits = P.hits;
+  g.profile_misses.clear();
+  for (auto& kv : P.misses) g.profile_misses.push_back({kv.first, kv.second});
   return DNNF_OK;
 }
 

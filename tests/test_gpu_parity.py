@@ -9,6 +9,7 @@ import pytest
 
 from paper_2108_13342_b200 import binding as B
 from paper_2108_13342_b200 import workloads as W
+from oracle import interp as O
 from util import RTOL_BF16, RTOL_F32, check, close, graph, rnd, run_both
 
 pytestmark = pytest.mark.gpu
@@ -197,3 +198,50 @@ def test_layernorm_from_primitives_unfused_and_strict():
     wl = W.Workload(g, {"x": rnd((40, 96), 60), "g": rnd((96,), 61, 0.9, 1.1), "b": rnd((96,), 62)})
     check(wl, RTOL_F32, UNFUSED)
     check(wl, RTOL_F32, FUSED)
+
+
+def test_tensor_read_outside_its_block_is_written_in_full_when_a_slice_follows():
+    """t = X + b is a graph output AND feeds Slice -> Relu.  A block {Add, Slice, Relu} would iterate over the slice
+    only and leave two thirds of t unwritten: the planner has to keep the Slice out of the block that stores t."""
+    g = graph()
+    g.ext("X", (4, 8, 12)); g.ext("b", (12,))
+    t = g.add("Add", ["X", "b"], out="T")
+    g.mark_output(t)
+    s = g.add("Slice", [t], axis=-1, start=4, end=8)
+    g.mark_output(g.add("Relu", [s], out="Y"))
+    wl = W.Workload(g, {"X": rnd((4, 8, 12), 1), "b": rnd((12,), 2)})
+    sess = Session_poisoned(wl)
+    ref = O.run_graph(wl.graph, wl.inputs)
+    for n in ("T", "Y"):
+        close(sess.output(n), ref[n], RTOL_F32)
+
+
+def Session_poisoned(wl):
+    """A session whose output buffers start as NaN: an element that no kernel writes is caught."""
+    from paper_2108_13342_b200.runtime import Session
+    s = Session(wl, plan_flags=B.PLAN_FUSED, rewrite_flags=B.REWRITE_NONE)
+    for n in wl.graph.outputs:
+        s.buffers[n].fill_(float("nan"))
+    s.run()
+    assert s.g.status()[0] == 0
+    return s
+
+
+def test_profiling_database_measured_on_the_device_drives_the_plan():
+    """Section 4.3: candidate blocks of profile-dependent decisions are measured on the device, the plan is rebuilt
+    from the measurements alone, and it still computes the oracle's result."""
+    import torch
+    from paper_2108_13342_b200 import profile_db
+    B.profile_db_clear()
+    wl = W.encoder(layers=1, batch=2, seq=32, hidden=64, heads=4, ffn=128)
+    rounds = profile_db.fill(wl.graph, torch.device("cuda:0"), B.REWRITE_CANON_MACRO, scratch_bytes=64 << 20, iters=5)
+    assert rounds[0]["misses"] > 0 and rounds[0]["measured"] == rounds[0]["misses"], rounds
+    assert rounds[-1]["misses"] == 0 and rounds[-1]["hits"] > 0, rounds
+    assert B.profile_db_size() >= rounds[0]["measured"]
+    try:
+        s, got, ref = run_both(wl, B.PLAN_FUSED, B.REWRITE_CANON_MACRO)
+        (name,) = wl.graph.outputs
+        close(got[name], ref[name], RTOL_BF16)
+        assert s.plan_stats.n_profile_misses == 0
+    finally:
+        B.profile_db_clear()

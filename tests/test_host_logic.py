@@ -328,3 +328,63 @@ def test_unsupported_block_fails_the_plan_instead_of_falling_back():
     with pytest.raises(B.DnnfError) as e:
         gg.plan()
     assert e.value.code == B.ERR_UNSUPPORTED_OP
+
+
+# ---- profiling database (Section 4.3, Step 2.3) ----------------------------------------------------
+
+def _matmul_then_transpose():
+    g = W.GraphDesc("mm_t")
+    g.ext("A", (512, 64), "bf16"); g.ext("Bm", (64, 256), "bf16")
+    t = g.add("MatMul", ["A", "Bm"])
+    t = g.add("Relu", [t])                      # the One-to-One seed of Listing 1
+    g.mark_output(g.add("Transpose", [t], perm=(1, 0), out="Y"))
+    return g
+
+
+def test_profile_database_round_trip(tmp_path):
+    B.profile_db_clear()
+    assert B.profile_db_size() == 0 and B.profile_db_get("x|y") is None
+    B.profile_db_set("gemm|MatMul|bf16,bf16,->bf16,|M1N2K3B1v0|bytes10", 12.5)
+    B.profile_db_set("row|Softmax|f32,->f32,|rows8L16|bytes1024", 3.25)
+    assert B.profile_db_size() == 2
+    assert B.profile_db_get("row|Softmax|f32,->f32,|rows8L16|bytes1024") == 3.25
+    path = str(tmp_path / "db.tsv")
+    B.profile_db_save(path)
+    B.profile_db_clear()
+    assert B.profile_db_load(path) == 2
+    assert B.profile_db_get("gemm|MatMul|bf16,bf16,->bf16,|M1N2K3B1v0|bytes10") == 12.5
+    with pytest.raises(ValueError):
+        B.profile_db_set("bad", -1.0)
+    B.profile_db_clear()
+
+
+def test_yellow_decision_follows_the_profiling_database():
+    """Many-to-Many followed by Shuffle is a profile-dependent (yellow) cell of Table 3: with measured latencies in
+    the database the planner fuses exactly when the fused block is not slower than the two separate ones."""
+    B.profile_db_clear()
+    g = build_graph(_matmul_then_transpose())[0]
+    g.rewrite(B.REWRITE_NONE)
+    st = g.plan(B.PLAN_FUSED)
+    assert st.n_yellow_decisions >= 1 and st.n_profile_hits == 0 and st.n_profile_misses >= 3
+    misses = g.profile_misses()
+    fused = [m for m in misses if m.startswith("gemm|") and "Transpose" in m]
+    alone_mm = [m for m in misses if m.startswith("gemm|MatMul|")]
+    alone_t = [m for m in misses if m.startswith("transpose|")]
+    assert len(fused) == 1 and len(alone_mm) == 1 and len(alone_t) == 1, misses
+
+    # measured: fusing is a loss -> two kernels
+    B.profile_db_set(fused[0], 50.0); B.profile_db_set(alone_mm[0], 5.0); B.profile_db_set(alone_t[0], 4.0)
+    g2 = build_graph(_matmul_then_transpose())[0]
+    g2.rewrite(B.REWRITE_NONE)
+    st2 = g2.plan(B.PLAN_FUSED)
+    assert st2.n_kernels == 2 and st2.n_profile_hits >= 3 and st2.n_profile_misses == 0
+    assert g2.block_signature(0) == alone_mm[0]
+
+    # measured: fusing wins -> one kernel
+    B.profile_db_set(fused[0], 6.0)
+    g3 = build_graph(_matmul_then_transpose())[0]
+    g3.rewrite(B.REWRITE_NONE)
+    st3 = g3.plan(B.PLAN_FUSED)
+    assert st3.n_kernels == 1 and st3.n_yellow_fused >= 1
+    assert g3.block_signature(0) == fused[0]
+    B.profile_db_clear()
