@@ -139,6 +139,20 @@ def encoder_report(dev, pk, layers=12):
         per.append({"ops": "+".join(blocks[b]["ops"][:10]), "family": blocks[b]["family"], "us_warm_l2": round(t, 3), "bytes": by,
                     "flops": fl, "roofline_us": round(roof, 3), "frac_of_roofline": round(roof / t, 3)})
     out["layer_blocks_canon_plan"] = per
+    # Same graph planned from measured latencies (profiling database, Section 4.3) instead of the analytic model.
+    from . import profile_db
+    del s
+    torch.cuda.empty_cache()
+    B.profile_db_clear()
+    try:
+        rounds = profile_db.fill(wl.graph, dev, B.REWRITE_CANON_MACRO, scratch_bytes=1 << 30, iters=20)
+        r = measure_workload(torch, dev, wl, pk, B.PLAN_FUSED, 1, iters=10, rewrite=B.REWRITE_CANON_MACRO, per_block_limit=0)
+        r["profiling_rounds"] = rounds
+        r["database_entries"] = B.profile_db_size()
+        out["fused+layernorm-canon+profiled-plan"] = r
+    finally:
+        B.profile_db_clear()
+    torch.cuda.empty_cache()
     out["speedup_fused_vs_unfused_graph"] = round(out["unfused"]["us_cuda_graph"] / out["fused+layernorm-canon"]["us_cuda_graph"], 2)
     out["speedup_fused_vs_unfused_plain"] = round(out["unfused"]["us_plain_launches"] / out["fused+layernorm-canon"]["us_plain_launches"], 2)
     return out
