@@ -140,7 +140,9 @@ struct Rewriter {
   // Returns the factor list after one simplification step, or empty if none applies.
   bool simplify_factors(std::vector<int>& f, int& rule, std::vector<std::function<int()>>& make) {
     // two Sqrt of the same tensor -> that tensor                          (Table 4, Associative row 2)
+    // (a negative entry stands for a node that an earlier step of this simplification will create)
     for (size_t i = 0; i < f.size(); ++i) for (size_t j = i + 1; j < f.size(); ++j) {
+      if (f[i] < 0 || f[j] < 0) continue;
       const Op *a = producer(f[i]), *b = producer(f[j]);
       if (a && b && a->kind == DNNF_OP_SQRT && b->kind == DNNF_OP_SQRT && a->in[0] == b->in[0] && uses(f[i]) <= (f[i] == f[j] ? 2 : 1) && uses(f[j]) <= (f[i] == f[j] ? 2 : 1)) {
         int x = a->in[0];
@@ -151,7 +153,7 @@ struct Rewriter {
     }
     // the same factor twice -> Square(factor)                               (row 4)
     for (size_t i = 0; i < f.size(); ++i) for (size_t j = i + 1; j < f.size(); ++j) {
-      if (f[i] == f[j] && !g.tensors[f[i]].external) {
+      if (f[i] >= 0 && f[i] == f[j] && !g.tensors[f[i]].external) {
         int x = f[i];
         f.erase(f.begin() + j); f.erase(f.begin() + i);
         f.push_back(-(int)make.size() - 1);

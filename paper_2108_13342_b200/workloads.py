@@ -368,8 +368,87 @@ def encoder(layers=12, batch=8, seq=128, hidden=768, heads=12, ffn=3072,
     return Workload(g, inputs)
 
 
+# --------------------------------------------------------------------------
+# Workload 6: GPT-2 style decoder as primitive operators (pre-LayerNorm blocks, causal attention,
+# GELU in its tanh form spelled out; 53 operators per layer plus a final LayerNorm)
+# --------------------------------------------------------------------------
+
+def _gelu_tanh_primitives(g, x):
+    x2 = g.add("Mul", [x, x])
+    x3 = g.add("Mul", [x2, x])
+    t = g.add("MulC", [x3], c=0.044715)
+    t = g.add("Add", [x, t])
+    t = g.add("MulC", [t], c=math.sqrt(2.0 / math.pi))
+    t = g.add("Tanh", [t])
+    t = g.add("AddC", [t], c=1.0)
+    t = g.add("Mul", [x, t])
+    return g.add("MulC", [t], c=0.5)
+
+
+def decoder(layers=12, batch=8, seq=128, hidden=768, heads=12, ffn=3072, seed=BASE_SEED) -> Workload:
+    d = _Draw(seed + 6)
+    hd = hidden // heads
+    g = GraphDesc("decoder")
+    inputs = {}
+
+    def ext(name, shape, dtype, kind, arr):
+        g.ext(name, shape, dtype, kind)
+        inputs[name] = round_to_bf16(arr) if dtype == "bf16" else arr
+        return name
+
+    def vec(name, n, mean):
+        return ext(name, (n,), "f32", "weight", d.normal((n,), mean, 0.02))
+
+    x = ext("x", (batch, seq, hidden), "bf16", "input", d.normal((batch, seq, hidden), 0.0, 1.0))
+    ext("mask", (seq, seq), "f32", "weight", causal_mask(seq))
+    for l in range(layers):
+        p = f"L{l}."
+        g1, be1 = vec(p + "ln1.g", hidden, 1.0), vec(p + "ln1.b", hidden, 0.0)
+        wqkv = ext(p + "Wqkv", (hidden, 3 * hidden), "bf16", "weight", d.normal((hidden, 3 * hidden), 0.0, 0.02))
+        bqkv = vec(p + "bqkv", 3 * hidden, 0.0)
+        wo = ext(p + "Wo", (hidden, hidden), "bf16", "weight", d.normal((hidden, hidden), 0.0, 0.02))
+        bo = vec(p + "bo", hidden, 0.0)
+        g2, be2 = vec(p + "ln2.g", hidden, 1.0), vec(p + "ln2.b", hidden, 0.0)
+        w1 = ext(p + "W1", (hidden, ffn), "bf16", "weight", d.normal((hidden, ffn), 0.0, 0.02))
+        b1 = vec(p + "b1", ffn, 0.0)
+        w2 = ext(p + "W2", (ffn, hidden), "bf16", "weight", d.normal((ffn, hidden), 0.0, 0.02))
+        b2 = vec(p + "b2", hidden, 0.0)
+
+        h1 = _layernorm_primitives(g, x, g1, be1, 1e-5)
+        qkv = g.add("MatMul", [h1, wqkv])
+        qkv = g.add("Add", [qkv, bqkv])
+        q, k, v = g.add("Split", [qkv], n_out=3, axis=-1, sizes=(hidden, hidden, hidden))
+        hs = []
+        for t in (q, k, v):
+            t = g.add("Reshape", [t], shape=(batch, seq, heads, hd))
+            hs.append(g.add("Transpose", [t], perm=(0, 2, 1, 3)))
+        q, k, v = hs
+        kt = g.add("Transpose", [k], perm=(0, 1, 3, 2))
+        s = g.add("MatMul", [q, kt])
+        s = g.add("MulC", [s], c=1.0 / math.sqrt(hd))
+        s = g.add("Add", [s, "mask"])
+        pr = g.add("Softmax", [s], axis=-1)
+        a = g.add("MatMul", [pr, v])
+        a = g.add("Transpose", [a], perm=(0, 2, 1, 3))
+        a = g.add("Reshape", [a], shape=(batch, seq, hidden))
+        o = g.add("MatMul", [a, wo])
+        o = g.add("Add", [o, bo])
+        x = g.add("Add", [x, o])
+        h2 = _layernorm_primitives(g, x, g2, be2, 1e-5)
+        f = g.add("MatMul", [h2, w1])
+        f = g.add("Add", [f, b1])
+        f = _gelu_tanh_primitives(g, f)
+        f = g.add("MatMul", [f, w2])
+        f = g.add("Add", [f, b2])
+        x = g.add("Add", [x, f])
+    gf, bf = vec("lnf.g", hidden, 1.0), vec("lnf.b", hidden, 0.0)
+    x = _layernorm_primitives(g, x, gf, bf, 1e-5)
+    g.mark_output(x)
+    return Workload(g, inputs)
+
+
 def by_name(name: str, **kw) -> Workload:
     table = {"swish_transpose": swish_transpose, "masked_softmax": masked_softmax,
              "add_layernorm_gelu": add_layernorm_gelu, "ffn_block": ffn_block,
-             "mbconv_block": mbconv_block, "encoder": encoder}
+             "mbconv_block": mbconv_block, "encoder": encoder, "decoder": decoder}
     return table[name](**kw)

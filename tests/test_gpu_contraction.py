@@ -255,6 +255,17 @@ def test_encoder_small(flags, rewrite):
         assert s.plan_stats.n_kernels <= 2 * 11
 
 
+@pytest.mark.parametrize("flags,rewrite", [(FUSED, B.REWRITE_NONE), (UNFUSED, B.REWRITE_NONE), (FUSED, B.REWRITE_DEFAULT), (FUSED, B.REWRITE_CANON_MACRO)])
+def test_decoder_small(flags, rewrite):
+    """GPT-2 style decoder (pre-LayerNorm, GELU by tanh spelled out in primitives, final LayerNorm)."""
+    wl = W.decoder(layers=2, batch=2, seq=32, hidden=64, heads=4, ffn=128)
+    s, got, ref = run_both(wl, flags, rewrite)
+    (name,) = wl.graph.outputs
+    close(got[name], ref[name], RTOL_BF16)
+    if flags == FUSED:
+        assert s.plan_stats.n_kernels <= 2 * 12 + 1
+
+
 def test_encoder_full_size_one_layer_elementwise():
     wl = W.encoder(layers=1)
     for flags, rw, kernels in [(FUSED, B.REWRITE_CANON_MACRO, 9), (FUSED, B.REWRITE_DEFAULT, 11)]:

@@ -63,6 +63,7 @@ def _mixed_graph():
 CASES = [("mixed", _mixed_graph, B.REWRITE_NONE, RTOL_F32),
          ("encoder", lambda: W.encoder(layers=2, batch=2, seq=32, hidden=64, heads=4, ffn=128), B.REWRITE_CANON_MACRO, RTOL_BF16),
          ("encoder-primitive", lambda: W.encoder(layers=1, batch=2, seq=32, hidden=64, heads=4, ffn=128), B.REWRITE_DEFAULT, RTOL_BF16),
+         ("decoder", lambda: W.decoder(layers=1, batch=2, seq=32, hidden=64, heads=4, ffn=128), B.REWRITE_CANON_MACRO, RTOL_BF16),
          ("mbconv", lambda: W.mbconv_block(2, 14, 14, 24, 144), B.REWRITE_NONE, RTOL_F32),
          ("ffn", lambda: W.ffn_block(256, 64, 128), B.REWRITE_NONE, RTOL_BF16)]
 

@@ -330,6 +330,22 @@ def test_unsupported_block_fails_the_plan_instead_of_falling_back():
     assert e.value.code == B.ERR_UNSUPPORTED_OP
 
 
+def test_product_of_three_equal_computed_factors_is_handled():
+    """x*x*x with x computed inside the graph: the associative Square rule is tried (Square(x) * x has the same #FLOPS,
+    so it need not be kept); the placeholder for the not-yet-created Square must not be looked up as a tensor by the
+    next simplification step (that was an out-of-bounds read)."""
+    g = W.GraphDesc("cube")
+    g.ext("A", (8, 16)); g.ext("Bv", (16,))
+    x = g.add("Add", ["A", "Bv"])
+    x2 = g.add("Mul", [x, x])
+    g.mark_output(g.add("Mul", [x2, x], out="Y"))
+    G = build_graph(g)[0]
+    st = G.rewrite(B.REWRITE_DEFAULT)
+    kinds = sorted(B.OP_NAMES[G.op_kind(i)[0]] for i in range(G.op_count()) if G.op_kind(i)[1])
+    assert kinds in (["Add", "Mul", "Mul"], ["Add", "Mul", "Square"]), kinds
+    assert st.ops_after == 3 and st.flops_after <= st.flops_before
+
+
 # ---- profiling database (Section 4.3, Step 2.3) ----------------------------------------------------
 
 def _matmul_then_transpose():
