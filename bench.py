@@ -353,6 +353,10 @@ def main():
             line["detail"]["cfg5 12-layer encoder (576 primitive operators)"] = report.encoder_report(dev, pk)
         except Exception as e:
             line["detail"]["cfg5 12-layer encoder (576 primitive operators)"] = {"error": repr(e)}
+        try:
+            line["detail"]["next: 12-layer GPT-2 style decoder (633 primitive operators)"] = report.decoder_report(dev, pk)
+        except Exception as e:  # noqa: BLE001
+            line["detail"]["next: 12-layer GPT-2 style decoder (633 primitive operators)"] = {"error": repr(e)}
         line["paper_context"] = {"note": "mobile-device figures from the paper, not comparable hardware",
                                  "fusion_rate_vs_other_frameworks": "up to 8.8x", "speedup_vs_other_frameworks": "up to 9.3x",
                                  "speedup_vs_own_unfused_backend": "1.5-5.8x"}

@@ -141,7 +141,7 @@ __device__ __forceinline__ void apply_op(int op, float (&acc)[VV], const float (
       break;
     case M_TANH:
 #pragma unroll
-      for (int v = 0; v < VV; ++v) acc[v] = tanhf(acc[v]);
+      for (int v = 0; v < VV; ++v) acc[v] = kFast ? fast_tanh(acc[v]) : tanhf(acc[v]);
       break;
     case M_ERF:
 #pragma unroll

@@ -240,8 +240,12 @@ DNNF_SP_BEGIN(EP_ScaleMask, 4) MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_CONST, 0), MO
 DNNF_SP_BEGIN(EP_BiasGeluPrimitives, 9)
   MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_SAVE, S_TMP, 0), MO(M_MUL, S_CONST, 0), MO(M_ERF, S_NONE, 0), MO(M_ADD, S_CONST, 1),
   MO(M_MUL, S_TMP, 0), MO(M_MUL, S_CONST, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(EP_BiasGeluTanhPrimitives, 13)
+  MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_SAVE, S_TMP, 0), MO(M_SQUARE, S_NONE, 0), MO(M_MUL, S_TMP, 0), MO(M_MUL, S_CONST, 0),
+  MO(M_ADD, S_TMP, 0), MO(M_MUL, S_CONST, 1), MO(M_TANH, S_NONE, 0), MO(M_ADD, S_CONST, 2), MO(M_MUL, S_TMP, 0), MO(M_MUL, S_CONST, 3),
+  MO(M_STORE, S_NONE, 0) DNNF_SP_END
 #undef MO
-using EpiStatic = TypeList<EP_Store, EP_Bias, EP_BiasGeluTanh, EP_BiasResidual, EP_ScaleMask, EP_BiasGeluPrimitives>;
+using EpiStatic = TypeList<EP_Store, EP_Bias, EP_BiasGeluTanh, EP_BiasResidual, EP_ScaleMask, EP_BiasGeluPrimitives, EP_BiasGeluTanhPrimitives>;
 
 // ---- host side --------------------------------------------------------------------------------------
 static GemmParams& gp_of(Launch& L) { return *reinterpret_cast<GemmParams*>(L.blob.data()); }

@@ -156,3 +156,19 @@ def encoder_report(dev, pk, layers=12):
     out["speedup_fused_vs_unfused_graph"] = round(out["unfused"]["us_cuda_graph"] / out["fused+layernorm-canon"]["us_cuda_graph"], 2)
     out["speedup_fused_vs_unfused_plain"] = round(out["unfused"]["us_plain_launches"] / out["fused+layernorm-canon"]["us_plain_launches"], 2)
     return out
+
+
+def decoder_report(dev, pk, layers=12):
+    """Second whole-graph workload: a GPT-2 style decoder as primitive operators.  The analogue of the paper's
+    optimisation breakdown: one kernel per operator / fusion without rewriting / fusion after the printed rewriting
+    rules / fusion after LayerNorm canonicalisation."""
+    import torch
+    wl = W.decoder(layers=layers)
+    out = {}
+    for name, flags, rw in [("unfused", B.PLAN_UNFUSED, B.REWRITE_NONE), ("fused, no rewriting", B.PLAN_FUSED, B.REWRITE_NONE),
+                            ("fused + printed rules", B.PLAN_FUSED, B.REWRITE_DEFAULT),
+                            ("fused + layernorm-canon", B.PLAN_FUSED, B.REWRITE_CANON_MACRO)]:
+        out[name] = measure_workload(torch, dev, wl, pk, flags, 1, iters=10, rewrite=rw, per_block_limit=0)
+        torch.cuda.empty_cache()
+    out["speedup_fused_vs_unfused_graph"] = round(out["unfused"]["us_cuda_graph"] / out["fused + layernorm-canon"]["us_cuda_graph"], 2)
+    return out
