@@ -79,6 +79,11 @@ DNNF_SP_BEGIN(SP_BiasResidualLayerNorm, 16)
   MO(M_MOV, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_ADD, S_IN, 2), MO(M_SAVE, S_TMP, 0), MO(M_ROWMEAN, S_NONE, 0),
   MO(M_RSUB, S_TMP, 0), MO(M_SAVE, S_TMP, 0), MO(M_SQUARE, S_NONE, 0), MO(M_ROWMEAN, S_NONE, 0), MO(M_ADD, S_CONST, 0),
   MO(M_SQRT, S_NONE, 0), MO(M_RECIP, S_NONE, 0), MO(M_MUL, S_TMP, 0), MO(M_MUL, S_IN, 3), MO(M_ADD, S_IN, 4), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+// the same with the sum also stored (pre-LayerNorm blocks keep the residual stream): outputs 0 = sum, 1 = normalised
+DNNF_SP_BEGIN(SP_BiasResidualStoreLayerNorm, 17)
+  MO(M_MOV, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_ADD, S_IN, 2), MO(M_STORE, S_NONE, 0), MO(M_SAVE, S_TMP, 0), MO(M_ROWMEAN, S_NONE, 0),
+  MO(M_RSUB, S_TMP, 0), MO(M_SAVE, S_TMP, 0), MO(M_SQUARE, S_NONE, 0), MO(M_ROWMEAN, S_NONE, 0), MO(M_ADD, S_CONST, 0),
+  MO(M_SQRT, S_NONE, 0), MO(M_RECIP, S_NONE, 0), MO(M_MUL, S_TMP, 0), MO(M_MUL, S_IN, 3), MO(M_ADD, S_IN, 4), MO(M_STORE, S_NONE, 1) DNNF_SP_END
 
 #undef MO
 
@@ -87,7 +92,8 @@ using EwStatic = TypeList<SP_Move, SP_BiasScaleSwish, SP_AddIn, SP_MulIn, SP_Mul
                           SP_GeluPrimitives, SP_ScaleShift, SP_Clip, SP_AddC, SP_Erf, SP_GeluTanh, SP_SubIn, SP_DivIn, SP_Square, SP_Sqrt,
                           SP_Relu>;
 using TrStatic = TypeList<SP_Move, SP_BiasScaleSwish>;
-using RowStatic = TypeList<SP_ScaleMaskSoftmax, SP_Softmax, SP_AddLayerNormGelu, SP_LayerNorm, SP_BiasResidualLayerNorm>;
+using RowStatic = TypeList<SP_ScaleMaskSoftmax, SP_Softmax, SP_AddLayerNormGelu, SP_LayerNorm, SP_BiasResidualLayerNorm,
+                           SP_BiasResidualStoreLayerNorm>;
 
 template <class SP>
 inline bool program_matches(const Program& p) {
