@@ -53,7 +53,7 @@ def build(force=False, verbose=False):
         f.write("\n".join(log))
     if verbose:
         print("\n".join(log))
-    cmd = [NVCC, "-shared", "-o", LIB, *objs, "-Xlinker", "--exclude-libs,ALL"]
+    cmd = [NVCC, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB, *objs, "-Xlinker", "--exclude-libs,ALL"]
     subprocess.check_call(cmd)
     return LIB
 
