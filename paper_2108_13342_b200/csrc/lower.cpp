@@ -652,7 +652,11 @@ static int lower_elementwise_or_row(const Graph& g, const std::vector<int>& ops,
   if (ref < 0) { why = "block has no output"; return DNNF_ERR_UNSUPPORTED_OP; }
   cx.ext = g.tensors[ref].dims;
   if (cx.ext.empty()) cx.ext.push_back(1);
+  const int64_t row_len = cx.ext.back();
   if (!derive_views(cx, ref, {})) { why = cx.why; return DNNF_ERR_UNSUPPORTED_OP; }
+  // Aligning the views may split iteration dims (a Reshape across a Slice, say).  The reduced axis has to stay one
+  // dim: the row kernels reduce over the innermost dim only.
+  if (anchor >= 0 && cx.ext.back() != row_len) { why = "the reduced axis is not a single run of elements in every operand"; return DNNF_ERR_UNSUPPORTED_OP; }
   if (!emit_program(cx, -1, anchor >= 0 ? 2 : kMaxTmp)) { why = cx.why; return DNNF_ERR_UNSUPPORTED_OP; }
 
   Packed p;

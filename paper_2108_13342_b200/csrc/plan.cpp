@@ -329,6 +329,19 @@ double block_cost_us(const Graph& g, const Block& b) {
 
 int plan_graph(Graph& g, uint32_t flags) {
   g.relink();
+  // Operators whose results nobody reads (not a graph output, no live consumer) are not planned: they would
+  // form blocks without an output.  (The rewriting pass removes them as well; a graph planned without rewriting
+  // may still carry some.)
+  for (bool changed = true; changed;) {
+    changed = false;
+    for (auto& o : g.ops) {
+      if (!o.alive) continue;
+      bool used = false;
+      for (int t : o.out) if (g.tensors[t].is_output || !g.tensors[t].consumers.empty()) used = true;
+      if (!used) { o.alive = false; changed = true; }
+    }
+    if (changed) g.relink();
+  }
   g.blocks.clear(); g.run_order.clear();
   g.planned = false;
   for (auto& o : g.ops) { o.block = -1; if (o.alive) o.mapping = node_mapping(g, o); }

@@ -1,0 +1,136 @@
+"""Random operator graphs against the oracle.  A seeded generator strings bounded element-wise operators, broadcasts
+against vectors and full tensors, transposes, reshapes, slices, last-axis reductions, Softmax / LayerNorm and
+matrix products into DAGs with several outputs; every graph runs fused (and un-fused) with outputs and workspace
+poisoned by NaN, and has to reproduce the oracle."""
+import numpy as np
+import pytest
+
+from paper_2108_13342_b200 import binding as B
+from paper_2108_13342_b200 import workloads as W
+from paper_2108_13342_b200.runtime import Session
+from oracle import interp as O
+from util import RTOL_F32, close, graph
+
+pytestmark = pytest.mark.gpu
+
+
+class _Rng:
+    """Counter-based draws from the shared input generator (no method arithmetic here)."""
+    def __init__(self, seed):
+        self.seed, self.n = seed, 0
+
+    def u(self):
+        self.n += 1
+        return float(W.uniform(4242 + self.seed, self.n, (1,), 0.0, 1.0)[0])
+
+    def pick(self, xs):
+        return xs[min(int(self.u() * len(xs)), len(xs) - 1)]
+
+
+def _build(seed):
+    r = _Rng(seed)
+    bsz, rows, cols = r.pick([1, 2, 3]), r.pick([5, 8, 16, 33]), r.pick([8, 12, 32, 64])
+    g = graph("rand%d" % seed)
+    ins = {}
+    g.ext("X", (bsz, rows, cols)); ins["X"] = W.uniform(777, 1000 + seed, (bsz, rows, cols), -1.0, 1.0)
+    g.ext("X2", (bsz, rows, cols)); ins["X2"] = W.uniform(777, 2000 + seed, (bsz, rows, cols), -1.0, 1.0)
+    pool = [("X", (bsz, rows, cols)), ("X2", (bsz, rows, cols))]
+    n_ext = [0]
+
+    def vec(n, lo, hi):
+        n_ext[0] += 1
+        name = "v%d" % n_ext[0]
+        g.ext(name, (n,)); ins[name] = W.uniform(777, 3000 + 10 * seed + n_ext[0], (n,), lo, hi)
+        return name
+
+    def mat(k, n):
+        n_ext[0] += 1
+        name = "m%d" % n_ext[0]
+        g.ext(name, (k, n)); ins[name] = W.uniform(777, 4000 + 10 * seed + n_ext[0], (k, n), -0.3, 0.3)
+        return name
+
+    n_ops = 4 + int(r.u() * 9)
+    for _ in range(n_ops):
+        t, shp = r.pick(pool[-4:])                      # prefer recent values: longer chains
+        kind = r.pick(["unary", "unary", "vec", "full", "transpose", "reshape", "slice", "reduce", "softmax", "layernorm", "matmul"])
+        if kind == "unary":
+            op, at = r.pick([("Tanh", {}), ("Sigmoid", {}), ("Relu", {}), ("Abs", {}), ("Square", {}), ("Neg", {}),
+                             ("MulC", {"c": 0.5}), ("AddC", {"c": 0.25}), ("Gelu", {"approx": "erf"}), ("Erf", {})])
+            if op == "Square":
+                t = g.add("Tanh", [t])                  # keep magnitudes bounded
+            o = g.add(op, [t], **at)
+        elif kind == "vec":
+            o = g.add(r.pick(["Add", "Mul", "Sub"]), [t, vec(shp[-1], 0.5, 1.5)])
+        elif kind == "full":
+            cands = [p for p in pool if p[1] == shp and p[0] != t]
+            if not cands:
+                continue
+            o = g.add(r.pick(["Add", "Mul", "Sub"]), [t, r.pick(cands)[0]])
+            o = g.add("Tanh", [o])
+        elif kind == "transpose":
+            if len(shp) < 2:
+                continue
+            perm = list(range(len(shp)))
+            i, j = len(shp) - 1, int(r.u() * (len(shp) - 1))
+            perm[i], perm[j] = perm[j], perm[i]
+            o = g.add("Transpose", [t], perm=tuple(perm))
+            shp = tuple(shp[p] for p in perm)
+        elif kind == "reshape":
+            if len(shp) == 3:
+                new = (shp[0] * shp[1], shp[2]) if r.u() < 0.5 else (shp[0], shp[1] * shp[2])
+            elif len(shp) == 2 and shp[0] % 2 == 0:
+                new = (2, shp[0] // 2, shp[1])
+            else:
+                continue
+            o = g.add("Reshape", [t], shape=new)
+            shp = new
+        elif kind == "slice":
+            ax = int(r.u() * len(shp))
+            if shp[ax] < 4:
+                continue
+            a = int(r.u() * (shp[ax] // 2)); e = a + max(1, int(r.u() * (shp[ax] - a)))
+            o = g.add("Slice", [t], axis=ax, start=a, end=e)
+            shp = shp[:ax] + (e - a,) + shp[ax + 1:]
+        elif kind == "reduce":
+            o = g.add(r.pick(["ReduceSum", "ReduceMean", "ReduceMax"]), [t], axis=-1, keepdims=1)
+            shp = shp[:-1] + (1,)
+        elif kind == "softmax":
+            o = g.add("Softmax", [t], axis=-1)
+        elif kind == "layernorm":
+            if shp[-1] < 4:
+                continue
+            o = g.add("LayerNorm", [t, vec(shp[-1], 0.8, 1.2), vec(shp[-1], -0.2, 0.2)], axis=-1, eps=1e-5)
+        else:
+            n = r.pick([8, 16, 24])
+            o = g.add("MatMul", [t, mat(shp[-1], n)])
+            shp = shp[:-1] + (n,)
+        if kind not in ("transpose", "reshape", "slice", "reduce", "matmul"):
+            pass
+        pool.append((o, shp))
+    outs = {pool[-1][0]}
+    for _ in range(int(r.u() * 3)):
+        cand = r.pick(pool[2:])
+        outs.add(cand[0])
+    for i, o in enumerate(sorted(outs)):
+        g.mark_output(o)
+    return W.Workload(g, ins)
+
+
+@pytest.mark.parametrize("seed", range(200))
+def test_random_graph(seed):
+    wl = _build(seed)
+    ref = O.run_graph(wl.graph, wl.inputs)
+    for flags in (B.PLAN_FUSED, B.PLAN_UNFUSED):
+        s = Session(wl, plan_flags=flags, rewrite_flags=B.REWRITE_NONE)
+        s.workspace[s.g.workspace_zero_bytes():].fill_(0xFF)
+        for n in wl.graph.outputs:
+            s.buffers[n].fill_(float("nan"))
+        s.run()
+        assert s.g.status()[0] == 0
+        for n in wl.graph.outputs:
+            got = s.output(n)
+            assert np.isfinite(got).all(), (n, "unwritten elements", [b["ops"] for b in s.g.blocks()])
+            try:
+                close(got, ref[n], 2e-5)
+            except AssertionError as e:
+                raise AssertionError(f"{n} plan {[b['ops'] for b in s.g.blocks()]}: {e}") from None
