@@ -27,9 +27,11 @@ class _Rng:
         return xs[min(int(self.u() * len(xs)), len(xs) - 1)]
 
 
-def _build(seed):
+def _build(seed, big=False):
     r = _Rng(seed)
     bsz, rows, cols = r.pick([1, 2, 3]), r.pick([5, 8, 16, 33]), r.pick([8, 12, 32, 64])
+    if big:      # sizes that reach the vectorised, multi-vector, multi-warp and tensor-core variants
+        bsz, rows, cols = r.pick([1, 2, 4]), r.pick([96, 256, 520, 1024]), r.pick([128, 256, 768, 1000, 2048])
     g = graph("rand%d" % seed)
     ins = {}
     g.ext("X", (bsz, rows, cols)); ins["X"] = W.uniform(777, 1000 + seed, (bsz, rows, cols), -1.0, 1.0)
@@ -51,14 +53,42 @@ def _build(seed):
 
     n_ops = 4 + int(r.u() * 9)
     for _ in range(n_ops):
-        t, shp = r.pick(pool[-4:])                      # prefer recent values: longer chains
-        kind = r.pick(["unary", "unary", "vec", "full", "transpose", "reshape", "slice", "reduce", "softmax", "layernorm", "matmul"])
+        t, shp = r.pick(pool[-4:]) if r.u() < 0.7 else r.pick(pool)      # mostly recent values (long chains), sometimes old ones (diamonds)
+        kind = r.pick(["unary", "unary", "vec", "full", "transpose", "reshape", "slice", "reduce", "softmax", "layernorm", "matmul",
+                       "rowvec", "exp", "div", "reduce0", "permute"])
+        if kind in ("reduce", "reduce0", "softmax", "layernorm") and shp[-1] > 8192:
+            continue                                    # longer rows than the row kernels take (the plan says so)
         if kind == "unary":
             op, at = r.pick([("Tanh", {}), ("Sigmoid", {}), ("Relu", {}), ("Abs", {}), ("Square", {}), ("Neg", {}),
                              ("MulC", {"c": 0.5}), ("AddC", {"c": 0.25}), ("Gelu", {"approx": "erf"}), ("Erf", {})])
             if op == "Square":
                 t = g.add("Tanh", [t])                  # keep magnitudes bounded
             o = g.add(op, [t], **at)
+        elif kind == "exp":
+            o = g.add("Exp", [g.add("MulC", [g.add("Tanh", [t])], c=0.5)])
+        elif kind == "div":
+            cands = [p for p in pool if p[1] == shp]
+            den = g.add("AddC", [g.add("Abs", [g.add("Tanh", [r.pick(cands)[0]])])], c=1.5)
+            o = g.add("Div", [g.add("Tanh", [t]), den])
+        elif kind == "rowvec":
+            if len(shp) < 2:
+                continue
+            n_ext[0] += 1
+            name = "c%d" % n_ext[0]
+            cshape = shp[:-1] + (1,)
+            g.ext(name, cshape); ins[name] = W.uniform(777, 5000 + 10 * seed + n_ext[0], cshape, 0.5, 1.5)
+            o = g.add(r.pick(["Add", "Mul"]), [t, name])
+        elif kind == "reduce0":
+            if len(shp) < 2:
+                continue
+            o = g.add(r.pick(["ReduceSum", "ReduceMax"]), [g.add("Tanh", [t])], axis=-1, keepdims=0)
+            shp = shp[:-1]
+        elif kind == "permute":
+            if len(shp) != 3:
+                continue
+            perm = r.pick([(0, 2, 1), (1, 0, 2), (2, 1, 0), (1, 2, 0), (2, 0, 1)])
+            o = g.add("Transpose", [t], perm=perm)
+            shp = tuple(shp[p] for p in perm)
         elif kind == "vec":
             o = g.add(r.pick(["Add", "Mul", "Sub"]), [t, vec(shp[-1], 0.5, 1.5)])
         elif kind == "full":
@@ -116,21 +146,45 @@ def _build(seed):
     return W.Workload(g, ins)
 
 
-@pytest.mark.parametrize("seed", range(200))
+def _random_db(wl, seed):
+    """Pseudo-random latencies for every candidate block the planner asks about (odd seeds: growing with block size)."""
+    from paper_2108_13342_b200.runtime import build_graph
+    for rnd_ in range(4):
+        g = build_graph(wl.graph)[0]
+        g.rewrite(B.REWRITE_NONE)
+        g.plan(B.PLAN_FUSED)
+        misses = g.profile_misses()
+        if not misses:
+            break
+        for i, sig in enumerate(misses):
+            u = float(W.uniform(9100 + seed, 100 * rnd_ + i, (1,), 1.0, 20.0)[0])
+            if seed % 2:
+                u *= 1 + 3 * sig.split("|")[1].count("+")
+            B.profile_db_set(sig, u)
+
+
+@pytest.mark.parametrize("seed", [pytest.param(i, id=str(i)) for i in range(300)] + [pytest.param(-i - 1, id="big%d" % i) for i in range(60)])
 def test_random_graph(seed):
-    wl = _build(seed)
+    wl = _build(seed, False) if seed >= 0 else _build(1000 - seed, True)
     ref = O.run_graph(wl.graph, wl.inputs)
-    for flags in (B.PLAN_FUSED, B.PLAN_UNFUSED):
-        s = Session(wl, plan_flags=flags, rewrite_flags=B.REWRITE_NONE)
-        s.workspace[s.g.workspace_zero_bytes():].fill_(0xFF)
-        for n in wl.graph.outputs:
-            s.buffers[n].fill_(float("nan"))
-        s.run()
-        assert s.g.status()[0] == 0
-        for n in wl.graph.outputs:
-            got = s.output(n)
-            assert np.isfinite(got).all(), (n, "unwritten elements", [b["ops"] for b in s.g.blocks()])
-            try:
-                close(got, ref[n], 2e-5)
-            except AssertionError as e:
-                raise AssertionError(f"{n} plan {[b['ops'] for b in s.g.blocks()]}: {e}") from None
+    for flags, rewrite, db in ((B.PLAN_FUSED, B.REWRITE_NONE, False), (B.PLAN_UNFUSED, B.REWRITE_NONE, False),
+                               (B.PLAN_FUSED, B.REWRITE_DEFAULT, False), (B.PLAN_FUSED, B.REWRITE_NONE, True)):
+        B.profile_db_clear()
+        try:
+            if db:
+                _random_db(wl, seed)
+            s = Session(wl, plan_flags=flags, rewrite_flags=rewrite)
+            s.workspace[s.g.workspace_zero_bytes():].fill_(0xFF)
+            for n in wl.graph.outputs:
+                s.buffers[n].fill_(float("nan"))
+            s.run()
+            assert s.g.status()[0] == 0
+            for n in wl.graph.outputs:
+                got = s.output(n)
+                assert np.isfinite(got).all(), (n, "unwritten elements", [b["ops"] for b in s.g.blocks()])
+                try:
+                    close(got, ref[n], 2e-5)
+                except AssertionError as e:
+                    raise AssertionError(f"{n} flags {flags} rewrite {rewrite} db {db} plan {[b['ops'] for b in s.g.blocks()]}: {e}") from None
+        finally:
+            B.profile_db_clear()
