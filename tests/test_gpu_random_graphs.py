@@ -27,15 +27,17 @@ class _Rng:
         return xs[min(int(self.u() * len(xs)), len(xs) - 1)]
 
 
-def _build(seed, big=False):
+def _build(seed, big=False, dtype="f32"):
     r = _Rng(seed)
     bsz, rows, cols = r.pick([1, 2, 3]), r.pick([5, 8, 16, 33]), r.pick([8, 12, 32, 64])
     if big:      # sizes that reach the vectorised, multi-vector, multi-warp and tensor-core variants
         bsz, rows, cols = r.pick([1, 2, 4]), r.pick([96, 256, 520, 1024]), r.pick([128, 256, 768, 1000, 2048])
     g = graph("rand%d" % seed)
     ins = {}
-    g.ext("X", (bsz, rows, cols)); ins["X"] = W.uniform(777, 1000 + seed, (bsz, rows, cols), -1.0, 1.0)
-    g.ext("X2", (bsz, rows, cols)); ins["X2"] = W.uniform(777, 2000 + seed, (bsz, rows, cols), -1.0, 1.0)
+    def data(a):
+        return W.round_to_bf16(a) if dtype == "bf16" else a
+    g.ext("X", (bsz, rows, cols), dtype); ins["X"] = data(W.uniform(777, 1000 + seed, (bsz, rows, cols), -1.0, 1.0))
+    g.ext("X2", (bsz, rows, cols), dtype); ins["X2"] = data(W.uniform(777, 2000 + seed, (bsz, rows, cols), -1.0, 1.0))
     pool = [("X", (bsz, rows, cols)), ("X2", (bsz, rows, cols))]
     n_ext = [0]
 
@@ -48,10 +50,10 @@ def _build(seed, big=False):
     def mat(k, n):
         n_ext[0] += 1
         name = "m%d" % n_ext[0]
-        g.ext(name, (k, n)); ins[name] = W.uniform(777, 4000 + 10 * seed + n_ext[0], (k, n), -0.3, 0.3)
+        g.ext(name, (k, n), dtype); ins[name] = data(W.uniform(777, 4000 + 10 * seed + n_ext[0], (k, n), -0.3, 0.3))
         return name
 
-    n_ops = 4 + int(r.u() * 9)
+    n_ops = 4 + int(r.u() * (4 if dtype == "bf16" else 9))
     for _ in range(n_ops):
         t, shp = r.pick(pool[-4:]) if r.u() < 0.7 else r.pick(pool)      # mostly recent values (long chains), sometimes old ones (diamonds)
         kind = r.pick(["unary", "unary", "vec", "full", "transpose", "reshape", "slice", "reduce", "softmax", "layernorm", "matmul",
@@ -188,3 +190,24 @@ def test_random_graph(seed):
                     raise AssertionError(f"{n} flags {flags} rewrite {rewrite} db {db} plan {[b['ops'] for b in s.g.blocks()]}: {e}") from None
         finally:
             B.profile_db_clear()
+
+
+@pytest.mark.parametrize("seed", range(80))
+def test_random_graph_bf16(seed):
+    """bf16 activations and weights (vectors stay fp32), short chains, fused plan: intermediates stay in fp32 inside a
+    block, every stored tensor is rounded to bf16."""
+    wl = _build(2000 + seed, seed % 4 == 3, "bf16")
+    ref = O.run_graph(wl.graph, wl.inputs)
+    s = Session(wl, plan_flags=B.PLAN_FUSED, rewrite_flags=B.REWRITE_NONE)
+    s.workspace[s.g.workspace_zero_bytes():].fill_(0xFF)
+    for n in wl.graph.outputs:
+        s.buffers[n].fill_(float("nan"))
+    s.run()
+    assert s.g.status()[0] == 0
+    for n in wl.graph.outputs:
+        got = s.output(n)
+        assert np.isfinite(got).all(), (n, "unwritten elements", [b["ops"] for b in s.g.blocks()])
+        try:
+            close(got, ref[n], 3e-2)
+        except AssertionError as e:
+            raise AssertionError(f"{n} plan {[b['ops'] for b in s.g.blocks()]}: {e}") from None
