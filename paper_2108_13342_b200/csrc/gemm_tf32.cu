@@ -585,6 +585,11 @@ bool tf32_gemm_eligible(const GemmParams& gp) {
   if (gp.K > 244) return false;                              // a whole row of A (padded) must fit one TMA box of 256 floats
   if (gp.N > 192 || gp.M < 4 * tf32::BM) return false;       // two accumulator stages and two A stages must fit in 512 TMEM columns
   if (tf32_b_bytes(gp) > tf32::kMaxBBytes) return false;
+  {   // tensor-memory budget (same arithmetic as the plan): never launch with fewer than two A stages
+    const int npad = tf32_npad(gp.N);
+    const bool dual = 4 * npad + 2 * tf32::kAStageCols <= 512;
+    if ((512 - 2 * (dual ? 2 : 1) * npad) / tf32::kAStageCols < 2) return false;
+  }
   // a whole tile of raw rows must be resident: the converter warps advance chunk by chunk together
   const int kr = (gp.K + 3) / 4 * 4, pitch = kr + ((kr / 4) % 2 == 0 ? 4 : 8);
   if ((tf32::kSmemMax - tf32::kFixed - tf32_b_bytes(gp)) / ((32 * pitch * 4 + 1023) / 1024 * 1024) < 4) return false;
@@ -611,7 +616,8 @@ void tf32_gemm_plan(Launch& L) {
   tf32::Params& q = fp_of(L);
   q.k_chunks = (gp.K + tf32::BK - 1) / tf32::BK;
   q.npad = tf32_npad(gp.N);
-  q.dual = 2 * q.npad <= 256 && !getenv("DNNF_TF32_NO_DUAL");
+  // tensor memory: two accumulator stages (twice as wide in the dual form) and at least two A stages must fit 512 columns
+  q.dual = 4 * q.npad + 2 * tf32::kAStageCols <= 512 && !getenv("DNNF_TF32_NO_DUAL");
   q.fast_epi = fast_epilogue(gp, q.slot) && !getenv("DNNF_TF32_GENERAL_EPILOGUE");
   q.b_static = gp.static_mask & 1u;
   q.fd_n = make_fastdiv((uint32_t)gp.N); q.fd_npad = make_fastdiv((uint32_t)q.npad); q.fd_kpad = make_fastdiv((uint32_t)(q.k_chunks * tf32::BK));

@@ -160,7 +160,8 @@ def test_conv1x1_with_epilogue(cfg):
 
 # fp32 blocks on the tensor cores (split-TF32): tall-and-skinny shapes, ragged M, N and K
 @pytest.mark.parametrize("cfg", [(2, 16, 16, 24, 144), (3, 19, 23, 144, 24), (1, 30, 31, 12, 20), (1, 40, 40, 36, 160), (4, 16, 16, 32, 192),
-                                 (1, 33, 33, 100, 8), (2, 24, 24, 96, 48)])
+                                 (1, 33, 33, 100, 8), (2, 24, 24, 96, 48),
+                                 (1, 29, 89, 32, 124), (1, 40, 40, 16, 100), (1, 40, 40, 16, 96)])
 @pytest.mark.parametrize("epi", ["clip", "residual", "none"])
 def test_conv1x1_tensor_core_fp32(cfg, epi):
     n, h, w, ci, co = cfg
