@@ -44,7 +44,7 @@ def _bf(a):
     return W.round_to_bf16(a)
 
 
-@pytest.mark.parametrize("seed", range(70))
+@pytest.mark.parametrize("seed", range(160))
 def test_random_bf16_gemm(seed):
     m = _pick(seed, 1, [1, 7, 64, 129, 256, 300, 512, 777, 1024, 1500])
     n = 8 * (1 + int(_u(seed, 2) * 90))
@@ -75,7 +75,7 @@ def test_random_bf16_gemm(seed):
     _run(W.Workload(g, ins), RTOL_BF16)
 
 
-@pytest.mark.parametrize("seed", range(40))
+@pytest.mark.parametrize("seed", range(120))
 def test_random_fp32_tall_skinny_gemm(seed):
     m = 512 + int(_u(seed, 1) * 4000)
     k = 4 * (1 + int(_u(seed, 2) * 59))
@@ -98,7 +98,7 @@ def test_random_fp32_tall_skinny_gemm(seed):
     _run(W.Workload(g, ins), RTOL_F32)
 
 
-@pytest.mark.parametrize("seed", range(40))
+@pytest.mark.parametrize("seed", range(100))
 def test_random_depthwise_and_pointwise_conv(seed):
     n = _pick(seed, 1, [1, 2, 5, 16, 40])
     h = 4 + int(_u(seed, 2) * 40)
