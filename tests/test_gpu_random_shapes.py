@@ -114,3 +114,34 @@ def test_random_depthwise_and_pointwise_conv(seed):
     y = g.add("Conv1x1", [e, "Wp"])
     g.mark_output(g.add("Add", [y, "u"], out="Y"))
     _run(W.Workload(g, ins), RTOL_F32)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_attention(seed):
+    """Q, K, V sliced out of one packed [B, S, 3*H*D] tensor, heads split by Reshape + Transpose, scores scaled and
+    masked, Softmax, P*V stored back to [B, S, H*D]: all index operators fold into operand strides of the two batched
+    GEMM blocks."""
+    import math
+    bsz = _pick(seed, 1, [1, 2, 3, 5])
+    s = _pick(seed, 2, [16, 32, 48, 100, 128, 200])
+    h = _pick(seed, 3, [1, 2, 3, 12])
+    d = _pick(seed, 4, [16, 32, 64, 128])
+    qkv = _bf(rnd((bsz, s, 3 * h * d), 5, -1, 1))
+    g = graph()
+    g.ext("QKV", qkv.shape, "bf16"); g.ext("mask", (s, s), "f32")
+    q, k, v = g.add("Split", ["QKV"], n_out=3, axis=-1, sizes=(h * d,) * 3)
+    hs = []
+    for t in (q, k, v):
+        t = g.add("Reshape", [t], shape=(bsz, s, h, d))
+        hs.append(g.add("Transpose", [t], perm=(0, 2, 1, 3)))
+    q, k, v = hs
+    kt = g.add("Transpose", [k], perm=(0, 1, 3, 2))
+    sc = g.add("MatMul", [q, kt])
+    sc = g.add("MulC", [sc], c=1.0 / math.sqrt(d))
+    sc = g.add("Add", [sc, "mask"])
+    p = g.add("Softmax", [sc], axis=-1)
+    a = g.add("MatMul", [p, v])
+    a = g.add("Transpose", [a], perm=(0, 2, 1, 3))
+    a = g.add("Reshape", [a], shape=(bsz, s, h * d), out="O")
+    g.mark_output(a)
+    _run(W.Workload(g, {"QKV": qkv, "mask": W.causal_mask(s)}), RTOL_BF16)
