@@ -124,6 +124,7 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, const void* 
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -378,9 +379,17 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
       for (int c = 0; c < chunks && ok; ++c, ++ccount) {
         const int buf = ccount & 1;
         io.chunk = cbuf + buf * kChunkBytes;
-        // the other buffer is free once the store issued from it two chunks ago has been read out
-        if (lane == 0) tma_store_wait_read();
+        // This chunk's buffer is free once the store issued from it two chunks ago has been read out: one store
+        // may stay in flight.  With a residual operand the OTHER buffer is about to be overwritten by the prefetch
+        // below, so the store issued from it one chunk ago has to be read out as well.
+#ifdef DNNF_TRACE
+        const long long tw0 = clock64();
+#endif
+        if (lane == 0) { if (q.c_input >= 0) tma_store_wait_read(); else tma_store_wait_read1(); }
         __syncwarp();
+#ifdef DNNF_TRACE
+        if (warp == 2 && lane == 0) T2ACC(9, clock64() - tw0);
+#endif
         {   // prefetch the next residual chunk (possibly of the next item) into the other buffer
           int nt = item, nc = c + 1;
           if (nc == chunks) { nt = item + n_pairs; nc = 0; }
@@ -413,8 +422,15 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
 #pragma unroll 1
         for (int h = 0; h < 2; ++h) {
           uint32_t raw[32];
+#ifdef DNNF_TRACE
+          const long long tl0 = clock64();
+#endif
           tc_ld32(t_row + c * 64 + h * 32, raw);
           tc_ld_wait();
+#ifdef DNNF_TRACE
+          const long long tl1 = clock64();
+          if (warp == 2 && lane == 0) T2ACC(6, tl1 - tl0);
+#endif
 #pragma unroll
           for (int i = 0; i < 32; ++i) io.accv[i] = __uint_as_float(raw[i]);
           if (others) {
@@ -428,13 +444,22 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
           io.col_in_chunk = h * 32;
           io.col_in_half = c * 64 + h * 32;
           run_program<32, SP, true>(p.prog, io);
+#ifdef DNNF_TRACE
+          if (warp == 2 && lane == 0) T2ACC(7, clock64() - tl1);
+#endif
         }
+#ifdef DNNF_TRACE
+        const long long ts0 = clock64();
+#endif
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
           tma_store_2d(&q.tmD, io.chunk, nw0 + c * 64, m0);
           tma_store_commit();
         }
+#ifdef DNNF_TRACE
+        if (warp == 2 && lane == 0) T2ACC(8, clock64() - ts0);
+#endif
       }
       tc_fence_before();
       __syncwarp();
