@@ -90,13 +90,31 @@ typedef enum {
   DNNF_OP_REDUCESUM, DNNF_OP_REDUCEMEAN, DNNF_OP_REDUCEMAX, DNNF_OP_REDUCEPROD, /* AXIS (last), KEEPDIMS */
   DNNF_OP_EXPAND,                                   /* attribute SHAPE */
   DNNF_OP_BITSHIFT,                                 /* attribute BITS; planning/rewriting only */
+  /* Table 2 operators that are index maps of an NHWC tensor [N,H,W,C].  dnnf_add_op records them in the ECG as the
+   * Reshape / Transpose / Expand operators they are made of, the way a Split becomes Slices, so that they fuse
+   * into their neighbours as changed load and store indices (Section 4.4.2):                                     */
+  DNNF_OP_DEPTHTOSPACE,                             /* Shuffle; attribute BLOCK b: y[n,h*b+i,w*b+j,c] = x[n,h,w,(i*b+j)*C/b^2+c] */
+  DNNF_OP_SPACETODEPTH,                             /* Shuffle; attribute BLOCK b: the inverse map */
+  DNNF_OP_RESIZE,                                   /* One-to-Many; nearest neighbour, integer attribute SCALE s:
+                                                       y[n,h,w,c] = x[n,h/s,w/s,c] */
+  DNNF_OP_CONCAT,                                   /* One-to-One (Table 2); 2 to 4 inputs, attribute AXIS.  Recorded as one
+                                                       ConcatPart per input: each writes its input's values into its
+                                                       range of the result, which all parts share in place, so that an
+                                                       input's producer block stores straight into the result (the
+                                                       Concat becomes changed store indices, Section 4.4.2) */
+  DNNF_OP_MAXPOOL, DNNF_OP_AVGPOOL,                 /* Many-to-Many (Table 2); NHWC fp32; attributes KERNEL k, STRIDE s, PAD p < k:
+                                                       result [N,(H+2p-k)/s+1,(W+2p-k)/s+1,C]; MaxPool ignores the padding,
+                                                       AveragePool divides by the number of elements inside the image;
+                                                       a global pool is KERNEL = H = W, STRIDE 1, PAD 0 */
+  DNNF_OP_CONCATPART,                               /* internal (made by Concat): (x [, result so far]); AXIS, START, SHAPE */
   DNNF_OP__COUNT
 } dnnf_op_t;
 
 typedef enum {
   DNNF_ATTR_C = 1, DNNF_ATTR_LO, DNNF_ATTR_HI, DNNF_ATTR_P, DNNF_ATTR_EPS,   /* use f */
   DNNF_ATTR_APPROX, DNNF_ATTR_AXIS, DNNF_ATTR_KEEPDIMS, DNNF_ATTR_START, DNNF_ATTR_END, DNNF_ATTR_BITS, /* use i[0] */
-  DNNF_ATTR_PERM, DNNF_ATTR_SHAPE, DNNF_ATTR_SIZES, DNNF_ATTR_AXES            /* use i[0..n) */
+  DNNF_ATTR_PERM, DNNF_ATTR_SHAPE, DNNF_ATTR_SIZES, DNNF_ATTR_AXES,           /* use i[0..n) */
+  DNNF_ATTR_BLOCK, DNNF_ATTR_SCALE, DNNF_ATTR_KERNEL, DNNF_ATTR_STRIDE, DNNF_ATTR_PAD   /* use i[0] */
 } dnnf_attr_key_t;
 
 typedef struct {
@@ -147,7 +165,8 @@ typedef enum {
   DNNF_FAMILY_ROW = 3,         /* chain around a last-axis reduction (Softmax, LayerNorm, Reduce*) */
   DNNF_FAMILY_GEMM = 4,        /* tensor-core GEMM anchor with an epilogue chain */
   DNNF_FAMILY_CONV1X1 = 5,     /* fp32 pointwise convolution with an epilogue chain */
-  DNNF_FAMILY_DWCONV = 6       /* fp32 depthwise 3x3 with an epilogue chain */
+  DNNF_FAMILY_DWCONV = 6,      /* fp32 depthwise 3x3 with an epilogue chain */
+  DNNF_FAMILY_POOL = 7         /* fp32 MaxPool / AveragePool with an epilogue chain */
 } dnnf_family_t;
 
 typedef struct {

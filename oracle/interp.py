@@ -140,6 +140,40 @@ def op_expand(x, shape):
     return np.ascontiguousarray(np.broadcast_to(x, tuple(int(s) for s in shape)))
 
 
+def op_depthtospace(x, block):
+    """NHWC, depth-column-row order: y[n, h*b+i, w*b+j, c] = x[n, h, w, (i*b+j)*C' + c] with C' = C / b^2
+    (Table 2 lists DepthToSpace under Shuffle)."""
+    b = int(block)
+    n, h, w, c = x.shape
+    cp = c // (b * b)
+    y = np.zeros((n, h * b, w * b, cp), dtype=np.float64)
+    for i in range(b):
+        for j in range(b):
+            y[:, i::b, j::b, :] = x[:, :, :, (i * b + j) * cp:(i * b + j + 1) * cp]
+    return y
+
+
+def op_spacetodepth(x, block):
+    """Inverse of op_depthtospace: y[n, h, w, (i*b+j)*C + c] = x[n, h*b+i, w*b+j, c]."""
+    b = int(block)
+    n, h, w, c = x.shape
+    y = np.zeros((n, h // b, w // b, b * b * c), dtype=np.float64)
+    for i in range(b):
+        for j in range(b):
+            y[:, :, :, (i * b + j) * c:(i * b + j + 1) * c] = x[:, i::b, j::b, :]
+    return y
+
+
+def op_resize_nearest(x, scale):
+    """NHWC nearest-neighbour enlargement by an integer factor: y[n, h, w, c] = x[n, h // s, w // s, c]
+    (Table 2 lists Resize / Upsample under One-to-Many)."""
+    s = int(scale)
+    n, h, w, c = x.shape
+    hi = np.arange(h * s) // s
+    wi = np.arange(w * s) // s
+    return x[:, hi][:, :, wi]
+
+
 def op_gather(x, indices, axis=0):
     return np.take(x, np.rint(indices).astype(np.int64), axis=_axis(axis, x.ndim))
 
@@ -167,6 +201,25 @@ def op_dwconv3x3(x, k):
         for dw in range(3):
             y += xp[:, dh:dh + h, dw:dw + w, :] * k[dh, dw, :]
     return y
+
+
+def _pool(x, kernel, stride, pad, is_max):
+    """NHWC pooling window by window: result[n, i, j, c] reduces x[n, i*s-p : i*s-p+k, j*s-p : j*s-p+k, c]
+    restricted to the image.  MaxPool takes the maximum of those elements, AveragePool their mean (elements of
+    the padding are neither compared nor counted).  Table 2 lists both under Many-to-Many."""
+    k, s, p = int(kernel), int(stride), int(pad)
+    n, h, w, c = x.shape
+    ho, wo = (h + 2 * p - k) // s + 1, (w + 2 * p - k) // s + 1
+    y = np.zeros((n, ho, wo, c), dtype=np.float64)
+    for i in range(ho):
+        for j in range(wo):
+            win = x[:, max(i * s - p, 0):min(i * s - p + k, h), max(j * s - p, 0):min(j * s - p + k, w), :]
+            y[:, i, j, :] = win.max(axis=(1, 2)) if is_max else win.mean(axis=(1, 2))
+    return y
+
+
+def op_maxpool(x, kernel, stride=1, pad=0): return _pool(x, kernel, stride, pad, True)
+def op_avgpool(x, kernel, stride=1, pad=0): return _pool(x, kernel, stride, pad, False)
 
 
 def op_softmax(x, axis=-1):
@@ -231,10 +284,15 @@ def _apply(op, ins, at):
     if op == "Concat": return [op_concat(ins, at["axis"])]
     if op == "Slice": return [op_slice(ins[0], at["axis"], at["start"], at["end"])]
     if op == "Expand": return [op_expand(ins[0], at["shape"])]
+    if op == "DepthToSpace": return [op_depthtospace(ins[0], at["block"])]
+    if op == "SpaceToDepth": return [op_spacetodepth(ins[0], at["block"])]
+    if op == "Resize": return [op_resize_nearest(ins[0], at["scale"])]
     if op == "Gather": return [op_gather(ins[0], ins[1], g("axis", 0))]
     if op == "MatMul": return [op_matmul(ins[0], ins[1])]
     if op == "Conv1x1": return [op_conv1x1(ins[0], ins[1])]
     if op == "DwConv3x3": return [op_dwconv3x3(ins[0], ins[1])]
+    if op == "MaxPool": return [op_maxpool(ins[0], at["kernel"], g("stride", 1), g("pad", 0))]
+    if op == "AveragePool": return [op_avgpool(ins[0], at["kernel"], g("stride", 1), g("pad", 0))]
     if op == "Softmax": return [op_softmax(ins[0], g("axis", -1))]
     if op == "LayerNorm": return [op_layernorm(ins[0], ins[1], ins[2], g("axis", -1), g("eps", 1e-5))]
     if op == "ReduceSum": return [op_reducesum(ins[0], g("axis", -1), g("keepdims", 1))]

@@ -79,6 +79,11 @@ static int parse_attrs(const dnnf_attr* a, int n, Attrs& at, std::string& err) {
       case DNNF_ATTR_SHAPE: at.shape = v; break;
       case DNNF_ATTR_SIZES: at.sizes = v; break;
       case DNNF_ATTR_AXES: at.axes = v; break;
+      case DNNF_ATTR_BLOCK: at.block = x.i[0]; break;
+      case DNNF_ATTR_SCALE: at.scale = x.i[0]; break;
+      case DNNF_ATTR_KERNEL: at.kernel = x.i[0]; break;
+      case DNNF_ATTR_STRIDE: at.stride = x.i[0]; break;
+      case DNNF_ATTR_PAD: at.pad = x.i[0]; break;
       default: err = "unknown attribute key"; return DNNF_ERR_INVALID_ARG;
     }
   }
@@ -121,6 +126,68 @@ int dnnf_add_op(dnnf_graph* g, int op_kind, int n_in, const int* in_ids, const d
       G.ops.push_back(o);
       start += s;
     }
+  } else if (op_kind == DNNF_OP_CONCATPART) {
+    return fail(g, DNNF_ERR_UNSUPPORTED_OP, "ConcatPart is made by Concat only");
+  } else if (op_kind == DNNF_OP_CONCAT) {
+    // One ConcatPart per input, chained through the result they fill in place.
+    if (n_in < 2) return fail(g, DNNF_ERR_INVALID_ARG, "Concat takes 2 to 4 inputs");
+    const Tensor& X0 = G.tensors[in_ids[0]];
+    int rank = (int)X0.dims.size();
+    int64_t ax = at.axis < 0 ? at.axis + rank : at.axis;
+    if (ax < 0 || ax >= rank) return fail(g, DNNF_ERR_SHAPE, "Concat: axis");
+    std::vector<int64_t> full = X0.dims;
+    full[ax] = 0;
+    for (int i = 0; i < n_in; ++i) {
+      const Tensor& Xi = G.tensors[in_ids[i]];
+      if ((int)Xi.dims.size() != rank || Xi.dtype != X0.dtype) return fail(g, DNNF_ERR_SHAPE, "Concat: inputs differ in rank or type");
+      full[ax] += Xi.dims[ax];
+    }
+    int64_t start = 0;
+    int carrier = -1;
+    for (int i = 0; i < n_in; ++i) {
+      Op o; o.id = (int)G.ops.size(); o.kind = DNNF_OP_CONCATPART; o.source_id = source;
+      o.in = {in_ids[i]};
+      if (carrier >= 0) o.in.push_back(carrier);
+      o.at.axis = ax; o.at.start = start; o.at.shape = full;
+      rc = infer_shapes(G, o, err);
+      if (rc) { rollback(); G.err = err; return rc; }
+      carrier = o.out[0];
+      start += G.tensors[in_ids[i]].dims[ax];
+      G.ops.push_back(o);
+    }
+    outs = {carrier};
+  } else if (op_kind == DNNF_OP_DEPTHTOSPACE || op_kind == DNNF_OP_SPACETODEPTH || op_kind == DNNF_OP_RESIZE) {
+    // Index maps of an NHWC tensor, recorded as the Reorganize / Shuffle / One-to-Many operators they consist of.
+    const Tensor& X = G.tensors[in_ids[0]];
+    if (X.dims.size() != 4) return fail(g, DNNF_ERR_SHAPE, "DepthToSpace / SpaceToDepth / Resize take an NHWC tensor");
+    const int64_t N = X.dims[0], H = X.dims[1], W = X.dims[2], Cc = X.dims[3];
+    const int64_t b = op_kind == DNNF_OP_RESIZE ? at.scale : at.block;
+    if (b < 1) return fail(g, DNNF_ERR_INVALID_ARG, "block size / scale must be a positive integer");
+    int cur = in_ids[0];
+    auto emit = [&](int kind, const Attrs& a) -> int {
+      Op o; o.id = (int)G.ops.size(); o.kind = kind; o.source_id = source; o.in = {cur}; o.at = a;
+      int r = infer_shapes(G, o, err);
+      if (r) return r;
+      cur = o.out[0];
+      G.ops.push_back(o);
+      return DNNF_OK;
+    };
+    Attrs a1, a2, a3;
+    int k2 = DNNF_OP_TRANSPOSE;
+    if (op_kind == DNNF_OP_DEPTHTOSPACE) {
+      if (Cc % (b * b)) return fail(g, DNNF_ERR_SHAPE, "DepthToSpace: channels are not a multiple of block^2");
+      a1.shape = {N, H, W, b, b, Cc / (b * b)}; a2.perm = {0, 1, 3, 2, 4, 5}; a3.shape = {N, H * b, W * b, Cc / (b * b)};
+    } else if (op_kind == DNNF_OP_SPACETODEPTH) {
+      if (H % b || W % b) return fail(g, DNNF_ERR_SHAPE, "SpaceToDepth: height or width is not a multiple of block");
+      a1.shape = {N, H / b, b, W / b, b, Cc}; a2.perm = {0, 1, 3, 2, 4, 5}; a3.shape = {N, H / b, W / b, b * b * Cc};
+    } else {
+      a1.shape = {N, H, 1, W, 1, Cc}; k2 = DNNF_OP_EXPAND; a2.shape = {N, H, b, W, b, Cc}; a3.shape = {N, H * b, W * b, Cc};
+    }
+    rc = emit(DNNF_OP_RESHAPE, a1);
+    if (!rc) rc = emit(k2, a2);
+    if (!rc) rc = emit(DNNF_OP_RESHAPE, a3);
+    if (rc) { rollback(); G.err = err; return rc; }
+    outs = {cur};
   } else {
     Op o; o.id = (int)G.ops.size(); o.kind = op_kind; o.source_id = source; o.in.assign(in_ids, in_ids + n_in); o.at = at;
     rc = infer_shapes(G, o, err);
@@ -206,7 +273,7 @@ int dnnf_block_info(const dnnf_graph* g, int bi, dnnf_block_desc* out) {
   out->n_inputs = (int)b.inputs.size();
   out->n_outputs = (int)b.outputs.size();
   for (int t : b.inputs) out->bytes_in += G.tensors[t].bytes();
-  for (int t : b.outputs) out->bytes_out += G.tensors[t].bytes();
+  for (int t : b.outputs) out->bytes_out += written_bytes(G, t);
   out->flops = b.launch.flops;
   { const Program* pr = program_of(b.launch); out->n_microops = pr ? pr->n : 0; }
   out->grid = b.launch.grid;

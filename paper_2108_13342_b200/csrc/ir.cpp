@@ -59,14 +59,14 @@ const char* op_name(int k) {
   static const char* names[] = {"?", "Add", "Sub", "Mul", "Div", "MulC", "AddC", "Sigmoid", "Tanh", "Erf", "Exp", "Log",
     "Sqrt", "Abs", "Neg", "Recip", "Square", "Relu", "Clip", "Pow", "Gelu", "ScaleShift", "Transpose", "Reshape",
     "Flatten", "Squeeze", "Unsqueeze", "Split", "Slice", "MatMul", "Conv1x1", "DwConv3x3", "Softmax", "LayerNorm",
-    "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift"};
+    "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift", "DepthToSpace", "SpaceToDepth", "Resize", "Concat", "MaxPool", "AveragePool", "ConcatPart"};
   if (k <= 0 || k >= DNNF_OP__COUNT) return "?";
   return names[k];
 }
 
 bool is_index_only(int k) {
   return k == DNNF_OP_TRANSPOSE || k == DNNF_OP_RESHAPE || k == DNNF_OP_FLATTEN || k == DNNF_OP_SQUEEZE ||
-         k == DNNF_OP_UNSQUEEZE || k == DNNF_OP_SLICE || k == DNNF_OP_SPLIT || k == DNNF_OP_EXPAND;
+         k == DNNF_OP_UNSQUEEZE || k == DNNF_OP_SLICE || k == DNNF_OP_SPLIT || k == DNNF_OP_EXPAND || k == DNNF_OP_CONCATPART;
 }
 bool is_elementwise(int k) {
   return (k >= DNNF_OP_ADD && k <= DNNF_OP_SCALESHIFT) || k == DNNF_OP_BITSHIFT;
@@ -74,7 +74,9 @@ bool is_elementwise(int k) {
 bool is_row_anchor(int k) {
   return k == DNNF_OP_SOFTMAX || k == DNNF_OP_LAYERNORM || (k >= DNNF_OP_REDUCESUM && k <= DNNF_OP_REDUCEPROD);
 }
-bool is_contraction(int k) { return k == DNNF_OP_MATMUL || k == DNNF_OP_CONV1X1 || k == DNNF_OP_DWCONV3X3; }
+bool is_contraction(int k) {      // anchors that take an epilogue chain and nothing in front
+  return k == DNNF_OP_MATMUL || k == DNNF_OP_CONV1X1 || k == DNNF_OP_DWCONV3X3 || k == DNNF_OP_MAXPOOL || k == DNNF_OP_AVGPOOL;
+}
 
 // Associative / commutative / distributive flags (Section 3.2).  Operators with
 // none of them are the partition points of the rewriting pass (Section 4.2).
@@ -122,10 +124,11 @@ int node_mapping(const Graph& g, const Op& op) {
     case DNNF_OP_SCALESHIFT: return DNNF_ONE_TO_ONE;     // BatchNormalization is listed One-to-One
     case DNNF_OP_TRANSPOSE: return DNNF_SHUFFLE;
     case DNNF_OP_RESHAPE: case DNNF_OP_FLATTEN: case DNNF_OP_SQUEEZE: case DNNF_OP_UNSQUEEZE: return DNNF_REORGANIZE;
-    case DNNF_OP_SPLIT: case DNNF_OP_SLICE: return DNNF_ONE_TO_ONE;
+    case DNNF_OP_SPLIT: case DNNF_OP_SLICE: case DNNF_OP_CONCAT: case DNNF_OP_CONCATPART: return DNNF_ONE_TO_ONE;
     case DNNF_OP_EXPAND: return DNNF_ONE_TO_MANY;
     case DNNF_OP_MATMUL: case DNNF_OP_CONV1X1: case DNNF_OP_DWCONV3X3: case DNNF_OP_SOFTMAX: case DNNF_OP_LAYERNORM:
     case DNNF_OP_REDUCESUM: case DNNF_OP_REDUCEMEAN: case DNNF_OP_REDUCEMAX: case DNNF_OP_REDUCEPROD:
+    case DNNF_OP_MAXPOOL: case DNNF_OP_AVGPOOL:
       return DNNF_MANY_TO_MANY;
     default: return DNNF_ONE_TO_ONE;
   }
@@ -263,6 +266,24 @@ int infer_shapes(Graph& g, Op& op, std::string& err) {
     op.at.axis = ax;
     auto d = in(0).dims; d[ax] = op.at.end - op.at.start;
     outs.push_back(d);
+  } else if (k == DNNF_OP_MAXPOOL || k == DNNF_OP_AVGPOOL) {
+    if (!need(1)) return DNNF_ERR_INVALID_ARG;
+    if (in(0).dims.size() != 4) { err = "pooling takes an NHWC tensor"; return DNNF_ERR_SHAPE; }
+    const int64_t kk = op.at.kernel, st = op.at.stride, pd = op.at.pad;
+    if (kk < 1 || st < 1 || pd < 0 || pd >= kk || kk > in(0).dims[1] + 2 * pd || kk > in(0).dims[2] + 2 * pd) { err = "pooling: kernel, stride or pad"; return DNNF_ERR_SHAPE; }
+    auto d = in(0).dims;
+    d[1] = (d[1] + 2 * pd - kk) / st + 1;
+    d[2] = (d[2] + 2 * pd - kk) / st + 1;
+    outs.push_back(d);
+  } else if (k == DNNF_OP_CONCATPART) {
+    if (op.in.size() != 1 && op.in.size() != 2) { err = "ConcatPart: operand count"; return DNNF_ERR_INVALID_ARG; }
+    int rank = (int)in(0).dims.size();
+    int ax = (int)op.at.axis;
+    if ((int)op.at.shape.size() != rank || ax < 0 || ax >= rank) { err = "Concat: rank or axis"; return DNNF_ERR_SHAPE; }
+    for (int d = 0; d < rank; ++d) if (d != ax && in(0).dims[d] != op.at.shape[d]) { err = "Concat: inputs differ off the axis"; return DNNF_ERR_SHAPE; }
+    if (op.at.start < 0 || op.at.start + in(0).dims[ax] > op.at.shape[ax]) { err = "Concat: range"; return DNNF_ERR_SHAPE; }
+    if (op.in.size() == 2 && (in(1).dims != op.at.shape || in(1).dtype != in(0).dtype)) { err = "Concat: inputs differ in type"; return DNNF_ERR_SHAPE; }
+    outs.push_back(op.at.shape);
   } else if (k == DNNF_OP_EXPAND) {
     if (!need(1)) return DNNF_ERR_INVALID_ARG;
     std::vector<int64_t> o;

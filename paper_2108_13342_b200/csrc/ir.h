@@ -14,7 +14,7 @@ namespace dnnf {
 
 struct Attrs {
   double c = 0, lo = 0, hi = 0, p = 0, eps = 1e-5;
-  int64_t approx = 0, axis = -1, keepdims = 1, start = 0, end = 0, bits = 0;
+  int64_t approx = 0, axis = -1, keepdims = 1, start = 0, end = 0, bits = 0, block = 0, scale = 0, kernel = 0, stride = 1, pad = 0;
   std::vector<int64_t> perm, shape, sizes, axes;
 };
 
@@ -117,6 +117,13 @@ bool is_elementwise(int kind);
 bool is_row_anchor(int kind);
 bool is_contraction(int kind);
 const char* op_name(int kind);
+// Bytes a block stores when tensor t is one of its outputs: the whole tensor, except for a Concat's part, which
+// fills only its own range of the shared result.
+inline int64_t written_bytes(const Graph& g, int t) {
+  const Tensor& T = g.tensors[t];
+  if (T.producer >= 0 && g.ops[T.producer].kind == DNNF_OP_CONCATPART) return g.tensors[g.ops[T.producer].in[0]].bytes();
+  return T.bytes();
+}
 int infer_shapes(Graph& g, Op& op, std::string& err);           // creates output tensors
 
 // ---- rewrite.cpp ----

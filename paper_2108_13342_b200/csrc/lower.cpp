@@ -154,6 +154,19 @@ bool backward_views(LowerCtx& cx, const Op& op, const View& vout, std::vector<Vi
     vin[0] = v;
     return true;
   }
+  if (k == DNNF_OP_CONCATPART) {
+    // the iteration space is the part's: the result's view starts inside the part's range of the axis
+    Aligned al;
+    if (!align_view(cx, vout, out.dims, al)) return false;
+    auto is = contiguous_strides(in(0).dims);
+    View v; v.coef.assign(cx.ext.size(), 0);
+    for (size_t d = 0; d < cx.ext.size(); ++d) if (al.tdim[d] >= 0) v.coef[d] = al.mult[d] * is[al.tdim[d]];
+    for (size_t j = 0; j < out.dims.size(); ++j) v.c0 += al.cst[j] * is[j];
+    v.c0 -= op.at.start * is[op.at.axis];
+    if (v.c0 < 0) { cx.why = "Concat: view outside the part"; return false; }
+    vin[0] = v;                         // the result so far (second operand) is extended in place, never read
+    return true;
+  }
   if (k == DNNF_OP_SOFTMAX) { vin[0] = vout; return true; }
   if (k >= DNNF_OP_REDUCESUM && k <= DNNF_OP_REDUCEPROD) {
     cx.why = "cannot derive a reduction's input from its output";
@@ -191,6 +204,17 @@ static int forward_view_i(LowerCtx& cx, const Op& op, int slot, const View& vi, 
     vo.coef.assign(cx.ext.size(), 0); vo.c0 = 0;
     for (size_t d = 0; d < cx.ext.size(); ++d) if (al.tdim[d] >= 0 && al.tdim[d] != last) vo.coef[d] = al.mult[d] * os[al.tdim[d]];
     for (int j = 0; j < last; ++j) vo.c0 += al.cst[j] * os[j];
+    return 1;
+  }
+  if (k == DNNF_OP_CONCATPART) {
+    if (slot != 0) { cx.why = "a Concat's result so far cannot be produced in the block that extends it"; return -1; }
+    Aligned al;
+    if (!align_view(cx, vi, in.dims, al)) return -1;
+    auto os = contiguous_strides(out.dims);
+    vo.coef.assign(cx.ext.size(), 0); vo.c0 = 0;
+    for (size_t d = 0; d < cx.ext.size(); ++d) if (al.tdim[d] >= 0) vo.coef[d] = al.mult[d] * os[al.tdim[d]];
+    for (size_t j = 0; j < in.dims.size(); ++j) vo.c0 += al.cst[j] * os[j];
+    vo.c0 += op.at.start * os[op.at.axis];
     return 1;
   }
   if (k == DNNF_OP_SLICE || k == DNNF_OP_EXPAND) { cx.why = "partial iteration space"; return -1; }
@@ -454,6 +478,7 @@ bool emit_program(LowerCtx& cx, int anchor_out, int max_tmp) {
     std::vector<Val> vals;
     for (size_t s = 0; s < op.in.size(); ++s) {
       int t = op.in[s];
+      if (op.kind == DNNF_OP_CONCATPART && s > 0) break;      // extended in place, not an operand of the kernel
       if (is_in_block_tensor(t)) {
         auto r = E.root_of.find(t);
         if (r == E.root_of.end()) { cx.why = "internal: operand before producer"; return false; }
@@ -489,7 +514,8 @@ bool emit_program(LowerCtx& cx, int anchor_out, int max_tmp) {
       {
         int64_t covered = 1;
         for (size_t d = 0; d < vit->second.coef.size() && d < cx.ext.size(); ++d) if (vit->second.coef[d] != 0) covered *= cx.ext[d];
-        if (covered != T.numel() || vit->second.c0 != 0) { cx.why = "a tensor that is read outside the block would be written only in part"; return false; }
+        const bool part = T.producer >= 0 && g.ops[T.producer].kind == DNNF_OP_CONCATPART;   // writes its own range only
+        if (part ? covered != g.tensors[g.ops[T.producer].in[0]].numel() : (covered != T.numel() || vit->second.c0 != 0)) { cx.why = "a tensor that is read outside the block would be written only in part"; return false; }
       }
       int oi = find_or_add_arg(cx.outs, t, vit->second);
       E.stores[E.root_of[t]].push_back(oi);
@@ -648,6 +674,7 @@ static int lower_elementwise_or_row(const Graph& g, const std::vector<int>& ops,
         if (outside) ref = t;              // the last one in topological order wins
       }
     }
+    for (int oid : ops) if (g.ops[oid].kind == DNNF_OP_CONCATPART) ref = g.ops[oid].in[0];   // the part, not the whole result
   }
   if (ref < 0) { why = "block has no output"; return DNNF_ERR_UNSUPPORTED_OP; }
   cx.ext = g.tensors[ref].dims;
@@ -743,6 +770,7 @@ static int lower_elementwise_or_row(const Graph& g, const std::vector<int>& ops,
   // A pure Reorganize block whose output walks its input in the same flat order is a zero-copy alias.
   if ((cx.prog.flags & kProgPureMove) && n_in == 1 && n_out == 1 && nd == 1 && ep.in[0].stride[0] == 1 && ep.out[0].stride[0] == 1 &&
       ep.in[0].base == 0 && ep.out[0].base == 0 && !g.tensors[cx.outs[0].tensor].is_output &&
+      g.tensors[cx.ins[0].tensor].numel() == g.tensors[cx.outs[0].tensor].numel() &&
       g.tensors[cx.ins[0].tensor].dtype == g.tensors[cx.outs[0].tensor].dtype) {
     L_.family = DNNF_FAMILY_ALIAS;
     out.lowered = true;
@@ -802,6 +830,18 @@ int lower_block(const Graph& g, const std::vector<int>& ops_in, uint32_t flags, 
     if (k == DNNF_OP_BITSHIFT) { why = "BitShift has no device code"; return DNNF_ERR_UNSUPPORTED_OP; }
   }
   if (n_anchor > 1) { why = "more than one Many-to-Many operator in a block"; return DNNF_ERR_UNSUPPORTED_OP; }
+  // A ConcatPart ends its block: it stores the block's values into its range of the Concat's result.  The
+  // operators that read the whole result, and the one that produced the result so far, run in other blocks.
+  {
+    int parts = 0;
+    for (int o : ops) {
+      const Op& P = g.ops[o];
+      if (P.kind != DNNF_OP_CONCATPART) continue;
+      if (++parts > 1) { why = "two parts of a Concat in one block"; return DNNF_ERR_UNSUPPORTED_OP; }
+      for (int c : g.tensors[P.out[0]].consumers) if (std::find(ops.begin(), ops.end(), c) != ops.end()) { why = "a Concat's result is complete only after its last part's block"; return DNNF_ERR_UNSUPPORTED_OP; }
+      if (P.in.size() > 1) { int pp = g.tensors[P.in[1]].producer; if (pp >= 0 && std::find(ops.begin(), ops.end(), pp) != ops.end()) { why = "two parts of a Concat in one block"; return DNNF_ERR_UNSUPPORTED_OP; } }
+    }
+  }
   // fused mapping type of the block: fold Table 3 along the topological order
   int m = g.ops[ops[0]].mapping;
   for (size_t i = 1; i < ops.size(); ++i) { int f, c; table3(m, g.ops[ops[i]].mapping, &f, &c); m = f; }

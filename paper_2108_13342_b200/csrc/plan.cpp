@@ -301,15 +301,15 @@ double block_cost_us(const Graph& g, const Block& b) {
   const Launch& L = b.launch;
   if (L.family == DNNF_FAMILY_ALIAS) return 0.0;
   double bytes = 0;
-  auto add = [&](int tensor, int mode) {
+  auto add = [&](int tensor, int mode, bool is_out = false) {
     const Tensor& T = g.tensors[tensor];
-    double e = (double)T.bytes();
-    if (mode == 2) e = (double)T.numel() * 32.0;
+    double e = (double)(is_out ? written_bytes(g, tensor) : T.bytes());
+    if (mode == 2) e = e / (T.dtype == DNNF_BF16 ? 2 : 4) * 32.0;
     bytes += e;
   };
   if (L.family == DNNF_FAMILY_ELEMENTWISE || L.family == DNNF_FAMILY_TRANSPOSE) {
     for (int i = 0; i < L.ew.n_in; ++i) add(L.in_tensors[i], L.ew.in[i].mode);
-    for (int i = 0; i < L.ew.n_out; ++i) add(L.out_tensors[i], L.ew.out[i].mode);
+    for (int i = 0; i < L.ew.n_out; ++i) add(L.out_tensors[i], L.ew.out[i].mode, true);
   } else if (L.family == DNNF_FAMILY_GEMM || L.family == DNNF_FAMILY_CONV1X1) {
     // operands: what the contraction reads (a strided view may cover part of a larger tensor)
     const GemmParams& gp = *reinterpret_cast<const GemmParams*>(L.blob.data());
@@ -320,7 +320,7 @@ double block_cost_us(const Graph& g, const Block& b) {
     for (int t : L.out_tensors) add(t, 0);
   } else {
     for (int t : b.inputs) add(t, 0);
-    for (int t : b.outputs) add(t, 0);
+    for (int t : b.outputs) add(t, 0, true);
   }
   double t_mem = bytes / 6.5e6;                       // us at 6.5 TB/s
   double t_cmp = (double)L.flops / 1.4e9;             // us at 1.4 PFLOP/s
@@ -418,6 +418,12 @@ int plan_graph(Graph& g, uint32_t flags) {
     g.tensors[b.launch.out_tensors[0]].alias_of = b.launch.in_tensors[0];
     irs_fused -= g.tensors[b.launch.out_tensors[0]].bytes();
   }
+  // A Concat's parts fill one result in place: the result so far shares storage with the extended one.
+  for (auto& o : g.ops) if (o.alive && o.kind == DNNF_OP_CONCATPART && o.in.size() > 1) {
+    g.tensors[o.in[1]].alias_of = o.out[0];
+    irs_fused -= g.tensors[o.in[1]].bytes();
+    irs_unfused -= g.tensors[o.in[1]].bytes();
+  }
   // Workspace: first-fit over live ranges in block order.
   struct Range { int64_t off, size; int last_use; };
   std::vector<Range> active;
@@ -428,13 +434,18 @@ int plan_graph(Graph& g, uint32_t flags) {
   g.ws_zero_bytes = (size_t)header;
   auto root = [&](int t) { while (g.tensors[t].alias_of >= 0) t = g.tensors[t].alias_of; return t; };
   std::vector<int> last_use(g.tensors.size(), -1);
-  for (size_t bi = 0; bi < g.blocks.size(); ++bi) for (int t : g.blocks[bi].inputs) last_use[root(t)] = (int)bi;
+  for (size_t bi = 0; bi < g.blocks.size(); ++bi) {
+    for (int t : g.blocks[bi].inputs) last_use[root(t)] = (int)bi;
+    for (int t : g.blocks[bi].outputs) last_use[root(t)] = std::max(last_use[root(t)], (int)bi);
+  }
   for (size_t bi = 0; bi < g.blocks.size(); ++bi) {
     Block& b = g.blocks[bi];
     if (!b.lowered || b.launch.family == DNNF_FAMILY_ALIAS) continue;
-    for (int t : b.outputs) {
+    for (int t0 : b.outputs) {
+      const int t = root(t0);             // a Concat's parts: the shared result, placed when its first part runs
       Tensor& T = g.tensors[t];
       if (T.is_output) continue;          // bound by the caller
+      if (T.ws_offset >= 0) continue;
       int64_t size = (T.bytes() + 255) / 256 * 256;
       // free ranges whose last use is before this block
       std::vector<Range> keep;

@@ -1,0 +1,138 @@
+// MaxPool / AveragePool over an NHWC fp32 tensor with a fused epilogue chain.
+//
+// Table 2 lists both under Many-to-Many; like the other Many-to-Many anchors they take One-to-One successors as
+// an epilogue (Table 3, Many-to-Many followed by One-to-One) and nothing in front.
+//
+// One thread owns four neighbouring channels of one output pixel and walks its window with 128-bit loads;
+// neighbouring lanes hold neighbouring channels, so every load of a warp is one run of bytes.  The window's rows
+// overlap between neighbouring outputs (stride < kernel) and are served by L1/L2; the kernel's HBM traffic is the
+// input once plus the output once.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <set>
+
+#include "conv_params.h"
+#include "launch_util.h"
+#include "lower.h"
+
+namespace dnnf {
+
+struct PoolParams {
+  DwParams d;              // N, H, W, C: the RESULT's dims; x: the pooled tensor; k unused; epilogue operands
+  int32_t Hi, Wi;          // pooled tensor's height and width
+  int32_t kernel, stride, pad;
+  int32_t is_max;
+  FastDiv fd_c4, fd_w, fd_h;
+};
+
+template <class SP>
+__global__ void __launch_bounds__(256) pool_kernel(const __grid_constant__ PoolParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const uint32_t C4 = (uint32_t)p.d.C / 4;
+  const uint32_t t = blockIdx.x * 256u + threadIdx.x;
+  const uint32_t total = (uint32_t)p.d.N * p.d.H * p.d.W * C4;
+  if (t >= total) return;
+  const uint32_t q0 = fd_div(t, p.fd_c4), c4 = t - q0 * C4;
+  const uint32_t q1 = fd_div(q0, p.fd_w), wo = q0 - q1 * (uint32_t)p.d.W;
+  const uint32_t n = fd_div(q1, p.fd_h), ho = q1 - n * (uint32_t)p.d.H;
+  const int h0 = (int)ho * p.stride - p.pad, w0 = (int)wo * p.stride - p.pad;
+  const int ha = max(h0, 0), hb = min(h0 + p.kernel, p.Hi);
+  const int wa = max(w0, 0), wb = min(w0 + p.kernel, p.Wi);
+  const float* xb = p.d.x + ((size_t)n * p.Hi * p.Wi) * p.d.C + c4 * 4;
+  DwIO io{p.d};
+  const float init = p.is_max ? -INFINITY : 0.0f;
+  io.accv[0] = io.accv[1] = io.accv[2] = io.accv[3] = init;
+  for (int h = ha; h < hb; ++h) {
+    const float* row = xb + ((size_t)h * p.Wi) * p.d.C;
+    for (int w = wa; w < wb; ++w) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(row + (size_t)w * p.d.C));
+      if (p.is_max) { io.accv[0] = fmaxf(io.accv[0], v.x); io.accv[1] = fmaxf(io.accv[1], v.y); io.accv[2] = fmaxf(io.accv[2], v.z); io.accv[3] = fmaxf(io.accv[3], v.w); }
+      else { io.accv[0] += v.x; io.accv[1] += v.y; io.accv[2] += v.z; io.accv[3] += v.w; }
+    }
+  }
+  if (!p.is_max) {                                  // mean over the elements inside the image (padding is not counted)
+    const float inv = 1.0f / (float)((hb - ha) * (wb - wa));
+#pragma unroll
+    for (int v = 0; v < 4; ++v) io.accv[v] *= inv;
+  }
+  io.n = n; io.h = ho; io.w = wo; io.c = c4 * 4;
+  run_program<4, SP>(p.d.prog, io);
+}
+
+static const PoolParams& pool_of(const Launch& L) { return *reinterpret_cast<const PoolParams*>(L.blob.data()); }
+
+struct PoolLauncher {
+  const Launch& L; cudaStream_t st;
+  template <class SP> void run() { launch_pdl(pool_kernel<SP>, L.grid, 256, 0, st, pool_of(L)); }
+};
+
+int pool_launch(const Launch& L, cudaStream_t st) {
+  PoolLauncher F{L, st};
+  if (!(L.static_id > 0 && StaticSet<ConvStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
+  return cudaGetLastError() == cudaSuccess ? 0 : 1;
+}
+
+void pool_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op) {
+  PoolParams& pp = *reinterpret_cast<PoolParams*>(L.blob.data());
+  pp.d.x = reinterpret_cast<const float*>(ip[0]);
+  for (int i = 0; i < pp.d.n_in; ++i) pp.d.in[i].ptr = ip[1 + i];
+  for (int i = 0; i < pp.d.n_out; ++i) pp.d.out[i].ptr = op[i];
+}
+
+int lower_pool(const Graph& g, const std::vector<int>& ops, int anchor, Block& out, std::string& why) {
+  const Op& A = g.ops[anchor];
+  const Tensor& X = g.tensors[A.in[0]];
+  const Tensor& Y = g.tensors[A.out[0]];
+  std::set<int> in_block(ops.begin(), ops.end());
+  if (X.dtype != DNNF_F32) { why = "pooling is fp32 only"; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (X.dims[3] % 4) { why = "pooling needs a channel count that is a multiple of 4"; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (in_block.count(X.producer)) { why = "operators in front of a pooling anchor (no prologue fusion)"; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (X.numel() >= (1ll << 31) || Y.numel() >= (1ll << 31)) { why = "tensor too large"; return DNNF_ERR_UNSUPPORTED_OP; }
+  LowerCtx cx(g);
+  cx.ops = ops; cx.in_block = in_block;
+  cx.ext = Y.dims;
+  if (!derive_views(cx, A.out[0], {anchor})) { why = cx.why; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (cx.ext != Y.dims) { why = "epilogue reshapes a pooling result"; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (!emit_program(cx, A.out[0], 2)) { why = cx.why; return DNNF_ERR_UNSUPPORTED_OP; }
+  Launch& L = out.launch;
+  L = Launch{};
+  L.blob.assign(sizeof(PoolParams), 0);
+  PoolParams& pp = *reinterpret_cast<PoolParams*>(L.blob.data());
+  DwParams& dp = pp.d;
+  dp.N = (int)Y.dims[0]; dp.H = (int)Y.dims[1]; dp.W = (int)Y.dims[2]; dp.C = (int)Y.dims[3];
+  pp.Hi = (int)X.dims[1]; pp.Wi = (int)X.dims[2];
+  pp.kernel = (int)A.at.kernel; pp.stride = (int)A.at.stride; pp.pad = (int)A.at.pad;
+  pp.is_max = A.kind == DNNF_OP_MAXPOOL;
+  pp.fd_c4 = make_fastdiv((uint32_t)dp.C / 4); pp.fd_w = make_fastdiv((uint32_t)dp.W); pp.fd_h = make_fastdiv((uint32_t)dp.H);
+  dp.n_in = (int)cx.ins.size(); dp.n_out = (int)cx.outs.size();
+  auto fill = [&](TensorArg& a, const ExtArg& e, bool is_out) {
+    a.ptr = nullptr; a.base = (int32_t)e.view.c0; a.dtype = g.tensors[e.tensor].dtype; a.mode = 0;
+    for (int d = 0; d < kMaxDims; ++d) a.stride[d] = d < 4 ? (int32_t)e.view.coef[3 - d] : 0;
+    if (a.dtype != DNNF_F32) return false;
+    if (a.stride[0] == 1) { if (a.base % 4) return false; for (int d = 1; d < 4; ++d) if (a.stride[d] % 4) return false; }
+    else if (!(a.stride[0] == 0 && !is_out)) return false;
+    return true;
+  };
+  for (size_t i = 0; i < cx.ins.size(); ++i) if (!fill(dp.in[i], cx.ins[i], false)) { why = "pooling epilogue operand is not fp32 / channel-contiguous"; return DNNF_ERR_UNSUPPORTED_OP; }
+  for (size_t i = 0; i < cx.outs.size(); ++i) if (!fill(dp.out[i], cx.outs[i], true)) { why = "pooling epilogue output is not fp32 / channel-contiguous"; return DNNF_ERR_UNSUPPORTED_OP; }
+  dp.prog = cx.prog;
+  L.ew.prog = cx.prog;
+  L.in_tensors = {A.in[0]};
+  out.inputs = {A.in[0]};
+  out.outputs.clear();
+  for (auto& a : cx.ins) { L.in_tensors.push_back(a.tensor); if (std::find(out.inputs.begin(), out.inputs.end(), a.tensor) == out.inputs.end()) out.inputs.push_back(a.tensor); }
+  for (auto& a : cx.outs) { L.out_tensors.push_back(a.tensor); out.outputs.push_back(a.tensor); }
+  L.family = DNNF_FAMILY_POOL;
+  L.flops = (int64_t)Y.numel() * pp.kernel * pp.kernel;
+  const int64_t total = Y.numel() / 4;
+  L.grid = (int)((total + 255) / 256);
+  L.threads = 256;
+  L.variant = pp.is_max;
+  L.static_id = StaticSet<ConvStatic>::find(dp.prog);
+  out.lowered = true;
+  return DNNF_OK;
+}
+
+}  // namespace dnnf

@@ -284,6 +284,52 @@ def mbconv_block(n=32, h=56, w=56, cin=24, cexp=144, seed=BASE_SEED) -> Workload
     return Workload(g, inputs)
 
 
+def cnn_neck(n=8, h=64, w=64, c=32, seed=BASE_SEED) -> Workload:
+    """A detection-style feature-pyramid fragment in NHWC fp32 that uses the rest of Table 2's operator set
+    around the convolution blocks: a pointwise stem, MaxPool and SpaceToDepth downsampling, nearest-neighbour
+    Resize and DepthToSpace upsampling, channel Concat with skip connections, a global AveragePool gate.
+    Synthetic shapes in the range of the paper's mobile CNNs (Section 5: 224-416 pixel inputs, stride 4-8 maps)."""
+    d = _Draw(seed + 9)
+    g = GraphDesc("cnn_neck")
+    ins = {}
+
+    def ext(name, shape, lo=None, hi=None, std=None):
+        g.ext(name, shape, kind="input" if name == "X" else "weight")
+        ins[name] = d.normal(shape, 0.0, std) if std is not None else d.uniform(shape, lo, hi)
+        return name
+
+    def conv_bn_relu6(x, cin, cout, tag):
+        wn = ext("W" + tag, (cin, cout), std=math.sqrt(2.0 / cin))
+        sn = ext("s" + tag, (cout,), 0.5, 1.5); tn = ext("t" + tag, (cout,), -0.5, 0.5)
+        e = g.add("Conv1x1", [x, wn])
+        e = g.add("ScaleShift", [e, sn, tn], axis=-1)
+        return g.add("Clip", [e], lo=0.0, hi=6.0)
+
+    ext("X", (n, h, w, c), 0.0, 1.0)
+    stem = conv_bn_relu6("X", c, 2 * c, "0")                              # [n, h, w, 2c]
+    p1 = g.add("MaxPool", [stem], kernel=3, stride=2, pad=1)              # [n, h/2, w/2, 2c]
+    s2d = g.add("SpaceToDepth", [stem], block=2)                          # [n, h/2, w/2, 8c]
+    lat = conv_bn_relu6(s2d, 8 * c, 2 * c, "1")                           # [n, h/2, w/2, 2c]
+    mid = g.add("Concat", [p1, lat], axis=3)                              # [n, h/2, w/2, 4c]
+    kd = ext("Kd", (3, 3, 4 * c), std=math.sqrt(2.0 / 9.0))
+    sd = ext("sd", (4 * c,), 0.5, 1.5); td = ext("td", (4 * c,), -0.5, 0.5)
+    dw = g.add("DwConv3x3", [mid, kd])
+    dw = g.add("ScaleShift", [dw, sd, td], axis=-1)
+    dw = g.add("Clip", [dw], lo=0.0, hi=6.0)                              # [n, h/2, w/2, 4c]
+    # squeeze-and-excitation style gate from a global average pool
+    gap = g.add("AveragePool", [dw], kernel=h // 2, stride=1, pad=0)      # [n, 1, 1, 4c]
+    wg = ext("Wg", (4 * c, 4 * c), std=math.sqrt(1.0 / (4 * c)))
+    gate = g.add("Sigmoid", [g.add("Conv1x1", [gap, wg])])                # [n, 1, 1, 4c]
+    gated = g.add("Mul", [dw, gate])                                      # broadcast over the image
+    up_a = g.add("DepthToSpace", [gated], block=2)                        # [n, h, w, c]
+    up_b = g.add("Resize", [conv_bn_relu6(gated, 4 * c, c, "2")], scale=2)   # [n, h, w, c]
+    top = g.add("Concat", [up_a, up_b, "X"], axis=3)                      # [n, h, w, 3c]
+    y = conv_bn_relu6(top, 3 * c, c, "3")
+    y = g.add("Add", [y, "X"], out="Y")
+    g.mark_output(y)
+    return Workload(g, ins, note="fp32 NHWC")
+
+
 # --------------------------------------------------------------------------
 # Workload 5: transformer encoder as primitive operators (48 per layer)
 # --------------------------------------------------------------------------
@@ -450,5 +496,5 @@ def decoder(layers=12, batch=8, seq=128, hidden=768, heads=12, ffn=3072, seed=BA
 def by_name(name: str, **kw) -> Workload:
     table = {"swish_transpose": swish_transpose, "masked_softmax": masked_softmax,
              "add_layernorm_gelu": add_layernorm_gelu, "ffn_block": ffn_block,
-             "mbconv_block": mbconv_block, "encoder": encoder, "decoder": decoder}
+             "mbconv_block": mbconv_block, "encoder": encoder, "decoder": decoder, "cnn_neck": cnn_neck}
     return table[name](**kw)

@@ -133,6 +133,8 @@ def _build(seed, big=False, dtype="f32"):
                 continue
             o = g.add("LayerNorm", [t, vec(shp[-1], 0.8, 1.2), vec(shp[-1], -0.2, 0.2)], axis=-1, eps=1e-5)
         else:
+            if len(shp) < 2:
+                continue                                # MatMul takes a matrix on the left
             n = r.pick([8, 16, 24])
             o = g.add("MatMul", [t, mat(shp[-1], n)])
             shp = shp[:-1] + (n,)

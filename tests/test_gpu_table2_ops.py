@@ -1,0 +1,171 @@
+"""Parity of the remaining Table 2 operators against the oracle: DepthToSpace / SpaceToDepth (Shuffle), Resize
+(One-to-Many), Concat (One-to-One, as changed store indices of its inputs' producer blocks, Section 4.4.2),
+MaxPool / AveragePool (Many-to-Many anchors with an epilogue), alone and fused with their neighbours, and a
+CNN fragment that uses all of them."""
+import numpy as np
+import pytest
+
+from paper_2108_13342_b200 import binding as B
+from paper_2108_13342_b200 import workloads as W
+from util import RTOL_F32, check, graph, rnd, run_both, close
+
+pytestmark = pytest.mark.gpu
+
+PLANS = [B.PLAN_FUSED, B.PLAN_UNFUSED]
+
+
+def _exact(wl, flags):
+    s, got, ref = run_both(wl, flags)
+    for n in wl.graph.outputs:
+        assert np.array_equal(got[n].astype(np.float64), ref[n]), (n, s.g.blocks())
+    return s
+
+
+@pytest.mark.parametrize("flags", PLANS)
+@pytest.mark.parametrize("shape,b", [((2, 8, 8, 16), 2), ((1, 5, 7, 36), 3), ((3, 4, 6, 8), 2), ((2, 9, 3, 64), 4)])
+def test_depthtospace_and_back_are_exact_moves(shape, b, flags):
+    g = graph("d2s")
+    g.ext("X", shape)
+    y = g.add("DepthToSpace", ["X"], block=b)
+    z = g.add("SpaceToDepth", [y], block=b)
+    g.mark_output(y); g.mark_output(z)
+    _exact(W.Workload(g, {"X": rnd(shape, 1)}), flags)
+
+
+@pytest.mark.parametrize("flags", PLANS)
+@pytest.mark.parametrize("shape,b", [((2, 8, 8, 16), 2), ((1, 6, 9, 18), 3)])
+def test_shuffle_ops_inside_a_chain(shape, b, flags):
+    n, h, w, c = shape
+    g = graph("d2s_chain")
+    g.ext("X", shape); g.ext("Y", (n, h * b, w * b, c // (b * b))); g.ext("v", (c // (b * b),))
+    t = g.add("Relu", ["X"])
+    t = g.add("DepthToSpace", [t], block=b)
+    t = g.add("Add", [g.add("Mul", [t, "v"]), "Y"])
+    u = g.add("Sigmoid", [g.add("SpaceToDepth", [t], block=b)])
+    g.mark_output(t); g.mark_output(u)
+    wl = W.Workload(g, {"X": rnd(shape, 2), "Y": rnd((n, h * b, w * b, c // (b * b)), 3), "v": rnd((c // (b * b),), 4, 0.5, 1.5)})
+    check(wl, RTOL_F32, flags)
+
+
+@pytest.mark.parametrize("flags", PLANS)
+def test_spacetodepth_in_front_of_a_pointwise_convolution(flags):
+    g = graph("s2d_conv")
+    g.ext("X", (2, 12, 12, 8)); g.ext("Wt", (32, 24), kind="weight")
+    t = g.add("Conv1x1", [g.add("SpaceToDepth", ["X"], block=2), "Wt"])
+    g.mark_output(g.add("Relu", [t]))
+    check(W.Workload(g, {"X": rnd((2, 12, 12, 8), 5), "Wt": rnd((32, 24), 6, -0.3, 0.3)}), RTOL_F32, flags)
+
+
+@pytest.mark.parametrize("flags", PLANS)
+@pytest.mark.parametrize("shape,s", [((2, 8, 8, 16), 2), ((1, 5, 7, 6), 3), ((2, 3, 4, 5), 2)])
+def test_resize_nearest(shape, s, flags):
+    n, h, w, c = shape
+    g = graph("up")
+    g.ext("X", shape); g.ext("Y", (n, h * s, w * s, c))
+    r = g.add("Resize", ["X"], scale=s)
+    t = g.add("Add", [g.add("Resize", [g.add("Tanh", ["X"])], scale=s), "Y"])
+    g.mark_output(r); g.mark_output(t)
+    sess, got, ref = run_both(W.Workload(g, {"X": rnd(shape, 7), "Y": rnd((n, h * s, w * s, c), 8)}), flags)
+    names = list(g.outputs)
+    assert np.array_equal(got[names[0]].astype(np.float64), ref[names[0]])
+    close(got[names[1]], ref[names[1]], RTOL_F32)
+
+
+@pytest.mark.parametrize("flags", PLANS)
+@pytest.mark.parametrize("axis,shapes", [
+    (3, [(2, 8, 8, 16), (2, 8, 8, 24), (2, 8, 8, 8)]),
+    (3, [(1, 5, 3, 5), (1, 5, 3, 7)]),                       # ragged channel counts: unaligned bases
+    (0, [(2, 4, 4, 8), (3, 4, 4, 8), (1, 4, 4, 8), (2, 4, 4, 8)]),
+    (1, [(2, 3, 5, 4), (2, 6, 5, 4)]),
+    (-1, [(7, 33), (7, 31)]),
+])
+def test_concat_of_external_and_produced_tensors(axis, shapes, flags):
+    g = graph("cat")
+    ins = {}
+    parts = []
+    for i, shp in enumerate(shapes):
+        g.ext(f"X{i}", shp); ins[f"X{i}"] = rnd(shp, 10 + i)
+        parts.append(f"X{i}" if i % 2 else g.add("Tanh", [f"X{i}"]))
+    c = g.add("Concat", parts, axis=axis)
+    g.mark_output(c)
+    g.mark_output(g.add("Sigmoid", [c]))
+    s = check(W.Workload(g, ins), RTOL_F32, flags)
+    if flags == B.PLAN_FUSED and all(shp[-1] % 4 == 0 for shp in shapes):
+        # each producer stores straight into the result: no kernel for the Concat itself (with ragged channel counts
+        # the stores would be scalar and the cost model may prefer a separate copy)
+        fams = [b["ops"] for b in s.g.blocks()]
+        assert ["Tanh", "ConcatPart"] in fams, fams
+
+
+@pytest.mark.parametrize("flags", PLANS)
+def test_concat_is_exact_and_nests(flags):
+    g = graph("cat_exact")
+    g.ext("A", (3, 4, 8)); g.ext("Bt", (3, 2, 8)); g.ext("Ct", (3, 6, 5))
+    ab = g.add("Concat", ["A", "Bt"], axis=1)                # [3, 6, 8]
+    abc = g.add("Concat", [ab, "Ct", ab], axis=2)            # [3, 6, 21]: a Concat's result as a part, twice
+    g.mark_output(abc)
+    _exact(W.Workload(g, {"A": rnd((3, 4, 8), 20), "Bt": rnd((3, 2, 8), 21), "Ct": rnd((3, 6, 5), 22)}), flags)
+
+
+@pytest.mark.parametrize("flags", PLANS)
+def test_concat_fed_by_row_and_convolution_blocks(flags):
+    g = graph("cat_blocks")
+    g.ext("X", (2, 10, 10, 16)); g.ext("W1", (16, 24), kind="weight"); g.ext("s", (24,)); g.ext("t", (24,))
+    g.ext("Kd", (3, 3, 16), kind="weight"); g.ext("ga", (16,)); g.ext("be", (16,))
+    a = g.add("Clip", [g.add("ScaleShift", [g.add("Conv1x1", ["X", "W1"]), "s", "t"], axis=-1)], lo=0.0, hi=6.0)
+    b = g.add("Relu", [g.add("DwConv3x3", ["X", "Kd"])])
+    c = g.add("LayerNorm", ["X", "ga", "be"], axis=-1, eps=1e-5)
+    d = g.add("MaxPool", ["X"], kernel=3, stride=1, pad=1)
+    y = g.add("Concat", [a, b, c, d], axis=3)                 # [2, 10, 10, 72]
+    g.mark_output(g.add("MulC", [y], c=0.5))
+    ins = {"X": rnd((2, 10, 10, 16), 30), "W1": rnd((16, 24), 31, -0.3, 0.3), "s": rnd((24,), 32, 0.5, 1.5),
+           "t": rnd((24,), 33, -0.5, 0.5), "Kd": rnd((3, 3, 16), 34, -0.5, 0.5), "ga": rnd((16,), 35, 0.8, 1.2),
+           "be": rnd((16,), 36, -0.2, 0.2)}
+    s = check(W.Workload(g, ins), 2e-4, flags)                # the convolution part runs as split TF32 when eligible
+    if flags == B.PLAN_FUSED:
+        assert s.plan_stats.n_kernels == 5, s.g.blocks()      # four producers (each ends in its part) + the consumer
+
+
+@pytest.mark.parametrize("flags", PLANS)
+def test_concat_bf16(flags):
+    g = graph("cat_bf16")
+    g.ext("X", (4, 64, 32), "bf16"); g.ext("Y", (4, 64, 16), "bf16")
+    c = g.add("Concat", [g.add("Relu", ["X"]), "Y"], axis=2)
+    g.mark_output(c)
+    ins = {"X": W.round_to_bf16(rnd((4, 64, 32), 40)), "Y": W.round_to_bf16(rnd((4, 64, 16), 41))}
+    _exact(W.Workload(g, ins), flags)
+
+
+@pytest.mark.parametrize("flags", PLANS)
+@pytest.mark.parametrize("kind", ["MaxPool", "AveragePool"])
+@pytest.mark.parametrize("shape,k,s,p", [((2, 16, 16, 8), 2, 2, 0), ((1, 15, 13, 12), 3, 2, 1), ((3, 7, 9, 4), 3, 1, 1),
+                                         ((2, 8, 8, 32), 8, 1, 0), ((1, 11, 11, 20), 5, 3, 2), ((2, 6, 10, 8), 2, 1, 0)])
+def test_pooling_with_epilogue(kind, shape, k, s, p, flags):
+    c = shape[3]
+    g = graph("pool")
+    g.ext("X", shape); g.ext("sc", (c,)); g.ext("sh", (c,))
+    y = g.add(kind, ["X"], kernel=k, stride=s, pad=p)
+    z = g.add("Relu", [g.add("ScaleShift", [y, "sc", "sh"], axis=-1)])
+    g.mark_output(y); g.mark_output(z)
+    sess = check(W.Workload(g, {"X": rnd(shape, 50), "sc": rnd((c,), 51, 0.5, 1.5), "sh": rnd((c,), 52, -0.5, 0.5)}),
+                 RTOL_F32, flags)
+    if flags == B.PLAN_FUSED:
+        assert sess.plan_stats.n_kernels == 1, sess.g.blocks()
+
+
+def test_maxpool_is_exact():
+    g = graph("maxpool_exact")
+    g.ext("X", (2, 17, 19, 8))
+    g.mark_output(g.add("MaxPool", ["X"], kernel=3, stride=2, pad=1))
+    _exact(W.Workload(g, {"X": rnd((2, 17, 19, 8), 53)}), B.PLAN_FUSED)
+
+
+@pytest.mark.parametrize("flags,rewrite", [(B.PLAN_FUSED, B.REWRITE_DEFAULT), (B.PLAN_FUSED, B.REWRITE_NONE), (B.PLAN_UNFUSED, B.REWRITE_NONE)])
+@pytest.mark.parametrize("dims", [(2, 16, 16, 8), (1, 24, 40, 16), (3, 64, 64, 32)])
+def test_cnn_fragment(dims, flags, rewrite):
+    wl = W.cnn_neck(*dims) if dims[1] == dims[2] else None
+    if wl is None:      # the global pool of the fragment takes a square map: use the nearest square
+        wl = W.cnn_neck(dims[0], dims[1], dims[1], dims[3])
+    s = check(wl, 5e-4, flags, rewrite)          # several split-TF32 convolutions in sequence
+    if flags == B.PLAN_FUSED:
+        assert s.plan_stats.n_kernels < s.plan_stats.n_ops

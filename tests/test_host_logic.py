@@ -404,3 +404,90 @@ def test_yellow_decision_follows_the_profiling_database():
     assert st3.n_kernels == 1 and st3.n_yellow_fused >= 1
     assert g3.block_signature(0) == fused[0]
     B.profile_db_clear()
+
+
+# ---- the rest of Table 2: index operators recorded as their parts, Concat as in-place parts, pooling -------------
+
+def _desc():
+    from paper_2108_13342_b200.workloads import GraphDesc
+    return GraphDesc("t")
+
+
+def _plan_desc(desc, flags=B.PLAN_FUSED):
+    from paper_2108_13342_b200.runtime import build_graph
+    G, ids = build_graph(desc)
+    G.rewrite(B.REWRITE_NONE)
+    st = G.plan(flags)
+    return G, ids, st
+
+
+def test_shuffle_and_resize_operators_are_recorded_as_index_operators():
+    g = _desc(); g.ext("X", (2, 8, 8, 16))
+    g.mark_output(g.add("Sigmoid", [g.add("DepthToSpace", [g.add("Relu", ["X"])], block=2)]))
+    G, ids, st = _plan_desc(g)
+    assert st.n_ops == 3 and st.n_kernels == 1
+    assert G.blocks()[0]["ops"] == ["Relu", "Reshape", "Transpose", "Reshape", "Sigmoid"]
+    assert G.tensor_info(ids[g.outputs[0]])[1] == (2, 16, 16, 4)
+    g = _desc(); g.ext("X", (2, 8, 8, 16))
+    g.mark_output(g.add("Resize", ["X"], scale=3))
+    G, ids, st = _plan_desc(g)
+    assert G.blocks()[0]["ops"] == ["Reshape", "Expand", "Reshape"] and G.blocks()[0]["mapping"] == "One-to-Many"
+    assert G.tensor_info(ids[g.outputs[0]])[1] == (2, 24, 24, 16)
+    g = _desc(); g.ext("X", (2, 8, 6, 4))
+    g.mark_output(g.add("SpaceToDepth", ["X"], block=2))
+    G, ids, st = _plan_desc(g)
+    assert G.tensor_info(ids[g.outputs[0]])[1] == (2, 4, 3, 16)
+    for bad in [dict(op="DepthToSpace", block=3), dict(op="SpaceToDepth", block=4), dict(op="Resize", scale=0)]:
+        g = _desc(); g.ext("X", (2, 8, 6, 4))
+        op = bad.pop("op")
+        g.add(op, ["X"], **bad)
+        with pytest.raises(B.DnnfError):
+            _plan_desc(g)
+
+
+def test_concat_parts_fuse_into_their_producers_and_share_the_result():
+    g = _desc(); g.ext("X", (2, 8, 8, 16)); g.ext("Y", (2, 8, 8, 24)); g.ext("Z", (2, 8, 8, 8))
+    c = g.add("Concat", [g.add("Relu", ["X"]), g.add("Sigmoid", ["Y"]), "Z"], axis=3)
+    g.mark_output(g.add("Tanh", [c]))
+    G, ids, st = _plan_desc(g)
+    ops = [b["ops"] for b in G.blocks()]
+    assert ops == [["Relu", "ConcatPart"], ["Sigmoid", "ConcatPart"], ["ConcatPart"], ["Tanh"]]
+    assert st.n_ops == 4                                   # the three parts count as the one Concat they came from
+    assert all(b["mapping"] == "One-to-One" for b in G.blocks())
+    full = 2 * 8 * 8 * 48 * 4
+    assert st.workspace_bytes - G.workspace_zero_bytes() == full          # one buffer for the result, none per part
+    assert st.irs_bytes_fused == full
+    assert [b["bytes"] for b in G.blocks()[:3]] == [2 * 2 * 8 * 8 * n * 4 for n in (16, 24, 8)]   # a part writes its range only
+    # unfused: one copy kernel per part, still one shared result
+    G, ids, st = _plan_desc(g, B.PLAN_UNFUSED)
+    assert [b["ops"] for b in G.blocks()].count(["ConcatPart"]) == 3
+    for bad_axis, shapes in [(3, [(2, 8, 8, 16), (2, 8, 7, 16)]), (5, [(2, 8), (2, 8)]), (0, [(2, 8), (2, 8, 1)])]:
+        g = _desc()
+        for i, shp in enumerate(shapes):
+            g.ext(f"X{i}", shp)
+        g.add("Concat", [f"X{i}" for i in range(len(shapes))], axis=bad_axis)
+        with pytest.raises(B.DnnfError):
+            _plan_desc(g)
+    g = _desc(); g.ext("X", (2, 8))
+    g.add("ConcatPart", ["X"], axis=0, start=0, shape=(4, 8))
+    with pytest.raises(B.DnnfError):
+        _plan_desc(g)
+
+
+def test_pooling_shapes_types_and_epilogue_fusion():
+    g = _desc(); g.ext("X", (2, 15, 13, 12)); g.ext("s", (12,)); g.ext("t", (12,))
+    y = g.add("MaxPool", ["X"], kernel=3, stride=2, pad=1)
+    g.mark_output(g.add("Relu", [g.add("ScaleShift", [y, "s", "t"], axis=-1)]))
+    G, ids, st = _plan_desc(g)
+    assert G.tensor_info(ids[g.outputs[0]])[1] == (2, 8, 7, 12)
+    assert st.n_kernels == 1 and G.blocks()[0]["family"] == "pool" and G.blocks()[0]["mapping"] == "Many-to-Many"
+    # Many-to-Many followed by Many-to-Many is a red cell: two pools never share a block
+    g = _desc(); g.ext("X", (2, 16, 16, 8))
+    g.mark_output(g.add("AveragePool", [g.add("MaxPool", ["X"], kernel=2, stride=2, pad=0)], kernel=8, stride=1, pad=0))
+    G, ids, st = _plan_desc(g)
+    assert st.n_kernels == 2 and G.tensor_info(ids[g.outputs[0]])[1] == (2, 1, 1, 8)
+    for at in [dict(kernel=0), dict(kernel=3, pad=3), dict(kernel=3, stride=0), dict(kernel=40)]:
+        g = _desc(); g.ext("X", (2, 16, 16, 8))
+        g.add("MaxPool", ["X"], **at)
+        with pytest.raises(B.DnnfError):
+            _plan_desc(g)

@@ -165,7 +165,52 @@ def test_gather():
     assert np.array_equal(y, np.stack([x[4], x[0], x[4]]))
 
 
+def test_depthtospace_spacetodepth_resize_index_loops():
+    """Each element against the index formula of the operator's definition, in pure-Python loops; the two Shuffle
+    operators undo each other; nearest-neighbour enlargement equals numpy's repeat along both image axes."""
+    b = 2
+    x = rnd((2, 3, 2, 12), 21)
+    y = O.op_depthtospace(x, b)
+    assert y.shape == (2, 6, 4, 3)
+    for n, h, w, i, j, c in itertools.product(range(2), range(3), range(2), range(b), range(b), range(3)):
+        assert y[n, h * b + i, w * b + j, c] == x[n, h, w, (i * b + j) * 3 + c]
+    assert np.array_equal(O.op_spacetodepth(y, b), x)
+    z = rnd((1, 6, 9, 2), 22)
+    s2d = O.op_spacetodepth(z, 3)
+    assert s2d.shape == (1, 2, 3, 18)
+    for h, w, i, j, c in itertools.product(range(2), range(3), range(3), range(3), range(2)):
+        assert s2d[0, h, w, (i * 3 + j) * 2 + c] == z[0, h * 3 + i, w * 3 + j, c]
+    assert np.array_equal(O.op_depthtospace(s2d, 3), z)
+    r = O.op_resize_nearest(z, 2)
+    assert r.shape == (1, 12, 18, 2)
+    for h, w, c in itertools.product(range(12), range(18), range(2)):
+        assert r[0, h, w, c] == z[0, h // 2, w // 2, c]
+    assert np.array_equal(r, np.repeat(np.repeat(z, 2, axis=1), 2, axis=2))
+    assert np.array_equal(O.op_resize_nearest(z, 1), z)
+
+
 # ---- Many-to-Many --------------------------------------------------------------
+
+def test_pooling_bruteforce_and_special_cases():
+    """Scalar loops from the definition (window clipped to the image; the mean counts only elements inside it);
+    a global average pool is the mean over the image; a 1x1 window is the identity; a constant image stays
+    constant under AveragePool whatever the padding; non-overlapping 2x2 MaxPool equals a reshape + max."""
+    x = rnd((2, 5, 7, 3), 31)
+    for k, s, p in [(3, 2, 1), (2, 2, 0), (3, 1, 1), (2, 1, 0), (3, 2, 0)]:
+        ho, wo = (5 + 2 * p - k) // s + 1, (7 + 2 * p - k) // s + 1
+        mx, av = O.op_maxpool(x, k, s, p), O.op_avgpool(x, k, s, p)
+        assert mx.shape == av.shape == (2, ho, wo, 3)
+        for n, i, j, c in itertools.product(range(2), range(ho), range(wo), range(3)):
+            vals = [x[n, a, b, c] for a in range(i * s - p, i * s - p + k) for b in range(j * s - p, j * s - p + k)
+                    if 0 <= a < 5 and 0 <= b < 7]
+            assert mx[n, i, j, c] == max(vals)
+            assert abs(av[n, i, j, c] - sum(vals) / len(vals)) < 1e-14
+    sq = rnd((2, 6, 6, 4), 32)
+    assert np.allclose(O.op_avgpool(sq, 6, 1, 0)[:, 0, 0, :], sq.mean(axis=(1, 2)), atol=1e-14)
+    assert np.array_equal(O.op_maxpool(sq, 1, 1, 0), sq)
+    assert np.allclose(O.op_avgpool(np.full((1, 5, 5, 2), 3.25), 3, 2, 1), 3.25)
+    assert np.array_equal(O.op_maxpool(sq, 2, 2, 0), sq.reshape(2, 3, 2, 3, 2, 4).max(axis=(2, 4)))
+
 
 def test_matmul_bruteforce_and_identities():
     a = rnd((2, 3, 4, 5), 9)
