@@ -40,7 +40,7 @@ int lower_dwconv(const Graph& g, const std::vector<int>& ops, int anchor, Block&
 int dwconv_launch(const Launch& L, void* status_words, int block_index, cudaStream_t st);
 void dwconv_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
 int lower_pool(const Graph& g, const std::vector<int>& ops, int anchor, Block& out, std::string& why);
-int pool_launch(const Launch& L, cudaStream_t st);
+int pool_launch(const Launch& L, void* ws_base, cudaStream_t st);
 void pool_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
 
 static GemmParams& gp_of(Launch& L) { return *reinterpret_cast<GemmParams*>(L.blob.data()); }
@@ -51,7 +51,7 @@ static const GemmParams& gp_of(const Launch& L) { return *reinterpret_cast<const
 // Handles any dtype and any operand strides; used when the tensor-core path's
 // alignment rules do not hold (and for fp32 MatMul).
 // ---------------------------------------------------------------------------
-constexpr int FB_T = 64, FB_K = 16;
+constexpr int FB_T = 64, FB_K = 32;
 
 __device__ __forceinline__ float ld_operand(const GemmOperand& o, int64_t off) {
   if (o.dtype == 0) return __ldg(reinterpret_cast<const float*>(o.ptr) + off);
@@ -121,15 +121,30 @@ __global__ void __launch_bounds__(256) gemm_fallback_kernel(const __grid_constan
   const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
   float acc[4][4] = {};
   for (int k0 = 0; k0 < p.K; k0 += FB_K) {
-    for (int i = threadIdx.x; i < FB_T * FB_K; i += 256) {
+    // All of a chunk's loads are issued before the first store to shared memory (the operand pointers are generic,
+    // so a load placed after a store would have to wait for it): small problems are bound by this latency.
+    constexpr int kLoads = FB_T * FB_K / 256;
+    float va[kLoads], vb[kLoads];
+#pragma unroll
+    for (int u = 0; u < kLoads; ++u) {
+      const int i = threadIdx.x + u * 256;
       int kk, mm;
       if (p.A.stride_col == 1) { kk = i % FB_K; mm = i / FB_K; } else { mm = i % FB_T; kk = i / FB_T; }
       int m = tile_m * FB_T + mm, k = k0 + kk;
-      As[kk][mm] = (m < p.M && k < p.K) ? ld_operand(p.A, a_base + (int64_t)m * p.A.stride_row + (int64_t)k * p.A.stride_col) : 0.0f;
+      va[u] = (m < p.M && k < p.K) ? ld_operand(p.A, a_base + (int64_t)m * p.A.stride_row + (int64_t)k * p.A.stride_col) : 0.0f;
       int nn;
       if (p.B.stride_col == 1) { nn = i % FB_T; kk = i / FB_T; } else { kk = i % FB_K; nn = i / FB_K; }
       int n = tile_n * FB_T + nn; k = k0 + kk;
-      Bs[kk][nn] = (n < p.N && k < p.K) ? ld_operand(p.B, b_base + (int64_t)k * p.B.stride_row + (int64_t)n * p.B.stride_col) : 0.0f;
+      vb[u] = (n < p.N && k < p.K) ? ld_operand(p.B, b_base + (int64_t)k * p.B.stride_row + (int64_t)n * p.B.stride_col) : 0.0f;
+    }
+#pragma unroll
+    for (int u = 0; u < kLoads; ++u) {
+      const int i = threadIdx.x + u * 256;
+      int kk, mm, nn;
+      if (p.A.stride_col == 1) { kk = i % FB_K; mm = i / FB_K; } else { mm = i % FB_T; kk = i / FB_T; }
+      As[kk][mm] = va[u];
+      if (p.B.stride_col == 1) { nn = i % FB_T; kk = i / FB_T; } else { kk = i % FB_K; nn = i / FB_K; }
+      Bs[kk][nn] = vb[u];
     }
     __syncthreads();
 #pragma unroll
@@ -482,7 +497,7 @@ void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vecto
 }
 
 int launch_contraction(const Launch& L, void* status_words, int block_index, cudaStream_t st, std::string& err) {
-  if (L.family == DNNF_FAMILY_POOL) { int rc = pool_launch(L, st); if (rc) err = "pooling launch failed"; return rc; }
+  if (L.family == DNNF_FAMILY_POOL) { int rc = pool_launch(L, status_words, st); if (rc) err = "pooling launch failed"; return rc; }
   if (L.family == DNNF_FAMILY_DWCONV) { int rc = dwconv_launch(L, status_words, block_index, st); if (rc) err = "depthwise convolution launch failed"; return rc; }
   if (L.variant == 2) { int rc = conv1x1_direct_launch(L, st); if (rc) err = "pointwise convolution launch failed"; return rc; }
   GemmParams gp = gp_of(L);

@@ -160,6 +160,7 @@ static bool pw_shape(int n, PwShape& s) {
 bool conv1x1_direct_eligible(const GemmParams& gp) {
   if (gp.A.dtype != 0 || gp.B.dtype != 0) return false;
   if (gp.batch_ext[0] * gp.batch_ext[1] != 1) return false;
+  if (gp.M < 128) return false;      // a handful of rows: one CTA would fetch all of B alone; the tiled kernel spreads N over CTAs
   if (gp.A.stride_col != 1 || gp.A.stride_row % 4 || gp.A.base % 4) return false;
   if (gp.B.stride_col != 1 || gp.B.stride_row != gp.N || gp.B.base % 4) return false;
   if (gp.N % 4 || gp.K % 4 || (int64_t)gp.K * gp.N * 4 > 96 * 1024) return false;

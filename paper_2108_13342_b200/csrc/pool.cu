@@ -10,6 +10,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <set>
 
 #include "conv_params.h"
@@ -24,6 +25,10 @@ struct PoolParams {
   int32_t kernel, stride, pad;
   int32_t is_max;
   FastDiv fd_c4, fd_w, fd_h;
+  // wide windows (a global pool): CTAs per (pixel, 128-channel group) and how the window is sliced over them
+  int32_t groups, slices, per_slice;
+  float* scratch;          // [unit][slice][128] partial results of a sliced window
+  int32_t* counters;       // [unit] arrivals, zero between runs
 };
 
 template <class SP>
@@ -61,14 +66,101 @@ __global__ void __launch_bounds__(256) pool_kernel(const __grid_constant__ PoolP
   run_program<4, SP>(p.d.prog, io);
 }
 
+// Wide windows.  A CTA reduces one slice of one output pixel's window for 128 neighbouring channels: its eight
+// warps stride over the slice's elements (a warp reads 512 contiguous bytes per element), then combine through
+// shared memory.  With one slice the CTA finishes the pixel itself; otherwise the partial goes to scratch, an
+// arrival counter per (pixel, channel group) finds the last CTA, and that CTA combines the slices in slice order
+// (the result does not depend on which CTA came last) and runs the epilogue.
+template <class SP>
+__global__ void __launch_bounds__(256) pool_wide_kernel(const __grid_constant__ PoolParams p) {
+  __shared__ float4 part[8][32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t slice = blockIdx.x % (uint32_t)p.slices;
+  const uint32_t unit = blockIdx.x / (uint32_t)p.slices;
+  const uint32_t grp = unit % (uint32_t)p.groups, pix = unit / (uint32_t)p.groups;
+  const uint32_t q1 = fd_div(pix, p.fd_w), wo = pix - q1 * (uint32_t)p.d.W;
+  const uint32_t n = fd_div(q1, p.fd_h), ho = q1 - n * (uint32_t)p.d.H;
+  const int h0 = (int)ho * p.stride - p.pad, w0 = (int)wo * p.stride - p.pad;
+  const int ha = max(h0, 0), hb = min(h0 + p.kernel, p.Hi);
+  const int wa = max(w0, 0), wb = min(w0 + p.kernel, p.Wi);
+  const int ww = wb - wa, count = (hb - ha) * ww;
+  const int c = (int)grp * 128 + lane * 4;
+  const bool live = c < p.d.C;
+  const float init = p.is_max ? -INFINITY : 0.0f;
+  float4 acc = make_float4(init, init, init, init);
+  const float* xb = p.d.x + ((size_t)n * p.Hi * p.Wi) * p.d.C + c;
+  const int e0 = (int)slice * p.per_slice, e1 = min(count, e0 + p.per_slice);
+  if (live) {
+    for (int eb = e0 + warp; eb < e1; eb += 32) {
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {            // four independent loads in flight per warp
+        const int e = eb + 8 * u;
+        v[u] = make_float4(init, init, init, init);
+        if (e < e1) {
+          const int dh = e / ww, dw = e - dh * ww;
+          v[u] = __ldg(reinterpret_cast<const float4*>(xb + ((size_t)(ha + dh) * p.Wi + (wa + dw)) * p.d.C));
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (p.is_max) { acc.x = fmaxf(acc.x, v[u].x); acc.y = fmaxf(acc.y, v[u].y); acc.z = fmaxf(acc.z, v[u].z); acc.w = fmaxf(acc.w, v[u].w); }
+        else { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+      }
+    }
+  }
+  part[warp][lane] = acc;
+  __syncthreads();
+  if (warp != 0) return;
+  auto combine = [&](float4& a, const float4& b) {
+    if (p.is_max) { a.x = fmaxf(a.x, b.x); a.y = fmaxf(a.y, b.y); a.z = fmaxf(a.z, b.z); a.w = fmaxf(a.w, b.w); }
+    else { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
+  };
+  acc = part[0][lane];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) combine(acc, part[w][lane]);
+  if (p.slices > 1) {
+    float4* mine = reinterpret_cast<float4*>(p.scratch) + ((size_t)unit * p.slices + slice) * 32;
+    mine[lane] = acc;
+    __threadfence();                         // the partial is visible before the counter moves
+    __syncwarp();
+    int old = 0;
+    if (lane == 0) old = atomicAdd(&p.counters[unit], 1);
+    old = __shfl_sync(0xffffffffu, old, 0);
+    if (old != p.slices - 1) return;         // another CTA finishes this pixel
+    if (lane == 0) p.counters[unit] = 0;     // ready for the next run
+    __threadfence();
+    const float4* all = reinterpret_cast<const float4*>(p.scratch) + (size_t)unit * p.slices * 32;
+    acc = __ldcg(all + lane);
+    for (int s = 1; s < p.slices; ++s) combine(acc, __ldcg(all + (size_t)s * 32 + lane));
+  }
+  if (!live) return;
+  DwIO io{p.d};
+  const float inv = p.is_max ? 1.0f : 1.0f / (float)count;
+  io.accv[0] = acc.x * inv; io.accv[1] = acc.y * inv; io.accv[2] = acc.z * inv; io.accv[3] = acc.w * inv;
+  io.n = n; io.h = ho; io.w = wo; io.c = (uint32_t)c;
+  run_program<4, SP>(p.d.prog, io);
+}
+
 static const PoolParams& pool_of(const Launch& L) { return *reinterpret_cast<const PoolParams*>(L.blob.data()); }
 
 struct PoolLauncher {
   const Launch& L; cudaStream_t st;
-  template <class SP> void run() { launch_pdl(pool_kernel<SP>, L.grid, 256, 0, st, pool_of(L)); }
+  template <class SP> void run() {
+    if (pool_of(L).slices > 0) launch_pdl(pool_wide_kernel<SP>, L.grid, 256, 0, st, pool_of(L));
+    else launch_pdl(pool_kernel<SP>, L.grid, 256, 0, st, pool_of(L));
+  }
 };
 
-int pool_launch(const Launch& L, cudaStream_t st) {
+int pool_launch(const Launch& L, void* ws_base, cudaStream_t st) {
+  {
+    PoolParams& pp = *reinterpret_cast<PoolParams*>(const_cast<Launch&>(L).blob.data());
+    pp.scratch = L.scratch_off >= 0 ? reinterpret_cast<float*>(reinterpret_cast<char*>(ws_base) + L.scratch_off) : nullptr;
+    pp.counters = L.counter_off >= 0 ? reinterpret_cast<int32_t*>(reinterpret_cast<char*>(ws_base) + L.counter_off) : nullptr;
+    if (pp.slices > 1 && (!pp.scratch || !pp.counters)) return 1;
+  }
   PoolLauncher F{L, st};
   if (!(L.static_id > 0 && StaticSet<ConvStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
   return cudaGetLastError() == cudaSuccess ? 0 : 1;
@@ -129,6 +221,22 @@ int lower_pool(const Graph& g, const std::vector<int>& ops, int anchor, Block& o
   const int64_t total = Y.numel() / 4;
   L.grid = (int)((total + 255) / 256);
   L.threads = 256;
+  pp.slices = 0;
+  if (pp.kernel * pp.kernel >= 64 && !getenv("DNNF_NO_WIDE_POOL")) {
+    // one thread per output would walk the window alone: give the window to whole CTAs instead
+    pp.groups = (dp.C + 127) / 128;
+    const int64_t units = (int64_t)dp.N * dp.H * dp.W * pp.groups;
+    const int window = pp.kernel * pp.kernel;
+    int slices = (int)std::min<int64_t>(std::max<int64_t>(1, (2 * 148 + units - 1) / units), std::max(1, window / 32));
+    pp.per_slice = (window + slices - 1) / slices;
+    pp.slices = (window + pp.per_slice - 1) / pp.per_slice;
+    if (units * pp.slices < (1ll << 31)) {
+      L.grid = (int)(units * pp.slices);
+      if (pp.slices > 1) { L.counter_bytes = units * 4; L.scratch_bytes = units * pp.slices * 128 * 4; }
+    } else {
+      pp.slices = 0;
+    }
+  }
   L.variant = pp.is_max;
   L.static_id = StaticSet<ConvStatic>::find(dp.prog);
   out.lowered = true;

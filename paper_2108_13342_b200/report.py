@@ -38,7 +38,7 @@ def _graph_of(torch, dev, fn):
     return g
 
 
-def measure_workload(torch, dev, wl, pk, flags, copies, iters=20, rewrite=B.REWRITE_NONE, per_block_limit=16):
+def measure_workload(torch, dev, wl, pk, flags, copies, iters=20, rewrite=B.REWRITE_NONE, per_block_limit=40):
     """`copies` sessions with distinct buffers, run round-robin so that every launch
     sees cold data when copies * footprint exceeds L2."""
     sess = [Session(wl, plan_flags=flags, rewrite_flags=rewrite, device=dev) for _ in range(copies)]
@@ -96,6 +96,7 @@ def per_config(dev, pk, only=None):
         ("cfg2b 131072-row variant", W.add_layernorm_gelu(rows=131072), 1),
         ("cfg3 GEMM+bias+GELU ; GEMM+bias+residual bf16 [4096,768,3072]", W.ffn_block(), 8),
         ("cfg4 MBConv fp32 NHWC [32,56,56,24->144->24]", W.mbconv_block(), 2),
+        ("next: CNN fragment with pooling, SpaceToDepth/DepthToSpace, Resize, Concat fp32 NHWC [32,64,64,32]", W.cnn_neck(n=32), 2),
     ]
     for name, wl, copies in cases:
         if only and only not in name:

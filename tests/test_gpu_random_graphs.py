@@ -27,7 +27,7 @@ class _Rng:
         return xs[min(int(self.u() * len(xs)), len(xs) - 1)]
 
 
-def _build(seed, big=False, dtype="f32"):
+def _build(seed, big=False, dtype="f32", extended=False):
     r = _Rng(seed)
     bsz, rows, cols = r.pick([1, 2, 3]), r.pick([5, 8, 16, 33]), r.pick([8, 12, 32, 64])
     if big:      # sizes that reach the vectorised, multi-vector, multi-warp and tensor-core variants
@@ -47,6 +47,12 @@ def _build(seed, big=False, dtype="f32"):
         g.ext(name, (n,)); ins[name] = W.uniform(777, 3000 + 10 * seed + n_ext[0], (n,), lo, hi)
         return name
 
+    def vec_like(shape):
+        n_ext[0] += 1
+        name = "f%d" % n_ext[0]
+        g.ext(name, shape, dtype); ins[name] = data(W.uniform(777, 6000 + 10 * seed + n_ext[0], shape, -1.0, 1.0))
+        return name
+
     def mat(k, n):
         n_ext[0] += 1
         name = "m%d" % n_ext[0]
@@ -57,7 +63,7 @@ def _build(seed, big=False, dtype="f32"):
     for _ in range(n_ops):
         t, shp = r.pick(pool[-4:]) if r.u() < 0.7 else r.pick(pool)      # mostly recent values (long chains), sometimes old ones (diamonds)
         kind = r.pick(["unary", "unary", "vec", "full", "transpose", "reshape", "slice", "reduce", "softmax", "layernorm", "matmul",
-                       "rowvec", "exp", "div", "reduce0", "permute"])
+                       "rowvec", "exp", "div", "reduce0", "permute"] + (["concat", "concat", "concat"] if extended else []))
         if kind in ("reduce", "reduce0", "softmax", "layernorm") and shp[-1] > 8192:
             continue                                    # longer rows than the row kernels take (the plan says so)
         if kind == "unary":
@@ -72,6 +78,13 @@ def _build(seed, big=False, dtype="f32"):
             cands = [p for p in pool if p[1] == shp]
             den = g.add("AddC", [g.add("Abs", [g.add("Tanh", [r.pick(cands)[0]])])], c=1.5)
             o = g.add("Div", [g.add("Tanh", [t]), den])
+        elif kind == "concat":
+            cands = [p for p in pool if p[1] == shp]
+            other = r.pick(cands)[0]
+            ax = int(r.u() * len(shp))
+            third = [vec_like(shp)] if r.u() < 0.3 else []
+            o = g.add("Concat", [t, other] + third, axis=ax)
+            shp = shp[:ax] + ((2 + len(third)) * shp[ax],) + shp[ax + 1:]
         elif kind == "rowvec":
             if len(shp) < 2:
                 continue
@@ -192,6 +205,28 @@ def test_random_graph(seed):
                     raise AssertionError(f"{n} flags {flags} rewrite {rewrite} db {db} plan {[b['ops'] for b in s.g.blocks()]}: {e}") from None
         finally:
             B.profile_db_clear()
+
+
+@pytest.mark.parametrize("seed", [pytest.param(i, id=str(i)) for i in range(120)] + [pytest.param(-i - 1, id="big%d" % i) for i in range(30)])
+def test_random_graph_with_concat(seed):
+    """The same generator with Concat among the operators: parts stored by producer blocks of every family,
+    results read through views, nested and repeated inputs."""
+    wl = _build(5000 + seed, False, extended=True) if seed >= 0 else _build(6000 - seed, True, extended=True)
+    ref = O.run_graph(wl.graph, wl.inputs)
+    for flags in (B.PLAN_FUSED, B.PLAN_UNFUSED):
+        s = Session(wl, plan_flags=flags, rewrite_flags=B.REWRITE_NONE)
+        s.workspace[s.g.workspace_zero_bytes():].fill_(0xFF)
+        for n in wl.graph.outputs:
+            s.buffers[n].fill_(float("nan"))
+        s.run()
+        assert s.g.status()[0] == 0
+        for n in wl.graph.outputs:
+            got = s.output(n)
+            assert np.isfinite(got).all(), (n, "unwritten elements", [b["ops"] for b in s.g.blocks()])
+            try:
+                close(got, ref[n], 2e-4 if seed < 0 else 2e-5)
+            except AssertionError as e:
+                raise AssertionError(f"{n} plan {[b['ops'] for b in s.g.blocks()]}: {e}") from None
 
 
 @pytest.mark.parametrize("seed", range(80))
