@@ -106,6 +106,13 @@ typedef enum {
                                                        result [N,(H+2p-k)/s+1,(W+2p-k)/s+1,C]; MaxPool ignores the padding,
                                                        AveragePool divides by the number of elements inside the image;
                                                        a global pool is KERNEL = H = W, STRIDE 1, PAD 0 */
+  /* more One-to-One operators of Table 2 */
+  DNNF_OP_SIN, DNNF_OP_COS, DNNF_OP_ASIN, DNNF_OP_CEIL, DNNF_OP_FLOOR,
+  DNNF_OP_ROUND,                                    /* to nearest, ties to even */
+  DNNF_OP_LEAKYRELU,                                /* attribute C: the slope for negative inputs */
+  DNNF_OP_NOT,                                      /* on 0 / 1 valued tensors: 1 where the input is 0, else 0 */
+  DNNF_OP_GREATER,                                  /* (a, b) with broadcasting: 1 where a > b, else 0 */
+  DNNF_OP_PRELU,                                    /* (x, slope) with broadcasting: x where x > 0, else slope * x */
   DNNF_OP_CONCATPART,                               /* internal (made by Concat): (x [, result so far]); AXIS, START, SHAPE */
   DNNF_OP__COUNT
 } dnnf_op_t;

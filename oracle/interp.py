@@ -249,6 +249,20 @@ def op_reduceprod(x, axis=-1, keepdims=1): return _reduce(np.prod, x, axis, keep
 def op_reducemax(x, axis=-1, keepdims=1): return _reduce(np.max, x, axis, keepdims)
 
 
+# ---- further One-to-One operators of Table 2 ---------------------------------
+
+def op_sin(x): return np.sin(x)
+def op_cos(x): return np.cos(x)
+def op_asin(x): return np.arcsin(x)
+def op_ceil(x): return np.ceil(x)
+def op_floor(x): return np.floor(x)
+def op_round(x): return np.rint(x)                         # to nearest, ties to even (ONNX Round)
+def op_leakyrelu(x, alpha): return np.where(x > 0, x, float(alpha) * x)
+def op_not(x): return np.where(x == 0, 1.0, 0.0)           # on 0 / 1 valued tensors
+def op_greater(a, b): return np.where(a > b, 1.0, 0.0)     # multidirectional broadcasting
+def op_prelu(x, slope): return np.where(x > 0, x, slope * x)
+
+
 # ---- dispatcher -------------------------------------------------------------
 
 def _apply(op, ins, at):
@@ -270,6 +284,16 @@ def _apply(op, ins, at):
     if op == "Recip": return [op_recip(ins[0])]
     if op == "Square": return [op_square(ins[0])]
     if op == "Relu": return [op_relu(ins[0])]
+    if op == "Sin": return [op_sin(ins[0])]
+    if op == "Cos": return [op_cos(ins[0])]
+    if op == "Asin": return [op_asin(ins[0])]
+    if op == "Ceil": return [op_ceil(ins[0])]
+    if op == "Floor": return [op_floor(ins[0])]
+    if op == "Round": return [op_round(ins[0])]
+    if op == "LeakyRelu": return [op_leakyrelu(ins[0], g("alpha", g("c", 0.01)))]
+    if op == "Not": return [op_not(ins[0])]
+    if op == "Greater": return [op_greater(ins[0], ins[1])]
+    if op == "PRelu": return [op_prelu(ins[0], ins[1])]
     if op == "Clip": return [op_clip(ins[0], at["lo"], at["hi"])]
     if op == "Pow": return [op_pow(ins[0], at["p"])]
     if op == "BitShift": return [op_bitshift(ins[0], at["bits"], g("direction", "left"))]

@@ -31,12 +31,14 @@ FAMILY_NAMES = ["alias", "elementwise", "transpose", "row", "gemm", "conv1x1", "
 OP_NAMES = ["?", "Add", "Sub", "Mul", "Div", "MulC", "AddC", "Sigmoid", "Tanh", "Erf", "Exp", "Log", "Sqrt", "Abs",
             "Neg", "Recip", "Square", "Relu", "Clip", "Pow", "Gelu", "ScaleShift", "Transpose", "Reshape", "Flatten",
             "Squeeze", "Unsqueeze", "Split", "Slice", "MatMul", "Conv1x1", "DwConv3x3", "Softmax", "LayerNorm",
-            "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift", "DepthToSpace", "SpaceToDepth", "Resize", "Concat", "MaxPool", "AveragePool", "ConcatPart"]
+            "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift", "DepthToSpace", "SpaceToDepth", "Resize", "Concat", "MaxPool", "AveragePool", "Sin", "Cos", "Asin", "Ceil",
+            "Floor", "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConcatPart"]
 OP = {n: i for i, n in enumerate(OP_NAMES) if i}
 
 ATTR = {"c": 1, "lo": 2, "hi": 3, "p": 4, "eps": 5, "approx": 6, "axis": 7, "keepdims": 8, "start": 9, "end": 10,
-        "bits": 11, "perm": 12, "shape": 13, "sizes": 14, "axes": 15, "block": 16, "scale": 17, "kernel": 18, "stride": 19, "pad": 20}
-_FLOAT_ATTRS = {"c", "lo", "hi", "p", "eps"}
+        "bits": 11, "perm": 12, "shape": 13, "sizes": 14, "axes": 15, "block": 16, "scale": 17, "kernel": 18, "stride": 19, "pad": 20,
+        "alpha": 1}      # LeakyRelu's slope travels as attribute C
+_FLOAT_ATTRS = {"c", "lo", "hi", "p", "eps", "alpha"}
 
 REWRITE_DEFAULT, REWRITE_NONE, REWRITE_CANON_MACRO = 0, 1, 2
 PLAN_FUSED, PLAN_UNFUSED, PLAN_STRICT_TABLE3, PLAN_ALLOW_PROLOGUE = 0, 1, 2, 4

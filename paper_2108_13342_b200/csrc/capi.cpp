@@ -286,7 +286,7 @@ int dnnf_block_program(const dnnf_graph* g, int bi, char* buf, size_t cap) {
   if (!g || !buf || cap == 0 || bi < 0 || bi >= (int)g->g.blocks.size()) return DNNF_ERR_INVALID_ARG;
   static const char* on[] = {"END", "MOV", "SAVE", "STORE", "ADD", "SUB", "RSUB", "MUL", "DIV", "RDIV", "MAX", "MIN", "NEG", "ABS",
     "RECIP", "SQUARE", "SQRT", "EXP", "LOG", "TANH", "ERF", "SIGMOID", "RELU", "GELU_ERF", "GELU_TANH", "CLIP", "POW",
-    "ROWSUM", "ROWMEAN", "ROWMAX", "ROWPROD"};
+    "SIN", "COS", "ASIN", "CEIL", "FLOOR", "ROUND", "NOT", "LEAKY", "GT", "LT", "PRELU", "RPRELU", "ROWSUM", "ROWMEAN", "ROWMAX", "ROWPROD"};
   const Block& b = g->g.blocks[bi];
   const Program* pr = program_of(b.launch);
   std::string s;

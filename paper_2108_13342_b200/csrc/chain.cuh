@@ -171,6 +171,54 @@ __device__ __forceinline__ void apply_op(int op, float (&acc)[VV], const float (
 #pragma unroll
       for (int v = 0; v < VV; ++v) acc[v] = powf(acc[v], c0);
       break;
+    case M_SIN:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = sinf(acc[v]);
+      break;
+    case M_COS:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = cosf(acc[v]);
+      break;
+    case M_ASIN:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = asinf(acc[v]);
+      break;
+    case M_CEIL:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = ceilf(acc[v]);
+      break;
+    case M_FLOOR:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = floorf(acc[v]);
+      break;
+    case M_ROUND:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = rintf(acc[v]);
+      break;
+    case M_NOT:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = acc[v] == 0.0f ? 1.0f : 0.0f;
+      break;
+    case M_LEAKY:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = acc[v] > 0.0f ? acc[v] : c0 * acc[v];
+      break;
+    case M_GT:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = acc[v] > src[v] ? 1.0f : 0.0f;
+      break;
+    case M_LT:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = acc[v] < src[v] ? 1.0f : 0.0f;
+      break;
+    case M_PRELU:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = acc[v] > 0.0f ? acc[v] : src[v] * acc[v];
+      break;
+    case M_RPRELU:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = src[v] > 0.0f ? src[v] : acc[v] * src[v];
+      break;
     default: break;
   }
 }

@@ -59,7 +59,8 @@ const char* op_name(int k) {
   static const char* names[] = {"?", "Add", "Sub", "Mul", "Div", "MulC", "AddC", "Sigmoid", "Tanh", "Erf", "Exp", "Log",
     "Sqrt", "Abs", "Neg", "Recip", "Square", "Relu", "Clip", "Pow", "Gelu", "ScaleShift", "Transpose", "Reshape",
     "Flatten", "Squeeze", "Unsqueeze", "Split", "Slice", "MatMul", "Conv1x1", "DwConv3x3", "Softmax", "LayerNorm",
-    "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift", "DepthToSpace", "SpaceToDepth", "Resize", "Concat", "MaxPool", "AveragePool", "ConcatPart"};
+    "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift", "DepthToSpace", "SpaceToDepth", "Resize", "Concat", "MaxPool", "AveragePool", "Sin", "Cos", "Asin", "Ceil", "Floor",
+    "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConcatPart"};
   if (k <= 0 || k >= DNNF_OP__COUNT) return "?";
   return names[k];
 }
@@ -69,7 +70,10 @@ bool is_index_only(int k) {
          k == DNNF_OP_UNSQUEEZE || k == DNNF_OP_SLICE || k == DNNF_OP_SPLIT || k == DNNF_OP_EXPAND || k == DNNF_OP_CONCATPART;
 }
 bool is_elementwise(int k) {
-  return (k >= DNNF_OP_ADD && k <= DNNF_OP_SCALESHIFT) || k == DNNF_OP_BITSHIFT;
+  return (k >= DNNF_OP_ADD && k <= DNNF_OP_SCALESHIFT) || k == DNNF_OP_BITSHIFT || (k >= DNNF_OP_SIN && k <= DNNF_OP_PRELU);
+}
+bool is_binary_elementwise(int k) {
+  return k == DNNF_OP_ADD || k == DNNF_OP_SUB || k == DNNF_OP_MUL || k == DNNF_OP_DIV || k == DNNF_OP_GREATER || k == DNNF_OP_PRELU;
 }
 bool is_row_anchor(int k) {
   return k == DNNF_OP_SOFTMAX || k == DNNF_OP_LAYERNORM || (k >= DNNF_OP_REDUCESUM && k <= DNNF_OP_REDUCEPROD);
@@ -105,7 +109,7 @@ int edge_mapping(const Graph& g, const Op& op, int slot) {
   const Tensor& in = g.tensors[op.in[slot]];
   const Tensor& out = g.tensors[op.out[0]];
   int k = op.kind;
-  if (k == DNNF_OP_ADD || k == DNNF_OP_SUB || k == DNNF_OP_MUL || k == DNNF_OP_DIV)
+  if (is_binary_elementwise(k))
     return same_shape(in, out) ? DNNF_ONE_TO_ONE : DNNF_ONE_TO_MANY;     // "elementwise w/ broadcast"
   if (k == DNNF_OP_SCALESHIFT) return slot == 0 ? DNNF_ONE_TO_ONE : DNNF_ONE_TO_MANY;
   if (k == DNNF_OP_LAYERNORM) return slot == 0 ? DNNF_MANY_TO_MANY : DNNF_ONE_TO_MANY;
@@ -115,7 +119,7 @@ int edge_mapping(const Graph& g, const Op& op, int slot) {
 int node_mapping(const Graph& g, const Op& op) {
   int k = op.kind;
   switch (k) {
-    case DNNF_OP_ADD: case DNNF_OP_SUB: case DNNF_OP_MUL: case DNNF_OP_DIV: {
+    case DNNF_OP_ADD: case DNNF_OP_SUB: case DNNF_OP_MUL: case DNNF_OP_DIV: case DNNF_OP_GREATER: case DNNF_OP_PRELU: {
       // most complex pair decides (Section 3.1)
       int m = DNNF_ONE_TO_ONE;
       for (int s = 0; s < (int)op.in.size(); ++s) m = std::max(m, edge_mapping(g, op, s));
@@ -177,7 +181,7 @@ int infer_shapes(Graph& g, Op& op, std::string& err) {
   std::vector<std::vector<int64_t>> outs;
   int k = op.kind;
   auto norm_axis = [&](int64_t a, int rank) { return a < 0 ? a + rank : a; };
-  if (k == DNNF_OP_ADD || k == DNNF_OP_SUB || k == DNNF_OP_MUL || k == DNNF_OP_DIV) {
+  if (is_binary_elementwise(k)) {
     if (!need(2)) return DNNF_ERR_INVALID_ARG;
     std::vector<int64_t> o;
     if (!broadcast_dims(in(0).dims, in(1).dims, o)) { err = "broadcast mismatch"; return DNNF_ERR_SHAPE; }

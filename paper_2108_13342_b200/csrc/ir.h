@@ -116,6 +116,7 @@ bool is_index_only(int kind);       // Reorganize / Shuffle / Slice: no arithmet
 bool is_elementwise(int kind);
 bool is_row_anchor(int kind);
 bool is_contraction(int kind);
+bool is_binary_elementwise(int kind);   // two operands with multidirectional broadcasting
 const char* op_name(int kind);
 // Bytes a block stores when tensor t is one of its outputs: the whole tensor, except for a Concat's part, which
 // fills only its own range of the shared result.

@@ -111,7 +111,7 @@ bool backward_views(LowerCtx& cx, const Op& op, const View& vout, std::vector<Vi
     vin[0] = vout;                      // same flat order
     return true;
   }
-  if (k == DNNF_OP_ADD || k == DNNF_OP_SUB || k == DNNF_OP_MUL || k == DNNF_OP_DIV || k == DNNF_OP_EXPAND) {
+  if (is_binary_elementwise(k) || k == DNNF_OP_EXPAND) {
     bool need_align = false;
     for (size_t i = 0; i < op.in.size(); ++i) if (in(i).dims != out.dims) need_align = true;
     Aligned al;
@@ -549,6 +549,16 @@ bool emit_program(LowerCtx& cx, int anchor_out, int max_tmp) {
       case DNNF_OP_LOG: E.unary(v[0], M_LOG); break;
       case DNNF_OP_SQRT: E.unary(v[0], M_SQRT); break;
       case DNNF_OP_ABS: E.unary(v[0], M_ABS); break;
+      case DNNF_OP_SIN: E.unary(v[0], M_SIN); break;
+      case DNNF_OP_COS: E.unary(v[0], M_COS); break;
+      case DNNF_OP_ASIN: E.unary(v[0], M_ASIN); break;
+      case DNNF_OP_CEIL: E.unary(v[0], M_CEIL); break;
+      case DNNF_OP_FLOOR: E.unary(v[0], M_FLOOR); break;
+      case DNNF_OP_ROUND: E.unary(v[0], M_ROUND); break;
+      case DNNF_OP_NOT: E.unary(v[0], M_NOT); break;
+      case DNNF_OP_LEAKYRELU: E.unary(v[0], M_LEAKY, S_CONST, (uint8_t)E.cst((float)op.at.c)); break;
+      case DNNF_OP_GREATER: E.binary(v[0], v[1], M_GT, M_LT, false); break;
+      case DNNF_OP_PRELU: E.binary(v[0], v[1], M_PRELU, M_RPRELU, false); break;
       case DNNF_OP_NEG: E.unary(v[0], M_NEG); break;
       case DNNF_OP_RECIP: E.unary(v[0], M_RECIP); break;
       case DNNF_OP_SQUARE: E.unary(v[0], M_SQUARE); break;

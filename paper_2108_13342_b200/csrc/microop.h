@@ -30,6 +30,11 @@ enum MOp : uint8_t {
   M_GELU_ERF, M_GELU_TANH,
   M_CLIP,       // acc = min(max(acc, const[idx]), const[idx+1])
   M_POW,        // acc = pow(acc, const[idx])
+  M_SIN, M_COS, M_ASIN, M_CEIL, M_FLOOR, M_ROUND,
+  M_NOT,        // acc = acc == 0 ? 1 : 0
+  M_LEAKY,      // acc = acc > 0 ? acc : const[idx] * acc
+  M_GT, M_LT,   // acc = acc > src ? 1 : 0 ; acc = acc < src ? 1 : 0
+  M_PRELU, M_RPRELU,   // acc = acc > 0 ? acc : src * acc ; acc = src > 0 ? src : acc * src
   M_ROWSUM, M_ROWMEAN, M_ROWMAX, M_ROWPROD,   // row kernels only: acc = reduce over the row, broadcast
   M__COUNT
 };

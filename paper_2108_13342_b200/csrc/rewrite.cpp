@@ -108,6 +108,9 @@ struct Rewriter {
       snprintf(buf, sizeof buf, "|%a|%a|%a|%a|%a|%lld|%lld|%lld|%lld|%lld|%lld", o.at.c, o.at.lo, o.at.hi, o.at.p, o.at.eps, (long long)o.at.approx,
                (long long)o.at.axis, (long long)o.at.keepdims, (long long)o.at.start, (long long)o.at.end, (long long)o.at.bits);
       key += buf;
+      snprintf(buf, sizeof buf, "|%lld|%lld|%lld|%lld|%lld", (long long)o.at.block, (long long)o.at.scale, (long long)o.at.kernel,
+               (long long)o.at.stride, (long long)o.at.pad);
+      key += buf;
       for (auto v : o.at.perm) key += "p" + std::to_string(v);
       for (auto v : o.at.shape) key += "s" + std::to_string(v);
       for (auto v : o.at.axes) key += "a" + std::to_string(v);

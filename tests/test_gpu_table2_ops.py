@@ -169,3 +169,45 @@ def test_cnn_fragment(dims, flags, rewrite):
     s = check(wl, 5e-4, flags, rewrite)          # several split-TF32 convolutions in sequence
     if flags == B.PLAN_FUSED:
         assert s.plan_stats.n_kernels < s.plan_stats.n_ops
+
+
+# ---- further One-to-One operators of Table 2 -------------------------------------------------------------------
+
+@pytest.mark.parametrize("flags", PLANS)
+@pytest.mark.parametrize("shape", [(3, 37, 20), (2, 64, 256), (5, 7)])
+def test_further_one_to_one_operators(shape, flags):
+    """Sin / Cos / Asin in a chain; the discrete operators (Ceil, Floor, Round, Greater, Not) applied to inputs, where both
+    sides see the same fp32-representable values, and their 0 / 1 or integer results used further down the chain."""
+    g = graph("more_ops")
+    g.ext("X", shape); g.ext("U", shape); g.ext("v", (shape[-1],)); g.ext("H", shape)
+    t = g.add("Asin", [g.add("Mul", [g.add("Sin", ["X"]), g.add("Cos", ["X"])])])          # |sin cos| <= 1/2
+    t = g.add("LeakyRelu", [g.add("Sub", [t, "U"])], alpha=0.125)
+    t = g.add("PRelu", [g.add("Sub", [t, "v"]), "v"])                                      # slope broadcast along the rows
+    g.mark_output(t)
+    gt = g.add("Greater", ["X", "U"])
+    sel = g.add("Add", [g.add("Mul", [gt, "X"]), g.add("Mul", [g.add("Not", [gt]), "U"])])  # max(X, U) spelled with a mask
+    g.mark_output(sel)
+    g.mark_output(g.add("Greater", ["X", "v"]))
+    r = g.add("Add", [g.add("Ceil", ["H"]), g.add("Add", [g.add("Floor", ["H"]), g.add("Round", ["H"])])])
+    g.mark_output(r)
+    halves = np.round(rnd(shape, 63, -8.0, 8.0) * 2.0) / 2.0          # multiples of 1/2: ties included
+    ins = {"X": rnd(shape, 60), "U": rnd(shape, 61), "v": rnd((shape[-1],), 62, 0.1, 0.9), "H": halves.astype(np.float32)}
+    s, got, ref = run_both(W.Workload(g, ins), flags)
+    names = list(g.outputs)
+    close(got[names[0]], ref[names[0]], RTOL_F32)
+    for n in names[1:]:
+        assert np.array_equal(got[n].astype(np.float64), ref[n]), n
+    assert np.array_equal(got[names[1]], np.maximum(ins["X"], ins["U"]))
+
+
+@pytest.mark.parametrize("flags", PLANS)
+def test_prelu_and_leakyrelu_in_a_convolution_epilogue(flags):
+    g = graph("conv_prelu")
+    g.ext("X", (2, 12, 12, 16)); g.ext("Wt", (16, 32), kind="weight"); g.ext("b", (32,)); g.ext("a", (32,))
+    t = g.add("PRelu", [g.add("Add", [g.add("Conv1x1", ["X", "Wt"]), "b"]), "a"])
+    t = g.add("LeakyRelu", [g.add("AddC", [t], c=-0.1)], alpha=0.2)
+    g.mark_output(t)
+    ins = {"X": rnd((2, 12, 12, 16), 64), "Wt": rnd((16, 32), 65, -0.3, 0.3), "b": rnd((32,), 66, -0.5, 0.5), "a": rnd((32,), 67, 0.05, 0.3)}
+    s = check(W.Workload(g, ins), RTOL_F32, flags)
+    if flags == B.PLAN_FUSED:
+        assert s.plan_stats.n_kernels == 1, s.g.blocks()

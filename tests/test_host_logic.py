@@ -491,3 +491,30 @@ def test_pooling_shapes_types_and_epilogue_fusion():
         g.add("MaxPool", ["X"], **at)
         with pytest.raises(B.DnnfError):
             _plan_desc(g)
+
+
+def test_further_one_to_one_operators_type_and_fuse():
+    g = _desc(); g.ext("X", (4, 8)); g.ext("v", (8,))
+    t = g.add("PRelu", [g.add("Sin", ["X"]), "v"])
+    t = g.add("Greater", [g.add("LeakyRelu", [t], alpha=0.1), g.add("Round", ["X"])])
+    g.mark_output(g.add("Not", [t]))
+    G, ids, st = _plan_desc(g)
+    assert st.n_ops == 6 and st.n_kernels == 1
+    kinds = G.blocks()[0]["ops"]
+    assert kinds == ["Sin", "PRelu", "LeakyRelu", "Round", "Greater", "Not"], kinds
+    prog = G.block_program(0)
+    for name in ("SIN", "PRELU", "LEAKY", "ROUND", "NOT"):
+        assert name in prog, prog
+    assert "GT" in prog or "LT" in prog
+    # the two pools differ only in attributes the common-subexpression pass must tell apart
+    g = _desc(); g.ext("X", (1, 8, 8, 4))
+    a = g.add("MaxPool", ["X"], kernel=2, stride=2, pad=0)
+    b = g.add("MaxPool", ["X"], kernel=2, stride=1, pad=0)
+    ra = g.add("Relu", [a]); rb = g.add("Relu", [b])
+    g.mark_output(ra); g.mark_output(rb)
+    from paper_2108_13342_b200.runtime import build_graph
+    G, ids = build_graph(g)
+    G.rewrite(B.REWRITE_DEFAULT)
+    G.plan(B.PLAN_FUSED)
+    assert G.tensor_info(ids[ra])[1] == (1, 4, 4, 4) and G.tensor_info(ids[rb])[1] == (1, 7, 7, 4)
+    assert len([x for x in G.blocks() if x["family"] == "pool"]) == 2

@@ -165,6 +165,27 @@ def test_gather():
     assert np.array_equal(y, np.stack([x[4], x[0], x[4]]))
 
 
+def test_further_one_to_one_operators_at_known_points():
+    assert np.allclose(O.op_sin(np.array([0.0, math.pi / 6, math.pi / 2, -math.pi / 2])), [0.0, 0.5, 1.0, -1.0], atol=1e-15)
+    assert np.allclose(O.op_cos(np.array([0.0, math.pi / 3, math.pi])), [1.0, 0.5, -1.0], atol=1e-15)
+    assert np.allclose(O.op_asin(np.array([0.0, 0.5, 1.0, -1.0])), [0.0, math.pi / 6, math.pi / 2, -math.pi / 2], atol=1e-15)
+    x = rnd((50,), 40, -1.0, 1.0)
+    assert np.allclose(O.op_sin(x) ** 2 + O.op_cos(x) ** 2, 1.0, atol=1e-15)
+    assert np.allclose(O.op_sin(O.op_asin(x)), x, atol=1e-15)
+    v = np.array([-2.5, -1.5, -0.5, -0.2, 0.0, 0.2, 0.5, 1.5, 2.5, 3.0])
+    assert np.array_equal(O.op_ceil(v), [-2, -1, -0, -0, 0, 1, 1, 2, 3, 3])
+    assert np.array_equal(O.op_floor(v), [-3, -2, -1, -1, 0, 0, 0, 1, 2, 3])
+    assert np.array_equal(O.op_round(v), [-2, -2, -0, -0, 0, 0, 0, 2, 2, 3])          # ties go to the even neighbour
+    assert np.array_equal(O.op_leakyrelu(np.array([-4.0, 0.0, 3.0]), 0.25), [-1.0, 0.0, 3.0])
+    assert np.array_equal(O.op_not(np.array([0.0, 1.0, 0.0])), [1.0, 0.0, 1.0])
+    a = np.array([[1.0, 5.0, 3.0], [4.0, 2.0, 6.0]])
+    assert np.array_equal(O.op_greater(a, np.array([2.0, 2.0, 6.0])), [[0, 1, 0], [1, 0, 0]])      # broadcast over rows
+    assert np.array_equal(O.op_greater(a, a), np.zeros((2, 3)))
+    assert np.array_equal(O.op_prelu(np.array([[-2.0, 4.0], [-1.0, -8.0]]), np.array([0.5, 0.25])), [[-1.0, 4.0], [-0.5, -2.0]])
+    assert np.array_equal(O.op_prelu(x, np.ones(50)), x)
+    assert np.array_equal(O.op_prelu(x, np.zeros(50)), O.op_relu(x))
+
+
 def test_depthtospace_spacetodepth_resize_index_loops():
     """Each element against the index formula of the operator's definition, in pure-Python loops; the two Shuffle
     operators undo each other; nearest-neighbour enlargement equals numpy's repeat along both image axes."""
