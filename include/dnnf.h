@@ -113,6 +113,11 @@ typedef enum {
   DNNF_OP_NOT,                                      /* on 0 / 1 valued tensors: 1 where the input is 0, else 0 */
   DNNF_OP_GREATER,                                  /* (a, b) with broadcasting: 1 where a > b, else 0 */
   DNNF_OP_PRELU,                                    /* (x, slope) with broadcasting: x where x > 0, else slope * x */
+  DNNF_OP_CONVTRANSPOSE,                            /* Many-to-Many; NHWC x [Cin,k,k,Cout] with stride = kernel = k (attribute KERNEL),
+                                                       no padding: y[n,h*k+i,w*k+j,o] = sum_c x[n,h,w,c] W[c,i,j,o].  Recorded as
+                                                       Reshape(W) -> Conv1x1 -> DepthToSpace, which it equals term by term */
+  DNNF_OP_GATHER,                                   /* One-to-Many; (table [V,D], indices [...]) along axis 0: y[..., :] = table[indices[...], :].
+                                                       Indices are integer-valued fp32 numbers; out-of-range ones are clamped */
   DNNF_OP_CONCATPART,                               /* internal (made by Concat): (x [, result so far]); AXIS, START, SHAPE */
   DNNF_OP__COUNT
 } dnnf_op_t;
@@ -173,7 +178,8 @@ typedef enum {
   DNNF_FAMILY_GEMM = 4,        /* tensor-core GEMM anchor with an epilogue chain */
   DNNF_FAMILY_CONV1X1 = 5,     /* fp32 pointwise convolution with an epilogue chain */
   DNNF_FAMILY_DWCONV = 6,      /* fp32 depthwise 3x3 with an epilogue chain */
-  DNNF_FAMILY_POOL = 7         /* fp32 MaxPool / AveragePool with an epilogue chain */
+  DNNF_FAMILY_POOL = 7,        /* fp32 MaxPool / AveragePool with an epilogue chain */
+  DNNF_FAMILY_GATHER = 8       /* row gather by an index tensor */
 } dnnf_family_t;
 
 typedef struct {

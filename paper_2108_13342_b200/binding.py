@@ -26,13 +26,13 @@ INPUT, WEIGHT = 0, 1
 ONE_TO_ONE, REORGANIZE, SHUFFLE, ONE_TO_MANY, MANY_TO_MANY = range(5)
 GREEN, YELLOW, RED = range(3)
 MAPPING_NAMES = ["One-to-One", "Reorganize", "Shuffle", "One-to-Many", "Many-to-Many"]
-FAMILY_NAMES = ["alias", "elementwise", "transpose", "row", "gemm", "conv1x1", "dwconv", "pool"]
+FAMILY_NAMES = ["alias", "elementwise", "transpose", "row", "gemm", "conv1x1", "dwconv", "pool", "gather"]
 
 OP_NAMES = ["?", "Add", "Sub", "Mul", "Div", "MulC", "AddC", "Sigmoid", "Tanh", "Erf", "Exp", "Log", "Sqrt", "Abs",
             "Neg", "Recip", "Square", "Relu", "Clip", "Pow", "Gelu", "ScaleShift", "Transpose", "Reshape", "Flatten",
             "Squeeze", "Unsqueeze", "Split", "Slice", "MatMul", "Conv1x1", "DwConv3x3", "Softmax", "LayerNorm",
             "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift", "DepthToSpace", "SpaceToDepth", "Resize", "Concat", "MaxPool", "AveragePool", "Sin", "Cos", "Asin", "Ceil",
-            "Floor", "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConcatPart"]
+            "Floor", "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConvTranspose", "Gather", "ConcatPart"]
 OP = {n: i for i, n in enumerate(OP_NAMES) if i}
 
 ATTR = {"c": 1, "lo": 2, "hi": 3, "p": 4, "eps": 5, "approx": 6, "axis": 7, "keepdims": 8, "start": 9, "end": 10,

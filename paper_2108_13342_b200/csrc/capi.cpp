@@ -156,6 +156,34 @@ int dnnf_add_op(dnnf_graph* g, int op_kind, int n_in, const int* in_ids, const d
       G.ops.push_back(o);
     }
     outs = {carrier};
+  } else if (op_kind == DNNF_OP_CONVTRANSPOSE) {
+    // stride = kernel: every output element receives one term per input channel, so the operator is a pointwise
+    // convolution onto k*k*Cout channels followed by the DepthToSpace that spreads them over the k x k cell
+    if (n_in != 2) return fail(g, DNNF_ERR_INVALID_ARG, "ConvTranspose takes (x, W)");
+    const std::vector<int64_t> xd = G.tensors[in_ids[0]].dims, wd = G.tensors[in_ids[1]].dims;
+    const int64_t k = at.kernel;
+    if (xd.size() != 4 || wd.size() != 4 || k < 1 || wd[0] != xd[3] || wd[1] != k || wd[2] != k)
+      return fail(g, DNNF_ERR_SHAPE, "ConvTranspose: NHWC x [Cin,k,k,Cout] with stride = kernel = k");
+    if (at.stride != 1 && at.stride != k) return fail(g, DNNF_ERR_UNSUPPORTED_OP, "ConvTranspose: stride must equal the kernel size");
+    int cur = -1;
+    auto emit = [&](int kind, std::vector<int> ins, const Attrs& a) -> int {
+      Op o; o.id = (int)G.ops.size(); o.kind = kind; o.source_id = source; o.in = ins; o.at = a;
+      int r = infer_shapes(G, o, err);
+      if (r) return r;
+      cur = o.out[0];
+      G.ops.push_back(o);
+      return DNNF_OK;
+    };
+    Attrs a1, a2, a3, a4, a5;
+    a1.shape = {wd[0], k * k * wd[3]};
+    rc = emit(DNNF_OP_RESHAPE, {in_ids[1]}, a1);
+    if (!rc) rc = emit(DNNF_OP_CONV1X1, {in_ids[0], cur}, a2);
+    a3.shape = {xd[0], xd[1], xd[2], k, k, wd[3]}; a4.perm = {0, 1, 3, 2, 4, 5}; a5.shape = {xd[0], xd[1] * k, xd[2] * k, wd[3]};
+    if (!rc) rc = emit(DNNF_OP_RESHAPE, {cur}, a3);
+    if (!rc) rc = emit(DNNF_OP_TRANSPOSE, {cur}, a4);
+    if (!rc) rc = emit(DNNF_OP_RESHAPE, {cur}, a5);
+    if (rc) { rollback(); G.err = err; return rc; }
+    outs = {cur};
   } else if (op_kind == DNNF_OP_DEPTHTOSPACE || op_kind == DNNF_OP_SPACETODEPTH || op_kind == DNNF_OP_RESIZE) {
     // Index maps of an NHWC tensor, recorded as the Reorganize / Shuffle / One-to-Many operators they consist of.
     const Tensor& X = G.tensors[in_ids[0]];

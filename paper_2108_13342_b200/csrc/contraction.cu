@@ -39,6 +39,9 @@ int conv1x1_direct_launch(const Launch& L, cudaStream_t st);
 int lower_dwconv(const Graph& g, const std::vector<int>& ops, int anchor, Block& out, std::string& why);
 int dwconv_launch(const Launch& L, void* status_words, int block_index, cudaStream_t st);
 void dwconv_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
+int lower_gather(const Graph& g, const std::vector<int>& ops, int anchor, Block& out, std::string& why);
+int gather_launch(const Launch& L, cudaStream_t st);
+void gather_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
 int lower_pool(const Graph& g, const std::vector<int>& ops, int anchor, Block& out, std::string& why);
 int pool_launch(const Launch& L, void* ws_base, cudaStream_t st);
 void pool_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
@@ -256,6 +259,7 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
   const Op& A = g.ops[anchor];
   if (A.kind == DNNF_OP_DWCONV3X3) return lower_dwconv(g, ops, anchor, out, why);
   if (A.kind == DNNF_OP_MAXPOOL || A.kind == DNNF_OP_AVGPOOL) return lower_pool(g, ops, anchor, out, why);
+  if (A.kind == DNNF_OP_GATHER) return lower_gather(g, ops, anchor, out, why);
   std::set<int> in_block(ops.begin(), ops.end());
   const Tensor& C = g.tensors[A.out[0]];
   const Tensor& TA = g.tensors[A.in[0]];
@@ -479,6 +483,7 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
 void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op, std::string& err) {
   if (L.family == DNNF_FAMILY_DWCONV) { dwconv_patch(L, ip, op); return; }
   if (L.family == DNNF_FAMILY_POOL) { pool_patch(L, ip, op); return; }
+  if (L.family == DNNF_FAMILY_GATHER) { gather_patch(L, ip, op); return; }
   GemmParams& gp = gp_of(L);
   bool changed = gp.A.ptr != ip[0] || gp.B.ptr != ip[1];
   gp.A.ptr = ip[0]; gp.B.ptr = ip[1];
@@ -497,6 +502,7 @@ void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vecto
 }
 
 int launch_contraction(const Launch& L, void* status_words, int block_index, cudaStream_t st, std::string& err) {
+  if (L.family == DNNF_FAMILY_GATHER) { int rc = gather_launch(L, st); if (rc) err = "gather launch failed"; return rc; }
   if (L.family == DNNF_FAMILY_POOL) { int rc = pool_launch(L, status_words, st); if (rc) err = "pooling launch failed"; return rc; }
   if (L.family == DNNF_FAMILY_DWCONV) { int rc = dwconv_launch(L, status_words, block_index, st); if (rc) err = "depthwise convolution launch failed"; return rc; }
   if (L.variant == 2) { int rc = conv1x1_direct_launch(L, st); if (rc) err = "pointwise convolution launch failed"; return rc; }

@@ -60,7 +60,7 @@ const char* op_name(int k) {
     "Sqrt", "Abs", "Neg", "Recip", "Square", "Relu", "Clip", "Pow", "Gelu", "ScaleShift", "Transpose", "Reshape",
     "Flatten", "Squeeze", "Unsqueeze", "Split", "Slice", "MatMul", "Conv1x1", "DwConv3x3", "Softmax", "LayerNorm",
     "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift", "DepthToSpace", "SpaceToDepth", "Resize", "Concat", "MaxPool", "AveragePool", "Sin", "Cos", "Asin", "Ceil", "Floor",
-    "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConcatPart"};
+    "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConvTranspose", "Gather", "ConcatPart"};
   if (k <= 0 || k >= DNNF_OP__COUNT) return "?";
   return names[k];
 }
@@ -79,7 +79,8 @@ bool is_row_anchor(int k) {
   return k == DNNF_OP_SOFTMAX || k == DNNF_OP_LAYERNORM || (k >= DNNF_OP_REDUCESUM && k <= DNNF_OP_REDUCEPROD);
 }
 bool is_contraction(int k) {      // anchors that take an epilogue chain and nothing in front
-  return k == DNNF_OP_MATMUL || k == DNNF_OP_CONV1X1 || k == DNNF_OP_DWCONV3X3 || k == DNNF_OP_MAXPOOL || k == DNNF_OP_AVGPOOL;
+  return k == DNNF_OP_MATMUL || k == DNNF_OP_CONV1X1 || k == DNNF_OP_DWCONV3X3 || k == DNNF_OP_MAXPOOL || k == DNNF_OP_AVGPOOL ||
+         k == DNNF_OP_GATHER;
 }
 
 // Associative / commutative / distributive flags (Section 3.2).  Operators with
@@ -129,7 +130,7 @@ int node_mapping(const Graph& g, const Op& op) {
     case DNNF_OP_TRANSPOSE: return DNNF_SHUFFLE;
     case DNNF_OP_RESHAPE: case DNNF_OP_FLATTEN: case DNNF_OP_SQUEEZE: case DNNF_OP_UNSQUEEZE: return DNNF_REORGANIZE;
     case DNNF_OP_SPLIT: case DNNF_OP_SLICE: case DNNF_OP_CONCAT: case DNNF_OP_CONCATPART: return DNNF_ONE_TO_ONE;
-    case DNNF_OP_EXPAND: return DNNF_ONE_TO_MANY;
+    case DNNF_OP_EXPAND: case DNNF_OP_GATHER: return DNNF_ONE_TO_MANY;
     case DNNF_OP_MATMUL: case DNNF_OP_CONV1X1: case DNNF_OP_DWCONV3X3: case DNNF_OP_SOFTMAX: case DNNF_OP_LAYERNORM:
     case DNNF_OP_REDUCESUM: case DNNF_OP_REDUCEMEAN: case DNNF_OP_REDUCEMAX: case DNNF_OP_REDUCEPROD:
     case DNNF_OP_MAXPOOL: case DNNF_OP_AVGPOOL:
@@ -278,6 +279,12 @@ int infer_shapes(Graph& g, Op& op, std::string& err) {
     auto d = in(0).dims;
     d[1] = (d[1] + 2 * pd - kk) / st + 1;
     d[2] = (d[2] + 2 * pd - kk) / st + 1;
+    outs.push_back(d);
+  } else if (k == DNNF_OP_GATHER) {
+    if (!need(2)) return DNNF_ERR_INVALID_ARG;
+    if (in(0).dims.size() != 2 || in(1).dtype != DNNF_F32 || in(1).dims.size() + 1 > (size_t)kMaxDims) { err = "Gather: table [V,D] and fp32 indices"; return DNNF_ERR_SHAPE; }
+    if (op.at.axis != 0 && op.at.axis != -2) { err = "Gather: axis 0 only"; return DNNF_ERR_UNSUPPORTED_OP; }
+    auto d = in(1).dims; d.push_back(in(0).dims[1]);
     outs.push_back(d);
   } else if (k == DNNF_OP_CONCATPART) {
     if (op.in.size() != 1 && op.in.size() != 2) { err = "ConcatPart: operand count"; return DNNF_ERR_INVALID_ARG; }

@@ -25,7 +25,7 @@ static const char* dtype_tag(int dt) { return dt == DNNF_BF16 ? "bf16" : "f32"; 
 std::string block_signature(const Graph& g, const Block& b) {
   const Launch& L = b.launch;
   std::ostringstream s;
-  static const char* fam[] = {"alias", "ew", "transpose", "row", "gemm", "conv1x1", "dwconv", "pool"};
+  static const char* fam[] = {"alias", "ew", "transpose", "row", "gemm", "conv1x1", "dwconv", "pool", "gather"};
   s << fam[L.family] << '|';
   std::vector<int> ops = b.ops;                 // canonical order: the same operator set gives the same signature
   std::sort(ops.begin(), ops.end());

@@ -211,3 +211,54 @@ def test_prelu_and_leakyrelu_in_a_convolution_epilogue(flags):
     s = check(W.Workload(g, ins), RTOL_F32, flags)
     if flags == B.PLAN_FUSED:
         assert s.plan_stats.n_kernels == 1, s.g.blocks()
+
+
+# ---- ConvTranspose (stride = kernel) and Gather ------------------------------------------------------------------
+
+@pytest.mark.parametrize("flags", PLANS)
+@pytest.mark.parametrize("shape,k,cout", [((2, 8, 8, 16), 2, 8), ((1, 5, 7, 12), 3, 4), ((3, 16, 16, 32), 2, 32)])
+def test_convtranspose_relu_concat(shape, k, cout, flags):
+    """The paper's ConvTranspose + ReLU + Concat example: the transposed convolution's epilogue spreads each pixel's
+    k x k cell over the result and stores it straight into the Concat."""
+    n, h, w, c = shape
+    g = graph("deconv")
+    g.ext("X", shape); g.ext("Wt", (c, k, k, cout), kind="weight"); g.ext("S", (n, h * k, w * k, 8))
+    t = g.add("Relu", [g.add("ConvTranspose", ["X", "Wt"], kernel=k)])
+    y = g.add("Concat", [t, "S"], axis=3)
+    g.mark_output(y)
+    ins = {"X": rnd(shape, 70), "Wt": rnd((c, k, k, cout), 71, -0.3, 0.3), "S": rnd((n, h * k, w * k, 8), 72)}
+    s = check(W.Workload(g, ins), 2e-4, flags)
+    if flags == B.PLAN_FUSED and cout % 8 == 0:
+        assert s.plan_stats.n_kernels == 2, s.g.blocks()      # the convolution block and the copy of the external part
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("v,d,idx_shape", [(50, 64, (7, 9)), (11, 5, (33,)), (1000, 768, (4, 128)), (3, 8, (2, 2, 2))])
+def test_gather_rows(v, d, idx_shape, dtype):
+    g = graph("gather")
+    g.ext("T", (v, d), dtype); g.ext("I", idx_shape); g.ext("P", idx_shape[-1:] + (d,), dtype)
+    e = g.add("Gather", ["T", "I"], axis=0)
+    g.mark_output(e)
+    g.mark_output(g.add("Add", [e, "P"]))                        # an embedding lookup plus a position table
+    idx = np.floor(W.uniform(777, 80, idx_shape, 0.0, float(v))).clip(0, v - 1)
+    tab = rnd((v, d), 81); pos = rnd(idx_shape[-1:] + (d,), 82)
+    if dtype == "bf16":
+        tab, pos = W.round_to_bf16(tab), W.round_to_bf16(pos)
+    s, got, ref = run_both(W.Workload(g, {"T": tab, "I": idx, "P": pos}), B.PLAN_FUSED)
+    names = list(g.outputs)
+    assert np.array_equal(got[names[0]].astype(np.float64), ref[names[0]])
+    close(got[names[1]], ref[names[1]], RTOL_F32 if dtype == "f32" else 1e-2)
+    assert [b["family"] for b in s.g.blocks()][0] == "gather"
+
+
+def test_gather_clamps_indices_outside_the_table():
+    g = graph("gather_clamp")
+    g.ext("T", (6, 12)); g.ext("I", (5,))
+    g.mark_output(g.add("Gather", ["T", "I"], axis=0))
+    tab = rnd((6, 12), 83)
+    from paper_2108_13342_b200.runtime import Session
+    s = Session(W.Workload(g, {"T": tab, "I": np.array([-3.0, 0.0, 5.0, 6.0, 1e9], dtype=np.float32)}))
+    s.run()
+    assert s.g.status()[0] == 0
+    got = s.output(g.outputs[0])
+    assert np.array_equal(got, tab[[0, 0, 5, 5, 5]].astype(np.float32))

@@ -518,3 +518,28 @@ def test_further_one_to_one_operators_type_and_fuse():
     G.plan(B.PLAN_FUSED)
     assert G.tensor_info(ids[ra])[1] == (1, 4, 4, 4) and G.tensor_info(ids[rb])[1] == (1, 7, 7, 4)
     assert len([x for x in G.blocks() if x["family"] == "pool"]) == 2
+
+
+def test_convtranspose_and_gather_recording_and_errors():
+    g = _desc(); g.ext("X", (2, 8, 8, 16)); g.ext("Wt", (16, 2, 2, 8), kind="weight"); g.ext("S", (2, 16, 16, 8))
+    t = g.add("Relu", [g.add("ConvTranspose", ["X", "Wt"], kernel=2)])
+    g.mark_output(g.add("Concat", [t, "S"], axis=3))
+    G, ids, st = _plan_desc(g)
+    assert st.n_ops == 3 and st.n_kernels == 2
+    assert ["Conv1x1", "Reshape", "Transpose", "Reshape", "Relu", "ConcatPart"] in [b["ops"] for b in G.blocks()]
+    assert G.tensor_info(ids[g.outputs[0]])[1] == (2, 16, 16, 16)
+    for wshape, at in [((16, 2, 3, 8), dict(kernel=2)), ((8, 2, 2, 8), dict(kernel=2)), ((16, 2, 2, 8), dict(kernel=2, stride=3))]:
+        g = _desc(); g.ext("X", (2, 8, 8, 16)); g.ext("Wt", wshape, kind="weight")
+        g.add("ConvTranspose", ["X", "Wt"], **at)
+        with pytest.raises(B.DnnfError):
+            _plan_desc(g)
+    g = _desc(); g.ext("T", (50, 64)); g.ext("I", (7, 9))
+    g.mark_output(g.add("Relu", [g.add("Gather", ["T", "I"], axis=0)]))
+    G, ids, st = _plan_desc(g)
+    assert [b["family"] for b in G.blocks()] == ["gather", "elementwise"]
+    assert G.blocks()[0]["mapping"] == "One-to-Many"
+    assert G.tensor_info(ids[g.outputs[0]])[1] == (7, 9, 64)
+    g = _desc(); g.ext("T", (50, 64)); g.ext("I", (7, 9))
+    g.add("Gather", ["T", "I"], axis=1)
+    with pytest.raises(B.DnnfError):
+        _plan_desc(g)

@@ -212,6 +212,21 @@ def test_depthtospace_spacetodepth_resize_index_loops():
 
 # ---- Many-to-Many --------------------------------------------------------------
 
+def test_convtranspose_bruteforce_and_pointwise_case():
+    """Scalar loops from the scatter definition, with overlapping patches too (stride < kernel); a 1x1 kernel at
+    stride 1 is the pointwise convolution."""
+    x = rnd((2, 3, 4, 3), 41); w = rnd((3, 2, 2, 5), 42)
+    for s in (2, 1):
+        y = O.op_convtranspose(x, w, s)
+        ref = np.zeros_like(y)
+        for n, h, ww, c, i, j, o in itertools.product(range(2), range(3), range(4), range(3), range(2), range(2), range(5)):
+            ref[n, h * s + i, ww * s + j, o] += x[n, h, ww, c] * w[c, i, j, o]
+        assert y.shape == (2, (3 - 1) * s + 2, (4 - 1) * s + 2, 5)
+        assert np.max(np.abs(y - ref)) < 1e-14
+    w1 = rnd((3, 1, 1, 5), 43)
+    assert np.allclose(O.op_convtranspose(x, w1, 1), O.op_conv1x1(x, w1[:, 0, 0, :]), atol=1e-14)
+
+
 def test_pooling_bruteforce_and_special_cases():
     """Scalar loops from the definition (window clipped to the image; the mean counts only elements inside it);
     a global average pool is the mean over the image; a 1x1 window is the identity; a constant image stays
