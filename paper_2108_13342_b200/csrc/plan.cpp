@@ -68,6 +68,31 @@ struct Planner {
     return true;
   }
 
+  // Convexity looks at one block.  Two convex blocks can still need each other (a1 -> b1 and b2 -> a2 with b1, b2
+  // joined only through a common consumer), so the block graph itself has to stay acyclic: starting from the
+  // candidate block's successors and walking whole blocks at a time, no path may lead back into the candidate.
+  bool no_cycle(const std::vector<int>& members) const {
+    const int n = (int)g.ops.size();
+    std::vector<char> in(n, 0), seen(n, 0);
+    for (int m : members) in[m] = 1;
+    std::vector<int> stack;
+    auto visit = [&](int o) {
+      if (seen[o] || in[o]) return;
+      const int b = block_of[o];
+      if (b >= 0) { for (int x : blocks[b]) if (!seen[x] && !in[x]) { seen[x] = 1; stack.push_back(x); } }
+      if (!seen[o]) { seen[o] = 1; stack.push_back(o); }
+    };
+    for (int m : members) for (int s : successors(m)) visit(s);
+    while (!stack.empty()) {
+      int o = stack.back(); stack.pop_back();
+      for (int s : successors(o)) {
+        if (in[s]) return false;
+        visit(s);
+      }
+    }
+    return true;
+  }
+
   // Mapping type of `op` as met along the edge from `from` (Section 3.1 defines
   // types per input/output pair).  With STRICT_TABLE3 the node type is used.
   int type_along(int op, int from_tensor) const {
@@ -123,7 +148,7 @@ struct Planner {
   // threshold" (register pressure etc.) becomes: the merged block must lower
   // to one kernel within the register / argument / program-length budgets.
   bool check_constraint(const std::vector<int>& merged) {
-    if (!convex(merged)) return false;
+    if (!convex(merged) || !no_cycle(merged)) return false;
     int anchors = 0;
     for (int m : merged) if (g.ops[m].mapping == DNNF_MANY_TO_MANY) anchors++;
     if (anchors > 1) return false;
@@ -212,7 +237,7 @@ struct Planner {
           if (tb == bi) continue;
           std::vector<int> merged = blocks[tb];
           merged.push_back(o);
-          if (!convex(merged)) continue;
+          if (!convex(merged) || !no_cycle(merged)) continue;
           Block m, a, b;
           if (!lowers(merged, &m)) continue;
           if (lowers(blocks[tb], &a) && lowers({o}, &b) && cost(m) > cost(a) + cost(b)) continue;
@@ -252,7 +277,7 @@ struct Planner {
         std::vector<int> xs, ys = blocks[y];
         for (int m : blocks[x]) if (m != o) xs.push_back(m);
         ys.push_back(o);
-        if (!convex(ys) || (!xs.empty() && !convex(xs))) continue;
+        if (!convex(ys) || (!xs.empty() && !convex(xs)) || !no_cycle(ys)) continue;
         double before = cost_of(blocks[x]) + cost_of(blocks[y]);
         double after = cost_of(xs) + cost_of(ys);
         if (after >= 1e30 || after > before) continue;

@@ -100,6 +100,7 @@ struct Rewriter {
     for (int oid : g.topo_order()) {
       Op& o = g.ops[oid];
       if (o.out.size() != 1 || g.tensors[o.out[0]].is_output) continue;
+      if (o.kind == DNNF_OP_CONCATPART) continue;      // a part extends its Concat's result in place: not a value of its own
       std::string key = std::to_string(o.kind) + ":";
       std::vector<int> ins = o.in;
       if ((o.kind == DNNF_OP_ADD || o.kind == DNNF_OP_MUL) && ins.size() == 2 && ins[0] > ins[1]) std::swap(ins[0], ins[1]);

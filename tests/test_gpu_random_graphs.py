@@ -207,7 +207,8 @@ def test_random_graph(seed):
             B.profile_db_clear()
 
 
-@pytest.mark.parametrize("seed", [pytest.param(i, id=str(i)) for i in range(120)] + [pytest.param(-i - 1, id="big%d" % i) for i in range(30)])
+@pytest.mark.parametrize("seed", [pytest.param(i, id=str(i)) for i in list(range(120)) + [2334]]     # 2334: two convex blocks that needed each other
+                         + [pytest.param(-i - 1, id="big%d" % i) for i in range(30)])
 def test_random_graph_with_concat(seed):
     """The same generator with Concat among the operators: parts stored by producer blocks of every family,
     results read through views, nested and repeated inputs."""
@@ -227,6 +228,121 @@ def test_random_graph_with_concat(seed):
                 close(got, ref[n], 2e-4 if seed < 0 else 2e-5)
             except AssertionError as e:
                 raise AssertionError(f"{n} plan {[b['ops'] for b in s.g.blocks()]}: {e}") from None
+
+
+def _build_cnn(seed):
+    """Random NHWC fp32 graphs over the convolution-side operators: pointwise / depthwise / transposed convolutions with
+    folded-BN epilogues, pooling, SpaceToDepth / DepthToSpace, Resize, channel and spatial Concat, residual adds."""
+    r = _Rng(seed)
+    n, hw, c = r.pick([1, 2, 3]), r.pick([4, 8, 12, 16]), r.pick([4, 8, 16, 24])
+    g = graph("cnn%d" % seed)
+    ins = {}
+    g.ext("X", (n, hw, hw, c)); ins["X"] = W.uniform(778, 1000 + seed, (n, hw, hw, c), -1.0, 1.0)
+    pool = [("X", (n, hw, hw, c))]
+    cnt = [0]
+
+    def ext(shape, lo, hi, kind="weight"):
+        cnt[0] += 1
+        name = "w%d" % cnt[0]
+        g.ext(name, shape, kind=kind); ins[name] = W.uniform(778, 3000 + 20 * seed + cnt[0], shape, lo, hi)
+        return name
+
+    def bn_act(t, ch):
+        t = g.add("ScaleShift", [t, ext((ch,), 0.5, 1.5), ext((ch,), -0.5, 0.5)], axis=-1)
+        act = r.pick(["clip", "relu", "leaky", "none", "sigmoid"])
+        if act == "clip": t = g.add("Clip", [t], lo=0.0, hi=6.0)
+        elif act == "relu": t = g.add("Relu", [t])
+        elif act == "leaky": t = g.add("LeakyRelu", [t], alpha=0.1)
+        elif act == "sigmoid": t = g.add("Sigmoid", [t])
+        return t
+
+    for _ in range(5 + int(r.u() * 8)):
+        t, shp = r.pick(pool[-3:]) if r.u() < 0.7 else r.pick(pool)
+        N, H, Wd, C = shp
+        kind = r.pick(["conv", "conv", "dw", "maxpool", "avgpool", "gap", "s2d", "d2s", "resize", "catc", "cath", "add", "deconv", "unary"])
+        if kind in ("dw", "maxpool", "avgpool", "gap") and C % 4:
+            continue                                  # these kernels move four channels per thread
+        if kind == "conv":
+            co = r.pick([4, 8, 16, 24, 32])
+            o = bn_act(g.add("Conv1x1", [t, ext((C, co), -0.4, 0.4)]), co); shp = (N, H, Wd, co)
+        elif kind == "dw":
+            o = bn_act(g.add("DwConv3x3", [t, ext((3, 3, C), -0.4, 0.4)]), C)
+        elif kind in ("maxpool", "avgpool"):
+            k, s_, p = r.pick([(2, 2, 0), (3, 2, 1), (3, 1, 1), (2, 1, 0)])
+            if H + 2 * p < k or Wd + 2 * p < k:
+                continue
+            o = g.add("MaxPool" if kind == "maxpool" else "AveragePool", [t], kernel=k, stride=s_, pad=p)
+            shp = (N, (H + 2 * p - k) // s_ + 1, (Wd + 2 * p - k) // s_ + 1, C)
+            if r.u() < 0.5:
+                o = bn_act(o, C)
+        elif kind == "gap":
+            if H != Wd or H < 2:
+                continue
+            o = g.add("AveragePool", [t], kernel=H, stride=1, pad=0)
+            gate = g.add("Sigmoid", [g.add("Conv1x1", [o, ext((C, C), -0.4, 0.4)])])
+            o = g.add("Mul", [t, gate])
+        elif kind == "s2d":
+            if H % 2 or Wd % 2 or C * 4 > 128:
+                continue
+            o = g.add("SpaceToDepth", [t], block=2); shp = (N, H // 2, Wd // 2, C * 4)
+        elif kind == "d2s":
+            if C % 4 or H * 2 > 48:
+                continue
+            o = g.add("DepthToSpace", [t], block=2); shp = (N, H * 2, Wd * 2, C // 4)
+        elif kind == "resize":
+            if H * 2 > 48:
+                continue
+            o = g.add("Resize", [t], scale=2); shp = (N, H * 2, Wd * 2, C)
+        elif kind in ("catc", "cath"):
+            ax = 3 if kind == "catc" else 1
+            cands = [p for p in pool if all(p[1][d] == shp[d] for d in range(4) if d != ax) and p[1][ax] + shp[ax] <= 160]
+            if not cands:
+                continue
+            other = r.pick(cands)
+            o = g.add("Concat", [t, other[0]], axis=ax)
+            shp = tuple(shp[d] + (other[1][d] if d == ax else 0) for d in range(4))
+        elif kind == "add":
+            cands = [p for p in pool if p[1] == shp and p[0] != t]
+            if not cands:
+                continue
+            o = g.add("Add", [t, r.pick(cands)[0]])
+        elif kind == "deconv":
+            if H * 2 > 48:
+                continue
+            co = r.pick([4, 8, 16])
+            o = bn_act(g.add("ConvTranspose", [t, ext((C, 2, 2, co), -0.4, 0.4)], kernel=2), co); shp = (N, H * 2, Wd * 2, co)
+        else:
+            o = g.add(r.pick(["Tanh", "Relu", "Abs", "Sin"]), [t])
+        pool.append((o, shp))
+    outs = {pool[-1][0]}
+    for _ in range(int(r.u() * 3)):
+        outs.add(r.pick(pool[1:])[0]) if len(pool) > 1 else None
+    for o in sorted(outs):
+        if o != "X":
+            g.mark_output(o)
+    if not g.outputs:
+        g.mark_output(g.add("Relu", ["X"]))
+    return W.Workload(g, ins)
+
+
+@pytest.mark.parametrize("seed", range(160))
+def test_random_cnn_graph(seed):
+    wl = _build_cnn(7000 + seed)
+    ref = O.run_graph(wl.graph, wl.inputs)
+    for flags, rewrite in ((B.PLAN_FUSED, B.REWRITE_NONE), (B.PLAN_UNFUSED, B.REWRITE_NONE), (B.PLAN_FUSED, B.REWRITE_DEFAULT)):
+        s = Session(wl, plan_flags=flags, rewrite_flags=rewrite)
+        s.workspace[s.g.workspace_zero_bytes():].fill_(0xFF)
+        for n in wl.graph.outputs:
+            s.buffers[n].fill_(float("nan"))
+        s.run()
+        assert s.g.status()[0] == 0
+        for n in wl.graph.outputs:
+            got = s.output(n)
+            assert np.isfinite(got).all(), (n, "unwritten elements", [b["ops"] for b in s.g.blocks()])
+            try:
+                close(got, ref[n], 1e-4)
+            except AssertionError as e:
+                raise AssertionError(f"{n} flags {flags} rewrite {rewrite} plan {[b['ops'] for b in s.g.blocks()]}: {e}") from None
 
 
 @pytest.mark.parametrize("seed", range(80))

@@ -107,6 +107,20 @@ def test_concat_is_exact_and_nests(flags):
     _exact(W.Workload(g, {"A": rnd((3, 4, 8), 20), "Bt": rnd((3, 2, 8), 21), "Ct": rnd((3, 6, 5), 22)}), flags)
 
 
+def test_identical_concats_survive_common_subexpression_elimination():
+    """Two Concats of the same inputs (and two that share a first input) under the rewriting pass: the parts fill their
+    own results in place and are never merged."""
+    g = graph("cat_cse")
+    g.ext("X", (3, 12, 12, 4))
+    a = g.add("DepthToSpace", ["X"], block=2)
+    b = g.add("Sin", [a])
+    c1 = g.add("Concat", [a, b], axis=3)
+    c2 = g.add("Concat", [a, a], axis=3)
+    c3 = g.add("Concat", [a, a], axis=3)
+    g.mark_output(c1); g.mark_output(c2); g.mark_output(g.add("Relu", [c3]))
+    check(W.Workload(g, {"X": rnd((3, 12, 12, 4), 25)}), RTOL_F32, B.PLAN_FUSED, B.REWRITE_DEFAULT)
+
+
 @pytest.mark.parametrize("flags", PLANS)
 def test_concat_fed_by_row_and_convolution_blocks(flags):
     g = graph("cat_blocks")
