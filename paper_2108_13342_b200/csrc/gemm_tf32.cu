@@ -562,8 +562,13 @@ DNNF_SP_BEGIN(FP_ScaleShiftResidual, 5)
   MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_ADD, S_IN, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
 DNNF_SP_BEGIN(FP_ScaleShiftClipResidual, 6)
   MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_CLIP, S_CONST, 0), MO(M_ADD, S_IN, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+// the later slices of a contraction that the planner split along K: the partial sum arrives as a residual
+DNNF_SP_BEGIN(FP_Residual, 3) MO(M_MOV, S_IN, 0), MO(M_ADD, S_ANCHOR, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(FP_ResidualScaleShiftClip, 6)
+  MO(M_MOV, S_IN, 0), MO(M_ADD, S_ANCHOR, 0), MO(M_MUL, S_IN, 1), MO(M_ADD, S_IN, 2), MO(M_CLIP, S_CONST, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
 #undef MO
-using Static = TypeList<FP_Store, FP_Bias, FP_ScaleShiftClip, FP_ScaleShiftResidual, FP_ScaleShiftClipResidual>;
+using Static = TypeList<FP_Store, FP_Bias, FP_ScaleShiftClip, FP_ScaleShiftResidual, FP_ScaleShiftClipResidual, FP_Residual,
+                        FP_ResidualScaleShiftClip>;
 
 }  // namespace tf32
 
@@ -577,25 +582,32 @@ static const tf32::Params& fp_of(const Launch& L) { return *reinterpret_cast<con
 size_t tf32_blob_bytes() { return sizeof(tf32::Params); }
 
 static int tf32_npad(int n) { return (n + 15) / 16 * 16; }
-static int tf32_b_bytes(const GemmParams& gp) { return 2 * tf32_npad(gp.N) * 128 * ((gp.K + tf32::BK - 1) / tf32::BK); }
+static int tf32_b_bytes_of(int N, int K) { return 2 * tf32_npad(N) * 128 * ((K + tf32::BK - 1) / tf32::BK); }
+static int tf32_b_bytes(const GemmParams& gp) { return tf32_b_bytes_of(gp.N, gp.K); }
 
-bool tf32_gemm_eligible(const GemmParams& gp) {
+// The part of the eligibility test that depends on the problem's shape alone (the planner asks it before it
+// splits a contraction that is too deep into several that fit).
+bool tf32_shape_fits(int64_t M, int64_t N, int64_t K) {
   if (getenv("DNNF_NO_TF32_GEMM")) return false;
-  if (gp.A.dtype != DNNF_F32 || gp.B.dtype != DNNF_F32) return false;
-  if (gp.batch_ext[0] * gp.batch_ext[1] != 1) return false;
-  if (gp.A.stride_col != 1 || gp.A.stride_row % 4 || gp.A.base % 4 || gp.A.stride_row <= 0) return false;
-  if (gp.K > 244) return false;                              // a whole row of A (padded) must fit one TMA box of 256 floats
-  if (gp.N > 192 || gp.M < 4 * tf32::BM) return false;       // two accumulator stages and two A stages must fit in 512 TMEM columns
-  if (tf32_b_bytes(gp) > tf32::kMaxBBytes) return false;
+  if (K < 1 || K > 244) return false;                        // a whole row of A (padded) must fit one TMA box of 256 floats
+  if (N < 1 || N > 192 || M < 4 * tf32::BM) return false;    // two accumulator stages and two A stages must fit in 512 TMEM columns
+  if (tf32_b_bytes_of((int)N, (int)K) > tf32::kMaxBBytes) return false;
   {   // tensor-memory budget (same arithmetic as the plan): never launch with fewer than two A stages
-    const int npad = tf32_npad(gp.N);
+    const int npad = tf32_npad((int)N);
     const bool dual = 4 * npad + 2 * tf32::kAStageCols <= 512;
     if ((512 - 2 * (dual ? 2 : 1) * npad) / tf32::kAStageCols < 2) return false;
   }
   // a whole tile of raw rows must be resident: the converter warps advance chunk by chunk together
-  const int kr = (gp.K + 3) / 4 * 4, pitch = kr + ((kr / 4) % 2 == 0 ? 4 : 8);
-  if ((tf32::kSmemMax - tf32::kFixed - tf32_b_bytes(gp)) / ((32 * pitch * 4 + 1023) / 1024 * 1024) < 4) return false;
+  const int kr = ((int)K + 3) / 4 * 4, pitch = kr + ((kr / 4) % 2 == 0 ? 4 : 8);
+  if ((tf32::kSmemMax - tf32::kFixed - tf32_b_bytes_of((int)N, (int)K)) / ((32 * pitch * 4 + 1023) / 1024 * 1024) < 4) return false;
   return true;
+}
+
+bool tf32_gemm_eligible(const GemmParams& gp) {
+  if (gp.A.dtype != DNNF_F32 || gp.B.dtype != DNNF_F32) return false;
+  if (gp.batch_ext[0] * gp.batch_ext[1] != 1) return false;
+  if (gp.A.stride_col != 1 || gp.A.stride_row % 4 || gp.A.base % 4 || gp.A.stride_row <= 0) return false;
+  return tf32_shape_fits(gp.M, gp.N, gp.K);
 }
 
 // The fast epilogue form: one dense fp32 output [M x N] (unit stride along n, rows 16-byte aligned),

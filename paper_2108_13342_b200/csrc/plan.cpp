@@ -352,8 +352,67 @@ double block_cost_us(const Graph& g, const Block& b) {
   return std::max(t_mem, t_cmp) + 2.0;
 }
 
+bool tf32_shape_fits(int64_t M, int64_t N, int64_t K);
+
+// An fp32 pointwise convolution too deep for the tensor-core kernel (its B images and a tile of whole A rows must
+// fit in shared memory) would run on the FMA pipes at a quarter of the speed.  It is split along K into 2-8
+// convolutions that fit, chained through Adds: sum_k = sum_{k < K/s} + ... .  The slices of x and W are views, the
+// Add joins the next slice's epilogue, so the cost is one extra write and read of the partial sum.  (A lowering
+// decision, not one of the paper's rewriting rules: it is applied to every plan, fused or not.)
+static void split_deep_pointwise(Graph& g) {
+  if (getenv("DNNF_NO_K_SPLIT")) return;
+  const size_t n_ops = g.ops.size();
+  bool any = false;
+  for (size_t oi = 0; oi < n_ops; ++oi) {
+    if (!g.ops[oi].alive || g.ops[oi].kind != DNNF_OP_CONV1X1) continue;
+    const int x = g.ops[oi].in[0], w = g.ops[oi].in[1], y = g.ops[oi].out[0];
+    if (g.tensors[x].dtype != DNNF_F32 || g.tensors[w].dtype != DNNF_F32) continue;
+    const int64_t K = g.tensors[w].dims[0], N = g.tensors[w].dims[1], M = g.tensors[x].numel() / K;
+    if (tf32_shape_fits(M, N, K)) continue;
+    int s = 0;
+    for (int c : {2, 3, 4, 5, 6, 8}) if (K % (4 * c) == 0 && tf32_shape_fits(M, N, K / c)) { s = c; break; }
+    if (!s) continue;
+    const int source = g.ops[oi].source_id;
+    auto add = [&](int kind, std::vector<int> in, const Attrs& at, int reuse_out) -> int {
+      Op o; o.id = (int)g.ops.size(); o.kind = kind; o.in = std::move(in); o.at = at; o.source_id = source;
+      std::string err;
+      const size_t nt = g.tensors.size();
+      if (infer_shapes(g, o, err) != DNNF_OK) { g.tensors.resize(nt); return -1; }
+      if (reuse_out >= 0) { g.tensors.resize(nt); o.out[0] = reuse_out; g.tensors[reuse_out].producer = o.id; }
+      o.mapping = node_mapping(g, o);
+      o.props = math_props(kind);
+      g.ops.push_back(o);
+      return o.out[0];
+    };
+    // as matrix products over [pixels, K]: a MatMul takes its operands through Slice / Reshape views
+    const int64_t ks = K / s;
+    Attrs r2; r2.shape = {M, K};
+    const int x2 = add(DNNF_OP_RESHAPE, {x}, r2, -1);
+    int acc = -1;
+    bool ok = x2 >= 0;
+    for (int i = 0; i < s && ok; ++i) {
+      Attrs ax, aw;
+      ax.axis = 1; ax.start = i * ks; ax.end = (i + 1) * ks;
+      aw.axis = 0; aw.start = i * ks; aw.end = (i + 1) * ks;
+      const int xs = add(DNNF_OP_SLICE, {x2}, ax, -1), ws = add(DNNF_OP_SLICE, {w}, aw, -1);
+      if (xs < 0 || ws < 0) { ok = false; break; }
+      const int c = add(DNNF_OP_MATMUL, {xs, ws}, Attrs{}, -1);
+      if (c < 0) { ok = false; break; }
+      acc = acc < 0 ? c : add(DNNF_OP_ADD, {c, acc}, Attrs{}, -1);
+      if (acc < 0) ok = false;
+    }
+    if (ok) {
+      Attrs r4; r4.shape = g.tensors[y].dims;
+      if (add(DNNF_OP_RESHAPE, {acc}, r4, y) < 0) ok = false;
+    }
+    if (ok) { g.ops[oi].alive = false; any = true; }
+  }
+  if (any) g.relink();
+}
+
 int plan_graph(Graph& g, uint32_t flags) {
   g.relink();
+  split_deep_pointwise(g);
   // Operators whose results nobody reads (not a graph output, no live consumer) are not planned: they would
   // form blocks without an output.  (The rewriting pass removes them as well; a graph planned without rewriting
   // may still carry some.)

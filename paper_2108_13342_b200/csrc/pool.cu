@@ -49,12 +49,30 @@ __global__ void __launch_bounds__(256) pool_kernel(const __grid_constant__ PoolP
   DwIO io{p.d};
   const float init = p.is_max ? -INFINITY : 0.0f;
   io.accv[0] = io.accv[1] = io.accv[2] = io.accv[3] = init;
-  for (int h = ha; h < hb; ++h) {
-    const float* row = xb + ((size_t)h * p.Wi) * p.d.C;
-    for (int w = wa; w < wb; ++w) {
-      const float4 v = __ldg(reinterpret_cast<const float4*>(row + (size_t)w * p.d.C));
-      if (p.is_max) { io.accv[0] = fmaxf(io.accv[0], v.x); io.accv[1] = fmaxf(io.accv[1], v.y); io.accv[2] = fmaxf(io.accv[2], v.z); io.accv[3] = fmaxf(io.accv[3], v.w); }
-      else { io.accv[0] += v.x; io.accv[1] += v.y; io.accv[2] += v.z; io.accv[3] += v.w; }
+  if (p.kernel <= 3) {
+    // up to nine loads, all issued before the first use (the window loop below would wait for each in turn)
+    float4 v[9];
+#pragma unroll
+    for (int dh = 0; dh < 3; ++dh)
+#pragma unroll
+      for (int dw = 0; dw < 3; ++dw) {
+        const int h = h0 + dh, w = w0 + dw;
+        const bool ok = dh < p.kernel && dw < p.kernel && h >= 0 && h < p.Hi && w >= 0 && w < p.Wi;
+        v[dh * 3 + dw] = ok ? __ldg(reinterpret_cast<const float4*>(xb + ((size_t)h * p.Wi + w) * p.d.C)) : make_float4(init, init, init, init);
+      }
+#pragma unroll
+    for (int e = 0; e < 9; ++e) {
+      if (p.is_max) { io.accv[0] = fmaxf(io.accv[0], v[e].x); io.accv[1] = fmaxf(io.accv[1], v[e].y); io.accv[2] = fmaxf(io.accv[2], v[e].z); io.accv[3] = fmaxf(io.accv[3], v[e].w); }
+      else { io.accv[0] += v[e].x; io.accv[1] += v[e].y; io.accv[2] += v[e].z; io.accv[3] += v[e].w; }
+    }
+  } else {
+    for (int h = ha; h < hb; ++h) {
+      const float* row = xb + ((size_t)h * p.Wi) * p.d.C;
+      for (int w = wa; w < wb; ++w) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(row + (size_t)w * p.d.C));
+        if (p.is_max) { io.accv[0] = fmaxf(io.accv[0], v.x); io.accv[1] = fmaxf(io.accv[1], v.y); io.accv[2] = fmaxf(io.accv[2], v.z); io.accv[3] = fmaxf(io.accv[3], v.w); }
+        else { io.accv[0] += v.x; io.accv[1] += v.y; io.accv[2] += v.z; io.accv[3] += v.w; }
+      }
     }
   }
   if (!p.is_max) {                                  // mean over the elements inside the image (padding is not counted)

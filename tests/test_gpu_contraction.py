@@ -285,3 +285,26 @@ def test_encoder_full_size_twelve_layers():
     rel = np.linalg.norm(got[name] - ref[name]) / np.linalg.norm(ref[name])
     assert rel < 2e-2, rel
     assert s.plan_stats.n_kernels == 108 and np.all(np.isfinite(got[name]))
+
+
+@pytest.mark.parametrize("flags", [B.PLAN_FUSED, B.PLAN_UNFUSED])
+@pytest.mark.parametrize("nhw,cin,cout,slices", [((2, 32, 32), 256, 64, 2), ((1, 40, 40), 384, 32, 2), ((1, 24, 24), 576, 48, 3),
+                                                  ((1, 24, 24), 960, 24, 4), ((2, 16, 16), 248, 40, 2)])
+def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, flags):
+    """fp32 pointwise convolutions deeper than the split-TF32 kernel takes (K > 244) are planned as 2-4 tensor-core
+    contractions over K slices (as few as fit the kernel's shared memory), the partial sums riding in a later slice's
+    epilogue."""
+    import os
+    n, h, w = nhw
+    g = graph("deep_pw")
+    g.ext("X", (n, h, w, cin)); g.ext("Wt", (cin, cout), kind="weight"); g.ext("s", (cout,)); g.ext("t", (cout,))
+    y = g.add("Clip", [g.add("ScaleShift", [g.add("Conv1x1", ["X", "Wt"]), "s", "t"], axis=-1)], lo=0.0, hi=6.0)
+    g.mark_output(y)
+    ins = {"X": rnd((n, h, w, cin), 90, 0.0, 1.0), "Wt": rnd((cin, cout), 91, -0.2, 0.2), "s": rnd((cout,), 92, 0.5, 1.5),
+           "t": rnd((cout,), 93, -0.5, 0.5)}
+    s = check(W.Workload(g, ins), 2e-5, flags)
+    if not (os.environ.get("DNNF_NO_K_SPLIT") or os.environ.get("DNNF_NO_TF32_GEMM")):
+        gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
+        assert len(gemms) >= slices and all(b["variant"] == 4 for b in gemms), s.g.blocks()
+        assert not [b for b in s.g.blocks() if b["family"] == "conv1x1"], s.g.blocks()
+        assert s.plan_stats.n_ops == 3          # the slices count as the one convolution they came from
