@@ -354,7 +354,7 @@ double block_cost_us(const Graph& g, const Block& b) {
 
 bool tf32_shape_fits(int64_t M, int64_t N, int64_t K);
 
-// An fp32 pointwise convolution too deep for the tensor-core kernel (its B images and a tile of whole A rows must
+// An fp32 pointwise convolution (or plain fp32 matrix product) too deep for the tensor-core kernel (its B images and a tile of whole A rows must
 // fit in shared memory) would run on the FMA pipes at a quarter of the speed.  It is split along K into 2-8
 // convolutions that fit, chained through Adds: sum_k = sum_{k < K/s} + ... .  The slices of x and W are views, the
 // Add joins the next slice's epilogue, so the cost is one extra write and read of the partial sum.  (A lowering
@@ -364,9 +364,10 @@ static void split_deep_pointwise(Graph& g) {
   const size_t n_ops = g.ops.size();
   bool any = false;
   for (size_t oi = 0; oi < n_ops; ++oi) {
-    if (!g.ops[oi].alive || g.ops[oi].kind != DNNF_OP_CONV1X1) continue;
+    if (!g.ops[oi].alive || (g.ops[oi].kind != DNNF_OP_CONV1X1 && g.ops[oi].kind != DNNF_OP_MATMUL)) continue;
     const int x = g.ops[oi].in[0], w = g.ops[oi].in[1], y = g.ops[oi].out[0];
     if (g.tensors[x].dtype != DNNF_F32 || g.tensors[w].dtype != DNNF_F32) continue;
+    if (g.ops[oi].kind == DNNF_OP_MATMUL && (g.tensors[x].dims.size() != 2 || g.tensors[w].dims.size() != 2)) continue;   // plain matrix products only
     const int64_t K = g.tensors[w].dims[0], N = g.tensors[w].dims[1], M = g.tensors[x].numel() / K;
     if (tf32_shape_fits(M, N, K)) continue;
     int s = 0;

@@ -308,3 +308,16 @@ def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, fla
         assert len(gemms) >= slices and all(b["variant"] == 4 for b in gemms), s.g.blocks()
         assert not [b for b in s.g.blocks() if b["family"] == "conv1x1"], s.g.blocks()
         assert s.plan_stats.n_ops == 3          # the slices count as the one convolution they came from
+
+
+@pytest.mark.parametrize("mnk", [(2048, 64, 512), (700, 100, 300), (4096, 16, 1024)])
+def test_deep_fp32_matrix_product_is_split_along_k(mnk):
+    import os
+    m, n, k = mnk
+    g = graph("deep_mm")
+    g.ext("A", (m, k)); g.ext("Bm", (k, n), kind="weight"); g.ext("b", (n,))
+    g.mark_output(g.add("Relu", [g.add("Add", [g.add("MatMul", ["A", "Bm"]), "b"])]))
+    s = check(W.Workload(g, {"A": rnd((m, k), 94, -1.0, 1.0), "Bm": rnd((k, n), 95, -0.2, 0.2), "b": rnd((n,), 96)}), 2e-5)
+    if not (os.environ.get("DNNF_NO_K_SPLIT") or os.environ.get("DNNF_NO_TF32_GEMM")):
+        gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
+        assert len(gemms) >= 2 and all(b["variant"] == 4 for b in gemms), s.g.blocks()
