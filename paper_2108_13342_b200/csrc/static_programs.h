@@ -41,6 +41,11 @@ DNNF_SP_BEGIN(SP_Sigmoid, 3) MO(M_MOV, S_IN, 0), MO(M_SIGMOID, S_NONE, 0), MO(M_
 DNNF_SP_BEGIN(SP_GeluErf, 3) MO(M_MOV, S_IN, 0), MO(M_GELU_ERF, S_NONE, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
 DNNF_SP_BEGIN(SP_ScaleShiftClip, 5)
   MO(M_MOV, S_IN, 0), MO(M_MUL, S_IN, 1), MO(M_ADD, S_IN, 2), MO(M_CLIP, S_CONST, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+// the same chains with the value stored twice (itself and through an index map: SpaceToDepth / DepthToSpace / a Concat part)
+DNNF_SP_BEGIN(SP_ScaleShiftClip2, 6)
+  MO(M_MOV, S_IN, 0), MO(M_MUL, S_IN, 1), MO(M_ADD, S_IN, 2), MO(M_CLIP, S_CONST, 0), MO(M_STORE, S_NONE, 0), MO(M_STORE, S_NONE, 1) DNNF_SP_END
+DNNF_SP_BEGIN(SP_SigmoidMul2, 5)
+  MO(M_MOV, S_IN, 0), MO(M_SIGMOID, S_NONE, 0), MO(M_MUL, S_IN, 1), MO(M_STORE, S_NONE, 0), MO(M_STORE, S_NONE, 1) DNNF_SP_END
 // x * 0.5 * (1 + erf(x / sqrt 2)) spelled as five primitive operators
 DNNF_SP_BEGIN(SP_GeluPrimitives, 8)
   MO(M_MOV, S_IN, 0), MO(M_SAVE, S_TMP, 0), MO(M_MUL, S_CONST, 0), MO(M_ERF, S_NONE, 0), MO(M_ADD, S_CONST, 1),
@@ -90,7 +95,7 @@ DNNF_SP_BEGIN(SP_BiasResidualStoreLayerNorm, 17)
 template <class... T> struct TypeList {};
 using EwStatic = TypeList<SP_Move, SP_BiasScaleSwish, SP_AddIn, SP_MulIn, SP_MulC, SP_Sigmoid, SP_GeluErf, SP_ScaleShiftClip,
                           SP_GeluPrimitives, SP_ScaleShift, SP_Clip, SP_AddC, SP_Erf, SP_GeluTanh, SP_SubIn, SP_DivIn, SP_Square, SP_Sqrt,
-                          SP_Relu>;
+                          SP_Relu, SP_ScaleShiftClip2, SP_SigmoidMul2>;
 using TrStatic = TypeList<SP_Move, SP_BiasScaleSwish>;
 using RowStatic = TypeList<SP_ScaleMaskSoftmax, SP_Softmax, SP_AddLayerNormGelu, SP_LayerNorm, SP_BiasResidualLayerNorm,
                            SP_BiasResidualStoreLayerNorm>;
