@@ -116,6 +116,28 @@ def test_random_depthwise_and_pointwise_conv(seed):
     _run(W.Workload(g, ins), RTOL_F32)
 
 
+@pytest.mark.parametrize("seed", range(60))
+def test_random_deep_pointwise_conv(seed):
+    """Channel counts beyond what the split-TF32 kernel takes in one pass (K up to 1024): the planner's K slices, with
+    slice counts 2-8 or none when K has no suitable divisor, and three kinds of epilogue."""
+    n = _pick(seed, 1, [1, 2, 3])
+    h = 8 + int(_u(seed, 2) * 40)
+    w = 8 + int(_u(seed, 3) * 40)
+    c = 4 * (62 + int(_u(seed, 4) * 195))             # 248 .. 1024
+    co = 4 * (1 + int(_u(seed, 6) * 47))              # 4 .. 188
+    g = graph()
+    g.ext("X", (n, h, w, c)); g.ext("Wp", (c, co)); g.ext("s", (co,)); g.ext("t", (co,)); g.ext("R", (n, h, w, co))
+    ins = {"X": rnd((n, h, w, c), 61, -1, 1), "Wp": rnd((c, co), 62, -0.1, 0.1), "s": rnd((co,), 63, 0.5, 1.5),
+           "t": rnd((co,), 64, -0.5, 0.5), "R": rnd((n, h, w, co), 65, -1, 1)}
+    y = g.add("Conv1x1", ["X", "Wp"])
+    kind = _pick(seed, 7, ["bias", "bn_clip", "bn_res", "plain"])
+    if kind == "bias": y = g.add("Add", [y, "t"])
+    elif kind == "bn_clip": y = g.add("Clip", [g.add("ScaleShift", [y, "s", "t"], axis=-1)], lo=-1.0, hi=1.0)
+    elif kind == "bn_res": y = g.add("Add", [g.add("ScaleShift", [y, "s", "t"], axis=-1), "R"])
+    g.mark_output(y)
+    _run(W.Workload(g, ins), 2e-5)
+
+
 @pytest.mark.parametrize("seed", range(40))
 def test_random_attention(seed):
     """Q, K, V sliced out of one packed [B, S, 3*H*D] tensor, heads split by Reshape + Transpose, scores scaled and
