@@ -543,3 +543,41 @@ def test_convtranspose_and_gather_recording_and_errors():
     g.add("Gather", ["T", "I"], axis=1)
     with pytest.raises(B.DnnfError):
         _plan_desc(g)
+
+
+def test_deep_pointwise_convolution_is_planned_as_k_slices():
+    g = _desc(); g.ext("X", (2, 32, 32, 256)); g.ext("Wt", (256, 64), kind="weight"); g.ext("s", (64,)); g.ext("t", (64,))
+    g.mark_output(g.add("Clip", [g.add("ScaleShift", [g.add("Conv1x1", ["X", "Wt"]), "s", "t"], axis=-1)], lo=0.0, hi=6.0))
+    G, ids, st = _plan_desc(g)
+    fams = [(b["family"], b["variant"]) for b in G.blocks() if b["family"] != "alias"]
+    assert fams == [("gemm", 4), ("gemm", 4)], G.blocks()
+    assert st.n_ops == 3 and st.n_kernels == 2                    # the slices count as the convolution they came from
+    assert G.blocks()[-1]["ops"][-3:] == ["ScaleShift", "Clip"][-3:] or "Clip" in G.blocks()[-1]["ops"]
+    assert "ADD anchor" in G.block_program(G.block_count() - 1)   # the partial sum rides in the last slice's epilogue
+    # shallow enough, too few rows for the tensor-core kernel, or bf16: left alone
+    for shape, wshape, dt in [((2, 32, 32, 240), (240, 24), "f32"), ((1, 8, 8, 256), (256, 64), "f32"), ((2, 32, 32, 256), (256, 64), "bf16")]:
+        g = _desc(); g.ext("X", shape, dt); g.ext("Wt", wshape, dt, kind="weight")
+        g.mark_output(g.add("Conv1x1", ["X", "Wt"]))
+        G, ids, st = _plan_desc(g)
+        assert st.n_kernels == 1, G.blocks()
+
+
+def test_blocks_that_would_need_each_other_are_not_formed():
+    """a1 -> b1 and b2 -> a2, with b1 and b2 joined only through their common consumer b3: {a1, a2} and {b1, b2, b3}
+    are each convex, together they would be a cycle of two blocks.  Whatever the planner merges, the blocks it
+    returns must admit a launch order (plan_graph reports an internal error otherwise)."""
+    for perm in range(4):
+        g = _desc(); g.ext("X", (64, 32)); g.ext("Y", (64, 32)); g.ext("ga", (32,)); g.ext("be", (32,))
+        a1 = g.add("Tanh", ["X"])
+        b2 = g.add("Sigmoid", ["Y"])
+        a2 = g.add("Mul", [a1, b2]) if perm & 1 else g.add("Add", [b2, a1])
+        b1 = g.add("Relu", [a1])
+        b3 = g.add("Sub", [b1, b2]) if perm & 2 else g.add("Mul", [b2, b1])
+        g.mark_output(g.add("LayerNorm", [a2, "ga", "be"], axis=-1, eps=1e-5))
+        g.mark_output(g.add("Softmax", [b3], axis=-1))
+        G, ids, st = _plan_desc(g)
+        order = {}
+        for i, b in enumerate(G.blocks()):
+            for o in b["ops"]:
+                order.setdefault(o, i)
+        assert st.n_kernels >= 2
