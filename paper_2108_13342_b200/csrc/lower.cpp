@@ -616,6 +616,22 @@ bool emit_program(LowerCtx& cx, int anchor_out, int max_tmp) {
   }
   if (E.fail) return false;
   if (cx.prog.n == 0) { cx.why = "empty program"; return false; }
+  // Number the external inputs in the order the program first reads them: the same chain then gives the same
+  // program whatever order its operators were declared in, and finds its compile-time table.
+  {
+    const int n_in = (int)cx.ins.size();
+    std::vector<int> map(n_in, -1);
+    int next = 0;
+    for (int i = 0; i < cx.prog.n; ++i) {
+      const MicroOp& m = cx.prog.ops[i];
+      if (m.src == S_IN && m.idx < n_in && map[m.idx] < 0) map[m.idx] = next++;
+    }
+    for (int k = 0; k < n_in; ++k) if (map[k] < 0) map[k] = next++;
+    std::vector<ExtArg> ins(n_in);
+    for (int k = 0; k < n_in; ++k) ins[map[k]] = cx.ins[k];
+    cx.ins.swap(ins);
+    for (int i = 0; i < cx.prog.n; ++i) if (cx.prog.ops[i].src == S_IN && cx.prog.ops[i].idx < n_in) cx.prog.ops[i].idx = (uint8_t)map[cx.prog.ops[i].idx];
+  }
   return true;
 }
 

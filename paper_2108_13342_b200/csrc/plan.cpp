@@ -342,7 +342,7 @@ double block_cost_us(const Graph& g, const Block& b) {
     bytes += nb * gp.M * gp.K * (gp.A.dtype ? 2 : 4) * ((gp.A.batch_stride[0] || gp.A.batch_stride[1] || nb == 1) ? 1.0 : 1.0 / nb);
     bytes += nb * gp.K * gp.N * (gp.B.dtype ? 2 : 4) * ((gp.B.batch_stride[0] || gp.B.batch_stride[1] || nb == 1) ? 1.0 : 1.0 / nb);
     for (size_t i = 2; i < L.in_tensors.size(); ++i) add(L.in_tensors[i], 0);
-    for (int t : L.out_tensors) add(t, 0);
+    for (int t : L.out_tensors) add(t, 0, true);
   } else {
     for (int t : b.inputs) add(t, 0);
     for (int t : b.outputs) add(t, 0, true);
@@ -353,6 +353,18 @@ double block_cost_us(const Graph& g, const Block& b) {
 }
 
 bool tf32_shape_fits(int64_t M, int64_t N, int64_t K);
+
+// Whether a split into parts x slices tensor-core kernels beats the tiled FMA kernel the contraction would otherwise
+// run on.  Both sides are rough models fitted to measurements on this GPU: the FMA kernels reach about 10 TFLOP/s
+// on such shapes; a split kernel costs about 9 us of launch, setup and tail, every part reads A again, every slice
+// but the last writes a partial sum that a later one reads.
+static bool split_pays(int64_t M, int64_t N, int64_t K, int64_t parts, int64_t slices) {
+  if (getenv("DNNF_SPLIT_ALWAYS")) return true;      // development switch: the tests use it to reach the split at small sizes
+  const double unsplit_us = 2.0 * (double)M * (double)N * (double)K / 1e7;
+  const double bytes = 4.0 * (double)M * ((double)parts * (double)K + (double)N * (1.0 + 2.0 * (double)(slices - 1)));
+  const double split_us = 9.0 * (double)(parts * slices) + bytes / 4e6;
+  return split_us < unsplit_us;
+}
 
 // An fp32 pointwise convolution (or plain fp32 matrix product) too deep for the tensor-core kernel (its B images and a tile of whole A rows must
 // fit in shared memory) would run on the FMA pipes at a quarter of the speed.  It is split along K into 2-8
@@ -372,7 +384,7 @@ static void split_deep_pointwise(Graph& g) {
     if (tf32_shape_fits(M, N, K)) continue;
     int s = 0;
     for (int c : {2, 3, 4, 5, 6, 8}) if (K % (4 * c) == 0 && tf32_shape_fits(M, N, K / c)) { s = c; break; }
-    if (!s) continue;
+    if (!s || !split_pays(M, N, K, 1, s)) continue;
     const int source = g.ops[oi].source_id;
     auto add = [&](int kind, std::vector<int> in, const Attrs& at, int reuse_out) -> int {
       Op o; o.id = (int)g.ops.size(); o.kind = kind; o.in = std::move(in); o.at = at; o.source_id = source;
@@ -387,6 +399,13 @@ static void split_deep_pointwise(Graph& g) {
     };
     // as matrix products over [pixels, K]: a MatMul takes its operands through Slice / Reshape views
     const int64_t ks = K / s;
+    int wcol = -1; int64_t wc0 = 0, wc1 = 0;
+    {
+      const int pw = g.tensors[w].producer;
+      if (pw >= 0 && g.ops[pw].alive && g.ops[pw].kind == DNNF_OP_SLICE && g.ops[pw].at.axis == 1 && g.tensors[g.ops[pw].in[0]].dims.size() == 2) {
+        wcol = g.ops[pw].in[0]; wc0 = g.ops[pw].at.start; wc1 = g.ops[pw].at.end;
+      }
+    }
     Attrs r2; r2.shape = {M, K};
     const int x2 = add(DNNF_OP_RESHAPE, {x}, r2, -1);
     int acc = -1;
@@ -395,7 +414,15 @@ static void split_deep_pointwise(Graph& g) {
       Attrs ax, aw;
       ax.axis = 1; ax.start = i * ks; ax.end = (i + 1) * ks;
       aw.axis = 0; aw.start = i * ks; aw.end = (i + 1) * ks;
-      const int xs = add(DNNF_OP_SLICE, {x2}, ax, -1), ws = add(DNNF_OP_SLICE, {w}, aw, -1);
+      int ws;
+      if (wcol >= 0) {                       // W is itself a column block of a wider matrix: rows first, then the columns
+        Attrs ac; ac.axis = 1; ac.start = wc0; ac.end = wc1;
+        const int wr = add(DNNF_OP_SLICE, {wcol}, aw, -1);
+        ws = wr < 0 ? -1 : add(DNNF_OP_SLICE, {wr}, ac, -1);
+      } else {
+        ws = add(DNNF_OP_SLICE, {w}, aw, -1);
+      }
+      const int xs = add(DNNF_OP_SLICE, {x2}, ax, -1);
       if (xs < 0 || ws < 0) { ok = false; break; }
       const int c = add(DNNF_OP_MATMUL, {xs, ws}, Attrs{}, -1);
       if (c < 0) { ok = false; break; }
@@ -411,8 +438,137 @@ static void split_deep_pointwise(Graph& g) {
   if (any) g.relink();
 }
 
+// An fp32 pointwise convolution with more output channels than the tensor-core kernel's accumulators hold (N > 192),
+// or whose B images do not fit its shared memory at any depth the K split can reach, becomes several convolutions over column blocks of W whose results are the parts of a Concat along the channel
+// axis.  The One-to-One operators that follow the convolution and work channel by channel (folded BN, activations,
+// bias, a residual of the same shape) are applied per part, with Slice views of their vector / tensor operands, so that
+// they stay in the convolutions' epilogues and each part is stored straight into the result.  The part width is the one
+// that needs the fewest kernels once the K split below has been applied to the parts as well (at most 32; every part
+// reads x again, but the tiled FMA kernel such a convolution would otherwise run on is slower by an order of magnitude).
+static void split_wide_pointwise(Graph& g) {
+  if (getenv("DNNF_NO_N_SPLIT") || getenv("DNNF_NO_TF32_GEMM")) return;
+  g.relink();
+  const size_t n_ops = g.ops.size();
+  bool any = false;
+  for (size_t oi = 0; oi < n_ops; ++oi) {
+    if (!g.ops[oi].alive || g.ops[oi].kind != DNNF_OP_CONV1X1) continue;
+    const int x = g.ops[oi].in[0], w = g.ops[oi].in[1], y = g.ops[oi].out[0];
+    if (g.tensors[x].dtype != DNNF_F32 || g.tensors[w].dtype != DNNF_F32) continue;
+    const int64_t K = g.tensors[w].dims[0], N = g.tensors[w].dims[1], M = g.tensors[x].numel() / K;
+    if (M < 512 || N % 4 || tf32_shape_fits(M, N, K)) continue;
+    // the widest part (a multiple of 16 columns) that the kernel takes at this depth; every part reads x again, so
+    // only splits into a few parts are worth it (deeper or wider problems stay with the FMA kernel)
+    int64_t nw = 0, best = 1 << 30;
+    for (int64_t c = std::min<int64_t>(192, (N + 15) / 16 * 16); c >= 48; c -= 16)
+      for (int sl : {1, 2, 3, 4, 5, 6, 8}) {
+        if (K % (4 * sl) || !tf32_shape_fits(M, c, K / sl)) continue;
+        const int64_t kernels = (N + c - 1) / c * sl;
+        if (kernels < best) { best = kernels; nw = c; }
+        break;                                                              // more slices at this width only cost more
+      }
+    if (!nw || best > 32) continue;
+    const int64_t parts = (N + nw - 1) / nw;
+    if (parts == 1) continue;                                              // the K split alone does it
+    if (!split_pays(M, N, K, parts, best / parts)) continue;
+    nw = ((N + parts - 1) / parts + 15) / 16 * 16;                        // even the parts out
+    const std::vector<int64_t> ydims = g.tensors[y].dims;
+    // the chain of channel-wise operators behind the convolution
+    struct Link { int op; int other; int other_kind; };                   // other_kind: 0 none, 1 vector [N], 2 tensor like y; ScaleShift: two vectors
+    std::vector<Link> chain;
+    int t = y;
+    for (;;) {
+      const Tensor& T = g.tensors[t];
+      if (T.is_output || T.consumers.size() != 1) break;
+      const Op& c = g.ops[T.consumers[0]];
+      if (!c.alive || c.out.size() != 1 || g.tensors[c.out[0]].dims != ydims) break;
+      Link l{c.id, -1, 0};
+      if (c.kind == DNNF_OP_SCALESHIFT) {
+        if (c.in[0] != t || (c.at.axis != 3 && c.at.axis != -1)) break;
+      } else if (is_binary_elementwise(c.kind)) {
+        if (c.in[0] == c.in[1]) break;
+        const int o = c.in[0] == t ? c.in[1] : c.in[0];
+        const Tensor& O = g.tensors[o];
+        if (O.dims == std::vector<int64_t>{N}) l.other_kind = 1;
+        else if (O.dims == ydims) l.other_kind = 2;
+        else break;
+        l.other = o;
+      } else if (!(is_elementwise(c.kind) && c.in.size() == 1)) {
+        break;
+      }
+      chain.push_back(l);
+      t = c.out[0];
+    }
+    const int result = t;                                                  // the tensor the Concat will write
+    const int source = g.ops[oi].source_id;
+    auto add = [&](int kind, std::vector<int> in, const Attrs& at, int src_id, int reuse_out) -> int {
+      Op o; o.id = (int)g.ops.size(); o.kind = kind; o.in = std::move(in); o.at = at; o.source_id = src_id;
+      std::string err;
+      const size_t nt = g.tensors.size();
+      if (infer_shapes(g, o, err) != DNNF_OK) { g.tensors.resize(nt); return -1; }
+      if (reuse_out >= 0) { g.tensors.resize(nt); o.out[0] = reuse_out; g.tensors[reuse_out].producer = o.id; }
+      o.mapping = node_mapping(g, o);
+      o.props = math_props(kind);
+      g.ops.push_back(o);
+      return o.out[0];
+    };
+    auto slice = [&](int tensor, int axis, int64_t a, int64_t b, int src_id) {
+      Attrs at; at.axis = axis; at.start = a; at.end = b;
+      return add(DNNF_OP_SLICE, {tensor}, at, src_id, -1);
+    };
+    Attrs r2; r2.shape = {M, K};
+    const int x2 = add(DNNF_OP_RESHAPE, {x}, r2, source, -1);
+    bool ok = x2 >= 0;
+    int carrier = -1;
+    for (int64_t n0 = 0; n0 < N && ok; n0 += nw) {
+      const int64_t n1 = std::min(N, n0 + nw);
+      const int wj = slice(w, 1, n0, n1, source);
+      if (wj < 0) { ok = false; break; }
+      int v = add(DNNF_OP_MATMUL, {x2, wj}, Attrs{}, source, -1);
+      if (v < 0) { ok = false; break; }
+      Attrs r4; r4.shape = ydims; r4.shape[3] = n1 - n0;
+      v = add(DNNF_OP_RESHAPE, {v}, r4, source, -1);
+      for (const Link& l : chain) {
+        if (v < 0) break;
+        const Op c = g.ops[l.op];                                          // copy: g.ops grows below
+        if (c.kind == DNNF_OP_SCALESHIFT) {
+          const int sc = slice(c.in[1], 0, n0, n1, c.source_id), sh = slice(c.in[2], 0, n0, n1, c.source_id);
+          Attrs at = c.at; at.axis = 3;
+          v = (sc < 0 || sh < 0) ? -1 : add(c.kind, {v, sc, sh}, at, c.source_id, -1);
+        } else if (l.other_kind) {
+          const int o = slice(l.other, l.other_kind == 1 ? 0 : 3, n0, n1, c.source_id);
+          if (o < 0) { v = -1; break; }
+          std::vector<int> in = c.in[0] == l.other ? std::vector<int>{o, v} : std::vector<int>{v, o};
+          v = add(c.kind, in, c.at, c.source_id, -1);
+        } else {
+          v = add(c.kind, {v}, c.at, c.source_id, -1);
+        }
+      }
+      if (v < 0) { ok = false; break; }
+      Op part; part.id = (int)g.ops.size(); part.kind = DNNF_OP_CONCATPART; part.source_id = source;
+      part.in = {v};
+      if (carrier >= 0) part.in.push_back(carrier);
+      part.at.axis = 3; part.at.start = n0; part.at.shape = ydims;
+      std::string err;
+      const size_t nt = g.tensors.size();
+      if (infer_shapes(g, part, err) != DNNF_OK) { g.tensors.resize(nt); ok = false; break; }
+      if (n1 == N) { g.tensors.resize(nt); part.out[0] = result; g.tensors[result].producer = part.id; }
+      part.mapping = node_mapping(g, part);
+      part.props = 0;
+      carrier = part.out[0];
+      g.ops.push_back(part);
+    }
+    if (!ok) continue;                       // what was added stays unused and is dropped as dead code below
+    g.ops[oi].alive = false;
+    for (const Link& l : chain) g.ops[l.op].alive = false;
+    any = true;
+    g.relink();
+  }
+  if (any) g.relink();
+}
+
 int plan_graph(Graph& g, uint32_t flags) {
   g.relink();
+  split_wide_pointwise(g);
   split_deep_pointwise(g);
   // Operators whose results nobody reads (not a graph output, no live consumer) are not planned: they would
   // form blocks without an output.  (The rewriting pass removes them as well; a graph planned without rewriting

@@ -290,11 +290,12 @@ def test_encoder_full_size_twelve_layers():
 @pytest.mark.parametrize("flags", [B.PLAN_FUSED, B.PLAN_UNFUSED])
 @pytest.mark.parametrize("nhw,cin,cout,slices", [((2, 32, 32), 256, 64, 2), ((1, 40, 40), 384, 32, 2), ((1, 24, 24), 576, 48, 3),
                                                   ((1, 24, 24), 960, 24, 4), ((2, 16, 16), 248, 40, 2)])
-def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, flags):
+def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, flags, monkeypatch):
     """fp32 pointwise convolutions deeper than the split-TF32 kernel takes (K > 244) are planned as 2-4 tensor-core
     contractions over K slices (as few as fit the kernel's shared memory), the partial sums riding in a later slice's
     epilogue."""
     import os
+    monkeypatch.setenv("DNNF_SPLIT_ALWAYS", "1")       # the sizes here are below the planner's break-even
     n, h, w = nhw
     g = graph("deep_pw")
     g.ext("X", (n, h, w, cin)); g.ext("Wt", (cin, cout), kind="weight"); g.ext("s", (cout,)); g.ext("t", (cout,))
@@ -311,8 +312,9 @@ def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, fla
 
 
 @pytest.mark.parametrize("mnk", [(2048, 64, 512), (700, 100, 300), (4096, 16, 1024)])
-def test_deep_fp32_matrix_product_is_split_along_k(mnk):
+def test_deep_fp32_matrix_product_is_split_along_k(mnk, monkeypatch):
     import os
+    monkeypatch.setenv("DNNF_SPLIT_ALWAYS", "1")
     m, n, k = mnk
     g = graph("deep_mm")
     g.ext("A", (m, k)); g.ext("Bm", (k, n), kind="weight"); g.ext("b", (n,))
@@ -321,3 +323,54 @@ def test_deep_fp32_matrix_product_is_split_along_k(mnk):
     if not (os.environ.get("DNNF_NO_K_SPLIT") or os.environ.get("DNNF_NO_TF32_GEMM")):
         gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
         assert len(gemms) >= 2 and all(b["variant"] == 4 for b in gemms), s.g.blocks()
+
+
+@pytest.mark.parametrize("flags", [B.PLAN_FUSED, B.PLAN_UNFUSED])
+@pytest.mark.parametrize("nhw,cin,cout,tail", [((2, 32, 32), 64, 384, "bn_clip_res_relu"), ((1, 40, 40), 96, 200, "bn_clip"),
+                                               ((2, 24, 24), 32, 256, "none"), ((1, 32, 32), 24, 240, "bias_two_readers"),
+                                               ((3, 16, 16), 48, 512, "prelu")])
+def test_wide_pointwise_convolution_is_split_into_channel_blocks(nhw, cin, cout, tail, flags, monkeypatch):
+    """fp32 pointwise convolutions with more output channels than the split-TF32 kernel's accumulators hold (N > 192) are
+    planned as tensor-core contractions over column blocks of W; the channel-wise operators behind the convolution move
+    into each block's epilogue and the blocks store straight into the result (parts of a Concat)."""
+    import os
+    monkeypatch.setenv("DNNF_SPLIT_ALWAYS", "1")
+    n, h, w = nhw
+    g = graph("wide_pw")
+    g.ext("X", (n, h, w, cin)); g.ext("Wt", (cin, cout), kind="weight"); g.ext("s", (cout,)); g.ext("t", (cout,)); g.ext("R", (n, h, w, cout))
+    y = g.add("Conv1x1", ["X", "Wt"])
+    if tail == "bn_clip_res_relu":
+        y = g.add("Relu", [g.add("Add", [g.add("Clip", [g.add("ScaleShift", [y, "s", "t"], axis=-1)], lo=0.0, hi=6.0), "R"])])
+    elif tail == "bn_clip":
+        y = g.add("Clip", [g.add("ScaleShift", [y, "s", "t"], axis=-1)], lo=0.0, hi=6.0)
+    elif tail == "bias_two_readers":
+        y = g.add("Add", [y, "t"])
+        g.mark_output(g.add("Tanh", [y]))            # a second reader ends the chain that moves into the blocks
+        y = g.add("Sigmoid", [y])
+    elif tail == "prelu":
+        y = g.add("PRelu", [g.add("Sub", ["R", y]), "s"])
+    g.mark_output(y)
+    ins = {"X": rnd((n, h, w, cin), 97, 0.0, 1.0), "Wt": rnd((cin, cout), 98, -0.2, 0.2), "s": rnd((cout,), 99, 0.5, 1.5),
+           "t": rnd((cout,), 100, -0.5, 0.5), "R": rnd((n, h, w, cout), 101, -1.0, 1.0)}
+    s = check(W.Workload(g, ins), 2e-5, flags)
+    if not (os.environ.get("DNNF_NO_N_SPLIT") or os.environ.get("DNNF_NO_TF32_GEMM")):
+        gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
+        assert len(gemms) >= 2 and all(b["variant"] == 4 for b in gemms), s.g.blocks()
+        assert not [b for b in s.g.blocks() if b["family"] == "conv1x1"], s.g.blocks()
+        if flags == B.PLAN_FUSED and tail in ("bn_clip_res_relu", "bn_clip", "none", "prelu"):
+            assert s.plan_stats.n_kernels == len(gemms), s.g.blocks()      # nothing but the column blocks runs
+
+
+def test_split_decision_follows_the_cost_model():
+    """At 25088 pixels a 160 -> 960 convolution is worth 18 tensor-core kernels; a 576 -> 160 one at 6272 pixels is not
+    worth 12 (measured: 263 us against 675 us, and 123 us against 111 us)."""
+    for (n, hw, cin, cout), split in [((32, 28, 160, 960), True), ((32, 14, 576, 160), False)]:
+        g = graph("split_cost")
+        g.ext("X", (n, hw, hw, cin)); g.ext("Wt", (cin, cout), kind="weight")
+        g.mark_output(g.add("Conv1x1", ["X", "Wt"]))
+        from paper_2108_13342_b200.runtime import build_graph
+        G, ids = build_graph(g)
+        G.rewrite(B.REWRITE_NONE)
+        G.plan(B.PLAN_FUSED)
+        fams = {b["family"] for b in G.blocks()}
+        assert ("gemm" in fams) == split, G.blocks()

@@ -545,7 +545,8 @@ def test_convtranspose_and_gather_recording_and_errors():
         _plan_desc(g)
 
 
-def test_deep_pointwise_convolution_is_planned_as_k_slices():
+def test_deep_pointwise_convolution_is_planned_as_k_slices(monkeypatch):
+    monkeypatch.setenv("DNNF_SPLIT_ALWAYS", "1")       # below the planner's break-even size
     g = _desc(); g.ext("X", (2, 32, 32, 256)); g.ext("Wt", (256, 64), kind="weight"); g.ext("s", (64,)); g.ext("t", (64,))
     g.mark_output(g.add("Clip", [g.add("ScaleShift", [g.add("Conv1x1", ["X", "Wt"]), "s", "t"], axis=-1)], lo=0.0, hi=6.0))
     G, ids, st = _plan_desc(g)
