@@ -371,7 +371,7 @@ static bool split_pays(int64_t M, int64_t N, int64_t K, int64_t parts, int64_t s
 // convolutions that fit, chained through Adds: sum_k = sum_{k < K/s} + ... .  The slices of x and W are views, the
 // Add joins the next slice's epilogue, so the cost is one extra write and read of the partial sum.  (A lowering
 // decision, not one of the paper's rewriting rules: it is applied to every plan, fused or not.)
-static void split_deep_pointwise(Graph& g) {
+static void split_deep_pointwise(Graph& g, const std::set<int>& decided) {
   if (getenv("DNNF_NO_K_SPLIT")) return;
   const size_t n_ops = g.ops.size();
   bool any = false;
@@ -384,7 +384,7 @@ static void split_deep_pointwise(Graph& g) {
     if (tf32_shape_fits(M, N, K)) continue;
     int s = 0;
     for (int c : {2, 3, 4, 5, 6, 8}) if (K % (4 * c) == 0 && tf32_shape_fits(M, N, K / c)) { s = c; break; }
-    if (!s || !split_pays(M, N, K, 1, s)) continue;
+    if (!s || (!decided.count((int)oi) && !split_pays(M, N, K, 1, s))) continue;      // parts of a column split were costed as a whole
     const int source = g.ops[oi].source_id;
     auto add = [&](int kind, std::vector<int> in, const Attrs& at, int reuse_out) -> int {
       Op o; o.id = (int)g.ops.size(); o.kind = kind; o.in = std::move(in); o.at = at; o.source_id = source;
@@ -407,7 +407,7 @@ static void split_deep_pointwise(Graph& g) {
       }
     }
     Attrs r2; r2.shape = {M, K};
-    const int x2 = add(DNNF_OP_RESHAPE, {x}, r2, -1);
+    const int x2 = g.tensors[x].dims == r2.shape ? x : add(DNNF_OP_RESHAPE, {x}, r2, -1);
     int acc = -1;
     bool ok = x2 >= 0;
     for (int i = 0; i < s && ok; ++i) {
@@ -445,7 +445,7 @@ static void split_deep_pointwise(Graph& g) {
 // they stay in the convolutions' epilogues and each part is stored straight into the result.  The part width is the one
 // that needs the fewest kernels once the K split below has been applied to the parts as well (at most 32; every part
 // reads x again, but the tiled FMA kernel such a convolution would otherwise run on is slower by an order of magnitude).
-static void split_wide_pointwise(Graph& g) {
+static void split_wide_pointwise(Graph& g, std::set<int>& decided) {
   if (getenv("DNNF_NO_N_SPLIT") || getenv("DNNF_NO_TF32_GEMM")) return;
   g.relink();
   const size_t n_ops = g.ops.size();
@@ -525,6 +525,7 @@ static void split_wide_pointwise(Graph& g) {
       if (wj < 0) { ok = false; break; }
       int v = add(DNNF_OP_MATMUL, {x2, wj}, Attrs{}, source, -1);
       if (v < 0) { ok = false; break; }
+      decided.insert((int)g.ops.size() - 1);
       Attrs r4; r4.shape = ydims; r4.shape[3] = n1 - n0;
       v = add(DNNF_OP_RESHAPE, {v}, r4, source, -1);
       for (const Link& l : chain) {
@@ -568,8 +569,11 @@ static void split_wide_pointwise(Graph& g) {
 
 int plan_graph(Graph& g, uint32_t flags) {
   g.relink();
-  split_wide_pointwise(g);
-  split_deep_pointwise(g);
+  {
+    std::set<int> decided;                  // matrix products made by the column split: their K split is part of that decision
+    split_wide_pointwise(g, decided);
+    split_deep_pointwise(g, decided);
+  }
   // Operators whose results nobody reads (not a graph output, no live consumer) are not planned: they would
   // form blocks without an output.  (The rewriting pass removes them as well; a graph planned without rewriting
   // may still carry some.)

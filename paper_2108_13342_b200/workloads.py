@@ -330,6 +330,47 @@ def cnn_neck(n=8, h=64, w=64, c=32, seed=BASE_SEED) -> Workload:
     return Workload(g, ins, note="fp32 NHWC")
 
 
+def mbconv_stack(n=32, hw=56, seed=BASE_SEED) -> Workload:
+    """A MobileNetV2-shaped stack of inverted-residual blocks in NHWC fp32 (expand 1x1 + BN + ReLU6, depthwise 3x3 + BN +
+    ReLU6, project 1x1 + BN, residual where the shapes agree) with the channel progression 16-24-32-64-96-160 and
+    expansion 6, MaxPool 3x3 / 2 between the stages (the library's depthwise kernel has stride 1), a 1x1 head, global
+    average pool and a classifier: the convolution side of the paper's model zoo (Section 5) as one synthetic graph.
+    Expansions beyond 192 channels and projections deeper than 244 exercise the planner's column-block and K splits."""
+    d = _Draw(seed + 11)
+    g = GraphDesc("mbconv_stack")
+    ins = {}
+    cnt = [0]
+
+    def ext(shape, lo=None, hi=None, std=None, name=None):
+        cnt[0] += 1
+        name = name or "p%d" % cnt[0]
+        g.ext(name, shape, kind="input" if name == "X" else "weight")
+        ins[name] = d.normal(shape, 0.0, std) if std is not None else d.uniform(shape, lo, hi)
+        return name
+
+    def bn(x, c):
+        return g.add("ScaleShift", [x, ext((c,), 0.5, 1.5), ext((c,), -0.5, 0.5)], axis=-1)
+
+    def block(x, cin, cout, t=6):
+        e = cin * t
+        y = g.add("Clip", [bn(g.add("Conv1x1", [x, ext((cin, e), std=math.sqrt(2.0 / cin))]), e)], lo=0.0, hi=6.0)
+        y = g.add("Clip", [bn(g.add("DwConv3x3", [y, ext((3, 3, e), std=math.sqrt(2.0 / 9.0))]), e)], lo=0.0, hi=6.0)
+        y = bn(g.add("Conv1x1", [y, ext((e, cout), std=math.sqrt(1.0 / e))]), cout)
+        return g.add("Add", [y, x]) if cin == cout else y
+
+    x = ext((n, hw, hw, 16), 0.0, 1.0, name="X")
+    x = block(x, 16, 24); x = block(x, 24, 24)
+    x = g.add("MaxPool", [x], kernel=3, stride=2, pad=1)
+    x = block(x, 24, 32); x = block(x, 32, 32); x = block(x, 32, 64)
+    x = g.add("MaxPool", [x], kernel=3, stride=2, pad=1)
+    x = block(x, 64, 64); x = block(x, 64, 96); x = block(x, 96, 96); x = block(x, 96, 160)
+    x = g.add("Clip", [bn(g.add("Conv1x1", [x, ext((160, 320), std=math.sqrt(2.0 / 160))]), 320)], lo=0.0, hi=6.0)
+    x = g.add("AveragePool", [x], kernel=hw // 4, stride=1, pad=0)                 # [n, 1, 1, 320]
+    x = g.add("Add", [g.add("Conv1x1", [x, ext((320, 100), std=math.sqrt(1.0 / 320))]), ext((100,), -0.1, 0.1)], out="logits")
+    g.mark_output(x)
+    return Workload(g, ins, note="fp32 NHWC")
+
+
 # --------------------------------------------------------------------------
 # Workload 5: transformer encoder as primitive operators (48 per layer)
 # --------------------------------------------------------------------------
@@ -496,5 +537,6 @@ def decoder(layers=12, batch=8, seq=128, hidden=768, heads=12, ffn=3072, seed=BA
 def by_name(name: str, **kw) -> Workload:
     table = {"swish_transpose": swish_transpose, "masked_softmax": masked_softmax,
              "add_layernorm_gelu": add_layernorm_gelu, "ffn_block": ffn_block,
-             "mbconv_block": mbconv_block, "encoder": encoder, "decoder": decoder, "cnn_neck": cnn_neck}
+             "mbconv_block": mbconv_block, "encoder": encoder, "decoder": decoder, "cnn_neck": cnn_neck,
+             "mbconv_stack": mbconv_stack}
     return table[name](**kw)

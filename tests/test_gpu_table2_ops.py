@@ -276,3 +276,20 @@ def test_gather_clamps_indices_outside_the_table():
     assert s.g.status()[0] == 0
     got = s.output(g.outputs[0])
     assert np.array_equal(got, tab[[0, 0, 5, 5, 5]].astype(np.float32))
+
+
+@pytest.mark.parametrize("flags,always", [(B.PLAN_FUSED, False), (B.PLAN_FUSED, True), (B.PLAN_UNFUSED, True)])
+def test_mobilenet_shaped_stack(flags, always, monkeypatch):
+    """Nine inverted-residual blocks, pooling between the stages, head and classifier: expansions wider than 192 channels
+    and projections deeper than 244 go through the planner's column-block and K splits (forced at this small size in two
+    of the three variants, decided by the cost model in the first)."""
+    if always:
+        monkeypatch.setenv("DNNF_SPLIT_ALWAYS", "1")
+    wl = W.mbconv_stack(n=4, hw=48)
+    s = check(wl, 5e-4, flags, B.REWRITE_DEFAULT)
+    fams = [b["family"] for b in s.g.blocks()]
+    assert "dwconv" in fams and "pool" in fams
+    if always:
+        assert fams.count("gemm") >= 20, fams          # the split pieces
+    if flags == B.PLAN_FUSED:
+        assert s.plan_stats.n_kernels < s.plan_stats.n_ops
