@@ -1,14 +1,29 @@
 #!/usr/bin/env python
 """Benchmark of the fused-block executor on one B200.
 
-Default arm: `python bench.py --gpus N --steps K --warmup W` prints ONE JSON line.
-A step is one pass of the hot path -- dnnf_run of the fused scale+mask+softmax
-block and of the fused add+LayerNorm+GELU block (fp32, the attention-score /
-norm configuration) -- over a batch of R independent instances that live in
-distinct buffers larger than L2.  `value` is algorithmic GB/s over the whole
-step, inputs already in HBM; `e2e` is the same through host buffers.
+Default arm: `python bench.py --gpus N --steps K --warmup W` prints ONE short JSON line
+(the last line of stdout).
 
-`--impl reference` times the CPU oracle on the same workload (bounded sample).
+A step is one pass of the hot path -- dnnf_run of the fused MobileNetV2-style
+inverted-residual block (fp32 NHWC [32,56,56,24 -> 144 -> 24]: pointwise expansion +
+BN + ReLU6, depthwise 3x3 + BN + ReLU6, pointwise projection + BN + residual; three
+kernels) -- over one batch of 32 synthetic images.  It is the largest memory-bound
+configuration: 260.1 MB of algorithmic traffic per step.  Consecutive steps rotate
+over SETS complete, independent buffer sets (inputs, intermediates, outputs) so that
+no step finds its data in L2.
+
+  value     algorithmic GB/s over the whole step (every block's external inputs and
+            outputs once), inputs resident in HBM, plain stream launches of dnnf_run
+  roofline  the longest kernel of the step by its own CUDA-event time (a second pass
+            over the same steps with an event between the blocks)
+  e2e       the same step with the images copied from pinned host memory and the
+            result copied back inside the timed region
+  graph_latency  the metric's second half: the 12-layer encoder (576 primitive
+            operators) fused against one kernel per operator, CUDA-graph replays
+
+`--detail` writes the per-configuration / per-block tables to
+gpurun_out/bench_detail.json.  `--impl reference` times the CPU oracle on the same
+workload (bounded sample).
 """
 from __future__ import annotations
 
@@ -25,9 +40,10 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-METRIC = "fused-block GB/s (algorithmic bytes / time) on the attention-score and norm blocks; % of HBM peak in roofline"
+METRIC = "fused-block GB/s as % of HBM peak; graph latency fused vs unfused per-op"
 UNIT = "GB/s"
-R_INSTANCES = 24
+SETS = 3
+WORKLOAD = "configs[3]: MobileNetV2-style inverted-residual block, fp32 NHWC [32,56,56,24->144->24], 3 fused kernels"
 
 
 def peaks():
@@ -103,42 +119,55 @@ def rank_seed(base_seed, rank):
 
 
 def block_bytes(sess):
-    tot = 0
-    for b in range(sess.g.block_count()):
-        d = sess.g.block_info(b)
-        tot += d.bytes_in + d.bytes_out
-    return tot
+    return [sess.g.block_info(b).bytes_in + sess.g.block_info(b).bytes_out for b in range(sess.g.block_count())]
+
+
+def mbconv_algorithmic_bytes(n=32, h=56, w=56, cin=24, cexp=144):
+    """External inputs and outputs of the three fused blocks, each once (fp32)."""
+    x, e = n * h * w * cin, n * h * w * cexp
+    blocks = [x + cin * cexp + 2 * cexp + e,            # expansion: X, W1, scale, shift -> E
+              e + 9 * cexp + 2 * cexp + e,              # depthwise: E, Kd, scale, shift -> E2
+              e + cexp * cin + 2 * cin + x + x]         # projection: E2, W3, scale, shift, X -> Y
+    return [4 * b for b in blocks]
+
+
+def oracle_pass_timer(wl):
+    """Times the oracle on the workload; returns (seconds per pass, passes, threads it kept busy)."""
+    from oracle import interp as O
+    O.run_graph(wl.graph, wl.inputs)
+    n, t0, c0 = 0, time.perf_counter(), time.process_time()
+    while time.perf_counter() - t0 < 10.0 or n < 2:
+        O.run_graph(wl.graph, wl.inputs)
+        n += 1
+    wall, cpu = time.perf_counter() - t0, time.process_time() - c0
+    return wall / n, n, max(1, int(round(cpu / wall)))
 
 
 # --------------------------------------------------------------------------------------
 def run_reference(args):
-    """CPU oracle arm: the unfused fp64 interpreter on the host cores."""
+    """CPU oracle arm: the unfused fp64 interpreter on the host cores, same workload and metric."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from oracle import interp as O
     from paper_2108_13342_b200 import workloads as W
-    try:
-        from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
-    except Exception:
-        cores = 1
-    wa, wb = W.masked_softmax(), W.add_layernorm_gelu()
-    bytes_step = 12648448 + 9443328
+    n_img = 4                                         # bounded sample: 4 of the step's 32 images per reference step
+    wl = W.mbconv_block(n=n_img)
+    bytes_step = sum(mbconv_algorithmic_bytes(n=n_img))      # the step's algorithmic bytes, scaled to the sample
     for _ in range(max(1, min(args.warmup, 1))):
-        O.run_graph(wa.graph, wa.inputs); O.run_graph(wb.graph, wb.inputs)
-    t0 = time.perf_counter()
+        O.run_graph(wl.graph, wl.inputs)
+    t0, c0 = time.perf_counter(), time.process_time()
     for _ in range(args.steps):
-        O.run_graph(wa.graph, wa.inputs); O.run_graph(wb.graph, wb.inputs)
-    dt = (time.perf_counter() - t0) / args.steps
+        O.run_graph(wl.graph, wl.inputs)
+    wall, cpu = time.perf_counter() - t0, time.process_time() - c0
+    dt = wall / args.steps
+    cores = max(1, int(round(cpu / wall)))
     val = bytes_step / dt / 1e9
+    sample = f"{n_img} of the step's 32 images per reference step, numpy fp64 unfused interpreter"
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "configs[1]: scale+mask+softmax [8,12,128,128] + add+LayerNorm+GELU [1024,768]; "
-                                   "one instance per step (bounded sample of the 24-instance GPU step)"},
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
-                             "sample": "1 of 24 instances per step, numpy fp64 unfused interpreter"},
+            "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD + "; " + sample},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -147,14 +176,12 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="dnnf")
-    ap.add_argument("--no-detail", action="store_true")
+    ap.add_argument("--detail", action="store_true", help="also write per-configuration / per-block tables to gpurun_out/bench_detail.json")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--no-graph", action="store_true", help="time plain dnnf_run launches instead of a captured CUDA graph")
-    ap.add_argument("--branches", type=int, default=4,
-                    help="parallel branches of the captured graph: the step's instances are independent, so they may overlap on the GPU")
+    ap.add_argument("--no-graph-latency", action="store_true", help="skip the encoder fused / unfused latency pair")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -177,211 +204,163 @@ def main():
     pk = peaks()
     steps, warm = args.steps, max(args.warmup, 3)
 
-    # ---- the step: R instances of each block, distinct buffers (footprint > L2) ------------------
-    wa, wb = W.masked_softmax(seed=rank_seed(W.BASE_SEED, rank)), W.add_layernorm_gelu(seed=rank_seed(W.BASE_SEED, rank))
-    A = [Session(wa, rewrite_flags=B.REWRITE_NONE, device=dev) for _ in range(R_INSTANCES)]
-    Bn = [Session(wb, rewrite_flags=B.REWRITE_NONE, device=dev) for _ in range(R_INSTANCES)]
-    bytes_a, bytes_b = block_bytes(A[0]), block_bytes(Bn[0])
-    bytes_step = R_INSTANCES * (bytes_a + bytes_b)
+    # ---- the step: dnnf_run of the fused block on one of SETS independent buffer sets ------------
+    wl = W.mbconv_block(seed=rank_seed(W.BASE_SEED, rank))
+    S = [Session(wl, rewrite_flags=B.REWRITE_NONE, device=dev) for _ in range(SETS)]
+    nb = S[0].g.block_count()
+    bbytes = block_bytes(S[0])
+    assert bbytes == mbconv_algorithmic_bytes(), (bbytes, mbconv_algorithmic_bytes())
+    bytes_step = sum(bbytes)
     stream = torch.cuda.current_stream(dev)
     sptr = stream.cuda_stream
 
-    def part_a():
-        for s in A:
-            s.g.run(sptr)
-
-    def part_b():
-        for s in Bn:
-            s.g.run(sptr)
-
-    for _ in range(warm):
-        part_a(); part_b()
+    for i in range(warm):
+        S[i % SETS].g.run(sptr)
     torch.cuda.synchronize(dev)
-    plain_a, plain_b = part_a, part_b
-    if not args.no_graph:
-        # The step is launch-bound (48 kernels of a few microseconds): capture it once, replay it.
-        # dnnf_run neither allocates nor synchronises, so it can be captured as is.
-        # The instances of a step share no buffer, so the graph gets `branches` parallel chains: a kernel
-        # of one instance may run beside a kernel of another (each fills about a third of the SMs).
-        side = torch.cuda.Stream(dev)
-        nbr = max(1, min(args.branches, R_INSTANCES))
-        lanes = [torch.cuda.Stream(dev) for _ in range(nbr - 1)]
-        side.wait_stream(stream)
-        graphs = []
-        with torch.cuda.stream(side):
-            for sess in (A, Bn):
-                cg = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(cg, stream=side):
-                    for ln in lanes:
-                        ln.wait_stream(side)                       # fork
-                    for i, x in enumerate(sess):
-                        st = side if i % nbr == 0 else lanes[i % nbr - 1]
-                        x.g.run(st.cuda_stream)
-                    for ln in lanes:
-                        side.wait_stream(ln)                       # join
-                graphs.append(cg)
-        stream.wait_stream(side)
-        part_a, part_b = graphs[0].replay, graphs[1].replay
-        for _ in range(warm):
-            part_a(); part_b()
-        torch.cuda.synchronize(dev)
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize(dev)
     with ClockSampler(local) as clk:
+        e0.record(stream)
         for i in range(steps):
-            ev[i][0].record(stream); part_a(); ev[i][1].record(stream); part_b(); ev[i][2].record(stream)
+            S[i % SETS].g.run(sptr)
+        e1.record(stream)
         torch.cuda.synchronize(dev)
-        t_total = ev[0][0].elapsed_time(ev[-1][2])                      # ms, whole timed region
-        # keep the GPU busy a little longer so the sampler sees clocks under load
+        ms_step = e0.elapsed_time(e1) / steps
+        # second pass over the same steps with an event between the blocks: each kernel's own duration
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(nb + 1)] for _ in range(steps)]
+        for i in range(steps):
+            g = S[i % SETS].g
+            ev[i][0].record(stream)
+            for b in range(nb):
+                g.run_block(b, sptr)
+                ev[i][b + 1].record(stream)
+        torch.cuda.synchronize(dev)
+        # keep the GPU busy a little longer so that the sampler sees clocks under load
         t_end = time.time() + 1.0
+        i = 0
         while time.time() < t_end:
-            part_a(); part_b()
+            S[i % SETS].g.run(sptr)
+            i += 1
+            if i % 64 == 0:
+                torch.cuda.synchronize(dev)
         torch.cuda.synchronize(dev)
     if world > 1:
         dist.barrier()
-    t_a = sum(e[0].elapsed_time(e[1]) for e in ev) / steps             # ms per step in part a
-    t_b = sum(e[1].elapsed_time(e[2]) for e in ev) / steps
-    ms_step = t_total / steps
+    for s in S:
+        st, blk = s.g.status()
+        if st != 0:
+            raise SystemExit(f"device status {st} from block {blk}")
     ms_step = max_over_ranks(ms_step, dev)
     value = aggregate_throughput(bytes_step, ms_step, world)
 
-    # ---- roofline of the dominant kernel (the softmax row kernel) ---------------------------------
-    dur_a = t_a * 1e-3 / R_INSTANCES
-    ach = bytes_a / dur_a / 1e9
-    def kernel_name(sess):
-        b = sess.g.blocks()[0]
-        v = b["variant"]                          # row family: V*100000 + NV*1000 + WPR*10 + RPW
-        return "row_kernel<V=%d,NV=%d,WPR=%d,RPW=%d> running %s, one launch per instance" % (
-            v // 100000, v // 1000 % 100, v // 10 % 100, v % 10, "+".join(b["ops"]))
-    roof = {"bound": "hbm", "kernel": kernel_name(A[0]), "achieved": ach, "peak": pk["hbm_gbs"],
-            "unit": "GB/s", "frac": ach / pk["hbm_gbs"], "peak_source": pk["source"], "traffic": None,
-            "bytes_per_launch": bytes_a, "us_per_launch": dur_a * 1e6,
-            "second_kernel": {"kernel": kernel_name(Bn[0]), "bytes_per_launch": bytes_b,
-                              "us_per_launch": t_b * 1e3 / R_INSTANCES, "achieved": bytes_b / (t_b * 1e-3 / R_INSTANCES) / 1e9,
-                              "frac": bytes_b / (t_b * 1e-3 / R_INSTANCES) / 1e9 / pk["hbm_gbs"]}}
+    blocks = S[0].g.blocks()
+    k_us = [sum(e[b].elapsed_time(e[b + 1]) for e in ev) / steps * 1e3 for b in range(nb)]
+    kernels = [{"ops": "+".join(blocks[b]["ops"]), "us": round(k_us[b], 2), "bytes": bbytes[b],
+                "frac": round(bbytes[b] / (k_us[b] * 1e-6) / 1e9 / pk["hbm_gbs"], 3)} for b in range(nb)]
+    top = max(range(nb), key=lambda b: k_us[b])
+    ach = bbytes[top] / (k_us[top] * 1e-6) / 1e9
+    roof = {"bound": "hbm", "kernel": "%s kernel of block %d (%s)" % (blocks[top]["family"], top, "+".join(blocks[top]["ops"])),
+            "achieved": round(ach, 1), "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": round(ach / pk["hbm_gbs"], 4),
+            "peak_source": pk["source"], "traffic": None, "bytes_per_launch": bbytes[top], "us_per_launch": round(k_us[top], 3)}
     tp = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tp):                       # DRAM bytes per launch from the committed ncu capture (see profiles/)
+    if os.path.exists(tp):                       # DRAM bytes per launch of that kernel from the committed ncu capture
         with open(tp) as f:
             tj = json.load(f)
-        roof["traffic"] = tj.get("masked_softmax_bytes_per_launch")
-        roof["traffic_source"] = tj.get("source")
+        ent = tj.get("mbconv_block", {}).get(str(top))
+        if ent:
+            roof["traffic"] = ent["dram_bytes_per_launch"]
+            roof["traffic_source"] = ent["source"]
 
-    # ---- end to end: host buffers in, host result out, through the same C-ABI calls -----------------
-    hin_a = [torch.from_numpy(wa.inputs["S"]).pin_memory() for _ in range(2)]
-    hin_b = [(torch.from_numpy(wb.inputs["H"]).pin_memory(), torch.from_numpy(wb.inputs["R"]).pin_memory()) for _ in range(2)]
-    hout_a = torch.empty_like(hin_a[0]).pin_memory()
-    hout_b = torch.empty_like(hin_b[0][0]).pin_memory()
-    h2d = R_INSTANCES * (hin_a[0].numel() + 2 * hin_b[0][0].numel()) * 4
-    d2h = R_INSTANCES * (hout_a.numel() + hout_b.numel()) * 4
-
-    # Three streams: host->device copies, the blocks, device->host copies.  The two copy directions use different
-    # DMA engines, so instance i+1's input travels while instance i computes and instance i-1's result goes back.
-    # Events order copy-in -> run -> copy-out per instance, and the next step's copy-in of an instance after its
-    # previous copy-out (its buffers are reused).
+    # ---- end to end: images from pinned host memory, result back to the host, same C-ABI calls --------
+    hin = [torch.from_numpy(wl.inputs["X"]).pin_memory() for _ in range(SETS)]
+    hout = [torch.empty_like(hin[0]).pin_memory() for _ in range(SETS)]
+    h2d = hin[0].numel() * 4
+    d2h = hout[0].numel() * 4
+    # Three streams: host->device copies, the blocks, device->host copies (two DMA directions beside the kernels).
+    # Events order copy-in -> run -> copy-out per buffer set, and a set's next copy-in after its previous copy-out.
     s_in, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
-    n_inst = 2 * R_INSTANCES
-    ev_in = [torch.cuda.Event() for _ in range(n_inst)]
-    ev_run = [torch.cuda.Event() for _ in range(n_inst)]
-    ev_out = [torch.cuda.Event() for _ in range(n_inst)]
-    for e in ev_out:
+    ev_in = [torch.cuda.Event() for _ in range(SETS)]
+    ev_run = [torch.cuda.Event() for _ in range(SETS)]
+    ev_out = [torch.cuda.Event() for _ in range(SETS)]
+    for e in ev_out + ev_run:
         e.record(stream)
 
-    def e2e_step():
-        for k in range(n_inst):
-            is_a = k < R_INSTANCES
-            sess = A[k] if is_a else Bn[k - R_INSTANCES]
-            s_in.wait_event(ev_out[k])
-            with torch.cuda.stream(s_in):
-                if is_a:
-                    sess.buffers["S"].copy_(hin_a[k & 1], non_blocking=True)
-                else:
-                    sess.buffers["H"].copy_(hin_b[k & 1][0], non_blocking=True)
-                    sess.buffers["R"].copy_(hin_b[k & 1][1], non_blocking=True)
-                ev_in[k].record(s_in)
-            stream.wait_event(ev_in[k])
-            sess.g.run(sptr)
-            ev_run[k].record(stream)
-            s_out.wait_event(ev_run[k])
-            with torch.cuda.stream(s_out):
-                if is_a:
-                    hout_a.copy_(sess.buffers["P"], non_blocking=True)
-                else:
-                    hout_b.copy_(sess.buffers["Y"], non_blocking=True)
-                ev_out[k].record(s_out)
+    def e2e_step(i):
+        k = i % SETS
+        sess = S[k]
+        s_in.wait_event(ev_out[k])
+        s_in.wait_event(ev_run[k])                 # the residual reads X until the set's last kernel ends
+        with torch.cuda.stream(s_in):
+            sess.buffers["X"].copy_(hin[k], non_blocking=True)
+            ev_in[k].record(s_in)
+        stream.wait_event(ev_in[k])
+        stream.wait_event(ev_out[k])
+        sess.g.run(sptr)
+        ev_run[k].record(stream)
+        s_out.wait_event(ev_run[k])
+        with torch.cuda.stream(s_out):
+            hout[k].copy_(sess.buffers["Y"], non_blocking=True)
+            ev_out[k].record(s_out)
 
-    def e2e_join():
-        stream.wait_stream(s_in)
-        stream.wait_stream(s_out)
-
-    e2e_steps = max(3, min(steps, 10))
-    for _ in range(2):
-        e2e_step()
-    e2e_join()
+    e2e_steps = max(3, min(steps, 60))
+    for i in range(SETS):
+        e2e_step(i)
+    stream.wait_stream(s_in); stream.wait_stream(s_out)
     torch.cuda.synchronize(dev)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(e2e_steps):
-        e2e_step()
-    e2e_join()                                 # the timed region ends when the last result has reached the host
-    e1.record(stream)
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for i in range(e2e_steps):
+        e2e_step(i)
+    stream.wait_stream(s_in); stream.wait_stream(s_out)     # the region ends when the last result has reached the host
+    f1.record(stream)
     torch.cuda.synchronize(dev)
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    e2e_ms = max_over_ranks(e2e_ms, dev)
-    e2e = {"value": aggregate_throughput(bytes_step, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms}
+    e2e_ms = max_over_ranks(f0.elapsed_time(f1) / e2e_steps, dev)
+    e2e = {"value": round(aggregate_throughput(bytes_step, e2e_ms, world), 1), "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4)}
 
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+    line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
+            "ms_per_step": round(ms_step, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
-            "config": {"workload": f"configs[1]: fused scale+mask+softmax [8,12,128,128] and fused add+LayerNorm+GELU "
-                                   f"[1024,768], fp32; {R_INSTANCES} independent instances of each per step",
-                       "l2": f"inputs larger than L2: {bytes_step / 1e6:.0f} MB of distinct buffers per step",
-                       "bytes_per_step": bytes_step, "launches_per_step": 2 * R_INSTANCES,
-                       "launch_mode": "plain stream launches" if args.no_graph else
-                       ("CUDA-graph replay of the captured step with %d parallel branches over the step's independent instances; "
-                        "kernels use programmatic dependent launch" % max(1, min(args.branches, R_INSTANCES)))},
-            "clocks": clk.summary(), "e2e": e2e, "gpu_launches": steps * 2 * R_INSTANCES, "roofline": roof}
+            "config": {"workload": WORKLOAD, "bytes_per_step": bytes_step, "launches_per_step": nb,
+                       "l2": f"steps rotate over {SETS} independent buffer sets of {bytes_step // 2 // 1000000} MB each (> L2)",
+                       "launch_mode": "plain stream launches of dnnf_run; kernels chained by programmatic dependent launch"},
+            "frac_of_hbm_peak": round(value / world / pk["hbm_gbs"], 4),
+            "clocks": clk.summary(), "e2e": e2e, "gpu_launches": steps * nb, "roofline": roof, "kernels": kernels}
 
-    if rank == 0 and not args.no_cpu:
-        line["cpu_baseline"] = cpu_baseline(wa, wb, bytes_a + bytes_b)
-    if rank == 0 and not args.no_detail:
+    del S
+    torch.cuda.empty_cache()
+    if rank == 0 and not args.no_graph_latency:
         from paper_2108_13342_b200 import report
-        line["detail"] = report.per_config(dev, pk)
         try:
-            line["detail"]["cfg5 12-layer encoder (576 primitive operators)"] = report.encoder_report(dev, pk)
-        except Exception as e:
-            line["detail"]["cfg5 12-layer encoder (576 primitive operators)"] = {"error": repr(e)}
-        try:
-            line["detail"]["next: 12-layer GPT-2 style decoder (633 primitive operators)"] = report.decoder_report(dev, pk)
-        except Exception as e:  # noqa: BLE001
-            line["detail"]["next: 12-layer GPT-2 style decoder (633 primitive operators)"] = {"error": repr(e)}
-        line["paper_context"] = {"note": "mobile-device figures from the paper, not comparable hardware",
-                                 "fusion_rate_vs_other_frameworks": "up to 8.8x", "speedup_vs_other_frameworks": "up to 9.3x",
-                                 "speedup_vs_own_unfused_backend": "1.5-5.8x"}
+            line["graph_latency"] = report.encoder_latency_pair(dev, pk)
+        except Exception as e:      # report, never hide
+            line["graph_latency"] = {"error": repr(e)[:200]}
+    if rank == 0 and not args.no_cpu:
+        sec, n, cores = oracle_pass_timer(W.mbconv_block(n=4))
+        line["cpu_baseline"] = {"value": round(sum(mbconv_algorithmic_bytes(n=4)) / sec / 1e9, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{n} passes over 4 of the step's 32 images (about {sec * n:.0f} s of CPU work)"}
+    if rank == 0 and args.detail:
+        from paper_2108_13342_b200 import report
+        detail = report.per_config(dev, pk)
+        for name, fn in [("cfg5 12-layer encoder (576 primitive operators)", report.encoder_report),
+                         ("next: 12-layer GPT-2 style decoder (633 primitive operators)", report.decoder_report)]:
+            try:
+                detail[name] = fn(dev, pk)
+            except Exception as e:  # noqa: BLE001
+                detail[name] = {"error": repr(e)}
+        detail["paper_context"] = {"note": "mobile-device figures from the paper, not comparable hardware",
+                                   "fusion_rate_vs_other_frameworks": "up to 8.8x", "speedup_vs_other_frameworks": "up to 9.3x",
+                                   "speedup_vs_own_unfused_backend": "1.5-5.8x"}
+        os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
+        with open(os.path.join(ROOT, "gpurun_out", "bench_detail.json"), "w") as f:
+            json.dump(detail, f, indent=1)
     if rank == 0:
+        sys.stdout.flush()
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
-
-
-def cpu_baseline(wa, wb, bytes_instance):
-    from oracle import interp as O
-    try:
-        from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
-    except Exception:
-        cores = 1
-    O.run_graph(wa.graph, wa.inputs); O.run_graph(wb.graph, wb.inputs)
-    n, t0 = 0, time.perf_counter()
-    while time.perf_counter() - t0 < 10.0 or n < 2:
-        O.run_graph(wa.graph, wa.inputs); O.run_graph(wb.graph, wb.inputs)
-        n += 1
-    dt = (time.perf_counter() - t0) / n
-    return {"value": bytes_instance / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{n} passes over 1 of the {R_INSTANCES} instances (about {dt * n:.0f} s of CPU work)",
-            "ms_per_instance": dt * 1e3}
 
 
 if __name__ == "__main__":

@@ -433,6 +433,7 @@ int dnnf_bind_workspace(dnnf_graph* g, void* dev_ptr, size_t bytes) {
   if (!dev_ptr || ((uintptr_t)dev_ptr & 255)) return fail(g, DNNF_ERR_INVALID_ARG, "workspace must be non-null and 256-byte aligned");
   if (bytes < G.ws_bytes) return fail(g, DNNF_ERR_WORKSPACE, "workspace too small");
   G.ws_ptr = dev_ptr; G.ws_bound_bytes = bytes;
+  G.last_status_base = nullptr;      // no run yet on this workspace: dnnf_status reads the new one
   return DNNF_OK;
 }
 

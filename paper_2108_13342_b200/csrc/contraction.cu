@@ -38,7 +38,7 @@ void conv1x1_direct_plan(Launch& L);
 int conv1x1_direct_launch(const Launch& L, cudaStream_t st);
 int lower_dwconv(const Graph& g, const std::vector<int>& ops, int anchor, Block& out, std::string& why);
 int dwconv_launch(const Launch& L, void* status_words, int block_index, cudaStream_t st);
-void dwconv_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
+void dwconv_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op, std::string& err);
 int lower_gather(const Graph& g, const std::vector<int>& ops, int anchor, Block& out, std::string& why);
 int gather_launch(const Launch& L, cudaStream_t st);
 void gather_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
@@ -481,24 +481,23 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
 }
 
 void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op, std::string& err) {
-  if (L.family == DNNF_FAMILY_DWCONV) { dwconv_patch(L, ip, op); return; }
+  if (L.family == DNNF_FAMILY_DWCONV) { dwconv_patch(L, ip, op, err); return; }
   if (L.family == DNNF_FAMILY_POOL) { pool_patch(L, ip, op); return; }
   if (L.family == DNNF_FAMILY_GATHER) { gather_patch(L, ip, op); return; }
   GemmParams& gp = gp_of(L);
-  bool changed = gp.A.ptr != ip[0] || gp.B.ptr != ip[1];
   gp.A.ptr = ip[0]; gp.B.ptr = ip[1];
   for (int i = 0; i < gp.n_in; ++i) gp.in[i].ptr = ip[2 + i];
   for (int i = 0; i < gp.n_out; ++i) gp.out[i].ptr = op[i];
-  if (L.variant == 3) changed = changed || !L.tc_ready || gp.out[0].ptr != L.last_out || (gp.n_in > 0 && gp.in[0].ptr != L.last_in0) || (gp.n_in > 1 && gp.in[1].ptr != L.last_in1);
-  if (L.variant == 1 && (changed || !L.tc_ready)) { if (tc_gemm_prepare(L, err)) L.tc_ready = true; }
-  if (L.variant == 4 && (changed || !L.tc_ready || gp.out[0].ptr != L.last_out)) {
-    if (tf32_gemm_prepare(L, err)) L.tc_ready = true;
-    L.last_out = gp.out[0].ptr;
-  }
-  if (L.variant == 3 && changed) {
-    if (tc2_gemm_prepare(L, err)) L.tc_ready = true;
-    L.last_out = gp.out[0].ptr; L.last_in0 = gp.n_in > 0 ? gp.in[0].ptr : nullptr; L.last_in1 = gp.n_in > 1 ? gp.in[1].ptr : nullptr;
-  }
+  if (L.variant != 1 && L.variant != 3 && L.variant != 4) return;
+  // The tensor maps embed addresses: encode them again whenever ANY pointer of the block differs from the
+  // ones they were made for (an epilogue operand in any position may be read through a map).
+  std::vector<void*> now(ip);
+  now.insert(now.end(), op.begin(), op.end());
+  if (L.tc_ready && now == L.encoded_ptrs) return;
+  L.tc_ready = false;
+  bool ok = L.variant == 1 ? tc_gemm_prepare(L, err) : L.variant == 3 ? tc2_gemm_prepare(L, err) : tf32_gemm_prepare(L, err);
+  if (ok) { L.tc_ready = true; L.encoded_ptrs = now; }
+  else if (err.empty()) err = "cannot encode the tensor maps of a contraction block";
 }
 
 int launch_contraction(const Launch& L, void* status_words, int block_index, cudaStream_t st, std::string& err) {
@@ -506,6 +505,7 @@ int launch_contraction(const Launch& L, void* status_words, int block_index, cud
   if (L.family == DNNF_FAMILY_POOL) { int rc = pool_launch(L, status_words, st); if (rc) err = "pooling launch failed"; return rc; }
   if (L.family == DNNF_FAMILY_DWCONV) { int rc = dwconv_launch(L, status_words, block_index, st); if (rc) err = "depthwise convolution launch failed"; return rc; }
   if (L.variant == 2) { int rc = conv1x1_direct_launch(L, st); if (rc) err = "pointwise convolution launch failed"; return rc; }
+  if ((L.variant == 1 || L.variant == 3 || L.variant == 4) && !L.tc_ready) { err = "tensor maps of the block are not encoded"; return 1; }
   GemmParams gp = gp_of(L);
   gp.status = reinterpret_cast<int32_t*>(status_words);
   gp.block_index = block_index;

@@ -187,8 +187,8 @@ template <int TN, int CG, int PG>
 struct PwLauncher {
   const Launch& L; cudaStream_t st;
   template <class SP> void run() {
-    static bool attr = false;
-    if (!attr) { cudaFuncSetAttribute(conv1x1_kernel<TN, CG, PG, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024); attr = true; }
+    static PerDeviceOnce once;       // per instantiation
+    if (once.first_use()) cudaFuncSetAttribute(conv1x1_kernel<TN, CG, PG, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024);
     launch_pdl(conv1x1_kernel<TN, CG, PG, SP>, L.grid, CG * PG, L.smem, st, gp_of(L));
   }
 };
@@ -286,18 +286,19 @@ struct DwLauncher {
 };
 
 int dwconv_launch(const Launch& L, void* status_words, int block_index, cudaStream_t st) {
+  if (L.variant < 0 && !L.tc_ready) return 1;        // never launch with a tensor map that was not encoded
   if (L.variant < 0) return dwconv_tma_launch(L, reinterpret_cast<int32_t*>(status_words), block_index, st);
   DwLauncher F{L, st, L.variant};
   if (!(L.static_id > 0 && StaticSet<ConvStatic>::dispatch(L.static_id, F))) F.run<DynProg>();
   return cudaGetLastError() == cudaSuccess ? 0 : 1;
 }
 
-void dwconv_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op) {
+void dwconv_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op, std::string& err) {
   DwParams& dp = *reinterpret_cast<DwParams*>(L.blob.data());
   if (L.variant < 0 && (dp.x != ip[0] || !L.tc_ready)) {
     dp.x = reinterpret_cast<const float*>(ip[0]);
-    std::string err;
     L.tc_ready = dwconv_tma_prepare(L, err);
+    if (!L.tc_ready && err.empty()) err = "cannot encode the tensor map of a depthwise convolution block";
   }
   dp.x = reinterpret_cast<const float*>(ip[0]);
   dp.k = reinterpret_cast<const float*>(ip[1]);

@@ -253,8 +253,8 @@ bool dwconv_tma_prepare(Launch& L, std::string& err) {
 struct DwTmaLauncher {
   const Launch& L; cudaStream_t st; int32_t* status; int block_index;
   template <class SP> void run() {
-    static bool attr_set = false;     // per instantiation
-    if (!attr_set) { cudaFuncSetAttribute(dwt::dwconv_tma_kernel<SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024); attr_set = true; }
+    static PerDeviceOnce once;       // per instantiation
+    if (once.first_use()) cudaFuncSetAttribute(dwt::dwconv_tma_kernel<SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
     launch_pdl(dwt::dwconv_tma_kernel<SP>, L.grid, dwt::THREADS, L.smem, st, dw_of(L), tq_of(L), status, block_index);
   }
 };

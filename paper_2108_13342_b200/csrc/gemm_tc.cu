@@ -336,8 +336,8 @@ bool tc_gemm_prepare(Launch& L, std::string& err) {
 struct TcLauncher {
   const Launch& L; cudaStream_t st; int stages;
   template <class SP> void run() {
-    static bool attr_set = false;     // per instantiation
-    if (!attr_set) { cudaFuncSetAttribute(gemm_tc_kernel<SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax); attr_set = true; }
+    static PerDeviceOnce once;       // per instantiation
+    if (once.first_use()) cudaFuncSetAttribute(gemm_tc_kernel<SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
     launch_pdl(gemm_tc_kernel<SP>, L.grid, TC_THREADS, L.smem, st, gp_of(L), tc_of(L), tc_of(L).tmA, tc_of(L).tmB, stages);
   }
 };

@@ -631,8 +631,8 @@ bool tc2_gemm_prepare(Launch& L, std::string& err) {
 struct Tc2Launcher {
   const Launch& L; cudaStream_t st; cudaError_t rc;
   template <class SP> void run() {
-    static bool attr_set = false;
-    if (!attr_set) { cudaFuncSetAttribute(tc2::gemm_tc2_kernel<SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::kSmemMax); attr_set = true; }
+    static PerDeviceOnce once;       // per instantiation
+    if (once.first_use()) cudaFuncSetAttribute(tc2::gemm_tc2_kernel<SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::kSmemMax);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(L.grid); cfg.blockDim = dim3(tc2::THREADS); cfg.dynamicSmemBytes = L.smem; cfg.stream = st;
     cudaLaunchAttribute attr[2];

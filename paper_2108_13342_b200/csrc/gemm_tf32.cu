@@ -683,8 +683,8 @@ template <bool kFast>
 struct Tf32Launcher {
   const Launch& L; cudaStream_t st;
   template <class SP> void run() {
-    static bool attr_set = false;     // per instantiation
-    if (!attr_set) { cudaFuncSetAttribute(tf32::gemm_tf32_kernel<SP, kFast>, cudaFuncAttributeMaxDynamicSharedMemorySize, tf32::kSmemMax); attr_set = true; }
+    static PerDeviceOnce once;       // per instantiation
+    if (once.first_use()) cudaFuncSetAttribute(tf32::gemm_tf32_kernel<SP, kFast>, cudaFuncAttributeMaxDynamicSharedMemorySize, tf32::kSmemMax);
     launch_pdl(tf32::gemm_tf32_kernel<SP, kFast>, L.grid, tf32::THREADS, L.smem, st, gp_of(L), fp_of(L));
   }
 };

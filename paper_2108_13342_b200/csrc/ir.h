@@ -60,7 +60,7 @@ struct Launch {
   int family = DNNF_FAMILY_ALIAS;
   int variant = 0;
   bool tc_ready = false;      // tensor maps encoded for the currently bound pointers
-  void *last_out = nullptr, *last_in0 = nullptr, *last_in1 = nullptr;
+  std::vector<void*> encoded_ptrs;   // the pointers (operands, epilogue inputs, outputs) the tensor maps were encoded for
   int static_id = 0;          // compile-time program table the block runs on (0: interpreted)
   int grid = 0, threads = 0;
   size_t smem = 0;
@@ -97,6 +97,7 @@ struct Graph {
   size_t ws_zero_bytes = 256;            // leading bytes of the workspace that must be zero when a run starts
   void* ws_ptr = nullptr;
   size_t ws_bound_bytes = 0;
+  void* last_status_base = nullptr;   // workspace whose status words the most recent run used (dnnf_status reads these)
   dnnf_plan_stats pstats{};
   std::vector<ProfileMiss> profile_misses;   // of the last dnnf_plan, one per distinct signature
   int profile_hits = 0;

@@ -26,6 +26,7 @@ int run_blocks(Graph& g, int only, void* stream) {
   if (!g.planned) { g.err = "graph is not planned (or the plan is not runnable)"; return DNNF_ERR_STATE; }
   if (g.ws_bytes > 256 && !g.ws_ptr) { g.err = "workspace not bound"; return DNNF_ERR_WORKSPACE; }
   cudaStream_t st = (cudaStream_t)stream;
+  g.last_status_base = g.ws_ptr;
   // Resolve every pointer first so that a failure launches nothing.
   for (int bi : g.run_order) {
     if (only >= 0 && bi != only) continue;
@@ -144,9 +145,10 @@ int profile_measure(Graph& g, void* scratch, size_t scratch_bytes, void* stream,
 int read_status(Graph& g, int* status, int* block) {
   *status = 0;
   if (block) *block = -1;
-  if (!g.ws_ptr) return DNNF_OK;
+  void* base = g.last_status_base ? g.last_status_base : g.ws_ptr;
+  if (!base) return DNNF_OK;
   int words[2] = {0, 0};
-  if (cudaMemcpy(words, g.ws_ptr, sizeof words, cudaMemcpyDeviceToHost) != cudaSuccess) { g.err = "status read failed"; return DNNF_ERR_CUDA; }
+  if (cudaMemcpy(words, base, sizeof words, cudaMemcpyDeviceToHost) != cudaSuccess) { g.err = "status read failed"; return DNNF_ERR_CUDA; }
   *status = words[0];
   if (block) *block = words[0] ? words[1] : -1;
   return DNNF_OK;

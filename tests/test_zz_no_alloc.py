@@ -12,7 +12,7 @@ import pytest
 from paper_2108_13342_b200 import binding as B
 from paper_2108_13342_b200 import workloads as W
 from paper_2108_13342_b200.runtime import Session
-from util import RTOL_F32, close
+from util import RTOL_BF16, RTOL_F32, close
 
 pytestmark = pytest.mark.gpu
 
@@ -21,10 +21,13 @@ def _outputs(sess):
     return {n: sess.output(n) for n in sess.desc.outputs}
 
 
-@pytest.mark.parametrize("make", [lambda: W.add_layernorm_gelu(rows=64, hidden=768),
-                                  lambda: W.swish_transpose(n=2, c=64, h=12, w=20)],
-                         ids=["add_layernorm_gelu", "swish_transpose"])
-def test_static_workspace_matches_caller_workspace_twice(make):
+@pytest.mark.parametrize("make,rtol", [(lambda: W.add_layernorm_gelu(rows=64, hidden=768), RTOL_F32),
+                                       (lambda: W.swish_transpose(n=2, c=64, h=12, w=20), RTOL_F32),
+                                       # tensor-core blocks: their TMA descriptors must follow the intermediates into the
+                                       # built-in array, and the split-K arrival counters live in its cleared header
+                                       (lambda: W.ffn_block(m=1024, hidden=768, ffn=3072), RTOL_BF16)],
+                         ids=["add_layernorm_gelu", "swish_transpose", "ffn_block_gemm"])
+def test_static_workspace_matches_caller_workspace_twice(make, rtol):
     import torch
     wl = make()
     # one kernel per operator: every intermediate goes through the workspace
@@ -38,11 +41,23 @@ def test_static_workspace_matches_caller_workspace_twice(make):
     for call in range(2):
         for n in s.desc.outputs:
             s.buffers[n].fill_(float("nan"))          # a stale result cannot pass
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         s.g.run_static_ws(stream)
+        torch.cuda.synchronize()
+        if call == 1:                                 # the first call on a device may load the kernels' code
+            assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the amount of free device memory"
+        assert s.g.status() == (0, -1)                # read from the built-in array, where this run kept its status words
         got = _outputs(s)
         for n in want:
-            close(got[n], want[n], RTOL_F32)
-            assert np.array_equal(got[n], want[n]), f"call {call}: {n} differs from dnnf_run"
+            close(got[n], want[n], rtol)
+            if rtol == RTOL_F32:
+                assert np.array_equal(got[n], want[n]), f"call {call}: {n} differs from dnnf_run"
+    # the caller's own workspace is still bound and still works
+    s.run()
+    assert s.g.status() == (0, -1)
+    for n in want:
+        close(s.output(n), want[n], rtol)
 
 
 def test_static_workspace_rejects_plans_that_do_not_fit():
