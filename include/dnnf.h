@@ -147,6 +147,18 @@ typedef struct {
 #define DNNF_PLAN_STRICT_TABLE3     2u   /* type a broadcast operand's consumer One-to-Many on every edge */
 #define DNNF_PLAN_ALLOW_PROLOGUE    4u   /* planning only: let One-to-One predecessors fuse in front of a
                                             GEMM/conv anchor (Listing 1 literal); such plans cannot be run */
+/* Kernel-selection overrides.  The plan, its blocks and the results stay the same; a block is only lowered to another
+ * kernel of its family.  They exist so that every kernel, including the ones the planner rarely picks, can be
+ * tested and timed through this interface; the library reads no environment variable. */
+#define DNNF_PLAN_SPLIT_ALWAYS      0x100u   /* cut fp32 contractions into K slices / column blocks wherever that is possible,
+                                                not only where the cost model says it pays */
+#define DNNF_PLAN_NO_K_SLICES       0x200u   /* never cut an fp32 contraction along K */
+#define DNNF_PLAN_NO_COLUMN_BLOCKS  0x400u   /* never cut an fp32 contraction into column blocks */
+#define DNNF_PLAN_NO_TF32_GEMM      0x800u   /* fp32 contractions on the FMA pipes instead of split-TF32 tensor-core kernels */
+#define DNNF_PLAN_NO_PAIR_GEMM      0x1000u  /* bf16 GEMM blocks without the CTA-pair kernel */
+#define DNNF_PLAN_NO_SPLIT_K        0x2000u  /* bf16 GEMM blocks without a split over K */
+#define DNNF_PLAN_NO_TMA_DWCONV     0x4000u  /* depthwise convolutions without the TMA-tiled kernel */
+#define DNNF_PLAN_NO_TILE_GEMM      0x8000u  /* bf16 GEMM blocks without the one-tile-per-CTA kernel */
 
 typedef struct {
   int32_t ops_before, ops_after;

@@ -18,6 +18,19 @@ def sources():
     return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cpp")))
 
 
+def _deps_of(obj, src):
+    """Headers the object was built from (the compiler's dependency file of the last build); every header if unknown."""
+    dfile = obj + ".d"
+    if os.path.exists(dfile) and os.path.exists(obj) and os.path.getmtime(dfile) >= os.path.getmtime(obj) - 600:
+        with open(dfile) as f:
+            words = f.read().replace("\\\n", " ").split()
+        deps = [w for w in words[1:] if not w.endswith(":") and (w.startswith(HERE) or w.startswith(os.path.join(HERE, "..")) or not os.path.isabs(w))]
+        if deps:
+            return [src] + deps
+    return [src] + [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))] + \
+           [os.path.join(HERE, "..", "include", "dnnf.h")]
+
+
 def needs_build():
     if not os.path.exists(LIB):
         return True
@@ -36,11 +49,10 @@ def build(force=False, verbose=False):
     for src in sources():
         obj = os.path.join(odir, os.path.basename(src) + ".o")
         objs.append(obj)
-        deps = [src] + [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))] + \
-               [os.path.join(HERE, "..", "include", "dnnf.h")]
-        if not force and os.path.exists(obj) and all(os.path.getmtime(obj) > os.path.getmtime(d) for d in deps):
+        deps = _deps_of(obj, src)
+        if not force and os.path.exists(obj) and all(os.path.exists(d) and os.path.getmtime(obj) > os.path.getmtime(d) for d in deps):
             continue
-        cmd = [NVCC, *FLAGS, "-x", "cu", "-c", src, "-o", obj]
+        cmd = [NVCC, *FLAGS, "-MMD", "-MF", obj + ".d", "-x", "cu", "-c", src, "-o", obj]
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     log = []
     for src, p in procs:

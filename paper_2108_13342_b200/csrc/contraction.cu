@@ -28,6 +28,12 @@ void tc2_gemm_plan(Launch& L);
 bool tc2_gemm_prepare(Launch& L, std::string& err);
 int tc2_gemm_launch(const Launch& L, cudaStream_t st);
 void tc2_set_scratch(Launch& L, void* ws_base);
+size_t tile_blob_bytes();
+bool tile_gemm_eligible(const GemmParams& gp);
+bool tile_gemm_preferred(const GemmParams& gp);
+void tile_gemm_plan(Launch& L);
+bool tile_gemm_prepare(Launch& L, std::string& err);
+int tile_gemm_launch(const Launch& L, cudaStream_t st);
 size_t tf32_blob_bytes();
 bool tf32_gemm_eligible(const GemmParams& gp);
 void tf32_gemm_plan(Launch& L);
@@ -267,7 +273,7 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
 
   Launch& L = out.launch;
   L = Launch{};
-  L.blob.assign(sizeof(GemmParams) + sizeof(GemmTcParams) + std::max(tc2_blob_bytes(), tf32_blob_bytes()), 0);
+  L.blob.assign(sizeof(GemmParams) + sizeof(GemmTcParams) + std::max({tc2_blob_bytes(), tf32_blob_bytes(), tile_blob_bytes()}), 0);
   GemmParams& gp = gp_of(L);
 
   // ---- operands ----------------------------------------------------------------
@@ -462,7 +468,9 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
   L.flops = 2ll * gp.M * gp.N * gp.K * (fold_batch ? 1 : nbatch);
   L.family = A.kind == DNNF_OP_CONV1X1 ? DNNF_FAMILY_CONV1X1 : DNNF_FAMILY_GEMM;
 
-  if (tc2_gemm_eligible(gp)) {
+  if (tile_gemm_eligible(gp) && (tile_gemm_preferred(gp) || !tc2_gemm_eligible(gp))) {
+    tile_gemm_plan(L);
+  } else if (tc2_gemm_eligible(gp)) {
     tc2_gemm_plan(L);
   } else if (tc_gemm_eligible(gp)) {
     L.variant = 1;
@@ -488,14 +496,14 @@ void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vecto
   gp.A.ptr = ip[0]; gp.B.ptr = ip[1];
   for (int i = 0; i < gp.n_in; ++i) gp.in[i].ptr = ip[2 + i];
   for (int i = 0; i < gp.n_out; ++i) gp.out[i].ptr = op[i];
-  if (L.variant != 1 && L.variant != 3 && L.variant != 4) return;
+  if (L.variant != 1 && L.variant != 3 && L.variant != 4 && L.variant != 5) return;
   // The tensor maps embed addresses: encode them again whenever ANY pointer of the block differs from the
   // ones they were made for (an epilogue operand in any position may be read through a map).
   std::vector<void*> now(ip);
   now.insert(now.end(), op.begin(), op.end());
   if (L.tc_ready && now == L.encoded_ptrs) return;
   L.tc_ready = false;
-  bool ok = L.variant == 1 ? tc_gemm_prepare(L, err) : L.variant == 3 ? tc2_gemm_prepare(L, err) : tf32_gemm_prepare(L, err);
+  bool ok = L.variant == 1 ? tc_gemm_prepare(L, err) : L.variant == 3 ? tc2_gemm_prepare(L, err) : L.variant == 5 ? tile_gemm_prepare(L, err) : tf32_gemm_prepare(L, err);
   if (ok) { L.tc_ready = true; L.encoded_ptrs = now; }
   else if (err.empty()) err = "cannot encode the tensor maps of a contraction block";
 }
@@ -505,7 +513,7 @@ int launch_contraction(const Launch& L, void* status_words, int block_index, cud
   if (L.family == DNNF_FAMILY_POOL) { int rc = pool_launch(L, status_words, st); if (rc) err = "pooling launch failed"; return rc; }
   if (L.family == DNNF_FAMILY_DWCONV) { int rc = dwconv_launch(L, status_words, block_index, st); if (rc) err = "depthwise convolution launch failed"; return rc; }
   if (L.variant == 2) { int rc = conv1x1_direct_launch(L, st); if (rc) err = "pointwise convolution launch failed"; return rc; }
-  if ((L.variant == 1 || L.variant == 3 || L.variant == 4) && !L.tc_ready) { err = "tensor maps of the block are not encoded"; return 1; }
+  if ((L.variant == 1 || L.variant == 3 || L.variant == 4 || L.variant == 5) && !L.tc_ready) { err = "tensor maps of the block are not encoded"; return 1; }
   GemmParams gp = gp_of(L);
   gp.status = reinterpret_cast<int32_t*>(status_words);
   gp.block_index = block_index;
@@ -515,6 +523,13 @@ int launch_contraction(const Launch& L, void* status_words, int block_index, cud
     tc2_set_scratch(M, status_words);
     int rc = tc2_gemm_launch(L, st);
     if (rc) err = "tensor-core pair GEMM launch failed";
+    return rc;
+  }
+  if (L.variant == 5) {
+    Launch& M = const_cast<Launch&>(L);
+    gp_of(M).status = gp.status; gp_of(M).block_index = block_index;
+    int rc = tile_gemm_launch(L, st);
+    if (rc) err = "tensor-core tile GEMM launch failed";
     return rc;
   }
   if (L.variant == 4) {

@@ -206,7 +206,7 @@ size_t dwconv_tma_blob_bytes() { return sizeof(dwt::Params); }
 
 // Picks the tile; false when the shape does not suit this kernel.
 bool dwconv_tma_plan(Launch& L) {
-  if (getenv("DNNF_NO_TMA_DWCONV")) return false;
+  if (plan_flag(DNNF_PLAN_NO_TMA_DWCONV)) return false;
   const DwParams& dp = dw_of(L);
   dwt::Params& q = tq_of(L);
   if (dp.C % 4 || dp.H < 4 || dp.W < 4) return false;

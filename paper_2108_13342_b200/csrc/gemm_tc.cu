@@ -134,7 +134,7 @@ gemm_tc_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Gem
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         for (int kt = 0; kt < k_tiles; ++kt) {
           if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
-          tc_fence_after();
+          // (no tcgen05 fence: TMA wrote the operands and the barrier orders its completion before the MMAs' reads)
 #pragma unroll
           for (int kk = 0; kk < TC_BK / 16; ++kk)
             tc_mma_bf16(d_tmem, da_s + 2 * kk, db_s + dbk * kk, idesc, (kt | kk) ? 1u : 0u);
@@ -300,7 +300,7 @@ void tc_gemm_plan(Launch& L) {
   L.smem = (size_t)stages * stage_bytes + kSmemFixed;
   L.variant = 1;
   L.static_id = StaticSet<EpiStatic>::find(gp.prog);
-  tc.debug = getenv("DNNF_GEMM_DEBUG") ? atoi(getenv("DNNF_GEMM_DEBUG")) : 0;
+  tc.debug = dev_env("DNNF_GEMM_DEBUG") ? atoi(dev_env("DNNF_GEMM_DEBUG")) : 0;
 }
 
 // dims innermost first: {inner, outer, b0, b1}

@@ -27,30 +27,16 @@
 #include <cstdlib>
 #include <mutex>
 
-#include "chain.cuh"
-#include "gemm_params.h"
 #include "ir.h"
+#include "tc2_common.cuh"
 #include "tma_host.h"
 
 namespace dnnf {
 
 namespace tc2 {
 
-#ifdef DNNF_TRACE
-#define T2ACC(slot, v) do { if (blockIdx.x == 0 && p.status) atomicAdd(reinterpret_cast<unsigned long long*>(p.status) + 4 + (slot), (unsigned long long)(v)); } while (0)
-#else
-#define T2ACC(slot, v) do {} while (0)
-#endif
-
-constexpr int BM = 128, BK = 64, EPI_WARPS = 8, THREADS = 64 + 32 * EPI_WARPS;
-constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // 1 s
-constexpr int kSmemMax = 227 * 1024;
-constexpr int kChunkBytes = 32 * 128;                        // 32 rows x 64 bf16
-constexpr int kBiasFloats = 128;                             // per warp, per row-invariant operand
-constexpr int kMaxVec = 2;                                   // row-invariant operands staged in shared memory
-constexpr int kEpiBytes = EPI_WARPS * (2 * kChunkBytes + kMaxVec * kBiasFloats * 4);
-constexpr int kFixed = 1024 + 512 + kEpiBytes;               // alignment slack + barriers + epilogue buffers
-constexpr int kRingBudget = kSmemMax - kFixed;
+constexpr int kProducer2 = 2 + EPI_WARPS;       // the second producer warp sits behind the epilogue warps
+constexpr int kThreads2 = THREADS + 32;
 
 struct Params {
   CUtensorMap tmA, tmB, tmD, tmC;
@@ -65,154 +51,8 @@ struct Params {
   int32_t* counters;         // split-K arrival counters, one per unit (a warp's 32 x 64 chunk); zero between runs
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
-__device__ __forceinline__ uint32_t mapa(uint32_t saddr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// arrive on a barrier that lives in another CTA of the cluster (address from mapa)
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long wall_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-// Bounded wait: gives up after kWaitLimitNs of wall-clock time (or as soon as another role of the
-// CTA gave up), sets the CTA's abort flag and returns false.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try(bar, parity)) return true;
-  const unsigned long long t0 = wall_ns();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 64; ++i) if (mbar_try(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (wall_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
-  }
-}
-// Operand load of a CTA pair: the bytes land in THIS CTA's shared memory, the completion is
-// counted on the LEADER's barrier (cluster address), so the MMA thread waits on one barrier only.
-__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* tm, uint32_t leader_bar, int c0, int c1) {
-  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-               ::"r"(smem_u32(dst)), "l"(tm), "r"(leader_bar), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, uint64_t* bar, int c0, int c1) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-               ::"r"(smem_u32(dst)), "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, const void* src, int c0, int c1) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-               ::"l"(tm), "r"(smem_u32(src)), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// completion of all MMAs issued so far arrives on one barrier, given by its cluster address
-__device__ __forceinline__ void tc_commit2(uint32_t cluster_addr) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void tc_mma2(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
-  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
-               ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-                 "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]),
-                 "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]),
-                 "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-               : "r"(taddr));
-}
-__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-  d |= 1ull << 46;
-  d |= 2ull << 61;          // SWIZZLE_128B
-  return d;
-}
-
-// Epilogue IO on 32 consecutive columns of the thread's own row (TMEM layout: lane = row).
-// Chunk buffer: 32 rows x 128 B, 128-byte swizzle: the 16-byte piece j of row r sits at
-// r*128 + ((j ^ (r & 7)) * 16).
-struct EpiIO {
-  static constexpr int VV = 32;
-  const GemmParams& p;
-  float accv[32];
-  uint8_t* chunk;            // this warp's current chunk buffer
-  const float* vec_s;        // staged row-invariant operands: [kMaxVec][kBiasFloats]
-  int lane;
-  int col_in_chunk;          // 0 or 32: which half of the 64-column chunk
-  int col_in_half;           // column offset inside this warp's half of the tile (for vec_s)
-  int c_input;
-  __device__ __forceinline__ void load(int idx, float (&dst)[VV]) const {
-    const TensorArg& a = p.in[idx];
-    if (idx == c_input) {                      // full-tile operand, prefetched by TMA into the chunk buffer
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int piece = (col_in_chunk >> 3) + j;
-        uint4 w = *reinterpret_cast<const uint4*>(chunk + lane * 128 + ((piece ^ (lane & 7)) << 4));
-        float* d = &dst[8 * j];
-        d[0] = __uint_as_float(w.x << 16); d[1] = __uint_as_float(w.x & 0xffff0000u);
-        d[2] = __uint_as_float(w.y << 16); d[3] = __uint_as_float(w.y & 0xffff0000u);
-        d[4] = __uint_as_float(w.z << 16); d[5] = __uint_as_float(w.z & 0xffff0000u);
-        d[6] = __uint_as_float(w.w << 16); d[7] = __uint_as_float(w.w & 0xffff0000u);
-      }
-      return;
-    }
-    // row-invariant operand from shared memory (every lane reads the same words: broadcast)
-    const float* s = vec_s + a.mode * kBiasFloats + col_in_half;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      float4 w = *reinterpret_cast<const float4*>(s + 4 * j);
-      dst[4 * j] = w.x; dst[4 * j + 1] = w.y; dst[4 * j + 2] = w.z; dst[4 * j + 3] = w.w;
-    }
-  }
-  __device__ __forceinline__ void anchor(float (&dst)[VV]) const {
-#pragma unroll
-    for (int v = 0; v < VV; ++v) dst[v] = accv[v];
-  }
-  __device__ __forceinline__ void store(int, const float (&val)[VV]) const {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int piece = (col_in_chunk >> 3) + j;
-      __nv_bfloat162 a0 = __floats2bfloat162_rn(val[8 * j], val[8 * j + 1]), a1 = __floats2bfloat162_rn(val[8 * j + 2], val[8 * j + 3]);
-      __nv_bfloat162 a2 = __floats2bfloat162_rn(val[8 * j + 4], val[8 * j + 5]), a3 = __floats2bfloat162_rn(val[8 * j + 6], val[8 * j + 7]);
-      uint4 w = make_uint4(*reinterpret_cast<uint32_t*>(&a0), *reinterpret_cast<uint32_t*>(&a1), *reinterpret_cast<uint32_t*>(&a2),
-                           *reinterpret_cast<uint32_t*>(&a3));
-      *reinterpret_cast<uint4*>(chunk + lane * 128 + ((piece ^ (lane & 7)) << 4)) = w;
-    }
-  }
-  __device__ __forceinline__ void row_reduce(int, float (&)[VV]) const {}
-};
-
 template <class SP>
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(kThreads2, 1)
 gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Params q) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -255,11 +95,15 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
   const int n_tiles = q.total_tiles, k_tiles = q.k_tiles, tiles_n = q.tiles_n;
   const int total = n_tiles * q.ksplit;        // work items: (tile, K slice); item = slice * n_tiles + tile
 
-  if (warp == 0) {
+  if (warp == 0 || warp == kProducer2) {
     if (lane == 0) {
-      // ---------------- TMA producer (both CTAs): own 128 rows of A, own half of B ----------------
+      // ---------------- TMA producers (both CTAs): own 128 rows of A, own half of B ----------------
+      // Two producer threads take alternate ring stages: a stage costs its producer a wait, an expect and three or four
+      // TMA requests at 50 to 80 ns each, more than the MMA thread spends on it.
       // (stage index and phase advance by increments: a division by the run-time stage count costs this
       // single thread some 200 cycles of dependent instructions per k-tile)
+      const uint32_t mine = warp == 0 ? 0u : 1u;
+      uint32_t turn = 0;
       int s = 0; uint32_t ph = 0;
       bool ok = true;
       for (int item = pair; item < total && ok; item += n_pairs) {
@@ -267,20 +111,22 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
         const int tm = (int)fd_div((uint32_t)tile, q.fd_tiles_n), tn = tile - tm * tiles_n;
         const int m0 = tm * 256 + (int)rank * BM, n0 = tn * BN + (int)rank * HB;
         const int kt_end = min(k_tiles, (ks + 1) * q.kt_per);
-        for (int kt = ks * q.kt_per; kt < kt_end; kt += kpack) {
-          { long long t0 = clock64(); if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_flag)) { ok = false; break; } T2ACC(0, clock64() - t0); }
-          const uint32_t lbar = mapa(smem_u32(&full_bar[s]), 0);
-          if (leader) mbar_expect_tx(&full_bar[s], 2 * stage_bytes);
-          // (a k-tile past K, when k_tiles is odd and kpack is 2, arrives as zeros: its MMAs add nothing)
-          for (int u = 0; u < kpack; ++u) {
-            uint8_t* sa = smem + (size_t)s * stage_bytes + (size_t)u * sub_bytes;
-            uint8_t* sb = sa + a_bytes;
-            const int k0 = (kt + u) * BK;
-            tma_load_2d_pair(sa, &q.tmA, lbar, k0, m0);
-            if (q.b_kmajor) {
-              tma_load_2d_pair(sb, &q.tmB, lbar, k0, n0);
-            } else {
-              for (int j = 0; j < HB / 64; ++j) tma_load_2d_pair(sb + j * (64 * BK * 2), &q.tmB, lbar, n0 + j * 64, k0);
+        for (int kt = ks * q.kt_per; kt < kt_end; kt += kpack, turn ^= 1u) {
+          if (turn == mine) {
+            { long long t0 = clock64(); if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_flag)) { ok = false; break; } T2ACC(0, clock64() - t0); }
+            const uint32_t lbar = mapa(smem_u32(&full_bar[s]), 0);
+            if (leader) mbar_expect_tx(&full_bar[s], 2 * stage_bytes);
+            // (a k-tile past K, when k_tiles is odd and kpack is 2, arrives as zeros: its MMAs add nothing)
+            for (int u = 0; u < kpack; ++u) {
+              uint8_t* sa = smem + (size_t)s * stage_bytes + (size_t)u * sub_bytes;
+              uint8_t* sb = sa + a_bytes;
+              const int k0 = (kt + u) * BK;
+              tma_load_2d_pair(sa, &q.tmA, lbar, k0, m0);
+              if (q.b_kmajor) {
+                tma_load_2d_pair(sb, &q.tmB, lbar, k0, n0);
+              } else {
+                for (int j = 0; j < HB / 64; ++j) tma_load_2d_pair(sb + j * (64 * BK * 2), &q.tmB, lbar, n0 + j * 64, k0);
+              }
             }
           }
           if (++s == stages) { s = 0; ph ^= 1; }
@@ -296,24 +142,28 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
         uint32_t tcount = 0;
         int s = 0; uint32_t ph = 0;
         bool ok = true;
+        TR(long long r_tempty = 0, r_wait = 0, r_mma = 0, r_commit = 0, r_n = 0);
         // descriptors of stage 0; a stage further on adds stage_bytes / 16 to the address field, a k-step 2 (32 bytes)
         // or, for an MN-major B, 128 (2048 bytes); the barriers' cluster addresses are 8 bytes apart
         const uint64_t da0 = make_desc(smem_u32(smem), 16, 1024);
         const uint64_t db0 = q.b_kmajor ? make_desc(smem_u32(smem) + a_bytes, 16, 1024) : make_desc(smem_u32(smem) + a_bytes, 64 * BK * 2, 1024);
         const uint64_t dstage = stage_bytes >> 4, dsub = sub_bytes >> 4, dbk = q.b_kmajor ? 2 : 128;
-        const uint32_t e0 = mapa(smem_u32(&empty_bar[0]), 0), e1 = mapa(smem_u32(&empty_bar[0]), 1);
+        const uint32_t e_local = smem_u32(&empty_bar[0]);
         uint64_t da_s = da0, db_s = db0;
         for (int item = pair; item < total && ok; item += n_pairs, ++tcount) {
           const int acc = tcount & 1;
           const uint32_t aph = (tcount >> 1) & 1;
-          { long long t0 = clock64(); if (!mbar_wait(&tempty_bar[acc], aph ^ 1, abort_flag)) { ok = false; break; } T2ACC(1, clock64() - t0); }
+          { long long t0 = clock64(); if (!mbar_wait(&tempty_bar[acc], aph ^ 1, abort_flag)) { ok = false; break; } TR(r_tempty += clock64() - t0); }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
           const int ks = (int)fd_div((uint32_t)item, q.fd_tiles);
           const int kt_begin = ks * q.kt_per, kt_end = min(k_tiles, kt_begin + q.kt_per);
           for (int kt = kt_begin; kt < kt_end; kt += kpack) {
-            { long long t0 = clock64(); if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; } T2ACC(2, clock64() - t0); T2ACC(3, 1); }
-            tc_fence_after();
+            TR(const long long t0 = clock64());
+            if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
+            TR(const long long t1 = clock64());
+            // (no tcgen05 fence here: the operands were written by TMA, and the barrier orders its completion before
+            // the MMAs' reads.  Every instruction of this thread that goes to an asynchronous unit costs 50 to 80 ns.)
 #pragma unroll
             for (int kk = 0; kk < BK / 16; ++kk)
               tc_mma2(d_tmem, da_s + 2 * kk, db_s + dbk * kk, idesc, ((kt - kt_begin) | kk) ? 1u : 0u);
@@ -322,18 +172,20 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
               for (int kk = 0; kk < BK / 16; ++kk)
                 tc_mma2(d_tmem, da_s + dsub + 2 * kk, db_s + dsub + dbk * kk, idesc, 1u);
             }
-            // stage free in both CTAs once these MMAs have read it.  (Relaying the peer's signal through a helper
-            // warp instead of a second commit was measured: the extra hop starves the peer's producer, 40 % slower.)
-            tc_commit2(e0 + 8u * (uint32_t)s);
-            tc_commit2(e1 + 8u * (uint32_t)s);
+            // stage free in both CTAs once these MMAs have read it: ONE commit, delivered to the barrier at this offset
+            // in both CTAs of the pair.
+            TR(const long long t2 = clock64());
+            tc_commit2_both(e_local + 8u * (uint32_t)s);
+            TR(const long long t3 = clock64(); r_wait += t1 - t0; r_mma += t2 - t1; r_commit += t3 - t2; r_n += 1);
             da_s += dstage; db_s += dstage;
             if (++s == stages) { s = 0; ph ^= 1; da_s = da0; db_s = db0; }
           }
-          if (ok) { tc_commit2(mapa(smem_u32(&tfull_bar[acc]), 0)); tc_commit2(mapa(smem_u32(&tfull_bar[acc]), 1)); }
+          if (ok) tc_commit2_both(smem_u32(&tfull_bar[acc]));
         }
+        TR(if (blockIdx.x == 0 && p.status) { long long* t = reinterpret_cast<long long*>(p.status) + 4; t[10] = r_tempty; t[11] = r_wait; t[12] = r_mma; t[13] = r_commit; t[14] = r_n; t[15] = clock64() - t_begin; });
       }
     }
-  } else {
+  } else if (warp < 2 + EPI_WARPS) {
     // ---------------- epilogue warps (both CTAs) ----------------
     const int ew = warp - 2, sub = warp & 3, half = ew >> 2;
     uint8_t* cbuf = epi + ew * (2 * kChunkBytes);
@@ -487,22 +339,6 @@ gemm_tc2_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ Pa
 
 }  // namespace tc2
 
-// ---- static epilogue programs (same tables as the single-CTA kernel) -------------------------------
-#define MO(o, s, i) MicroOp{o, s, i, 0}
-DNNF_SP_BEGIN(E2_Store, 2) MO(M_MOV, S_ANCHOR, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-DNNF_SP_BEGIN(E2_Bias, 3) MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-DNNF_SP_BEGIN(E2_BiasGeluTanh, 4) MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_GELU_TANH, S_NONE, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-DNNF_SP_BEGIN(E2_BiasResidual, 4) MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-DNNF_SP_BEGIN(E2_BiasGeluPrimitives, 9)
-  MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_SAVE, S_TMP, 0), MO(M_MUL, S_CONST, 0), MO(M_ERF, S_NONE, 0), MO(M_ADD, S_CONST, 1),
-  MO(M_MUL, S_TMP, 0), MO(M_MUL, S_CONST, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-DNNF_SP_BEGIN(E2_BiasGeluTanhPrimitives, 13)
-  MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_SAVE, S_TMP, 0), MO(M_SQUARE, S_NONE, 0), MO(M_MUL, S_TMP, 0), MO(M_MUL, S_CONST, 0),
-  MO(M_ADD, S_TMP, 0), MO(M_MUL, S_CONST, 1), MO(M_TANH, S_NONE, 0), MO(M_ADD, S_CONST, 2), MO(M_MUL, S_TMP, 0), MO(M_MUL, S_CONST, 3),
-  MO(M_STORE, S_NONE, 0) DNNF_SP_END
-#undef MO
-using Epi2Static = TypeList<E2_Store, E2_Bias, E2_BiasGeluTanh, E2_BiasResidual, E2_BiasGeluPrimitives, E2_BiasGeluTanhPrimitives>;
-
 // ---- host side --------------------------------------------------------------------------------------
 static GemmParams& gp_of(Launch& L) { return *reinterpret_cast<GemmParams*>(L.blob.data()); }
 static const GemmParams& gp_of(const Launch& L) { return *reinterpret_cast<const GemmParams*>(L.blob.data()); }
@@ -516,7 +352,7 @@ bool tc_gemm_eligible(const GemmParams& gp);
 // The pair kernel takes plain 2-D problems whose epilogue operands and result are row-major
 // matrices over (m, n): one bf16 output, at most one bf16 full-tile input, row-invariant others.
 bool tc2_gemm_eligible(const GemmParams& gp) {
-  if (getenv("DNNF_NO_PAIR_GEMM")) return false;
+  if (plan_flag(DNNF_PLAN_NO_PAIR_GEMM)) return false;
   if (!tc_gemm_eligible(gp)) return false;
   if (gp.batch_ext[0] * gp.batch_ext[1] != 1) return false;
   if (gp.M < 256 || gp.N < 128) return false;
@@ -550,7 +386,7 @@ void tc2_gemm_plan(Launch& L) {
     double eff = (double)tiles / (waves * 74.0) * useful;
     if (eff > best + 1e-9) { best = eff; best_bn = bn; }
   }
-  if (getenv("DNNF_PAIR_BN")) best_bn = atoi(getenv("DNNF_PAIR_BN"));      // development switch
+  if (dev_env("DNNF_PAIR_BN")) best_bn = atoi(dev_env("DNNF_PAIR_BN"));      // development switch
   q.bn = best_bn;
   q.tiles_n = (gp.N + q.bn - 1) / q.bn;
   q.total_tiles = tiles_m * q.tiles_n;
@@ -561,16 +397,17 @@ void tc2_gemm_plan(Launch& L) {
   // two k-tiles per stage halve the issuing thread's per-stage cost (wait, fence, two commits); worth it when its
   // MMAs are short (BN = 128) or the k loop is long, as long as three stages still fit
   q.kpack = (q.k_tiles >= 4 && tc2::kRingBudget / (2 * sub_bytes) >= 3) ? 2 : 1;
-  if (getenv("DNNF_PAIR_KPACK")) q.kpack = atoi(getenv("DNNF_PAIR_KPACK")) == 2 ? 2 : 1;
+  if (dev_env("DNNF_PAIR_KPACK")) q.kpack = atoi(dev_env("DNNF_PAIR_KPACK")) == 2 ? 2 : 1;
   const int stage_bytes = sub_bytes * q.kpack;
   q.stages = std::min(8, tc2::kRingBudget / stage_bytes);
   // split-K when fewer than half of the 74 CTA pairs would have a tile and the k loop is long.  Handing partial
   // tiles over through L2 costs about 3 us (measured), a k-tile about 0.22 us: it pays from 32 k-tiles up, with
   // two or three slices (1024 x 768 x 3072: 15.7 -> 13.2 us; 1024 x 768 x 768: 7.2 -> 9.2 us, so not there).
   q.ksplit = 1; q.kt_per = q.k_tiles;
-  if (q.total_tiles * 2 <= 74 && q.k_tiles >= 32 && !getenv("DNNF_NO_SPLIT_K")) {
-    int want = std::min(3, 74 / q.total_tiles);
-    if (getenv("DNNF_SPLIT_K")) want = std::max(1, std::min(8, atoi(getenv("DNNF_SPLIT_K"))));
+  {
+    int want = 1;
+    if (q.total_tiles * 2 <= 74 && q.k_tiles >= 32 && !plan_flag(DNNF_PLAN_NO_SPLIT_K)) want = std::min(3, 74 / q.total_tiles);
+    if (dev_env("DNNF_SPLIT_K")) want = std::max(1, std::min(8, atoi(dev_env("DNNF_SPLIT_K"))));
     if (want > 1) {
       int per = (q.k_tiles + want - 1) / want;
       per = (per + q.kpack - 1) / q.kpack * q.kpack;
@@ -592,7 +429,7 @@ void tc2_gemm_plan(Launch& L) {
     else { q.c_input = i; gp.in[i].mode = 0; }
   }
   L.grid = 2 * std::min(q.total_tiles * q.ksplit, 74);
-  L.threads = tc2::THREADS;
+  L.threads = tc2::kThreads2;
   L.smem = (size_t)q.stages * stage_bytes + tc2::kFixed;
   L.variant = 3;
   L.static_id = StaticSet<Epi2Static>::find(gp.prog);
@@ -634,7 +471,7 @@ struct Tc2Launcher {
     static PerDeviceOnce once;       // per instantiation
     if (once.first_use()) cudaFuncSetAttribute(tc2::gemm_tc2_kernel<SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::kSmemMax);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(L.grid); cfg.blockDim = dim3(tc2::THREADS); cfg.dynamicSmemBytes = L.smem; cfg.stream = st;
+    cfg.gridDim = dim3(L.grid); cfg.blockDim = dim3(tc2::kThreads2); cfg.dynamicSmemBytes = L.smem; cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;

@@ -588,7 +588,7 @@ static int tf32_b_bytes(const GemmParams& gp) { return tf32_b_bytes_of(gp.N, gp.
 // The part of the eligibility test that depends on the problem's shape alone (the planner asks it before it
 // splits a contraction that is too deep into several that fit).
 bool tf32_shape_fits(int64_t M, int64_t N, int64_t K) {
-  if (getenv("DNNF_NO_TF32_GEMM")) return false;
+  if (plan_flag(DNNF_PLAN_NO_TF32_GEMM)) return false;
   if (K < 1 || K > 244) return false;                        // a whole row of A (padded) must fit one TMA box of 256 floats
   if (N < 1 || N > 192 || M < 4 * tf32::BM) return false;    // two accumulator stages and two A stages must fit in 512 TMEM columns
   if (tf32_b_bytes_of((int)N, (int)K) > tf32::kMaxBBytes) return false;
@@ -631,12 +631,12 @@ void tf32_gemm_plan(Launch& L) {
   q.k_chunks = (gp.K + tf32::BK - 1) / tf32::BK;
   q.npad = tf32_npad(gp.N);
   // tensor memory: two accumulator stages (twice as wide in the dual form) and at least two A stages must fit 512 columns
-  q.dual = 4 * q.npad + 2 * tf32::kAStageCols <= 512 && !getenv("DNNF_TF32_NO_DUAL");
-  q.fast_epi = fast_epilogue(gp, q.slot) && !getenv("DNNF_TF32_GENERAL_EPILOGUE");
+  q.dual = 4 * q.npad + 2 * tf32::kAStageCols <= 512 && !dev_env("DNNF_TF32_NO_DUAL");
+  q.fast_epi = fast_epilogue(gp, q.slot) && !dev_env("DNNF_TF32_GENERAL_EPILOGUE");
   q.b_static = gp.static_mask & 1u;
   q.fd_n = make_fastdiv((uint32_t)gp.N); q.fd_npad = make_fastdiv((uint32_t)q.npad); q.fd_kpad = make_fastdiv((uint32_t)(q.k_chunks * tf32::BK));
-  q.epi_warps = (gp.N <= 32 && !getenv("DNNF_TF32_EPI8")) ? 4 : 8;
-  q.debug = getenv("DNNF_TF32_DEBUG") ? atoi(getenv("DNNF_TF32_DEBUG")) : 0;
+  q.epi_warps = (gp.N <= 32 && !dev_env("DNNF_TF32_EPI8")) ? 4 : 8;
+  q.debug = dev_env("DNNF_TF32_DEBUG") ? atoi(dev_env("DNNF_TF32_DEBUG")) : 0;
   gp.tiles_m = (gp.M + tf32::BM - 1) / tf32::BM;
   gp.tiles_n = 1;
   q.total_tiles = gp.tiles_m;
@@ -653,7 +653,7 @@ void tf32_gemm_plan(Launch& L) {
   q.a_stages = std::min(4, (512 - 2 * (q.dual ? 2 : 1) * q.npad) / tf32::kAStageCols);
   L.smem = (size_t)tf32_b_bytes(gp) + (size_t)q.stages * q.unit_stride + tf32::kFixed;
   q.b_dense = gp.B.stride_col == 1 && gp.B.stride_row == gp.N && gp.N % 4 == 0 && gp.B.base % 4 == 0 &&
-              (int64_t)gp.K * gp.N * 4 <= tf32::kEpiBytes && !getenv("DNNF_TF32_NO_BULK_B");
+              (int64_t)gp.K * gp.N * 4 <= tf32::kEpiBytes && !dev_env("DNNF_TF32_NO_BULK_B");
   L.variant = 4;
   L.static_id = StaticSet<tf32::Static>::find(gp.prog);
 }

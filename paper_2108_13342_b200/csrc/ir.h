@@ -2,6 +2,7 @@
 // mapping type per operator, IR_removable per tensor and mathematical-property
 // flags; fusion blocks and their lowered launches.
 #pragma once
+#include <cstdlib>
 #include <cstdint>
 #include <map>
 #include <string>
@@ -11,6 +12,21 @@
 #include "microop.h"
 
 namespace dnnf {
+
+// Plan flags of the dnnf_plan call that is being served on this thread (kernel-selection overrides, see dnnf.h).
+extern thread_local uint32_t tl_plan_flags;
+inline bool plan_flag(uint32_t f) { return (tl_plan_flags & f) != 0; }
+
+// Development switches: environment variables that tune or ablate a kernel.  They exist only in libraries built with
+// -DDNNF_DEV_SWITCHES; a normal build never reads the environment.
+inline const char* dev_env(const char* name) {
+#ifdef DNNF_DEV_SWITCHES
+  return getenv(name);
+#else
+  (void)name;
+  return nullptr;
+#endif
+}
 
 struct Attrs {
   double c = 0, lo = 0, hi = 0, p = 0, eps = 1e-5;

@@ -42,8 +42,8 @@ bool finalize_row(Launch& L) {
   // (shorter per-thread chains), with many short rows a warp takes several rows (more loads in flight).
   // 4000 (27 warps per SM): measured best when independent blocks overlap on the GPU, 6 % slower than
   // 148 * 32 for a lone 1024-row launch.
-  static const long target = getenv("DNNF_ROW_TARGET_WARPS") ? atol(getenv("DNNF_ROW_TARGET_WARPS")) : 4000L;
-  static const long split_target = getenv("DNNF_ROW_SPLIT_TARGET") ? atol(getenv("DNNF_ROW_SPLIT_TARGET")) : 4000L;   // (2000 is 3 % better when independent blocks overlap, 20 % worse for a lone 1024-row launch)
+  static const long target = dev_env("DNNF_ROW_TARGET_WARPS") ? atol(dev_env("DNNF_ROW_TARGET_WARPS")) : 4000L;
+  static const long split_target = dev_env("DNNF_ROW_SPLIT_TARGET") ? atol(dev_env("DNNF_ROW_SPLIT_TARGET")) : 4000L;   // (2000 is 3 % better when independent blocks overlap, 20 % worse for a lone 1024-row launch)
   if (V == 4) {
     const int vectors = (Lr + 3) / 4;
     auto fit = [&](int w) { int need = (vectors + 32 * w - 1) / (32 * w); return need; };   // vectors per lane with w warps per row

@@ -46,7 +46,11 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  static const bool pdl_off = getenv("DNNF_NO_PDL") != nullptr;       // development switch
+#ifdef DNNF_DEV_SWITCHES
+  static const bool pdl_off = getenv("DNNF_NO_PDL") != nullptr;
+#else
+  constexpr bool pdl_off = false;
+#endif
   attr[0].val.programmaticStreamSerializationAllowed = pdl_off ? 0 : 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);

@@ -840,6 +840,7 @@ const Program* program_of(const Launch& L) {
 }
 
 int lower_block(const Graph& g, const std::vector<int>& ops_in, uint32_t flags, Block& out, std::string& why) {
+  tl_plan_flags = flags;
   // topological order inside the block
   std::vector<int> ops = ops_in;
   {

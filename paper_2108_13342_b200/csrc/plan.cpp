@@ -33,7 +33,7 @@ struct Planner {
   std::vector<std::vector<int>> blocks;
   std::vector<int> btype;
   int yellow = 0, yellow_fused = 0;
-  bool debug = getenv("DNNF_DEBUG_PLAN") != nullptr;
+  bool debug = dev_env("DNNF_DEBUG_PLAN") != nullptr;
 
   Planner(Graph& gg, uint32_t f) : g(gg), flags(f) {}
 
@@ -359,7 +359,7 @@ bool tf32_shape_fits(int64_t M, int64_t N, int64_t K);
 // on such shapes; a split kernel costs about 9 us of launch, setup and tail, every part reads A again, every slice
 // but the last writes a partial sum that a later one reads.
 static bool split_pays(int64_t M, int64_t N, int64_t K, int64_t parts, int64_t slices) {
-  if (getenv("DNNF_SPLIT_ALWAYS")) return true;      // development switch: the tests use it to reach the split at small sizes
+  if (plan_flag(DNNF_PLAN_SPLIT_ALWAYS)) return true;      // development switch: the tests use it to reach the split at small sizes
   const double unsplit_us = 2.0 * (double)M * (double)N * (double)K / 1e7;
   const double bytes = 4.0 * (double)M * ((double)parts * (double)K + (double)N * (1.0 + 2.0 * (double)(slices - 1)));
   const double split_us = 9.0 * (double)(parts * slices) + bytes / 4e6;
@@ -372,7 +372,7 @@ static bool split_pays(int64_t M, int64_t N, int64_t K, int64_t parts, int64_t s
 // Add joins the next slice's epilogue, so the cost is one extra write and read of the partial sum.  (A lowering
 // decision, not one of the paper's rewriting rules: it is applied to every plan, fused or not.)
 static void split_deep_pointwise(Graph& g, const std::set<int>& decided) {
-  if (getenv("DNNF_NO_K_SPLIT")) return;
+  if (plan_flag(DNNF_PLAN_NO_K_SLICES)) return;
   const size_t n_ops = g.ops.size();
   bool any = false;
   for (size_t oi = 0; oi < n_ops; ++oi) {
@@ -446,7 +446,7 @@ static void split_deep_pointwise(Graph& g, const std::set<int>& decided) {
 // that needs the fewest kernels once the K split below has been applied to the parts as well (at most 32; every part
 // reads x again, but the tiled FMA kernel such a convolution would otherwise run on is slower by an order of magnitude).
 static void split_wide_pointwise(Graph& g, std::set<int>& decided) {
-  if (getenv("DNNF_NO_N_SPLIT") || getenv("DNNF_NO_TF32_GEMM")) return;
+  if (plan_flag(DNNF_PLAN_NO_COLUMN_BLOCKS) || plan_flag(DNNF_PLAN_NO_TF32_GEMM)) return;
   g.relink();
   const size_t n_ops = g.ops.size();
   bool any = false;
@@ -567,7 +567,10 @@ static void split_wide_pointwise(Graph& g, std::set<int>& decided) {
   if (any) g.relink();
 }
 
+thread_local uint32_t tl_plan_flags = 0;
+
 int plan_graph(Graph& g, uint32_t flags) {
+  tl_plan_flags = flags;
   g.relink();
   {
     std::set<int> decided;                  // matrix products made by the column split: their K split is part of that decision

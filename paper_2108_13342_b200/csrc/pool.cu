@@ -240,7 +240,7 @@ int lower_pool(const Graph& g, const std::vector<int>& ops, int anchor, Block& o
   L.grid = (int)((total + 255) / 256);
   L.threads = 256;
   pp.slices = 0;
-  if (pp.kernel * pp.kernel >= 64 && !getenv("DNNF_NO_WIDE_POOL")) {
+  if (pp.kernel * pp.kernel >= 64 && !dev_env("DNNF_NO_WIDE_POOL")) {
     // one thread per output would walk the window alone: give the window to whole CTAs instead
     pp.groups = (dp.C + 127) / 128;
     const int64_t units = (int64_t)dp.N * dp.H * dp.W * pp.groups;

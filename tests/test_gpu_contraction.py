@@ -12,12 +12,9 @@ FUSED, UNFUSED = B.PLAN_FUSED, B.PLAN_UNFUSED
 
 
 
-def _expect_variant(sess, variant, switch):
-    """The block must run on the named kernel variant -- unless the development switch that disables it is set
-    (the suite is also run with those switches to cover the fall-back kernels)."""
-    import os
-    if not os.environ.get(switch):
-        assert sess.g.blocks()[0]["variant"] == variant, sess.g.blocks()
+def _expect_variant(sess, variant):
+    """The block must run on the named kernel variant."""
+    assert sess.g.blocks()[0]["variant"] == variant, sess.g.blocks()
 
 def _bf(x):
     return W.round_to_bf16(x)
@@ -47,14 +44,16 @@ def test_ffn_block(cfg, flags):
     s = check(W.ffn_block(m, hidden, ffn), RTOL_BF16, flags, expect_blocks=2 if flags == FUSED else 6)
     if flags == FUSED:
         assert [b["family"] for b in s.g.blocks()] == ["gemm", "gemm"]
-        assert all(b["variant"] in (1, 3) for b in s.g.blocks()), "expected a tensor-core kernel"
+        assert all(b["variant"] in (1, 3, 5) for b in s.g.blocks()), "expected a tensor-core kernel"
 
 
 @pytest.mark.parametrize("mnk", [(256, 128, 64), (300, 200, 72), (1000, 328, 264), (257, 136, 8), (512, 2304, 768), (512, 128, 448)])
 @pytest.mark.parametrize("kmajor_b", [False, True])
 @pytest.mark.parametrize("epi", ["none", "bias_gelu", "bias_residual"])
-def test_pair_gemm_shapes_and_epilogues(mnk, kmajor_b, epi):
-    """The CTA-pair kernel (M >= 256, N >= 128): ragged edges in M, N and K, both operand layouts for B."""
+@pytest.mark.parametrize("kernel", ["pair", "tile"])
+def test_pair_gemm_shapes_and_epilogues(mnk, kmajor_b, epi, kernel):
+    """The CTA-pair kernel (M >= 256, N >= 128) and the one-tile-per-CTA kernel, which the planner prefers at these
+    sizes: ragged edges in M, N and K, both operand layouts for B."""
     m, n, k = mnk
     g = graph()
     g.ext("A", (m, k), "bf16")
@@ -74,8 +73,8 @@ def test_pair_gemm_shapes_and_epilogues(mnk, kmajor_b, epi):
         g.ext("R", (m, n), "bf16"); ins["R"] = _bf(rnd((m, n), 34, -1, 1))
         t = g.add("Add", [t, "R"])
     g.mark_output(t)
-    s = check(W.Workload(g, ins), RTOL_BF16, FUSED, expect_blocks=1)
-    _expect_variant(s, 3, "DNNF_NO_PAIR_GEMM")
+    s = check(W.Workload(g, ins), RTOL_BF16, FUSED | (B.PLAN_NO_TILE_GEMM if kernel == "pair" else 0), expect_blocks=1)
+    _expect_variant(s, 3 if kernel == "pair" else 5)
 
 
 @pytest.mark.parametrize("mnk", [(4000, 3000, 776), (2304, 2304, 264), (2500, 1104, 264), (8192, 1024, 128), (5000, 1544, 72)])
@@ -101,7 +100,7 @@ def test_pair_gemm_more_tiles_than_cta_pairs(mnk, epi):
     s, got, ref = run_both(wl, FUSED)
     (name,) = wl.graph.outputs
     close(got[name], ref[name], RTOL_BF16)
-    _expect_variant(s, 3, "DNNF_NO_PAIR_GEMM")
+    _expect_variant(s, 3)
     s.buffers[name].fill_(float("nan"))
     s.run()
     close(s.output(name), ref[name], RTOL_BF16)
@@ -132,8 +131,7 @@ def test_pair_gemm_split_k(mnk, epi):
     s, got, ref = run_both(wl, FUSED)
     (name,) = wl.graph.outputs
     close(got[name], ref[name], RTOL_BF16)
-    if not (os.environ.get("DNNF_NO_PAIR_GEMM") or os.environ.get("DNNF_NO_SPLIT_K")):
-        assert s.g.blocks()[0]["variant"] == 3 and s.g.workspace_zero_bytes() > 256, (s.g.blocks(), s.g.workspace_zero_bytes())
+    assert s.g.blocks()[0]["variant"] == 3 and s.g.workspace_zero_bytes() > 256, (s.g.blocks(), s.g.workspace_zero_bytes())
     for _ in range(2):
         s.run()
         close(s.output(name), ref[name], RTOL_BF16)
@@ -212,7 +210,7 @@ def test_conv1x1_tensor_core_fp32(cfg, epi):
             g.ext("R", (n, h, w, co)); ins["R"] = rnd((n, h, w, co), 15, -1, 1)
             g.mark_output(g.add("Add", [e, "R"], out="Y"))
     s = check(W.Workload(g, ins), RTOL_F32, FUSED, expect_blocks=1)
-    _expect_variant(s, 4, "DNNF_NO_TF32_GEMM")
+    _expect_variant(s, 4)
 
 
 def test_matmul_fp32_tall_skinny_uses_tensor_cores():
@@ -223,7 +221,7 @@ def test_matmul_fp32_tall_skinny_uses_tensor_cores():
     t = g.add("Add", [t, "b"])
     g.mark_output(g.add("Tanh", [t], out="Y"))
     s = check(W.Workload(g, {"X": rnd((m, k), 3, -1, 1), "Wt": rnd((k, n), 4, -0.3, 0.3), "b": rnd((n,), 5)}), RTOL_F32, FUSED, expect_blocks=1)
-    _expect_variant(s, 4, "DNNF_NO_TF32_GEMM")
+    _expect_variant(s, 4)
 
 
 def test_matmul_fp32_tall_skinny_transposed_weight_and_second_output():
@@ -238,7 +236,7 @@ def test_matmul_fp32_tall_skinny_transposed_weight_and_second_output():
     g.mark_output(t)
     g.mark_output(g.add("Relu", [t], out="Y"))
     s = check(W.Workload(g, {"X": rnd((m, k), 3, -1, 1), "Wt": rnd((n, k), 4, -0.3, 0.3), "b": rnd((n,), 5)}), RTOL_F32, FUSED, expect_blocks=1)
-    _expect_variant(s, 4, "DNNF_NO_TF32_GEMM")
+    _expect_variant(s, 4)
 
 
 @pytest.mark.parametrize("cfg", [(1, 5, 6, 8), (2, 7, 9, 144), (1, 1, 1, 4), (1, 3, 1, 12), (2, 30, 17, 24)])
@@ -266,7 +264,7 @@ def test_dwconv3x3_tma_tiled(cfg):
     ins = {"X": rnd((n, h, w, c), 21, -1, 1), "Kd": rnd((3, 3, c), 22, -0.5, 0.5), "s": rnd((c,), 23, 0.5, 1.5), "t": rnd((c,), 24, -0.5, 0.5),
            "R": rnd((n, h, w, c), 25, -1, 1)}
     s = check(W.Workload(g, ins), RTOL_F32, FUSED, expect_blocks=1)
-    _expect_variant(s, -1, "DNNF_NO_TMA_DWCONV")
+    _expect_variant(s, -1)
     check(W.Workload(g, ins), RTOL_F32, UNFUSED, expect_blocks=3)
 
 
@@ -323,12 +321,11 @@ def test_encoder_full_size_twelve_layers():
 @pytest.mark.parametrize("flags", [B.PLAN_FUSED, B.PLAN_UNFUSED])
 @pytest.mark.parametrize("nhw,cin,cout,slices", [((2, 32, 32), 256, 64, 2), ((1, 40, 40), 384, 32, 2), ((1, 24, 24), 576, 48, 3),
                                                   ((1, 24, 24), 960, 24, 4), ((2, 16, 16), 248, 40, 2)])
-def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, flags, monkeypatch):
+def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, flags):
     """fp32 pointwise convolutions deeper than the split-TF32 kernel takes (K > 244) are planned as 2-4 tensor-core
     contractions over K slices (as few as fit the kernel's shared memory), the partial sums riding in a later slice's
     epilogue."""
-    import os
-    monkeypatch.setenv("DNNF_SPLIT_ALWAYS", "1")       # the sizes here are below the planner's break-even
+    flags |= B.PLAN_SPLIT_ALWAYS                       # the sizes here are below the planner's break-even
     n, h, w = nhw
     g = graph("deep_pw")
     g.ext("X", (n, h, w, cin)); g.ext("Wt", (cin, cout), kind="weight"); g.ext("s", (cout,)); g.ext("t", (cout,))
@@ -337,37 +334,34 @@ def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, fla
     ins = {"X": rnd((n, h, w, cin), 90, 0.0, 1.0), "Wt": rnd((cin, cout), 91, -0.2, 0.2), "s": rnd((cout,), 92, 0.5, 1.5),
            "t": rnd((cout,), 93, -0.5, 0.5)}
     s = check(W.Workload(g, ins), 2e-5, flags)
-    if not (os.environ.get("DNNF_NO_K_SPLIT") or os.environ.get("DNNF_NO_TF32_GEMM")):
-        gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
-        assert len(gemms) >= slices and all(b["variant"] == 4 for b in gemms), s.g.blocks()
-        assert not [b for b in s.g.blocks() if b["family"] == "conv1x1"], s.g.blocks()
-        assert s.plan_stats.n_ops == 3          # the slices count as the one convolution they came from
+    gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
+    assert len(gemms) >= slices and all(b["variant"] == 4 for b in gemms), s.g.blocks()
+    assert not [b for b in s.g.blocks() if b["family"] == "conv1x1"], s.g.blocks()
+    assert s.plan_stats.n_ops == 3          # the slices count as the one convolution they came from
 
 
 @pytest.mark.parametrize("mnk", [(2048, 64, 512), (700, 100, 300), (4096, 16, 1024)])
-def test_deep_fp32_matrix_product_is_split_along_k(mnk, monkeypatch):
-    import os
-    monkeypatch.setenv("DNNF_SPLIT_ALWAYS", "1")
+def test_deep_fp32_matrix_product_is_split_along_k(mnk):
     m, n, k = mnk
     g = graph("deep_mm")
     g.ext("A", (m, k)); g.ext("Bm", (k, n), kind="weight"); g.ext("b", (n,))
     g.mark_output(g.add("Relu", [g.add("Add", [g.add("MatMul", ["A", "Bm"]), "b"])]))
-    s = check(W.Workload(g, {"A": rnd((m, k), 94, -1.0, 1.0), "Bm": rnd((k, n), 95, -0.2, 0.2), "b": rnd((n,), 96)}), 2e-5)
-    if not (os.environ.get("DNNF_NO_K_SPLIT") or os.environ.get("DNNF_NO_TF32_GEMM")):
-        gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
-        assert len(gemms) >= 2 and all(b["variant"] == 4 for b in gemms), s.g.blocks()
+    s = check(W.Workload(g, {"A": rnd((m, k), 94, -1.0, 1.0), "Bm": rnd((k, n), 95, -0.2, 0.2), "b": rnd((n,), 96)}), 2e-5,
+              B.PLAN_FUSED | B.PLAN_SPLIT_ALWAYS)
+    gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
+    assert len(gemms) >= 2 and all(b["variant"] == 4 for b in gemms), s.g.blocks()
 
 
 @pytest.mark.parametrize("flags", [B.PLAN_FUSED, B.PLAN_UNFUSED])
 @pytest.mark.parametrize("nhw,cin,cout,tail", [((2, 32, 32), 64, 384, "bn_clip_res_relu"), ((1, 40, 40), 96, 200, "bn_clip"),
                                                ((2, 24, 24), 32, 256, "none"), ((1, 32, 32), 24, 240, "bias_two_readers"),
                                                ((3, 16, 16), 48, 512, "prelu")])
-def test_wide_pointwise_convolution_is_split_into_channel_blocks(nhw, cin, cout, tail, flags, monkeypatch):
+def test_wide_pointwise_convolution_is_split_into_channel_blocks(nhw, cin, cout, tail, flags):
     """fp32 pointwise convolutions with more output channels than the split-TF32 kernel's accumulators hold (N > 192) are
     planned as tensor-core contractions over column blocks of W; the channel-wise operators behind the convolution move
     into each block's epilogue and the blocks store straight into the result (parts of a Concat)."""
-    import os
-    monkeypatch.setenv("DNNF_SPLIT_ALWAYS", "1")
+    fused = flags == B.PLAN_FUSED
+    flags |= B.PLAN_SPLIT_ALWAYS
     n, h, w = nhw
     g = graph("wide_pw")
     g.ext("X", (n, h, w, cin)); g.ext("Wt", (cin, cout), kind="weight"); g.ext("s", (cout,)); g.ext("t", (cout,)); g.ext("R", (n, h, w, cout))
@@ -386,12 +380,11 @@ def test_wide_pointwise_convolution_is_split_into_channel_blocks(nhw, cin, cout,
     ins = {"X": rnd((n, h, w, cin), 97, 0.0, 1.0), "Wt": rnd((cin, cout), 98, -0.2, 0.2), "s": rnd((cout,), 99, 0.5, 1.5),
            "t": rnd((cout,), 100, -0.5, 0.5), "R": rnd((n, h, w, cout), 101, -1.0, 1.0)}
     s = check(W.Workload(g, ins), 2e-5, flags)
-    if not (os.environ.get("DNNF_NO_N_SPLIT") or os.environ.get("DNNF_NO_TF32_GEMM")):
-        gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
-        assert len(gemms) >= 2 and all(b["variant"] == 4 for b in gemms), s.g.blocks()
-        assert not [b for b in s.g.blocks() if b["family"] == "conv1x1"], s.g.blocks()
-        if flags == B.PLAN_FUSED and tail in ("bn_clip_res_relu", "bn_clip", "none", "prelu"):
-            assert s.plan_stats.n_kernels == len(gemms), s.g.blocks()      # nothing but the column blocks runs
+    gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
+    assert len(gemms) >= 2 and all(b["variant"] == 4 for b in gemms), s.g.blocks()
+    assert not [b for b in s.g.blocks() if b["family"] == "conv1x1"], s.g.blocks()
+    if fused and tail in ("bn_clip_res_relu", "bn_clip", "none", "prelu"):
+        assert s.plan_stats.n_kernels == len(gemms), s.g.blocks()      # nothing but the column blocks runs
 
 
 def test_split_decision_follows_the_cost_model():

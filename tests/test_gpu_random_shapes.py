@@ -21,9 +21,9 @@ def _pick(seed, i, xs):
     return xs[min(int(_u(seed, i) * len(xs)), len(xs) - 1)]
 
 
-def _run(wl, rtol):
+def _run(wl, rtol, plan_flags=B.PLAN_FUSED):
     ref = O.run_graph(wl.graph, wl.inputs)
-    s = Session(wl, plan_flags=B.PLAN_FUSED, rewrite_flags=B.REWRITE_NONE)
+    s = Session(wl, plan_flags=plan_flags, rewrite_flags=B.REWRITE_NONE)
     s.workspace[s.g.workspace_zero_bytes():].fill_(0xFF)
     for n in wl.graph.outputs:
         s.buffers[n].fill_(float("nan"))
@@ -117,11 +117,11 @@ def test_random_depthwise_and_pointwise_conv(seed):
 
 
 @pytest.mark.parametrize("seed", range(60))
-def test_random_deep_pointwise_conv(seed, monkeypatch):
+def test_random_deep_pointwise_conv(seed):
     """Channel counts beyond what the split-TF32 kernel takes in one pass (K up to 1024): the planner's K slices, with
     slice counts 2-8 or none when K has no suitable divisor, and three kinds of epilogue."""
-    if seed % 3:
-        monkeypatch.setenv("DNNF_SPLIT_ALWAYS", "1")  # most of these sizes are below the planner's break-even for a split
+    # most of these sizes are below the planner's break-even for a split
+    plan_flags = B.PLAN_FUSED | (B.PLAN_SPLIT_ALWAYS if seed % 3 else 0)
     n = _pick(seed, 1, [1, 2, 3])
     h = 8 + int(_u(seed, 2) * 40)
     w = 8 + int(_u(seed, 3) * 40)
@@ -137,7 +137,7 @@ def test_random_deep_pointwise_conv(seed, monkeypatch):
     elif kind == "bn_clip": y = g.add("Clip", [g.add("ScaleShift", [y, "s", "t"], axis=-1)], lo=-1.0, hi=1.0)
     elif kind == "bn_res": y = g.add("Add", [g.add("ScaleShift", [y, "s", "t"], axis=-1), "R"])
     g.mark_output(y)
-    _run(W.Workload(g, ins), 2e-5)
+    _run(W.Workload(g, ins), 2e-5, plan_flags)
 
 
 @pytest.mark.parametrize("seed", range(40))

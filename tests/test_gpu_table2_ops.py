@@ -279,14 +279,12 @@ def test_gather_clamps_indices_outside_the_table():
 
 
 @pytest.mark.parametrize("flags,always", [(B.PLAN_FUSED, False), (B.PLAN_FUSED, True), (B.PLAN_UNFUSED, True)])
-def test_mobilenet_shaped_stack(flags, always, monkeypatch):
+def test_mobilenet_shaped_stack(flags, always):
     """Nine inverted-residual blocks, pooling between the stages, head and classifier: expansions wider than 192 channels
     and projections deeper than 244 go through the planner's column-block and K splits (forced at this small size in two
     of the three variants, decided by the cost model in the first)."""
-    if always:
-        monkeypatch.setenv("DNNF_SPLIT_ALWAYS", "1")
     wl = W.mbconv_stack(n=4, hw=48)
-    s = check(wl, 5e-4, flags, B.REWRITE_DEFAULT)
+    s = check(wl, 5e-4, flags | (B.PLAN_SPLIT_ALWAYS if always else 0), B.REWRITE_DEFAULT)
     fams = [b["family"] for b in s.g.blocks()]
     assert "dwconv" in fams and "pool" in fams
     if always:

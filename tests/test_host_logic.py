@@ -545,11 +545,11 @@ def test_convtranspose_and_gather_recording_and_errors():
         _plan_desc(g)
 
 
-def test_deep_pointwise_convolution_is_planned_as_k_slices(monkeypatch):
-    monkeypatch.setenv("DNNF_SPLIT_ALWAYS", "1")       # below the planner's break-even size
+def test_deep_pointwise_convolution_is_planned_as_k_slices():
+    always = B.PLAN_FUSED | B.PLAN_SPLIT_ALWAYS        # below the planner's break-even size
     g = _desc(); g.ext("X", (2, 32, 32, 256)); g.ext("Wt", (256, 64), kind="weight"); g.ext("s", (64,)); g.ext("t", (64,))
     g.mark_output(g.add("Clip", [g.add("ScaleShift", [g.add("Conv1x1", ["X", "Wt"]), "s", "t"], axis=-1)], lo=0.0, hi=6.0))
-    G, ids, st = _plan_desc(g)
+    G, ids, st = _plan_desc(g, always)
     fams = [(b["family"], b["variant"]) for b in G.blocks() if b["family"] != "alias"]
     assert fams == [("gemm", 4), ("gemm", 4)], G.blocks()
     assert st.n_ops == 3 and st.n_kernels == 2                    # the slices count as the convolution they came from
@@ -559,7 +559,7 @@ def test_deep_pointwise_convolution_is_planned_as_k_slices(monkeypatch):
     for shape, wshape, dt in [((2, 32, 32, 144), (144, 24), "f32"), ((1, 8, 8, 256), (256, 64), "f32"), ((2, 32, 32, 256), (256, 64), "bf16")]:
         g = _desc(); g.ext("X", shape, dt); g.ext("Wt", wshape, dt, kind="weight")
         g.mark_output(g.add("Conv1x1", ["X", "Wt"]))
-        G, ids, st = _plan_desc(g)
+        G, ids, st = _plan_desc(g, always)
         assert st.n_kernels == 1, G.blocks()
 
 
