@@ -147,6 +147,9 @@ typedef struct {
 #define DNNF_PLAN_STRICT_TABLE3     2u   /* type a broadcast operand's consumer One-to-Many on every edge */
 #define DNNF_PLAN_ALLOW_PROLOGUE    4u   /* planning only: let One-to-One predecessors fuse in front of a
                                             GEMM/conv anchor (Listing 1 literal); such plans cannot be run */
+#define DNNF_PLAN_BEYOND_TABLE3      8u   /* an extension beyond the paper's rules: MatMul -> [scale] -> [+ mask] -> Softmax ->
+                                            MatMul runs as ONE kernel (Table 3 marks Many-to-Many followed by
+                                            Many-to-Many red, so the default plan keeps three blocks) */
 /* Kernel-selection overrides.  The plan, its blocks and the results stay the same; a block is only lowered to another
  * kernel of its family.  They exist so that every kernel, including the ones the planner rarely picks, can be
  * tested and timed through this interface; the library reads no environment variable. */
@@ -191,7 +194,8 @@ typedef enum {
   DNNF_FAMILY_CONV1X1 = 5,     /* fp32 pointwise convolution with an epilogue chain */
   DNNF_FAMILY_DWCONV = 6,      /* fp32 depthwise 3x3 with an epilogue chain */
   DNNF_FAMILY_POOL = 7,        /* fp32 MaxPool / AveragePool with an epilogue chain */
-  DNNF_FAMILY_GATHER = 8       /* row gather by an index tensor */
+  DNNF_FAMILY_GATHER = 8,      /* row gather by an index tensor */
+  DNNF_FAMILY_ATTENTION = 9    /* scores, softmax and weighted sum of a head in one kernel (DNNF_PLAN_BEYOND_TABLE3 only) */
 } dnnf_family_t;
 
 typedef struct {

@@ -569,6 +569,44 @@ static void split_wide_pointwise(Graph& g, std::set<int>& decided) {
 
 thread_local uint32_t tl_plan_flags = 0;
 
+// Beyond Table 3: a block that ends in the scores of an attention head, the Softmax block behind it and the block of
+// the product with V become one block where that lowers to the single-kernel form.  The scores have the Softmax as
+// their only reader and the probabilities the second product, so the union is convex and depends on nothing that
+// depends on it.
+static void fuse_attention_blocks(const Graph& g, uint32_t flags, std::vector<std::vector<int>>& live) {
+  std::vector<int> bo(g.ops.size(), -1);
+  for (size_t i = 0; i < live.size(); ++i) for (int o : live[i]) bo[o] = (int)i;
+  for (size_t r = 0; r < live.size(); ++r) {
+    // the Softmax block: its one Many-to-Many operator is the Softmax (the scale / mask chain may sit in it or in
+    // the block of the first product; lowering sorts that out)
+    int smo = -1, anchors = 0;
+    for (int o : live[r]) { const int k = g.ops[o].kind; if (is_row_anchor(k) || is_contraction(k)) { ++anchors; if (k == DNNF_OP_SOFTMAX) smo = o; } }
+    if (anchors != 1 || smo < 0) continue;
+    const Op& sm = g.ops[smo];
+    const Tensor& pr = g.tensors[sm.out[0]];
+    if (pr.is_output || pr.consumers.size() != 1) continue;
+    // back along the chain in front of the Softmax to the tensor that enters this block
+    int t = sm.in[0];
+    while (g.tensors[t].producer >= 0 && bo[g.tensors[t].producer] == (int)r) t = g.ops[g.tensors[t].producer].in[0];
+    const Tensor& sc = g.tensors[t];
+    if (sc.producer < 0 || sc.is_output || sc.consumers.size() != 1) continue;
+    const int a = bo[sc.producer], c = bo[pr.consumers[0]];
+    if (a < 0 || c < 0 || a == c || a == (int)r || c == (int)r || live[a].empty() || live[c].empty()) continue;
+    if (g.ops[pr.consumers[0]].kind != DNNF_OP_MATMUL) continue;
+    std::vector<int> merged = live[a];
+    merged.insert(merged.end(), live[r].begin(), live[r].end());
+    merged.insert(merged.end(), live[c].begin(), live[c].end());
+    Block trial; std::string why;
+    if (lower_block(g, merged, flags, trial, why) != DNNF_OK || trial.launch.family != DNNF_FAMILY_ATTENTION) { if (dev_env("DNNF_DEBUG_PLAN")) fprintf(stderr, "attention not fused: %s\n", why.c_str()); continue; }
+    for (int o : live[r]) bo[o] = a;
+    for (int o : live[c]) bo[o] = a;
+    live[a] = merged; live[r].clear(); live[c].clear();
+  }
+  std::vector<std::vector<int>> keep;
+  for (auto& b : live) if (!b.empty()) keep.push_back(b);
+  live.swap(keep);
+}
+
 int plan_graph(Graph& g, uint32_t flags) {
   tl_plan_flags = flags;
   g.relink();
@@ -612,6 +650,7 @@ int plan_graph(Graph& g, uint32_t flags) {
   // is not enough after predecessor fusion: sort blocks topologically).
   std::vector<std::vector<int>> live;
   for (auto& b : P.blocks) if (!b.empty()) live.push_back(b);
+  if ((flags & DNNF_PLAN_BEYOND_TABLE3) && !(flags & (DNNF_PLAN_UNFUSED | DNNF_PLAN_ALLOW_PROLOGUE))) fuse_attention_blocks(g, flags, live);
   int nb = (int)live.size();
   std::vector<int> bo(g.ops.size(), -1);
   for (int i = 0; i < nb; ++i) for (int o : live[i]) bo[o] = i;
