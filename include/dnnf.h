@@ -162,6 +162,9 @@ typedef struct {
 #define DNNF_PLAN_NO_SPLIT_K        0x2000u  /* bf16 GEMM blocks without a split over K */
 #define DNNF_PLAN_NO_TMA_DWCONV     0x4000u  /* depthwise convolutions without the TMA-tiled kernel */
 #define DNNF_PLAN_NO_TILE_GEMM      0x8000u  /* bf16 GEMM blocks without the one-tile-per-CTA kernel */
+#define DNNF_PLAN_CLUSTER_SPLIT_K   0x10000u /* one-tile-per-CTA kernel: clusters of 2 or 4 CTAs share a tile's k-tiles and add their
+                                                partial sums through distributed shared memory (measured slower at the sizes
+                                                tried, so not the default) */
 
 typedef struct {
   int32_t ops_before, ops_after;

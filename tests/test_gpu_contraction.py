@@ -97,7 +97,7 @@ def test_pair_gemm_more_tiles_than_cta_pairs(mnk, epi):
         t = g.add("Add", [t, "R"])
     g.mark_output(t)
     wl = W.Workload(g, ins)
-    s, got, ref = run_both(wl, FUSED)
+    s, got, ref = run_both(wl, FUSED | B.PLAN_NO_TILE_GEMM)
     (name,) = wl.graph.outputs
     close(got[name], ref[name], RTOL_BF16)
     _expect_variant(s, 3)
@@ -107,28 +107,31 @@ def test_pair_gemm_more_tiles_than_cta_pairs(mnk, epi):
     assert s.g.status()[0] == 0
 
 
-@pytest.mark.parametrize("mnk", [(512, 128, 2048), (256, 256, 2304), (1024, 768, 3072), (300, 136, 2120), (512, 384, 2056)])
-@pytest.mark.parametrize("epi", ["none", "bias_gelu", "bias_residual"])
-def test_pair_gemm_split_k(mnk, epi):
-    """Few output tiles and a long K: several CTA pairs share a tile (split-K).  Three runs in a row on the same
-    workspace: the arrival counters must come back to zero by themselves."""
-    import os
-    m, n, k = mnk
+def _gemm_with_epilogue(m, n, k, epi, seed0):
     g = graph()
     g.ext("A", (m, k), "bf16"); g.ext("Bm", (k, n), "bf16")
-    ins = {"A": _bf(rnd((m, k), 41, -1, 1)), "Bm": _bf(rnd((k, n), 42, -0.1, 0.1))}
+    ins = {"A": _bf(rnd((m, k), seed0, -1, 1)), "Bm": _bf(rnd((k, n), seed0 + 1, -0.1, 0.1))}
     t = g.add("MatMul", ["A", "Bm"])
     if epi != "none":
-        g.ext("bias", (n,), "f32"); ins["bias"] = rnd((n,), 43, -0.5, 0.5)
+        g.ext("bias", (n,), "f32"); ins["bias"] = rnd((n,), seed0 + 2, -0.5, 0.5)
         t = g.add("Add", [t, "bias"])
     if epi == "bias_gelu":
         t = g.add("Gelu", [t], approx="tanh")
     if epi == "bias_residual":
-        g.ext("R", (m, n), "bf16"); ins["R"] = _bf(rnd((m, n), 44, -1, 1))
+        g.ext("R", (m, n), "bf16"); ins["R"] = _bf(rnd((m, n), seed0 + 3, -1, 1))
         t = g.add("Add", [t, "R"])
     g.mark_output(t)
-    wl = W.Workload(g, ins)
-    s, got, ref = run_both(wl, FUSED)
+    return W.Workload(g, ins)
+
+
+@pytest.mark.parametrize("mnk", [(512, 128, 2048), (256, 256, 2304), (1024, 768, 3072), (300, 136, 2120), (512, 384, 2056)])
+@pytest.mark.parametrize("epi", ["none", "bias_gelu", "bias_residual"])
+def test_pair_gemm_split_k(mnk, epi):
+    """Few output tiles and a long K: several CTA pairs share a tile (split-K through the workspace).  Three runs in a row
+    on the same workspace: the arrival counters must come back to zero by themselves."""
+    m, n, k = mnk
+    wl = _gemm_with_epilogue(m, n, k, epi, 41)
+    s, got, ref = run_both(wl, FUSED | B.PLAN_NO_TILE_GEMM)
     (name,) = wl.graph.outputs
     close(got[name], ref[name], RTOL_BF16)
     assert s.g.blocks()[0]["variant"] == 3 and s.g.workspace_zero_bytes() > 256, (s.g.blocks(), s.g.workspace_zero_bytes())
@@ -136,6 +139,32 @@ def test_pair_gemm_split_k(mnk, epi):
         s.run()
         close(s.output(name), ref[name], RTOL_BF16)
         assert s.g.status()[0] == 0
+
+
+@pytest.mark.parametrize("mnk", [(512, 128, 2048), (256, 256, 2304), (1024, 768, 3072), (1024, 768, 768), (1024, 2304, 768), (300, 136, 2120),
+                                 (512, 384, 2056), (129, 72, 1032), (1000, 200, 392), (128, 128, 832)])
+@pytest.mark.parametrize("epi", ["none", "bias_gelu", "bias_residual"])
+def test_tile_gemm_cluster_split_k(mnk, epi):
+    """The one-tile-per-CTA kernel with a cluster of 2 or 4 CTAs per tile (an option: measured slower than no split): each takes a range of the k-tiles, the partial
+    sums meet through distributed shared memory and every CTA finishes its own column slice.  Ragged M, N and K, a
+    last CTA with fewer k-tiles than the others, both cluster sizes, every epilogue; nothing goes through the
+    workspace."""
+    m, n, k = mnk
+    wl = _gemm_with_epilogue(m, n, k, epi, 71)
+    s, got, ref = run_both(wl, FUSED | B.PLAN_CLUSTER_SPLIT_K)
+    (name,) = wl.graph.outputs
+    close(got[name], ref[name], RTOL_BF16)
+    b = s.g.blocks()[0]
+    tiles = -(-m // 128) * -(-n // (128 if n > 64 else 64))
+    assert b["variant"] == 5 and b["grid"] in (2 * tiles, 4 * tiles) and s.g.workspace_zero_bytes() == 256, (b, tiles)
+    s.buffers[name].fill_(float("nan"))
+    s.run()
+    close(s.output(name), ref[name], RTOL_BF16)
+    assert s.g.status() == (0, -1)
+    # the same block without the split
+    s1, got1, _ = run_both(wl, FUSED | B.PLAN_CLUSTER_SPLIT_K | B.PLAN_NO_SPLIT_K)
+    assert s1.g.blocks()[0]["variant"] == 5 and s1.g.blocks()[0]["grid"] == tiles
+    close(got1[name], ref[name], RTOL_BF16)
 
 
 def test_batched_matmul_with_transposed_and_strided_operands():
