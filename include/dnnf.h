@@ -269,6 +269,15 @@ DNNF_API const char* dnnf_rule_name(int rule_index);
 DNNF_API int dnnf_plan(dnnf_graph* g, uint32_t flags, dnnf_plan_stats* host_stats);
 DNNF_API int dnnf_block_count(const dnnf_graph* g, int* n_blocks);
 DNNF_API int dnnf_block_info(const dnnf_graph* g, int block, dnnf_block_desc* host_out);
+/* External tensors of a planned block: what it reads from and writes to memory (ids as returned by dnnf_add_tensor /
+ * dnnf_add_op; capacities in entries, counts always written). */
+DNNF_API int dnnf_block_tensors(const dnnf_graph* g, int block, int* host_in_ids, int cap_in, int* n_in,
+                                int* host_out_ids, int cap_out, int* n_out);
+/* Where a tensor lives after dnnf_plan: *where = 0 caller-bound (external input or marked output), 1 in the workspace at
+ * *workspace_offset bytes, 2 nowhere (it stays inside its block: IR_removable, Section 3.2), 3 it shares the caller-bound
+ * storage of tensor *workspace_offset (a zero-copy Reshape).  With dnnf_run_block this lets a caller feed one block with
+ * inputs of its own and read its results (per-block parity tests, per-block timing on chosen data). */
+DNNF_API int dnnf_tensor_location(const dnnf_graph* g, int tensor_id, int* where, int64_t* workspace_offset);
 /* Writes the block's micro-op program as text ("MOV in0; ADD in1; MUL c0=0.5; ...")
  * into host_buf (capacity bytes, NUL-terminated, truncated if needed): the linearised
  * data-flow tree of Section 4.4, every value computed once. */

@@ -75,7 +75,7 @@ class BlockDesc(C.Structure):
 
 EXPORTS = ["dnnf_graph_create", "dnnf_graph_destroy", "dnnf_add_tensor", "dnnf_add_op", "dnnf_mark_output",
            "dnnf_tensor_info", "dnnf_op_mapping", "dnnf_mapping_check", "dnnf_rewrite", "dnnf_rule_name", "dnnf_plan",
-           "dnnf_block_count", "dnnf_block_info", "dnnf_block_program", "dnnf_op_block", "dnnf_op_count", "dnnf_op_kind",
+           "dnnf_block_count", "dnnf_block_info", "dnnf_block_tensors", "dnnf_tensor_location", "dnnf_block_program", "dnnf_op_block", "dnnf_op_count", "dnnf_op_kind",
            "dnnf_workspace_size", "dnnf_workspace_zero_bytes", "dnnf_bind", "dnnf_bind_workspace", "dnnf_run", "dnnf_run_static_ws", "dnnf_run_block", "dnnf_status",
            "dnnf_launch_count", "dnnf_last_error", "dnnf_version",
            "dnnf_profile_db_set", "dnnf_profile_db_get", "dnnf_profile_db_size", "dnnf_profile_db_clear", "dnnf_profile_db_save",
@@ -106,6 +106,8 @@ def _load():
     lib.dnnf_block_count.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
     lib.dnnf_block_info.argtypes = [C.c_void_p, C.c_int, C.POINTER(BlockDesc)]
     lib.dnnf_block_program.argtypes = [C.c_void_p, C.c_int, C.c_char_p, C.c_size_t]
+    lib.dnnf_block_tensors.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_int, C.POINTER(C.c_int)]
+    lib.dnnf_tensor_location.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int64)]
     lib.dnnf_op_block.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int)]
     lib.dnnf_op_count.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
     lib.dnnf_op_kind.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
@@ -226,6 +228,19 @@ class Graph:
         d = BlockDesc()
         self._check(lib.dnnf_block_info(self.h, b, C.byref(d)))
         return d
+
+    def block_tensors(self, b):
+        """(input tensor ids, output tensor ids) of a planned block."""
+        ins, outs = (C.c_int * 16)(), (C.c_int * 16)()
+        ni, no = C.c_int(), C.c_int()
+        self._check(lib.dnnf_block_tensors(self.h, b, ins, 16, C.byref(ni), outs, 16, C.byref(no)))
+        return [ins[i] for i in range(min(ni.value, 16))], [outs[i] for i in range(min(no.value, 16))]
+
+    def tensor_location(self, tid):
+        """(where, offset): 0 caller-bound, 1 workspace at `offset` bytes, 2 inside its block, 3 alias of bound tensor `offset`."""
+        w, off = C.c_int(), C.c_int64()
+        self._check(lib.dnnf_tensor_location(self.h, tid, C.byref(w), C.byref(off)))
+        return w.value, off.value
 
     def block_program(self, b):
         buf = C.create_string_buffer(4096)

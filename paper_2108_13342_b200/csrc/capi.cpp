@@ -310,6 +310,29 @@ int dnnf_block_info(const dnnf_graph* g, int bi, dnnf_block_desc* out) {
   return DNNF_OK;
 }
 
+int dnnf_block_tensors(const dnnf_graph* g, int bi, int* in_ids, int cap_in, int* n_in, int* out_ids, int cap_out, int* n_out) {
+  if (!g || !n_in || !n_out || bi < 0 || bi >= (int)g->g.blocks.size()) return DNNF_ERR_INVALID_ARG;
+  const Block& b = g->g.blocks[bi];
+  *n_in = (int)b.inputs.size(); *n_out = (int)b.outputs.size();
+  for (int i = 0; in_ids && i < cap_in && i < *n_in; ++i) in_ids[i] = b.inputs[i];
+  for (int i = 0; out_ids && i < cap_out && i < *n_out; ++i) out_ids[i] = b.outputs[i];
+  return DNNF_OK;
+}
+
+int dnnf_tensor_location(const dnnf_graph* g, int tensor_id, int* where, int64_t* workspace_offset) {
+  if (!g || !where || tensor_id < 0 || tensor_id >= (int)g->g.tensors.size()) return DNNF_ERR_INVALID_ARG;
+  const Graph& G = g->g;
+  if (!G.planned) return DNNF_ERR_STATE;
+  int t = tensor_id;
+  while (G.tensors[t].alias_of >= 0) t = G.tensors[t].alias_of;
+  const Tensor& T = G.tensors[t];
+  if (workspace_offset) *workspace_offset = -1;
+  if (T.external || T.is_output) { *where = t == tensor_id ? 0 : 3; if (workspace_offset && t != tensor_id) *workspace_offset = t; return DNNF_OK; }
+  if (T.ws_offset >= 0) { *where = 1; if (workspace_offset) *workspace_offset = T.ws_offset; return DNNF_OK; }
+  *where = 2;
+  return DNNF_OK;
+}
+
 int dnnf_block_program(const dnnf_graph* g, int bi, char* buf, size_t cap) {
   if (!g || !buf || cap == 0 || bi < 0 || bi >= (int)g->g.blocks.size()) return DNNF_ERR_INVALID_ARG;
   static const char* on[] = {"END", "MOV", "SAVE", "STORE", "ADD", "SUB", "RSUB", "MUL", "DIV", "RDIV", "MAX", "MIN", "NEG", "ABS",
