@@ -356,6 +356,13 @@ DNNF_API int dnnf_run_static_ws(dnnf_graph* g, void* cuda_stream);
  * (0 = ok, DNNF_ERR_TIMEOUT if a bounded wait inside a kernel ran out) and the
  * block that reported it. */
 DNNF_API int dnnf_status(dnnf_graph* g, int* device_status, int* block);
+/* Self-test of the failure path (no counterpart in the paper).  Every wait inside the tensor-core kernels is bounded;
+ * when a bound runs out the kernel records DNNF_ERR_TIMEOUT in the workspace's status words and returns instead of
+ * hanging.  This call launches one tiny kernel on `cuda_stream` that waits, with the kernels' own wait routine, on a
+ * barrier nobody signals, for at most limit_ns (1 .. 100,000,000).  After a stream synchronisation dnnf_status()
+ * reports DNNF_ERR_TIMEOUT from block -2; the caller then clears the workspace's first dnnf_workspace_zero_bytes bytes
+ * and the graph runs as before.  Needs a bound workspace; nothing faults, traps or hangs. */
+DNNF_API int dnnf_selftest_wait_expiry(dnnf_graph* g, uint64_t limit_ns, void* cuda_stream);
 /* Number of kernels one dnnf_run launches. */
 DNNF_API int dnnf_launch_count(const dnnf_graph* g, int* n);
 

@@ -76,7 +76,7 @@ class BlockDesc(C.Structure):
 EXPORTS = ["dnnf_graph_create", "dnnf_graph_destroy", "dnnf_add_tensor", "dnnf_add_op", "dnnf_mark_output",
            "dnnf_tensor_info", "dnnf_op_mapping", "dnnf_mapping_check", "dnnf_rewrite", "dnnf_rule_name", "dnnf_plan",
            "dnnf_block_count", "dnnf_block_info", "dnnf_block_tensors", "dnnf_tensor_location", "dnnf_block_program", "dnnf_op_block", "dnnf_op_count", "dnnf_op_kind",
-           "dnnf_workspace_size", "dnnf_workspace_zero_bytes", "dnnf_bind", "dnnf_bind_workspace", "dnnf_run", "dnnf_run_static_ws", "dnnf_run_block", "dnnf_status",
+           "dnnf_workspace_size", "dnnf_workspace_zero_bytes", "dnnf_bind", "dnnf_bind_workspace", "dnnf_run", "dnnf_run_static_ws", "dnnf_run_block", "dnnf_status", "dnnf_selftest_wait_expiry",
            "dnnf_launch_count", "dnnf_last_error", "dnnf_version",
            "dnnf_profile_db_set", "dnnf_profile_db_get", "dnnf_profile_db_size", "dnnf_profile_db_clear", "dnnf_profile_db_save",
            "dnnf_profile_db_load", "dnnf_block_signature", "dnnf_profile_miss_count", "dnnf_profile_miss", "dnnf_profile_measure"]
@@ -128,6 +128,7 @@ def _load():
     lib.dnnf_run_static_ws.argtypes = [C.c_void_p, C.c_void_p]
     lib.dnnf_run_block.argtypes = [C.c_void_p, C.c_int, C.c_void_p]
     lib.dnnf_status.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+    lib.dnnf_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
     lib.dnnf_launch_count.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
     return lib
 
@@ -307,6 +308,9 @@ class Graph:
 
     def run_block(self, b, stream=0):
         self._check(lib.dnnf_run_block(self.h, b, C.c_void_p(stream)))
+
+    def selftest_wait_expiry(self, limit_ns, stream=0):
+        self._check(lib.dnnf_selftest_wait_expiry(self.h, int(limit_ns), C.c_void_p(stream)))
 
     def status(self):
         s, b = C.c_int(), C.c_int()

@@ -22,6 +22,8 @@ int profile_measure(Graph& g, void* scratch, size_t scratch_bytes, void* stream,
 
 static int fail(dnnf_graph* g, int code, const char* msg) { if (g) g->g.err = msg; return code; }
 
+namespace dnnf { int selftest_wait_expiry(Graph& g, unsigned long long limit_ns, void* stream); }
+
 extern "C" {
 
 const char* dnnf_version(void) { return "dnnf-b200 0.1"; }
@@ -308,6 +310,11 @@ int dnnf_block_info(const dnnf_graph* g, int bi, dnnf_block_desc* out) {
   out->threads = b.launch.threads;
   out->variant = b.launch.variant;
   return DNNF_OK;
+}
+
+int dnnf_selftest_wait_expiry(dnnf_graph* g, uint64_t limit_ns, void* stream) {
+  if (!g) return DNNF_ERR_INVALID_ARG;
+  return dnnf::selftest_wait_expiry(g->g, limit_ns, stream);
 }
 
 int dnnf_block_tensors(const dnnf_graph* g, int bi, int* in_ids, int cap_in, int* n_in, int* out_ids, int cap_out, int* n_out) {

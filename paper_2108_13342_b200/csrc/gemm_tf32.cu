@@ -3,9 +3,11 @@
 // to live in shared memory.  On the FMA pipes such a block is bound by arithmetic; on the
 // tensor cores it becomes bound by HBM, which is where a fused block belongs.
 //
-// fp32 accuracy comes from splitting every operand into two TF32 numbers, x = hi + lo with
-// hi = tf32(x) and lo = tf32(x - hi), and accumulating the three products lo*hi + hi*lo + hi*hi
-// in fp32 (tensor memory); the dropped lo*lo term and the rounding of lo are O(2^-22) relative.
+// fp32 accuracy comes from splitting every operand into two TF32 numbers, x = hi + lo, and accumulating the three
+// products lo*hi + hi*lo + hi*hi in fp32 (tensor memory).  B is split once per CTA with rounding (hi = tf32(x),
+// lo = tf32(x - hi)); A, which is split on the fly for every tile, with a mask (hi = x cut to 11 significant bits,
+// lo = x - hi, cut once more by the tensor core): the dropped lo*lo term and the cut of lo are below 2^-20 relative
+// per product, against a parity bar of 1e-5.
 //
 // One persistent CTA per SM, 448 threads, warp-specialised:
 //   warp 0        TMA producer: raw fp32 row blocks of A (whole rows: one contiguous piece of memory
@@ -37,6 +39,7 @@
 
 #include "ir.h"
 #include "tc_common.cuh"
+#include "fp32_epilogues.h"
 #include "tma_host.h"
 
 namespace dnnf {
@@ -60,8 +63,19 @@ constexpr int kMaxStages = 8;                               // raw row blocks in
 constexpr int kAStageCols = 2 * BK;                         // TMEM columns of one A stage: hi, then lo
 constexpr int kChunkBytes = 32 * 128;                       // 32 rows x 32 fp32, swizzled
 constexpr int kMaxVec = 4, kVecFloats = 256 + 32;           // staged row-invariant operands
-constexpr int kEpiBytes = EPI_WARPS * 2 * kChunkBytes;      // >= EPI_WARPS * kStageWords * 4 (the general form's staging)
-constexpr int kFixed = 1024 + 512 + kEpiBytes + kMaxVec * kVecFloats * 4;   // alignment slack, barriers, epilogue buffers
+constexpr int kMinEpiBytes = EPI_WARPS * 2 * kChunkBytes;   // >= EPI_WARPS * kStageWords * 4 (the general form's staging)
+constexpr int kFixedNoEpi = 1024 + 512 + kMaxVec * kVecFloats * 4;          // alignment slack, barriers, staged vectors
+// chunk buffers of the fast epilogue: one per 32-column chunk a warp handles in a tile, so that a tile's stores are
+// issued together and the wait for the buffers falls a whole tile later
+inline int epi_bytes_for(int N, int K, bool fast) {
+  const int n_epi = N <= 32 ? 4 : 8;
+  const int chunks = (N + 31) / 32, per_warp = n_epi == 4 ? chunks : (chunks + 1) / 2;
+  int b = n_epi * per_warp * kChunkBytes;
+  if (!fast && b < kMinEpiBytes) b = kMinEpiBytes;                // the general form's transpose staging
+  const int raw_b = ((K * N * 4 + 1023) / 1024) * 1024;          // a dense B block lands here before it is split
+  return b < raw_b && raw_b <= 96 * 1024 ? raw_b : b;
+}
+
 constexpr int kMaxBBytes = 88 * 1024;                       // hi + lo images of B
 
 struct Params {
@@ -79,6 +93,8 @@ struct Params {
   int32_t b_dense;           // B is a dense row-major [K x N] block: fetched with one bulk copy
   int32_t fast_epi;          // the fast epilogue form applies
   int32_t debug;             // ablation switches (development only)
+  int32_t epi_bytes;         // chunk buffers / transpose staging / raw B
+  int32_t chunks_per_warp;   // fast epilogue: chunk buffers of one warp
   FastDiv fd_n, fd_npad, fd_kpad;   // element index of B -> (k, n)
   int32_t b_static;          // B is an external input: it may be read before the previous kernel ends
   int8_t slot[kMaxIn];       // fast form: staged-vector slot of epilogue input i, or -1 for a dense operand
@@ -136,6 +152,7 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, const void* 
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // Fast epilogue IO: a lane owns 32 consecutive columns [c, c+32) of its own row.
@@ -202,7 +219,7 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
   const uint32_t a_cols0 = 2u * (uint32_t)acc_cols;                // A stages follow the two accumulator stages
   uint8_t* ring = smem + (size_t)atom_bytes * k_chunks;            // raw row blocks of A
   uint8_t* epi = ring + (size_t)stages * q.unit_stride;            // chunk buffers (1024-aligned) / transpose staging / raw B
-  float* vec_s = reinterpret_cast<float*>(epi + kEpiBytes);
+  float* vec_s = reinterpret_cast<float*>(epi + q.epi_bytes);
   uint64_t* raw_bar = reinterpret_cast<uint64_t*>(vec_s + kMaxVec * kVecFloats);
   uint64_t* empty_bar = raw_bar + kMaxStages;    // [stages]   raw block consumed by the converters
   uint64_t* conv_bar = empty_bar + kMaxStages;   // [a_stages] A stage written
@@ -396,6 +413,7 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
       tc_fence_after();
       if (q.debug & 4) { __syncwarp(); if (lane == 0) mbar_arrive(&tempty_bar[acc]); continue; }
       const uint32_t t_row = tmem_base + ((uint32_t)(sub * 32) << 16) + (uint32_t)(acc * acc_cols);
+      bool released = false;
       if (kFast) {
         RowEpiIO io{p, q};
         io.lane = lane;
@@ -403,8 +421,16 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
         const int m = tile * BM + sub * 32 + lane;
         io.row_ok = m < p.M;
         io.row = io.row_ok ? (uint32_t)m : 0u;
-        for (int c = cgroup * 32; c < p.N; c += cstep, ++nstore) {
+        // One chunk buffer per 32-column chunk of this warp: the tile's stores are issued together at its end, and the
+        // wait for the buffers (the previous tile's stores have read them) comes a whole tile after they were issued.
+        // (With two buffers per warp, every chunk waited for the store of two chunks earlier: 1100 cycles per chunk.)
+        { const long long t0 = clock64(); if (lane == 0) tma_store_wait_read0();
+        __syncwarp(); if (warp == 2 && lane == 0) FACC(14, clock64() - t0); }
+        uint8_t* my_chunks = epi + (size_t)(warp - 2) * q.chunks_per_warp * kChunkBytes;
+        int slot = 0;
+        for (int c = cgroup * 32; c < p.N; c += cstep, ++slot) {
           uint32_t raw[32];
+          const long long t0 = clock64();
           tc_ld32_issue(t_row + c, raw);
           tc_ld_wait();
 #pragma unroll
@@ -415,16 +441,25 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
 #pragma unroll
             for (int j = 0; j < 32; ++j) io.accv[j] += __uint_as_float(raw[j]);
           }
+          const long long t1 = clock64();
           io.c = c;
-          io.chunk = epi + ((warp - 2) * 2 + (nstore & 1)) * kChunkBytes;
-          // the store issued two chunks ago read this buffer: it must have finished reading
-          if (lane == 0) tma_store_wait_read1();
-          __syncwarp();
+          io.chunk = my_chunks + slot * kChunkBytes;
           run_program<32, SP, false>(p.prog, io);
-          fence_async_smem();
-          __syncwarp();
-          if (lane == 0) { tma_store_2d(&q.tmD, io.chunk, c, tile * BM + sub * 32); tma_store_commit(); }
+          if (warp == 2 && lane == 0) { FACC(12, t1 - t0); FACC(13, clock64() - t1); }
         }
+        // the accumulator stage is free as soon as it has been read
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+        released = true;
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          slot = 0;
+          for (int c = cgroup * 32; c < p.N; c += cstep, ++slot) tma_store_2d(&q.tmD, my_chunks + slot * kChunkBytes, c, tile * BM + sub * 32);
+          tma_store_commit();
+        }
+        (void)nstore;
       } else {
         TcEpiIO io{p};
         uint32_t* stage = stage_area + (warp - 2) * kStageWords;
@@ -466,9 +501,11 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
           run_program<32, SP, false>(p.prog, io);
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+      if (!released) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+      }
       if (warp == 2 && lane == 0) FACC(6, clock64() - t_epi);
     }
     if (kFast && lane == 0) tma_store_wait_all();     // shared memory must outlive the last stores' reads
@@ -506,9 +543,12 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
             const float xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const float h = to_tf32(xs[e]);
-              hi[4 * j + e] = __float_as_uint(h);
-              lo[4 * j + e] = __float_as_uint(to_tf32(xs[e] - h));
+              // hi = x cut to TF32 precision by a mask, lo = x - hi (exact in fp32); the tensor core reads the upper 19
+              // bits of lo, i.e. cuts it once more: |a - (hi + lo')| < 2^-20 |a|.  Two full-rate instructions per value
+              // instead of two conversions and a subtraction (7 % of the 144 -> 24 block's time).
+              const uint32_t hb = __float_as_uint(xs[e]) & 0xffffe000u;
+              hi[4 * j + e] = hb;
+              lo[4 * j + e] = __float_as_uint(xs[e] - __uint_as_float(hb));
             }
           }
         }
@@ -552,24 +592,6 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
   }
 }
 
-// ---- static epilogue programs ------------------------------------------------------------------
-#define MO(o, s, i) MicroOp{o, s, i, 0}
-DNNF_SP_BEGIN(FP_Store, 2) MO(M_MOV, S_ANCHOR, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-DNNF_SP_BEGIN(FP_Bias, 3) MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-DNNF_SP_BEGIN(FP_ScaleShiftClip, 5)
-  MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_CLIP, S_CONST, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-DNNF_SP_BEGIN(FP_ScaleShiftResidual, 5)
-  MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_ADD, S_IN, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-DNNF_SP_BEGIN(FP_ScaleShiftClipResidual, 6)
-  MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_CLIP, S_CONST, 0), MO(M_ADD, S_IN, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-// the later slices of a contraction that the planner split along K: the partial sum arrives as a residual
-DNNF_SP_BEGIN(FP_Residual, 3) MO(M_MOV, S_IN, 0), MO(M_ADD, S_ANCHOR, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-DNNF_SP_BEGIN(FP_ResidualScaleShiftClip, 6)
-  MO(M_MOV, S_IN, 0), MO(M_ADD, S_ANCHOR, 0), MO(M_MUL, S_IN, 1), MO(M_ADD, S_IN, 2), MO(M_CLIP, S_CONST, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
-#undef MO
-using Static = TypeList<FP_Store, FP_Bias, FP_ScaleShiftClip, FP_ScaleShiftResidual, FP_ScaleShiftClipResidual, FP_Residual,
-                        FP_ResidualScaleShiftClip>;
-
 }  // namespace tf32
 
 // ---- host side ------------------------------------------------------------------------------------
@@ -599,7 +621,7 @@ bool tf32_shape_fits(int64_t M, int64_t N, int64_t K) {
   }
   // a whole tile of raw rows must be resident: the converter warps advance chunk by chunk together
   const int kr = ((int)K + 3) / 4 * 4, pitch = kr + ((kr / 4) % 2 == 0 ? 4 : 8);
-  if ((tf32::kSmemMax - tf32::kFixed - tf32_b_bytes_of((int)N, (int)K)) / ((32 * pitch * 4 + 1023) / 1024 * 1024) < 4) return false;
+  if ((tf32::kSmemMax - tf32::kFixedNoEpi - tf32::epi_bytes_for((int)N, (int)K, false) - tf32_b_bytes_of((int)N, (int)K)) / ((32 * pitch * 4 + 1023) / 1024 * 1024) < 4) return false;
   return true;
 }
 
@@ -646,14 +668,17 @@ void tf32_gemm_plan(Launch& L) {
   // number of 16-byte pieces (conflict-free 128-bit reads down a column of rows)
   const int kr = (gp.K + 3) / 4 * 4;
   q.pitch = kr + ((kr / 4) % 2 == 0 ? 4 : 8);
-  const int ring_budget = tf32::kSmemMax - tf32::kFixed - tf32_b_bytes(gp);
+  q.epi_bytes = tf32::epi_bytes_for(gp.N, gp.K, q.fast_epi != 0);
+  { const int chunks = (gp.N + 31) / 32; q.chunks_per_warp = q.epi_warps == 4 ? chunks : (chunks + 1) / 2; }
+  const int fixed = tf32::kFixedNoEpi + q.epi_bytes;
+  const int ring_budget = tf32::kSmemMax - fixed - tf32_b_bytes(gp);
   q.rb = 32;                                                 // one block per converter warp
   q.unit_stride = (q.rb * q.pitch * 4 + 1023) / 1024 * 1024;
   q.stages = std::min(tf32::kMaxStages, ring_budget / q.unit_stride);
-  q.a_stages = std::min(4, (512 - 2 * (q.dual ? 2 : 1) * q.npad) / tf32::kAStageCols);
-  L.smem = (size_t)tf32_b_bytes(gp) + (size_t)q.stages * q.unit_stride + tf32::kFixed;
+  q.a_stages = std::min(6, (512 - 2 * (q.dual ? 2 : 1) * q.npad) / tf32::kAStageCols);
+  L.smem = (size_t)tf32_b_bytes(gp) + (size_t)q.stages * q.unit_stride + fixed;
   q.b_dense = gp.B.stride_col == 1 && gp.B.stride_row == gp.N && gp.N % 4 == 0 && gp.B.base % 4 == 0 &&
-              (int64_t)gp.K * gp.N * 4 <= tf32::kEpiBytes && !dev_env("DNNF_TF32_NO_BULK_B");
+              (int64_t)gp.K * gp.N * 4 <= q.epi_bytes && !dev_env("DNNF_TF32_NO_BULK_B");
   L.variant = 4;
   L.static_id = StaticSet<tf32::Static>::find(gp.prog);
 }

@@ -6,6 +6,7 @@
 #include <map>
 
 #include "ir.h"
+#include "tc_common.cuh"
 
 namespace dnnf {
 
@@ -140,6 +141,34 @@ int profile_measure(Graph& g, void* scratch, size_t scratch_bytes, void* stream,
   if (n_measured) *n_measured = done;
   if (rc_all != DNNF_OK) g.err = "profiling run failed";
   return rc_all;
+}
+
+// Self-test of the bounded waits: one CTA waits, with the kernels' own wait routine, on a barrier that nothing will
+// ever signal.  The wait has to give up after `limit_ns`, raise the CTA's abort flag and come back; the kernel then
+// records DNNF_ERR_TIMEOUT in the status words the way every tensor-core kernel's tear-down does.  Nothing faults and
+// nothing hangs: this is the path a lost TMA completion or a missing commit would take.
+__global__ void wait_expiry_kernel(int32_t* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  bool ok = true;
+  if (threadIdx.x == 0) ok = mbar_wait(&bar, 0, &abort_flag, limit_ns);
+  __syncthreads();
+  if (threadIdx.x == 0 && abort_flag && !ok && status) { atomicExch(&status[0], DNNF_ERR_TIMEOUT); atomicExch(&status[1], -2); }
+}
+
+int selftest_wait_expiry(Graph& g, unsigned long long limit_ns, void* stream) {
+  if (!g.ws_ptr) { g.err = "bind a workspace first: the status words live in it"; return DNNF_ERR_WORKSPACE; }
+  if (limit_ns == 0 || limit_ns > 100000000ull) { g.err = "limit must be between 1 ns and 100 ms"; return DNNF_ERR_INVALID_ARG; }
+  g.last_status_base = g.ws_ptr;
+  wait_expiry_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(reinterpret_cast<int32_t*>(g.ws_ptr), limit_ns);
+  if (cudaGetLastError() != cudaSuccess) { g.err = "self-test launch failed"; return DNNF_ERR_CUDA; }
+  return DNNF_OK;
 }
 
 int read_status(Graph& g, int* status, int* block) {

@@ -37,14 +37,14 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ unsigned long long wall_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
 // Bounded wait: gives up after kWaitLimitNs of wall-clock time (or as soon as another role of the
 // CTA gave up), sets the CTA's abort flag and returns false.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = wall_ns();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 64; ++i) if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (wall_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    if (wall_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
   }
 }
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* tm, uint64_t* bar, int c0, int c1, int c2, int c3) {

@@ -245,3 +245,27 @@ def test_profiling_database_measured_on_the_device_drives_the_plan():
         assert s.plan_stats.n_profile_misses == 0
     finally:
         B.profile_db_clear()
+
+
+def test_bounded_wait_expires_and_the_graph_runs_on():
+    """The failure path of the tensor-core kernels without a failure: a wait on a barrier that nothing signals gives up
+    after its limit (1 ms here), the status words report DNNF_ERR_TIMEOUT, nothing hangs or faults, and after the
+    caller has cleared the status words the graph runs and is correct again."""
+    import time
+    import torch
+    wl = W.ffn_block(m=256, hidden=128, ffn=256)
+    s, got, ref = run_both(wl)
+    close(got["Y"], ref["Y"], RTOL_BF16)
+    stream = torch.cuda.current_stream().cuda_stream
+    t0 = time.perf_counter()
+    s.g.selftest_wait_expiry(1_000_000, stream)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 0.5                      # it gave up after about a millisecond, not a second
+    assert s.g.status() == (B.ERR_TIMEOUT, -2)
+    s.workspace[: s.g.workspace_zero_bytes()].zero_()
+    s.buffers["Y"].fill_(float("nan"))
+    s.run()
+    close(s.output("Y"), ref["Y"], RTOL_BF16)
+    assert s.g.status() == (0, -1)
+    with pytest.raises(B.DnnfError):
+        s.g.selftest_wait_expiry(10**12, stream)               # limits beyond 100 ms are refused
