@@ -14,6 +14,7 @@ def main():
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--unfused", action="store_true")
     ap.add_argument("--canon", action="store_true")
+    ap.add_argument("--beyond", action="store_true", help="plan with DNNF_PLAN_BEYOND_TABLE3 (single-kernel attention)")
     ap.add_argument("--instances", type=int, default=1, help="independent copies with their own buffers, run round-robin")
     args = ap.parse_args()
     import torch
@@ -22,7 +23,7 @@ def main():
     from .runtime import Session
     kw = {k: int(v) for k, v in (x.split("=") for x in args.kw)}
     wl = W.by_name(args.workload, **kw)
-    sess = [Session(wl, plan_flags=B.PLAN_UNFUSED if args.unfused else B.PLAN_FUSED,
+    sess = [Session(wl, plan_flags=B.PLAN_UNFUSED if args.unfused else (B.PLAN_FUSED | (B.PLAN_BEYOND_TABLE3 if args.beyond else 0)),
                     rewrite_flags=B.REWRITE_CANON_MACRO if args.canon else B.REWRITE_NONE) for _ in range(args.instances)]
     s = sess[0]
     for _ in range(args.iters):
