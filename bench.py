@@ -257,7 +257,7 @@ def main():
 
     blocks = S[0].g.blocks()
     k_us = [sum(e[b].elapsed_time(e[b + 1]) for e in ev) / steps * 1e3 for b in range(nb)]
-    kernels = [{"ops": "+".join(blocks[b]["ops"]), "us": round(k_us[b], 2), "bytes": bbytes[b],
+    kernels = [{"ops": "+".join(blocks[b]["ops"]), "us": round(k_us[b], 2),
                 "frac": round(bbytes[b] / (k_us[b] * 1e-6) / 1e9 / pk["hbm_gbs"], 3)} for b in range(nb)]
     top = max(range(nb), key=lambda b: k_us[b])
     ach = bbytes[top] / (k_us[top] * 1e-6) / 1e9
@@ -271,7 +271,7 @@ def main():
         ent = tj.get("mbconv_block", {}).get(str(top))
         if ent:
             roof["traffic"] = ent["dram_bytes_per_launch"]
-            roof["traffic_source"] = ent["source"]
+            roof["traffic_source"] = "committed ncu capture, profiles/mbconv_fp32_kernels.md"
 
     # ---- end to end: images from pinned host memory, result back to the host, same C-ABI calls --------
     hin = [torch.from_numpy(wl.inputs["X"]).pin_memory() for _ in range(SETS)]
@@ -324,8 +324,8 @@ def main():
             "ms_per_step": round(ms_step, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
             "config": {"workload": WORKLOAD, "bytes_per_step": bytes_step, "launches_per_step": nb,
-                       "l2": f"steps rotate over {SETS} independent buffer sets of {bytes_step // 2 // 1000000} MB each (> L2)",
-                       "launch_mode": "plain stream launches of dnnf_run; kernels chained by programmatic dependent launch"},
+                       "l2": f"steps rotate over {SETS} buffer sets of {bytes_step // 2 // 1000000} MB each (> L2)",
+                       "launch_mode": "plain stream launches, PDL between kernels"},
             "frac_of_hbm_peak": round(value / world / pk["hbm_gbs"], 4),
             "clocks": clk.summary(), "e2e": e2e, "gpu_launches": steps * nb, "roofline": roof, "kernels": kernels}
 
@@ -345,7 +345,8 @@ def main():
         from paper_2108_13342_b200 import report
         detail = report.per_config(dev, pk)
         for name, fn in [("cfg5 12-layer encoder (576 primitive operators)", report.encoder_report),
-                         ("next: 12-layer GPT-2 style decoder (633 primitive operators)", report.decoder_report)]:
+                         ("next: 12-layer GPT-2 style decoder (633 primitive operators)", report.decoder_report),
+                         ("next: layout selection on the MobileNetV2-shaped stack written channels-first", report.layout_report)]:
             try:
                 detail[name] = fn(dev, pk)
             except Exception as e:  # noqa: BLE001

@@ -141,6 +141,10 @@ typedef struct {
 #define DNNF_REWRITE_NONE           1u   /* leave the graph as given */
 #define DNNF_REWRITE_CANON_MACRO    2u   /* also fold the 9-operator LayerNorm expansion into one LayerNorm
                                             operator (an extension beyond the paper's printed rules) */
+#define DNNF_REWRITE_KEEP_LAYOUT    4u   /* skip the layout selection of Section 4.4.2: leave every Transpose where the graph
+                                            has it (by default element-wise operators and batch normalisation take the layout
+                                            of the convolution, pool, GEMM or Softmax they feed, and Transposes that then
+                                            meet their inverse disappear) */
 /* dnnf_plan flags */
 #define DNNF_PLAN_FUSED             0u
 #define DNNF_PLAN_UNFUSED           1u   /* one block per operator: the no-fusion baseline of Section 5 ("OurB") */
@@ -172,6 +176,7 @@ typedef struct {
   int32_t rules_applied;
   int32_t applied_by_rule[16];             /* index: see dnnf_rule_name() */
   int32_t folded_constants;
+  int32_t layout_transposes_removed;       /* Transposes the layout selection took out of the graph */
 } dnnf_rewrite_stats;
 
 typedef struct {

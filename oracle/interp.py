@@ -277,6 +277,54 @@ def op_greater(a, b): return np.where(a > b, 1.0, 0.0)     # multidirectional br
 def op_prelu(x, slope): return np.where(x > 0, x, slope * x)
 
 
+# ---- further Table 2 operators: Where, Cast (One-to-One); CumSum, InstanceNormalization (Many-to-Many) ----
+
+def op_where(cond, a, b):
+    """y = a where cond is non-zero, else b; cond is a 0 / 1 valued tensor; multidirectional broadcasting.
+    A selection, not arithmetic: an infinity or NaN in the branch that is not taken leaves no trace."""
+    return np.where(np.asarray(cond) != 0, a, b)
+
+
+def _round_to_bf16(x):
+    """Nearest bfloat16 (8 significand bits), ties to even, of the fp32 value nearest to x."""
+    bits = np.asarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    bits = (bits + 0x7FFF + ((bits >> 16) & 1)) & 0xFFFF0000
+    return bits.astype(np.uint32).view(np.float32).astype(np.float64)
+
+
+def op_cast(x, to):
+    """ONNX Cast between the value types a graph here can hold.  "f32": unchanged; "bf16": nearest bfloat16, ties to
+    even; "i32": the integer toward zero (the float-to-integer conversion); "bool": 1 where x is non-zero, else 0.
+    Integer and boolean results stay stored as floating-point numbers with those values."""
+    x = np.asarray(x, dtype=np.float64)
+    if to == "f32": return x
+    if to == "bf16": return _round_to_bf16(x).reshape(x.shape)
+    if to == "i32": return np.trunc(x)
+    if to == "bool": return np.where(x != 0, 1.0, 0.0)
+    raise ValueError(f"Cast: unknown target {to}")
+
+
+def op_cumsum(x, axis=-1, exclusive=0, reverse=0):
+    """ONNX CumSum along `axis`: y[i] = sum of x[j] over j <= i (j < i when exclusive), counted from the far end
+    when reverse."""
+    x = np.asarray(x, dtype=np.float64)
+    ax = _axis(axis, x.ndim)
+    if reverse: x = np.flip(x, ax)
+    y = np.cumsum(x, axis=ax)
+    if exclusive: y = y - x
+    if reverse: y = np.flip(y, ax)
+    return y
+
+
+def op_instancenorm(x, scale, bias, eps=1e-5):
+    """ONNX InstanceNormalization on an NHWC tensor: every image n and channel c is normalised by the mean and the
+    (biased) variance over its own H x W positions, then scaled and shifted per channel."""
+    x = np.asarray(x, dtype=np.float64)
+    mean = x.mean(axis=(1, 2), keepdims=True)
+    var = ((x - mean) ** 2).mean(axis=(1, 2), keepdims=True)
+    return (x - mean) / np.sqrt(var + float(eps)) * np.asarray(scale, dtype=np.float64) + np.asarray(bias, dtype=np.float64)
+
+
 # ---- dispatcher -------------------------------------------------------------
 
 def _apply(op, ins, at):
@@ -338,6 +386,10 @@ def _apply(op, ins, at):
     if op == "ReduceMean": return [op_reducemean(ins[0], g("axis", -1), g("keepdims", 1))]
     if op == "ReduceProd": return [op_reduceprod(ins[0], g("axis", -1), g("keepdims", 1))]
     if op == "ReduceMax": return [op_reducemax(ins[0], g("axis", -1), g("keepdims", 1))]
+    if op == "Where": return [op_where(ins[0], ins[1], ins[2])]
+    if op == "Cast": return [op_cast(ins[0], at["to"])]
+    if op == "CumSum": return [op_cumsum(ins[0], g("axis", -1), g("exclusive", 0), g("reverse", 0))]
+    if op == "InstanceNorm": return [op_instancenorm(ins[0], ins[1], ins[2], g("eps", 1e-5))]
     raise KeyError(f"oracle: unknown operator {op}")
 
 

@@ -40,7 +40,7 @@ ATTR = {"c": 1, "lo": 2, "hi": 3, "p": 4, "eps": 5, "approx": 6, "axis": 7, "kee
         "alpha": 1}      # LeakyRelu's slope travels as attribute C
 _FLOAT_ATTRS = {"c", "lo", "hi", "p", "eps", "alpha"}
 
-REWRITE_DEFAULT, REWRITE_NONE, REWRITE_CANON_MACRO = 0, 1, 2
+REWRITE_DEFAULT, REWRITE_NONE, REWRITE_CANON_MACRO, REWRITE_KEEP_LAYOUT = 0, 1, 2, 4
 PLAN_FUSED, PLAN_UNFUSED, PLAN_STRICT_TABLE3, PLAN_ALLOW_PROLOGUE, PLAN_BEYOND_TABLE3 = 0, 1, 2, 4, 8
 # kernel-selection overrides (same blocks and results, another kernel of the family)
 PLAN_SPLIT_ALWAYS, PLAN_NO_K_SLICES, PLAN_NO_COLUMN_BLOCKS, PLAN_NO_TF32_GEMM = 0x100, 0x200, 0x400, 0x800
@@ -56,7 +56,7 @@ class Attr(C.Structure):
 class RewriteStats(C.Structure):
     _fields_ = [("ops_before", C.c_int32), ("ops_after", C.c_int32), ("flops_before", C.c_int64),
                 ("flops_after", C.c_int64), ("rules_applied", C.c_int32), ("applied_by_rule", C.c_int32 * 16),
-                ("folded_constants", C.c_int32)]
+                ("folded_constants", C.c_int32), ("layout_transposes_removed", C.c_int32)]
 
 
 class PlanStats(C.Structure):
@@ -329,7 +329,8 @@ class Graph:
             out.append({"family": FAMILY_NAMES[d.family], "mapping": MAPPING_NAMES[d.mapping],
                         "ops": [OP_NAMES[d.op_kinds[i]] for i in range(min(d.n_ops, 48))],
                         "bytes": d.bytes_in + d.bytes_out, "flops": d.flops, "grid": d.grid,
-                        "threads": d.threads, "variant": d.variant, "n_microops": d.n_microops})
+                        "threads": d.threads, "variant": d.variant, "n_microops": d.n_microops,
+                        "n_inputs": d.n_inputs, "n_outputs": d.n_outputs})
         return out
 
 

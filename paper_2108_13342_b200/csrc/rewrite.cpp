@@ -127,6 +127,130 @@ struct Rewriter {
     return any;
   }
 
+  // ---- layout selection (Section 4.4.2, "inter-block optimization") -----------------------------
+  // The operators whose speed depends on the data layout -- convolutions, pools, GEMMs, Softmax and the
+  // other last-axis operators -- exist here in one layout each, so a graph written in another layout
+  // (a channels-first network) reaches them through Transposes: those Transposes state the layout the
+  // dominant operator of the coming block wants.  Element-wise operators and batch normalisation are
+  // indifferent to layout, so they take the dominant operator's: a Transpose is moved from the output
+  // of such an operator to its operands (f(x)^T = f(x^T), a per-channel operand follows its axis),
+  // and moved again, until it meets the Transpose that brought the tensor into the other layout; the
+  // two compose, to nothing when they are inverses.  What remains are Transposes of graph inputs and
+  // outputs.  The pass is kept only if the graph has fewer Transposes and no more #FLOPS than before.
+  static std::vector<int64_t> compose_perm(const std::vector<int64_t>& first, const std::vector<int64_t>& then) {
+    std::vector<int64_t> r(then.size());
+    for (size_t i = 0; i < then.size(); ++i) r[i] = first[then[i]];
+    return r;
+  }
+  static bool identity_perm(const std::vector<int64_t>& p) {
+    for (size_t i = 0; i < p.size(); ++i) if (p[i] != (int64_t)i) return false;
+    return true;
+  }
+  bool layout_indifferent(const Op& o) const {
+    if (!is_elementwise(o.kind) || o.out.size() != 1) return false;
+    return true;
+  }
+  // Can a Transpose by `perm` of tensor t be expressed without a new data movement?
+  bool transposable(int t, const std::vector<int64_t>& perm, int out_numel, std::map<int, bool>& memo, int depth = 0) {
+    auto it = memo.find(t);
+    if (it != memo.end()) return it->second;
+    bool ok = false;
+    const Tensor& T = g.tensors[t];
+    const Op* p = producer(t);
+    if (T.dims.size() != perm.size()) ok = false;
+    else if (p && p->kind == DNNF_OP_TRANSPOSE) ok = true;
+    else if (T.numel() < out_numel && !p) ok = true;               // a broadcast constant: permuting it costs no pass over the data
+    else if (p && layout_indifferent(*p) && depth < 64) {
+      ok = true;
+      for (size_t i = 0; i < p->in.size() && ok; ++i) {
+        if (p->kind == DNNF_OP_SCALESHIFT && i > 0) continue;
+        const Tensor& a = g.tensors[p->in[i]];
+        if (a.numel() == 1) continue;
+        ok = transposable(p->in[i], perm, out_numel, memo, depth + 1);
+      }
+    } else {
+      // some other consumer already reads this tensor through the same Transpose
+      for (int c : T.consumers) if (g.ops[c].alive && g.ops[c].kind == DNNF_OP_TRANSPOSE && g.ops[c].at.perm == perm) ok = true;
+      if (ok && depth == 0) ok = false;
+    }
+    memo[t] = ok;
+    return ok;
+  }
+  // Transposes of feature maps; one of a (broadcast) weight moves no data worth counting
+  int count_transposes() const {
+    int n = 0;
+    for (auto& o : g.ops) if (o.alive && o.kind == DNNF_OP_TRANSPOSE && !g.tensors[o.in[0]].weight) n++;
+    return n;
+  }
+
+  int crossings = 0;      // Transposes moved across a layout-indifferent operator
+  bool move_transposes_once() {
+    g.relink();
+    for (int oid : g.topo_order()) {
+      const Op T = g.ops[oid];
+      if (!T.alive || T.kind != DNNF_OP_TRANSPOSE) continue;
+      const int x = T.in[0], y = T.out[0];
+      const Op* P = producer(x);
+      if (!P) continue;
+      if (P->kind == DNNF_OP_TRANSPOSE) {
+        std::vector<int64_t> r = compose_perm(P->at.perm, T.at.perm);
+        const int src = P->in[0];
+        if (identity_perm(r)) {
+          if (g.tensors[y].is_output) continue;
+          for (auto& c : g.ops) if (c.alive) for (int& t : c.in) if (t == y) t = src;
+          g.ops[oid].alive = false;
+        } else {
+          Attrs at; at.perm = r;
+          if (add_op(DNNF_OP_TRANSPOSE, {src}, at, y) < 0) continue;
+        }
+        return true;
+      }
+      if (!layout_indifferent(*P)) continue;
+      std::map<int, bool> memo;
+      const int out_numel = (int)std::min<int64_t>(g.tensors[x].numel(), INT32_MAX);
+      if (!transposable(x, T.at.perm, out_numel, memo)) continue;
+      const Op Pc = *P;
+      std::vector<int> ins;
+      bool ok = true;
+      for (size_t i = 0; i < Pc.in.size() && ok; ++i) {
+        const Tensor& a = g.tensors[Pc.in[i]];
+        if ((Pc.kind == DNNF_OP_SCALESHIFT && i > 0) || a.numel() == 1) { ins.push_back(Pc.in[i]); continue; }
+        Attrs at; at.perm = T.at.perm;
+        int t = add_op(DNNF_OP_TRANSPOSE, {Pc.in[i]}, at);
+        if (t < 0) ok = false;
+        ins.push_back(t);
+      }
+      if (!ok) continue;
+      Attrs at = Pc.at;
+      if (Pc.kind == DNNF_OP_SCALESHIFT) {
+        const int64_t rank = (int64_t)T.at.perm.size();
+        const int64_t axis = Pc.at.axis < 0 ? Pc.at.axis + rank : Pc.at.axis;
+        for (int64_t i = 0; i < rank; ++i) if (T.at.perm[i] == axis) at.axis = i;
+      }
+      if (add_op(Pc.kind, ins, at, y) < 0) continue;
+      ++crossings;
+      return true;
+    }
+    return false;
+  }
+
+  void select_layouts() {
+    if (count_transposes() < 2) return;
+    Graph saved = g;
+    const int n_before = count_transposes();
+    const int64_t f_before = flops();
+    int moves = 0;
+    crossings = 0;
+    while (moves < 100000 && move_transposes_once()) { ++moves; }
+    while (cse()) {}
+    dce();
+    const int n_after = count_transposes();
+    // Back-to-back Transposes alone (the head split followed by K^T in attention) are left as the graph has them:
+    // they already share a block and compose there as index maps.
+    if (crossings == 0 || n_after >= n_before || flops() > f_before) { g = saved; g.relink(); return; }
+    st.layout_transposes_removed = n_before - n_after;
+  }
+
   // ---- product trees: flatten, simplify the multiset of factors, rebuild -----------------------
   void collect_factors(int t, int root, std::vector<int>& leaves, std::vector<int>& inner) {
     const Op* p = producer(t);
@@ -372,6 +496,7 @@ struct Rewriter {
     st.ops_before = 0;
     for (auto& o : g.ops) if (o.alive) st.ops_before++;
     st.flops_before = flops();
+    if (!(flags & DNNF_REWRITE_KEEP_LAYOUT)) select_layouts();
     for (int round = 0; round < 100000; ++round) {
       if (cse()) dce();
       std::vector<Candidate> cands;

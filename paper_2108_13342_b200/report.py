@@ -188,8 +188,22 @@ def encoder_latency_pair(dev, pk, layers=12):
     # reported apart: the plan that also fuses what Table 3 forbids (each attention head's three blocks as one kernel)
     x = measure_workload(torch, dev, wl, pk, B.PLAN_FUSED | B.PLAN_BEYOND_TABLE3, 1, iters=20, rewrite=B.REWRITE_CANON_MACRO, per_block_limit=0)
     torch.cuda.empty_cache()
-    return {"workload": "configs[4]: 12-layer encoder, 576 primitive operators, bf16", "cfg5_fused_us": f["us_cuda_graph"],
+    return {"workload": "configs[4]: 12-layer encoder, 576 operators, bf16; CUDA-graph replays", "cfg5_fused_us": f["us_cuda_graph"],
             "cfg5_beyond_table3_us": x["us_cuda_graph"], "cfg5_beyond_table3_kernels": x["kernels"],
             "cfg5_unfused_us": u["us_cuda_graph"], "cfg5_fused_plain_us": f["us_plain_launches"],
             "cfg5_unfused_plain_us": u["us_plain_launches"], "cfg5_fused_kernels": f["kernels"], "cfg5_unfused_kernels": u["kernels"],
             "cfg5_sum_of_block_rooflines_us": 160.0}
+
+
+def layout_report(dev, pk):
+    """Layout selection (Section 4.4.2) on the MobileNetV2-shaped stack: the network written channels-first with a
+    Transpose around every convolution and pool, planned with and without the pass, beside the channels-last network."""
+    import torch
+    out = {}
+    for name, wl, rw in [("channels-last graph", W.mbconv_stack(), B.REWRITE_DEFAULT),
+                         ("channels-first graph, layout selection", W.mbconv_stack(layout="nchw"), B.REWRITE_DEFAULT),
+                         ("channels-first graph, Transposes kept", W.mbconv_stack(layout="nchw"), B.REWRITE_KEEP_LAYOUT)]:
+        r = measure_workload(torch, dev, wl, pk, B.PLAN_FUSED, 1, iters=20, rewrite=rw, per_block_limit=0)
+        out[name] = {k: r[k] for k in ("ops", "kernels", "us_cuda_graph", "us_plain_launches", "irs_bytes")}
+        torch.cuda.empty_cache()
+    return out

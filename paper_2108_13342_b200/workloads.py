@@ -330,14 +330,23 @@ def cnn_neck(n=8, h=64, w=64, c=32, seed=BASE_SEED) -> Workload:
     return Workload(g, ins, note="fp32 NHWC")
 
 
-def mbconv_stack(n=32, hw=56, seed=BASE_SEED) -> Workload:
+def mbconv_stack(n=32, hw=56, seed=BASE_SEED, layout="nhwc") -> Workload:
     """A MobileNetV2-shaped stack of inverted-residual blocks in NHWC fp32 (expand 1x1 + BN + ReLU6, depthwise 3x3 + BN +
     ReLU6, project 1x1 + BN, residual where the shapes agree) with the channel progression 16-24-32-64-96-160 and
     expansion 6, MaxPool 3x3 / 2 between the stages (the library's depthwise kernel has stride 1), a 1x1 head, global
     average pool and a classifier: the convolution side of the paper's model zoo (Section 5) as one synthetic graph.
-    Expansions beyond 192 channels and projections deeper than 244 exercise the planner's column-block and K splits."""
+    Expansions beyond 192 channels and projections deeper than 244 exercise the planner's column-block and K splits.
+
+    layout="nchw" describes the same network the way a channels-first exporter writes it: the image X and every
+    feature map are [n, c, h, w], batch normalisation scales axis 1, ReLU6 and the residual Add act on channels-first
+    tensors, and each operator the library defines channels-last only (the convolutions and the pools) sits between a
+    Transpose to NHWC and a Transpose back.  The values are those of the NHWC graph with X transposed (same seeds), so
+    the logits agree: the case for inter-block layout selection (Section 4.4.2)."""
+    if layout not in ("nhwc", "nchw"):
+        raise ValueError("layout is 'nhwc' or 'nchw'")
+    cf = layout == "nchw"
     d = _Draw(seed + 11)
-    g = GraphDesc("mbconv_stack")
+    g = GraphDesc("mbconv_stack" + ("_nchw" if cf else ""))
     ins = {}
     cnt = [0]
 
@@ -349,26 +358,37 @@ def mbconv_stack(n=32, hw=56, seed=BASE_SEED) -> Workload:
         return name
 
     def bn(x, c):
-        return g.add("ScaleShift", [x, ext((c,), 0.5, 1.5), ext((c,), -0.5, 0.5)], axis=-1)
+        return g.add("ScaleShift", [x, ext((c,), 0.5, 1.5), ext((c,), -0.5, 0.5)], axis=1 if cf else -1)
+
+    def channels_last(kind, ins, **attrs):
+        """An operator the library defines on NHWC tensors; in the channels-first graph it is wrapped in Transposes."""
+        if not cf:
+            return g.add(kind, ins, **attrs)
+        y = g.add(kind, [g.add("Transpose", [ins[0]], perm=(0, 2, 3, 1))] + list(ins[1:]), **attrs)
+        return g.add("Transpose", [y], perm=(0, 3, 1, 2))
 
     def block(x, cin, cout, t=6):
         e = cin * t
-        y = g.add("Clip", [bn(g.add("Conv1x1", [x, ext((cin, e), std=math.sqrt(2.0 / cin))]), e)], lo=0.0, hi=6.0)
-        y = g.add("Clip", [bn(g.add("DwConv3x3", [y, ext((3, 3, e), std=math.sqrt(2.0 / 9.0))]), e)], lo=0.0, hi=6.0)
-        y = bn(g.add("Conv1x1", [y, ext((e, cout), std=math.sqrt(1.0 / e))]), cout)
+        y = g.add("Clip", [bn(channels_last("Conv1x1", [x, ext((cin, e), std=math.sqrt(2.0 / cin))]), e)], lo=0.0, hi=6.0)
+        y = g.add("Clip", [bn(channels_last("DwConv3x3", [y, ext((3, 3, e), std=math.sqrt(2.0 / 9.0))]), e)], lo=0.0, hi=6.0)
+        y = bn(channels_last("Conv1x1", [y, ext((e, cout), std=math.sqrt(1.0 / e))]), cout)
         return g.add("Add", [y, x]) if cin == cout else y
 
-    x = ext((n, hw, hw, 16), 0.0, 1.0, name="X")
+    x = ext((n, 16, hw, hw) if cf else (n, hw, hw, 16), 0.0, 1.0, name="X")
+    if cf:
+        ins["X"] = np.ascontiguousarray(ins["X"].reshape(n, hw, hw, 16).transpose(0, 3, 1, 2))
     x = block(x, 16, 24); x = block(x, 24, 24)
-    x = g.add("MaxPool", [x], kernel=3, stride=2, pad=1)
+    x = channels_last("MaxPool", [x], kernel=3, stride=2, pad=1)
     x = block(x, 24, 32); x = block(x, 32, 32); x = block(x, 32, 64)
-    x = g.add("MaxPool", [x], kernel=3, stride=2, pad=1)
+    x = channels_last("MaxPool", [x], kernel=3, stride=2, pad=1)
     x = block(x, 64, 64); x = block(x, 64, 96); x = block(x, 96, 96); x = block(x, 96, 160)
-    x = g.add("Clip", [bn(g.add("Conv1x1", [x, ext((160, 320), std=math.sqrt(2.0 / 160))]), 320)], lo=0.0, hi=6.0)
-    x = g.add("AveragePool", [x], kernel=hw // 4, stride=1, pad=0)                 # [n, 1, 1, 320]
+    x = g.add("Clip", [bn(channels_last("Conv1x1", [x, ext((160, 320), std=math.sqrt(2.0 / 160))]), 320)], lo=0.0, hi=6.0)
+    x = channels_last("AveragePool", [x], kernel=hw // 4, stride=1, pad=0)                 # [n, 1, 1, 320] (NHWC)
+    if cf:
+        x = g.add("Transpose", [x], perm=(0, 2, 3, 1))
     x = g.add("Add", [g.add("Conv1x1", [x, ext((320, 100), std=math.sqrt(1.0 / 320))]), ext((100,), -0.1, 0.1)], out="logits")
     g.mark_output(x)
-    return Workload(g, ins, note="fp32 NHWC")
+    return Workload(g, ins, note="fp32 " + layout.upper())
 
 
 # --------------------------------------------------------------------------

@@ -291,3 +291,37 @@ def test_mobilenet_shaped_stack(flags, always):
         assert fams.count("gemm") >= 20, fams          # the split pieces
     if flags == B.PLAN_FUSED:
         assert s.plan_stats.n_kernels < s.plan_stats.n_ops
+
+
+# ---- Section 4.4.2: layout selection ---------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("rewrite", [B.REWRITE_DEFAULT, B.REWRITE_KEEP_LAYOUT])
+def test_channels_first_stack_with_and_without_layout_selection(rewrite):
+    """The MobileNetV2-shaped stack written channels-first (a Transpose around every convolution and pool, batch
+    normalisation on axis 1): same logits as the oracle's evaluation of that graph, whether the layout selection
+    re-expresses the element-wise operators channels-last or every Transpose stays an index map."""
+    wl = W.mbconv_stack(n=4, hw=48, layout="nchw")
+    s = check(wl, 5e-4, B.PLAN_FUSED, rewrite)
+    kinds = [k for b in s.g.blocks() for k in b["ops"]]
+    assert kinds.count("Transpose") == (1 if rewrite == B.REWRITE_DEFAULT else 63)
+
+
+def test_layout_selection_keeps_values_on_small_graphs():
+    # composed (non-inverse) Transposes, a per-channel operand that follows its axis, a broadcast operand of full rank
+    g = graph(); g.ext("X", (3, 5, 6, 7)); g.ext("s", (7,), kind="weight"); g.ext("t", (7,), kind="weight"); g.ext("b", (1, 7, 1, 1), kind="weight")
+    y = g.add("Transpose", [g.add("Sigmoid", ["X"])], perm=(0, 3, 1, 2))                    # [3, 7, 5, 6]
+    y = g.add("Add", [g.add("ScaleShift", [y, "s", "t"], axis=1), "b"])
+    y = g.add("Transpose", [g.add("Tanh", [y])], perm=(0, 1, 3, 2))                          # [3, 7, 6, 5]
+    g.mark_output(g.add("Softmax", [y], axis=-1))
+    ins = {"X": rnd((3, 5, 6, 7), 1), "s": rnd((7,), 2, 0.5, 1.5), "t": rnd((7,), 3), "b": rnd((1, 7, 1, 1), 4)}
+    s = check(W.Workload(g, ins), RTOL_F32, B.PLAN_FUSED, B.REWRITE_DEFAULT)
+    assert s.rewrite_stats.layout_transposes_removed == 1
+    # a residual Add whose operands both come back from the other layout, between two convolutions
+    g = graph(); g.ext("X", (2, 9, 9, 16)); g.ext("W", (16, 16), kind="weight"); g.ext("s", (16,), kind="weight"); g.ext("t", (16,), kind="weight")
+    a = g.add("Transpose", [g.add("Conv1x1", ["X", "W"])], perm=(0, 3, 1, 2))
+    a = g.add("Clip", [g.add("ScaleShift", [a, "s", "t"], axis=1)], lo=0.0, hi=6.0)
+    y = g.add("Transpose", [g.add("Add", [a, g.add("Transpose", ["X"], perm=(0, 3, 1, 2))])], perm=(0, 2, 3, 1))
+    g.mark_output(g.add("Conv1x1", [y, "W"]))
+    ins = {"X": rnd((2, 9, 9, 16), 5), "W": rnd((16, 16), 6, -0.3, 0.3), "s": rnd((16,), 7, 0.5, 1.5), "t": rnd((16,), 8)}
+    s = check(W.Workload(g, ins), 5e-4, B.PLAN_FUSED, B.REWRITE_DEFAULT)
+    assert s.rewrite_stats.layout_transposes_removed == 3

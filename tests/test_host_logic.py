@@ -582,3 +582,67 @@ def test_blocks_that_would_need_each_other_are_not_formed():
             for o in b["ops"]:
                 order.setdefault(o, i)
         assert st.n_kernels >= 2
+
+
+# ---- Section 4.4.2: layout selection ---------------------------------------------------------------------------------
+
+def _rewritten_kinds(desc, flags=B.REWRITE_DEFAULT):
+    G, ids = build_graph(desc)
+    st = G.rewrite(flags)
+    G.plan(B.PLAN_FUSED)
+    kinds = [k for b in G.blocks() for k in b["ops"]]
+    return G, st, kinds
+
+
+def test_layout_selection_gives_elementwise_operators_the_layout_of_the_dominant_one():
+    """A channels-first network reaches the channels-last convolutions and pools through Transposes.  Batch normalisation,
+    ReLU6 and the residual Adds take the convolutions' layout, every Transpose pair between them cancels, and what is left
+    is the NHWC network behind one Transpose of the input image."""
+    nhwc = W.mbconv_stack(n=2, hw=16)
+    nchw = W.mbconv_stack(n=2, hw=16, layout="nchw")
+    Ga, sa, ka = _rewritten_kinds(nhwc.graph)
+    Gb, sb, kb = _rewritten_kinds(nchw.graph)
+    assert sa.layout_transposes_removed == 0
+    assert sb.ops_before == 147 and sb.ops_after == sa.ops_after + 1
+    assert sb.layout_transposes_removed == 62 and kb.count("Transpose") == 1
+    assert sb.flops_after == sa.flops_after
+    fam = lambda G: sorted(b["family"] for b in G.blocks())
+    assert fam(Gb) == sorted(fam(Ga) + ["transpose"])
+    assert all(b["n_outputs"] == 1 for b in Gb.blocks())
+    # without the pass the residual sources are stored twice, once per layout
+    Gc, sc, kc = _rewritten_kinds(nchw.graph, B.REWRITE_KEEP_LAYOUT)
+    assert sc.layout_transposes_removed == 0 and sc.ops_after == 147
+    assert sum(b["n_outputs"] for b in Gc.blocks()) > len(Gc.blocks())
+
+
+def test_layout_selection_small_cases():
+    # inverse Transposes around a layout-indifferent chain cancel; the per-channel operand follows its axis
+    g = _desc(); g.ext("X", (2, 5, 6, 7)); g.ext("s", (7,), kind="weight"); g.ext("t", (7,), kind="weight")
+    y = g.add("Transpose", [g.add("Relu", ["X"])], perm=(0, 3, 1, 2))
+    y = g.add("Clip", [g.add("ScaleShift", [y, "s", "t"], axis=1)], lo=0.0, hi=6.0)
+    g.mark_output(g.add("Sigmoid", [g.add("Transpose", [y], perm=(0, 2, 3, 1))]))
+    G, st, kinds = _rewritten_kinds(g)
+    assert st.layout_transposes_removed == 2 and kinds == ["Relu", "ScaleShift", "Clip", "Sigmoid"]
+    # Transposes that are not inverses compose into one
+    g = _desc(); g.ext("X", (2, 5, 6, 7))
+    y = g.add("Tanh", [g.add("Transpose", [g.add("Relu", ["X"])], perm=(0, 3, 1, 2))])
+    g.mark_output(g.add("Transpose", [y], perm=(0, 1, 3, 2)))
+    G, st, kinds = _rewritten_kinds(g)
+    assert st.layout_transposes_removed == 1 and kinds.count("Transpose") == 1
+    # an operator that fixes a layout (Softmax on the last axis) is not crossed
+    g = _desc(); g.ext("X", (2, 5, 6, 7))
+    y = g.add("Softmax", [g.add("Transpose", ["X"], perm=(0, 3, 1, 2))], axis=-1)
+    g.mark_output(g.add("Transpose", [y], perm=(0, 2, 3, 1)))
+    G, st, kinds = _rewritten_kinds(g)
+    assert st.layout_transposes_removed == 0 and kinds.count("Transpose") == 2
+    # a lone Transpose behind element-wise operators stays where the graph has it (nothing to meet)
+    G, st, kinds = _rewritten_kinds(W.swish_transpose(n=1, c=8, h=4, w=4).graph)
+    assert st.layout_transposes_removed == 0 and kinds[-1] == "Transpose"
+    # both operands of a residual Add come back from the other layout
+    g = _desc(); g.ext("X", (2, 4, 4, 8)); g.ext("W", (8, 8), kind="weight")
+    a = g.add("Transpose", [g.add("Conv1x1", ["X", "W"])], perm=(0, 3, 1, 2))
+    b = g.add("Transpose", ["X"], perm=(0, 3, 1, 2))
+    y = g.add("Transpose", [g.add("Add", [g.add("Relu", [a]), b])], perm=(0, 2, 3, 1))
+    g.mark_output(g.add("Conv1x1", [y, "W"]))
+    G, st, kinds = _rewritten_kinds(g)
+    assert st.layout_transposes_removed == 3 and "Transpose" not in kinds

@@ -441,3 +441,116 @@ def test_generators_are_counter_based_and_distributed():
     r = W.round_to_bf16(np.array([1.0, 1.00390625, 1.01171875, 3.14159], dtype=np.float32))
     assert r[0] == 1.0 and r[1] == 1.0 and r[2] == 1.015625    # ties to even, both directions
     assert np.array_equal(W.bf16_bits_to_f32(W.bf16_bits(r)), r)
+
+
+# ---- Where, Cast, CumSum, InstanceNormalization (Table 2) -------------------------------------------------------------
+
+def test_where_index_loops_and_selection_semantics():
+    r = np.random.default_rng(5)
+    cond = (r.random((3, 1, 5)) > 0.5).astype(np.float64)
+    a = r.standard_normal((1, 4, 5)); b = r.standard_normal((3, 4, 1))
+    y = O.op_where(cond, a, b)
+    assert y.shape == (3, 4, 5)
+    for i, j, k in itertools.product(range(3), range(4), range(5)):
+        assert y[i, j, k] == (a[0, j, k] if cond[i, 0, k] != 0 else b[i, j, 0])
+    np.testing.assert_array_equal(O.op_where(np.ones((2, 3)), a[0, :2, :3], 7.0), a[0, :2, :3])
+    np.testing.assert_array_equal(O.op_where(np.zeros((2, 3)), a[0, :2, :3], 7.0), np.full((2, 3), 7.0))
+    # the branch that is not taken leaves no trace: the usual masking with -inf, and a NaN on the other side
+    y = O.op_where(np.array([1.0, 0.0, 1.0]), np.array([1.0, np.nan, 3.0]), np.array([-np.inf, 2.0, -np.inf]))
+    np.testing.assert_array_equal(y, [1.0, 2.0, 3.0])
+    # Where(Greater(x, 0), x, 0) is Relu; Where(Not(c), a, b) swaps the branches
+    x = r.standard_normal(50)
+    np.testing.assert_array_equal(O.op_where(O.op_greater(x, 0.0), x, 0.0), O.op_relu(x))
+    c = (r.random(50) > 0.5).astype(float)
+    np.testing.assert_array_equal(O.op_where(O.op_not(c), x, -x), O.op_where(c, -x, x))
+
+
+def test_cast_points_and_properties():
+    import torch
+    # bfloat16 keeps 8 significand bits: spacing 2^-7 in [1, 2); ties go to the even neighbour
+    e = 2.0 ** -7
+    pts = {1.0: 1.0, 1.0 + e / 2: 1.0, 1.0 + 3 * e / 2: 1.0 + 2 * e, 1.0 + e / 2 + 2.0 ** -20: 1.0 + e, -1.0 - 3 * e / 2: -1.0 - 2 * e,
+           3.140625: 3.140625, 0.0: 0.0, 2.0 ** -130: 2.0 ** -130, 65280.0: 65280.0, 1e-3: 131 / 128 * 2.0 ** -10}        # 0.001 = 1.024 * 2^-10 and 1.024 * 128 = 131.07
+    for x, want in pts.items():
+        assert O.op_cast(np.array([x]), "bf16")[0] == want, (x, want)
+    r = np.random.default_rng(6)
+    x = np.concatenate([r.standard_normal(4000) * 10.0 ** r.integers(-6, 6, 4000), [0.0, -0.0, 1e30, -1e-30]])
+    y = O.op_cast(x, "bf16")
+    x32 = x.astype(np.float32).astype(np.float64)
+    assert np.all(np.abs(y - x32) <= 2.0 ** -8 * np.abs(x32))                         # half a unit in the last place: 2^-8 * 2^exponent
+    assert np.all((y.astype(np.float32).view(np.uint32) & 0xFFFF) == 0)               # representable in 16 bits
+    np.testing.assert_array_equal(O.op_cast(y, "bf16"), y)                            # idempotent
+    lib = torch.from_numpy(x.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    np.testing.assert_array_equal(y, lib)                                             # the library's conversion
+    # float -> integer conversion goes toward zero; bool is "non-zero"; f32 leaves values alone
+    v = np.array([-2.7, -2.0, -0.5, 0.0, 0.5, 1.999, 2.0, 1e6 + 0.75])
+    np.testing.assert_array_equal(O.op_cast(v, "i32"), [float(int(t)) for t in v])
+    np.testing.assert_array_equal(O.op_cast(v, "bool"), [1, 1, 1, 0, 1, 1, 1, 1])
+    np.testing.assert_array_equal(O.op_cast(v, "f32"), v)
+    np.testing.assert_array_equal(O.op_cast(v, "bool"), O.op_not(O.op_not(v)))
+
+
+def test_cumsum_running_loops_and_closed_forms():
+    r = np.random.default_rng(7)
+    x = r.standard_normal((3, 4, 6))
+    for axis in (0, 1, 2, -1):
+        for exclusive in (0, 1):
+            for reverse in (0, 1):
+                y = O.op_cumsum(x, axis, exclusive, reverse)
+                ax = axis % 3
+                xm = np.moveaxis(x, ax, -1); ym = np.moveaxis(y, ax, -1)
+                L = xm.shape[-1]
+                for i, j in itertools.product(range(xm.shape[0]), range(xm.shape[1])):
+                    order = range(L - 1, -1, -1) if reverse else range(L)
+                    run = 0.0
+                    for k in order:
+                        if exclusive:
+                            assert abs(ym[i, j, k] - run) < 1e-12
+                        run += xm[i, j, k]
+                        if not exclusive:
+                            assert abs(ym[i, j, k] - run) < 1e-12
+    n = 37
+    np.testing.assert_array_equal(O.op_cumsum(np.ones(n)), np.arange(1, n + 1))
+    np.testing.assert_array_equal(O.op_cumsum(np.ones(n), exclusive=1), np.arange(n))
+    np.testing.assert_array_equal(O.op_cumsum(np.ones(n), reverse=1), np.arange(n, 0, -1))
+    np.testing.assert_array_equal(O.op_cumsum(np.arange(1, n + 1)), [k * (k + 1) // 2 for k in range(1, n + 1)])   # triangular numbers
+    q = 0.5 ** np.arange(20)
+    np.testing.assert_allclose(O.op_cumsum(q), 2.0 - q, rtol=1e-15)                                                # geometric series
+    y = O.op_cumsum(x, -1)
+    np.testing.assert_allclose(y[..., -1], O.op_reducesum(x, -1, 0), rtol=1e-14)                                    # last element is the sum
+    np.testing.assert_allclose(np.diff(y, axis=-1), x[..., 1:], atol=1e-14)                                         # differences give x back
+    np.testing.assert_allclose(O.op_cumsum(x, -1) - O.op_cumsum(x, -1, exclusive=1), x, atol=1e-14)
+    np.testing.assert_allclose(O.op_cumsum(x, -1) + O.op_cumsum(x, -1, exclusive=1, reverse=1),
+                               np.broadcast_to(x.sum(-1, keepdims=True), x.shape), atol=1e-13)
+
+
+def test_instancenorm_index_loops_and_invariants():
+    r = np.random.default_rng(8)
+    N, H, Wd, Cc = 2, 3, 5, 4
+    x = r.standard_normal((N, H, Wd, Cc)) * 3 + 1
+    s = r.uniform(0.5, 1.5, Cc); b = r.uniform(-1, 1, Cc)
+    eps = 1e-5
+    y = O.op_instancenorm(x, s, b, eps)
+    for n, c in itertools.product(range(N), range(Cc)):
+        vals = [x[n, h, w, c] for h in range(H) for w in range(Wd)]
+        m = sum(vals) / len(vals)
+        v = sum((t - m) ** 2 for t in vals) / len(vals)
+        for h, w in itertools.product(range(H), range(Wd)):
+            assert abs(y[n, h, w, c] - ((x[n, h, w, c] - m) / math.sqrt(v + eps) * s[c] + b[c])) < 1e-12
+    # unit scale, zero shift: every (image, channel) plane has mean 0 and variance var / (var + eps)
+    z = O.op_instancenorm(x, np.ones(Cc), np.zeros(Cc), eps)
+    var = x.var(axis=(1, 2))
+    np.testing.assert_allclose(z.mean(axis=(1, 2)), 0.0, atol=1e-14)
+    np.testing.assert_allclose(z.var(axis=(1, 2)), var / (var + eps), rtol=1e-12)
+    # a per-plane affine change of the input is removed (exactly so as eps -> 0); planes do not see each other
+    a = r.uniform(0.5, 2.0, (N, 1, 1, Cc)); t = r.standard_normal((N, 1, 1, Cc))
+    np.testing.assert_allclose(O.op_instancenorm(a * x + t, s, b, 0.0), O.op_instancenorm(x, s, b, 0.0), atol=1e-12)
+    x2 = x.copy(); x2[1, :, :, 2] = r.standard_normal((H, Wd))
+    y2 = O.op_instancenorm(x2, s, b, eps)
+    mask = np.ones_like(x, dtype=bool); mask[1, :, :, 2] = False
+    np.testing.assert_array_equal(y2[mask], y[mask])
+    # a constant plane maps to the shift; it is LayerNorm over the H*W positions of the channels-first view
+    np.testing.assert_allclose(O.op_instancenorm(np.full((1, 2, 2, Cc), 5.0), s, b, eps), np.broadcast_to(b, (1, 2, 2, Cc)), atol=1e-12)
+    xt = x.transpose(0, 3, 1, 2).reshape(N, Cc, H * Wd)
+    ln = O.op_layernorm(xt, np.ones(H * Wd), np.zeros(H * Wd), -1, eps).reshape(N, Cc, H, Wd).transpose(0, 2, 3, 1)
+    np.testing.assert_allclose(y, ln * s + b, atol=1e-12)
