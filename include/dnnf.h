@@ -86,7 +86,7 @@ typedef enum {
   DNNF_OP_CONV1X1,                                  /* NHWC x [Cin,Cout] */
   DNNF_OP_DWCONV3X3,                                /* NHWC x [3,3,C], stride 1, zero pad 1 */
   DNNF_OP_SOFTMAX,                                  /* attribute AXIS (last axis only) */
-  DNNF_OP_LAYERNORM,                                /* (x, gamma, beta); attributes AXIS, EPS */
+  DNNF_OP_LAYERNORM,                                /* (x, gamma, beta), or (x) alone for no scale and shift; attributes AXIS, EPS */
   DNNF_OP_REDUCESUM, DNNF_OP_REDUCEMEAN, DNNF_OP_REDUCEMAX, DNNF_OP_REDUCEPROD, /* AXIS (last), KEEPDIMS */
   DNNF_OP_EXPAND,                                   /* attribute SHAPE */
   DNNF_OP_BITSHIFT,                                 /* attribute BITS; planning/rewriting only */
@@ -118,6 +118,18 @@ typedef enum {
                                                        Reshape(W) -> Conv1x1 -> DepthToSpace, which it equals term by term */
   DNNF_OP_GATHER,                                   /* One-to-Many; (table [V,D], indices [...]) along axis 0: y[..., :] = table[indices[...], :].
                                                        Indices are integer-valued fp32 numbers; out-of-range ones are clamped */
+  DNNF_OP_WHERE,                                    /* One-to-One (Table 2); (cond, a, b) with broadcasting: a where the 0 / 1 valued cond
+                                                       is non-zero, else b.  A selection: the other branch's value is never touched */
+  DNNF_OP_CAST,                                     /* One-to-One (Table 2); attribute TO: DNNF_CAST_F32 (values unchanged), DNNF_CAST_BF16
+                                                       (nearest bfloat16, ties to even; the result tensor is bf16), DNNF_CAST_I32 (the integer
+                                                       toward zero) or DNNF_CAST_BOOL (1 where non-zero, else 0); integer and boolean
+                                                       results are stored as fp32 numbers with those values */
+  DNNF_OP_CUMSUM,                                   /* Many-to-Many (Table 2); running sum along the last axis (attribute AXIS must name it);
+                                                       attributes EXCLUSIVE (sum of the elements before) and REVERSE (from the far end) */
+  DNNF_OP_INSTANCENORM,                             /* Many-to-Many (Table 2); (x NHWC, scale[C], shift[C]), attribute EPS: each image and
+                                                       channel is normalised by the mean and biased variance over its H x W positions.
+                                                       Recorded as Transpose -> Reshape [N,C,HW] -> LayerNorm (no scale / shift) ->
+                                                       Reshape -> Transpose -> ScaleShift, which it equals term by term */
   DNNF_OP_CONCATPART,                               /* internal (made by Concat): (x [, result so far]); AXIS, START, SHAPE */
   DNNF_OP__COUNT
 } dnnf_op_t;
@@ -126,8 +138,15 @@ typedef enum {
   DNNF_ATTR_C = 1, DNNF_ATTR_LO, DNNF_ATTR_HI, DNNF_ATTR_P, DNNF_ATTR_EPS,   /* use f */
   DNNF_ATTR_APPROX, DNNF_ATTR_AXIS, DNNF_ATTR_KEEPDIMS, DNNF_ATTR_START, DNNF_ATTR_END, DNNF_ATTR_BITS, /* use i[0] */
   DNNF_ATTR_PERM, DNNF_ATTR_SHAPE, DNNF_ATTR_SIZES, DNNF_ATTR_AXES,           /* use i[0..n) */
-  DNNF_ATTR_BLOCK, DNNF_ATTR_SCALE, DNNF_ATTR_KERNEL, DNNF_ATTR_STRIDE, DNNF_ATTR_PAD   /* use i[0] */
+  DNNF_ATTR_BLOCK, DNNF_ATTR_SCALE, DNNF_ATTR_KERNEL, DNNF_ATTR_STRIDE, DNNF_ATTR_PAD,  /* use i[0] */
+  DNNF_ATTR_TO, DNNF_ATTR_EXCLUSIVE, DNNF_ATTR_REVERSE                                    /* use i[0] */
 } dnnf_attr_key_t;
+
+/* Cast targets (attribute TO) */
+#define DNNF_CAST_F32   0
+#define DNNF_CAST_BF16  1
+#define DNNF_CAST_I32   2
+#define DNNF_CAST_BOOL  3
 
 typedef struct {
   int32_t key;      /* dnnf_attr_key_t */

@@ -32,12 +32,15 @@ OP_NAMES = ["?", "Add", "Sub", "Mul", "Div", "MulC", "AddC", "Sigmoid", "Tanh", 
             "Neg", "Recip", "Square", "Relu", "Clip", "Pow", "Gelu", "ScaleShift", "Transpose", "Reshape", "Flatten",
             "Squeeze", "Unsqueeze", "Split", "Slice", "MatMul", "Conv1x1", "DwConv3x3", "Softmax", "LayerNorm",
             "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift", "DepthToSpace", "SpaceToDepth", "Resize", "Concat", "MaxPool", "AveragePool", "Sin", "Cos", "Asin", "Ceil",
-            "Floor", "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConvTranspose", "Gather", "ConcatPart"]
+            "Floor", "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConvTranspose", "Gather", "Where", "Cast", "CumSum", "InstanceNorm",
+            "ConcatPart"]
 OP = {n: i for i, n in enumerate(OP_NAMES) if i}
 
 ATTR = {"c": 1, "lo": 2, "hi": 3, "p": 4, "eps": 5, "approx": 6, "axis": 7, "keepdims": 8, "start": 9, "end": 10,
         "bits": 11, "perm": 12, "shape": 13, "sizes": 14, "axes": 15, "block": 16, "scale": 17, "kernel": 18, "stride": 19, "pad": 20,
+        "to": 21, "exclusive": 22, "reverse": 23,
         "alpha": 1}      # LeakyRelu's slope travels as attribute C
+CAST_TO = {"f32": 0, "bf16": 1, "i32": 2, "bool": 3}
 _FLOAT_ATTRS = {"c", "lo", "hi", "p", "eps", "alpha"}
 
 REWRITE_DEFAULT, REWRITE_NONE, REWRITE_CANON_MACRO, REWRITE_KEEP_LAYOUT = 0, 1, 2, 4
@@ -179,6 +182,8 @@ class Graph:
                 v = {"erf": 0, "tanh": 1}[v]
             if k == "direction":
                 continue
+            if k == "to" and isinstance(v, str):
+                v = CAST_TO[v]
             a = Attr()
             a.key = ATTR[k]
             if k in _FLOAT_ATTRS:

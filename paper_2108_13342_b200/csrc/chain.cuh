@@ -219,6 +219,14 @@ __device__ __forceinline__ void apply_op(int op, float (&acc)[VV], const float (
 #pragma unroll
       for (int v = 0; v < VV; ++v) acc[v] = src[v] > 0.0f ? src[v] : acc[v] * src[v];
       break;
+    case M_BF16R:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = __bfloat162float(__float2bfloat16_rn(acc[v]));
+      break;
+    case M_TRUNC:
+#pragma unroll
+      for (int v = 0; v < VV; ++v) acc[v] = truncf(acc[v]);
+      break;
     default: break;
   }
 }
@@ -250,6 +258,22 @@ __device__ __forceinline__ void exec_one(const MicroOp m, ChainState<VV>& st, IO
   }
   if (m.op == M_STORE) { io.store(m.idx, st.acc); return; }
   if (m.op >= M_ROWSUM) { io.row_reduce(m.op, st.acc); return; }
+  if (m.op == M_SELECT || m.op == M_RSELECT) {       // acc = condition (saved value number m.pad) ? acc : operand, or the reverse
+    float src[VV];
+    if (m.src == S_IN) io.load(m.idx, src);
+    else if (m.src == S_ANCHOR) io.anchor(src);
+    else {
+      const float c = m.src == S_CONST ? prog.consts[m.idx] : 0.0f;
+#pragma unroll
+      for (int v = 0; v < VV; ++v) src[v] = m.src == S_TMP ? (m.idx == 0 ? st.t0[v] : st.t1[v]) : c;
+    }
+#pragma unroll
+    for (int v = 0; v < VV; ++v) {
+      const bool take_acc = ((m.pad == 0 ? st.t0[v] : st.t1[v]) != 0.0f) == (m.op == M_SELECT);
+      st.acc[v] = take_acc ? st.acc[v] : src[v];
+    }
+    return;
+  }
   float c0 = 0.0f, c1 = 0.0f;
   if (m.src == S_IN) {
     float src[VV];

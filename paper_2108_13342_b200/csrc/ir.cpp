@@ -60,7 +60,7 @@ const char* op_name(int k) {
     "Sqrt", "Abs", "Neg", "Recip", "Square", "Relu", "Clip", "Pow", "Gelu", "ScaleShift", "Transpose", "Reshape",
     "Flatten", "Squeeze", "Unsqueeze", "Split", "Slice", "MatMul", "Conv1x1", "DwConv3x3", "Softmax", "LayerNorm",
     "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift", "DepthToSpace", "SpaceToDepth", "Resize", "Concat", "MaxPool", "AveragePool", "Sin", "Cos", "Asin", "Ceil", "Floor",
-    "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConvTranspose", "Gather", "ConcatPart"};
+    "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConvTranspose", "Gather", "Where", "Cast", "CumSum", "InstanceNorm", "ConcatPart"};
   if (k <= 0 || k >= DNNF_OP__COUNT) return "?";
   return names[k];
 }
@@ -70,13 +70,15 @@ bool is_index_only(int k) {
          k == DNNF_OP_UNSQUEEZE || k == DNNF_OP_SLICE || k == DNNF_OP_SPLIT || k == DNNF_OP_EXPAND || k == DNNF_OP_CONCATPART;
 }
 bool is_elementwise(int k) {
-  return (k >= DNNF_OP_ADD && k <= DNNF_OP_SCALESHIFT) || k == DNNF_OP_BITSHIFT || (k >= DNNF_OP_SIN && k <= DNNF_OP_PRELU);
+  return (k >= DNNF_OP_ADD && k <= DNNF_OP_SCALESHIFT) || k == DNNF_OP_BITSHIFT || (k >= DNNF_OP_SIN && k <= DNNF_OP_PRELU) ||
+         k == DNNF_OP_WHERE || k == DNNF_OP_CAST;
 }
+bool is_broadcasting_elementwise(int k) { return is_binary_elementwise(k) || k == DNNF_OP_WHERE; }
 bool is_binary_elementwise(int k) {
   return k == DNNF_OP_ADD || k == DNNF_OP_SUB || k == DNNF_OP_MUL || k == DNNF_OP_DIV || k == DNNF_OP_GREATER || k == DNNF_OP_PRELU;
 }
 bool is_row_anchor(int k) {
-  return k == DNNF_OP_SOFTMAX || k == DNNF_OP_LAYERNORM || (k >= DNNF_OP_REDUCESUM && k <= DNNF_OP_REDUCEPROD);
+  return k == DNNF_OP_SOFTMAX || k == DNNF_OP_LAYERNORM || (k >= DNNF_OP_REDUCESUM && k <= DNNF_OP_REDUCEPROD) || k == DNNF_OP_CUMSUM;
 }
 bool is_contraction(int k) {      // anchors that take an epilogue chain and nothing in front
   return k == DNNF_OP_MATMUL || k == DNNF_OP_CONV1X1 || k == DNNF_OP_DWCONV3X3 || k == DNNF_OP_MAXPOOL || k == DNNF_OP_AVGPOOL ||
@@ -110,7 +112,7 @@ int edge_mapping(const Graph& g, const Op& op, int slot) {
   const Tensor& in = g.tensors[op.in[slot]];
   const Tensor& out = g.tensors[op.out[0]];
   int k = op.kind;
-  if (is_binary_elementwise(k))
+  if (is_broadcasting_elementwise(k))
     return same_shape(in, out) ? DNNF_ONE_TO_ONE : DNNF_ONE_TO_MANY;     // "elementwise w/ broadcast"
   if (k == DNNF_OP_SCALESHIFT) return slot == 0 ? DNNF_ONE_TO_ONE : DNNF_ONE_TO_MANY;
   if (k == DNNF_OP_LAYERNORM) return slot == 0 ? DNNF_MANY_TO_MANY : DNNF_ONE_TO_MANY;
@@ -120,7 +122,7 @@ int edge_mapping(const Graph& g, const Op& op, int slot) {
 int node_mapping(const Graph& g, const Op& op) {
   int k = op.kind;
   switch (k) {
-    case DNNF_OP_ADD: case DNNF_OP_SUB: case DNNF_OP_MUL: case DNNF_OP_DIV: case DNNF_OP_GREATER: case DNNF_OP_PRELU: {
+    case DNNF_OP_ADD: case DNNF_OP_SUB: case DNNF_OP_MUL: case DNNF_OP_DIV: case DNNF_OP_GREATER: case DNNF_OP_PRELU: case DNNF_OP_WHERE: {
       // most complex pair decides (Section 3.1)
       int m = DNNF_ONE_TO_ONE;
       for (int s = 0; s < (int)op.in.size(); ++s) m = std::max(m, edge_mapping(g, op, s));
@@ -133,7 +135,7 @@ int node_mapping(const Graph& g, const Op& op) {
     case DNNF_OP_EXPAND: case DNNF_OP_GATHER: return DNNF_ONE_TO_MANY;
     case DNNF_OP_MATMUL: case DNNF_OP_CONV1X1: case DNNF_OP_DWCONV3X3: case DNNF_OP_SOFTMAX: case DNNF_OP_LAYERNORM:
     case DNNF_OP_REDUCESUM: case DNNF_OP_REDUCEMEAN: case DNNF_OP_REDUCEMAX: case DNNF_OP_REDUCEPROD:
-    case DNNF_OP_MAXPOOL: case DNNF_OP_AVGPOOL:
+    case DNNF_OP_MAXPOOL: case DNNF_OP_AVGPOOL: case DNNF_OP_CUMSUM:
       return DNNF_MANY_TO_MANY;
     default: return DNNF_ONE_TO_ONE;
   }
@@ -195,10 +197,24 @@ int infer_shapes(Graph& g, Op& op, std::string& err) {
     op.at.axis = ax;
     outs.push_back(in(0).dims);
   } else if (k == DNNF_OP_LAYERNORM) {
-    if (!need(3)) return DNNF_ERR_INVALID_ARG;
+    if (op.in.size() != 1 && !need(3)) return DNNF_ERR_INVALID_ARG;
     int rank = (int)in(0).dims.size();
     if (norm_axis(op.at.axis, rank) != rank - 1) { err = "LayerNorm: last axis only"; return DNNF_ERR_UNSUPPORTED_OP; }
-    if (in(1).numel() != in(0).dims.back() || in(2).numel() != in(0).dims.back()) { err = "LayerNorm: parameter length"; return DNNF_ERR_SHAPE; }
+    if (op.in.size() == 3 && (in(1).numel() != in(0).dims.back() || in(2).numel() != in(0).dims.back())) { err = "LayerNorm: parameter length"; return DNNF_ERR_SHAPE; }
+    outs.push_back(in(0).dims);
+  } else if (k == DNNF_OP_WHERE) {
+    if (!need(3)) return DNNF_ERR_INVALID_ARG;
+    std::vector<int64_t> ab, o;
+    if (!broadcast_dims(in(1).dims, in(2).dims, ab) || !broadcast_dims(in(0).dims, ab, o)) { err = "broadcast mismatch"; return DNNF_ERR_SHAPE; }
+    outs.push_back(o);
+  } else if (k == DNNF_OP_CAST) {
+    if (!need(1)) return DNNF_ERR_INVALID_ARG;
+    if (op.at.to < DNNF_CAST_F32 || op.at.to > DNNF_CAST_BOOL) { err = "Cast: unknown target type"; return DNNF_ERR_INVALID_ARG; }
+    outs.push_back(in(0).dims);
+  } else if (k == DNNF_OP_CUMSUM) {
+    if (!need(1)) return DNNF_ERR_INVALID_ARG;
+    int rank = (int)in(0).dims.size();
+    if (norm_axis(op.at.axis, rank) != rank - 1) { err = "CumSum: last axis only"; return DNNF_ERR_UNSUPPORTED_OP; }
     outs.push_back(in(0).dims);
   } else if (is_elementwise(k)) {
     if (!need(1)) return DNNF_ERR_INVALID_ARG;
@@ -324,7 +340,10 @@ int infer_shapes(Graph& g, Op& op, std::string& err) {
   for (auto& d : outs) {
     if (d.size() > (size_t)kMaxDims) { err = "rank above 6"; return DNNF_ERR_SHAPE; }
     for (auto v : d) if (v <= 0) { err = "empty dimension"; return DNNF_ERR_SHAPE; }
-    int t = g.add_tensor("", in(0).dtype, d);
+    int dt = in(0).dtype;
+    if (k == DNNF_OP_WHERE) dt = in(1).dtype;
+    if (k == DNNF_OP_CAST) dt = op.at.to == DNNF_CAST_BF16 ? DNNF_BF16 : DNNF_F32;
+    int t = g.add_tensor("", dt, d);
     g.tensors[t].producer = op.id;
     op.out.push_back(t);
   }

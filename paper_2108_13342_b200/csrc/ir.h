@@ -31,6 +31,7 @@ inline const char* dev_env(const char* name) {
 struct Attrs {
   double c = 0, lo = 0, hi = 0, p = 0, eps = 1e-5;
   int64_t approx = 0, axis = -1, keepdims = 1, start = 0, end = 0, bits = 0, block = 0, scale = 0, kernel = 0, stride = 1, pad = 0;
+  int64_t to = 0, exclusive = 0, reverse = 0;
   std::vector<int64_t> perm, shape, sizes, axes;
 };
 
@@ -134,6 +135,7 @@ bool is_elementwise(int kind);
 bool is_row_anchor(int kind);
 bool is_contraction(int kind);
 bool is_binary_elementwise(int kind);   // two operands with multidirectional broadcasting
+bool is_broadcasting_elementwise(int kind);   // the binary ones and the ternary Where
 const char* op_name(int kind);
 // Bytes a block stores when tensor t is one of its outputs: the whole tensor, except for a Concat's part, which
 // fills only its own range of the shared result.

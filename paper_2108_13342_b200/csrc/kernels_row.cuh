@@ -83,7 +83,63 @@ struct RowIO {
       }
     }
   }
+  // Running sum along the row (CumSum).  The row's elements sit in scan order first inside a thread's vector, then
+  // across the lanes (and warps) of one chunk of 32 * WPR vectors, then across the NV chunks: a serial scan of the
+  // vector, a shuffle scan of the vector totals, one shared-memory exchange of the warp totals, and a carry from
+  // chunk to chunk.  Exclusive: each element gets the sum of those before it; reverse: scan order runs from the far end.
+  __device__ __forceinline__ void row_scan(int op, float (&acc)[VV]) const {
+    const bool excl = op == M_ROWSCAN_X || op == M_ROWSCAN_RX, rev = op == M_ROWSCAN_R || op == M_ROWSCAN_RX;
+    const int lane = threadIdx.x & 31;
+    pdl_launch_dependents();
+#pragma unroll
+    for (int r = 0; r < RPW; ++r) {
+      float carry = 0.0f;
+#pragma unroll
+      for (int jj = 0; jj < NV; ++jj) {
+        const int j = rev ? NV - 1 - jj : jj;
+        float* a = &acc[(r * NV + j) * V];
+        const bool inside = col(j) < p.L;
+        float run = 0.0f;
+#pragma unroll
+        for (int vv = 0; vv < V; ++vv) {
+          const int v = rev ? V - 1 - vv : vv;
+          const float x = inside ? a[v] : 0.0f;
+          a[v] = excl ? run : run + x;
+          run += x;
+        }
+        float incl = run;                              // inclusive scan of the vector totals over the warp's lanes
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const float y = rev ? __shfl_down_sync(0xffffffffu, incl, o) : __shfl_up_sync(0xffffffffu, incl, o);
+          if (rev ? lane + o < 32 : lane >= o) incl += y;
+        }
+        float before = rev ? __shfl_down_sync(0xffffffffu, incl, 1) : __shfl_up_sync(0xffffffffu, incl, 1);
+        if (lane == (rev ? 31 : 0)) before = 0.0f;
+        float chunk_total = __shfl_sync(0xffffffffu, incl, rev ? 0 : 31);
+        if (WPR > 1) {
+          float* x = xchg + xslot * WPR;
+          xslot ^= 1;
+          const int warp = threadIdx.x >> 5;
+          if (lane == 0) x[warp] = chunk_total;
+          __syncthreads();
+          float wb = 0.0f, tot = 0.0f;
+#pragma unroll
+          for (int w = 0; w < WPR; ++w) {
+            const float y = x[w];
+            tot += y;
+            if (rev ? w > warp : w < warp) wb += y;
+          }
+          before += wb;
+          chunk_total = tot;
+        }
+#pragma unroll
+        for (int v = 0; v < V; ++v) a[v] += before + carry;
+        carry += chunk_total;
+      }
+    }
+  }
   __device__ __forceinline__ void row_reduce(int op, float (&acc)[VV]) const {
+    if (op >= M_ROWSCAN) { row_scan(op, acc); return; }
     // The row's loads have been issued by now: let the next kernel's CTAs start arriving.  (Triggering at
     // kernel entry parks them on the SMs for this kernel's whole load latency, where they take the
     // slots of independent kernels that could run.)  Only the first trigger of a CTA counts.

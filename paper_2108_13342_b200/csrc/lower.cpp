@@ -111,7 +111,7 @@ bool backward_views(LowerCtx& cx, const Op& op, const View& vout, std::vector<Vi
     vin[0] = vout;                      // same flat order
     return true;
   }
-  if (is_binary_elementwise(k) || k == DNNF_OP_EXPAND) {
+  if (is_broadcasting_elementwise(k) || k == DNNF_OP_EXPAND) {
     bool need_align = false;
     for (size_t i = 0; i < op.in.size(); ++i) if (in(i).dims != out.dims) need_align = true;
     Aligned al;
@@ -125,7 +125,7 @@ bool backward_views(LowerCtx& cx, const Op& op, const View& vout, std::vector<Vi
     Aligned al;
     if (!align_view(cx, vout, out.dims, al)) return false;
     int ax = k == DNNF_OP_SCALESHIFT ? (int)op.at.axis : (int)out.dims.size() - 1;
-    for (int s = 1; s < 3; ++s) {
+    for (int s = 1; s < (int)op.in.size(); ++s) {
       View v; v.coef.assign(cx.ext.size(), 0);
       for (size_t d = 0; d < cx.ext.size(); ++d) if (al.tdim[d] == ax) v.coef[d] = al.mult[d];
       v.c0 = al.cst[ax];
@@ -167,7 +167,7 @@ bool backward_views(LowerCtx& cx, const Op& op, const View& vout, std::vector<Vi
     vin[0] = v;                         // the result so far (second operand) is extended in place, never read
     return true;
   }
-  if (k == DNNF_OP_SOFTMAX) { vin[0] = vout; return true; }
+  if (k == DNNF_OP_SOFTMAX || k == DNNF_OP_CUMSUM) { vin[0] = vout; return true; }
   if (k >= DNNF_OP_REDUCESUM && k <= DNNF_OP_REDUCEPROD) {
     cx.why = "cannot derive a reduction's input from its output";
     return false;
@@ -218,7 +218,7 @@ static int forward_view_i(LowerCtx& cx, const Op& op, int slot, const View& vi, 
     return 1;
   }
   if (k == DNNF_OP_SLICE || k == DNNF_OP_EXPAND) { cx.why = "partial iteration space"; return -1; }
-  if (k == DNNF_OP_SOFTMAX) { vo = vi; return 1; }
+  if (k == DNNF_OP_SOFTMAX || k == DNNF_OP_CUMSUM) { vo = vi; return 1; }
   if (k == DNNF_OP_LAYERNORM || k == DNNF_OP_SCALESHIFT) { if (slot != 0) return 0; vo = vi; return 1; }
   if (is_elementwise(k)) {
     if (in.dims == out.dims) { vo = vi; return 1; }
@@ -324,9 +324,9 @@ struct Emitter {
 
   Emitter(LowerCtx& c, int mt) : cx(c), max_tmp(mt) {}
 
-  bool push(uint8_t op, uint8_t src = S_NONE, uint8_t idx = 0) {
+  bool push(uint8_t op, uint8_t src = S_NONE, uint8_t idx = 0, uint8_t pad = 0) {
     if (cx.prog.n >= kMaxOps) { cx.why = "fused chain is longer than the micro-op budget"; fail = true; return false; }
-    cx.prog.ops[cx.prog.n++] = MicroOp{op, src, idx, 0};
+    cx.prog.ops[cx.prog.n++] = MicroOp{op, src, idx, pad};
     return true;
   }
   int cst(float v) {
@@ -407,6 +407,54 @@ struct Emitter {
     protect_operand_in_acc(a, 1);
     push(op, src, idx);
     consume(a);
+  }
+  // Where: the condition is parked in a saved value, a goes to acc, b is the operand of the selection
+  void select(const Val& c, const Val& a, const Val& b) {
+    bool parked_here = false;
+    if (!tmp_of.count(c)) {
+      load_acc(c);
+      if (fail) return;
+      int t = alloc_tmp();
+      if (fail) return;
+      tmp_of[c] = t;
+      push(M_SAVE, S_TMP, (uint8_t)t);
+      parked_here = true;
+    }
+    const int tc = tmp_of[c];
+    if (in_acc(b) && !(a == b)) {                    // b is at hand: select the other way round
+      protect_operand_in_acc(b, 1);
+      if (fail) return;
+      uint8_t s, i;
+      if (!src_of(a, s, i)) return;
+      push(M_RSELECT, s, i, (uint8_t)tc);
+      consume(a); consume(b);
+      if (c.kind == 0) { if (--uses[c] <= 0) release(c); }
+      else if (parked_here) { tmp_busy[tc] = false; tmp_of.erase(c); }
+      return;
+    }
+    if (!in_acc(a)) {
+      // the value now in acc (the condition, or an operand that lives only there) is kept if still needed
+      if (acc_valid && !(acc == c)) spill_acc_if_live();
+      if (fail) return;
+      uint8_t s, i;
+      if (!src_of(a, s, i)) return;
+      push(M_MOV, s, i);
+      acc = a; acc_valid = true;
+    }
+    if (!(a == b)) {
+      protect_operand_in_acc(a, 1);
+      if (fail) return;
+      uint8_t s, i;
+      if (!src_of(b, s, i)) return;
+      push(M_SELECT, s, i, (uint8_t)tc);
+    }
+    consume(a); consume(b);
+    // the condition leaves its slot unless an in-block value that is still needed sits there
+    if (c.kind == 0) {
+      if (--uses[c] <= 0) release(c);
+    } else if (parked_here) {
+      tmp_busy[tc] = false; tmp_of.erase(c);
+    }
   }
   void binary(const Val& a, const Val& b, uint8_t op, uint8_t rop, bool commutative) {
     if (a == b) {
@@ -579,6 +627,14 @@ bool emit_program(LowerCtx& cx, int anchor_out, int max_tmp) {
         E.consume(v[0]);
         break;
       }
+      case DNNF_OP_WHERE: E.select(v[0], v[1], v[2]); break;
+      case DNNF_OP_CAST:
+        if (op.at.to == DNNF_CAST_BF16) E.unary(v[0], M_BF16R);
+        else if (op.at.to == DNNF_CAST_I32) E.unary(v[0], M_TRUNC);
+        else if (op.at.to == DNNF_CAST_BOOL) { E.unary(v[0], M_NOT); E.push(M_NOT); }
+        else { E.load_acc(v[0]); E.protect_operand_in_acc(v[0], 1); E.consume(v[0]); }
+        break;
+      case DNNF_OP_CUMSUM: E.unary(v[0], (uint8_t)(M_ROWSCAN + (op.at.exclusive ? 1 : 0) + (op.at.reverse ? 2 : 0))); break;
       case DNNF_OP_SOFTMAX: {
         E.load_acc(v[0]); E.protect_operand_in_acc(v[0], 1);
         int t = E.alloc_tmp(); if (E.fail) break;
@@ -596,9 +652,11 @@ bool emit_program(LowerCtx& cx, int anchor_out, int max_tmp) {
         E.push(M_SAVE, S_TMP, (uint8_t)t); E.push(M_SQUARE); E.push(M_ROWMEAN);
         E.push(M_ADD, S_CONST, (uint8_t)E.cst((float)op.at.eps)); E.push(M_SQRT); E.push(M_RECIP); E.push(M_MUL, S_TMP, (uint8_t)t);
         E.tmp_busy[t] = false;
-        uint8_t s, i;
-        if (!E.src_of(v[1], s, i)) break; E.push(M_MUL, s, i);
-        if (!E.src_of(v[2], s, i)) break; E.push(M_ADD, s, i);
+        if (v.size() >= 3) {
+          uint8_t s, i;
+          if (!E.src_of(v[1], s, i)) break; E.push(M_MUL, s, i);
+          if (!E.src_of(v[2], s, i)) break; E.push(M_ADD, s, i);
+        }
         E.consume(v[0]);
         break;
       }

@@ -35,7 +35,12 @@ enum MOp : uint8_t {
   M_LEAKY,      // acc = acc > 0 ? acc : const[idx] * acc
   M_GT, M_LT,   // acc = acc > src ? 1 : 0 ; acc = acc < src ? 1 : 0
   M_PRELU, M_RPRELU,   // acc = acc > 0 ? acc : src * acc ; acc = src > 0 ? src : acc * src
+  M_SELECT,     // acc = tmp[pad] != 0 ? acc : src   (Where: the condition waits in a saved value)
+  M_RSELECT,    // acc = tmp[pad] != 0 ? src : acc
+  M_BF16R,      // acc = nearest bfloat16 (ties to even) of acc
+  M_TRUNC,      // acc = the integer toward zero
   M_ROWSUM, M_ROWMEAN, M_ROWMAX, M_ROWPROD,   // row kernels only: acc = reduce over the row, broadcast
+  M_ROWSCAN, M_ROWSCAN_X, M_ROWSCAN_R, M_ROWSCAN_RX,   // row kernels only: running sum along the row; X exclusive, R from the far end
   M__COUNT
 };
 

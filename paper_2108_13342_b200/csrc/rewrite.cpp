@@ -112,6 +112,8 @@ struct Rewriter {
       snprintf(buf, sizeof buf, "|%lld|%lld|%lld|%lld|%lld", (long long)o.at.block, (long long)o.at.scale, (long long)o.at.kernel,
                (long long)o.at.stride, (long long)o.at.pad);
       key += buf;
+      snprintf(buf, sizeof buf, "|%lld|%lld|%lld", (long long)o.at.to, (long long)o.at.exclusive, (long long)o.at.reverse);
+      key += buf;
       for (auto v : o.at.perm) key += "p" + std::to_string(v);
       for (auto v : o.at.shape) key += "s" + std::to_string(v);
       for (auto v : o.at.axes) key += "a" + std::to_string(v);

@@ -325,3 +325,94 @@ def test_layout_selection_keeps_values_on_small_graphs():
     ins = {"X": rnd((2, 9, 9, 16), 5), "W": rnd((16, 16), 6, -0.3, 0.3), "s": rnd((16,), 7, 0.5, 1.5), "t": rnd((16,), 8)}
     s = check(W.Workload(g, ins), 5e-4, B.PLAN_FUSED, B.REWRITE_DEFAULT)
     assert s.rewrite_stats.layout_transposes_removed == 3
+
+
+# ---- Where, Cast, CumSum, InstanceNormalization (Table 2) ------------------------------------------------------------
+
+def test_where_is_a_selection_with_broadcasting():
+    cond = (rnd((5, 1, 33), 1, 0.0, 1.0) > 0.5).astype(np.float32)
+    a = rnd((1, 7, 33), 2); b = rnd((5, 7, 1), 3)
+    b[0, 0, 0] = -np.inf; a[0, 1, 4] = np.inf                      # infinities pass through or stay out untouched
+    g = graph(); g.ext("C", cond.shape); g.ext("A", a.shape); g.ext("Bv", b.shape)
+    g.mark_output(g.add("Where", ["C", "A", "Bv"]))
+    s, got, ref = run_both(W.Workload(g, {"C": cond, "A": a, "Bv": b}))
+    assert s.plan_stats.n_kernels == 1
+    np.testing.assert_array_equal(got[g.outputs[0]], ref[g.outputs[0]].astype(np.float32))          # bit-exact
+    # inside a chain: Where(Greater(x, y), x * 2, Neg(y)) with every operand computed in the block
+    g = graph(); g.ext("X", (64, 257)); g.ext("Y", (64, 257))
+    c = g.add("Greater", ["X", "Y"])
+    g.mark_output(g.add("Tanh", [g.add("Where", [c, g.add("MulC", ["X"], c=2.0), g.add("Neg", ["Y"])])]))
+    s = check(W.Workload(g, {"X": rnd((64, 257), 4), "Y": rnd((64, 257), 5)}), RTOL_F32)
+    assert s.plan_stats.n_kernels == 1
+
+
+def test_where_masks_attention_scores_in_front_of_softmax():
+    # the usual masking: scores where the mask is set, -1e9 elsewhere, then Softmax over the row
+    S = 96
+    mask = (np.tril(np.ones((S, S))) != 0).astype(np.float32)
+    g = graph(); g.ext("Sc", (4, 3, S, S)); g.ext("M", (S, S), kind="weight"); g.ext("neg", (1,), kind="weight")
+    w = g.add("Where", ["M", g.add("MulC", ["Sc"], c=0.125), "neg"])
+    g.mark_output(g.add("Softmax", [w], axis=-1))
+    s = check(W.Workload(g, {"Sc": rnd((4, 3, S, S), 6, -8, 8), "M": mask, "neg": np.full((1,), -1e9, np.float32)}), RTOL_F32)
+    assert s.plan_stats.n_kernels == 1 and s.g.blocks()[0]["family"] == "row"
+    y = s.output(g.outputs[0])
+    assert np.all(y[..., np.triu_indices(S, 1)[0], np.triu_indices(S, 1)[1]] == 0.0)
+
+
+@pytest.mark.parametrize("to", ["bf16", "i32", "bool", "f32"])
+def test_cast_on_inputs_is_bit_exact(to):
+    x = rnd((37, 130), 7, -300.0, 300.0)
+    x[0, :6] = [0.0, -0.0, 0.5, -0.5, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8]          # zeros, halves and bfloat16 ties
+    g = graph(); g.ext("X", x.shape)
+    g.mark_output(g.add("Cast", ["X"], to=to))
+    s, got, ref = run_both(W.Workload(g, {"X": x}))
+    np.testing.assert_array_equal(got[g.outputs[0]].astype(np.float64), ref[g.outputs[0]])
+    dt, _ = s.g.tensor_info(s.ids[g.outputs[0]])
+    assert dt == (B.BF16 if to == "bf16" else B.F32)
+
+
+def test_cast_inside_a_chain_rounds_the_value_its_consumers_see():
+    # Sigmoid -> Cast(bf16) -> MulC -> Cast(i32): the second operator works on the rounded value
+    x = rnd((64, 512), 8, -4.0, 4.0)
+    g = graph(); g.ext("X", x.shape)
+    k = g.add("Cast", [g.add("Sigmoid", ["X"])], to="bf16")
+    g.mark_output(g.add("Cast", [g.add("MulC", [k], c=1024.0)], to="f32"))
+    s, got, ref = run_both(W.Workload(g, {"X": x}))
+    assert s.plan_stats.n_kernels == 1
+    y, r = got[g.outputs[0]].astype(np.float64), ref[g.outputs[0]]
+    # values are multiples of 1024 * 2^-9 at most apart by one bfloat16 step where fp32 and fp64 Sigmoid straddle a tie
+    assert np.mean(y == r) > 0.99 and np.all(np.abs(y - r) <= 2.0 ** -7 * np.abs(r) + 1e-12)
+
+
+@pytest.mark.parametrize("shape", [(5, 8), (33, 100), (16, 128), (7, 3, 1024), (6, 4096), (3, 8192), (64, 24), (9, 2052)])
+@pytest.mark.parametrize("exclusive,reverse", [(0, 0), (1, 0), (0, 1), (1, 1)])
+def test_cumsum_rows(shape, exclusive, reverse):
+    g = graph(); g.ext("X", shape)
+    g.mark_output(g.add("CumSum", ["X"], axis=-1, exclusive=exclusive, reverse=reverse))
+    s = check(W.Workload(g, {"X": rnd(shape, 9)}), RTOL_F32)
+    assert s.plan_stats.n_kernels == 1 and s.g.blocks()[0]["family"] == "row"
+
+
+def test_cumsum_counts_exactly_and_fuses_with_its_neighbours():
+    # running count of ones: integers, exact in fp32
+    x = (rnd((11, 4096), 10, 0.0, 1.0) > 0.7).astype(np.float32)
+    g = graph(); g.ext("X", x.shape)
+    g.mark_output(g.add("CumSum", ["X"], axis=-1))
+    s, got, ref = run_both(W.Workload(g, {"X": x}))
+    np.testing.assert_array_equal(got[g.outputs[0]].astype(np.float64), ref[g.outputs[0]])
+    # Exp in front, a normalisation by the row total behind: a cumulative distribution in one kernel
+    g = graph(); g.ext("X", (40, 768))
+    e = g.add("Exp", ["X"])
+    g.mark_output(g.add("Div", [g.add("CumSum", [e], axis=-1), g.add("ReduceSum", [e], axis=-1, keepdims=1)]))
+    s = check(W.Workload(g, {"X": rnd((40, 768), 11)}), RTOL_F32)
+    assert s.plan_stats.n_kernels <= 2
+
+
+@pytest.mark.parametrize("shape", [(2, 12, 12, 16), (3, 7, 9, 40), (4, 56, 56, 24)])
+def test_instance_normalization(shape):
+    c = shape[3]
+    g = graph(); g.ext("X", shape); g.ext("s", (c,), kind="weight"); g.ext("t", (c,), kind="weight")
+    g.mark_output(g.add("Relu", [g.add("InstanceNorm", ["X", "s", "t"], eps=1e-5)]))
+    ins = {"X": rnd(shape, 12, -1.0, 3.0), "s": rnd((c,), 13, 0.5, 1.5), "t": rnd((c,), 14, -0.5, 0.5)}
+    s = check(W.Workload(g, ins), RTOL_F32)
+    assert s.plan_stats.n_ops == 2

@@ -646,3 +646,38 @@ def test_layout_selection_small_cases():
     g.mark_output(g.add("Conv1x1", [y, "W"]))
     G, st, kinds = _rewritten_kinds(g)
     assert st.layout_transposes_removed == 3 and "Transpose" not in kinds
+
+
+# ---- Where, Cast, CumSum, InstanceNormalization (Table 2) ------------------------------------------------------------
+
+def test_where_cast_cumsum_instancenorm_recording_types_and_plans():
+    # Table 2: Where and Cast are One-to-One (Where with a broadcast operand takes the operand's One-to-Many), CumSum and
+    # InstanceNormalization Many-to-Many
+    g = _desc(); g.ext("C", (4, 1, 8)); g.ext("A", (4, 6, 8)); g.ext("Bv", (8,))
+    w = g.add("Where", ["C", "A", "Bv"])
+    k = g.add("Cast", [w], to="bf16")
+    g.mark_output(g.add("CumSum", [g.add("Cast", [k], to="f32")], axis=-1, exclusive=1))
+    G, ids, st = _plan_desc(g)
+    assert [G.op_mapping(i) for i in range(4)] == [OM, OO, OO, MM]
+    assert G.tensor_info(ids[w]) == (B.F32, (4, 6, 8)) and G.tensor_info(ids[k])[0] == B.BF16
+    assert st.n_kernels == 1 and G.blocks()[0]["family"] == "row"
+    prog = G.block_program(0)
+    assert "SELECT" in prog and "BF16R" in prog and "ROWSCAN_X" in prog, prog
+    g = _desc(); g.ext("C", (4, 8)); g.ext("A", (4, 8)); g.ext("Bv", (4, 8))
+    g.mark_output(g.add("Where", ["C", "A", "Bv"]))
+    G, ids, st = _plan_desc(g)
+    assert G.op_mapping(0) == OO and G.block_program(0) == "MOV in0; SAVE t0; MOV in1; SELECT in2; STORE out0"
+    # InstanceNormalization is recorded as its channels-first row normalisation between index operators
+    g = _desc(); g.ext("X", (2, 6, 6, 8)); g.ext("s", (8,), kind="weight"); g.ext("t", (8,), kind="weight")
+    g.mark_output(g.add("Relu", [g.add("InstanceNorm", ["X", "s", "t"], eps=1e-5)]))
+    G, ids, st = _plan_desc(g)
+    kinds = [k for b in G.blocks() for k in b["ops"]]
+    assert sorted(kinds) == sorted(["Transpose", "Reshape", "LayerNorm", "Reshape", "Transpose", "ScaleShift", "Relu"])
+    assert st.n_ops == 2 and any(b["family"] == "row" for b in G.blocks())
+    # errors
+    for op, ins, at in [("Where", ["X", "s"], {}), ("Cast", ["X"], dict(to=7)), ("CumSum", ["X"], dict(axis=1)),
+                        ("InstanceNorm", ["X", "s"], {}), ("InstanceNorm", ["s", "s", "t"], {})]:
+        g2 = _desc(); g2.ext("X", (2, 6, 6, 8)); g2.ext("s", (8,), kind="weight"); g2.ext("t", (8,), kind="weight")
+        g2.add(op, ins, **at)
+        with pytest.raises(B.DnnfError):
+            _plan_desc(g2)
