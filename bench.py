@@ -228,14 +228,16 @@ def main():
         e1.record(stream)
         torch.cuda.synchronize(dev)
         ms_step = e0.elapsed_time(e1) / steps
-        # second pass over the same steps with an event between the blocks: each kernel's own duration
-        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(nb + 1)] for _ in range(steps)]
-        for i in range(steps):
-            g = S[i % SETS].g
-            ev[i][0].record(stream)
-            for b in range(nb):
-                g.run_block(b, sptr)
-                ev[i][b + 1].record(stream)
+        # second pass, one kernel at a time: the same `steps` launches of block b over the rotating buffer sets, back
+        # to back on the same stream and with the same launch attributes as inside dnnf_run, between two events.
+        # (An event between the blocks of a step would add the gap it creates to every kernel: those figures summed
+        # to a quarter more than the step itself; these sum to the step.)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(nb)]
+        for b in range(nb):
+            ev[b][0].record(stream)
+            for i in range(steps):
+                S[i % SETS].g.run_block(b, sptr)
+            ev[b][1].record(stream)
         torch.cuda.synchronize(dev)
         # keep the GPU busy a little longer so that the sampler sees clocks under load
         t_end = time.time() + 1.0
@@ -256,7 +258,7 @@ def main():
     value = aggregate_throughput(bytes_step, ms_step, world)
 
     blocks = S[0].g.blocks()
-    k_us = [sum(e[b].elapsed_time(e[b + 1]) for e in ev) / steps * 1e3 for b in range(nb)]
+    k_us = [ev[b][0].elapsed_time(ev[b][1]) / steps * 1e3 for b in range(nb)]
     kernels = [{"ops": "+".join(blocks[b]["ops"]), "us": round(k_us[b], 2),
                 "frac": round(bbytes[b] / (k_us[b] * 1e-6) / 1e9 / pk["hbm_gbs"], 3)} for b in range(nb)]
     top = max(range(nb), key=lambda b: k_us[b])

@@ -14,7 +14,8 @@ FUSED, UNFUSED = B.PLAN_FUSED, B.PLAN_UNFUSED
 
 def _expect_variant(sess, variant):
     """The block must run on the named kernel variant."""
-    assert sess.g.blocks()[0]["variant"] == variant, sess.g.blocks()
+    ok = variant if isinstance(variant, tuple) else (variant,)
+    assert sess.g.blocks()[0]["variant"] in ok, sess.g.blocks()
 
 def _bf(x):
     return W.round_to_bf16(x)
@@ -464,3 +465,4 @@ def test_rebinding_any_epilogue_operand_reencodes_the_tensor_maps():
     s.run()
     close(s.output("Y"), O.run_graph(wl.graph, ins)["Y"], RTOL_BF16)
     assert s.g.status() == (0, -1)
+
