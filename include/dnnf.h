@@ -171,8 +171,9 @@ typedef struct {
 #define DNNF_PLAN_ALLOW_PROLOGUE    4u   /* planning only: let One-to-One predecessors fuse in front of a
                                             GEMM/conv anchor (Listing 1 literal); such plans cannot be run */
 #define DNNF_PLAN_BEYOND_TABLE3      8u   /* an extension beyond the paper's rules: MatMul -> [scale] -> [+ mask] -> Softmax ->
-                                            MatMul runs as ONE kernel (Table 3 marks Many-to-Many followed by
-                                            Many-to-Many red, so the default plan keeps three blocks) */
+                                            MatMul runs as ONE kernel, and so does Conv1x1 -> DwConv3x3 -> Conv1x1 with
+                                            their chains (Table 3 marks Many-to-Many followed by Many-to-Many red, so the
+                                            default plan keeps three blocks each) */
 /* Kernel-selection overrides.  The plan, its blocks and the results stay the same; a block is only lowered to another
  * kernel of its family.  They exist so that every kernel, including the ones the planner rarely picks, can be
  * tested and timed through this interface; the library reads no environment variable. */
@@ -185,6 +186,9 @@ typedef struct {
 #define DNNF_PLAN_NO_SPLIT_K        0x2000u  /* bf16 GEMM blocks without a split over K */
 #define DNNF_PLAN_NO_TMA_DWCONV     0x4000u  /* depthwise convolutions without the TMA-tiled kernel */
 #define DNNF_PLAN_NO_TILE_GEMM      0x8000u  /* bf16 GEMM blocks without the one-tile-per-CTA kernel */
+#define DNNF_PLAN_MBCONV_ALWAYS     0x20000u /* with DNNF_PLAN_BEYOND_TABLE3: form the single-kernel inverted-residual block whatever its
+                                                size (by default only while its 8 x 16 pixel tiles fit one wave of CTAs, where it was
+                                                measured faster than the three kernels; this flag changes the plan, not only a kernel) */
 #define DNNF_PLAN_CLUSTER_SPLIT_K   0x10000u /* one-tile-per-CTA kernel: clusters of 2 or 4 CTAs share a tile's k-tiles and add their
                                                 partial sums through distributed shared memory (measured slower at the sizes
                                                 tried, so not the default) */
@@ -222,7 +226,9 @@ typedef enum {
   DNNF_FAMILY_DWCONV = 6,      /* fp32 depthwise 3x3 with an epilogue chain */
   DNNF_FAMILY_POOL = 7,        /* fp32 MaxPool / AveragePool with an epilogue chain */
   DNNF_FAMILY_GATHER = 8,      /* row gather by an index tensor */
-  DNNF_FAMILY_ATTENTION = 9    /* scores, softmax and weighted sum of a head in one kernel (DNNF_PLAN_BEYOND_TABLE3 only) */
+  DNNF_FAMILY_ATTENTION = 9,   /* scores, softmax and weighted sum of a head in one kernel (DNNF_PLAN_BEYOND_TABLE3 only) */
+  DNNF_FAMILY_MBCONV = 10      /* pointwise expansion, depthwise 3x3 and pointwise projection of an inverted-residual block in one
+                                  kernel, the expanded tensor kept in shared memory (DNNF_PLAN_BEYOND_TABLE3 only) */
 } dnnf_family_t;
 
 typedef struct {

@@ -26,7 +26,7 @@ INPUT, WEIGHT = 0, 1
 ONE_TO_ONE, REORGANIZE, SHUFFLE, ONE_TO_MANY, MANY_TO_MANY = range(5)
 GREEN, YELLOW, RED = range(3)
 MAPPING_NAMES = ["One-to-One", "Reorganize", "Shuffle", "One-to-Many", "Many-to-Many"]
-FAMILY_NAMES = ["alias", "elementwise", "transpose", "row", "gemm", "conv1x1", "dwconv", "pool", "gather", "attention"]
+FAMILY_NAMES = ["alias", "elementwise", "transpose", "row", "gemm", "conv1x1", "dwconv", "pool", "gather", "attention", "mbconv"]
 
 OP_NAMES = ["?", "Add", "Sub", "Mul", "Div", "MulC", "AddC", "Sigmoid", "Tanh", "Erf", "Exp", "Log", "Sqrt", "Abs",
             "Neg", "Recip", "Square", "Relu", "Clip", "Pow", "Gelu", "ScaleShift", "Transpose", "Reshape", "Flatten",
@@ -48,6 +48,7 @@ PLAN_FUSED, PLAN_UNFUSED, PLAN_STRICT_TABLE3, PLAN_ALLOW_PROLOGUE, PLAN_BEYOND_T
 # kernel-selection overrides (same blocks and results, another kernel of the family)
 PLAN_SPLIT_ALWAYS, PLAN_NO_K_SLICES, PLAN_NO_COLUMN_BLOCKS, PLAN_NO_TF32_GEMM = 0x100, 0x200, 0x400, 0x800
 PLAN_NO_PAIR_GEMM, PLAN_NO_SPLIT_K, PLAN_NO_TMA_DWCONV, PLAN_NO_TILE_GEMM = 0x1000, 0x2000, 0x4000, 0x8000
+PLAN_MBCONV_ALWAYS = 0x20000
 PLAN_CLUSTER_SPLIT_K = 0x10000
 STATIC_WS_BYTES = 32 << 20
 

@@ -35,6 +35,8 @@ void tile_gemm_plan(Launch& L);
 bool tile_gemm_prepare(Launch& L, std::string& err);
 int tile_gemm_launch(const Launch& L, cudaStream_t st);
 void attention_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op, std::string& err);
+void mbconv_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
+int mbconv_launch(const Launch& L, cudaStream_t st);
 int attention_launch(const Launch& L, void* status_words, int block_index, cudaStream_t st);
 size_t tf32_blob_bytes();
 bool tf32_gemm_eligible(const GemmParams& gp);
@@ -494,6 +496,7 @@ void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vecto
   if (L.family == DNNF_FAMILY_DWCONV) { dwconv_patch(L, ip, op, err); return; }
   if (L.family == DNNF_FAMILY_POOL) { pool_patch(L, ip, op); return; }
   if (L.family == DNNF_FAMILY_GATHER) { gather_patch(L, ip, op); return; }
+  if (L.family == DNNF_FAMILY_MBCONV) { mbconv_patch(L, ip, op); return; }
   if (L.family == DNNF_FAMILY_ATTENTION) { attention_patch(L, ip, op, err); if (!L.tc_ready && err.empty()) err = "cannot encode the tensor maps of an attention block"; return; }
   GemmParams& gp = gp_of(L);
   gp.A.ptr = ip[0]; gp.B.ptr = ip[1];
@@ -512,6 +515,7 @@ void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vecto
 }
 
 int launch_contraction(const Launch& L, void* status_words, int block_index, cudaStream_t st, std::string& err) {
+  if (L.family == DNNF_FAMILY_MBCONV) { int rc = mbconv_launch(L, st); if (rc) err = "inverted-residual block launch failed"; return rc; }
   if (L.family == DNNF_FAMILY_ATTENTION) { int rc = attention_launch(L, status_words, block_index, st); if (rc) err = "attention launch failed"; return rc; }
   if (L.family == DNNF_FAMILY_GATHER) { int rc = gather_launch(L, st); if (rc) err = "gather launch failed"; return rc; }
   if (L.family == DNNF_FAMILY_POOL) { int rc = pool_launch(L, status_words, st); if (rc) err = "pooling launch failed"; return rc; }

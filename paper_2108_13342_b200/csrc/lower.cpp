@@ -914,7 +914,12 @@ int lower_block(const Graph& g, const std::vector<int>& ops_in, uint32_t flags, 
     if (is_row_anchor(k) || is_contraction(k)) { n_anchor++; anchor = o; }
     if (k == DNNF_OP_BITSHIFT) { why = "BitShift has no device code"; return DNNF_ERR_UNSUPPORTED_OP; }
   }
-  if (n_anchor == 3 && (flags & DNNF_PLAN_BEYOND_TABLE3)) { out.mapping = DNNF_MANY_TO_MANY; return lower_attention(g, ops, flags, out, why); }
+  if (n_anchor == 3 && (flags & DNNF_PLAN_BEYOND_TABLE3)) {
+    out.mapping = DNNF_MANY_TO_MANY;
+    bool conv = false;
+    for (int o : ops) if (g.ops[o].kind == DNNF_OP_DWCONV3X3) conv = true;
+    return conv ? lower_mbconv(g, ops, flags, out, why) : lower_attention(g, ops, flags, out, why);
+  }
   if (n_anchor > 1) { why = "more than one Many-to-Many operator in a block"; return DNNF_ERR_UNSUPPORTED_OP; }
   // A ConcatPart ends its block: it stores the block's values into its range of the Concat's result.  The
   // operators that read the whole result, and the one that produced the result so far, run in other blocks.

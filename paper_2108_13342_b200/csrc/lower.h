@@ -56,5 +56,7 @@ int find_or_add_arg(std::vector<ExtArg>& v, int tensor, const View& view);
 int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flags, int anchor, Block& out, std::string& why);
 // MatMul -> [scale] -> [+ mask] -> Softmax -> MatMul as one kernel (beyond Table 3)
 int lower_attention(const Graph& g, const std::vector<int>& ops, uint32_t flags, Block& out, std::string& why);
+// Conv1x1 + chain -> DwConv3x3 + chain -> Conv1x1 + chain as one kernel (beyond Table 3)
+int lower_mbconv(const Graph& g, const std::vector<int>& ops, uint32_t flags, Block& out, std::string& why);
 
 }  // namespace dnnf

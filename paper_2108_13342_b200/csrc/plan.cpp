@@ -607,6 +607,45 @@ static void fuse_attention_blocks(const Graph& g, uint32_t flags, std::vector<st
   live.swap(keep);
 }
 
+// Beyond Table 3, second case: the block of a depthwise 3x3 convolution between the blocks of the pointwise convolution
+// that makes its input and the one that reads its result (an inverted-residual block) becomes one block when the three
+// lower to the single kernel.
+static void fuse_mbconv_blocks(const Graph& g, uint32_t flags, std::vector<std::vector<int>>& live) {
+  std::vector<int> bo(g.ops.size(), -1);
+  for (size_t i = 0; i < live.size(); ++i) for (int o : live[i]) bo[o] = (int)i;
+  auto one_anchor = [&](const std::vector<int>& b, int kind) {
+    int n = 0, found = -1;
+    for (int o : b) { const int k = g.ops[o].kind; if (is_row_anchor(k) || is_contraction(k)) { ++n; if (k == kind) found = o; } }
+    return n == 1 ? found : -1;
+  };
+  for (size_t r = 0; r < live.size(); ++r) {
+    const int dwo = one_anchor(live[r], DNNF_OP_DWCONV3X3);
+    if (dwo < 0) continue;
+    const Tensor& e = g.tensors[g.ops[dwo].in[0]];
+    if (e.producer < 0 || e.is_output || e.consumers.size() != 1) continue;
+    const int a = bo[e.producer];
+    if (a < 0 || a == (int)r || live[a].empty() || one_anchor(live[a], DNNF_OP_CONV1X1) < 0) continue;
+    // forward along the chain behind the depthwise filter to the tensor that leaves this block
+    int t = g.ops[dwo].out[0];
+    while (g.tensors[t].consumers.size() == 1 && bo[g.tensors[t].consumers[0]] == (int)r && !g.tensors[t].is_output) t = g.ops[g.tensors[t].consumers[0]].out[0];
+    const Tensor& d = g.tensors[t];
+    if (d.is_output || d.consumers.size() != 1) continue;
+    const int c = bo[d.consumers[0]];
+    if (c < 0 || c == (int)r || c == a || live[c].empty() || one_anchor(live[c], DNNF_OP_CONV1X1) != d.consumers[0]) continue;
+    std::vector<int> merged = live[a];
+    merged.insert(merged.end(), live[r].begin(), live[r].end());
+    merged.insert(merged.end(), live[c].begin(), live[c].end());
+    Block trial; std::string why;
+    if (lower_block(g, merged, flags, trial, why) != DNNF_OK || trial.launch.family != DNNF_FAMILY_MBCONV) { if (dev_env("DNNF_DEBUG_PLAN")) fprintf(stderr, "inverted-residual block not fused: %s\n", why.c_str()); continue; }
+    for (int o : live[r]) bo[o] = a;
+    for (int o : live[c]) bo[o] = a;
+    live[a] = merged; live[r].clear(); live[c].clear();
+  }
+  std::vector<std::vector<int>> keep;
+  for (auto& b : live) if (!b.empty()) keep.push_back(b);
+  live.swap(keep);
+}
+
 int plan_graph(Graph& g, uint32_t flags) {
   tl_plan_flags = flags;
   g.relink();
@@ -650,7 +689,7 @@ int plan_graph(Graph& g, uint32_t flags) {
   // is not enough after predecessor fusion: sort blocks topologically).
   std::vector<std::vector<int>> live;
   for (auto& b : P.blocks) if (!b.empty()) live.push_back(b);
-  if ((flags & DNNF_PLAN_BEYOND_TABLE3) && !(flags & (DNNF_PLAN_UNFUSED | DNNF_PLAN_ALLOW_PROLOGUE))) fuse_attention_blocks(g, flags, live);
+  if ((flags & DNNF_PLAN_BEYOND_TABLE3) && !(flags & (DNNF_PLAN_UNFUSED | DNNF_PLAN_ALLOW_PROLOGUE))) { fuse_attention_blocks(g, flags, live); fuse_mbconv_blocks(g, flags, live); }
   int nb = (int)live.size();
   std::vector<int> bo(g.ops.size(), -1);
   for (int i = 0; i < nb; ++i) for (int o : live[i]) bo[o] = i;

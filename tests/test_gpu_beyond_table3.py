@@ -8,7 +8,7 @@ import pytest
 
 from paper_2108_13342_b200 import binding as B
 from paper_2108_13342_b200 import workloads as W
-from util import RTOL_BF16, check, close, graph, rnd, run_both
+from util import RTOL_BF16, RTOL_F32, check, close, graph, rnd, run_both
 
 pytestmark = pytest.mark.gpu
 BEYOND = B.PLAN_FUSED | B.PLAN_BEYOND_TABLE3
@@ -122,3 +122,95 @@ def test_encoder_full_size_one_layer_with_single_kernel_attention():
     (name,) = wl.graph.outputs
     close(got[name], ref[name], RTOL_BF16)
     assert s.plan_stats.n_kernels == 7
+
+
+# ---- the inverted-residual block as one kernel ---------------------------------------------------------------------------
+
+def _families(s):
+    return [b["family"] for b in s.g.blocks() if b["family"] != "alias"]
+
+
+@pytest.mark.parametrize("cfg", [(1, 8, 16, 24, 144), (2, 14, 14, 24, 144), (3, 19, 23, 24, 144), (1, 56, 56, 24, 144), (2, 9, 33, 24, 48),
+                                 (1, 17, 18, 24, 96), (2, 7, 5, 24, 144), (1, 2, 3, 24, 48), (5, 3, 70, 24, 96)])
+def test_inverted_residual_block_as_one_kernel(cfg):
+    """Expansion, depthwise filter and projection with their batch-norm / ReLU6 / residual chains in one kernel: same values
+    as the oracle at the tolerance of fp32 blocks, on tiles that are ragged in both directions, image borders inside and
+    outside a tile, one to several tiles per image."""
+    n, h, w, cin, cexp = cfg
+    wl = W.mbconv_block(n, h, w, cin, cexp)
+    s = check(wl, RTOL_F32, BEYOND | B.PLAN_MBCONV_ALWAYS, expect_blocks=1)
+    assert _families(s) == ["mbconv"]
+    # the paper's rules keep three kernels
+    assert len(_families(check(wl, RTOL_F32, B.PLAN_FUSED, expect_blocks=3))) == 3
+
+
+def test_inverted_residual_block_full_size():
+    """32 images are 896 tiles, six waves: the planner keeps the three kernels unless told otherwise (they are faster
+    there); the single kernel is checked on the full size all the same."""
+    s = check(W.mbconv_block(), RTOL_F32, BEYOND | B.PLAN_MBCONV_ALWAYS, expect_blocks=1)
+    assert _families(s) == ["mbconv"] and s.g.blocks()[0]["grid"] == 148
+    s = check(W.mbconv_block(), RTOL_F32, BEYOND, expect_blocks=3)
+    assert "mbconv" not in _families(s)
+    s = check(W.mbconv_block(n=1), RTOL_F32, BEYOND, expect_blocks=1)       # one image: 28 tiles
+    assert _families(s) == ["mbconv"]
+
+
+@pytest.mark.parametrize("cout,tail,act", [(32, "none", "clip"), (24, "relu", "relu"), (32, "two_outputs", "clip"), (24, "pixel_gate", "leaky")])
+def test_inverted_residual_block_other_chains(cout, tail, act):
+    """Chains without a compile-time table (interpreted), a projection without residual, onto 32 channels, with two
+    outputs, with an operand that depends on the pixel only."""
+    n, h, w, ce = 2, 21, 19, 96
+    cin = {"none": 16, "two_outputs": 40}.get(tail, 24)           # 40 input channels: a K with an 8-wide tail
+    g = graph("mb"); ins = {}
+
+    def ext(name, shape, lo, hi, seed, kind="weight"):
+        g.ext(name, shape, kind=kind); ins[name] = rnd(shape, seed, lo, hi); return name
+
+    def activation(x):
+        if act == "clip": return g.add("Clip", [x], lo=0.0, hi=6.0)
+        if act == "relu": return g.add("Relu", [x])
+        return g.add("LeakyRelu", [x], alpha=0.1)
+
+    ext("X", (n, h, w, cin), 0.0, 1.0, 1, kind="input")
+    e = g.add("Conv1x1", ["X", ext("W1", (cin, ce), -0.3, 0.3, 2)])
+    e = activation(g.add("ScaleShift", [e, ext("s1", (ce,), 0.5, 1.5, 3), ext("t1", (ce,), -0.5, 0.5, 4)], axis=-1))
+    e = g.add("DwConv3x3", [e, ext("Kd", (3, 3, ce), -0.5, 0.5, 5)])
+    e = activation(g.add("Add", [e, ext("b2", (ce,), -0.5, 0.5, 6)]))
+    e = g.add("Conv1x1", [e, ext("W3", (ce, cout), -0.2, 0.2, 7)])
+    e = g.add("ScaleShift", [e, ext("s3", (cout,), 0.5, 1.5, 8), ext("t3", (cout,), -0.5, 0.5, 9)], axis=-1)
+    if tail == "relu":
+        e = g.add("Relu", [g.add("Add", [e, "X"])])
+    elif tail == "two_outputs":
+        g.mark_output(e)
+        e = g.add("Sigmoid", [e])
+    elif tail == "pixel_gate":
+        e = g.add("Mul", [g.add("Add", [e, "X"]), ext("P", (n, h, w, 1), 0.5, 1.5, 10, kind="input")])
+    g.mark_output(e)
+    s = check(W.Workload(g, ins), RTOL_F32, BEYOND, expect_blocks=1)
+    assert _families(s) == ["mbconv"]
+
+
+def test_inverted_residual_blocks_that_stay_three_kernels():
+    # the expanded tensor is also a graph output; an operand behind the expansion depends on the pixel
+    wl = W.mbconv_block(2, 12, 12, 24, 48)
+    wl.graph.mark_output(wl.graph.ops[2].outputs[0])                      # the first ReLU6
+    s = check(wl, RTOL_F32, BEYOND)
+    assert "mbconv" not in _families(s)
+    g = graph("mb2"); n, h, w = 1, 10, 10
+    g.ext("X", (n, h, w, 24)); g.ext("W1", (24, 48), kind="weight"); g.ext("Kd", (3, 3, 48), kind="weight"); g.ext("W3", (48, 24), kind="weight")
+    g.ext("R", (n, h, w, 48))
+    e = g.add("Add", [g.add("Conv1x1", ["X", "W1"]), "R"])
+    g.mark_output(g.add("Conv1x1", [g.add("Relu", [g.add("DwConv3x3", [e, "Kd"])]), "W3"]))
+    ins = {"X": rnd((n, h, w, 24), 1), "W1": rnd((24, 48), 2, -0.3, 0.3), "Kd": rnd((3, 3, 48), 3, -0.5, 0.5), "W3": rnd((48, 24), 4, -0.3, 0.3),
+           "R": rnd((n, h, w, 48), 5)}
+    s = check(W.Workload(g, ins), RTOL_F32, BEYOND)
+    assert "mbconv" not in _families(s)
+
+
+def test_mobilenet_stack_with_single_kernel_blocks():
+    """The MobileNetV2-shaped stack: the inverted-residual blocks whose channel counts fit run as one kernel each, the others
+    keep the three kernels of the paper's rules; same logits as the oracle."""
+    wl = W.mbconv_stack(n=4, hw=48)
+    s = check(wl, 5e-4, BEYOND | B.PLAN_MBCONV_ALWAYS, B.REWRITE_DEFAULT)
+    fams = _families(s)
+    assert fams.count("mbconv") >= 2, fams

@@ -681,3 +681,20 @@ def test_where_cast_cumsum_instancenorm_recording_types_and_plans():
         g2.add(op, ins, **at)
         with pytest.raises(B.DnnfError):
             _plan_desc(g2)
+
+
+def test_beyond_table3_forms_the_single_kernel_inverted_residual_block_only_while_it_pays():
+    def fams(wl, flags):
+        G, ids = build_graph(wl.graph)
+        G.rewrite(B.REWRITE_NONE)
+        st = G.plan(flags)
+        return [b["family"] for b in G.blocks()], st
+    beyond = B.PLAN_FUSED | B.PLAN_BEYOND_TABLE3
+    small, full = W.mbconv_block(n=1, h=16, w=16), W.mbconv_block()
+    assert fams(small, B.PLAN_FUSED)[0] == ["conv1x1", "dwconv", "conv1x1"]          # Table 3: Many-to-Many + Many-to-Many is red
+    f, st = fams(small, beyond)
+    assert f == ["mbconv"] and st.n_kernels == 1 and st.n_ops == 9
+    assert fams(full, beyond)[0] == ["conv1x1", "dwconv", "conv1x1"]                 # 896 tiles: more than one wave
+    assert fams(full, beyond | B.PLAN_MBCONV_ALWAYS)[0] == ["mbconv"]
+    # the intermediate tensors of the single kernel never reach memory
+    assert fams(small, beyond)[1].irs_bytes_fused == 0 and fams(small, B.PLAN_FUSED)[1].irs_bytes_fused > 0
