@@ -14,7 +14,8 @@ def main():
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--unfused", action="store_true")
     ap.add_argument("--canon", action="store_true")
-    ap.add_argument("--beyond", action="store_true", help="plan with DNNF_PLAN_BEYOND_TABLE3 (single-kernel attention)")
+    ap.add_argument("--beyond", action="store_true", help="plan with DNNF_PLAN_BEYOND_TABLE3 (single-kernel attention and inverted-residual blocks)")
+    ap.add_argument("--plan-flags", type=lambda v: int(v, 0), default=0, help="further dnnf_plan flags, e.g. 0x20000 (DNNF_PLAN_MBCONV_ALWAYS)")
     ap.add_argument("--instances", type=int, default=1, help="independent copies with their own buffers, run round-robin")
     args = ap.parse_args()
     import torch
@@ -23,7 +24,7 @@ def main():
     from .runtime import Session
     kw = {k: int(v) for k, v in (x.split("=") for x in args.kw)}
     wl = W.by_name(args.workload, **kw)
-    sess = [Session(wl, plan_flags=B.PLAN_UNFUSED if args.unfused else (B.PLAN_FUSED | (B.PLAN_BEYOND_TABLE3 if args.beyond else 0)),
+    sess = [Session(wl, plan_flags=B.PLAN_UNFUSED if args.unfused else (B.PLAN_FUSED | (B.PLAN_BEYOND_TABLE3 if args.beyond else 0) | args.plan_flags),
                     rewrite_flags=B.REWRITE_CANON_MACRO if args.canon else B.REWRITE_NONE) for _ in range(args.instances)]
     s = sess[0]
     for _ in range(args.iters):
