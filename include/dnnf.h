@@ -130,6 +130,12 @@ typedef enum {
                                                        channel is normalised by the mean and biased variance over its H x W positions.
                                                        Recorded as Transpose -> Reshape [N,C,HW] -> LayerNorm (no scale / shift) ->
                                                        Reshape -> Transpose -> ScaleShift, which it equals term by term */
+  DNNF_OP_EINSUM,                                   /* Many-to-Many (Table 2); two operands, attributes LABELS_A, LABELS_B, LABELS_OUT: one small
+                                                       integer per axis (the letters of "bhqd,bhkd->bhqk").  Every label of the result comes
+                                                       from an operand, a label of both operands that is missing in the result is summed
+                                                       over (at least one), no label repeats inside an operand and none belongs to one
+                                                       operand only without reaching the result.  Recorded as Transpose / Reshape of the
+                                                       operands -> (batched) MatMul -> Reshape / Transpose, which it equals term by term */
   DNNF_OP_CONCATPART,                               /* internal (made by Concat): (x [, result so far]); AXIS, START, SHAPE */
   DNNF_OP__COUNT
 } dnnf_op_t;
@@ -139,7 +145,8 @@ typedef enum {
   DNNF_ATTR_APPROX, DNNF_ATTR_AXIS, DNNF_ATTR_KEEPDIMS, DNNF_ATTR_START, DNNF_ATTR_END, DNNF_ATTR_BITS, /* use i[0] */
   DNNF_ATTR_PERM, DNNF_ATTR_SHAPE, DNNF_ATTR_SIZES, DNNF_ATTR_AXES,           /* use i[0..n) */
   DNNF_ATTR_BLOCK, DNNF_ATTR_SCALE, DNNF_ATTR_KERNEL, DNNF_ATTR_STRIDE, DNNF_ATTR_PAD,  /* use i[0] */
-  DNNF_ATTR_TO, DNNF_ATTR_EXCLUSIVE, DNNF_ATTR_REVERSE                                    /* use i[0] */
+  DNNF_ATTR_TO, DNNF_ATTR_EXCLUSIVE, DNNF_ATTR_REVERSE,                                   /* use i[0] */
+  DNNF_ATTR_LABELS_A, DNNF_ATTR_LABELS_B, DNNF_ATTR_LABELS_OUT                            /* use i[0..n) */
 } dnnf_attr_key_t;
 
 /* Cast targets (attribute TO) */

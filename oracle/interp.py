@@ -325,6 +325,12 @@ def op_instancenorm(x, scale, bias, eps=1e-5):
     return (x - mean) / np.sqrt(var + float(eps)) * np.asarray(scale, dtype=np.float64) + np.asarray(bias, dtype=np.float64)
 
 
+def op_einsum(a, b, equation):
+    """ONNX Einsum of two operands in explicit form ("bhqd,bhkd->bhqk"): the sum over the labels that are missing in
+    the result of the products of the operands' elements (the library routine is the definition written out)."""
+    return np.einsum(equation, np.asarray(a, dtype=np.float64), np.asarray(b, dtype=np.float64))
+
+
 # ---- dispatcher -------------------------------------------------------------
 
 def _apply(op, ins, at):
@@ -389,6 +395,7 @@ def _apply(op, ins, at):
     if op == "Where": return [op_where(ins[0], ins[1], ins[2])]
     if op == "Cast": return [op_cast(ins[0], at["to"])]
     if op == "CumSum": return [op_cumsum(ins[0], g("axis", -1), g("exclusive", 0), g("reverse", 0))]
+    if op == "Einsum": return [op_einsum(ins[0], ins[1], at["equation"])]
     if op == "InstanceNorm": return [op_instancenorm(ins[0], ins[1], ins[2], g("eps", 1e-5))]
     raise KeyError(f"oracle: unknown operator {op}")
 

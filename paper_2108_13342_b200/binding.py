@@ -33,12 +33,12 @@ OP_NAMES = ["?", "Add", "Sub", "Mul", "Div", "MulC", "AddC", "Sigmoid", "Tanh", 
             "Squeeze", "Unsqueeze", "Split", "Slice", "MatMul", "Conv1x1", "DwConv3x3", "Softmax", "LayerNorm",
             "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift", "DepthToSpace", "SpaceToDepth", "Resize", "Concat", "MaxPool", "AveragePool", "Sin", "Cos", "Asin", "Ceil",
             "Floor", "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConvTranspose", "Gather", "Where", "Cast", "CumSum", "InstanceNorm",
-            "ConcatPart"]
+            "Einsum", "ConcatPart"]
 OP = {n: i for i, n in enumerate(OP_NAMES) if i}
 
 ATTR = {"c": 1, "lo": 2, "hi": 3, "p": 4, "eps": 5, "approx": 6, "axis": 7, "keepdims": 8, "start": 9, "end": 10,
         "bits": 11, "perm": 12, "shape": 13, "sizes": 14, "axes": 15, "block": 16, "scale": 17, "kernel": 18, "stride": 19, "pad": 20,
-        "to": 21, "exclusive": 22, "reverse": 23,
+        "to": 21, "exclusive": 22, "reverse": 23, "labels_a": 24, "labels_b": 25, "labels_out": 26,
         "alpha": 1}      # LeakyRelu's slope travels as attribute C
 CAST_TO = {"f32": 0, "bf16": 1, "i32": 2, "bool": 3}
 _FLOAT_ATTRS = {"c", "lo", "hi", "p", "eps", "alpha"}
@@ -177,6 +177,11 @@ class Graph:
         if isinstance(kind, str):
             kind = OP[kind]
         ins = (C.c_int * len(inputs))(*inputs)
+        if "equation" in attrs:                      # "bhqd,bhkd->bhqk": one integer per axis label
+            attrs = dict(attrs)
+            lhs, out = attrs.pop("equation").replace(" ", "").split("->")
+            a, b = lhs.split(",")
+            attrs.update(labels_a=[ord(c) for c in a], labels_b=[ord(c) for c in b], labels_out=[ord(c) for c in out])
         alist = []
         for k, v in attrs.items():
             if k == "approx" and isinstance(v, str):

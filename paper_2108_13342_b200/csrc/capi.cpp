@@ -89,6 +89,9 @@ static int parse_attrs(const dnnf_attr* a, int n, Attrs& at, std::string& err) {
       case DNNF_ATTR_TO: at.to = x.i[0]; break;
       case DNNF_ATTR_EXCLUSIVE: at.exclusive = x.i[0] != 0; break;
       case DNNF_ATTR_REVERSE: at.reverse = x.i[0] != 0; break;
+      case DNNF_ATTR_LABELS_A: at.perm = v; break;          // an Einsum has no other use for these three lists
+      case DNNF_ATTR_LABELS_B: at.sizes = v; break;
+      case DNNF_ATTR_LABELS_OUT: at.axes = v; break;
       default: err = "unknown attribute key"; return DNNF_ERR_INVALID_ARG;
     }
   }
@@ -187,6 +190,77 @@ int dnnf_add_op(dnnf_graph* g, int op_kind, int n_in, const int* in_ids, const d
     if (!rc) rc = emit(DNNF_OP_RESHAPE, {cur}, a3);
     if (!rc) rc = emit(DNNF_OP_TRANSPOSE, {cur}, a4);
     if (!rc) rc = emit(DNNF_OP_RESHAPE, {cur}, a5);
+    if (rc) { rollback(); G.err = err; return rc; }
+    outs = {cur};
+  } else if (op_kind == DNNF_OP_EINSUM) {
+    // Labels of both operands and of the result: batch.  Of both operands only: summed.  Of one operand and the
+    // result: that operand's free axes.  With the operands permuted to [batch, free, summed] and [batch, summed, free]
+    // and each group merged into one axis the operator is a batched matrix product.
+    if (n_in != 2) return fail(g, DNNF_ERR_INVALID_ARG, "Einsum takes two operands");
+    const std::vector<int64_t>& la = at.perm, & lb = at.sizes, & lo = at.axes;
+    const std::vector<int64_t> da = G.tensors[in_ids[0]].dims, db = G.tensors[in_ids[1]].dims;
+    if (la.size() != da.size() || lb.size() != db.size()) return fail(g, DNNF_ERR_SHAPE, "Einsum: one label per axis");
+    auto pos = [](const std::vector<int64_t>& l, int64_t x) { for (size_t i = 0; i < l.size(); ++i) if (l[i] == x) return (int)i; return -1; };
+    auto repeats = [](const std::vector<int64_t>& l) { for (size_t i = 0; i < l.size(); ++i) for (size_t j = i + 1; j < l.size(); ++j) if (l[i] == l[j]) return true; return false; };
+    if (repeats(la) || repeats(lb) || repeats(lo)) return fail(g, DNNF_ERR_UNSUPPORTED_OP, "Einsum: a label repeats inside one operand");
+    std::vector<int64_t> batch, fa, fb, sum;       // labels, in the order of the result (batch, free) or of A (summed)
+    for (auto x : lo) {
+      const int ia = pos(la, x), ib = pos(lb, x);
+      if (ia < 0 && ib < 0) return fail(g, DNNF_ERR_SHAPE, "Einsum: a result label is in no operand");
+      if (ia >= 0 && ib >= 0) { if (da[ia] != db[ib]) return fail(g, DNNF_ERR_SHAPE, "Einsum: extents of a label differ"); batch.push_back(x); }
+      else (ia >= 0 ? fa : fb).push_back(x);
+    }
+    for (auto x : la) if (pos(lo, x) < 0) {
+      const int ib = pos(lb, x);
+      if (ib < 0) return fail(g, DNNF_ERR_UNSUPPORTED_OP, "Einsum: a label of one operand only is summed away (use ReduceSum)");
+      if (da[pos(la, x)] != db[ib]) return fail(g, DNNF_ERR_SHAPE, "Einsum: extents of a label differ");
+      sum.push_back(x);
+    }
+    for (auto x : lb) if (pos(lo, x) < 0 && pos(la, x) < 0) return fail(g, DNNF_ERR_UNSUPPORTED_OP, "Einsum: a label of one operand only is summed away (use ReduceSum)");
+    if (sum.empty()) return fail(g, DNNF_ERR_UNSUPPORTED_OP, "Einsum without a summed label (an element-wise or outer product: use Mul)");
+    int cur = -1;
+    auto emit = [&](int kind, std::vector<int> ins, const Attrs& a) -> int {
+      Op o; o.id = (int)G.ops.size(); o.kind = kind; o.source_id = source; o.in = ins; o.at = a;
+      int r = infer_shapes(G, o, err);
+      if (r) return r;
+      cur = o.out[0];
+      G.ops.push_back(o);
+      return DNNF_OK;
+    };
+    auto identity = [](const std::vector<int64_t>& p) { for (size_t i = 0; i < p.size(); ++i) if (p[i] != (int64_t)i) return false; return true; };
+    auto prod = [&](const std::vector<int64_t>& labels, const std::vector<int64_t>& l, const std::vector<int64_t>& d) { int64_t n = 1; for (auto x : labels) n *= d[pos(l, x)]; return n; };
+    const int64_t Bt = prod(batch, la, da), M = prod(fa, la, da), K = prod(sum, la, da), Nn = prod(fb, lb, db);
+    // operand: permute to the group order, merge the groups
+    auto arrange = [&](int t, const std::vector<int64_t>& l, const std::vector<std::vector<int64_t>>& groups, const std::vector<int64_t>& shape) -> int {
+      Attrs ap, ar;
+      for (auto& grp : groups) for (auto x : grp) ap.perm.push_back(pos(l, x));
+      cur = t;
+      int r = DNNF_OK;
+      if (!identity(ap.perm)) r = emit(DNNF_OP_TRANSPOSE, {cur}, ap);
+      ar.shape = shape;
+      if (!r && G.tensors[cur].dims != shape) r = emit(DNNF_OP_RESHAPE, {cur}, ar);
+      return r;
+    };
+    const bool batched = !batch.empty();
+    std::vector<int64_t> sa = batched ? std::vector<int64_t>{Bt, M, K} : std::vector<int64_t>{M, K};
+    std::vector<int64_t> sb = batched ? std::vector<int64_t>{Bt, K, Nn} : std::vector<int64_t>{K, Nn};
+    rc = arrange(in_ids[0], la, {batch, fa, sum}, sa);
+    const int ta = cur;
+    if (!rc) rc = arrange(in_ids[1], lb, {batch, sum, fb}, sb);
+    const int tb = cur;
+    if (!rc) rc = emit(DNNF_OP_MATMUL, {ta, tb}, Attrs{});
+    if (!rc) {
+      // [batch, free of A, free of B] -> the separate axes -> the result's order
+      std::vector<int64_t> have = batch;
+      have.insert(have.end(), fa.begin(), fa.end());
+      have.insert(have.end(), fb.begin(), fb.end());
+      Attrs ar, ap;
+      for (auto x : have) ar.shape.push_back(pos(la, x) >= 0 ? da[pos(la, x)] : db[pos(lb, x)]);
+      if (ar.shape.empty()) ar.shape = {1};
+      if (G.tensors[cur].dims != ar.shape) rc = emit(DNNF_OP_RESHAPE, {cur}, ar);
+      for (auto x : lo) ap.perm.push_back(pos(have, x));
+      if (!rc && !lo.empty() && !identity(ap.perm)) rc = emit(DNNF_OP_TRANSPOSE, {cur}, ap);
+    }
     if (rc) { rollback(); G.err = err; return rc; }
     outs = {cur};
   } else if (op_kind == DNNF_OP_INSTANCENORM) {

@@ -416,3 +416,34 @@ def test_instance_normalization(shape):
     ins = {"X": rnd(shape, 12, -1.0, 3.0), "s": rnd((c,), 13, 0.5, 1.5), "t": rnd((c,), 14, -0.5, 0.5)}
     s = check(W.Workload(g, ins), RTOL_F32)
     assert s.plan_stats.n_ops == 2
+
+
+# ---- Einsum (Table 2, Many-to-Many) ---------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("eq,sa,sb,dtype", [
+    ("ik,kj->ij", (130, 72), (72, 40), "f32"),
+    ("ik,jk->ij", (100, 64), (48, 64), "f32"),                              # K-major second operand
+    ("bik,bkj->bij", (6, 70, 32), (6, 32, 24), "f32"),
+    ("nhwc,co->nhwo", (2, 20, 20, 24), (24, 48), "f32"),                   # a pointwise convolution
+    ("bhqd,bhkd->bhqk", (2, 4, 128, 64), (2, 4, 128, 64), "bf16"),         # attention scores
+    ("bhqk,bhkd->bhqd", (2, 4, 128, 128), (2, 4, 128, 64), "bf16"),        # probabilities times V
+    ("bqhd,bkhd->bhqk", (2, 128, 4, 64), (2, 128, 4, 64), "bf16"),         # heads inside: strided head views
+    ("mck,knc->nm", (33, 8, 16), (16, 40, 8), "f32"),                      # two summed labels, permuted result
+    ("ik,k->i", (257, 64), (64,), "f32"),
+])
+def test_einsum(eq, sa, sb, dtype):
+    g = graph(); g.ext("A", sa, dtype); g.ext("Bm", sb, dtype)
+    g.mark_output(g.add("Einsum", ["A", "Bm"], equation=eq))
+    a, b = rnd(sa, 21, -1.0, 1.0), rnd(sb, 22, -1.0, 1.0)
+    if dtype == "bf16":
+        a, b = W.round_to_bf16(a), W.round_to_bf16(b)
+    s = check(W.Workload(g, {"A": a, "Bm": b}), 2e-2 if dtype == "bf16" else RTOL_F32)
+    assert s.plan_stats.n_ops == 1
+
+
+def test_einsum_with_neighbours_fuses_like_a_matrix_product():
+    # bias and activation behind the contraction go into its epilogue
+    g = graph(); g.ext("A", (300, 48)); g.ext("Bm", (48, 64), kind="weight"); g.ext("b", (64,), kind="weight")
+    g.mark_output(g.add("Relu", [g.add("Add", [g.add("Einsum", ["A", "Bm"], equation="ik,kj->ij"), "b"])]))
+    s = check(W.Workload(g, {"A": rnd((300, 48), 23, -1, 1), "Bm": rnd((48, 64), 24, -0.3, 0.3), "b": rnd((64,), 25)}), RTOL_F32, expect_blocks=1)
+    assert s.g.blocks()[0]["family"] == "gemm"

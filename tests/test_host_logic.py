@@ -698,3 +698,33 @@ def test_beyond_table3_forms_the_single_kernel_inverted_residual_block_only_whil
     assert fams(full, beyond | B.PLAN_MBCONV_ALWAYS)[0] == ["mbconv"]
     # the intermediate tensors of the single kernel never reach memory
     assert fams(small, beyond)[1].irs_bytes_fused == 0 and fams(small, B.PLAN_FUSED)[1].irs_bytes_fused > 0
+
+
+def test_einsum_is_recorded_as_a_batched_matrix_product_between_index_operators():
+    def kinds_of(eq, sa, sb):
+        g = _desc(); g.ext("A", sa); g.ext("Bm", sb)
+        y = g.add("Einsum", ["A", "Bm"], equation=eq)
+        g.mark_output(y)
+        G, ids = build_graph(g)
+        kinds = [B.OP_NAMES[k] for k, alive in (G.op_kind(i) for i in range(G.op_count())) if alive]
+        return G, ids[y], kinds
+    G, y, kinds = kinds_of("ik,kj->ij", (4, 7), (7, 3))
+    assert kinds == ["MatMul"] and G.tensor_info(y)[1] == (4, 3) and G.op_mapping(0) == MM
+    G, y, kinds = kinds_of("bhqd,bhkd->bhqk", (2, 3, 4, 5), (2, 3, 6, 5))
+    assert kinds == ["Reshape", "Transpose", "Reshape", "MatMul", "Reshape"] and G.tensor_info(y)[1] == (2, 3, 4, 6)
+    G, y, kinds = kinds_of("mck,knc->nm", (3, 2, 4), (4, 5, 2))
+    assert kinds.count("MatMul") == 1 and kinds[-1] == "Transpose" and G.tensor_info(y)[1] == (5, 3)
+    G.rewrite(B.REWRITE_NONE)
+    assert G.plan().n_ops == 1                                        # the pieces count as the one operator they came from
+    for eq, sa, sb in [("ii,ij->j", (3, 3), (3, 4)), ("ik,kj->ijz", (2, 3), (3, 4)), ("ik,lj->ij", (2, 3), (3, 4)), ("ij,ij->ij", (2, 3), (2, 3)),
+                       ("ik,kj->ij", (2, 3), (4, 5)), ("ikl,kj->ij", (2, 3), (3, 4))]:
+        g = _desc(); g.ext("A", sa); g.ext("Bm", sb)
+        with pytest.raises(B.DnnfError):
+            build_graph_with(g, eq)
+    g = _desc(); g.ext("A", (2, 3)); g.ext("Bm", (3, 4))
+    assert g.add("Relu", ["A"])                                       # the graph stays usable after the refusals above
+
+
+def build_graph_with(g, eq):
+    g.add("Einsum", ["A", "Bm"], equation=eq)
+    return build_graph(g)

@@ -554,3 +554,27 @@ def test_instancenorm_index_loops_and_invariants():
     xt = x.transpose(0, 3, 1, 2).reshape(N, Cc, H * Wd)
     ln = O.op_layernorm(xt, np.ones(H * Wd), np.zeros(H * Wd), -1, eps).reshape(N, Cc, H, Wd).transpose(0, 2, 3, 1)
     np.testing.assert_allclose(y, ln * s + b, atol=1e-12)
+
+
+def test_einsum_index_loops_and_matrix_product_cases():
+    r = np.random.default_rng(9)
+    a = r.standard_normal((2, 3, 4, 5)); b = r.standard_normal((2, 3, 6, 5))
+    y = O.op_einsum(a, b, "bhqd,bhkd->bhqk")
+    assert y.shape == (2, 3, 4, 6)
+    for i, j, q, k in itertools.product(range(2), range(3), range(4), range(6)):
+        assert abs(y[i, j, q, k] - sum(a[i, j, q, d] * b[i, j, k, d] for d in range(5))) < 1e-12
+    np.testing.assert_allclose(y, O.op_matmul(a, np.swapaxes(b, -1, -2)), atol=1e-12)         # Q K^T
+    # a permuted result, two summed labels, free labels on both sides that are not adjacent
+    a = r.standard_normal((3, 2, 4)); b = r.standard_normal((4, 5, 2))
+    y = O.op_einsum(a, b, "mck,knc->nm")
+    for n, m in itertools.product(range(5), range(3)):
+        assert abs(y[n, m] - sum(a[m, c, k] * b[k, n, c] for c in range(2) for k in range(4))) < 1e-12
+    # plain cases: matrix product, matrix-vector, a 1x1 convolution over NHWC pixels
+    A = r.standard_normal((4, 7)); Bm = r.standard_normal((7, 3)); v = r.standard_normal(7)
+    np.testing.assert_allclose(O.op_einsum(A, Bm, "ik,kj->ij"), O.op_matmul(A, Bm), atol=1e-12)
+    np.testing.assert_allclose(O.op_einsum(A, v, "ik,k->i"), A @ v, atol=1e-12)
+    x = r.standard_normal((2, 3, 3, 7))
+    np.testing.assert_allclose(O.op_einsum(x, Bm, "nhwc,co->nhwo"), O.op_conv1x1(x, Bm), atol=1e-12)
+    # linear in each operand; ones as the second operand sum the label away
+    np.testing.assert_allclose(O.op_einsum(2.0 * A, Bm, "ik,kj->ij"), 2.0 * O.op_einsum(A, Bm, "ik,kj->ij"), atol=1e-12)
+    np.testing.assert_allclose(O.op_einsum(A, np.ones((7, 1)), "ik,kj->ij")[:, 0], O.op_reducesum(A, -1, 0), atol=1e-12)
