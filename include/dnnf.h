@@ -117,7 +117,10 @@ typedef enum {
                                                        no padding: y[n,h*k+i,w*k+j,o] = sum_c x[n,h,w,c] W[c,i,j,o].  Recorded as
                                                        Reshape(W) -> Conv1x1 -> DepthToSpace, which it equals term by term */
   DNNF_OP_GATHER,                                   /* One-to-Many; (table [V,D], indices [...]) along axis 0: y[..., :] = table[indices[...], :].
-                                                       Indices are integer-valued fp32 numbers; out-of-range ones are clamped */
+                                                       Indices are integer-valued fp32 numbers; out-of-range ones are clamped.  A table of
+                                                       another rank or another AXIS is recorded as Transpose / Reshape to that form, the
+                                                       row gather, and Reshape / Transpose of the result (the index axes take the place of
+                                                       the gathered axis) */
   DNNF_OP_WHERE,                                    /* One-to-One (Table 2); (cond, a, b) with broadcasting: a where the 0 / 1 valued cond
                                                        is non-zero, else b.  A selection: the other branch's value is never touched */
   DNNF_OP_CAST,                                     /* One-to-One (Table 2); attribute TO: DNNF_CAST_F32 (values unchanged), DNNF_CAST_BF16

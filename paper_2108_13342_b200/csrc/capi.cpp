@@ -192,6 +192,47 @@ int dnnf_add_op(dnnf_graph* g, int op_kind, int n_in, const int* in_ids, const d
     if (!rc) rc = emit(DNNF_OP_RESHAPE, {cur}, a5);
     if (rc) { rollback(); G.err = err; return rc; }
     outs = {cur};
+  } else if (op_kind == DNNF_OP_GATHER && n_in == 2 &&
+             (G.tensors[in_ids[0]].dims.size() != 2 || !(at.axis == 0 || at.axis == -2))) {
+    // Gather along any axis of a table of any rank: the axis moves to the front, the other axes merge into the row of a
+    // [V, D] table, rows are gathered, and the index axes move to where the gathered axis was.
+    const std::vector<int64_t> d = G.tensors[in_ids[0]].dims, qd = G.tensors[in_ids[1]].dims;
+    const int r = (int)d.size(), nq = (int)qd.size();
+    const int a = (int)(at.axis < 0 ? at.axis + r : at.axis);
+    if (r < 1 || a < 0 || a >= r) return fail(g, DNNF_ERR_SHAPE, "Gather: axis");
+    if (r - 1 + nq > kMaxDims || r - 1 + nq < 1) return fail(g, DNNF_ERR_SHAPE, "Gather: rank of the result");
+    int cur = in_ids[0];
+    auto emit = [&](int kind, std::vector<int> ins, const Attrs& at2) -> int {
+      Op o; o.id = (int)G.ops.size(); o.kind = kind; o.source_id = source; o.in = ins; o.at = at2;
+      int rr = infer_shapes(G, o, err);
+      if (rr) return rr;
+      cur = o.out[0];
+      G.ops.push_back(o);
+      return DNNF_OK;
+    };
+    int64_t rest = 1;
+    std::vector<int64_t> others;
+    for (int i = 0; i < r; ++i) if (i != a) { rest *= d[i]; others.push_back(d[i]); }
+    Attrs a1, a2, a3, a4, a5;
+    a1.perm.push_back(a);
+    for (int i = 0; i < r; ++i) if (i != a) a1.perm.push_back(i);
+    rc = DNNF_OK;
+    if (a != 0) rc = emit(DNNF_OP_TRANSPOSE, {cur}, a1);
+    a2.shape = {d[a], rest};
+    if (!rc && G.tensors[cur].dims != a2.shape) rc = emit(DNNF_OP_RESHAPE, {cur}, a2);
+    a3.axis = 0;
+    if (!rc) rc = emit(DNNF_OP_GATHER, {cur, in_ids[1]}, a3);
+    a4.shape = qd;
+    a4.shape.insert(a4.shape.end(), others.begin(), others.end());
+    if (!rc && G.tensors[cur].dims != a4.shape) rc = emit(DNNF_OP_RESHAPE, {cur}, a4);
+    if (!rc && a != 0) {
+      for (int i = 0; i < a; ++i) a5.perm.push_back(nq + i);
+      for (int i = 0; i < nq; ++i) a5.perm.push_back(i);
+      for (int i = a; i < r - 1; ++i) a5.perm.push_back(nq + i);
+      rc = emit(DNNF_OP_TRANSPOSE, {cur}, a5);
+    }
+    if (rc) { rollback(); G.err = err; return rc; }
+    outs = {cur};
   } else if (op_kind == DNNF_OP_EINSUM) {
     // Labels of both operands and of the result: batch.  Of both operands only: summed.  Of one operand and the
     // result: that operand's free axes.  With the operands permuted to [batch, free, summed] and [batch, summed, free]

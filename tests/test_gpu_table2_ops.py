@@ -447,3 +447,16 @@ def test_einsum_with_neighbours_fuses_like_a_matrix_product():
     g.mark_output(g.add("Relu", [g.add("Add", [g.add("Einsum", ["A", "Bm"], equation="ik,kj->ij"), "b"])]))
     s = check(W.Workload(g, {"A": rnd((300, 48), 23, -1, 1), "Bm": rnd((48, 64), 24, -0.3, 0.3), "b": rnd((64,), 25)}), RTOL_F32, expect_blocks=1)
     assert s.g.blocks()[0]["family"] == "gemm"
+
+
+@pytest.mark.parametrize("shape,axis,idx_shape", [((6, 40, 32), 1, (7,)), ((5, 9, 64), 2, (3, 4)), ((12, 8, 4, 16), 0, (5,)), ((50,), 0, (4, 6)),
+                                                  ((3, 20, 8), -2, (2, 2))])
+def test_gather_along_any_axis(shape, axis, idx_shape):
+    g = graph("gather_axis"); g.ext("T", shape); g.ext("I", idx_shape)
+    g.mark_output(g.add("Relu", [g.add("Gather", ["T", "I"], axis=axis)]))
+    v = shape[axis]
+    idx = np.floor(W.uniform(777, 90, idx_shape, 0.0, float(v))).clip(0, v - 1)
+    s, got, ref = run_both(W.Workload(g, {"T": rnd(shape, 91), "I": idx}))
+    name = g.outputs[0]
+    assert np.array_equal(got[name].astype(np.float64), ref[name])          # a selection followed by max(x, 0): bit-exact
+    assert s.plan_stats.n_ops == 2

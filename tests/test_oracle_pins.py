@@ -166,6 +166,16 @@ def test_gather():
     x = rnd((5, 3), 8)
     y = O.op_gather(x, np.array([4.0, 0.0, 4.0]), 0)
     assert np.array_equal(y, np.stack([x[4], x[0], x[4]]))
+    # any axis, index tensors of any rank: the index axes take the place of the gathered axis
+    t = rnd((3, 4, 5), 9)
+    idx = np.array([[3.0, 0.0], [1.0, 1.0], [2.0, 3.0]])
+    y = O.op_gather(t, idx, 1)
+    assert y.shape == (3, 3, 2, 5)
+    for a, i, j, c in itertools.product(range(3), range(3), range(2), range(5)):
+        assert y[a, i, j, c] == t[a, int(idx[i, j]), c]
+    y = O.op_gather(t, np.array([4.0, 4.0, 0.0]), -1)
+    for a, b, i in itertools.product(range(3), range(4), range(3)):
+        assert y[a, b, i] == t[a, b, [4, 4, 0][i]]
 
 
 def test_further_one_to_one_operators_at_known_points():
