@@ -27,7 +27,7 @@ class _Rng:
         return xs[min(int(self.u() * len(xs)), len(xs) - 1)]
 
 
-def _build(seed, big=False, dtype="f32", extended=False):
+def _build(seed, big=False, dtype="f32", extended=False, table2=False):
     r = _Rng(seed)
     bsz, rows, cols = r.pick([1, 2, 3]), r.pick([5, 8, 16, 33]), r.pick([8, 12, 32, 64])
     if big:      # sizes that reach the vectorised, multi-vector, multi-warp and tensor-core variants
@@ -63,8 +63,9 @@ def _build(seed, big=False, dtype="f32", extended=False):
     for _ in range(n_ops):
         t, shp = r.pick(pool[-4:]) if r.u() < 0.7 else r.pick(pool)      # mostly recent values (long chains), sometimes old ones (diamonds)
         kind = r.pick(["unary", "unary", "vec", "full", "transpose", "reshape", "slice", "reduce", "softmax", "layernorm", "matmul",
-                       "rowvec", "exp", "div", "reduce0", "permute"] + (["concat", "concat", "concat"] if extended else []))
-        if kind in ("reduce", "reduce0", "softmax", "layernorm") and shp[-1] > 8192:
+                       "rowvec", "exp", "div", "reduce0", "permute"] + (["concat", "concat", "concat"] if extended else [])
+                      + (["where", "where", "cumsum", "cumsum", "where_vec"] if table2 else []))
+        if kind in ("reduce", "reduce0", "softmax", "layernorm", "cumsum") and shp[-1] > 8192:
             continue                                    # longer rows than the row kernels take (the plan says so)
         if kind == "unary":
             op, at = r.pick([("Tanh", {}), ("Sigmoid", {}), ("Relu", {}), ("Abs", {}), ("Square", {}), ("Neg", {}),
@@ -72,6 +73,15 @@ def _build(seed, big=False, dtype="f32", extended=False):
             if op == "Square":
                 t = g.add("Tanh", [t])                  # keep magnitudes bounded
             o = g.add(op, [t], **at)
+        elif kind == "where":                          # the condition and both branches are values of the graph
+            cands = [p for p in pool if p[1] == shp]
+            a, b, c = r.pick(cands)[0], r.pick(cands)[0], r.pick(cands)[0]
+            o = g.add("Where", [g.add("Greater", [t, a]), b, g.add("Neg", [c])])
+        elif kind == "where_vec":                      # a broadcast condition and a broadcast branch
+            o = g.add("Where", [g.add("Greater", [vec(shp[-1], -1.0, 1.0), vec(shp[-1], -1.0, 1.0)]), t, vec(shp[-1], -1.0, 1.0)])
+        elif kind == "cumsum":
+            o = g.add("CumSum", [g.add("Tanh", [t])], axis=-1, exclusive=int(r.u() < 0.3), reverse=int(r.u() < 0.3))
+            o = g.add("MulC", [o], c=1.0 / max(1, shp[-1]) ** 0.5)
         elif kind == "exp":
             o = g.add("Exp", [g.add("MulC", [g.add("Tanh", [t])], c=0.5)])
         elif kind == "div":
@@ -364,3 +374,25 @@ def test_random_graph_bf16(seed):
             close(got, ref[n], 3e-2)
         except AssertionError as e:
             raise AssertionError(f"{n} plan {[b['ops'] for b in s.g.blocks()]}: {e}") from None
+
+
+@pytest.mark.parametrize("seed", [pytest.param(i, id=str(i)) for i in range(100)] + [pytest.param(-i - 1, id="big%d" % i) for i in range(24)])
+def test_random_graph_with_where_and_cumsum(seed):
+    """The same generator with Where (conditions and branches computed in the graph, or broadcast) and CumSum (inclusive,
+    exclusive, reverse) among the operators."""
+    wl = _build(8000 + seed, False, table2=True) if seed >= 0 else _build(9000 - seed, True, table2=True)
+    ref = O.run_graph(wl.graph, wl.inputs)
+    for flags, rewrite in ((B.PLAN_FUSED, B.REWRITE_NONE), (B.PLAN_UNFUSED, B.REWRITE_NONE), (B.PLAN_FUSED, B.REWRITE_DEFAULT)):
+        s = Session(wl, plan_flags=flags, rewrite_flags=rewrite)
+        s.workspace[s.g.workspace_zero_bytes():].fill_(0xFF)
+        for n in wl.graph.outputs:
+            s.buffers[n].fill_(float("nan"))
+        s.run()
+        assert s.g.status()[0] == 0
+        for n in wl.graph.outputs:
+            got = s.output(n)
+            assert np.isfinite(got).all(), (n, "unwritten elements", [b["ops"] for b in s.g.blocks()])
+            try:
+                close(got, ref[n], 2e-5)
+            except AssertionError as e:
+                raise AssertionError(f"{n} flags {flags} rewrite {rewrite} plan {[b['ops'] for b in s.g.blocks()]}: {e}") from None
