@@ -113,9 +113,12 @@ typedef enum {
   DNNF_OP_NOT,                                      /* on 0 / 1 valued tensors: 1 where the input is 0, else 0 */
   DNNF_OP_GREATER,                                  /* (a, b) with broadcasting: 1 where a > b, else 0 */
   DNNF_OP_PRELU,                                    /* (x, slope) with broadcasting: x where x > 0, else slope * x */
-  DNNF_OP_CONVTRANSPOSE,                            /* Many-to-Many; NHWC x [Cin,k,k,Cout] with stride = kernel = k (attribute KERNEL),
-                                                       no padding: y[n,h*k+i,w*k+j,o] = sum_c x[n,h,w,c] W[c,i,j,o].  Recorded as
-                                                       Reshape(W) -> Conv1x1 -> DepthToSpace, which it equals term by term */
+  DNNF_OP_CONVTRANSPOSE,                            /* Many-to-Many; NHWC x [Cin,k,k,Cout], attributes KERNEL k, STRIDE s <= k (default: k) and PAD
+                                                       p < k: y[n,h*s+i-p,w*s+j-p,o] += sum_c x[n,h,w,c] W[c,i,j,o], the result has
+                                                       (H-1)*s + k - 2p rows.  With s = k and p = 0 the patches do not overlap and the operator is
+                                                       recorded as Reshape(W) -> Conv1x1 -> DepthToSpace; otherwise as Reshape(W) -> Conv1x1
+                                                       (all k*k*Cout patch values of every pixel) -> Col2Im (each output element adds the at most
+                                                       ceil(k/s)^2 patch values that land on it; Cout a multiple of 4) */
   DNNF_OP_GATHER,                                   /* One-to-Many; (table [V,D], indices [...]) along axis 0: y[..., :] = table[indices[...], :].
                                                        Indices are integer-valued fp32 numbers; out-of-range ones are clamped.  A table of
                                                        another rank or another AXIS is recorded as Transpose / Reshape to that form, the
@@ -139,6 +142,7 @@ typedef enum {
                                                        over (at least one), no label repeats inside an operand and none belongs to one
                                                        operand only without reaching the result.  Recorded as Transpose / Reshape of the
                                                        operands -> (batched) MatMul -> Reshape / Transpose, which it equals term by term */
+  DNNF_OP_COL2IM,                                   /* internal (made by ConvTranspose): ([N,H,W,k*k*C]); KERNEL, STRIDE, PAD; Many-to-Many */
   DNNF_OP_CONCATPART,                               /* internal (made by Concat): (x [, result so far]); AXIS, START, SHAPE */
   DNNF_OP__COUNT
 } dnnf_op_t;

@@ -222,18 +222,18 @@ def op_maxpool(x, kernel, stride=1, pad=0): return _pool(x, kernel, stride, pad,
 def op_avgpool(x, kernel, stride=1, pad=0): return _pool(x, kernel, stride, pad, False)
 
 
-def op_convtranspose(x, w, stride):
-    """NHWC transposed convolution without padding, weights [Cin, k, k, Cout]: every input pixel adds its
-    k x k x Cout patch at (h*s, w*s): y[n, h*s+i, w*s+j, o] += sum_c x[n,h,w,c] W[c,i,j,o]
-    (Table 2 lists ConvTranspose under Many-to-Many)."""
-    s = int(stride)
+def op_convtranspose(x, w, stride, pad=0):
+    """NHWC transposed convolution, weights [Cin, k, k, Cout]: every input pixel adds its k x k x Cout patch at
+    (h*s, w*s): y[n, h*s+i, w*s+j, o] += sum_c x[n,h,w,c] W[c,i,j,o]; `pad` rows and columns are then cut from every
+    border (ONNX pads), leaving (H-1)*s + k - 2*pad rows (Table 2 lists ConvTranspose under Many-to-Many)."""
+    s, p = int(stride), int(pad)
     n, h, wd, c = x.shape
     _, k, _, co = w.shape
     y = np.zeros((n, (h - 1) * s + k, (wd - 1) * s + k, co), dtype=np.float64)
     for a in range(h):
         for b in range(wd):
             y[:, a * s:a * s + k, b * s:b * s + k, :] += np.einsum("nc,cijo->nijo", x[:, a, b, :], w)
-    return y
+    return y[:, p:y.shape[1] - p, p:y.shape[2] - p, :] if p else y
 
 
 def op_softmax(x, axis=-1):
@@ -385,7 +385,7 @@ def _apply(op, ins, at):
     if op == "DwConv3x3": return [op_dwconv3x3(ins[0], ins[1])]
     if op == "MaxPool": return [op_maxpool(ins[0], at["kernel"], g("stride", 1), g("pad", 0))]
     if op == "AveragePool": return [op_avgpool(ins[0], at["kernel"], g("stride", 1), g("pad", 0))]
-    if op == "ConvTranspose": return [op_convtranspose(ins[0], ins[1], at["kernel"])]
+    if op == "ConvTranspose": return [op_convtranspose(ins[0], ins[1], g("stride", at["kernel"]), g("pad", 0))]
     if op == "Softmax": return [op_softmax(ins[0], g("axis", -1))]
     if op == "LayerNorm": return [op_layernorm(ins[0], ins[1], ins[2], g("axis", -1), g("eps", 1e-5))]
     if op == "ReduceSum": return [op_reducesum(ins[0], g("axis", -1), g("keepdims", 1))]

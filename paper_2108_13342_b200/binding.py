@@ -33,7 +33,7 @@ OP_NAMES = ["?", "Add", "Sub", "Mul", "Div", "MulC", "AddC", "Sigmoid", "Tanh", 
             "Squeeze", "Unsqueeze", "Split", "Slice", "MatMul", "Conv1x1", "DwConv3x3", "Softmax", "LayerNorm",
             "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift", "DepthToSpace", "SpaceToDepth", "Resize", "Concat", "MaxPool", "AveragePool", "Sin", "Cos", "Asin", "Ceil",
             "Floor", "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConvTranspose", "Gather", "Where", "Cast", "CumSum", "InstanceNorm",
-            "Einsum", "ConcatPart"]
+            "Einsum", "Col2Im", "ConcatPart"]
 OP = {n: i for i, n in enumerate(OP_NAMES) if i}
 
 ATTR = {"c": 1, "lo": 2, "hi": 3, "p": 4, "eps": 5, "approx": 6, "axis": 7, "keepdims": 8, "start": 9, "end": 10,

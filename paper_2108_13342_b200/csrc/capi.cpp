@@ -172,7 +172,13 @@ int dnnf_add_op(dnnf_graph* g, int op_kind, int n_in, const int* in_ids, const d
     const int64_t k = at.kernel;
     if (xd.size() != 4 || wd.size() != 4 || k < 1 || wd[0] != xd[3] || wd[1] != k || wd[2] != k)
       return fail(g, DNNF_ERR_SHAPE, "ConvTranspose: NHWC x [Cin,k,k,Cout] with stride = kernel = k");
-    if (at.stride != 1 && at.stride != k) return fail(g, DNNF_ERR_UNSUPPORTED_OP, "ConvTranspose: stride must equal the kernel size");
+    // STRIDE defaults to 1 in the attribute block; a ConvTranspose without the attribute means stride = kernel
+    bool has_stride = false;
+    for (int i = 0; i < n_attrs; ++i) if (attrs[i].key == DNNF_ATTR_STRIDE) has_stride = true;
+    const int64_t st = has_stride ? at.stride : k, pd = at.pad;
+    if (st < 1 || st > k || pd < 0 || pd >= k) return fail(g, DNNF_ERR_SHAPE, "ConvTranspose: 1 <= stride <= kernel and 0 <= pad < kernel");
+    if ((xd[1] - 1) * st + k - 2 * pd < 1 || (xd[2] - 1) * st + k - 2 * pd < 1) return fail(g, DNNF_ERR_SHAPE, "ConvTranspose: empty result");
+    const bool overlap = st != k || pd != 0;
     int cur = -1;
     auto emit = [&](int kind, std::vector<int> ins, const Attrs& a) -> int {
       Op o; o.id = (int)G.ops.size(); o.kind = kind; o.source_id = source; o.in = ins; o.at = a;
@@ -187,9 +193,15 @@ int dnnf_add_op(dnnf_graph* g, int op_kind, int n_in, const int* in_ids, const d
     rc = emit(DNNF_OP_RESHAPE, {in_ids[1]}, a1);
     if (!rc) rc = emit(DNNF_OP_CONV1X1, {in_ids[0], cur}, a2);
     a3.shape = {xd[0], xd[1], xd[2], k, k, wd[3]}; a4.perm = {0, 1, 3, 2, 4, 5}; a5.shape = {xd[0], xd[1] * k, xd[2] * k, wd[3]};
-    if (!rc) rc = emit(DNNF_OP_RESHAPE, {cur}, a3);
-    if (!rc) rc = emit(DNNF_OP_TRANSPOSE, {cur}, a4);
-    if (!rc) rc = emit(DNNF_OP_RESHAPE, {cur}, a5);
+    if (overlap) {
+      // patches overlap (or are cropped): every output element adds the patch values that land on it
+      Attrs a6; a6.kernel = k; a6.stride = st; a6.pad = pd;
+      if (!rc) rc = emit(DNNF_OP_COL2IM, {cur}, a6);
+    } else {
+      if (!rc) rc = emit(DNNF_OP_RESHAPE, {cur}, a3);
+      if (!rc) rc = emit(DNNF_OP_TRANSPOSE, {cur}, a4);
+      if (!rc) rc = emit(DNNF_OP_RESHAPE, {cur}, a5);
+    }
     if (rc) { rollback(); G.err = err; return rc; }
     outs = {cur};
   } else if (op_kind == DNNF_OP_GATHER && n_in == 2 &&

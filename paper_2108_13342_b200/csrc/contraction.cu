@@ -268,7 +268,7 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
   (void)flags;
   const Op& A = g.ops[anchor];
   if (A.kind == DNNF_OP_DWCONV3X3) return lower_dwconv(g, ops, anchor, out, why);
-  if (A.kind == DNNF_OP_MAXPOOL || A.kind == DNNF_OP_AVGPOOL) return lower_pool(g, ops, anchor, out, why);
+  if (A.kind == DNNF_OP_MAXPOOL || A.kind == DNNF_OP_AVGPOOL || A.kind == DNNF_OP_COL2IM) return lower_pool(g, ops, anchor, out, why);
   if (A.kind == DNNF_OP_GATHER) return lower_gather(g, ops, anchor, out, why);
   std::set<int> in_block(ops.begin(), ops.end());
   const Tensor& C = g.tensors[A.out[0]];

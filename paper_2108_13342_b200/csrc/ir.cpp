@@ -60,7 +60,7 @@ const char* op_name(int k) {
     "Sqrt", "Abs", "Neg", "Recip", "Square", "Relu", "Clip", "Pow", "Gelu", "ScaleShift", "Transpose", "Reshape",
     "Flatten", "Squeeze", "Unsqueeze", "Split", "Slice", "MatMul", "Conv1x1", "DwConv3x3", "Softmax", "LayerNorm",
     "ReduceSum", "ReduceMean", "ReduceMax", "ReduceProd", "Expand", "BitShift", "DepthToSpace", "SpaceToDepth", "Resize", "Concat", "MaxPool", "AveragePool", "Sin", "Cos", "Asin", "Ceil", "Floor",
-    "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConvTranspose", "Gather", "Where", "Cast", "CumSum", "InstanceNorm", "Einsum", "ConcatPart"};
+    "Round", "LeakyRelu", "Not", "Greater", "PRelu", "ConvTranspose", "Gather", "Where", "Cast", "CumSum", "InstanceNorm", "Einsum", "Col2Im", "ConcatPart"};
   if (k <= 0 || k >= DNNF_OP__COUNT) return "?";
   return names[k];
 }
@@ -81,7 +81,7 @@ bool is_row_anchor(int k) {
   return k == DNNF_OP_SOFTMAX || k == DNNF_OP_LAYERNORM || (k >= DNNF_OP_REDUCESUM && k <= DNNF_OP_REDUCEPROD) || k == DNNF_OP_CUMSUM;
 }
 bool is_contraction(int k) {      // anchors that take an epilogue chain and nothing in front
-  return k == DNNF_OP_MATMUL || k == DNNF_OP_CONV1X1 || k == DNNF_OP_DWCONV3X3 || k == DNNF_OP_MAXPOOL || k == DNNF_OP_AVGPOOL ||
+  return k == DNNF_OP_MATMUL || k == DNNF_OP_CONV1X1 || k == DNNF_OP_DWCONV3X3 || k == DNNF_OP_MAXPOOL || k == DNNF_OP_AVGPOOL || k == DNNF_OP_COL2IM ||
          k == DNNF_OP_GATHER;
 }
 
@@ -135,7 +135,7 @@ int node_mapping(const Graph& g, const Op& op) {
     case DNNF_OP_EXPAND: case DNNF_OP_GATHER: return DNNF_ONE_TO_MANY;
     case DNNF_OP_MATMUL: case DNNF_OP_CONV1X1: case DNNF_OP_DWCONV3X3: case DNNF_OP_SOFTMAX: case DNNF_OP_LAYERNORM:
     case DNNF_OP_REDUCESUM: case DNNF_OP_REDUCEMEAN: case DNNF_OP_REDUCEMAX: case DNNF_OP_REDUCEPROD:
-    case DNNF_OP_MAXPOOL: case DNNF_OP_AVGPOOL: case DNNF_OP_CUMSUM:
+    case DNNF_OP_MAXPOOL: case DNNF_OP_AVGPOOL: case DNNF_OP_CUMSUM: case DNNF_OP_COL2IM:
       return DNNF_MANY_TO_MANY;
     default: return DNNF_ONE_TO_ONE;
   }
@@ -295,6 +295,15 @@ int infer_shapes(Graph& g, Op& op, std::string& err) {
     auto d = in(0).dims;
     d[1] = (d[1] + 2 * pd - kk) / st + 1;
     d[2] = (d[2] + 2 * pd - kk) / st + 1;
+    outs.push_back(d);
+  } else if (k == DNNF_OP_COL2IM) {
+    if (!need(1)) return DNNF_ERR_INVALID_ARG;
+    const int64_t kk = op.at.kernel, st = op.at.stride, pd = op.at.pad;
+    if (in(0).dims.size() != 4 || kk < 1 || st < 1 || st > kk || pd < 0 || pd >= kk || in(0).dims[3] % (kk * kk)) { err = "Col2Im: patch tensor, kernel, stride or pad"; return DNNF_ERR_SHAPE; }
+    auto d = in(0).dims;
+    d[1] = (d[1] - 1) * st + kk - 2 * pd;
+    d[2] = (d[2] - 1) * st + kk - 2 * pd;
+    d[3] = d[3] / (kk * kk);
     outs.push_back(d);
   } else if (k == DNNF_OP_GATHER) {
     if (!need(2)) return DNNF_ERR_INVALID_ARG;

@@ -24,6 +24,8 @@ struct PoolParams {
   int32_t Hi, Wi;          // pooled tensor's height and width
   int32_t kernel, stride, pad;
   int32_t is_max;
+  int32_t col2im;          // the tensor holds k x k patches per pixel ([N,Hi,Wi,k*k*C]); an output element adds the values that land on it
+  int32_t Ci;              // channels per pixel of the tensor that is read (C, or k*k*C for col2im)
   FastDiv fd_c4, fd_w, fd_h;
   // wide windows (a global pool): CTAs per (pixel, 128-channel group) and how the window is sliced over them
   int32_t groups, slices, per_slice;
@@ -45,10 +47,29 @@ __global__ void __launch_bounds__(256) pool_kernel(const __grid_constant__ PoolP
   const int h0 = (int)ho * p.stride - p.pad, w0 = (int)wo * p.stride - p.pad;
   const int ha = max(h0, 0), hb = min(h0 + p.kernel, p.Hi);
   const int wa = max(w0, 0), wb = min(w0 + p.kernel, p.Wi);
-  const float* xb = p.d.x + ((size_t)n * p.Hi * p.Wi) * p.d.C + c4 * 4;
+  const float* xb = p.d.x + ((size_t)n * p.Hi * p.Wi) * p.Ci + c4 * 4;
   DwIO io{p.d};
   const float init = p.is_max ? -INFINITY : 0.0f;
   io.accv[0] = io.accv[1] = io.accv[2] = io.accv[3] = init;
+  if (p.col2im) {
+    // transposed convolution, gather form: output row ho receives tap i of input row h where ho + pad = h * stride + i,
+    // likewise for columns; at most ceil(k / s)^2 terms, added in a fixed order
+    const int s = p.stride, k = p.kernel;
+    const int hp = (int)ho + p.pad, wp = (int)wo + p.pad;
+    for (int i = hp % s; i < k; i += s) {
+      const int h = (hp - i) / s;
+      if (hp - i < 0 || h >= p.Hi) continue;
+      for (int j = wp % s; j < k; j += s) {
+        const int w = (wp - j) / s;
+        if (wp - j < 0 || w >= p.Wi) continue;
+        const float4 v = __ldg(reinterpret_cast<const float4*>(xb + ((size_t)h * p.Wi + w) * p.Ci + (size_t)(i * k + j) * p.d.C));
+        io.accv[0] += v.x; io.accv[1] += v.y; io.accv[2] += v.z; io.accv[3] += v.w;
+      }
+    }
+    io.n = n; io.h = ho; io.w = wo; io.c = c4 * 4;
+    run_program<4, SP>(p.d.prog, io);
+    return;
+  }
   if (p.kernel <= 3) {
     // up to nine loads, all issued before the first use (the window loop below would wait for each in turn)
     float4 v[9];
@@ -197,7 +218,7 @@ int lower_pool(const Graph& g, const std::vector<int>& ops, int anchor, Block& o
   const Tensor& Y = g.tensors[A.out[0]];
   std::set<int> in_block(ops.begin(), ops.end());
   if (X.dtype != DNNF_F32) { why = "pooling is fp32 only"; return DNNF_ERR_UNSUPPORTED_OP; }
-  if (X.dims[3] % 4) { why = "pooling needs a channel count that is a multiple of 4"; return DNNF_ERR_UNSUPPORTED_OP; }
+  if (Y.dims[3] % 4) { why = "pooling / col2im needs a channel count that is a multiple of 4"; return DNNF_ERR_UNSUPPORTED_OP; }
   if (in_block.count(X.producer)) { why = "operators in front of a pooling anchor (no prologue fusion)"; return DNNF_ERR_UNSUPPORTED_OP; }
   if (X.numel() >= (1ll << 31) || Y.numel() >= (1ll << 31)) { why = "tensor too large"; return DNNF_ERR_UNSUPPORTED_OP; }
   LowerCtx cx(g);
@@ -215,6 +236,8 @@ int lower_pool(const Graph& g, const std::vector<int>& ops, int anchor, Block& o
   pp.Hi = (int)X.dims[1]; pp.Wi = (int)X.dims[2];
   pp.kernel = (int)A.at.kernel; pp.stride = (int)A.at.stride; pp.pad = (int)A.at.pad;
   pp.is_max = A.kind == DNNF_OP_MAXPOOL;
+  pp.col2im = A.kind == DNNF_OP_COL2IM;
+  pp.Ci = (int)X.dims[3];
   pp.fd_c4 = make_fastdiv((uint32_t)dp.C / 4); pp.fd_w = make_fastdiv((uint32_t)dp.W); pp.fd_h = make_fastdiv((uint32_t)dp.H);
   dp.n_in = (int)cx.ins.size(); dp.n_out = (int)cx.outs.size();
   auto fill = [&](TensorArg& a, const ExtArg& e, bool is_out) {
@@ -240,7 +263,7 @@ int lower_pool(const Graph& g, const std::vector<int>& ops, int anchor, Block& o
   L.grid = (int)((total + 255) / 256);
   L.threads = 256;
   pp.slices = 0;
-  if (pp.kernel * pp.kernel >= 64 && !dev_env("DNNF_NO_WIDE_POOL")) {
+  if (!pp.col2im && pp.kernel * pp.kernel >= 64 && !dev_env("DNNF_NO_WIDE_POOL")) {
     // one thread per output would walk the window alone: give the window to whole CTAs instead
     pp.groups = (dp.C + 127) / 128;
     const int64_t units = (int64_t)dp.N * dp.H * dp.W * pp.groups;

@@ -40,6 +40,7 @@ int64_t op_flops(const Graph& g, const Op& o) {
   if (o.kind == DNNF_OP_MATMUL) { const Tensor& a = g.tensors[o.in[0]]; return 2 * g.tensors[o.out[0]].numel() * a.dims.back(); }
   if (o.kind == DNNF_OP_CONV1X1) return 2 * g.tensors[o.out[0]].numel() * g.tensors[o.in[1]].dims[0];
   if (o.kind == DNNF_OP_DWCONV3X3) return 18 * g.tensors[o.out[0]].numel();
+  if (o.kind == DNNF_OP_COL2IM) return g.tensors[o.in[0]].numel();
   if (o.kind == DNNF_OP_SCALESHIFT) return 2 * g.tensors[o.out[0]].numel();
   return g.tensors[o.out[0]].numel();
 }

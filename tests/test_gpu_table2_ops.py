@@ -460,3 +460,24 @@ def test_gather_along_any_axis(shape, axis, idx_shape):
     name = g.outputs[0]
     assert np.array_equal(got[name].astype(np.float64), ref[name])          # a selection followed by max(x, 0): bit-exact
     assert s.plan_stats.n_ops == 2
+
+
+@pytest.mark.parametrize("flags", [B.PLAN_FUSED, B.PLAN_UNFUSED])
+@pytest.mark.parametrize("shape,k,s,p,cout", [((2, 9, 11, 16), 4, 2, 1, 8), ((1, 16, 16, 32), 3, 2, 1, 16), ((3, 5, 7, 8), 3, 1, 1, 12),
+                                               ((2, 6, 6, 24), 2, 1, 0, 4), ((1, 12, 10, 16), 4, 2, 0, 32), ((2, 8, 8, 8), 5, 3, 2, 8),
+                                               ((4, 28, 28, 64), 4, 2, 1, 32)])
+def test_convtranspose_with_overlapping_patches(shape, k, s, p, cout, flags):
+    """Transposed convolutions whose patches overlap (stride < kernel) or are cropped (pad): the pointwise convolution onto
+    all k x k x Cout patch values followed by the gather that adds, per output element, the values that land on it;
+    ReLU and a residual ride in the gather's epilogue."""
+    n, h, w, c = shape
+    ho, wo = (h - 1) * s + k - 2 * p, (w - 1) * s + k - 2 * p
+    g = graph("deconv2")
+    g.ext("X", shape); g.ext("Wt", (c, k, k, cout), kind="weight"); g.ext("R", (n, ho, wo, cout))
+    t = g.add("Relu", [g.add("ConvTranspose", ["X", "Wt"], kernel=k, stride=s, pad=p)])
+    g.mark_output(g.add("Add", [t, "R"]))
+    ins = {"X": rnd(shape, 73), "Wt": rnd((c, k, k, cout), 74, -0.3, 0.3), "R": rnd((n, ho, wo, cout), 75)}
+    sess = check(W.Workload(g, ins), 2e-5, flags)
+    assert sess.g.tensor_info(sess.ids[g.outputs[0]])[1] == (n, ho, wo, cout)
+    if flags == B.PLAN_FUSED:
+        assert sess.plan_stats.n_ops == 3 and [b["ops"] for b in sess.g.blocks()][-1] == ["Col2Im", "Relu", "Add"]

@@ -728,3 +728,23 @@ def test_einsum_is_recorded_as_a_batched_matrix_product_between_index_operators(
 def build_graph_with(g, eq):
     g.add("Einsum", ["A", "Bm"], equation=eq)
     return build_graph(g)
+
+
+def test_convtranspose_with_overlap_is_recorded_as_patches_plus_gather():
+    g = _desc(); g.ext("X", (2, 8, 8, 16)); g.ext("Wt", (16, 4, 4, 8), kind="weight")
+    y = g.add("ConvTranspose", ["X", "Wt"], kernel=4, stride=2, pad=1)
+    g.mark_output(g.add("Relu", [y]))
+    G, ids, st = _plan_desc(g)
+    assert G.tensor_info(ids[y])[1] == (2, 16, 16, 8)
+    assert [b["ops"] for b in G.blocks() if b["family"] != "alias"] == [["Conv1x1"], ["Col2Im", "Relu"]]
+    assert st.n_ops == 2 and G.blocks()[-1]["family"] == "pool" and G.blocks()[-1]["mapping"] == "Many-to-Many"
+    # stride = kernel without padding stays the index-only form; bad strides and pads are refused
+    g = _desc(); g.ext("X", (2, 8, 8, 16)); g.ext("Wt", (16, 2, 2, 8), kind="weight")
+    g.mark_output(g.add("ConvTranspose", ["X", "Wt"], kernel=2, stride=2))
+    G, ids, st = _plan_desc(g)
+    assert "Col2Im" not in [k for b in G.blocks() for k in b["ops"]]
+    for at in (dict(kernel=2, stride=3), dict(kernel=2, stride=0), dict(kernel=3, stride=1, pad=3), dict(kernel=3, stride=1, pad=-1)):
+        g = _desc(); g.ext("X", (2, 8, 8, 16)); g.ext("Wt", (16, at["kernel"], at["kernel"], 8), kind="weight")
+        g.add("ConvTranspose", ["X", "Wt"], **at)
+        with pytest.raises(B.DnnfError):
+            _plan_desc(g)

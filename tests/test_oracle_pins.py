@@ -238,6 +238,29 @@ def test_convtranspose_bruteforce_and_pointwise_case():
         assert np.max(np.abs(y - ref)) < 1e-14
     w1 = rnd((3, 1, 1, 5), 43)
     assert np.allclose(O.op_convtranspose(x, w1, 1), O.op_conv1x1(x, w1[:, 0, 0, :]), atol=1e-14)
+    # padding cuts the border: the gather form, written as index loops over the OUTPUT (kernel 4, stride 2, pad 1: the
+    # result is exactly twice the input's size), and kernel 3, stride 2, pad 1
+    for k, s, p in ((4, 2, 1), (3, 2, 1), (3, 1, 1)):
+        w = rnd((3, k, k, 2), 44 + k)
+        y = O.op_convtranspose(x, w, s, p)
+        ho, wo = (3 - 1) * s + k - 2 * p, (4 - 1) * s + k - 2 * p
+        assert y.shape == (2, ho, wo, 2)
+        ref = np.zeros_like(y)
+        for n, oh, ow, o in itertools.product(range(2), range(ho), range(wo), range(2)):
+            acc = 0.0
+            for i, j in itertools.product(range(k), range(k)):
+                if (oh + p - i) % s or (ow + p - j) % s:
+                    continue
+                h, ww = (oh + p - i) // s, (ow + p - j) // s
+                if 0 <= h < 3 and 0 <= ww < 4:
+                    acc += sum(x[n, h, ww, c] * w[c, i, j, o] for c in range(3))
+            ref[n, oh, ow, o] = acc
+        assert np.max(np.abs(y - ref)) < 1e-13
+    assert O.op_convtranspose(x, rnd((3, 4, 4, 2), 50), 2, 1).shape == (2, 6, 8, 2)
+    # stride 1, kernel 3, pad 1 is a same-size correlation with the flipped kernel: a delta input returns the flipped taps
+    d = np.zeros((1, 5, 5, 1)); d[0, 2, 2, 0] = 1.0
+    wk = rnd((1, 3, 3, 1), 51)
+    assert np.allclose(O.op_convtranspose(d, wk, 1, 1)[0, 1:4, 1:4, 0], wk[0, :, :, 0], atol=1e-15)
 
 
 def test_pooling_bruteforce_and_special_cases():
