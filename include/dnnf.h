@@ -133,9 +133,8 @@ typedef enum {
   DNNF_OP_CUMSUM,                                   /* Many-to-Many (Table 2); running sum along the last axis (attribute AXIS must name it);
                                                        attributes EXCLUSIVE (sum of the elements before) and REVERSE (from the far end) */
   DNNF_OP_INSTANCENORM,                             /* Many-to-Many (Table 2); (x NHWC, scale[C], shift[C]), attribute EPS: each image and
-                                                       channel is normalised by the mean and biased variance over its H x W positions.
-                                                       Recorded as Transpose -> Reshape [N,C,HW] -> LayerNorm (no scale / shift) ->
-                                                       Reshape -> Transpose -> ScaleShift, which it equals term by term */
+                                                       channel is normalised by the mean and biased variance over its H x W positions,
+                                                       then scaled and shifted per channel; C a multiple of 4 */
   DNNF_OP_EINSUM,                                   /* Many-to-Many (Table 2); two operands, attributes LABELS_A, LABELS_B, LABELS_OUT: one small
                                                        integer per axis (the letters of "bhqd,bhkd->bhqk").  Every label of the result comes
                                                        from an operand, a label of both operands that is missing in the result is summed
@@ -241,6 +240,7 @@ typedef enum {
   DNNF_FAMILY_POOL = 7,        /* fp32 MaxPool / AveragePool with an epilogue chain */
   DNNF_FAMILY_GATHER = 8,      /* row gather by an index tensor */
   DNNF_FAMILY_ATTENTION = 9,   /* scores, softmax and weighted sum of a head in one kernel (DNNF_PLAN_BEYOND_TABLE3 only) */
+  DNNF_FAMILY_INSTNORM = 11,   /* fp32 InstanceNormalization with an epilogue chain */
   DNNF_FAMILY_MBCONV = 10      /* pointwise expansion, depthwise 3x3 and pointwise projection of an inverted-residual block in one
                                   kernel, the expanded tensor kept in shared memory (DNNF_PLAN_BEYOND_TABLE3 only) */
 } dnnf_family_t;

@@ -26,7 +26,7 @@ INPUT, WEIGHT = 0, 1
 ONE_TO_ONE, REORGANIZE, SHUFFLE, ONE_TO_MANY, MANY_TO_MANY = range(5)
 GREEN, YELLOW, RED = range(3)
 MAPPING_NAMES = ["One-to-One", "Reorganize", "Shuffle", "One-to-Many", "Many-to-Many"]
-FAMILY_NAMES = ["alias", "elementwise", "transpose", "row", "gemm", "conv1x1", "dwconv", "pool", "gather", "attention", "mbconv"]
+FAMILY_NAMES = ["alias", "elementwise", "transpose", "row", "gemm", "conv1x1", "dwconv", "pool", "gather", "attention", "mbconv", "instnorm"]
 
 OP_NAMES = ["?", "Add", "Sub", "Mul", "Div", "MulC", "AddC", "Sigmoid", "Tanh", "Erf", "Exp", "Log", "Sqrt", "Abs",
             "Neg", "Recip", "Square", "Relu", "Clip", "Pow", "Gelu", "ScaleShift", "Transpose", "Reshape", "Flatten",

@@ -316,34 +316,6 @@ int dnnf_add_op(dnnf_graph* g, int op_kind, int n_in, const int* in_ids, const d
     }
     if (rc) { rollback(); G.err = err; return rc; }
     outs = {cur};
-  } else if (op_kind == DNNF_OP_INSTANCENORM) {
-    // Per (image, channel) statistics over the H x W positions: in the channels-first view [N, C, H*W] that is a
-    // normalisation of each row, so the operator is recorded as the index operators that give that view around a
-    // LayerNorm without scale and shift, and the per-channel scale and shift as a ScaleShift on the NHWC result.
-    if (n_in != 3) return fail(g, DNNF_ERR_INVALID_ARG, "InstanceNorm takes (x, scale, shift)");
-    const std::vector<int64_t> xd = G.tensors[in_ids[0]].dims;
-    if (xd.size() != 4) return fail(g, DNNF_ERR_SHAPE, "InstanceNorm takes an NHWC tensor");
-    if (G.tensors[in_ids[1]].numel() != xd[3] || G.tensors[in_ids[2]].numel() != xd[3]) return fail(g, DNNF_ERR_SHAPE, "InstanceNorm: parameter length");
-    int cur = in_ids[0];
-    auto emit = [&](int kind, std::vector<int> ins, const Attrs& a) -> int {
-      Op o; o.id = (int)G.ops.size(); o.kind = kind; o.source_id = source; o.in = ins; o.at = a;
-      int r = infer_shapes(G, o, err);
-      if (r) return r;
-      cur = o.out[0];
-      G.ops.push_back(o);
-      return DNNF_OK;
-    };
-    Attrs a1, a2, a3, a4, a5, a6;
-    a1.perm = {0, 3, 1, 2}; a2.shape = {xd[0], xd[3], xd[1] * xd[2]}; a3.axis = -1; a3.eps = at.eps;
-    a4.shape = {xd[0], xd[3], xd[1], xd[2]}; a5.perm = {0, 2, 3, 1}; a6.axis = 3;
-    rc = emit(DNNF_OP_TRANSPOSE, {cur}, a1);
-    if (!rc) rc = emit(DNNF_OP_RESHAPE, {cur}, a2);
-    if (!rc) rc = emit(DNNF_OP_LAYERNORM, {cur}, a3);
-    if (!rc) rc = emit(DNNF_OP_RESHAPE, {cur}, a4);
-    if (!rc) rc = emit(DNNF_OP_TRANSPOSE, {cur}, a5);
-    if (!rc) rc = emit(DNNF_OP_SCALESHIFT, {cur, in_ids[1], in_ids[2]}, a6);
-    if (rc) { rollback(); G.err = err; return rc; }
-    outs = {cur};
   } else if (op_kind == DNNF_OP_DEPTHTOSPACE || op_kind == DNNF_OP_SPACETODEPTH || op_kind == DNNF_OP_RESIZE) {
     // Index maps of an NHWC tensor, recorded as the Reorganize / Shuffle / One-to-Many operators they consist of.
     const Tensor& X = G.tensors[in_ids[0]];

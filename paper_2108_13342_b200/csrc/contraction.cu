@@ -53,6 +53,9 @@ int lower_gather(const Graph& g, const std::vector<int>& ops, int anchor, Block&
 int gather_launch(const Launch& L, cudaStream_t st);
 void gather_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
 int lower_pool(const Graph& g, const std::vector<int>& ops, int anchor, Block& out, std::string& why);
+int lower_instnorm(const Graph& g, const std::vector<int>& ops, int anchor, Block& out, std::string& why);
+int instnorm_launch(const Launch& L, cudaStream_t st);
+void instnorm_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
 int pool_launch(const Launch& L, void* ws_base, cudaStream_t st);
 void pool_patch(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op);
 
@@ -269,6 +272,7 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
   const Op& A = g.ops[anchor];
   if (A.kind == DNNF_OP_DWCONV3X3) return lower_dwconv(g, ops, anchor, out, why);
   if (A.kind == DNNF_OP_MAXPOOL || A.kind == DNNF_OP_AVGPOOL || A.kind == DNNF_OP_COL2IM) return lower_pool(g, ops, anchor, out, why);
+  if (A.kind == DNNF_OP_INSTANCENORM) return lower_instnorm(g, ops, anchor, out, why);
   if (A.kind == DNNF_OP_GATHER) return lower_gather(g, ops, anchor, out, why);
   std::set<int> in_block(ops.begin(), ops.end());
   const Tensor& C = g.tensors[A.out[0]];
@@ -495,6 +499,7 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
 void patch_contraction(Launch& L, const std::vector<void*>& ip, const std::vector<void*>& op, std::string& err) {
   if (L.family == DNNF_FAMILY_DWCONV) { dwconv_patch(L, ip, op, err); return; }
   if (L.family == DNNF_FAMILY_POOL) { pool_patch(L, ip, op); return; }
+  if (L.family == DNNF_FAMILY_INSTNORM) { instnorm_patch(L, ip, op); return; }
   if (L.family == DNNF_FAMILY_GATHER) { gather_patch(L, ip, op); return; }
   if (L.family == DNNF_FAMILY_MBCONV) { mbconv_patch(L, ip, op); return; }
   if (L.family == DNNF_FAMILY_ATTENTION) { attention_patch(L, ip, op, err); if (!L.tc_ready && err.empty()) err = "cannot encode the tensor maps of an attention block"; return; }
@@ -519,6 +524,7 @@ int launch_contraction(const Launch& L, void* status_words, int block_index, cud
   if (L.family == DNNF_FAMILY_ATTENTION) { int rc = attention_launch(L, status_words, block_index, st); if (rc) err = "attention launch failed"; return rc; }
   if (L.family == DNNF_FAMILY_GATHER) { int rc = gather_launch(L, st); if (rc) err = "gather launch failed"; return rc; }
   if (L.family == DNNF_FAMILY_POOL) { int rc = pool_launch(L, status_words, st); if (rc) err = "pooling launch failed"; return rc; }
+  if (L.family == DNNF_FAMILY_INSTNORM) { int rc = instnorm_launch(L, st); if (rc) err = "instance normalisation launch failed"; return rc; }
   if (L.family == DNNF_FAMILY_DWCONV) { int rc = dwconv_launch(L, status_words, block_index, st); if (rc) err = "depthwise convolution launch failed"; return rc; }
   if (L.variant == 2) { int rc = conv1x1_direct_launch(L, st); if (rc) err = "pointwise convolution launch failed"; return rc; }
   if ((L.variant == 1 || L.variant == 3 || L.variant == 4 || L.variant == 5) && !L.tc_ready) { err = "tensor maps of the block are not encoded"; return 1; }

@@ -198,6 +198,50 @@ struct RowEpiIO {
   __device__ __forceinline__ void row_reduce(int, float (&)[VV]) const {}
 };
 
+// The same for a result of at most 8 columns (a convolution onto a few channels): the chain runs on 8 values per row
+// instead of 32, of which 24 would be padding.
+struct RowEpiIO8 {
+  static constexpr int VV = 8;
+  const GemmParams& p;
+  const Params& q;
+  float accv[8];
+  uint8_t* chunk;
+  const float* vec_s;
+  uint32_t row;
+  bool row_ok;
+  int lane;
+  __device__ __forceinline__ void load(int idx, float (&dst)[VV]) const {
+    const int slot = q.slot[idx];
+    if (slot >= 0) {
+      const float* s = vec_s + slot * kVecFloats;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        float4 w = *reinterpret_cast<const float4*>(s + 4 * j);
+        dst[4 * j] = w.x; dst[4 * j + 1] = w.y; dst[4 * j + 2] = w.z; dst[4 * j + 3] = w.w;
+      }
+      return;
+    }
+    const TensorArg& a = p.in[idx];
+    const float* src = reinterpret_cast<const float*>(a.ptr) + a.base + (int64_t)row * a.stride[1];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      float4 w = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (row_ok && 4 * j < p.N) w = __ldg(reinterpret_cast<const float4*>(src + 4 * j));
+      dst[4 * j] = w.x; dst[4 * j + 1] = w.y; dst[4 * j + 2] = w.z; dst[4 * j + 3] = w.w;
+    }
+  }
+  __device__ __forceinline__ void anchor(float (&dst)[VV]) const {
+#pragma unroll
+    for (int v = 0; v < VV; ++v) dst[v] = accv[v];
+  }
+  __device__ __forceinline__ void store(int, const float (&val)[VV]) const {
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+      *reinterpret_cast<float4*>(chunk + lane * 128 + ((j ^ (lane & 7)) << 4)) = make_float4(val[4 * j], val[4 * j + 1], val[4 * j + 2], val[4 * j + 3]);
+  }
+  __device__ __forceinline__ void row_reduce(int, float (&)[VV]) const {}
+};
+
 // byte offset of element (row, k) inside a K-major, 128-byte-swizzled image whose 32-wide K atoms
 // are `atom_bytes` apart
 __device__ __forceinline__ uint32_t sw128_offset(uint32_t row, uint32_t k, uint32_t atom_bytes) {
@@ -428,6 +472,23 @@ gemm_tf32_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ P
         __syncwarp(); if (warp == 2 && lane == 0) FACC(14, clock64() - t0); }
         uint8_t* my_chunks = epi + (size_t)(warp - 2) * q.chunks_per_warp * kChunkBytes;
         int slot = 0;
+        if (p.N <= 8) {                                   // one narrow chunk (cgroup 0 only: four epilogue warps)
+          RowEpiIO8 io8{p, q};
+          io8.lane = lane; io8.vec_s = vec_s; io8.row_ok = io.row_ok; io8.row = io.row;
+          uint32_t raw[8];
+          tc_ld8_issue(t_row, raw);
+          tc_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) io8.accv[j] = __uint_as_float(raw[j]);
+          for (int r = 1; r < nranges; ++r) {
+            tc_ld8_issue(t_row + r * NP, raw);
+            tc_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) io8.accv[j] += __uint_as_float(raw[j]);
+          }
+          io8.chunk = my_chunks;
+          run_program<8, SP, false>(p.prog, io8);
+        } else
         for (int c = cgroup * 32; c < p.N; c += cstep, ++slot) {
           uint32_t raw[32];
           const long long t0 = clock64();

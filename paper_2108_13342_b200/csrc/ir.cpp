@@ -81,7 +81,7 @@ bool is_row_anchor(int k) {
   return k == DNNF_OP_SOFTMAX || k == DNNF_OP_LAYERNORM || (k >= DNNF_OP_REDUCESUM && k <= DNNF_OP_REDUCEPROD) || k == DNNF_OP_CUMSUM;
 }
 bool is_contraction(int k) {      // anchors that take an epilogue chain and nothing in front
-  return k == DNNF_OP_MATMUL || k == DNNF_OP_CONV1X1 || k == DNNF_OP_DWCONV3X3 || k == DNNF_OP_MAXPOOL || k == DNNF_OP_AVGPOOL || k == DNNF_OP_COL2IM ||
+  return k == DNNF_OP_MATMUL || k == DNNF_OP_CONV1X1 || k == DNNF_OP_DWCONV3X3 || k == DNNF_OP_MAXPOOL || k == DNNF_OP_AVGPOOL || k == DNNF_OP_COL2IM || k == DNNF_OP_INSTANCENORM ||
          k == DNNF_OP_GATHER;
 }
 
@@ -115,7 +115,7 @@ int edge_mapping(const Graph& g, const Op& op, int slot) {
   if (is_broadcasting_elementwise(k))
     return same_shape(in, out) ? DNNF_ONE_TO_ONE : DNNF_ONE_TO_MANY;     // "elementwise w/ broadcast"
   if (k == DNNF_OP_SCALESHIFT) return slot == 0 ? DNNF_ONE_TO_ONE : DNNF_ONE_TO_MANY;
-  if (k == DNNF_OP_LAYERNORM) return slot == 0 ? DNNF_MANY_TO_MANY : DNNF_ONE_TO_MANY;
+  if (k == DNNF_OP_LAYERNORM || k == DNNF_OP_INSTANCENORM) return slot == 0 ? DNNF_MANY_TO_MANY : DNNF_ONE_TO_MANY;
   return node_mapping(g, op);
 }
 
@@ -135,7 +135,7 @@ int node_mapping(const Graph& g, const Op& op) {
     case DNNF_OP_EXPAND: case DNNF_OP_GATHER: return DNNF_ONE_TO_MANY;
     case DNNF_OP_MATMUL: case DNNF_OP_CONV1X1: case DNNF_OP_DWCONV3X3: case DNNF_OP_SOFTMAX: case DNNF_OP_LAYERNORM:
     case DNNF_OP_REDUCESUM: case DNNF_OP_REDUCEMEAN: case DNNF_OP_REDUCEMAX: case DNNF_OP_REDUCEPROD:
-    case DNNF_OP_MAXPOOL: case DNNF_OP_AVGPOOL: case DNNF_OP_CUMSUM: case DNNF_OP_COL2IM:
+    case DNNF_OP_MAXPOOL: case DNNF_OP_AVGPOOL: case DNNF_OP_CUMSUM: case DNNF_OP_COL2IM: case DNNF_OP_INSTANCENORM:
       return DNNF_MANY_TO_MANY;
     default: return DNNF_ONE_TO_ONE;
   }
@@ -296,6 +296,11 @@ int infer_shapes(Graph& g, Op& op, std::string& err) {
     d[1] = (d[1] + 2 * pd - kk) / st + 1;
     d[2] = (d[2] + 2 * pd - kk) / st + 1;
     outs.push_back(d);
+  } else if (k == DNNF_OP_INSTANCENORM) {
+    if (!need(3)) return DNNF_ERR_INVALID_ARG;
+    if (in(0).dims.size() != 4) { err = "InstanceNorm takes an NHWC tensor"; return DNNF_ERR_SHAPE; }
+    if (in(1).numel() != in(0).dims[3] || in(2).numel() != in(0).dims[3]) { err = "InstanceNorm: parameter length"; return DNNF_ERR_SHAPE; }
+    outs.push_back(in(0).dims);
   } else if (k == DNNF_OP_COL2IM) {
     if (!need(1)) return DNNF_ERR_INVALID_ARG;
     const int64_t kk = op.at.kernel, st = op.at.stride, pd = op.at.pad;

@@ -36,7 +36,7 @@ int64_t op_flops(const Graph& g, const Op& o) {
   if (is_index_only(o.kind)) return 0;
   if (o.kind >= DNNF_OP_REDUCESUM && o.kind <= DNNF_OP_REDUCEPROD) return g.tensors[o.in[0]].numel();
   if (o.kind == DNNF_OP_SOFTMAX) return 5 * g.tensors[o.in[0]].numel();
-  if (o.kind == DNNF_OP_LAYERNORM) return 7 * g.tensors[o.in[0]].numel();
+  if (o.kind == DNNF_OP_LAYERNORM || o.kind == DNNF_OP_INSTANCENORM) return 7 * g.tensors[o.in[0]].numel();
   if (o.kind == DNNF_OP_MATMUL) { const Tensor& a = g.tensors[o.in[0]]; return 2 * g.tensors[o.out[0]].numel() * a.dims.back(); }
   if (o.kind == DNNF_OP_CONV1X1) return 2 * g.tensors[o.out[0]].numel() * g.tensors[o.in[1]].dims[0];
   if (o.kind == DNNF_OP_DWCONV3X3) return 18 * g.tensors[o.out[0]].numel();

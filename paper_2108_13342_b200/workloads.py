@@ -391,6 +391,42 @@ def mbconv_stack(n=32, hw=56, seed=BASE_SEED, layout="nhwc") -> Workload:
     return Workload(g, ins, note="fp32 " + layout.upper())
 
 
+def style_decoder(n=8, hw=64, c=64, seed=BASE_SEED) -> Workload:
+    """The decoder half of a style-transfer / image-to-image generator in NHWC fp32: a residual block (pointwise
+    convolution, instance normalisation, ReLU, depthwise 3x3, instance normalisation, skip), two transposed
+    convolutions with overlapping patches (kernel 4, stride 2, pad 1: each doubles the image) with instance
+    normalisation and ReLU, and a pointwise convolution to 4 output channels with Tanh.  Synthetic shapes in the range of
+    the paper's image-to-image models (Section 5); it exercises InstanceNormalization and ConvTranspose at sizes where
+    they dominate."""
+    d = _Draw(seed + 13)
+    g = GraphDesc("style_decoder")
+    ins = {}
+    cnt = [0]
+
+    def ext(shape, lo=None, hi=None, std=None, name=None):
+        cnt[0] += 1
+        name = name or "p%d" % cnt[0]
+        g.ext(name, shape, kind="input" if name == "X" else "weight")
+        ins[name] = d.normal(shape, 0.0, std) if std is not None else d.uniform(shape, lo, hi)
+        return name
+
+    def inorm(x, ch):
+        return g.add("InstanceNorm", [x, ext((ch,), 0.5, 1.5), ext((ch,), -0.5, 0.5)], eps=1e-5)
+
+    x = ext((n, hw, hw, c), -1.0, 1.0, name="X")
+    y = g.add("Relu", [inorm(g.add("Conv1x1", [x, ext((c, c), std=math.sqrt(2.0 / c))]), c)])
+    y = inorm(g.add("DwConv3x3", [y, ext((3, 3, c), std=math.sqrt(2.0 / 9.0))]), c)
+    y = g.add("Add", [y, x])
+    ch = c
+    for _ in range(2):
+        y = g.add("ConvTranspose", [y, ext((ch, 4, 4, ch // 2), std=math.sqrt(2.0 / (4 * ch)))], kernel=4, stride=2, pad=1)
+        ch //= 2
+        y = g.add("Relu", [inorm(y, ch)])
+    y = g.add("Tanh", [g.add("Add", [g.add("Conv1x1", [y, ext((ch, 4), std=math.sqrt(1.0 / ch))]), ext((4,), -0.1, 0.1)])], out="image")
+    g.mark_output(y)
+    return Workload(g, ins, note="fp32 NHWC")
+
+
 # --------------------------------------------------------------------------
 # Workload 5: transformer encoder as primitive operators (48 per layer)
 # --------------------------------------------------------------------------
@@ -558,5 +594,5 @@ def by_name(name: str, **kw) -> Workload:
     table = {"swish_transpose": swish_transpose, "masked_softmax": masked_softmax,
              "add_layernorm_gelu": add_layernorm_gelu, "ffn_block": ffn_block,
              "mbconv_block": mbconv_block, "encoder": encoder, "decoder": decoder, "cnn_neck": cnn_neck,
-             "mbconv_stack": mbconv_stack}
+             "mbconv_stack": mbconv_stack, "style_decoder": style_decoder}
     return table[name](**kw)

@@ -45,3 +45,16 @@ def test_decoder_twelve_layers_every_block(flags, rewrite):
     """The full-size GPT-2 style decoder (12 layers, 633 primitive operators)."""
     checked, skipped = check_blocks(W.decoder(), flags, rewrite, min_checked=60)
     print("decoder: blocks checked", checked, "skipped", skipped)
+
+
+@pytest.mark.parametrize("flags", [B.PLAN_FUSED, B.PLAN_UNFUSED])
+def test_style_transfer_decoder_blocks(flags):
+    """Instance normalisation, overlapping transposed convolutions (pointwise convolution onto the patch values + gather),
+    depthwise convolution: every block at the single-block tolerance."""
+    checked, skipped = check_blocks(W.style_decoder(n=4, hw=32, c=64), flags, min_checked=6)
+    print("style decoder: blocks checked", checked, "skipped", skipped)
+
+
+def test_channels_first_stack_blocks_after_layout_selection():
+    checked, skipped = check_blocks(W.mbconv_stack(n=4, hw=48, layout="nchw"), B.PLAN_FUSED, B.REWRITE_DEFAULT, min_checked=20)
+    print("channels-first stack: blocks checked", checked, "skipped", skipped)

@@ -481,3 +481,25 @@ def test_convtranspose_with_overlapping_patches(shape, k, s, p, cout, flags):
     assert sess.g.tensor_info(sess.ids[g.outputs[0]])[1] == (n, ho, wo, cout)
     if flags == B.PLAN_FUSED:
         assert sess.plan_stats.n_ops == 3 and [b["ops"] for b in sess.g.blocks()][-1] == ["Col2Im", "Relu", "Add"]
+
+
+@pytest.mark.parametrize("shape", [(1, 64, 64, 128), (16, 20, 20, 8), (2, 33, 17, 36), (300, 4, 4, 64)])
+def test_instance_normalization_channel_group_widths(shape):
+    """One image with many channels, many images with few, a channel count that leaves a narrow last group, many small
+    planes: the CTA's channel group goes from one to eight 128-bit lanes; a residual and an activation ride in the epilogue."""
+    c = shape[3]
+    g = graph(); g.ext("X", shape); g.ext("s", (c,), kind="weight"); g.ext("t", (c,), kind="weight"); g.ext("R", shape)
+    g.mark_output(g.add("LeakyRelu", [g.add("Add", [g.add("InstanceNorm", ["X", "s", "t"], eps=1e-3), "R"])], alpha=0.2))
+    ins = {"X": rnd(shape, 12, -1.0, 5.0), "s": rnd((c,), 13, 0.5, 1.5), "t": rnd((c,), 14, -0.5, 0.5), "R": rnd(shape, 15)}
+    s = check(W.Workload(g, ins), RTOL_F32, expect_blocks=1)
+    assert s.g.blocks()[0]["family"] == "instnorm"
+
+
+@pytest.mark.parametrize("flags", [B.PLAN_FUSED, B.PLAN_UNFUSED])
+def test_style_transfer_decoder(flags):
+    """Residual block with instance normalisation, two overlapping transposed convolutions, Tanh head."""
+    wl = W.style_decoder(n=2, hw=24, c=32)
+    s = check(wl, 2e-4, flags)
+    if flags == B.PLAN_FUSED:
+        fams = [b["family"] for b in s.g.blocks() if b["family"] != "alias"]
+        assert fams.count("instnorm") == 4 and fams.count("pool") == 2 and s.plan_stats.n_kernels == 11, s.g.blocks()

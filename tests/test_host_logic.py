@@ -667,13 +667,12 @@ def test_where_cast_cumsum_instancenorm_recording_types_and_plans():
     g.mark_output(g.add("Where", ["C", "A", "Bv"]))
     G, ids, st = _plan_desc(g)
     assert G.op_mapping(0) == OO and G.block_program(0) == "MOV in0; SAVE t0; MOV in1; SELECT in2; STORE out0"
-    # InstanceNormalization is recorded as its channels-first row normalisation between index operators
-    g = _desc(); g.ext("X", (2, 6, 6, 8)); g.ext("s", (8,), kind="weight"); g.ext("t", (8,), kind="weight")
-    g.mark_output(g.add("Relu", [g.add("InstanceNorm", ["X", "s", "t"], eps=1e-5)]))
+    # InstanceNormalization is a Many-to-Many anchor of its own: One-to-One successors ride in its epilogue, nothing in front
+    g = _desc(); g.ext("X", (2, 6, 6, 8)); g.ext("s", (8,), kind="weight"); g.ext("t", (8,), kind="weight"); g.ext("R", (2, 6, 6, 8))
+    g.mark_output(g.add("Add", [g.add("Relu", [g.add("InstanceNorm", [g.add("Tanh", ["X"]), "s", "t"], eps=1e-5)]), "R"]))
     G, ids, st = _plan_desc(g)
-    kinds = [k for b in G.blocks() for k in b["ops"]]
-    assert sorted(kinds) == sorted(["Transpose", "Reshape", "LayerNorm", "Reshape", "Transpose", "ScaleShift", "Relu"])
-    assert st.n_ops == 2 and any(b["family"] == "row" for b in G.blocks())
+    assert [(b["family"], b["ops"]) for b in G.blocks()] == [("elementwise", ["Tanh"]), ("instnorm", ["InstanceNorm", "Relu", "Add"])]
+    assert G.op_mapping(1) == MM and st.n_ops == 4 and st.n_kernels == 2
     # errors
     for op, ins, at in [("Where", ["X", "s"], {}), ("Cast", ["X"], dict(to=7)), ("CumSum", ["X"], dict(axis=1)),
                         ("InstanceNorm", ["X", "s"], {}), ("InstanceNorm", ["s", "s", "t"], {})]:
