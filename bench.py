@@ -348,7 +348,8 @@ def main():
         detail = report.per_config(dev, pk)
         for name, fn in [("cfg5 12-layer encoder (576 primitive operators)", report.encoder_report),
                          ("next: 12-layer GPT-2 style decoder (633 primitive operators)", report.decoder_report),
-                         ("next: layout selection on the MobileNetV2-shaped stack written channels-first", report.layout_report)]:
+                         ("next: layout selection on the MobileNetV2-shaped stack written channels-first", report.layout_report),
+                         ("beyond Table 3: the inverted-residual block as one kernel", report.mbconv_single_kernel_report)]:
             try:
                 detail[name] = fn(dev, pk)
             except Exception as e:  # noqa: BLE001

@@ -271,16 +271,9 @@ __global__ void __launch_bounds__(THREADS, 1) mbconv_kernel(const __grid_constan
   cp_async_wait_all();
   __syncthreads();
 
-#ifdef DNNF_MB_TRACE
-  long long tc[6] = {0, 0, 0, 0, 0, 0}; long long tq = clock64();
-#define MBT(i) do { long long now_ = clock64(); tc[i] += now_ - tq; tq = now_; } while (0)
-#else
-#define MBT(i) do {} while (0)
-#endif
   for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
     const int n = tile / tiles_per_image, tr = tile - n * tiles_per_image;
     const int h0 = (tr / p.tiles_w) * TH, w0 = (tr % p.tiles_w) * TW;
-    MBT(0);
 
     // ---- stage 1: expansion of the halo tile; a unit is 16 halo pixels x 24 channels ----
     for (int unit = warp; unit < M1 * (NT1 / 3); unit += WARPS) {
@@ -335,8 +328,6 @@ __global__ void __launch_bounds__(THREADS, 1) mbconv_kernel(const __grid_constan
       }
     }
     __syncthreads();
-
-    MBT(1);
     // The halo tile of X is consumed: the next tile's copy starts now and lands while stages 2 and 3 run.
     if (tile + (int)gridDim.x < p.total_tiles) load_x(tile + gridDim.x);
     cp_async_commit();
@@ -435,7 +426,6 @@ __global__ void __launch_bounds__(THREADS, 1) mbconv_kernel(const __grid_constan
         }
       }
     }
-    MBT(2);
     __syncthreads();                       // every warp is done with the expanded tile: its place takes the partial sums
     float* part = es;                      // [pixel group][quarter][2 NT3 x 4 values][32 lanes]
     constexpr int kVals = 2 * NT3 * 4, kFrags = 2 * NT3;
@@ -449,7 +439,6 @@ __global__ void __launch_bounds__(THREADS, 1) mbconv_kernel(const __grid_constan
           for (int v = 0; v < 4; ++v) r[((u * NT3 + j) * 4 + v) * 32] = acc3[u][j][v];
     }
     __syncthreads();
-    MBT(3);
     {
       // the group's fragments are shared out over its four warps: each adds the four partial sums of its fragments
       // (always in the same order) and runs the last chain on them
@@ -471,15 +460,9 @@ __global__ void __launch_bounds__(THREADS, 1) mbconv_kernel(const __grid_constan
         else run_program<4, SP3>(p.prog3, io3);
       }
     }
-    MBT(4);
     cp_async_wait_all();
     __syncthreads();                       // the partial sums are read, the next halo tile of X has landed
-    MBT(5);
   }
-#ifdef DNNF_MB_TRACE
-  if (blockIdx.x == 0 && (threadIdx.x == 0 || threadIdx.x == 33))
-    printf("mb trace t%d: head %lld expand+sync %lld dw+proj %lld sync %lld epi %lld wait+sync %lld\n", threadIdx.x, tc[0], tc[1], tc[2], tc[3], tc[4], tc[5]);
-#endif
 }
 
 #define MO(o, s, i) MicroOp{o, s, i, 0}

@@ -208,3 +208,19 @@ def layout_report(dev, pk):
         out[name] = {k: r[k] for k in ("ops", "kernels", "us_cuda_graph", "us_plain_launches", "irs_bytes")}
         torch.cuda.empty_cache()
     return out
+
+
+def mbconv_single_kernel_report(dev, pk):
+    """The inverted-residual block of configs[3] as three kernels (the paper's rules) and as one (beyond Table 3), from one
+    image to the full batch; the planner forms the single kernel only while its tiles fit one wave."""
+    import torch
+    out = {}
+    for n, hw in [(1, 14), (1, 56), (4, 28), (8, 56), (32, 56)]:
+        wl = W.mbconv_block(n, hw, hw)
+        a = measure_workload(torch, dev, wl, pk, B.PLAN_FUSED, 3, iters=20, per_block_limit=0)
+        b = measure_workload(torch, dev, wl, pk, B.PLAN_FUSED | B.PLAN_BEYOND_TABLE3 | B.PLAN_MBCONV_ALWAYS, 3, iters=20, per_block_limit=0)
+        c = measure_workload(torch, dev, wl, pk, B.PLAN_FUSED | B.PLAN_BEYOND_TABLE3, 3, iters=20, per_block_limit=0)
+        out["[%d,%d,%d,24->144->24]" % (n, hw, hw)] = {"three_kernels_us": a["us_cuda_graph"], "one_kernel_us": b["us_cuda_graph"],
+                                                        "planner_forms_it": c["kernels"] == 1}
+        torch.cuda.empty_cache()
+    return out
