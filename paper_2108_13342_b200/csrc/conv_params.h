@@ -39,6 +39,35 @@ struct DwIO {
   __device__ __forceinline__ void row_reduce(int, float (&)[4]) const {}
 };
 
+// P results of a kernel's own IO side by side: one pass of the chain serves 4 * P values, so an interpreted chain pays
+// its dispatch once per 4 * P values instead of once per 4 (and the P loads of an operand are in flight together).
+template <class IO, int P>
+struct BatchIO {
+  static constexpr int VV = 4 * P;
+  IO io[P];
+  bool on[P];
+  __device__ __forceinline__ void load(int idx, float (&dst)[VV]) const {
+#pragma unroll
+    for (int u = 0; u < P; ++u) {
+      float (&d)[4] = *reinterpret_cast<float (*)[4]>(&dst[4 * u]);
+      if (on[u]) io[u].load(idx, d);
+      else d[0] = d[1] = d[2] = d[3] = 0.0f;
+    }
+  }
+  __device__ __forceinline__ void anchor(float (&dst)[VV]) const {
+#pragma unroll
+    for (int u = 0; u < P; ++u)
+#pragma unroll
+      for (int v = 0; v < 4; ++v) dst[4 * u + v] = io[u].accv[v];
+  }
+  __device__ __forceinline__ void store(int idx, const float (&val)[VV]) const {
+#pragma unroll
+    for (int u = 0; u < P; ++u)
+      if (on[u]) io[u].store(idx, *reinterpret_cast<const float (*)[4]>(&val[4 * u]));
+  }
+  __device__ __forceinline__ void row_reduce(int, float (&)[VV]) const {}
+};
+
 #define MO(o, s, i) MicroOp{o, s, i, 0}
 DNNF_SP_BEGIN(CP_ScaleShiftClip, 5)
   MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_CLIP, S_CONST, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END

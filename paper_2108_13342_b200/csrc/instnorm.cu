@@ -92,20 +92,29 @@ __global__ void __launch_bounds__(kThreads) instnorm_kernel(const __grid_constan
   const float inv = 1.0f / (float)HW;
 
   float4 s = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+  const float4 zero4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
   if (live)
-    for (int q = q_begin + pr; q < q_end; q += prs) {
-      const float4 v = __ldg(reinterpret_cast<const float4*>(xb + (size_t)q * p.d.C));
-      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    for (int q = q_begin + pr; q < q_end; q += 4 * prs) {          // four loads in flight per thread
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[u] = q + u * prs < q_end ? __ldg(reinterpret_cast<const float4*>(xb + (size_t)(q + u * prs) * p.d.C)) : zero4;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
     }
   s = cluster_sum<kCluster>(plane_sum(s, lanes, xchg), cpart[0], lanes, split);
   const float4 mean = make_float4(s.x * inv, s.y * inv, s.z * inv, s.w * inv);
 
   float4 m2 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
   if (live)
-    for (int q = q_begin + pr; q < q_end; q += prs) {
-      const float4 v = __ldg(reinterpret_cast<const float4*>(xb + (size_t)q * p.d.C));
-      const float a = v.x - mean.x, b = v.y - mean.y, e = v.z - mean.z, f = v.w - mean.w;
-      m2.x = fmaf(a, a, m2.x); m2.y = fmaf(b, b, m2.y); m2.z = fmaf(e, e, m2.z); m2.w = fmaf(f, f, m2.w);
+    for (int q = q_begin + pr; q < q_end; q += 4 * prs) {
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[u] = q + u * prs < q_end ? __ldg(reinterpret_cast<const float4*>(xb + (size_t)(q + u * prs) * p.d.C)) : mean;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {                                 // (a pixel past the end was given the mean: deviation 0)
+        const float a = v[u].x - mean.x, b = v[u].y - mean.y, e = v[u].z - mean.z, f = v[u].w - mean.w;
+        m2.x = fmaf(a, a, m2.x); m2.y = fmaf(b, b, m2.y); m2.z = fmaf(e, e, m2.z); m2.w = fmaf(f, f, m2.w);
+      }
     }
   m2 = cluster_sum<kCluster>(plane_sum(m2, lanes, xchg), cpart[1], lanes, split);
   if (live) {
@@ -113,14 +122,25 @@ __global__ void __launch_bounds__(kThreads) instnorm_kernel(const __grid_constan
   // y = (x - mean) / sqrt(var + eps) * scale + shift
   const float4 g = make_float4(sc.x / sqrtf(m2.x * inv + p.eps), sc.y / sqrtf(m2.y * inv + p.eps), sc.z / sqrtf(m2.z * inv + p.eps),
                                sc.w / sqrtf(m2.w * inv + p.eps));
-  DwIO io{p.d};
-  io.n = n; io.c = c;
-  for (int q = q_begin + pr; q < q_end; q += prs) {
-    const float4 v = __ldg(reinterpret_cast<const float4*>(xb + (size_t)q * p.d.C));
-    io.accv[0] = fmaf(v.x - mean.x, g.x, sh.x); io.accv[1] = fmaf(v.y - mean.y, g.y, sh.y);
-    io.accv[2] = fmaf(v.z - mean.z, g.z, sh.z); io.accv[3] = fmaf(v.w - mean.w, g.w, sh.w);
-    io.h = q / p.d.W; io.w = q - io.h * p.d.W;
-    run_program<4, SP>(p.d.prog, io);
+  // four pixels per pass of the chain
+  BatchIO<DwIO, 4> b{{DwIO{p.d}, DwIO{p.d}, DwIO{p.d}, DwIO{p.d}}, {false, false, false, false}};
+  for (int q = q_begin + pr; q < q_end; q += 4 * prs) {
+    float4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int qq = q + u * prs;
+      b.on[u] = qq < q_end;
+      v[u] = b.on[u] ? __ldg(reinterpret_cast<const float4*>(xb + (size_t)qq * p.d.C)) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int qq = q + u * prs;
+      DwIO& io = b.io[u];
+      io.accv[0] = fmaf(v[u].x - mean.x, g.x, sh.x); io.accv[1] = fmaf(v[u].y - mean.y, g.y, sh.y);
+      io.accv[2] = fmaf(v[u].z - mean.z, g.z, sh.z); io.accv[3] = fmaf(v[u].w - mean.w, g.w, sh.w);
+      io.n = n; io.c = c; io.h = qq / p.d.W; io.w = qq - io.h * p.d.W;
+    }
+    run_program<16, SP>(p.d.prog, b);
   }
   }
   if (kCluster) cooperative_groups::this_cluster().sync();      // nobody leaves while its sums may still be read
