@@ -22,10 +22,12 @@ no step finds its data in L2.
             operators) fused against one kernel per operator, CUDA-graph replays
 
 `--detail` writes the per-configuration / per-block tables to
-gpurun_out/bench_detail.json.  `--impl reference` times the CPU oracle on the same
+bench_detail.json in the output folder (OUT_DIR below).  `--impl reference` times the CPU oracle on the same
 workload (bounded sample).
 """
 from __future__ import annotations
+
+OUT_DIR = "gpurun_out"      # where files that a run produces go
 
 import argparse
 import json
@@ -179,7 +181,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="dnnf")
-    ap.add_argument("--detail", action="store_true", help="also write per-configuration / per-block tables to gpurun_out/bench_detail.json")
+    ap.add_argument("--detail", action="store_true", help="also write per-configuration / per-block tables to bench_detail.json in the output folder")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-graph-latency", action="store_true", help="skip the encoder fused / unfused latency pair")
     args = ap.parse_args()
@@ -357,8 +359,8 @@ def main():
         detail["paper_context"] = {"note": "mobile-device figures from the paper, not comparable hardware",
                                    "fusion_rate_vs_other_frameworks": "up to 8.8x", "speedup_vs_other_frameworks": "up to 9.3x",
                                    "speedup_vs_own_unfused_backend": "1.5-5.8x"}
-        os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-        with open(os.path.join(ROOT, "gpurun_out", "bench_detail.json"), "w") as f:
+        os.makedirs(os.path.join(ROOT, OUT_DIR), exist_ok=True)
+        with open(os.path.join(ROOT, OUT_DIR, "bench_detail.json"), "w") as f:
             json.dump(detail, f, indent=1)
     if rank == 0:
         sys.stdout.flush()
