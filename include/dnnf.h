@@ -199,6 +199,7 @@ typedef struct {
 #define DNNF_PLAN_NO_SPLIT_K        0x2000u  /* bf16 GEMM blocks without a split over K */
 #define DNNF_PLAN_NO_TMA_DWCONV     0x4000u  /* depthwise convolutions without the TMA-tiled kernel */
 #define DNNF_PLAN_NO_TILE_GEMM      0x8000u  /* bf16 GEMM blocks without the one-tile-per-CTA kernel */
+#define DNNF_PLAN_NO_SMALL_CONV     0x40000u /* fp32 contractions with few rows without the one-tile-per-CTA mma.sync kernel */
 #define DNNF_PLAN_MBCONV_ALWAYS     0x20000u /* with DNNF_PLAN_BEYOND_TABLE3: form the single-kernel inverted-residual block whatever its
                                                 size (by default only while its 8 x 16 pixel tiles fit one wave of CTAs, where it was
                                                 measured faster than the three kernels; this flag changes the plan, not only a kernel) */

@@ -49,6 +49,7 @@ PLAN_FUSED, PLAN_UNFUSED, PLAN_STRICT_TABLE3, PLAN_ALLOW_PROLOGUE, PLAN_BEYOND_T
 PLAN_SPLIT_ALWAYS, PLAN_NO_K_SLICES, PLAN_NO_COLUMN_BLOCKS, PLAN_NO_TF32_GEMM = 0x100, 0x200, 0x400, 0x800
 PLAN_NO_PAIR_GEMM, PLAN_NO_SPLIT_K, PLAN_NO_TMA_DWCONV, PLAN_NO_TILE_GEMM = 0x1000, 0x2000, 0x4000, 0x8000
 PLAN_MBCONV_ALWAYS = 0x20000
+PLAN_NO_SMALL_CONV = 0x40000
 PLAN_CLUSTER_SPLIT_K = 0x10000
 STATIC_WS_BYTES = 32 << 20
 

