@@ -353,6 +353,9 @@ int lower_dwconv(const Graph& g, const std::vector<int>& ops, int anchor, Block&
   int hs = dp.H;
   int64_t threads_full = (int64_t)dp.N * dp.W * (dp.C / 4);
   while (hs > 7 && threads_full * ((dp.H + hs - 1) / hs) < 148 * 1024 * 4) hs = (hs + 1) / 2;
+  // a problem with fewer threads than one CTA per SM is a chain of dependent row loads per thread: shorter strips, at
+  // the price of reading the strips' halo rows again
+  while (hs > 2 && threads_full * ((dp.H + hs - 1) / hs) < (int64_t)sm_count() * 256) hs = (hs + 1) / 2;
   L.variant = hs;
   int64_t total = threads_full * ((dp.H + hs - 1) / hs);
   L.grid = (int)((total + 255) / 256);
