@@ -98,6 +98,7 @@ def per_config(dev, pk, only=None):
         ("cfg4 MBConv fp32 NHWC [32,56,56,24->144->24]", W.mbconv_block(), 2),
         ("next: CNN fragment with pooling, SpaceToDepth/DepthToSpace, Resize, Concat fp32 NHWC [32,64,64,32]", W.cnn_neck(n=32), 2),
         ("next: MobileNetV2-shaped stack of 9 inverted-residual blocks + head, fp32 NHWC [32,56,56,16] (84 operators)", W.mbconv_stack(), 1),
+        ("next: the same stack on ONE image [1,56,56,16] (the paper's operating point)", W.mbconv_stack(n=1), 4),
         ("next: style-transfer decoder with InstanceNormalization and overlapping ConvTranspose, fp32 NHWC [8,64,64,64] -> [8,256,256,4]", W.style_decoder(), 1),
     ]
     for name, wl, copies in cases:
