@@ -560,10 +560,14 @@ int lower_mbconv(const Graph& g, const std::vector<int>& ops, uint32_t flags, Bl
   if (total >= (1ll << 31)) return refuse("too many tiles");
   q.total_tiles = (int)total;
   // Measured (B200, CUDA-graph replays of the 24 -> 144 -> 24 block): one kernel against three is 15.1 against 21.7 us
-  // on one 56 x 56 image (28 tiles) and 14.6 against 38.2 us on a 14 x 14 image, but 30.1 against 26.8 us on 8 images
+  // on one 56 x 56 image (28 tiles; 17.3 against 20.4 us once the small-M pointwise kernel existed), but 30.1 against 26.8 us on 8 images
   // and 94.9 against 63.0 us on 32: once the tiles exceed one wave the kernel is bound by instruction issue and
   // shared-memory bandwidth (split-TF32 on warp-level instructions, the depthwise taps), the three kernels by HBM.
   if (total > sm_count() && !plan_flag(DNNF_PLAN_MBCONV_ALWAYS)) return refuse("more than one wave of tiles: the three kernels are faster");
+  // ... and below 16 tiles its set-up (both weight matrices into fragment order, once per CTA) is not paid back: one
+  // 14 x 14 image is 17.2 us against 11.5 us for the three kernels since the small-M pointwise kernel exists.
+  { const char* e = dev_env("DNNF_MB_MIN_TILES"); const int min_tiles = e ? atoi(e) : 16;
+    if (total < min_tiles && !plan_flag(DNNF_PLAN_MBCONV_ALWAYS)) return refuse("too few tiles to pay for the set-up: the three kernels are faster"); }
   q.prog1 = ga.prog; q.prog2 = db.prog; q.prog3 = gc.prog;
   q.n_in1 = ga.n_in; q.n_in2 = db.n_in; q.n_in3 = gc.n_in; q.n_out3 = gc.n_out;
   for (int i = 0; i < ga.n_in; ++i) q.in1[i] = ga.in[i];

@@ -153,6 +153,10 @@ def test_inverted_residual_block_full_size():
     assert "mbconv" not in _families(s)
     s = check(W.mbconv_block(n=1), RTOL_F32, BEYOND, expect_blocks=1)       # one image: 28 tiles
     assert _families(s) == ["mbconv"]
+    s = check(W.mbconv_block(n=1, h=14, w=14), RTOL_F32, BEYOND, expect_blocks=3)       # two tiles: not worth the set-up
+    assert "mbconv" not in _families(s)
+    s = check(W.mbconv_block(n=1, h=14, w=14), RTOL_F32, BEYOND | B.PLAN_MBCONV_ALWAYS, expect_blocks=1)
+    assert _families(s) == ["mbconv"]
 
 
 @pytest.mark.parametrize("cout,tail,act", [(32, "none", "clip"), (24, "relu", "relu"), (32, "two_outputs", "clip"), (24, "pixel_gate", "leaky")])
@@ -186,7 +190,7 @@ def test_inverted_residual_block_other_chains(cout, tail, act):
     elif tail == "pixel_gate":
         e = g.add("Mul", [g.add("Add", [e, "X"]), ext("P", (n, h, w, 1), 0.5, 1.5, 10, kind="input")])
     g.mark_output(e)
-    s = check(W.Workload(g, ins), RTOL_F32, BEYOND, expect_blocks=1)
+    s = check(W.Workload(g, ins), RTOL_F32, BEYOND | B.PLAN_MBCONV_ALWAYS, expect_blocks=1)       # (12 tiles: below the planner's own bar)
     assert _families(s) == ["mbconv"]
 
 

@@ -689,7 +689,7 @@ def test_beyond_table3_forms_the_single_kernel_inverted_residual_block_only_whil
         st = G.plan(flags)
         return [b["family"] for b in G.blocks()], st
     beyond = B.PLAN_FUSED | B.PLAN_BEYOND_TABLE3
-    small, full = W.mbconv_block(n=1, h=16, w=16), W.mbconv_block()
+    small, full = W.mbconv_block(n=1, h=56, w=56), W.mbconv_block()
     assert fams(small, B.PLAN_FUSED)[0] == ["conv1x1", "dwconv", "conv1x1"]          # Table 3: Many-to-Many + Many-to-Many is red
     f, st = fams(small, beyond)
     assert f == ["mbconv"] and st.n_kernels == 1 and st.n_ops == 9
