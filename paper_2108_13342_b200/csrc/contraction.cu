@@ -271,7 +271,8 @@ bool pack_operand(const Graph& g, const std::vector<int64_t>& orig_dims, const s
 }  // namespace
 
 // Up to this many rows an fp32 contraction goes to the one-tile-per-CTA kernel even where the tall-and-skinny tensor-core
-// kernel would take it: that kernel has one 128-row tile per CTA and nothing to spread over the GPU.
+// kernel would take it: that kernel has one 128-row tile per CTA and nothing to spread over the GPU.  (Where the
+// tensor-core kernel does not apply, the one-tile-per-CTA kernel is taken up to 65536 rows.)
 static int small_m_limit() { const char* e = dev_env("DNNF_SMALL_M"); return e ? atoi(e) : 1024; }
 
 int lower_contraction(const Graph& g, const std::vector<int>& ops, uint32_t flags, int anchor, Block& out, std::string& why) {
