@@ -78,8 +78,9 @@ DNNF_SP_BEGIN(CP_ScaleShiftClipResidual, 6)
   MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_CLIP, S_CONST, 0), MO(M_ADD, S_IN, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
 DNNF_SP_BEGIN(CP_Relu, 3) MO(M_MOV, S_ANCHOR, 0), MO(M_RELU, S_NONE, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
 DNNF_SP_BEGIN(CP_Residual, 3) MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+DNNF_SP_BEGIN(CP_ScaleShift, 4) MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_STORE, S_NONE, 0) DNNF_SP_END
 #undef MO
-using ConvStatic = TypeList<CP_ScaleShiftClip, CP_ScaleShiftResidual, CP_Store, CP_ScaleShiftClipResidual, CP_Relu, CP_Residual>;
+using ConvStatic = TypeList<CP_ScaleShiftClip, CP_ScaleShiftResidual, CP_Store, CP_ScaleShiftClipResidual, CP_Relu, CP_Residual, CP_ScaleShift>;
 
 
 }  // namespace dnnf

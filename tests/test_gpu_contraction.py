@@ -223,7 +223,7 @@ def test_conv1x1_with_epilogue(cfg):
 @pytest.mark.parametrize("cfg", [(2, 16, 16, 24, 144), (3, 19, 23, 144, 24), (1, 30, 31, 12, 20), (1, 40, 40, 36, 160), (4, 16, 16, 32, 192),
                                  (1, 33, 33, 100, 8), (2, 24, 24, 96, 48),
                                  (1, 29, 89, 32, 124), (1, 40, 40, 16, 100), (1, 40, 40, 16, 96)])
-@pytest.mark.parametrize("epi", ["clip", "residual", "none"])
+@pytest.mark.parametrize("epi", ["clip", "residual", "affine", "none"])
 def test_conv1x1_tensor_core_fp32(cfg, epi):
     n, h, w, ci, co = cfg
     g = graph()
@@ -236,6 +236,8 @@ def test_conv1x1_tensor_core_fp32(cfg, epi):
         e = g.add("ScaleShift", [e, "s", "t"], axis=-1)
         if epi == "clip":
             g.mark_output(g.add("Clip", [e], lo=0.0, hi=6.0, out="Y"))
+        elif epi == "affine":                  # a projection whose channel count changes: no residual
+            g.mark_output(e)
         else:
             g.ext("R", (n, h, w, co)); ins["R"] = rnd((n, h, w, co), 15, -1, 1)
             g.mark_output(g.add("Add", [e, "R"], out="Y"))
@@ -351,7 +353,8 @@ def test_encoder_full_size_twelve_layers():
 @pytest.mark.parametrize("flags", [B.PLAN_FUSED, B.PLAN_UNFUSED])
 @pytest.mark.parametrize("nhw,cin,cout,slices", [((2, 32, 32), 256, 64, 2), ((1, 40, 40), 384, 32, 2), ((1, 24, 24), 576, 48, 3),
                                                   ((1, 24, 24), 960, 24, 4), ((2, 16, 16), 248, 40, 2)])
-def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, flags):
+@pytest.mark.parametrize("tail", ["bn_clip", "bn"])
+def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, flags, tail):
     """fp32 pointwise convolutions deeper than the split-TF32 kernel takes (K > 244) are planned as 2-4 tensor-core
     contractions over K slices (as few as fit the kernel's shared memory), the partial sums riding in a later slice's
     epilogue."""
@@ -359,7 +362,9 @@ def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, fla
     n, h, w = nhw
     g = graph("deep_pw")
     g.ext("X", (n, h, w, cin)); g.ext("Wt", (cin, cout), kind="weight"); g.ext("s", (cout,)); g.ext("t", (cout,))
-    y = g.add("Clip", [g.add("ScaleShift", [g.add("Conv1x1", ["X", "Wt"]), "s", "t"], axis=-1)], lo=0.0, hi=6.0)
+    y = g.add("ScaleShift", [g.add("Conv1x1", ["X", "Wt"]), "s", "t"], axis=-1)
+    if tail == "bn_clip":
+        y = g.add("Clip", [y], lo=0.0, hi=6.0)
     g.mark_output(y)
     ins = {"X": rnd((n, h, w, cin), 90, 0.0, 1.0), "Wt": rnd((cin, cout), 91, -0.2, 0.2), "s": rnd((cout,), 92, 0.5, 1.5),
            "t": rnd((cout,), 93, -0.5, 0.5)}
@@ -367,7 +372,7 @@ def test_deep_pointwise_convolution_is_split_along_k(nhw, cin, cout, slices, fla
     gemms = [b for b in s.g.blocks() if b["family"] == "gemm"]
     assert len(gemms) >= slices and all(b["variant"] in (4, 7) for b in gemms), s.g.blocks()
     assert not [b for b in s.g.blocks() if b["family"] == "conv1x1"], s.g.blocks()
-    assert s.plan_stats.n_ops == 3          # the slices count as the one convolution they came from
+    assert s.plan_stats.n_ops == (3 if tail == "bn_clip" else 2)          # the slices count as the one convolution they came from
 
 
 @pytest.mark.parametrize("mnk", [(2048, 64, 512), (700, 100, 300), (4096, 16, 1024)])
@@ -472,7 +477,7 @@ def test_rebinding_any_epilogue_operand_reencodes_the_tensor_maps():
 @pytest.mark.parametrize("cfg", [(1, 14, 14, 384, 64), (1, 14, 14, 64, 384), (1, 7, 7, 576, 160), (1, 28, 28, 24, 144), (2, 9, 11, 40, 24),
                                  (1, 5, 3, 16, 8), (1, 20, 20, 144, 24), (1, 1, 1, 320, 104), (1, 30, 30, 72, 200),
                                  (1, 1, 1, 320, 100), (2, 3, 3, 64, 20), (4, 1, 1, 48, 2)])
-@pytest.mark.parametrize("epi", ["clip", "residual", "chain", "none"])
+@pytest.mark.parametrize("epi", ["clip", "residual", "affine", "chain", "none"])
 def test_conv1x1_few_rows(cfg, epi):
     n, h, w, ci, co = cfg
     g = graph()
@@ -490,6 +495,8 @@ def test_conv1x1_few_rows(cfg, epi):
         e = g.add("ScaleShift", [e, "s", "t"], axis=-1)
         if epi == "clip":
             g.mark_output(g.add("Clip", [e], lo=0.0, hi=6.0, out="Y"))
+        elif epi == "affine":
+            g.mark_output(e)
         else:
             g.ext("R", (n, h, w, co)); ins["R"] = rnd((n, h, w, co), 15, -1, 1)
             g.mark_output(g.add("Add", [e, "R"], out="Y"))
