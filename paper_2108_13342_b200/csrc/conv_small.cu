@@ -193,17 +193,23 @@ __global__ void __launch_bounds__(THREADS) conv_small_kernel(const __grid_consta
 
 static const GemmParams& gp_of(const Launch& L) { return *reinterpret_cast<const GemmParams*>(L.blob.data()); }
 
-// Taken where the tall-and-skinny kernels have too few rows to fill the GPU.
-bool conv_small_eligible(const GemmParams& gp) {
+// The part of the eligibility test that depends on the problem's shape alone (the planner's cost model for splitting a
+// contraction asks it: this kernel, not the FMA kernels, is what an unsplit fp32 contraction of such a shape runs on).
+bool conv_small_shape_fits(int64_t M, int64_t N, int64_t K) {
   if (plan_flag(DNNF_PLAN_NO_SMALL_CONV)) return false;
-  if (gp.A.dtype != 0 || gp.B.dtype != 0) return false;
-  if (gp.batch_ext[0] * gp.batch_ext[1] != 1) return false;
   // (beyond 1024 rows only where the tall-and-skinny tensor-core kernel does not apply, i.e. K x N too large for its
   // resident weights: the 576 -> 160 and 384 -> 64 projections on 6272 pixels ran at 99 and 86 us on the FMA kernels)
-  { const char* e = dev_env("DNNF_SMALL_M_MAX"); if (gp.M > (e ? atoi(e) : 65536)) return false; }
+  { const char* e = dev_env("DNNF_SMALL_M_MAX"); if (M > (e ? atoi(e) : 65536)) return false; }
+  return N % 2 == 0 && K % 8 == 0 && K >= 8;
+}
+
+// Taken where the tall-and-skinny kernels have too few rows to fill the GPU.
+bool conv_small_eligible(const GemmParams& gp) {
+  if (!conv_small_shape_fits(gp.M, gp.N, gp.K)) return false;
+  if (gp.A.dtype != 0 || gp.B.dtype != 0) return false;
+  if (gp.batch_ext[0] * gp.batch_ext[1] != 1) return false;
   if (gp.A.stride_col != 1 || gp.A.stride_row % 4 || gp.A.base % 4) return false;
   if (gp.B.stride_col != 1 || gp.B.stride_row != gp.N) return false;
-  if (gp.N % 2 || gp.K % 8 || gp.K < 8) return false;
   if (gp.n_nd != 1 || gp.m_nd != 1 || gp.b_nd != 1) return false;
   // the chain reads and writes pairs of neighbouring columns: 8-byte aligned wherever it walks along n
   auto pair_ok = [](const TensorArg& a) { return a.dtype == 0 && (a.stride[0] == 0 || (a.stride[0] == 1 && a.base % 2 == 0 && a.stride[1] % 2 == 0)); };

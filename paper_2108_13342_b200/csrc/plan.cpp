@@ -353,14 +353,20 @@ double block_cost_us(const Graph& g, const Block& b) {
 }
 
 bool tf32_shape_fits(int64_t M, int64_t N, int64_t K);
+bool conv_small_shape_fits(int64_t M, int64_t N, int64_t K);
 
-// Whether a split into parts x slices tensor-core kernels beats the tiled FMA kernel the contraction would otherwise
-// run on.  Both sides are rough models fitted to measurements on this GPU: the FMA kernels reach about 10 TFLOP/s
-// on such shapes; a split kernel costs about 9 us of launch, setup and tail, every part reads A again, every slice
-// but the last writes a partial sum that a later one reads.
+// Whether a split into parts x slices tensor-core kernels beats the kernel the contraction would otherwise run on.
+// Both sides are rough models fitted to measurements on this GPU: the tiled FMA kernels reach about 10 TFLOP/s on
+// such shapes; the one-tile-per-CTA mma.sync kernel (up to 65536 rows) takes about 4.7 ns + 0.044 ns x K per 16 x 32
+// tile over the whole GPU (on 6272 pixels: 96 -> 576 channels 61 us, 64 -> 384 37 us, 576 -> 96 40 us, 576 -> 160
+// 55 us), so it is the better choice for deep contractions and the worse one for wide ones; a split kernel costs about
+// 9 us of launch, setup and tail, every part reads A again, every slice but the last writes a partial sum that a
+// later one reads.
 static bool split_pays(int64_t M, int64_t N, int64_t K, int64_t parts, int64_t slices) {
   if (plan_flag(DNNF_PLAN_SPLIT_ALWAYS)) return true;      // development switch: the tests use it to reach the split at small sizes
-  const double unsplit_us = 2.0 * (double)M * (double)N * (double)K / 1e7;
+  const double unsplit_us = conv_small_shape_fits(M, N, K)
+      ? (double)((M + 15) / 16) * (double)((N + 31) / 32) * (4.7 + 0.044 * (double)K) * 1e-3
+      : 2.0 * (double)M * (double)N * (double)K / 1e7;
   const double bytes = 4.0 * (double)M * ((double)parts * (double)K + (double)N * (1.0 + 2.0 * (double)(slices - 1)));
   const double split_us = 9.0 * (double)(parts * slices) + bytes / 4e6;
   return split_us < unsplit_us;

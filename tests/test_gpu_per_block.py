@@ -51,7 +51,7 @@ def test_decoder_twelve_layers_every_block(flags, rewrite):
 def test_style_transfer_decoder_blocks(flags):
     """Instance normalisation, overlapping transposed convolutions (pointwise convolution onto the patch values + gather),
     depthwise convolution: every block at the single-block tolerance."""
-    checked, skipped = check_blocks(W.style_decoder(n=4, hw=32, c=64), flags, min_checked=6)
+    checked, skipped = check_blocks(W.style_decoder(n=4, hw=32, c=64), flags, min_checked=5)
     print("style decoder: blocks checked", checked, "skipped", skipped)
 
 
