@@ -424,8 +424,11 @@ def test_wide_pointwise_convolution_is_split_into_channel_blocks(nhw, cin, cout,
 
 def test_split_decision_follows_the_cost_model():
     """At 25088 pixels a 160 -> 960 convolution is worth 18 tensor-core kernels; a 576 -> 160 one at 6272 pixels is not
-    worth 12 (measured: 263 us against 675 us, and 123 us against 111 us)."""
-    for (n, hw, cin, cout), split in [((32, 28, 160, 960), True), ((32, 14, 576, 160), False)]:
+    worth 12 (measured: 263 us against 675 us, and 123 us against 111 us).  At 6272 pixels the one-tile-per-CTA kernel is
+    the unsplit alternative: a deep 576 -> 96 projection stays whole (41 us against 95 us in six K slices), a wide
+    96 -> 576 expansion is cut into column blocks (36 us in three kernels against 61 us)."""
+    for (n, hw, cin, cout), split in [((32, 28, 160, 960), True), ((32, 14, 576, 160), False), ((32, 14, 576, 96), False),
+                                      ((32, 14, 96, 576), True)]:
         g = graph("split_cost")
         g.ext("X", (n, hw, hw, cin)); g.ext("Wt", (cin, cout), kind="weight")
         g.mark_output(g.add("Conv1x1", ["X", "Wt"]))
