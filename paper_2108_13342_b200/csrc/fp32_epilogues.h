@@ -25,9 +25,11 @@ DNNF_SP_BEGIN(FP_ResidualScaleShiftClip, 6)
 DNNF_SP_BEGIN(FP_ScaleShift, 4) MO(M_MOV, S_ANCHOR, 0), MO(M_MUL, S_IN, 0), MO(M_ADD, S_IN, 1), MO(M_STORE, S_NONE, 0) DNNF_SP_END
 DNNF_SP_BEGIN(FP_ResidualScaleShift, 5)
   MO(M_MOV, S_IN, 0), MO(M_ADD, S_ANCHOR, 0), MO(M_MUL, S_IN, 1), MO(M_ADD, S_IN, 2), MO(M_STORE, S_NONE, 0) DNNF_SP_END
+// the last layer of an image decoder: bias, Tanh
+DNNF_SP_BEGIN(FP_BiasTanh, 4) MO(M_MOV, S_ANCHOR, 0), MO(M_ADD, S_IN, 0), MO(M_TANH, S_NONE, 0), MO(M_STORE, S_NONE, 0) DNNF_SP_END
 #undef MO
 using Static = TypeList<FP_Store, FP_Bias, FP_ScaleShiftClip, FP_ScaleShiftResidual, FP_ScaleShiftClipResidual, FP_Residual,
-                        FP_ResidualScaleShiftClip, FP_ScaleShift, FP_ResidualScaleShift>;
+                        FP_ResidualScaleShiftClip, FP_ScaleShift, FP_ResidualScaleShift, FP_BiasTanh>;
 
 
 }  // namespace tf32
