@@ -26,7 +26,7 @@ struct PoolParams {
   int32_t is_max;
   int32_t col2im;          // the tensor holds k x k patches per pixel ([N,Hi,Wi,k*k*C]); an output element adds the values that land on it
   int32_t Ci;              // channels per pixel of the tensor that is read (C, or k*k*C for col2im)
-  FastDiv fd_c4, fd_w, fd_h;
+  FastDiv fd_c4, fd_w, fd_h, fd_s;   // fd_s: by the stride (col2im)
   // wide windows (a global pool): CTAs per (pixel, 128-channel group) and how the window is sliced over them
   int32_t groups, slices, per_slice;
   float* scratch;          // [unit][slice][128] partial results of a sliced window
@@ -56,6 +56,23 @@ __global__ void __launch_bounds__(256) pool_kernel(const __grid_constant__ PoolP
     // likewise for columns; at most ceil(k / s)^2 terms, added in a fixed order
     const int s = p.stride, k = p.kernel;
     const int hp = (int)ho + p.pad, wp = (int)wo + p.pad;
+    if (k <= 2 * s) {
+      // at most 2 x 2 terms (the usual k = 2s): their loads are issued together, then added in the same fixed order
+      const int hq = (int)fd_div((uint32_t)hp, p.fd_s), wq = (int)fd_div((uint32_t)wp, p.fd_s);
+      const int i0 = hp - hq * s, j0 = wp - wq * s;
+      float4 v[4];
+#pragma unroll
+      for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+          const int i = i0 + a * s, j = j0 + b * s, h = hq - a, w = wq - b;
+          const bool ok = i < k && j < k && h >= 0 && h < p.Hi && w >= 0 && w < p.Wi;
+          v[a * 2 + b] = ok ? __ldg(reinterpret_cast<const float4*>(xb + ((size_t)h * p.Wi + w) * p.Ci + (size_t)(i * k + j) * p.d.C))
+                            : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { io.accv[0] += v[e].x; io.accv[1] += v[e].y; io.accv[2] += v[e].z; io.accv[3] += v[e].w; }
+    } else
     for (int i = hp % s; i < k; i += s) {
       const int h = (hp - i) / s;
       if (hp - i < 0 || h >= p.Hi) continue;
@@ -239,6 +256,7 @@ int lower_pool(const Graph& g, const std::vector<int>& ops, int anchor, Block& o
   pp.col2im = A.kind == DNNF_OP_COL2IM;
   pp.Ci = (int)X.dims[3];
   pp.fd_c4 = make_fastdiv((uint32_t)dp.C / 4); pp.fd_w = make_fastdiv((uint32_t)dp.W); pp.fd_h = make_fastdiv((uint32_t)dp.H);
+  pp.fd_s = make_fastdiv((uint32_t)std::max(pp.stride, 1));
   dp.n_in = (int)cx.ins.size(); dp.n_out = (int)cx.outs.size();
   auto fill = [&](TensorArg& a, const ExtArg& e, bool is_out) {
     a.ptr = nullptr; a.base = (int32_t)e.view.c0; a.dtype = g.tensors[e.tensor].dtype; a.mode = 0;
